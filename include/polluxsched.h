@@ -1,0 +1,200 @@
+/*
+ * polluxsched.h - C ABI of the B200-native PolluxSched optimizer core.
+ *
+ * The library evaluates, on one GPU, the data-parallel part of the cluster-wide
+ * optimisation of Pollux (Qiao et al., OSDI'21, Sec. 4.2-4.3): per-job speedup tables
+ * from the goodput model (Eq. 4-11, 13, 15), the fitness of a population of allocation
+ * matrices (Eq. 14 with the re-allocation penalty), and the population search
+ * ("perturbs and combines candidate allocation matrices ... and finally modifies them
+ * to satisfy node resource constraints and interference avoidance", Sec. 4.3).
+ *
+ * Conventions
+ *  - Every function returns SCHED_OK (0) or a negative SCHED_ERR_* code; nothing throws,
+ *    aborts or traps.  sched_last_error() gives a human-readable reason.
+ *  - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  All buffers passed in
+ *    are owned by the caller; the library never frees or resizes them.  The context owns
+ *    only its internal scratch (allocated in sched_init / on first use, freed in
+ *    sched_destroy).
+ *  - All work is enqueued on the CUDA stream given to sched_init; calls with device
+ *    buffers are asynchronous with respect to the host, calls with host buffers
+ *    (`*_host`) return after their results are in the host buffers.
+ *  - Matrices are row-major.  An allocation matrix A is int16 [J][num_nodes] (node index
+ *    fastest, A[j][n] = GPUs of node n given to job j, Sec. 4.2); a population is
+ *    int16 [P][J][num_nodes].  Tables are fp32 [J][k_max+1][n_max+1] indexed by
+ *    (job, replicas K, occupied nodes N).
+ *  - Entries of allocation matrices are expected in [0, 32767].  Out-of-range values never
+ *    cause out-of-bounds accesses: the fitness clamps (K, N) into the table, the
+ *    operators first clamp every entry into [0, capacity of its node].
+ *  - One context must not be used from two host threads at once.
+ */
+#ifndef POLLUXSCHED_H_
+#define POLLUXSCHED_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SCHED_OK 0
+#define SCHED_ERR_INVALID_ARG (-1) /* null pointer, negative size, misaligned buffer   */
+#define SCHED_ERR_BAD_CONFIG (-2)  /* a sched_config field outside its documented range */
+#define SCHED_ERR_CUDA (-3)        /* a CUDA runtime call failed                        */
+#define SCHED_ERR_TIMEOUT (-4)     /* a bounded device-side wait ran out                */
+#define SCHED_ERR_NOT_FINITE (-5)  /* reserved                                          */
+#define SCHED_ERR_TOO_LARGE (-6)   /* a size exceeds a documented fixed maximum         */
+
+/* Limits checked by sched_init. */
+#define SCHED_MAX_NODES 8192
+#define SCHED_MAX_K 1024
+#define SCHED_MAX_N 1024
+
+typedef struct sched_ctx sched_ctx; /* opaque, library-owned */
+
+typedef struct {
+  int32_t num_nodes;   /* nodes in the cluster, 1..SCHED_MAX_NODES                       */
+  int32_t num_jobs;    /* J: rows of every allocation matrix (running + pending jobs)     */
+  int32_t k_max;       /* largest replica count tabulated, 1..SCHED_MAX_K                 */
+  int32_t n_max;       /* largest node count tabulated, 1..SCHED_MAX_N                    */
+  int32_t grid_m;      /* per-GPU batch sizes per job in the (m, s) grid, >= 1            */
+  int32_t grid_s;      /* accumulation steps s = 0..grid_s-1; grid_m*grid_s <= 65535      */
+  int32_t population;  /* P: candidates evolved by ga_generation / schedule_round, >= 1   */
+  float p;             /* exponent of the power mean in Eq. 14 (schedule_round)           */
+  float delta_sec;     /* re-allocation delay estimate delta (Sec. 4.2), >= 0             */
+  float speedup_floor; /* lower bound applied to every penalised speedup, >= 0            */
+  uint32_t thr_mutate; /* a row is perturbed when a 32-bit draw is below this value       */
+  uint32_t thr_init;   /* same, for the initial population of a round                     */
+  int32_t num_elite;   /* best candidates copied unchanged into the next generation, 0..P */
+  uint64_t seed;       /* seed of the counter-based random stream                         */
+} sched_config;
+
+/* Per-job inputs, structure of arrays.  The struct lives on the host; for the device
+ * entry points every member is a DEVICE pointer to J elements (m_grid: J*grid_m), for
+ * the *_host entry points every member is a HOST pointer.  (theta_sys, phi, M0) of
+ * Eq. 12 specify each job's goodput function. */
+typedef struct {
+  const float *alpha_grad, *beta_grad;   /* T_grad(m) = alpha + beta m           (Eq. 8) */
+  const float *alpha_local, *beta_local; /* T_sync, all replicas on one node     (Eq. 9) */
+  const float *alpha_node, *beta_node;   /* T_sync, replicas on several nodes    (Eq. 9) */
+  const float *gamma;                    /* overlap exponent, >= 1               (Eq. 10) */
+  const float *phi;                      /* gradient noise scale                 (Eq. 6) */
+  const float *m0;                       /* initial batch size M0 (an exact integer)      */
+  const float *m_max_total;              /* upper limit of the total batch size M         */
+  const int32_t *m_grid;                 /* [J][grid_m] ascending per-GPU batch sizes     */
+  const int32_t *k_cap;                  /* max replicas per job (Sec. 4.1 exploration cap);
+                                            nullable = k_max                              */
+  const int32_t *fair_k, *fair_n;        /* (K, N) of the fair allocation a_f    (Eq. 15) */
+  const float *age_sec;                  /* T_j, nullable when no penalty is needed       */
+  const int32_t *num_restarts;           /* R_j, nullable likewise                        */
+  const uint8_t *active;                 /* nullable = all jobs active; inactive jobs are
+                                            left out of Eq. 14 and get empty rows         */
+} sched_jobs;
+
+/* Creates a context.  h_node_capacity: HOST array [num_nodes] of GPUs per node (>= 0).
+ * cuda_stream: a cudaStream_t (may be NULL for the default stream).  Allocates the
+ * context's device scratch (cudaMalloc); the device current at this call is the
+ * device the context lives on.  Errors: INVALID_ARG, BAD_CONFIG, TOO_LARGE, CUDA. */
+int sched_init(const sched_config *cfg, const int16_t *h_node_capacity, void *cuda_stream,
+               sched_ctx **out);
+
+/* Frees the context and its scratch.  NULL is accepted. */
+int sched_destroy(sched_ctx *ctx);
+
+/* Reason of the last failure on this context (or of the last failed sched_init when ctx
+ * is NULL).  The string is owned by the library and valid until the next call. */
+const char *sched_last_error(const sched_ctx *ctx);
+
+/* Waits for the stream and returns the device-side status word (SCHED_OK unless a
+ * kernel recorded an error such as an exhausted bounded wait). */
+int sched_sync_status(sched_ctx *ctx);
+
+/* Number of kernels this context has launched so far (for accounting in benchmarks). */
+int64_t sched_launch_count(const sched_ctx *ctx);
+
+/* Speedup tables (Eq. 13 and 15).  For every job and every (K, N) with 1 <= N <= n_max,
+ * N <= K <= k_max and K no larger than the N largest nodes together:
+ *   goodput[j][K][N] = max over the grid {m_grid[j][i]} x {s} of GOODPUT(a, m, s) (Eq. 4)
+ *                      subject to M0 <= K m (s+1) <= m_max_total,
+ *   argmax[j][K][N]  = i * grid_s + s of a maximiser,
+ *   speedup[j][K][N] = goodput[j][K][N] / goodput[j][fair_k][fair_n].
+ * All other entries are 0 (argmax 0xFFFF); so are entries with no feasible grid point,
+ * and a job's whole speedup slab when its fair-share goodput is 0.  Outputs are
+ * fp32/uint16 [J][k_max+1][n_max+1]; d_goodput and d_argmax may be NULL.  Batch sizes
+ * must satisfy K m (s+1) < 2^24 for the feasibility test to be exact.
+ * Uses: all fp32 members of jobs, m_grid, fair_k, fair_n. */
+int build_speedup_table(sched_ctx *ctx, const sched_jobs *d_jobs, float *d_goodput,
+                        float *d_speedup, uint16_t *d_argmax);
+
+/* REALLOC_FACTOR_j(delta) = (T_j - R_j delta) / (T_j + delta) clamped to [0, 1]
+ * (Sec. 4.2), with delta = cfg.delta_sec.  d_out: fp32 [J].  Uses age_sec, num_restarts. */
+int compute_realloc_factor(sched_ctx *ctx, const sched_jobs *d_jobs, float *d_out);
+
+/* Fitness of `count` candidates (Eq. 14).  d_pop: int16 [count][J][num_nodes].  For each
+ * active job the speedup is read at (K, N) = (sum of the row, entries > 0), clamped to
+ * the table; if d_cur (int16 [J][num_nodes]) and d_realloc_factor (fp32 [J]) are both
+ * given, a row that differs from a non-empty current row is multiplied by the job's
+ * factor; the result is raised to cfg.speedup_floor; the power mean with exponent p
+ * over the active jobs is written to d_fitness[count] (p = 0: geometric mean; no active
+ * job: 0).  d_active: uint8 [J], nullable.  `count` may differ from cfg.population. */
+int eval_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const float *d_speedup,
+                 const int16_t *d_cur, const float *d_realloc_factor, const uint8_t *d_active,
+                 float p, float *d_fitness);
+
+/* The repair step alone, in place, on `count` matrices: entries into [0, node size], per-job
+ * replica cap (k_cap, highest node index first) and n_max, then at most one distributed
+ * job per node (interference avoidance, Sec. 4.2) and node capacity, the last two with
+ * job order rotated by draws of the random stream addressed by (round, first_candidate
+ * + c, generation).  Removal only; feasible matrices are left unchanged.
+ * Uses k_cap, active (jobs may be NULL: no cap beyond k_max, all active). */
+int repair_population(sched_ctx *ctx, const sched_jobs *d_jobs, int16_t *d_pop, int32_t count,
+                      uint32_t first_candidate, uint32_t round, uint32_t generation);
+
+/* Initial population of a round: candidate 0 is d_cur (NULL = empty cluster), candidates
+ * 1..P-1 are d_cur with rows perturbed with threshold thr_init; all repaired.
+ * d_pop_out: int16 [P][J][num_nodes]. */
+int init_population(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cur,
+                    uint32_t round, int16_t *d_pop_out);
+
+/* One generation of the population search (Sec. 4.3).  Children 0..num_elite-1 are the
+ * best-ranked parents (fitness descending, index ascending, compared by bit pattern);
+ * every other child takes each job's row from one of two parents (each the better of two
+ * random candidates), perturbs it with threshold thr_mutate (grow / shrink / relocate)
+ * and is repaired.  d_pop_in, d_pop_out: int16 [P][J][num_nodes], must not overlap;
+ * d_fitness_in: fp32 [P].  The result is a pure function of the inputs, cfg.seed, round
+ * and generation.  Uses k_cap, active (jobs may be NULL). */
+int ga_generation(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_pop_in,
+                  const float *d_fitness_in, int16_t *d_pop_out, uint32_t round,
+                  uint32_t generation);
+
+/* A whole scheduling round: tables, re-allocation factors, initial population and its
+ * fitness, `generations` x (ga_generation, eval_fitness), then the best candidate of the
+ * last population.  d_cur: int16 [J][num_nodes] or NULL.  d_best: int16 [J][num_nodes],
+ * d_best_fitness: fp32 [1].  Population and table buffers are context scratch allocated
+ * on the first call. */
+int schedule_round(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cur, uint32_t round,
+                   int32_t generations, int16_t *d_best, float *d_best_fitness);
+
+/* Same with HOST buffers: copies the job arrays and h_cur to the device, runs the round,
+ * copies the result back and waits for it.  Every member of h_jobs is a host pointer. */
+int schedule_round_host(sched_ctx *ctx, const sched_jobs *h_jobs, const int16_t *h_cur,
+                        uint32_t round, int32_t generations, int16_t *h_best,
+                        float *h_best_fitness);
+
+/* Copies the population and fitness left by the last schedule_round into caller buffers
+ * (either may be NULL).  d_pop_out: int16 [P][J][num_nodes], d_fitness_out: fp32 [P]. */
+int sched_get_population(sched_ctx *ctx, int16_t *d_pop_out, float *d_fitness_out);
+
+/* Pointer to the fp32 [J][k_max+1][n_max+1] speedup table built by the last schedule_round
+ * (context scratch, device memory), or NULL before the first round. */
+const float *sched_round_speedup_table(const sched_ctx *ctx);
+
+/* Fitness with HOST buffers (population, table, optional cur / factors / active mask are
+ * copied in, fitness copied out, the call waits).  Staging buffers are context scratch. */
+int eval_fitness_host(sched_ctx *ctx, const int16_t *h_pop, int32_t count, const float *h_speedup,
+                      const int16_t *h_cur, const float *h_realloc_factor,
+                      const uint8_t *h_active, float p, float *h_fitness);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* POLLUXSCHED_H_ */

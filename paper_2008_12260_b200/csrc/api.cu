@@ -1,0 +1,440 @@
+// C-ABI entry points: argument validation, context and scratch management, and the
+// scheduling-round driver.  All arithmetic of the method lives in the kernels.
+#include <stdarg.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+char g_init_error[256] = "";
+
+const char *set_error(sched_ctx *ctx, const char *fmt, ...) {
+  char *dst = ctx ? ctx->err : g_init_error;
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(dst, 256, fmt, ap);
+  va_end(ap);
+  return dst;
+}
+
+namespace {
+
+template <typename T>
+int dev_alloc(sched_ctx *ctx, T **p, size_t n) {
+  *p = nullptr;
+  if (n == 0) n = 1;
+  SCHED_CUDA_CHECK(ctx, cudaMalloc((void **)p, n * sizeof(T)));
+  return SCHED_OK;
+}
+
+#define REQUIRE(ctx, cond, code, ...)   \
+  do {                                  \
+    if (!(cond)) {                      \
+      set_error(ctx, __VA_ARGS__);      \
+      return code;                      \
+    }                                   \
+  } while (0)
+
+int check_table_jobs(sched_ctx *ctx, const sched_jobs *j) {
+  REQUIRE(ctx, j, SCHED_ERR_INVALID_ARG, "jobs is NULL");
+  REQUIRE(ctx, j->alpha_grad && j->beta_grad && j->alpha_local && j->beta_local && j->alpha_node &&
+                   j->beta_node && j->gamma && j->phi && j->m0 && j->m_max_total && j->m_grid &&
+                   j->fair_k && j->fair_n,
+          SCHED_ERR_INVALID_ARG, "jobs: a goodput-model array, m_grid, fair_k or fair_n is NULL");
+  return SCHED_OK;
+}
+
+int ensure_round_scratch(sched_ctx *ctx) {
+  if (ctx->round_ready) return SCHED_OK;
+  const sched_config &c = ctx->cfg;
+  const size_t pop = (size_t)c.population * c.num_jobs * c.num_nodes;
+  const size_t tab = (size_t)c.num_jobs * ctx->KD * ctx->ND;
+  int rc;
+  if ((rc = dev_alloc(ctx, &ctx->d_popA, pop)) != SCHED_OK) return rc;
+  if ((rc = dev_alloc(ctx, &ctx->d_popB, pop)) != SCHED_OK) return rc;
+  if ((rc = dev_alloc(ctx, &ctx->d_fit, (size_t)c.population)) != SCHED_OK) return rc;
+  if ((rc = dev_alloc(ctx, &ctx->d_tab_goodput, tab)) != SCHED_OK) return rc;
+  if ((rc = dev_alloc(ctx, &ctx->d_tab_speedup, tab)) != SCHED_OK) return rc;
+  if ((rc = dev_alloc(ctx, &ctx->d_rf, (size_t)c.num_jobs)) != SCHED_OK) return rc;
+  ctx->round_ready = true;
+  return SCHED_OK;
+}
+
+}  // namespace
+
+int ensure_fitness_scratch(sched_ctx *ctx, int32_t count, int chunks) {
+  const size_t need_p = (size_t)count * chunks * 2;
+  if (need_p > ctx->partial_cap) {
+    if (ctx->d_partial) {
+      SCHED_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
+      SCHED_CUDA_CHECK(ctx, cudaFree(ctx->d_partial));
+    }
+    int rc = dev_alloc(ctx, &ctx->d_partial, need_p);
+    if (rc != SCHED_OK) { ctx->partial_cap = 0; return rc; }
+    ctx->partial_cap = need_p;
+  }
+  if ((size_t)count > ctx->ticket_cap) {
+    if (ctx->d_ticket) {
+      SCHED_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
+      SCHED_CUDA_CHECK(ctx, cudaFree(ctx->d_ticket));
+    }
+    int rc = dev_alloc(ctx, &ctx->d_ticket, (size_t)count);
+    if (rc != SCHED_OK) { ctx->ticket_cap = 0; return rc; }
+    ctx->ticket_cap = (size_t)count;
+    SCHED_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->d_ticket, 0, (size_t)count * sizeof(unsigned int), ctx->stream));
+  }
+  return SCHED_OK;
+}
+
+int ensure_dflag(sched_ctx *ctx, int32_t count) {
+  const size_t need = (size_t)count * ctx->cfg.num_jobs;
+  if (need > ctx->dflag_cap) {
+    if (ctx->d_dflag) {
+      SCHED_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
+      SCHED_CUDA_CHECK(ctx, cudaFree(ctx->d_dflag));
+    }
+    int rc = dev_alloc(ctx, &ctx->d_dflag, need);
+    if (rc != SCHED_OK) { ctx->dflag_cap = 0; return rc; }
+    ctx->dflag_cap = need;
+  }
+  return SCHED_OK;
+}
+
+extern "C" {
+#pragma GCC visibility push(default)
+
+int sched_init(const sched_config *cfg, const int16_t *h_node_capacity, void *cuda_stream,
+               sched_ctx **out) {
+  if (out) *out = nullptr;
+  REQUIRE(nullptr, cfg && h_node_capacity && out, SCHED_ERR_INVALID_ARG,
+          "sched_init: cfg, h_node_capacity and out must be non-NULL");
+  REQUIRE(nullptr, cfg->num_nodes >= 1 && cfg->num_jobs >= 0 && cfg->k_max >= 1 && cfg->n_max >= 1 &&
+                       cfg->grid_m >= 1 && cfg->grid_s >= 1 && cfg->population >= 1,
+          SCHED_ERR_BAD_CONFIG, "sched_init: sizes must be positive (num_jobs may be 0)");
+  REQUIRE(nullptr, cfg->num_nodes <= SCHED_MAX_NODES && cfg->k_max <= SCHED_MAX_K &&
+                       cfg->n_max <= SCHED_MAX_N,
+          SCHED_ERR_TOO_LARGE, "sched_init: num_nodes <= %d, k_max <= %d, n_max <= %d",
+          SCHED_MAX_NODES, SCHED_MAX_K, SCHED_MAX_N);
+  REQUIRE(nullptr, (long long)cfg->grid_m * cfg->grid_s <= 65535, SCHED_ERR_TOO_LARGE,
+          "sched_init: grid_m * grid_s must be <= 65535");
+  REQUIRE(nullptr, cfg->num_elite >= 0 && cfg->num_elite <= cfg->population, SCHED_ERR_BAD_CONFIG,
+          "sched_init: num_elite must be in [0, population]");
+  REQUIRE(nullptr, cfg->delta_sec >= 0.f && cfg->speedup_floor >= 0.f && cfg->p == cfg->p,
+          SCHED_ERR_BAD_CONFIG, "sched_init: delta_sec and speedup_floor must be >= 0, p not NaN");
+  REQUIRE(nullptr, (long long)cfg->population * cfg->num_jobs < (1LL << 31), SCHED_ERR_TOO_LARGE,
+          "sched_init: population * num_jobs must be below 2^31");
+
+  sched_ctx *ctx = new (std::nothrow) sched_ctx();
+  REQUIRE(nullptr, ctx, SCHED_ERR_CUDA, "sched_init: out of host memory");
+  memset(ctx, 0, sizeof(*ctx));
+  ctx->cfg = *cfg;
+  ctx->stream = (cudaStream_t)cuda_stream;
+  ctx->KD = cfg->k_max + 1;
+  ctx->ND = cfg->n_max + 1;
+
+  auto fail = [&](int rc) {
+    strncpy(g_init_error, ctx->err, sizeof(g_init_error) - 1);
+    sched_destroy(ctx);
+    return rc;
+  };
+  cudaError_t e = cudaGetDevice(&ctx->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, ctx->device);
+  if (e != cudaSuccess) {
+    set_error(ctx, "sched_init: no usable CUDA device: %s", cudaGetErrorString(e));
+    return fail(SCHED_ERR_CUDA);
+  }
+
+  // replicas that fit on the N largest nodes, N = 0..n_max
+  std::vector<int16_t> sorted(h_node_capacity, h_node_capacity + cfg->num_nodes);
+  std::sort(sorted.begin(), sorted.end(), [](int16_t a, int16_t b) { return a > b; });
+  std::vector<int32_t> kfit(ctx->ND, 0);
+  for (int n = 1; n < ctx->ND; ++n) {
+    const int add = (n <= cfg->num_nodes && sorted[n - 1] > 0) ? sorted[n - 1] : 0;
+    kfit[n] = kfit[n - 1] + add;
+  }
+
+  const size_t J = (size_t)cfg->num_jobs, P = (size_t)cfg->population;
+  int rc;
+  if ((rc = dev_alloc(ctx, &ctx->d_cap, ((size_t)cfg->num_nodes + 7) & ~(size_t)7)) != SCHED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_kfit, (size_t)ctx->ND)) != SCHED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_gmax, J * ctx->KD * 2)) != SCHED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_amax, J * ctx->KD * 2)) != SCHED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_rank, P)) != SCHED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_order, P)) != SCHED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_pen, J)) != SCHED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_status, 1)) != SCHED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_best_idx, 1)) != SCHED_OK) return fail(rc);
+  e = cudaMemcpyAsync(ctx->d_cap, h_node_capacity, sizeof(int16_t) * cfg->num_nodes,
+                      cudaMemcpyHostToDevice, ctx->stream);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(ctx->d_kfit, kfit.data(), sizeof(int32_t) * ctx->ND, cudaMemcpyHostToDevice, ctx->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_status, 0, sizeof(int), ctx->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_gmax, 0, sizeof(float) * std::max<size_t>(J * ctx->KD * 2, 1), ctx->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_amax, 0xFF, sizeof(uint16_t) * std::max<size_t>(J * ctx->KD * 2, 1), ctx->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);   // host vectors go out of scope
+  if (e != cudaSuccess) {
+    set_error(ctx, "sched_init: upload failed: %s", cudaGetErrorString(e));
+    return fail(SCHED_ERR_CUDA);
+  }
+  *out = ctx;
+  return SCHED_OK;
+}
+
+int sched_destroy(sched_ctx *ctx) {
+  if (!ctx) return SCHED_OK;
+  cudaStreamSynchronize(ctx->stream);
+  void *ptrs[] = {ctx->d_cap, ctx->d_kfit, ctx->d_gmax, ctx->d_amax, ctx->d_rank, ctx->d_order,
+                  ctx->d_dflag, ctx->d_pen, ctx->d_partial, ctx->d_ticket, ctx->d_status,
+                  ctx->d_popA, ctx->d_popB, ctx->d_fit, ctx->d_tab_goodput, ctx->d_tab_speedup,
+                  ctx->d_rf, ctx->d_best_idx, ctx->d_stage, ctx->d_stage_fit};
+  for (void *p : ptrs)
+    if (p) cudaFree(p);
+  delete ctx;
+  return SCHED_OK;
+}
+
+const char *sched_last_error(const sched_ctx *ctx) { return ctx ? ctx->err : g_init_error; }
+
+int sched_sync_status(sched_ctx *ctx) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "sched_sync_status: ctx is NULL");
+  int status = 0;
+  SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(&status, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+  SCHED_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
+  if (status != SCHED_OK) set_error(ctx, "a kernel recorded device status %d", status);
+  return status;
+}
+
+int64_t sched_launch_count(const sched_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int build_speedup_table(sched_ctx *ctx, const sched_jobs *d_jobs, float *d_goodput,
+                        float *d_speedup, uint16_t *d_argmax) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "build_speedup_table: ctx is NULL");
+  int rc = check_table_jobs(ctx, d_jobs);
+  if (rc != SCHED_OK) return rc;
+  REQUIRE(ctx, d_speedup, SCHED_ERR_INVALID_ARG, "build_speedup_table: d_speedup is NULL");
+  return launch_speedup_table(ctx, d_jobs, d_goodput, d_speedup, d_argmax);
+}
+
+int compute_realloc_factor(sched_ctx *ctx, const sched_jobs *d_jobs, float *d_out) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "compute_realloc_factor: ctx is NULL");
+  REQUIRE(ctx, d_jobs && d_jobs->age_sec && d_jobs->num_restarts && d_out, SCHED_ERR_INVALID_ARG,
+          "compute_realloc_factor: jobs.age_sec, jobs.num_restarts and d_out must be non-NULL");
+  return launch_realloc_factor(ctx, d_jobs, d_out);
+}
+
+int eval_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const float *d_speedup,
+                 const int16_t *d_cur, const float *d_realloc_factor, const uint8_t *d_active,
+                 float p, float *d_fitness) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "eval_fitness: ctx is NULL");
+  REQUIRE(ctx, count >= 0, SCHED_ERR_INVALID_ARG, "eval_fitness: count is negative");
+  REQUIRE(ctx, count == 0 || (d_pop && d_speedup && d_fitness), SCHED_ERR_INVALID_ARG,
+          "eval_fitness: d_pop, d_speedup and d_fitness must be non-NULL");
+  REQUIRE(ctx, p == p, SCHED_ERR_INVALID_ARG, "eval_fitness: p is NaN");
+  REQUIRE(ctx, ((uintptr_t)d_pop & 1) == 0 && ((uintptr_t)d_cur & 1) == 0 &&
+                   ((uintptr_t)d_speedup & 3) == 0 && ((uintptr_t)d_fitness & 3) == 0,
+          SCHED_ERR_INVALID_ARG, "eval_fitness: a buffer is not aligned to its element size");
+  REQUIRE(ctx, (long long)count * ctx->cfg.num_jobs < (1LL << 31), SCHED_ERR_TOO_LARGE,
+          "eval_fitness: count * num_jobs must be below 2^31");
+  return launch_fitness(ctx, d_pop, count, d_speedup, d_cur, d_realloc_factor, d_active, p, d_fitness);
+}
+
+int repair_population(sched_ctx *ctx, const sched_jobs *d_jobs, int16_t *d_pop, int32_t count,
+                      uint32_t first_candidate, uint32_t round, uint32_t generation) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "repair_population: ctx is NULL");
+  REQUIRE(ctx, count >= 0 && (count == 0 || d_pop), SCHED_ERR_INVALID_ARG,
+          "repair_population: d_pop is NULL or count negative");
+  REQUIRE(ctx, ((uintptr_t)d_pop & 1) == 0, SCHED_ERR_INVALID_ARG, "repair_population: d_pop misaligned");
+  REQUIRE(ctx, (long long)count * ctx->cfg.num_jobs < (1LL << 31), SCHED_ERR_TOO_LARGE,
+          "repair_population: count * num_jobs must be below 2^31");
+  if (ctx->cfg.num_jobs == 0) return SCHED_OK;
+  return launch_repair(ctx, d_jobs ? d_jobs->k_cap : nullptr, d_jobs ? d_jobs->active : nullptr, d_pop,
+                       count, first_candidate, round, generation);
+}
+
+int init_population(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cur, uint32_t round,
+                    int16_t *d_pop_out) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "init_population: ctx is NULL");
+  REQUIRE(ctx, d_pop_out, SCHED_ERR_INVALID_ARG, "init_population: d_pop_out is NULL");
+  REQUIRE(ctx, ((uintptr_t)d_pop_out & 1) == 0 && ((uintptr_t)d_cur & 1) == 0, SCHED_ERR_INVALID_ARG,
+          "init_population: a buffer is misaligned");
+  if (ctx->cfg.num_jobs == 0) return SCHED_OK;
+  return launch_init_population(ctx, d_jobs ? d_jobs->k_cap : nullptr,
+                                d_jobs ? d_jobs->active : nullptr, d_cur, round, d_pop_out);
+}
+
+int ga_generation(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_pop_in,
+                  const float *d_fitness_in, int16_t *d_pop_out, uint32_t round, uint32_t generation) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "ga_generation: ctx is NULL");
+  REQUIRE(ctx, d_pop_in && d_fitness_in && d_pop_out, SCHED_ERR_INVALID_ARG,
+          "ga_generation: d_pop_in, d_fitness_in and d_pop_out must be non-NULL");
+  REQUIRE(ctx, d_pop_in != d_pop_out, SCHED_ERR_INVALID_ARG, "ga_generation: in and out must not overlap");
+  REQUIRE(ctx, (((uintptr_t)d_pop_in | (uintptr_t)d_pop_out) & 1) == 0 && ((uintptr_t)d_fitness_in & 3) == 0,
+          SCHED_ERR_INVALID_ARG, "ga_generation: a buffer is misaligned");
+  if (ctx->cfg.num_jobs == 0) return SCHED_OK;
+  return launch_generation(ctx, d_jobs ? d_jobs->k_cap : nullptr, d_jobs ? d_jobs->active : nullptr,
+                           d_pop_in, d_fitness_in, d_pop_out, round, generation);
+}
+
+int schedule_round(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cur, uint32_t round,
+                   int32_t generations, int16_t *d_best, float *d_best_fitness) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "schedule_round: ctx is NULL");
+  int rc = check_table_jobs(ctx, d_jobs);
+  if (rc != SCHED_OK) return rc;
+  REQUIRE(ctx, generations >= 0, SCHED_ERR_INVALID_ARG, "schedule_round: generations is negative");
+  REQUIRE(ctx, d_best && d_best_fitness, SCHED_ERR_INVALID_ARG,
+          "schedule_round: d_best and d_best_fitness must be non-NULL");
+  REQUIRE(ctx, ctx->cfg.num_jobs >= 1, SCHED_ERR_BAD_CONFIG, "schedule_round: needs at least one job");
+  const bool penalise = d_cur && d_jobs->age_sec && d_jobs->num_restarts;
+  if ((rc = ensure_round_scratch(ctx)) != SCHED_OK) return rc;
+  if ((rc = launch_speedup_table(ctx, d_jobs, ctx->d_tab_goodput, ctx->d_tab_speedup, nullptr)) != SCHED_OK) return rc;
+  if (penalise && (rc = launch_realloc_factor(ctx, d_jobs, ctx->d_rf)) != SCHED_OK) return rc;
+  const float *rf = penalise ? ctx->d_rf : nullptr;
+  int16_t *pa = ctx->d_popA, *pb = ctx->d_popB;
+  if ((rc = launch_init_population(ctx, d_jobs->k_cap, d_jobs->active, d_cur, round, pa)) != SCHED_OK) return rc;
+  if ((rc = launch_fitness(ctx, pa, ctx->cfg.population, ctx->d_tab_speedup, d_cur, rf, d_jobs->active,
+                           ctx->cfg.p, ctx->d_fit)) != SCHED_OK) return rc;
+  for (int g = 0; g < generations; ++g) {
+    if ((rc = launch_generation(ctx, d_jobs->k_cap, d_jobs->active, pa, ctx->d_fit, pb, round, (uint32_t)g)) != SCHED_OK) return rc;
+    std::swap(pa, pb);
+    if ((rc = launch_fitness(ctx, pa, ctx->cfg.population, ctx->d_tab_speedup, d_cur, rf, d_jobs->active,
+                             ctx->cfg.p, ctx->d_fit)) != SCHED_OK) return rc;
+  }
+  ctx->d_pop_last = pa;
+  return launch_select_best(ctx, pa, ctx->d_fit, d_best, d_best_fitness);
+}
+
+int sched_get_population(sched_ctx *ctx, int16_t *d_pop_out, float *d_fitness_out) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "sched_get_population: ctx is NULL");
+  REQUIRE(ctx, ctx->d_pop_last, SCHED_ERR_INVALID_ARG, "sched_get_population: no round has run yet");
+  const sched_config &c = ctx->cfg;
+  if (d_pop_out)
+    SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(d_pop_out, ctx->d_pop_last,
+                                          sizeof(int16_t) * (size_t)c.population * c.num_jobs * c.num_nodes,
+                                          cudaMemcpyDeviceToDevice, ctx->stream));
+  if (d_fitness_out)
+    SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(d_fitness_out, ctx->d_fit, sizeof(float) * c.population,
+                                          cudaMemcpyDeviceToDevice, ctx->stream));
+  return SCHED_OK;
+}
+
+const float *sched_round_speedup_table(const sched_ctx *ctx) {
+  return (ctx && ctx->round_ready) ? ctx->d_tab_speedup : nullptr;
+}
+
+// ---- host-buffer entry points ------------------------------------------------------------
+
+static size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+int schedule_round_host(sched_ctx *ctx, const sched_jobs *h_jobs, const int16_t *h_cur, uint32_t round,
+                        int32_t generations, int16_t *h_best, float *h_best_fitness) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "schedule_round_host: ctx is NULL");
+  int rc = check_table_jobs(ctx, h_jobs);
+  if (rc != SCHED_OK) return rc;
+  REQUIRE(ctx, h_best && h_best_fitness, SCHED_ERR_INVALID_ARG,
+          "schedule_round_host: h_best and h_best_fitness must be non-NULL");
+  const sched_config &c = ctx->cfg;
+  const size_t J = (size_t)c.num_jobs, mat = J * c.num_nodes * sizeof(int16_t);
+  // layout of the staging buffer: 10 fp32 arrays, m_grid, k_cap, fair_k, fair_n, age,
+  // restarts, active, cur, best, best_fitness - each 256-byte aligned
+  const size_t f32 = align256(J * 4), grid = align256(J * c.grid_m * 4), u8 = align256(J);
+  const size_t need = 10 * f32 + grid + 5 * f32 + u8 + 2 * align256(mat) + 256;
+  if (need > ctx->stage_bytes) {
+    if (ctx->d_stage) {
+      SCHED_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
+      SCHED_CUDA_CHECK(ctx, cudaFree(ctx->d_stage));
+      ctx->d_stage = nullptr;
+      ctx->stage_bytes = 0;
+    }
+    SCHED_CUDA_CHECK(ctx, cudaMalloc(&ctx->d_stage, need));
+    ctx->stage_bytes = need;
+  }
+  char *base = (char *)ctx->d_stage;
+  size_t off = 0;
+  auto up = [&](const void *h, size_t bytes, size_t slot) -> const void * {
+    void *d = base + off;
+    off += slot;
+    if (!h) return nullptr;
+    if (cudaMemcpyAsync(d, h, bytes, cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess) return (const void *)-1;
+    return d;
+  };
+  sched_jobs dj;
+  const float *const hf[10] = {h_jobs->alpha_grad, h_jobs->beta_grad, h_jobs->alpha_local, h_jobs->beta_local,
+                               h_jobs->alpha_node, h_jobs->beta_node, h_jobs->gamma, h_jobs->phi,
+                               h_jobs->m0, h_jobs->m_max_total};
+  const float **df[10] = {&dj.alpha_grad, &dj.beta_grad, &dj.alpha_local, &dj.beta_local, &dj.alpha_node,
+                          &dj.beta_node, &dj.gamma, &dj.phi, &dj.m0, &dj.m_max_total};
+  bool bad = false;
+  for (int i = 0; i < 10; ++i) {
+    *df[i] = (const float *)up(hf[i], J * 4, f32);
+    bad |= (*df[i] == (const float *)-1);
+  }
+  dj.m_grid = (const int32_t *)up(h_jobs->m_grid, J * c.grid_m * 4, grid);
+  dj.k_cap = (const int32_t *)up(h_jobs->k_cap, J * 4, f32);
+  dj.fair_k = (const int32_t *)up(h_jobs->fair_k, J * 4, f32);
+  dj.fair_n = (const int32_t *)up(h_jobs->fair_n, J * 4, f32);
+  dj.age_sec = (const float *)up(h_jobs->age_sec, J * 4, f32);
+  dj.num_restarts = (const int32_t *)up(h_jobs->num_restarts, J * 4, f32);
+  dj.active = (const uint8_t *)up(h_jobs->active, J, u8);
+  const int16_t *d_cur = (const int16_t *)up(h_cur, mat, align256(mat));
+  bad |= dj.m_grid == (const void *)-1 || dj.k_cap == (const void *)-1 || dj.fair_k == (const void *)-1 ||
+         dj.fair_n == (const void *)-1 || dj.age_sec == (const void *)-1 ||
+         dj.num_restarts == (const void *)-1 || dj.active == (const void *)-1 || d_cur == (const void *)-1;
+  REQUIRE(ctx, !bad, SCHED_ERR_CUDA, "schedule_round_host: a host-to-device copy failed: %s",
+          cudaGetErrorString(cudaGetLastError()));
+  int16_t *d_best = (int16_t *)(base + off);
+  off += align256(mat);
+  float *d_bf = (float *)(base + off);
+  rc = schedule_round(ctx, &dj, d_cur, round, generations, d_best, d_bf);
+  if (rc != SCHED_OK) return rc;
+  SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(h_best, d_best, mat, cudaMemcpyDeviceToHost, ctx->stream));
+  SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(h_best_fitness, d_bf, sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
+  SCHED_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
+  return SCHED_OK;
+}
+
+int eval_fitness_host(sched_ctx *ctx, const int16_t *h_pop, int32_t count, const float *h_speedup,
+                      const int16_t *h_cur, const float *h_realloc_factor, const uint8_t *h_active,
+                      float p, float *h_fitness) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "eval_fitness_host: ctx is NULL");
+  REQUIRE(ctx, count >= 0 && (count == 0 || (h_pop && h_speedup && h_fitness)), SCHED_ERR_INVALID_ARG,
+          "eval_fitness_host: h_pop, h_speedup and h_fitness must be non-NULL");
+  if (count == 0) return SCHED_OK;
+  const sched_config &c = ctx->cfg;
+  const size_t J = (size_t)c.num_jobs, mat = J * c.num_nodes * sizeof(int16_t);
+  const size_t pop_b = align256(mat * count), tab_b = align256(J * ctx->KD * ctx->ND * 4);
+  const size_t need = pop_b + tab_b + align256(mat) + align256(J * 4) + align256(J) + align256((size_t)count * 4);
+  if (need > ctx->stage_fit_bytes) {
+    if (ctx->d_stage_fit) {
+      SCHED_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
+      SCHED_CUDA_CHECK(ctx, cudaFree(ctx->d_stage_fit));
+      ctx->d_stage_fit = nullptr;
+      ctx->stage_fit_bytes = 0;
+    }
+    SCHED_CUDA_CHECK(ctx, cudaMalloc(&ctx->d_stage_fit, need));
+    ctx->stage_fit_bytes = need;
+  }
+  char *base = (char *)ctx->d_stage_fit;
+  int16_t *d_pop = (int16_t *)base;
+  float *d_tab = (float *)(base + pop_b);
+  int16_t *d_cur = (int16_t *)(base + pop_b + tab_b);
+  float *d_rf = (float *)(base + pop_b + tab_b + align256(mat));
+  uint8_t *d_act = (uint8_t *)(base + pop_b + tab_b + align256(mat) + align256(J * 4));
+  float *d_fit = (float *)(base + pop_b + tab_b + align256(mat) + align256(J * 4) + align256(J));
+  SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(d_pop, h_pop, mat * count, cudaMemcpyHostToDevice, ctx->stream));
+  SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(d_tab, h_speedup, J * ctx->KD * ctx->ND * 4, cudaMemcpyHostToDevice, ctx->stream));
+  if (h_cur) SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(d_cur, h_cur, mat, cudaMemcpyHostToDevice, ctx->stream));
+  if (h_realloc_factor) SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(d_rf, h_realloc_factor, J * 4, cudaMemcpyHostToDevice, ctx->stream));
+  if (h_active) SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(d_act, h_active, J, cudaMemcpyHostToDevice, ctx->stream));
+  int rc = eval_fitness(ctx, d_pop, count, d_tab, h_cur ? d_cur : nullptr, h_realloc_factor ? d_rf : nullptr,
+                        h_active ? d_act : nullptr, p, d_fit);
+  if (rc != SCHED_OK) return rc;
+  SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(h_fitness, d_fit, (size_t)count * 4, cudaMemcpyDeviceToHost, ctx->stream));
+  SCHED_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
+  return SCHED_OK;
+}
+
+#pragma GCC visibility pop
+}  // extern "C"

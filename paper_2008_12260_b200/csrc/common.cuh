@@ -1,0 +1,157 @@
+// Shared declarations of the PolluxSched CUDA library: context, error plumbing,
+// the counter-based random stream, small device helpers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "polluxsched.h"
+
+#define SLOT_SELECT 0u
+#define SLOT_XOVER 1u
+#define SLOT_MUTATE 2u
+#define SLOT_REPAIR_INTF 3u
+#define SLOT_REPAIR_CAP 4u
+#define SLOT_INIT 5u
+#define GEN_INIT 0xFFFFFFFFu
+
+struct sched_ctx {
+  sched_config cfg;
+  cudaStream_t stream;
+  int device;
+  int num_sms;
+  int KD, ND;
+  int64_t launches;
+  char err[256];
+
+  // device scratch owned by the context
+  int16_t *d_cap;        // [num_nodes]
+  int32_t *d_kfit;       // [ND] replicas that fit on the N largest nodes
+  float *d_gmax;         // [J][KD][2] compact goodput maxima (class local / node)
+  uint16_t *d_amax;      // [J][KD][2]
+  int32_t *d_rank;       // [P]
+  int32_t *d_order;      // [P] inverse of rank
+  uint8_t *d_dflag;      // [P][J] "row spans >= 2 nodes" after the row pass
+  float *d_pen;          // [J] effective penalty factor (1 when none applies)
+  double *d_partial;     // [count][chunks] partial sums of the fitness reduction
+  unsigned int *d_ticket;  // [count] arrival counters of the fitness reduction
+  size_t partial_cap, ticket_cap, dflag_cap;
+  int *d_status;         // device status word
+
+  // scratch of schedule_round (allocated on first use)
+  int16_t *d_popA, *d_popB;
+  float *d_fit;          // [P]
+  float *d_tab_goodput, *d_tab_speedup;
+  float *d_rf;           // [J]
+  int32_t *d_best_idx;
+  int16_t *d_pop_last;   // points at d_popA or d_popB after a round
+  bool round_ready;
+
+  // staging for the *_host entry points (allocated on first use)
+  void *d_stage;         // job arrays + cur + best
+  size_t stage_bytes;
+  void *d_stage_fit;     // eval_fitness_host staging
+  size_t stage_fit_bytes;
+};
+
+const char *set_error(sched_ctx *ctx, const char *fmt, ...);
+extern char g_init_error[256];
+
+#define SCHED_CUDA_CHECK(ctx, call)                                                        \
+  do {                                                                                     \
+    cudaError_t e__ = (call);                                                              \
+    if (e__ != cudaSuccess) {                                                              \
+      set_error(ctx, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e__), __FILE__,    \
+                __LINE__);                                                                 \
+      return SCHED_ERR_CUDA;                                                               \
+    }                                                                                      \
+  } while (0)
+
+#define SCHED_LAUNCH_CHECK(ctx)                                                            \
+  do {                                                                                     \
+    (ctx)->launches++;                                                                     \
+    cudaError_t e__ = cudaGetLastError();                                                  \
+    if (e__ != cudaSuccess) {                                                              \
+      set_error(ctx, "kernel launch failed: %s (%s:%d)", cudaGetErrorString(e__),          \
+                __FILE__, __LINE__);                                                       \
+      return SCHED_ERR_CUDA;                                                               \
+    }                                                                                      \
+  } while (0)
+
+// ---------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies; the key is
+// advanced by the Weyl constants before every round except the first.
+// ---------------------------------------------------------------------------------------
+struct u32x4 {
+  uint32_t x, y, z, w;
+};
+
+__host__ __device__ __forceinline__ u32x4 philox4x32_10(u32x4 c, uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+#ifdef __CUDA_ARCH__
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+#else
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c.x, p1 = (uint64_t)0xCD9E8D57u * c.z;
+    const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+    const uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
+#endif
+    u32x4 n;
+    n.x = hi1 ^ c.y ^ k0;
+    n.y = lo1;
+    n.z = hi0 ^ c.w ^ k1;
+    n.w = lo0;
+    c = n;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return c;
+}
+
+// Random stream of the operators: key = (seed_lo ^ seed_hi, round),
+// counter = (idx, candidate, generation, slot).
+struct RngKey {
+  uint32_t k0, k1;
+};
+
+__host__ __device__ __forceinline__ RngKey make_key(uint64_t seed, uint32_t round) {
+  RngKey k;
+  k.k0 = (uint32_t)seed ^ (uint32_t)(seed >> 32);
+  k.k1 = round;
+  return k;
+}
+
+__device__ __forceinline__ u32x4 draw(RngKey k, uint32_t idx, uint32_t cand, uint32_t gen,
+                                      uint32_t slot) {
+  u32x4 c = {idx, cand, gen, slot};
+  return philox4x32_10(c, k.k0, k.k1);
+}
+
+// floor(w * n / 2^32): an integer in [0, n)
+__device__ __forceinline__ uint32_t bounded(uint32_t w, uint32_t n) { return __umulhi(w, n); }
+
+// order-preserving integer image of an fp32 bit pattern
+__device__ __forceinline__ uint32_t order_key(uint32_t bits) {
+  return bits ^ ((bits >> 31) ? 0xFFFFFFFFu : 0x80000000u);
+}
+
+// kernels' launchers (defined in table.cu / fitness.cu / ga.cu)
+int launch_speedup_table(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodput, float *d_speedup,
+                         uint16_t *d_argmax);
+int launch_realloc_factor(sched_ctx *ctx, const sched_jobs *jobs, float *d_out);
+int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const float *d_speedup,
+                   const int16_t *d_cur, const float *d_rf, const uint8_t *d_active, float p,
+                   float *d_fitness);
+int launch_repair(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active, int16_t *d_pop,
+                  int32_t count, uint32_t first_candidate, uint32_t round, uint32_t generation);
+int launch_init_population(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active,
+                           const int16_t *d_cur, uint32_t round, int16_t *d_pop_out);
+int launch_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active,
+                      const int16_t *d_pop_in, const float *d_fitness_in, int16_t *d_pop_out,
+                      uint32_t round, uint32_t generation);
+int launch_select_best(sched_ctx *ctx, const int16_t *d_pop, const float *d_fitness,
+                       int16_t *d_best, float *d_best_fitness);
+int ensure_fitness_scratch(sched_ctx *ctx, int32_t count, int chunks);
+int ensure_dflag(sched_ctx *ctx, int32_t count);

@@ -1,0 +1,287 @@
+// Population fitness (Eq. 14): per (candidate, job) row summary (K = SUM(a), N = occupied
+// nodes, "row differs from the current allocation"), speedup gather, re-allocation
+// penalty, floor, and the power-mean reduction over the active jobs.
+//
+// The kernel streams the dense int16 population once with wide loads.  Rows are split
+// over LPR lanes (a power of two <= 32); a warp summarises 32 rows, parks each row's
+// packed (K, N, changed) in one lane, and then all 32 lanes do the gather / penalty /
+// power term for their row at once.  A block covers a contiguous chunk of one
+// candidate's rows; chunk sums go to a scratch array and the last block to arrive adds
+// them in index order, so results are bitwise reproducible.
+#include "common.cuh"
+
+namespace {
+
+enum { MODE_POW = 0, MODE_ARITH = 1, MODE_HARM = 2, MODE_GEO = 3, MODE_SQRT = 4 };
+
+template <int W>
+struct VecLoad;
+template <>
+struct VecLoad<16> {
+  static __device__ __forceinline__ uint4 ld(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+  }
+  static __device__ __forceinline__ uint4 ld_cached(const void *p) { return __ldg((const uint4 *)p); }
+};
+template <>
+struct VecLoad<8> {
+  static __device__ __forceinline__ uint4 ld(const void *p) {
+    const uint2 t = __ldg((const uint2 *)p);
+    return make_uint4(t.x, t.y, 0u, 0u);
+  }
+  static __device__ __forceinline__ uint4 ld_cached(const void *p) { return ld(p); }
+};
+template <>
+struct VecLoad<4> {
+  static __device__ __forceinline__ uint4 ld(const void *p) {
+    return make_uint4(__ldg((const uint32_t *)p), 0u, 0u, 0u);
+  }
+  static __device__ __forceinline__ uint4 ld_cached(const void *p) { return ld(p); }
+};
+template <>
+struct VecLoad<2> {
+  static __device__ __forceinline__ uint4 ld(const void *p) {
+    return make_uint4((uint32_t)__ldg((const uint16_t *)p), 0u, 0u, 0u);
+  }
+  static __device__ __forceinline__ uint4 ld_cached(const void *p) { return ld(p); }
+};
+
+// per 32-bit word (two int16 entries): signed sum, and count of entries > 0
+__device__ __forceinline__ void summarise_word(uint32_t w, int &ksum, uint32_t &npos) {
+  ksum = __dp2a_lo((int)w, 0x0101, ksum);
+  npos += __vimin_s16x2_relu(w, 0x00010001u);   // min(v, 1) floored at 0, per half
+}
+
+struct FitnessArgs {
+  const int16_t *pop;
+  const int16_t *cur;
+  const float *table;
+  const float *pen;       // [J] factor applied to changed rows, or NULL
+  const uint8_t *active;  // or NULL
+  int J, num_nodes, k_max, n_max;
+  int lpr_log2;           // lanes per row = 1 << lpr_log2
+  int rows_per_block, chunks;
+  int mode;
+  float p, floor_;
+  double *partial;        // [count][chunks][2]: sum of terms, number of active rows
+  unsigned int *ticket;   // [count]
+  float *fitness;
+};
+
+template <int W>
+__global__ void __launch_bounds__(256) fitness_kernel(FitnessArgs a) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const int cand = blockIdx.y, chunk = blockIdx.x;
+  const int LPR = 1 << a.lpr_log2, RPW = 32 >> a.lpr_log2;
+  const int group = lane >> a.lpr_log2, sub = lane & (LPR - 1);
+  const unsigned gmask = (LPR == 32) ? 0xffffffffu : (((1u << LPR) - 1u) << (group * LPR));
+  const int row_vecs = (a.num_nodes * 2) / W;
+  const int j0 = chunk * a.rows_per_block;
+  const int j1 = min(a.J, j0 + a.rows_per_block);
+  const int KD = a.k_max + 1, ND = a.n_max + 1;
+  const char *cand_base = (const char *)(a.pop + (size_t)cand * a.J * a.num_nodes);
+  const char *cur_base = (const char *)a.cur;
+  const size_t row_bytes = (size_t)a.num_nodes * 2;
+
+  double acc = 0.0;
+  int cnt = 0;
+  uint32_t mine = 0;
+  int myrow = -1;
+  int it = 0;
+  const int slots_per_fill = LPR;        // iterations that fill all 32 lanes
+
+  // warp-uniform loop: every lane takes part in the shuffles of every iteration
+  for (int jb = j0 + warp * RPW; jb < j1; jb += nwarps * RPW, ++it) {
+    const int j = jb + group;
+    const bool live = j < j1;
+    int ksum = 0;
+    uint32_t npos = 0, diff = 0;
+    if (live) {
+      const char *row = cand_base + (size_t)j * row_bytes;
+      const char *crow = cur_base ? cur_base + (size_t)j * row_bytes : nullptr;
+#pragma unroll 4
+      for (int v = sub; v < row_vecs; v += LPR) {
+        const uint4 x = VecLoad<W>::ld(row + (size_t)v * W);
+        if ((x.x | x.y | x.z | x.w) != 0u) {
+          summarise_word(x.x, ksum, npos);
+          if (W >= 8) summarise_word(x.y, ksum, npos);
+          if (W >= 16) { summarise_word(x.z, ksum, npos); summarise_word(x.w, ksum, npos); }
+        }
+        if (crow) {
+          const uint4 c = VecLoad<W>::ld_cached(crow + (size_t)v * W);
+          diff |= (x.x ^ c.x) | (x.y ^ c.y) | (x.z ^ c.z) | (x.w ^ c.w);
+        }
+      }
+    }
+    // saturate the lane-local counts so that the packed fields cannot overflow when
+    // 32 lanes are added: K in bits 0..15 (<= 32 * 2047), N in bits 16..31
+    int nl = (int)((npos & 0xFFFFu) + (npos >> 16));
+    ksum = max(0, min(ksum, 2047));
+    nl = min(nl, 2047);
+    uint32_t packed = (uint32_t)ksum | ((uint32_t)nl << 16);
+    for (int off = LPR >> 1; off >= 1; off >>= 1) packed += __shfl_xor_sync(0xffffffffu, packed, off);
+    const unsigned changed = __ballot_sync(0xffffffffu, diff != 0u) & gmask;
+    // lane `sub` of each group parks the row its group summarised in iteration `sub`
+    if (live && sub == (it & (LPR - 1))) {
+      // K <= 32*2047 < 2^16, N likewise; keep "changed" in the top bit of the N field
+      mine = (packed & 0x7FFFFFFFu) | (changed ? 0x80000000u : 0u);
+      myrow = j;
+    }
+    const bool flush = ((it + 1) % slots_per_fill == 0) || (jb + nwarps * RPW >= j1);
+    if (flush) {
+      if (myrow >= 0 && (!a.active || a.active[myrow])) {
+        const int K = min((int)(mine & 0xFFFFu), a.k_max);
+        const int N = min((int)((mine >> 16) & 0x7FFFu), a.n_max);
+        float x = __ldg(a.table + ((size_t)myrow * KD + K) * ND + N);
+        if (a.pen && (mine >> 31)) x *= a.pen[myrow];
+        x = fmaxf(x, a.floor_);
+        float t;
+        switch (a.mode) {
+          case MODE_ARITH: t = x; break;
+          case MODE_HARM: t = 1.f / x; break;
+          case MODE_GEO: t = logf(x); break;
+          case MODE_SQRT: t = sqrtf(x); break;
+          default: t = powf(x, a.p); break;
+        }
+        acc += (double)t;
+        cnt += 1;
+      }
+      myrow = -1;
+    }
+  }
+
+  // block reduction in a fixed order
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
+  }
+  __shared__ double s_acc[8];
+  __shared__ int s_cnt[8];
+  __shared__ bool s_last;
+  if (lane == 0) { s_acc[warp] = acc; s_cnt[warp] = cnt; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    int n = 0;
+    for (int w = 0; w < nwarps; ++w) { t += s_acc[w]; n += s_cnt[w]; }
+    double *dst = a.partial + ((size_t)cand * a.chunks + chunk) * 2;
+    dst[0] = t;
+    dst[1] = (double)n;
+    __threadfence();
+    const unsigned prev = atomicAdd(a.ticket + cand, 1u);
+    s_last = (prev == (unsigned)a.chunks - 1u);
+  }
+  __syncthreads();
+  if (s_last && threadIdx.x == 0) {
+    __threadfence();
+    const volatile double *src = a.partial + (size_t)cand * a.chunks * 2;
+    double t = 0.0, n = 0.0;
+    for (int c = 0; c < a.chunks; ++c) { t += src[2 * c]; n += src[2 * c + 1]; }
+    double f;
+    if (n == 0.0) f = 0.0;
+    else {
+      const double mean = t / n;
+      switch (a.mode) {
+        case MODE_ARITH: f = mean; break;
+        case MODE_HARM: f = 1.0 / mean; break;
+        case MODE_GEO: f = exp(mean); break;
+        case MODE_SQRT: f = mean * mean; break;
+        default: f = pow(mean, 1.0 / (double)a.p); break;
+      }
+    }
+    a.fitness[cand] = (float)f;
+    a.ticket[cand] = 0u;   // ready for the next call on this stream
+  }
+}
+
+// Effective penalty per job: the re-allocation factor when the job currently holds GPUs,
+// else 1 (pending jobs are never penalised).  One warp per job.
+__global__ void penalty_prep_kernel(const int16_t *__restrict__ cur, const float *__restrict__ rf,
+                                    int J, int num_nodes, float *__restrict__ pen) {
+  const int lane = threadIdx.x & 31;
+  const int j = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (j >= J) return;
+  long long k = 0;
+  for (int n = lane; n < num_nodes; n += 32) k += cur[(size_t)j * num_nodes + n];
+  for (int off = 16; off >= 1; off >>= 1) k += __shfl_xor_sync(0xffffffffu, k, off);
+  if (lane == 0) pen[j] = (k > 0) ? rf[j] : 1.f;
+}
+
+}  // namespace
+
+int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const float *d_speedup,
+                   const int16_t *d_cur, const float *d_rf, const uint8_t *d_active, float p,
+                   float *d_fitness) {
+  const sched_config &c = ctx->cfg;
+  const int J = c.num_jobs;
+  if (count == 0) return SCHED_OK;
+
+  const bool penalise = d_cur && d_rf;
+  if (penalise && J > 0) {
+    penalty_prep_kernel<<<(J * 32 + 255) / 256, 256, 0, ctx->stream>>>(d_cur, d_rf, J, c.num_nodes,
+                                                                       ctx->d_pen);
+    SCHED_LAUNCH_CHECK(ctx);
+  }
+
+  // widest vector that divides the row and keeps every row aligned
+  const size_t row_bytes = (size_t)c.num_nodes * 2;
+  const uintptr_t al = (uintptr_t)d_pop | (penalise ? (uintptr_t)d_cur : 0);
+  int W = 2;
+  if (row_bytes % 16 == 0 && al % 16 == 0) W = 16;
+  else if (row_bytes % 8 == 0 && al % 8 == 0) W = 8;
+  else if (row_bytes % 4 == 0 && al % 4 == 0) W = 4;
+  const int row_vecs = (int)(row_bytes / W);
+  int lpr_log2 = 0;
+  while ((1 << lpr_log2) < row_vecs && lpr_log2 < 5) ++lpr_log2;
+
+  // chunk of rows per block: about 1 MB of population, at least 32 rows per warp batch
+  int rows_per_block = (int)((1u << 20) / row_bytes);
+  if (rows_per_block < 256) rows_per_block = 256;
+  if (rows_per_block > J) rows_per_block = J > 0 ? J : 1;
+  // keep enough blocks in flight for small populations
+  while (rows_per_block > 256 && (long long)count * ((J + rows_per_block - 1) / rows_per_block) <
+                                     4LL * ctx->num_sms)
+    rows_per_block = (rows_per_block + 1) / 2;
+  const int chunks = J > 0 ? (J + rows_per_block - 1) / rows_per_block : 1;
+  int rc = ensure_fitness_scratch(ctx, count, chunks);
+  if (rc != SCHED_OK) return rc;
+
+  FitnessArgs a;
+  a.pop = d_pop;
+  a.cur = penalise ? d_cur : nullptr;
+  a.table = d_speedup;
+  a.pen = penalise ? ctx->d_pen : nullptr;
+  a.active = d_active;
+  a.J = J; a.num_nodes = c.num_nodes; a.k_max = c.k_max; a.n_max = c.n_max;
+  a.lpr_log2 = lpr_log2;
+  a.rows_per_block = rows_per_block; a.chunks = chunks;
+  a.p = p; a.floor_ = c.speedup_floor;
+  a.mode = (p == 1.f) ? MODE_ARITH : (p == -1.f) ? MODE_HARM : (p == 0.f) ? MODE_GEO
+           : (p == 0.5f) ? MODE_SQRT : MODE_POW;
+  a.partial = ctx->d_partial;
+  a.ticket = ctx->d_ticket;
+  a.fitness = d_fitness;
+
+  // grid.y is limited to 65535 candidates per launch
+  for (int32_t first = 0; first < count; first += 65535) {
+    const int32_t n = (count - first < 65535) ? (count - first) : 65535;
+    FitnessArgs b = a;
+    b.pop = d_pop + (size_t)first * J * c.num_nodes;
+    b.partial = ctx->d_partial + (size_t)first * chunks * 2;
+    b.ticket = ctx->d_ticket + first;
+    b.fitness = d_fitness + first;
+    dim3 grid((unsigned)chunks, (unsigned)n);
+    switch (W) {
+      case 16: fitness_kernel<16><<<grid, 256, 0, ctx->stream>>>(b); break;
+      case 8: fitness_kernel<8><<<grid, 256, 0, ctx->stream>>>(b); break;
+      case 4: fitness_kernel<4><<<grid, 256, 0, ctx->stream>>>(b); break;
+      default: fitness_kernel<2><<<grid, 256, 0, ctx->stream>>>(b); break;
+    }
+    SCHED_LAUNCH_CHECK(ctx);
+  }
+  return SCHED_OK;
+}

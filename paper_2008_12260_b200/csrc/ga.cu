@@ -1,0 +1,413 @@
+// Population-search operators (Sec. 4.3): ranking, parent selection + row-wise crossover
+// + row perturbation, and the repair that enforces node capacity and interference
+// avoidance (Sec. 4.2).  Integer work only; all randomness comes from the counter-based
+// stream, so every output is a pure function of the inputs.
+//
+// Structure: a row kernel (one warp per (candidate, job) row: build the child row in
+// shared memory, perturb, apply the per-row caps, write it and a "spans >= 2 nodes" flag)
+// followed by a column kernel (one thread per (candidate, node): interference and
+// capacity passes over the jobs of that node).
+#include "common.cuh"
+
+namespace {
+
+enum { ROWS_GENERATION = 0, ROWS_INIT = 1, ROWS_REPAIR = 2 };
+
+// rank[i] = number of candidates ordered before i (fitness descending, index ascending)
+__global__ void __launch_bounds__(128)
+rank_kernel(const uint32_t *__restrict__ fitness_bits, int P, int32_t *__restrict__ rank,
+            int32_t *__restrict__ order) {
+  __shared__ uint32_t tile[128];
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  const uint32_t ki = (i < P) ? order_key(fitness_bits[i]) : 0u;
+  int r = 0;
+  for (int base = 0; base < P; base += 128) {
+    const int o = base + threadIdx.x;
+    tile[threadIdx.x] = (o < P) ? order_key(fitness_bits[o]) : 0u;
+    __syncthreads();
+    const int lim = min(128, P - base);
+    for (int t = 0; t < lim; ++t) {
+      const uint32_t ko = tile[t];
+      r += (ko > ki || (ko == ki && base + t < i)) ? 1 : 0;
+    }
+    __syncthreads();
+  }
+  if (i < P) {
+    rank[i] = r;
+    order[r] = i;
+  }
+}
+
+struct RowsArgs {
+  const int16_t *src;       // parents [P][J][N], or the current allocation [J][N] (may be NULL), or dst
+  int16_t *dst;             // children [count][J][N]
+  const int16_t *cap;       // [N]
+  const int32_t *k_cap;     // [J] or NULL
+  const uint8_t *active;    // [J] or NULL
+  const int32_t *rank;      // [P]   (generation mode)
+  const int32_t *order;     // [P]
+  uint8_t *dflag;           // [count][J]
+  int mode, P, J, num_nodes, k_max, n_max, num_elite, count;
+  uint32_t thr, gen, first_cand;
+  RngKey key;
+};
+
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+  return v;
+}
+
+// node index of the t-th occupied entry (ascending) of a row held in shared memory
+__device__ __forceinline__ int nth_occupied(const int16_t *row, int num_nodes, uint32_t t, int lane) {
+  for (int base = 0; base < num_nodes; base += 32) {
+    const int n = base + lane;
+    const unsigned m = __ballot_sync(0xffffffffu, n < num_nodes && row[n] > 0);
+    const uint32_t c = __popc(m);
+    if (t < c) return base + (int)__fns(m, 0, (int)t + 1);
+    t -= c;
+  }
+  return -1;
+}
+
+__global__ void __launch_bounds__(256) rows_kernel(RowsArgs a) {
+  extern __shared__ __align__(16) int16_t s_rows[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const long long gw = (long long)blockIdx.x * (blockDim.x >> 5) + warp;
+  if (gw >= (long long)a.count * a.J) return;
+  const int cl = (int)(gw / a.J), j = (int)(gw % a.J);
+  const uint32_t c = a.first_cand + (uint32_t)cl;
+  const int NN = a.num_nodes;
+  const int row_stride = (NN + 7) & ~7;
+  int16_t *row = s_rows + (size_t)warp * row_stride;
+  int16_t *out = a.dst + ((size_t)cl * a.J + j) * NN;
+  const bool vec = ((NN & 7) == 0) && ((((uintptr_t)a.dst | (uintptr_t)a.src) & 15) == 0);
+
+  if (a.active && !a.active[j]) {
+    if (vec) for (int v = lane; v < NN / 8; v += 32) ((uint4 *)out)[v] = make_uint4(0, 0, 0, 0);
+    else for (int n = lane; n < NN; n += 32) out[n] = 0;
+    if (lane == 0) a.dflag[(size_t)cl * a.J + j] = 0;
+    return;
+  }
+
+  // which row feeds this child row, and the perturbation draw
+  const int16_t *src = nullptr;
+  bool mutate = false;
+  u32x4 mw = {0, 0, 0, 0};
+  if (a.mode == ROWS_GENERATION) {
+    int parent;
+    if ((int)c < a.num_elite) {
+      parent = a.order[c];
+    } else {
+      const u32x4 s = draw(a.key, 0u, c, a.gen, SLOT_SELECT);
+      const int i0 = bounded(s.x, a.P), i1 = bounded(s.y, a.P);
+      const int i2 = bounded(s.z, a.P), i3 = bounded(s.w, a.P);
+      const int pa = a.rank[i0] <= a.rank[i1] ? i0 : i1;
+      const int pb = a.rank[i2] <= a.rank[i3] ? i2 : i3;
+      const u32x4 x = draw(a.key, (uint32_t)j, c, a.gen, SLOT_XOVER);
+      parent = (x.x >> 31) ? pb : pa;
+      mw = draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE);
+      mutate = mw.x < a.thr;
+    }
+    src = a.src + ((size_t)parent * a.J + j) * NN;
+  } else if (a.mode == ROWS_INIT) {
+    src = a.src ? a.src + (size_t)j * NN : nullptr;
+    if (c > 0) {
+      mw = draw(a.key, (uint32_t)j, c, GEN_INIT, SLOT_INIT);
+      mutate = mw.x < a.thr;
+    }
+  } else {
+    src = out;
+  }
+
+  // load into shared memory, every entry forced into [0, capacity of its node]
+  int K = 0, N = 0;
+  if (!src) {
+    for (int n = lane; n < row_stride; n += 32) row[n] = 0;
+  } else if (vec) {
+    for (int v = lane; v < NN / 8; v += 32) {
+      uint4 x = __ldg((const uint4 *)src + v);
+      const uint4 cp = __ldg((const uint4 *)a.cap + v);
+      x.x = __vimin_s16x2_relu(x.x, __vimax_s16x2_relu(cp.x, 0u));
+      x.y = __vimin_s16x2_relu(x.y, __vimax_s16x2_relu(cp.y, 0u));
+      x.z = __vimin_s16x2_relu(x.z, __vimax_s16x2_relu(cp.z, 0u));
+      x.w = __vimin_s16x2_relu(x.w, __vimax_s16x2_relu(cp.w, 0u));
+      ((uint4 *)row)[v] = x;
+      const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        K += (int)(w[q] & 0xFFFFu) + (int)(w[q] >> 16);
+        N += ((w[q] & 0xFFFFu) != 0u) + ((w[q] >> 16) != 0u);
+      }
+    }
+  } else {
+    for (int n = lane; n < NN; n += 32) {
+      const int cp = max((int)a.cap[n], 0);
+      const int v = min(max((int)src[n], 0), cp);
+      row[n] = (int16_t)v;
+      K += v;
+      N += v > 0;
+    }
+  }
+  K = warp_sum(K);
+  N = warp_sum(N);
+  __syncwarp();
+
+  if (mutate) {
+    const uint32_t op = bounded(mw.y, 3u);
+    if (op == 0u) {
+      const int n = (int)bounded(mw.w, (uint32_t)NN);
+      if (lane == 0) row[n] = (int16_t)min((int)row[n] + 1, max((int)a.cap[n], 0));
+    } else if (N > 0) {
+      const int ns = nth_occupied(row, NN, bounded(mw.z, (uint32_t)N), lane);
+      if (op == 1u) {
+        if (lane == 0) row[ns] = (int16_t)(row[ns] - 1);
+      } else {
+        const int nd = (int)bounded(mw.w, (uint32_t)NN);
+        if (nd != ns && lane == 0) {
+          row[nd] = (int16_t)min((int)row[nd] + (int)row[ns], max((int)a.cap[nd], 0));
+          row[ns] = 0;
+        }
+      }
+    }
+    __syncwarp();
+    K = 0; N = 0;
+    for (int n = lane; n < NN; n += 32) { K += row[n]; N += row[n] > 0; }
+    K = warp_sum(K);
+    N = warp_sum(N);
+  }
+
+  // per-row caps: replicas above the job's cap leave from the highest node index down,
+  // then occupied nodes beyond n_max are cleared from the highest index down
+  int kc = a.k_cap ? a.k_cap[j] : a.k_max;
+  kc = max(0, min(kc, a.k_max));
+  if (K > kc || N > a.n_max) {
+    if (lane == 0) {
+      int excess = K - kc;
+      for (int n = NN - 1; n >= 0 && excess > 0; --n) {
+        const int take = min((int)row[n], excess);
+        row[n] = (int16_t)(row[n] - take);
+        excess -= take;
+      }
+      int occ = 0;
+      for (int n = 0; n < NN; ++n) {
+        if (row[n] > 0) {
+          ++occ;
+          if (occ > a.n_max) row[n] = 0;
+        }
+      }
+      N = min(occ, a.n_max);
+    }
+    N = __shfl_sync(0xffffffffu, N, 0);
+    __syncwarp();
+  }
+
+  if (vec) for (int v = lane; v < NN / 8; v += 32) ((uint4 *)out)[v] = ((const uint4 *)row)[v];
+  else for (int n = lane; n < NN; n += 32) out[n] = row[n];
+  if (lane == 0) a.dflag[(size_t)cl * a.J + j] = (N >= 2) ? 1 : 0;
+}
+
+struct ColsArgs {
+  int16_t *pop;             // [count][J][N], repaired in place
+  const uint8_t *dflag;     // [count][J]
+  const int16_t *cap;
+  int J, num_nodes, count;
+  uint32_t gen, first_cand;
+  RngKey key;
+};
+
+// One thread per (candidate, node).  Interference avoidance: of the jobs flagged as
+// distributed that occupy the node, only the first in job order rotated by the node's
+// draw stays.  Capacity: GPUs above the node's size are taken from its jobs in job order
+// rotated by a second draw.
+__global__ void __launch_bounds__(128) cols_kernel(ColsArgs a) {
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  const int cl = blockIdx.y;
+  if (n >= a.num_nodes) return;
+  const uint32_t c = a.first_cand + (uint32_t)cl;
+  const int J = a.J, NN = a.num_nodes;
+  int16_t *col = a.pop + (size_t)cl * J * NN + n;
+  const uint8_t *df = a.dflag + (size_t)cl * J;
+  int total = 0, nelig = 0;
+#pragma unroll 8
+  for (int j = 0; j < J; ++j) {
+    const int v = col[(size_t)j * NN];
+    total += v;
+    nelig += (v > 0 && df[j]) ? 1 : 0;
+  }
+  const int cp = max((int)a.cap[n], 0);
+  if (nelig <= 1 && total <= cp) return;
+  if (nelig >= 2) {
+    const int o = (int)bounded(draw(a.key, (uint32_t)n, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
+    int keep = -1, best = J;
+    for (int j = 0; j < J; ++j) {
+      if (df[j] && col[(size_t)j * NN] > 0) {
+        int t = j - o;
+        if (t < 0) t += J;
+        if (t < best) { best = t; keep = j; }
+      }
+    }
+    for (int j = 0; j < J; ++j) {
+      if (j != keep && df[j]) {
+        const int v = col[(size_t)j * NN];
+        if (v > 0) { total -= v; col[(size_t)j * NN] = 0; }
+      }
+    }
+  }
+  int excess = total - cp;
+  if (excess > 0) {
+    const int o = (int)bounded(draw(a.key, (uint32_t)n, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J);
+    for (int t = 0; t < J && excess > 0; ++t) {
+      int j = o + t;
+      if (j >= J) j -= J;
+      const int v = col[(size_t)j * NN];
+      if (v > 0) {
+        const int take = min(v, excess);
+        col[(size_t)j * NN] = (int16_t)(v - take);
+        excess -= take;
+      }
+    }
+  }
+}
+
+// index of the best candidate (largest key, lowest index on ties) and its fitness
+__global__ void __launch_bounds__(256)
+best_index_kernel(const uint32_t *__restrict__ fitness_bits, int P, int32_t *__restrict__ best_idx,
+                  float *__restrict__ best_fitness) {
+  __shared__ unsigned long long s[256];
+  unsigned long long best = 0ull;   // (key << 32) | (0xFFFFFFFF - index): larger is better
+  for (int i = threadIdx.x; i < P; i += blockDim.x) {
+    const unsigned long long v = ((unsigned long long)order_key(fitness_bits[i]) << 32) |
+                                 (unsigned long long)(0xFFFFFFFFu - (uint32_t)i);
+    best = v > best ? v : best;
+  }
+  s[threadIdx.x] = best;
+  __syncthreads();
+  for (int off = 128; off >= 1; off >>= 1) {
+    if ((int)threadIdx.x < off) s[threadIdx.x] = s[threadIdx.x] > s[threadIdx.x + off] ? s[threadIdx.x] : s[threadIdx.x + off];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const int idx = (int)(0xFFFFFFFFu - (uint32_t)(s[0] & 0xFFFFFFFFull));
+    *best_idx = idx;
+    if (best_fitness) *best_fitness = __uint_as_float(fitness_bits[idx]);
+  }
+}
+
+__global__ void copy_best_kernel(const int16_t *__restrict__ pop, const int32_t *__restrict__ best_idx,
+                                 size_t elems, int16_t *__restrict__ out) {
+  const int16_t *src = pop + (size_t)(*best_idx) * elems;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < elems;
+       i += (size_t)gridDim.x * blockDim.x)
+    out[i] = src[i];
+}
+
+int launch_rows(sched_ctx *ctx, RowsArgs &a) {
+  const long long warps = (long long)a.count * a.J;
+  if (warps == 0) return SCHED_OK;
+  const int wpb = 8;
+  const size_t smem = (size_t)wpb * ((a.num_nodes + 7) & ~7) * sizeof(int16_t);
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) {
+      set_error(ctx, "cudaFuncSetAttribute failed: %s", cudaGetErrorString(e));
+      return SCHED_ERR_CUDA;
+    }
+  }
+  const long long blocks = (warps + wpb - 1) / wpb;
+  rows_kernel<<<(unsigned)blocks, wpb * 32, smem, ctx->stream>>>(a);
+  SCHED_LAUNCH_CHECK(ctx);
+  return SCHED_OK;
+}
+
+int launch_cols(sched_ctx *ctx, int16_t *pop, int count, uint32_t first_cand, uint32_t round,
+                uint32_t gen) {
+  if (count == 0 || ctx->cfg.num_jobs == 0) return SCHED_OK;
+  ColsArgs a;
+  a.pop = pop; a.dflag = ctx->d_dflag; a.cap = ctx->d_cap;
+  a.J = ctx->cfg.num_jobs; a.num_nodes = ctx->cfg.num_nodes;
+  a.gen = gen; a.key = make_key(ctx->cfg.seed, round);
+  for (int first = 0; first < count; first += 65535) {
+    const int n = min(65535, count - first);
+    a.count = n;
+    a.first_cand = first_cand + (uint32_t)first;
+    a.pop = pop + (size_t)first * a.J * a.num_nodes;
+    a.dflag = ctx->d_dflag + (size_t)first * a.J;
+    dim3 grid((unsigned)((a.num_nodes + 127) / 128), (unsigned)n);
+    cols_kernel<<<grid, 128, 0, ctx->stream>>>(a);
+    SCHED_LAUNCH_CHECK(ctx);
+  }
+  return SCHED_OK;
+}
+
+RowsArgs base_rows_args(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active, int count) {
+  RowsArgs a;
+  const sched_config &c = ctx->cfg;
+  a.cap = ctx->d_cap; a.k_cap = d_k_cap; a.active = d_active;
+  a.rank = ctx->d_rank; a.order = ctx->d_order; a.dflag = ctx->d_dflag;
+  a.P = c.population; a.J = c.num_jobs; a.num_nodes = c.num_nodes;
+  a.k_max = c.k_max; a.n_max = c.n_max; a.num_elite = c.num_elite; a.count = count;
+  a.thr = 0; a.gen = 0; a.first_cand = 0;
+  a.key = make_key(c.seed, 0);
+  a.src = nullptr; a.dst = nullptr; a.mode = ROWS_REPAIR;
+  return a;
+}
+
+}  // namespace
+
+int launch_repair(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active, int16_t *d_pop,
+                  int32_t count, uint32_t first_candidate, uint32_t round, uint32_t generation) {
+  int rc = ensure_dflag(ctx, count);
+  if (rc != SCHED_OK) return rc;
+  RowsArgs a = base_rows_args(ctx, d_k_cap, d_active, count);
+  a.mode = ROWS_REPAIR; a.src = d_pop; a.dst = d_pop;
+  a.first_cand = first_candidate; a.gen = generation; a.key = make_key(ctx->cfg.seed, round);
+  rc = launch_rows(ctx, a);
+  if (rc != SCHED_OK) return rc;
+  return launch_cols(ctx, d_pop, count, first_candidate, round, generation);
+}
+
+int launch_init_population(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active,
+                           const int16_t *d_cur, uint32_t round, int16_t *d_pop_out) {
+  const int P = ctx->cfg.population;
+  int rc = ensure_dflag(ctx, P);
+  if (rc != SCHED_OK) return rc;
+  RowsArgs a = base_rows_args(ctx, d_k_cap, d_active, P);
+  a.mode = ROWS_INIT; a.src = d_cur; a.dst = d_pop_out;
+  a.thr = ctx->cfg.thr_init; a.gen = GEN_INIT; a.key = make_key(ctx->cfg.seed, round);
+  rc = launch_rows(ctx, a);
+  if (rc != SCHED_OK) return rc;
+  return launch_cols(ctx, d_pop_out, P, 0u, round, GEN_INIT);
+}
+
+int launch_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active,
+                      const int16_t *d_pop_in, const float *d_fitness_in, int16_t *d_pop_out,
+                      uint32_t round, uint32_t generation) {
+  const int P = ctx->cfg.population;
+  int rc = ensure_dflag(ctx, P);
+  if (rc != SCHED_OK) return rc;
+  rank_kernel<<<(P + 127) / 128, 128, 0, ctx->stream>>>((const uint32_t *)d_fitness_in, P,
+                                                         ctx->d_rank, ctx->d_order);
+  SCHED_LAUNCH_CHECK(ctx);
+  RowsArgs a = base_rows_args(ctx, d_k_cap, d_active, P);
+  a.mode = ROWS_GENERATION; a.src = d_pop_in; a.dst = d_pop_out;
+  a.thr = ctx->cfg.thr_mutate; a.gen = generation; a.key = make_key(ctx->cfg.seed, round);
+  rc = launch_rows(ctx, a);
+  if (rc != SCHED_OK) return rc;
+  return launch_cols(ctx, d_pop_out, P, 0u, round, generation);
+}
+
+int launch_select_best(sched_ctx *ctx, const int16_t *d_pop, const float *d_fitness,
+                       int16_t *d_best, float *d_best_fitness) {
+  const int P = ctx->cfg.population;
+  best_index_kernel<<<1, 256, 0, ctx->stream>>>((const uint32_t *)d_fitness, P, ctx->d_best_idx,
+                                                d_best_fitness);
+  SCHED_LAUNCH_CHECK(ctx);
+  const size_t elems = (size_t)ctx->cfg.num_jobs * ctx->cfg.num_nodes;
+  if (elems == 0) return SCHED_OK;
+  const int blocks = (int)((elems + 256 * 8 - 1) / (256 * 8));
+  copy_best_kernel<<<blocks > 1024 ? 1024 : blocks, 256, 0, ctx->stream>>>(d_pop, ctx->d_best_idx,
+                                                                           elems, d_best);
+  SCHED_LAUNCH_CHECK(ctx);
+  return SCHED_OK;
+}

@@ -1,0 +1,223 @@
+// Speedup-table builder: goodput sweep over the (m, s) grid (Eq. 4-11, 13) and
+// normalisation by the fair-share goodput (Eq. 15).
+//
+// The goodput of an allocation depends on the allocation only through K = SUM(a) and
+// whether one or several nodes are occupied (Eq. 9), so the sweep runs once per
+// (job, K, class) with class in {local, node}; a second kernel broadcasts the class
+// results along the N axis of the [J][K][N] tables and divides by the fair-share entry.
+#include "common.cuh"
+
+namespace {
+
+struct JobPtrs {
+  const float *alpha_grad, *beta_grad, *alpha_local, *beta_local, *alpha_node, *beta_node;
+  const float *gamma, *phi, *m0, *m_max_total;
+};
+
+__device__ __forceinline__ float lg2_approx(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// (T_grad^g + T_sync^g)^(1/g) in ratio form: hi * (1 + (lo/hi)^g)^(1/g).  Both exponent
+// arguments stay in [-inf, 1], so the approximate lg2/ex2 keep ~1e-7 relative accuracy.
+__device__ __forceinline__ float overlap_time(float tg, float ts, float gamma, float inv_gamma) {
+  if (ts <= 0.f) return tg;
+  const float hi = fmaxf(tg, ts), lo = fminf(tg, ts);
+  const float r = lo / hi;
+  const float x = ex2_approx(gamma * lg2_approx(r));
+  return hi * ex2_approx(lg2_approx(1.f + x) * inv_gamma);
+}
+
+// A candidate optimum: goodput = num / den; tie = (s << 16) | grid index (smaller wins).
+struct Best {
+  float num, den;
+  uint32_t tie;
+};
+
+__device__ __forceinline__ bool beats(const Best &a, const Best &b) {
+  const float l = a.num * b.den, r = b.num * a.den;
+  return (l > r) || (l == r && a.num > 0.f && a.tie < b.tie);
+}
+
+// One warp per (job, K, class).  Lane l owns grid indices l, l+32, ... (MQ of them per
+// pass); T_grad, the overlapped time and K*m of each are held in registers while the
+// warp sweeps s.  Goodput is compared as num/den by cross-multiplication:
+//   num = M,  den = T_iter * (phi + M) / (phi + M0)   =>  num/den = THROUGHPUT * EFFICIENCY.
+template <int MQ>
+__global__ void __launch_bounds__(256)
+goodput_sweep_kernel(JobPtrs jp, const int32_t *__restrict__ m_grid,
+                     const int32_t *__restrict__ kfit, int J, int k_max, int n_max, int Gm, int Gs,
+                     float *__restrict__ gmax, uint16_t *__restrict__ amax) {
+  const int lane = threadIdx.x & 31;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long total = (long long)J * k_max * 2;
+  if (warp >= total) return;
+  const int cls = (int)(warp & 1);
+  const int K = (int)((warp >> 1) % k_max) + 1;
+  const int j = (int)((warp >> 1) / k_max);
+  const int KD = k_max + 1;
+  const size_t out = ((size_t)j * KD + K) * 2 + cls;
+
+  bool valid;
+  if (cls == 0) valid = K <= kfit[1];
+  else valid = (n_max >= 2) && (K >= 2) && (K <= kfit[min(K, n_max)]);
+  if (!valid) {
+    if (lane == 0) { gmax[out] = 0.f; amax[out] = 0xFFFFu; }
+    return;
+  }
+
+  const float a_g = jp.alpha_grad[j], b_g = jp.beta_grad[j];
+  const float gamma = jp.gamma[j], inv_gamma = 1.f / gamma;
+  const float phi = jp.phi[j], M0 = jp.m0[j], Mmax = jp.m_max_total[j];
+  float ts = 0.f;
+  if (K >= 2) {
+    const float a = cls ? jp.alpha_node[j] : jp.alpha_local[j];
+    const float b = cls ? jp.beta_node[j] : jp.beta_local[j];
+    ts = fmaf(b, (float)(K - 2), a);
+  }
+  const float rinv = 1.f / (phi + M0);   // (phi + M) * rinv = 1 / EFFICIENCY
+  const float c0 = phi * rinv;
+  const float Kf = (float)K;
+
+  Best best = {0.f, 1.f, 0xFFFFFFFFu};
+  for (int base = 0; base < Gm; base += 32 * MQ) {
+    float tg[MQ], tov[MQ], km[MQ], mlo[MQ];
+#pragma unroll
+    for (int q = 0; q < MQ; ++q) {
+      const int i = base + lane + 32 * q;
+      const bool in = i < Gm;
+      const float mf = in ? (float)m_grid[(size_t)j * Gm + i] : 1.f;
+      tg[q] = fmaf(b_g, mf, a_g);
+      tov[q] = overlap_time(tg[q], ts, gamma, inv_gamma);
+      km[q] = Kf * mf;
+      mlo[q] = in ? M0 : __int_as_float(0x7f800000);
+    }
+    float bn = 0.f, bd = 1.f;
+    int code = -1;   // s * MQ + q of this pass's best
+#pragma unroll 4
+    for (int s = 0; s < Gs; ++s) {
+      const float sf = (float)s, sp1 = (float)(s + 1);
+#pragma unroll
+      for (int q = 0; q < MQ; ++q) {
+        const float tit = fmaf(sf, tg[q], tov[q]);
+        const float M = km[q] * sp1;
+        const float den = tit * fmaf(M, rinv, c0);
+        const bool better = (M >= mlo[q]) && (M <= Mmax) && (M * bd > bn * den);
+        bn = better ? M : bn;
+        bd = better ? den : bd;
+        code = better ? s * MQ + q : code;
+      }
+    }
+    if (code >= 0) {
+      Best b;
+      b.num = bn; b.den = bd;
+      b.tie = ((uint32_t)(code / MQ) << 16) | (uint32_t)(base + lane + 32 * (code % MQ));
+      if (beats(b, best)) best = b;
+    }
+  }
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    Best o;
+    o.num = __shfl_xor_sync(0xffffffffu, best.num, off);
+    o.den = __shfl_xor_sync(0xffffffffu, best.den, off);
+    o.tie = __shfl_xor_sync(0xffffffffu, best.tie, off);
+    if (beats(o, best)) best = o;
+  }
+  if (lane == 0) {
+    const bool found = best.num > 0.f;
+    gmax[out] = found ? best.num / best.den : 0.f;
+    amax[out] = found ? (uint16_t)((best.tie & 0xFFFFu) * Gs + (best.tie >> 16)) : (uint16_t)0xFFFFu;
+  }
+}
+
+__device__ __forceinline__ bool kn_valid(int K, int N, int k_max, int n_max,
+                                         const int32_t *__restrict__ kfit) {
+  return N >= 1 && N <= n_max && K >= N && K <= k_max && K <= kfit[N];
+}
+
+// Broadcast the class results along N and divide by the fair-share goodput (Eq. 15).
+__global__ void __launch_bounds__(256)
+speedup_expand_kernel(const float *__restrict__ gmax, const uint16_t *__restrict__ amax,
+                      const int32_t *__restrict__ kfit, const int32_t *__restrict__ fair_k,
+                      const int32_t *__restrict__ fair_n, int J, int k_max, int n_max,
+                      float *__restrict__ goodput, float *__restrict__ speedup,
+                      uint16_t *__restrict__ argmax) {
+  const int KD = k_max + 1, ND = n_max + 1;
+  const long long total = (long long)J * KD * ND;
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= total) return;
+  const int N = (int)(e % ND);
+  const int K = (int)((e / ND) % KD);
+  const int j = (int)(e / ((long long)ND * KD));
+  float g = 0.f;
+  uint16_t a = 0xFFFFu;
+  if (kn_valid(K, N, k_max, n_max, kfit)) {
+    const size_t src = ((size_t)j * KD + K) * 2 + (N >= 2 ? 1 : 0);
+    g = gmax[src];
+    a = amax[src];
+  }
+  const int kf = fair_k[j], nf = fair_n[j];
+  float denom = 0.f;
+  if (kn_valid(kf, nf, k_max, n_max, kfit)) denom = gmax[((size_t)j * KD + kf) * 2 + (nf >= 2 ? 1 : 0)];
+  if (goodput) goodput[e] = g;
+  if (argmax) argmax[e] = a;
+  speedup[e] = denom > 0.f ? g / denom : 0.f;
+}
+
+// REALLOC_FACTOR_j(delta) = (T_j - R_j delta) / (T_j + delta), clamped to [0, 1].
+__global__ void realloc_factor_kernel(const float *__restrict__ age, const int32_t *__restrict__ restarts,
+                                      float delta, int J, float *__restrict__ out) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= J) return;
+  const float T = age[j], R = (float)restarts[j];
+  float f = (T - R * delta) / (T + delta);
+  if (!(f >= 0.f)) f = 0.f;
+  out[j] = fminf(f, 1.f);
+}
+
+}  // namespace
+
+int launch_speedup_table(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodput, float *d_speedup,
+                         uint16_t *d_argmax) {
+  const sched_config &c = ctx->cfg;
+  const int J = c.num_jobs;
+  if (J == 0) return SCHED_OK;
+  JobPtrs jp = {jobs->alpha_grad, jobs->beta_grad, jobs->alpha_local, jobs->beta_local,
+                jobs->alpha_node, jobs->beta_node, jobs->gamma, jobs->phi, jobs->m0,
+                jobs->m_max_total};
+  const long long warps = (long long)J * c.k_max * 2;
+  const int block = 256;
+  const long long blocks = (warps * 32 + block - 1) / block;
+  const int mq = (c.grid_m + 31) / 32;
+#define SWEEP(MQ)                                                                              \
+  goodput_sweep_kernel<MQ><<<(unsigned)blocks, block, 0, ctx->stream>>>(                       \
+      jp, jobs->m_grid, ctx->d_kfit, J, c.k_max, c.n_max, c.grid_m, c.grid_s, ctx->d_gmax,    \
+      ctx->d_amax)
+  if (mq <= 1) SWEEP(1);
+  else if (mq == 2) SWEEP(2);
+  else SWEEP(4);
+#undef SWEEP
+  SCHED_LAUNCH_CHECK(ctx);
+  const long long entries = (long long)J * ctx->KD * ctx->ND;
+  speedup_expand_kernel<<<(unsigned)((entries + 255) / 256), 256, 0, ctx->stream>>>(
+      ctx->d_gmax, ctx->d_amax, ctx->d_kfit, jobs->fair_k, jobs->fair_n, J, c.k_max, c.n_max,
+      d_goodput, d_speedup, d_argmax);
+  SCHED_LAUNCH_CHECK(ctx);
+  return SCHED_OK;
+}
+
+int launch_realloc_factor(sched_ctx *ctx, const sched_jobs *jobs, float *d_out) {
+  const int J = ctx->cfg.num_jobs;
+  if (J == 0) return SCHED_OK;
+  realloc_factor_kernel<<<(J + 127) / 128, 128, 0, ctx->stream>>>(jobs->age_sec, jobs->num_restarts,
+                                                                   ctx->cfg.delta_sec, J, d_out);
+  SCHED_LAUNCH_CHECK(ctx);
+  return SCHED_OK;
+}

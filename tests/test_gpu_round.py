@@ -1,0 +1,155 @@
+"""The scheduling-round driver: equal to the step-by-step entry points, reproducible,
+feasible, consistent with the oracle's fitness, and the host-buffer variant."""
+import numpy as np
+import pytest
+
+from helpers import REL_TOL, assert_close, feasible, setup
+from paper_2008_12260_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    import torch
+    from paper_2008_12260_b200 import api
+    assert torch.cuda.is_available()
+    return torch, api
+
+
+def _round(gpu, cfg, jobs, cur, gens, rnd=0):
+    torch, api = gpu
+    s = api.scheduler_for(cfg, stream=torch.cuda.current_stream().cuda_stream)
+    dj = api.DeviceJobs(jobs, "cuda:0", torch)
+    best = torch.full((cfg.num_jobs, cfg.num_nodes), -1, dtype=torch.int16, device="cuda:0")
+    bf = torch.zeros(1, dtype=torch.float32, device="cuda:0")
+    d_cur = None if cur is None else torch.from_numpy(cur).cuda()
+    s.schedule_round(dj, d_cur, best, bf, round=rnd, generations=gens)
+    s.sync_status()
+    pop = torch.empty((cfg.population, cfg.num_jobs, cfg.num_nodes), dtype=torch.int16, device="cuda:0")
+    fit = torch.empty(cfg.population, dtype=torch.float32, device="cuda:0")
+    s.get_population(pop, fit)
+    torch.cuda.synchronize()
+    return s, dj, best.cpu().numpy(), float(bf.item()), pop.cpu().numpy(), fit.cpu().numpy()
+
+
+@pytest.mark.parametrize("cfg", [synth.TINY, synth.TESTBED], ids=lambda c: c.name)
+def test_round_equals_stepwise_calls_and_oracle_fitness(gpu, oracle, cfg):
+    torch, api = gpu
+    cl, jobs = setup(cfg)
+    cur = cfg.cur()
+    gens = min(cfg.generations, 25)
+    s, dj, best, bf, pop, fit = _round(gpu, cfg, jobs, cur, gens, rnd=2)
+
+    # the same round through the individual entry points
+    dev = "cuda:0"
+    sp = torch.empty(s.table_shape, dtype=torch.float32, device=dev)
+    s.build_speedup_table(dj, None, sp, None)
+    rf = torch.empty(cfg.num_jobs, dtype=torch.float32, device=dev)
+    s.compute_realloc_factor(dj, rf)
+    d_cur = torch.from_numpy(cur).cuda()
+    a = torch.empty((cfg.population, cfg.num_jobs, cfg.num_nodes), dtype=torch.int16, device=dev)
+    b = torch.empty_like(a)
+    f = torch.empty(cfg.population, dtype=torch.float32, device=dev)
+    s.init_population(dj, d_cur, a, round=2)
+    s.eval_fitness(a, sp, f, p=cfg.p, cur=d_cur, realloc_factor=rf, active=dj.tensors["active"])
+    f0 = f.cpu().numpy().copy()
+    for g in range(gens):
+        s.ga_generation(dj, a, f, b, round=2, generation=g)
+        a, b = b, a
+        s.eval_fitness(a, sp, f, p=cfg.p, cur=d_cur, realloc_factor=rf, active=dj.tensors["active"])
+    assert np.array_equal(a.cpu().numpy(), pop)
+    assert np.array_equal(f.cpu().numpy().view(np.uint32), fit.view(np.uint32))
+    i = int(np.argmax(fit))
+    assert np.array_equal(best, pop[i]) and bf == fit[i]
+    assert bf >= f0[0]                      # never worse than keeping the current allocation
+
+    # oracle: realloc factors, table, and the fitness of the final population
+    rf_ref = oracle.realloc_factor(jobs.age_sec, jobs.num_restarts, cfg.delta_sec)
+    assert_close(rf.cpu().numpy(), rf_ref, what="realloc factor")
+    _, sp_ref, _ = oracle.build_speedup_table(jobs, cl.node_capacity, cl.k_max, cl.n_max, cfg.grid_s)
+    assert_close(sp.cpu().numpy(), sp_ref, what="speedup")
+    fit_ref = oracle.eval_fitness(pop, sp_ref, cl.k_max, cl.n_max, cfg.p, cfg.speedup_floor, cur=cur,
+                                  realloc=rf_ref, active=jobs.active)
+    assert_close(fit, fit_ref, rel=3 * REL_TOL, what="fitness of the final population")
+    for c in range(cfg.population):
+        assert feasible(pop[c], cl.node_capacity, jobs.k_cap, cl.n_max)
+    s.close()
+
+
+def test_round_is_reproducible_and_round_number_matters(gpu):
+    cfg = synth.TESTBED
+    cl, jobs = setup(cfg)
+    cur = cfg.cur()
+    r1 = _round(gpu, cfg, jobs, cur, 10, rnd=5)
+    r2 = _round(gpu, cfg, jobs, cur, 10, rnd=5)
+    r3 = _round(gpu, cfg, jobs, cur, 10, rnd=6)
+    assert np.array_equal(r1[4], r2[4]) and np.array_equal(r1[2], r2[2]) and r1[3] == r2[3]
+    assert not np.array_equal(r1[4], r3[4])
+    for r in (r1, r2, r3):
+        r[0].close()
+
+
+def test_round_search_quality_against_oracle_round(gpu, oracle):
+    """The two rounds may fork at fp32/fp64 near-ties, so only the outcome is compared: the
+    CUDA round must reach a fitness close to the oracle's own round on the same inputs."""
+    cfg = synth.TINY
+    cl, jobs = setup(cfg)
+    s, dj, best, bf, pop, fit = _round(gpu, cfg, jobs, None, 40)
+    ob, of = oracle.schedule_round(jobs, cl.node_capacity, cl.k_max, cl.n_max, cfg.grid_s, cfg.population,
+                                   cfg.p, cfg.delta_sec, cfg.speedup_floor, cfg.num_elite,
+                                   synth.prob_to_threshold(cfg.mutate_prob),
+                                   synth.prob_to_threshold(cfg.init_prob), cfg.seed, 0, 40, None)
+    assert bf > 0.5 * of and of > 0.5 * bf
+    s.close()
+
+
+def test_zero_generations_and_no_current_allocation(gpu, oracle):
+    cfg = synth.TINY
+    cl, jobs = setup(cfg)
+    s, dj, best, bf, pop, fit = _round(gpu, cfg, jobs, None, 0)
+    ref = oracle.init_population(cfg.population, None, cfg.num_jobs, cl.node_capacity, jobs.k_cap, cl.k_max,
+                                 cl.n_max, synth.prob_to_threshold(cfg.init_prob), cfg.seed, 0,
+                                 active=jobs.active)
+    assert np.array_equal(pop, ref)
+    assert np.array_equal(best, pop[int(np.argmax(fit))])
+    s.close()
+
+
+def test_host_buffer_round(gpu):
+    torch, api = gpu
+    cfg = synth.TESTBED
+    cl, jobs = setup(cfg)
+    cur = cfg.cur()
+    s, dj, best, bf, pop, fit = _round(gpu, cfg, jobs, cur, 8, rnd=1)
+    hj = api.HostJobs(jobs, torch)
+    h_cur = torch.from_numpy(cur).pin_memory()
+    h_best = torch.empty((cfg.num_jobs, cfg.num_nodes), dtype=torch.int16).pin_memory()
+    h_bf = torch.zeros(1, dtype=torch.float32).pin_memory()
+    s.schedule_round_host(hj, h_cur, h_best, h_bf, round=1, generations=8)
+    assert np.array_equal(h_best.numpy(), best) and float(h_bf.item()) == bf
+    s.close()
+
+
+def test_argument_errors(gpu):
+    torch, api = gpu
+    cfg = synth.TINY
+    cl, jobs = setup(cfg)
+    s = api.scheduler_for(cfg)
+    dj = api.DeviceJobs(jobs, "cuda:0", torch)
+    best = torch.empty((cfg.num_jobs, cfg.num_nodes), dtype=torch.int16, device="cuda:0")
+    bf = torch.zeros(1, dtype=torch.float32, device="cuda:0")
+    with pytest.raises(api.SchedError) as e:
+        s.schedule_round(dj, None, None, bf, round=0, generations=1)
+    assert e.value.code == -1
+    with pytest.raises(api.SchedError):
+        s.schedule_round(dj, None, best, bf, round=0, generations=-1)
+    with pytest.raises(api.SchedError):
+        s.ga_generation(None, best, bf, best, round=0, generation=0)          # in == out
+    with pytest.raises(api.SchedError):
+        s.eval_fitness(best, None, bf, p=-1.0, count=1)
+    with pytest.raises(api.SchedError):
+        s.get_population(best, bf)                                            # no round yet
+    s.schedule_round(dj, None, best, bf, round=0, generations=1)              # still usable afterwards
+    s.sync_status()
+    s.close()
