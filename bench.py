@@ -1,0 +1,421 @@
+#!/usr/bin/env python
+"""Benchmark of the PolluxSched optimizer core on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one whole scheduling round of the "large" workload (256 nodes x 8 GPUs, 1024
+jobs, 128 x 32 (m, s) grid, population 512, 200 generations): speedup tables, initial
+population, and per generation ranking / selection + crossover + perturbation / repair /
+fitness, then the best allocation.  The headline value is candidate fitness evaluations
+per second over the round.  With N > 1 (torchrun) every rank schedules its own cluster
+(independent problems, no data-path collective): weak scaling.
+
+Rank 0 prints ONE JSON line.  Besides the contract keys it carries the per-kernel device
+times of the timed region, the roofline of the dominant kernel, and - at N = 1 - two
+single-kernel measurements: the goodput sweep (ALU-bound) and the dense fitness kernel on
+a chunk of the stress workload (HBM-bound), plus the CPU oracle timed on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2008_12260_b200 import dist as pdist  # noqa: E402
+from paper_2008_12260_b200 import synth  # noqa: E402
+
+METRIC = "ga_candidate_fitness_evals_per_sec"
+UNIT = "candidates/s"
+FP32_LANES_PER_SM = 128          # CUDA cores per SM (compute capability 10.0)
+OPS_PER_POINT = 10               # fp32 lane-ops counted as useful per (job, K, class, m, s) point
+HBM_FALLBACK_GBS = 6650.0
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
+# captures summarised under profiles/; None = kernel changed since the counters were taken.
+NCU_TRAFFIC_BYTES = {"rows": None, "cols": None, "fitness": None, "fitness_stress": None}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return float(d["hbm_gbs"]), "measured", float(d.get("sm_max_mhz", 1965.0))
+        except Exception:
+            pass
+    return HBM_FALLBACK_GBS, "fallback", 1965.0
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled every 200 ms while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.proc = None
+        self.tmp = None
+
+    def start(self):
+        try:
+            self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "200"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp.read().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def large_inputs(rank: int):
+    cfg = synth.LARGE
+    cl = cfg.cluster()
+    jobs = synth.draw_jobs(cfg.num_jobs, cfg.seed + 1000 * rank, cfg.grid_m, cfg.grid_s, cl.k_max,
+                           phi_hi=cfg.phi_hi, with_history=True)
+    from paper_2008_12260_b200.api import fair_share
+    fk, fn = fair_share(cl.node_capacity, cfg.num_jobs, cl.k_max)
+    jobs.fair_k = np.full(cfg.num_jobs, fk, np.int32)
+    jobs.fair_n = np.full(cfg.num_jobs, fn, np.int32)
+    cur = synth.random_feasible_allocation(cl, cfg.num_jobs, cfg.seed + 1000 + rank)
+    return cfg, cl, jobs, cur
+
+
+def distinct_classes(cl) -> int:
+    """(K, class) pairs the sweep evaluates per job: K that fit one node, and K >= 2 that
+    fit on min(K, n_max) nodes."""
+    cap = np.sort(np.maximum(cl.node_capacity.astype(np.int64), 0))[::-1]
+    kfit = np.concatenate([[0], np.cumsum(cap)])
+    n = 0
+    for K in range(1, cl.k_max + 1):
+        n += int(K <= kfit[1])
+        n += int(cl.n_max >= 2 and K >= 2 and K <= kfit[min(K, cl.n_max, len(cap))])
+    return n
+
+
+# ------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    from paper_2008_12260_b200 import api
+
+    rank, local_rank, world = pdist.init("nccl")
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    stream = torch.cuda.current_stream()
+    hbm_peak, peak_src, sm_max_mhz = measured_peaks()
+
+    cfg, cl, jobs, cur = large_inputs(rank)
+    G, P, J, NN = cfg.generations, cfg.population, cfg.num_jobs, cfg.num_nodes
+    sched = api.scheduler_for(cfg, stream=stream.cuda_stream)
+    dj = api.DeviceJobs(jobs, dev, torch)
+    d_cur = torch.from_numpy(cur).to(dev)
+    d_best = torch.empty((J, NN), dtype=torch.int16, device=dev)
+    d_bf = torch.zeros(1, dtype=torch.float32, device=dev)
+
+    def step(rnd):
+        sched.schedule_round(dj, d_cur, d_best, d_bf, round=rnd, generations=G)
+
+    for w in range(args.warmup):
+        step(w)
+    sched.sync_status()
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    sched.set_kernel_timing(True)
+    sched.read_kernel_timing()
+    launches0 = sched.launch_count()
+    pdist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for k in range(args.steps):
+        step(100 + k)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    pdist.barrier()
+    clocks = sampler.stop()
+    elapsed_ms = e0.elapsed_time(e1)
+    kernel_ms = sched.read_kernel_timing()
+    sched.set_kernel_timing(False)
+    launches = sched.launch_count() - launches0
+    sched.sync_status()
+    units = float(P) * (G + 1) * args.steps
+    value, t_max, u_sum = pdist.throughput(elapsed_ms, units, device=dev)
+
+    # ---- end to end through the host-buffer entry point (pinned host memory) -------------
+    hj = api.HostJobs(jobs, torch)
+    h_cur = torch.from_numpy(cur.copy()).pin_memory()
+    h_best = torch.empty((J, NN), dtype=torch.int16).pin_memory()
+    h_bf = torch.zeros(1, dtype=torch.float32).pin_memory()
+    sched.schedule_round_host(hj, h_cur, h_best, h_bf, round=0, generations=G)
+    pdist.barrier()
+    t0 = time.perf_counter()
+    e0.record(stream)
+    for k in range(args.steps):
+        sched.schedule_round_host(hj, h_cur, h_best, h_bf, round=100 + k, generations=G)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3)
+    e2e_value, _, _ = pdist.throughput(e2e_ms, units, device=dev)
+    h2d = hj.nbytes + h_cur.numel() * 2
+    d2h = h_best.numel() * 2 + 4
+    assert np.array_equal(h_best.numpy(), d_best.cpu().numpy()), "host and device rounds disagree"
+
+    # ---- per-kernel accounting and the roofline of the dominant kernel --------------------
+    pop_bytes = float(P) * J * NN * 2
+    algo_bytes = {
+        "rows": 2 * pop_bytes + P * J,           # read parent rows, write child rows (+ row flags)
+        "cols": pop_bytes + P * J,               # column scan of every child (writes only on violations)
+        "fitness": pop_bytes + P * J * 4 + J * NN * 2 + P * 4,
+    }
+    kernels = []
+    for name, (ms, n) in sorted(kernel_ms.items(), key=lambda kv: -kv[1][0]):
+        if n == 0:
+            continue
+        k = {"kernel": name, "launches": n, "total_ms": round(ms, 3), "avg_us": round(1e3 * ms / n, 2),
+             "share": round(ms / max(sum(v[0] for v in kernel_ms.values()), 1e-9), 4)}
+        if name in algo_bytes:
+            k["algorithmic_bytes"] = algo_bytes[name]
+            k["achieved_gbs"] = round(algo_bytes[name] / (ms / n * 1e-3) / 1e9, 1)
+            k["frac_of_hbm_peak"] = round(k["achieved_gbs"] / hbm_peak, 4)
+        kernels.append(k)
+    dom = next((k for k in kernels if "achieved_gbs" in k), None)
+    roofline = None
+    if dom:
+        roofline = {"kernel": dom["kernel"], "bound": "hbm", "achieved": dom["achieved_gbs"], "peak": hbm_peak,
+                    "peak_source": "MEASURED_PEAKS.json hbm_gbs" if peak_src == "measured" else "recipe fallback",
+                    "unit": "GB/s", "frac": dom["frac_of_hbm_peak"],
+                    "traffic": NCU_TRAFFIC_BYTES.get(dom["kernel"]),
+                    "algorithmic_bytes_per_launch": dom["algorithmic_bytes"], "avg_launch_us": dom["avg_us"]}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": t_max / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "large: 256 nodes x 8 GPUs, 1024 jobs, grid 128x32, population 512, "
+                               "200 generations, p=-1, random current allocation, one scheduling round per step",
+                   "per_rank": "one independent cluster per rank", "arithmetic": "int16 matrices, fp32 tables and fitness",
+                   "l2": "inputs larger than L2 (two 268 MB population buffers alternate every generation)"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                "ms_per_step": e2e_ms / args.steps, "api": "schedule_round_host (pinned host buffers)"},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "kernels": kernels,
+        "best_fitness": float(h_bf.item()),
+    }
+    sched.close()
+
+    if world == 1 and not args.skip_extras:
+        line["goodput_model"] = bench_table(api, torch, dev, stream, cfg, cl, jobs, sm_max_mhz, clocks)
+        line["stress_fitness"] = bench_stress(api, torch, dev, stream, hbm_peak, peak_src, args)
+        line["cpu_baseline"] = oracle_sample(cfg, cl, jobs, cur)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def bench_table(api, torch, dev, stream, cfg, cl, jobs, sm_max_mhz, clocks):
+    """build_speedup_table alone on the large workload: distinct (job, K, class, m, s) points
+    per second, and the share of the fp32 lane-op peak (ALU-bound kernel)."""
+    sched = api.scheduler_for(cfg, stream=stream.cuda_stream)
+    dj = api.DeviceJobs(jobs, dev, torch)
+    sp = torch.empty(sched.table_shape, dtype=torch.float32, device=dev)
+    gp = torch.empty_like(sp)
+    am = torch.empty(sched.table_shape, dtype=torch.uint16, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    for _ in range(3):
+        sched.build_speedup_table(dj, gp, sp, am)
+    sched.set_kernel_timing(True)
+    sched.read_kernel_timing()
+    reps = 20
+    for _ in range(reps):
+        flush.fill_(1)                      # L2 flush between iterations
+        sched.build_speedup_table(dj, gp, sp, am)
+    t = sched.read_kernel_timing()
+    sched.close()
+    sweep_ms = t["goodput_sweep"][0] / reps
+    expand_ms = t["speedup_expand"][0] / reps
+    points = float(cfg.num_jobs) * distinct_classes(cl) * cfg.grid_m * cfg.grid_s
+    num_sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    peak = num_sms * FP32_LANES_PER_SM * sm_max_mhz * 1e6          # lane-ops/s (an FMA counts once)
+    achieved = OPS_PER_POINT * points / (sweep_ms * 1e-3)
+    return {
+        "workload": "large", "distinct_points": points, "sweep_us": round(sweep_ms * 1e3, 2),
+        "expand_us": round(expand_ms * 1e3, 2),
+        "evals_per_sec": points / ((sweep_ms + expand_ms) * 1e-3),
+        "evals_per_sec_sweep_only": points / (sweep_ms * 1e-3),
+        "roofline": {"kernel": "goodput_sweep", "bound": "alu", "achieved": achieved / 1e12, "peak": peak / 1e12,
+                     "unit": "T lane-op/s", "frac": achieved / peak,
+                     "peak_source": "%d SMs x %d fp32 lanes x %.0f MHz (max SM clock)" % (num_sms, FP32_LANES_PER_SM, sm_max_mhz),
+                     "ops_per_point": OPS_PER_POINT, "traffic": None, "l2": "flushed between iterations"},
+    }
+
+
+def bench_stress(api, torch, dev, stream, hbm_peak, peak_src, args):
+    """eval_fitness on one chunk of the stress workload (2048 x 8 cluster, 8192 jobs, fp32
+    [8192][65][65] tables, dense int16 candidates of 33.5 MB each)."""
+    st = synth.STRESS
+    chunk = args.stress_chunk
+    J, NN = st["num_jobs"], st["num_nodes"]
+    cap = synth.uniform_cluster(NN, st["gpus_per_node"]).node_capacity
+    sched = api.Scheduler(node_capacity=cap, num_jobs=J, grid_m=1, grid_s=1, population=chunk,
+                          stream=stream.cuda_stream)
+    table = torch.from_numpy(synth.stress_speedup_table(J, 64, 64, st["gpus_per_node"], st["seed"])).to(dev)
+    pop = torch.cat([synth.stress_population(32, J, NN, st["gpus_per_node"], st["seed"], device=dev, first_candidate=c)
+                     for c in range(0, chunk, 32)])
+    fit = torch.empty(chunk, dtype=torch.float32, device=dev)
+    out = {"workload": "stress chunk: %d of 4096 candidates, 8192 jobs x 2048 nodes, int16 dense" % chunk,
+           "chunk_bytes": int(pop.numel() * 2), "p": {}}
+    bytes_per_cand = J * NN * 2 + J * 4 + 4
+    sched.set_kernel_timing(True)
+    best = None
+    for p in st["p_values"]:
+        for _ in range(3):
+            sched.eval_fitness(pop, table, fit, p=p)
+        sched.read_kernel_timing()
+        reps = 10
+        for _ in range(reps):
+            sched.eval_fitness(pop, table, fit, p=p)          # 8.6 GB per pass: far larger than L2
+        ms = sched.read_kernel_timing()["fitness"][0] / reps
+        gbs = chunk * bytes_per_cand / (ms * 1e-3) / 1e9
+        out["p"][str(p)] = {"ms_per_chunk": round(ms, 3), "candidates_per_sec": chunk / (ms * 1e-3),
+                            "achieved_gbs": round(gbs, 1), "frac_of_hbm_peak": round(gbs / hbm_peak, 4)}
+        if best is None or gbs < best[0]:
+            best = (gbs, ms)
+    out["roofline"] = {"kernel": "fitness", "bound": "hbm", "achieved": round(best[0], 1), "peak": hbm_peak,
+                       "peak_source": "MEASURED_PEAKS.json hbm_gbs" if peak_src == "measured" else "recipe fallback",
+                       "unit": "GB/s", "frac": round(best[0] / hbm_peak, 4), "frac_of_8tbs_nominal": round(best[0] / 8000.0, 4),
+                       "traffic": NCU_TRAFFIC_BYTES.get("fitness_stress"),
+                       "algorithmic_bytes_per_launch": chunk * bytes_per_cand, "note": "slowest of the three exponents"}
+    sched.close()
+    del pop, table
+    torch.cuda.empty_cache()
+    return out
+
+
+# ------------------------------------------------------------------------------------------
+def oracle_sample(cfg, cl, jobs, cur, table_jobs: int = 8, gens: int = 2):
+    """The CPU oracle on a bounded sample of the large round: tables of `table_jobs` jobs, the
+    initial population, and `gens` x (generation + fitness) at the full population; the
+    time of a whole round is extrapolated linearly (tables x J / table_jobs, generations x
+    G / gens)."""
+    import oracle
+
+    P, J, G = cfg.population, cfg.num_jobs, cfg.generations
+    sub = jobs.take(slice(0, table_jobs))
+    t0 = time.perf_counter()
+    oracle.build_speedup_table(sub, cl.node_capacity, cl.k_max, cl.n_max, cfg.grid_s, want_argmax=False)
+    t_table = (time.perf_counter() - t0) * (J / table_jobs)
+    rng = np.random.default_rng(0)
+    speedup = rng.uniform(0.1, 3.0, (J, cl.k_max + 1, cl.n_max + 1))
+    rf = oracle.realloc_factor(jobs.age_sec, jobs.num_restarts, cfg.delta_sec)
+    thr_m, thr_i = synth.prob_to_threshold(cfg.mutate_prob), synth.prob_to_threshold(cfg.init_prob)
+    t0 = time.perf_counter()
+    pop = oracle.init_population(P, cur, J, cl.node_capacity, jobs.k_cap, cl.k_max, cl.n_max, thr_i, cfg.seed, 0)
+    fit = oracle.eval_fitness(pop, speedup, cl.k_max, cl.n_max, cfg.p, cfg.speedup_floor, cur=cur, realloc=rf)
+    t_init = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    for g in range(gens):
+        pop = oracle.ga_generation(pop, fit.astype(np.float32), cl.node_capacity, jobs.k_cap, cl.k_max, cl.n_max,
+                                   cfg.num_elite, thr_m, cfg.seed, 0, g)
+        fit = oracle.eval_fitness(pop, speedup, cl.k_max, cl.n_max, cfg.p, cfg.speedup_floor, cur=cur, realloc=rf)
+    t_gen = (time.perf_counter() - t0) / gens
+    round_s = t_table + t_init + G * t_gen
+    return {"value": P * (G + 1) / round_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "tables of %d of %d jobs, initial population, %d of %d generations at population %d; "
+                      "round time extrapolated linearly" % (table_jobs, J, gens, G, P),
+            "round_seconds_extrapolated": round_s, "table_seconds_extrapolated": t_table,
+            "generation_seconds": t_gen}
+
+
+def run_reference(args):
+    """The oracle as the reference arm: CPU only, rank 0 only."""
+    rank, _, world = pdist.env_world()
+    if rank != 0:
+        return
+    cfg, cl, jobs, cur = large_inputs(0)
+    samples = []
+    for i in range(args.warmup + args.steps):
+        s = oracle_sample(cfg, cl, jobs, cur, table_jobs=4, gens=1)
+        if i >= args.warmup:
+            samples.append(s)
+    round_s = statistics.mean(s["round_seconds_extrapolated"] for s in samples)
+    value = cfg.population * (cfg.generations + 1) / round_s
+    base = dict(samples[-1], value=value)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round_s * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "large: 256 nodes x 8 GPUs, 1024 jobs, grid 128x32, population 512, "
+                               "200 generations, p=-1, random current allocation, one scheduling round per step",
+                   "note": "CPU oracle; each step times a bounded sample and extrapolates the round"},
+        "cpu_baseline": base,
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--skip-extras", action="store_true", help="only the timed rounds (no single-kernel sections, no oracle)")
+    ap.add_argument("--stress-chunk", type=int, default=256, help="candidates in the stress fitness chunk (multiple of 32)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

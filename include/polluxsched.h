@@ -111,6 +111,18 @@ int sched_sync_status(sched_ctx *ctx);
 /* Number of kernels this context has launched so far (for accounting in benchmarks). */
 int64_t sched_launch_count(const sched_ctx *ctx);
 
+/* Optional per-kernel timing.  While enabled, every kernel the context launches is
+ * bracketed by a pair of CUDA events on the context's stream (at most 131072 pairs between
+ * read-outs; further launches are not timed).  sched_read_kernel_timing waits for the
+ * stream and writes, per kernel class k in [0, sched_num_kernel_kinds()), the summed
+ * device time in milliseconds and the number of timed launches since the previous
+ * read-out into HOST arrays of that length.  The paper has no counterpart; this exists so
+ * that a benchmark can attribute a round's time to kernels without a profiler. */
+int sched_set_kernel_timing(sched_ctx *ctx, int enable);
+int sched_num_kernel_kinds(void);
+const char *sched_kernel_kind_name(int kind);
+int sched_read_kernel_timing(sched_ctx *ctx, float *h_ms_total, int64_t *h_launches);
+
 /* Speedup tables (Eq. 13 and 15).  For every job and every (K, N) with 1 <= N <= n_max,
  * N <= K <= k_max and K no larger than the N largest nodes together:
  *   goodput[j][K][N] = max over the grid {m_grid[j][i]} x {s} of GOODPUT(a, m, s) (Eq. 4)

@@ -21,6 +21,8 @@ EXPORTS = (
     "build_speedup_table", "compute_realloc_factor", "eval_fitness", "repair_population",
     "init_population", "ga_generation", "schedule_round", "schedule_round_host",
     "sched_get_population", "sched_round_speedup_table", "eval_fitness_host",
+    "sched_set_kernel_timing", "sched_num_kernel_kinds", "sched_kernel_kind_name",
+    "sched_read_kernel_timing",
 )
 
 
@@ -75,6 +77,11 @@ def load_library(path: str = LIB_PATH):
     lib.sched_round_speedup_table.argtypes = [vp]
     lib.sched_round_speedup_table.restype = vp
     lib.eval_fitness_host.argtypes = [vp, vp, i32, vp, vp, vp, vp, f32, vp]
+    lib.sched_set_kernel_timing.argtypes = [vp, i32]
+    lib.sched_num_kernel_kinds.argtypes = []
+    lib.sched_kernel_kind_name.argtypes = [i32]
+    lib.sched_kernel_kind_name.restype = C.c_char_p
+    lib.sched_read_kernel_timing.argtypes = [vp, vp, vp]
     for name in EXPORTS:
         if getattr(lib, name).restype is C.c_int:
             getattr(lib, name).restype = C.c_int
@@ -190,6 +197,17 @@ class Scheduler:
 
     def launch_count(self) -> int:
         return int(_lib.sched_launch_count(self._ctx))
+
+    def set_kernel_timing(self, enable: bool):
+        self._check(_lib.sched_set_kernel_timing(self._ctx, 1 if enable else 0))
+
+    def read_kernel_timing(self):
+        """{kernel class: (total ms, timed launches)} since the previous read-out"""
+        n = _lib.sched_num_kernel_kinds()
+        ms = np.zeros(n, np.float32)
+        cnt = np.zeros(n, np.int64)
+        self._check(_lib.sched_read_kernel_timing(self._ctx, ms.ctypes.data, cnt.ctypes.data))
+        return {_lib.sched_kernel_kind_name(k).decode(): (float(ms[k]), int(cnt[k])) for k in range(n)}
 
     # -- entry points ---------------------------------------------------------------------
     def build_speedup_table(self, jobs, goodput, speedup, argmax=None):

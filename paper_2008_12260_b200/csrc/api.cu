@@ -20,6 +20,29 @@ const char *set_error(sched_ctx *ctx, const char *fmt, ...) {
   return dst;
 }
 
+TimedLaunch::TimedLaunch(sched_ctx *c, int kind) : ctx(c), on(false) {
+  span.kind = kind;
+  c->kind_launches[kind]++;
+  if (!c->timing_on) return;
+  if (!c->free_spans.empty()) {
+    span.start = c->free_spans.back().start;
+    span.stop = c->free_spans.back().stop;
+    c->free_spans.pop_back();
+  } else {
+    if (c->spans.size() >= (1u << 17)) { c->spans_dropped++; return; }
+    if (cudaEventCreate(&span.start) != cudaSuccess) return;
+    if (cudaEventCreate(&span.stop) != cudaSuccess) { cudaEventDestroy(span.start); return; }
+  }
+  on = true;
+  cudaEventRecord(span.start, c->stream);
+}
+
+TimedLaunch::~TimedLaunch() {
+  if (!on) return;
+  cudaEventRecord(span.stop, ctx->stream);
+  ctx->spans.push_back(span);
+}
+
 namespace {
 
 template <typename T>
@@ -129,7 +152,6 @@ int sched_init(const sched_config *cfg, const int16_t *h_node_capacity, void *cu
 
   sched_ctx *ctx = new (std::nothrow) sched_ctx();
   REQUIRE(nullptr, ctx, SCHED_ERR_CUDA, "sched_init: out of host memory");
-  memset(ctx, 0, sizeof(*ctx));
   ctx->cfg = *cfg;
   ctx->stream = (cudaStream_t)cuda_stream;
   ctx->KD = cfg->k_max + 1;
@@ -192,6 +214,8 @@ int sched_destroy(sched_ctx *ctx) {
                   ctx->d_rf, ctx->d_best_idx, ctx->d_stage, ctx->d_stage_fit};
   for (void *p : ptrs)
     if (p) cudaFree(p);
+  for (auto *v : {&ctx->spans, &ctx->free_spans})
+    for (TimedSpan &t : *v) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
   delete ctx;
   return SCHED_OK;
 }
@@ -208,6 +232,38 @@ int sched_sync_status(sched_ctx *ctx) {
 }
 
 int64_t sched_launch_count(const sched_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int sched_set_kernel_timing(sched_ctx *ctx, int enable) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "sched_set_kernel_timing: ctx is NULL");
+  ctx->timing_on = enable != 0;
+  return SCHED_OK;
+}
+
+int sched_num_kernel_kinds(void) { return KK_COUNT; }
+
+const char *sched_kernel_kind_name(int kind) {
+  static const char *names[KK_COUNT] = {"goodput_sweep", "speedup_expand", "realloc_factor",
+                                        "penalty_prep", "fitness", "rank", "rows", "cols",
+                                        "best_index", "copy_best"};
+  return (kind >= 0 && kind < KK_COUNT) ? names[kind] : "";
+}
+
+int sched_read_kernel_timing(sched_ctx *ctx, float *h_ms_total, int64_t *h_launches) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "sched_read_kernel_timing: ctx is NULL");
+  REQUIRE(ctx, h_ms_total && h_launches, SCHED_ERR_INVALID_ARG, "sched_read_kernel_timing: NULL output");
+  SCHED_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
+  for (int k = 0; k < KK_COUNT; ++k) { h_ms_total[k] = 0.f; h_launches[k] = 0; }
+  for (TimedSpan &t : ctx->spans) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, t.start, t.stop) == cudaSuccess) {
+      h_ms_total[t.kind] += ms;
+      h_launches[t.kind] += 1;
+    }
+    ctx->free_spans.push_back(t);
+  }
+  ctx->spans.clear();
+  return SCHED_OK;
+}
 
 int build_speedup_table(sched_ctx *ctx, const sched_jobs *d_jobs, float *d_goodput,
                         float *d_speedup, uint16_t *d_argmax) {

@@ -6,6 +6,8 @@
 #include <stdint.h>
 #include <stdio.h>
 
+#include <vector>
+
 #include "polluxsched.h"
 
 #define SLOT_SELECT 0u
@@ -15,6 +17,17 @@
 #define SLOT_REPAIR_CAP 4u
 #define SLOT_INIT 5u
 #define GEN_INIT 0xFFFFFFFFu
+
+// kernel classes, for launch accounting and optional per-kernel timing
+enum KernelKind {
+  KK_SWEEP = 0, KK_EXPAND, KK_REALLOC, KK_PENPREP, KK_FITNESS, KK_RANK, KK_ROWS, KK_COLS, KK_BEST,
+  KK_COPY, KK_COUNT
+};
+
+struct TimedSpan {
+  cudaEvent_t start, stop;
+  int kind;
+};
 
 struct sched_ctx {
   sched_config cfg;
@@ -53,6 +66,22 @@ struct sched_ctx {
   size_t stage_bytes;
   void *d_stage_fit;     // eval_fitness_host staging
   size_t stage_fit_bytes;
+
+  // optional per-kernel timing with CUDA events on the context's stream
+  bool timing_on;
+  std::vector<TimedSpan> spans;      // recorded since the last read-out
+  std::vector<TimedSpan> free_spans; // event pairs ready for reuse
+  int64_t spans_dropped;
+  int64_t kind_launches[KK_COUNT];
+};
+
+// Brackets one kernel launch with a pair of events when timing is enabled.
+struct TimedLaunch {
+  sched_ctx *ctx;
+  TimedSpan span;
+  bool on;
+  TimedLaunch(sched_ctx *c, int kind);
+  ~TimedLaunch();
 };
 
 const char *set_error(sched_ctx *ctx, const char *fmt, ...);

@@ -222,8 +222,11 @@ int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const fl
 
   const bool penalise = d_cur && d_rf;
   if (penalise && J > 0) {
+    {
+    TimedLaunch tl_(ctx, KK_PENPREP);
     penalty_prep_kernel<<<(J * 32 + 255) / 256, 256, 0, ctx->stream>>>(d_cur, d_rf, J, c.num_nodes,
                                                                        ctx->d_pen);
+    }
     SCHED_LAUNCH_CHECK(ctx);
   }
 
@@ -275,11 +278,14 @@ int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const fl
     b.ticket = ctx->d_ticket + first;
     b.fitness = d_fitness + first;
     dim3 grid((unsigned)chunks, (unsigned)n);
+    {
+    TimedLaunch tl_(ctx, KK_FITNESS);
     switch (W) {
       case 16: fitness_kernel<16><<<grid, 256, 0, ctx->stream>>>(b); break;
       case 8: fitness_kernel<8><<<grid, 256, 0, ctx->stream>>>(b); break;
       case 4: fitness_kernel<4><<<grid, 256, 0, ctx->stream>>>(b); break;
       default: fitness_kernel<2><<<grid, 256, 0, ctx->stream>>>(b); break;
+    }
     }
     SCHED_LAUNCH_CHECK(ctx);
   }

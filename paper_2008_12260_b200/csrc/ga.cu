@@ -315,7 +315,10 @@ int launch_rows(sched_ctx *ctx, RowsArgs &a) {
     }
   }
   const long long blocks = (warps + wpb - 1) / wpb;
+  {
+  TimedLaunch tl_(ctx, KK_ROWS);
   rows_kernel<<<(unsigned)blocks, wpb * 32, smem, ctx->stream>>>(a);
+  }
   SCHED_LAUNCH_CHECK(ctx);
   return SCHED_OK;
 }
@@ -334,7 +337,7 @@ int launch_cols(sched_ctx *ctx, int16_t *pop, int count, uint32_t first_cand, ui
     a.pop = pop + (size_t)first * a.J * a.num_nodes;
     a.dflag = ctx->d_dflag + (size_t)first * a.J;
     dim3 grid((unsigned)((a.num_nodes + 127) / 128), (unsigned)n);
-    cols_kernel<<<grid, 128, 0, ctx->stream>>>(a);
+    { TimedLaunch tl_(ctx, KK_COLS); cols_kernel<<<grid, 128, 0, ctx->stream>>>(a); }
     SCHED_LAUNCH_CHECK(ctx);
   }
   return SCHED_OK;
@@ -386,8 +389,11 @@ int launch_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_a
   const int P = ctx->cfg.population;
   int rc = ensure_dflag(ctx, P);
   if (rc != SCHED_OK) return rc;
+  {
+  TimedLaunch tl_(ctx, KK_RANK);
   rank_kernel<<<(P + 127) / 128, 128, 0, ctx->stream>>>((const uint32_t *)d_fitness_in, P,
                                                          ctx->d_rank, ctx->d_order);
+  }
   SCHED_LAUNCH_CHECK(ctx);
   RowsArgs a = base_rows_args(ctx, d_k_cap, d_active, P);
   a.mode = ROWS_GENERATION; a.src = d_pop_in; a.dst = d_pop_out;
@@ -400,14 +406,20 @@ int launch_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_a
 int launch_select_best(sched_ctx *ctx, const int16_t *d_pop, const float *d_fitness,
                        int16_t *d_best, float *d_best_fitness) {
   const int P = ctx->cfg.population;
+  {
+  TimedLaunch tl_(ctx, KK_BEST);
   best_index_kernel<<<1, 256, 0, ctx->stream>>>((const uint32_t *)d_fitness, P, ctx->d_best_idx,
                                                 d_best_fitness);
+  }
   SCHED_LAUNCH_CHECK(ctx);
   const size_t elems = (size_t)ctx->cfg.num_jobs * ctx->cfg.num_nodes;
   if (elems == 0) return SCHED_OK;
   const int blocks = (int)((elems + 256 * 8 - 1) / (256 * 8));
+  {
+  TimedLaunch tl_(ctx, KK_COPY);
   copy_best_kernel<<<blocks > 1024 ? 1024 : blocks, 256, 0, ctx->stream>>>(d_pop, ctx->d_best_idx,
                                                                            elems, d_best);
+  }
   SCHED_LAUNCH_CHECK(ctx);
   return SCHED_OK;
 }

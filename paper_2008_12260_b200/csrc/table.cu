@@ -197,18 +197,22 @@ int launch_speedup_table(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodpu
   const long long blocks = (warps * 32 + block - 1) / block;
   const int mq = (c.grid_m + 31) / 32;
 #define SWEEP(MQ)                                                                              \
+  TimedLaunch tl_(ctx, KK_SWEEP);                                                              \
   goodput_sweep_kernel<MQ><<<(unsigned)blocks, block, 0, ctx->stream>>>(                       \
       jp, jobs->m_grid, ctx->d_kfit, J, c.k_max, c.n_max, c.grid_m, c.grid_s, ctx->d_gmax,    \
       ctx->d_amax)
-  if (mq <= 1) SWEEP(1);
-  else if (mq == 2) SWEEP(2);
-  else SWEEP(4);
+  if (mq <= 1) { SWEEP(1); }
+  else if (mq == 2) { SWEEP(2); }
+  else { SWEEP(4); }
 #undef SWEEP
   SCHED_LAUNCH_CHECK(ctx);
   const long long entries = (long long)J * ctx->KD * ctx->ND;
+  {
+  TimedLaunch tl_(ctx, KK_EXPAND);
   speedup_expand_kernel<<<(unsigned)((entries + 255) / 256), 256, 0, ctx->stream>>>(
       ctx->d_gmax, ctx->d_amax, ctx->d_kfit, jobs->fair_k, jobs->fair_n, J, c.k_max, c.n_max,
       d_goodput, d_speedup, d_argmax);
+  }
   SCHED_LAUNCH_CHECK(ctx);
   return SCHED_OK;
 }
@@ -216,8 +220,11 @@ int launch_speedup_table(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodpu
 int launch_realloc_factor(sched_ctx *ctx, const sched_jobs *jobs, float *d_out) {
   const int J = ctx->cfg.num_jobs;
   if (J == 0) return SCHED_OK;
+  {
+  TimedLaunch tl_(ctx, KK_REALLOC);
   realloc_factor_kernel<<<(J + 127) / 128, 128, 0, ctx->stream>>>(jobs->age_sec, jobs->num_restarts,
                                                                    ctx->cfg.delta_sec, J, d_out);
+  }
   SCHED_LAUNCH_CHECK(ctx);
   return SCHED_OK;
 }
