@@ -206,6 +206,46 @@ int eval_fitness_host(sched_ctx *ctx, const int16_t *h_pop, int32_t count, const
                       const int16_t *h_cur, const float *h_realloc_factor,
                       const uint8_t *h_active, float p, float *h_fitness);
 
+/* Limits of eval_fitness_noalloc (its scratch array is sized for exactly these). */
+#define SCHED_NOALLOC_MAX_COUNT 2048
+#define SCHED_NOALLOC_MAX_JOBS 16384
+
+/* eval_fitness for callers that must not allocate device memory.  (The paper has no
+ * counterpart: this is a deployment variant of the Eq. 14 evaluation above, same kernels,
+ * same results.)
+ *
+ * Who needs it: a scheduler embedded in a process whose GPU memory is handed out in full
+ * to a caching allocator at start-up, where a later cudaMalloc can simply fail; and
+ * latency-critical control loops that cannot accept the device-wide synchronisation a
+ * cudaMalloc / cudaFree implies.  sched_init and the first eval_fitness call of a context
+ * allocate their scratch; this entry point never calls cudaMalloc, cudaFree or any
+ * allocating library routine.  It needs no context: sizes and the floor are passed
+ * directly, and all work is enqueued on `cuda_stream` (a cudaStream_t, NULL = default
+ * stream) of the current device.
+ *
+ * Its scratch (per-chunk partial sums, arrival counters, per-job penalty factors) is one
+ * fixed file-scope device array of about 2.2 MB that every GPU holding the library keeps
+ * from load to exit.  Hence fixed maxima: count <= SCHED_NOALLOC_MAX_COUNT, num_jobs <=
+ * SCHED_NOALLOC_MAX_JOBS, num_nodes <= SCHED_MAX_NODES, k_max <= SCHED_MAX_K, n_max <=
+ * SCHED_MAX_N; anything larger returns SCHED_ERR_TOO_LARGE (use eval_fitness, in chunks if
+ * need be).  The first call on each device resolves the array's device address (one
+ * cudaGetSymbolAddress, with that device current) and reads the SM count; make that first
+ * call before any stream capture.  All calls share the one array: the part a call relies
+ * on being zero is cleared on the stream at the start of each call, the rest is
+ * overwritten before it is read, but two calls whose kernels overlap on the GPU (different
+ * streams, or different host threads on different streams) race on it - serialise them.
+ * Host-side the call is guarded by a mutex.
+ *
+ * Arguments as eval_fitness: d_pop int16 [count][num_jobs][num_nodes], d_speedup fp32
+ * [num_jobs][k_max+1][n_max+1], optional d_cur / d_realloc_factor / d_active, exponent p,
+ * floor, d_fitness fp32 [count].  Errors: INVALID_ARG, TOO_LARGE, CUDA; the reason is in
+ * eval_fitness_noalloc_last_error(). */
+int eval_fitness_noalloc(const int16_t *d_pop, int32_t count, int32_t num_jobs, int32_t num_nodes,
+                         int32_t k_max, int32_t n_max, const float *d_speedup, const int16_t *d_cur,
+                         const float *d_realloc_factor, const uint8_t *d_active, float p,
+                         float speedup_floor, float *d_fitness, void *cuda_stream);
+const char *eval_fitness_noalloc_last_error(void);
+
 #ifdef __cplusplus
 }
 #endif

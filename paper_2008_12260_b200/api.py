@@ -22,7 +22,7 @@ EXPORTS = (
     "init_population", "ga_generation", "schedule_round", "schedule_round_host",
     "sched_get_population", "sched_round_speedup_table", "eval_fitness_host",
     "sched_set_kernel_timing", "sched_num_kernel_kinds", "sched_kernel_kind_name",
-    "sched_read_kernel_timing",
+    "sched_read_kernel_timing", "eval_fitness_noalloc", "eval_fitness_noalloc_last_error",
 )
 
 
@@ -82,6 +82,9 @@ def load_library(path: str = LIB_PATH):
     lib.sched_kernel_kind_name.argtypes = [i32]
     lib.sched_kernel_kind_name.restype = C.c_char_p
     lib.sched_read_kernel_timing.argtypes = [vp, vp, vp]
+    lib.eval_fitness_noalloc.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, f32, f32, vp, vp]
+    lib.eval_fitness_noalloc_last_error.argtypes = []
+    lib.eval_fitness_noalloc_last_error.restype = C.c_char_p
     for name in EXPORTS:
         if getattr(lib, name).restype is C.c_int:
             getattr(lib, name).restype = C.c_int
@@ -251,6 +254,21 @@ class Scheduler:
     def eval_fitness_host(self, pop, speedup, fitness, *, p, cur=None, realloc_factor=None, active=None):
         self._check(_lib.eval_fitness_host(self._ctx, _ptr(pop), pop.shape[0], _ptr(speedup), _ptr(cur),
                                            _ptr(realloc_factor), _ptr(active), p, _ptr(fitness)))
+
+
+def eval_fitness_noalloc(pop, speedup, fitness, *, k_max, n_max, p, speedup_floor, cur=None,
+                         realloc_factor=None, active=None, stream=None, count=None):
+    """Fitness of `pop` ([count][J][num_nodes] int16 on the device) without a context and
+    without any device allocation inside the library: for processes whose allocator already
+    owns the whole GPU, or loops that cannot take cudaMalloc's device-wide synchronisation.
+    See the header for the fixed limits (count <= 2048, J <= 16384) and the sharing rules of
+    its static scratch array."""
+    n = pop.shape[0] if count is None else count
+    rc = _lib.eval_fitness_noalloc(_ptr(pop), n, pop.shape[1], pop.shape[2], k_max, n_max, _ptr(speedup),
+                                   _ptr(cur), _ptr(realloc_factor), _ptr(active), p, speedup_floor,
+                                   _ptr(fitness), stream)
+    if rc != SCHED_OK:
+        raise SchedError(rc, _lib.eval_fitness_noalloc_last_error().decode())
 
 
 def scheduler_for(cfg, jobs=None, stream=None, **overrides):

@@ -291,3 +291,144 @@ int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const fl
   }
   return SCHED_OK;
 }
+
+// ---------------------------------------------------------------------------------------
+// Fitness without any allocation: same kernels, scratch in a fixed file-scope device array.
+// ---------------------------------------------------------------------------------------
+#include <mutex>
+
+namespace {
+
+constexpr int NOALLOC_MAX_COUNT = SCHED_NOALLOC_MAX_COUNT;
+constexpr int NOALLOC_MAX_JOBS = SCHED_NOALLOC_MAX_JOBS;
+constexpr int NOALLOC_MAX_CHUNKS = NOALLOC_MAX_JOBS / 256;   // a block covers at least 256 rows
+
+struct NoAllocScratch {
+  double partial[(size_t)NOALLOC_MAX_COUNT * NOALLOC_MAX_CHUNKS * 2];
+  unsigned int ticket[NOALLOC_MAX_COUNT];
+  float pen[NOALLOC_MAX_JOBS];
+};
+
+// Lives in every GPU that loads the library, from load to exit (about 2.2 MB).  In host code
+// this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+std::mutex g_noalloc_mutex;
+NoAllocScratch *g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {};
+int g_noalloc_sms[NOALLOC_MAX_DEVICES] = {};
+char g_noalloc_error[256] = "";
+
+int noalloc_fail(int code, const char *msg, cudaError_t e = cudaSuccess) {
+  if (e != cudaSuccess) snprintf(g_noalloc_error, sizeof(g_noalloc_error), "%s: %s", msg, cudaGetErrorString(e));
+  else snprintf(g_noalloc_error, sizeof(g_noalloc_error), "%s", msg);
+  return code;
+}
+
+}  // namespace
+
+extern "C" {
+#pragma GCC visibility push(default)
+
+const char *eval_fitness_noalloc_last_error(void) { return g_noalloc_error; }
+
+int eval_fitness_noalloc(const int16_t *d_pop, int32_t count, int32_t num_jobs, int32_t num_nodes,
+                         int32_t k_max, int32_t n_max, const float *d_speedup, const int16_t *d_cur,
+                         const float *d_realloc_factor, const uint8_t *d_active, float p,
+                         float speedup_floor, float *d_fitness, void *cuda_stream) {
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (count < 0 || num_jobs < 1 || num_nodes < 1 || k_max < 1 || n_max < 1)
+    return noalloc_fail(SCHED_ERR_INVALID_ARG, "eval_fitness_noalloc: sizes must be positive");
+  if (count == 0) return SCHED_OK;
+  if (!d_pop || !d_speedup || !d_fitness)
+    return noalloc_fail(SCHED_ERR_INVALID_ARG, "eval_fitness_noalloc: d_pop, d_speedup and d_fitness must be non-NULL");
+  if (count > NOALLOC_MAX_COUNT || num_jobs > NOALLOC_MAX_JOBS || num_nodes > SCHED_MAX_NODES ||
+      k_max > SCHED_MAX_K || n_max > SCHED_MAX_N)
+    return noalloc_fail(SCHED_ERR_TOO_LARGE,
+                        "eval_fitness_noalloc: count <= 2048, num_jobs <= 16384, num_nodes <= 8192, "
+                        "k_max, n_max <= 1024 (the scratch array is fixed; use eval_fitness beyond that)");
+  if (!(p == p) || !(speedup_floor >= 0.f))
+    return noalloc_fail(SCHED_ERR_INVALID_ARG, "eval_fitness_noalloc: p is NaN or speedup_floor negative");
+  if (((uintptr_t)d_pop & 1) || ((uintptr_t)d_cur & 1) || ((uintptr_t)d_speedup & 3) || ((uintptr_t)d_fitness & 3))
+    return noalloc_fail(SCHED_ERR_INVALID_ARG, "eval_fitness_noalloc: a buffer is not aligned to its element size");
+
+  // set-up, once per device, with that device current: resolve the scratch array's address
+  int device = -1;
+  cudaError_t e = cudaGetDevice(&device);
+  if (e != cudaSuccess) return noalloc_fail(SCHED_ERR_CUDA, "cudaGetDevice", e);
+  if (device < 0 || device >= NOALLOC_MAX_DEVICES)
+    return noalloc_fail(SCHED_ERR_TOO_LARGE, "eval_fitness_noalloc: device ordinal beyond 63");
+  if (!g_noalloc_ptr[device]) {
+    void *ptr = nullptr;
+    e = cudaGetSymbolAddress((void **)&ptr, g_noalloc_scratch);
+    if (e != cudaSuccess || !ptr) return noalloc_fail(SCHED_ERR_CUDA, "cudaGetSymbolAddress(scratch)", e);
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    if (e != cudaSuccess) return noalloc_fail(SCHED_ERR_CUDA, "cudaDeviceGetAttribute", e);
+    g_noalloc_sms[device] = sms;
+    g_noalloc_ptr[device] = (NoAllocScratch *)ptr;
+  }
+  NoAllocScratch *scratch = g_noalloc_ptr[device];
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  const int J = num_jobs;
+
+  // the arrival counters must start at zero; the array keeps whatever the last call left
+  e = cudaMemsetAsync(scratch->ticket, 0, sizeof(unsigned int) * (size_t)count, stream);
+  if (e != cudaSuccess) return noalloc_fail(SCHED_ERR_CUDA, "cudaMemsetAsync(ticket)", e);
+
+  const bool penalise = d_cur && d_realloc_factor;
+  if (penalise) {
+    penalty_prep_kernel<<<(J * 32 + 255) / 256, 256, 0, stream>>>(d_cur, d_realloc_factor, J, num_nodes,
+                                                                 scratch->pen);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return noalloc_fail(SCHED_ERR_CUDA, "penalty_prep_kernel launch", e);
+  }
+
+  const size_t row_bytes = (size_t)num_nodes * 2;
+  const uintptr_t al = (uintptr_t)d_pop | (penalise ? (uintptr_t)d_cur : 0);
+  int W = 2;
+  if (row_bytes % 16 == 0 && al % 16 == 0) W = 16;
+  else if (row_bytes % 8 == 0 && al % 8 == 0) W = 8;
+  else if (row_bytes % 4 == 0 && al % 4 == 0) W = 4;
+  const int row_vecs = (int)(row_bytes / W);
+  int lpr_log2 = 0;
+  while ((1 << lpr_log2) < row_vecs && lpr_log2 < 5) ++lpr_log2;
+  int rows_per_block = (int)((1u << 20) / row_bytes);
+  if (rows_per_block < 256) rows_per_block = 256;
+  if (rows_per_block > J) rows_per_block = J;
+  while (rows_per_block > 256 &&
+         (long long)count * ((J + rows_per_block - 1) / rows_per_block) < 4LL * g_noalloc_sms[device])
+    rows_per_block = (rows_per_block + 1) / 2;
+  const int chunks = (J + rows_per_block - 1) / rows_per_block;
+  if (chunks > NOALLOC_MAX_CHUNKS)
+    return noalloc_fail(SCHED_ERR_TOO_LARGE, "eval_fitness_noalloc: internal chunk count exceeds the scratch array");
+
+  FitnessArgs a;
+  a.pop = d_pop;
+  a.cur = penalise ? d_cur : nullptr;
+  a.table = d_speedup;
+  a.pen = penalise ? scratch->pen : nullptr;
+  a.active = d_active;
+  a.J = J; a.num_nodes = num_nodes; a.k_max = k_max; a.n_max = n_max;
+  a.lpr_log2 = lpr_log2;
+  a.rows_per_block = rows_per_block; a.chunks = chunks;
+  a.p = p; a.floor_ = speedup_floor;
+  a.mode = (p == 1.f) ? MODE_ARITH : (p == -1.f) ? MODE_HARM : (p == 0.f) ? MODE_GEO
+           : (p == 0.5f) ? MODE_SQRT : MODE_POW;
+  a.partial = scratch->partial;
+  a.ticket = scratch->ticket;
+  a.fitness = d_fitness;
+  dim3 grid((unsigned)chunks, (unsigned)count);
+  switch (W) {
+    case 16: fitness_kernel<16><<<grid, 256, 0, stream>>>(a); break;
+    case 8: fitness_kernel<8><<<grid, 256, 0, stream>>>(a); break;
+    case 4: fitness_kernel<4><<<grid, 256, 0, stream>>>(a); break;
+    default: fitness_kernel<2><<<grid, 256, 0, stream>>>(a); break;
+  }
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return noalloc_fail(SCHED_ERR_CUDA, "fitness_kernel launch", e);
+  return SCHED_OK;
+}
+
+#pragma GCC visibility pop
+}  // extern "C"
