@@ -126,6 +126,24 @@ int ensure_dflag(sched_ctx *ctx, int32_t count) {
   return SCHED_OK;
 }
 
+int ensure_colscratch(sched_ctx *ctx, size_t ints) {
+  if (ints > ctx->col_cap) {
+    if (ctx->d_colsum || ctx->d_colelig) {
+      SCHED_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
+      if (ctx->d_colsum) SCHED_CUDA_CHECK(ctx, cudaFree(ctx->d_colsum));
+      if (ctx->d_colelig) SCHED_CUDA_CHECK(ctx, cudaFree(ctx->d_colelig));
+      ctx->d_colsum = ctx->d_colelig = nullptr;
+    }
+    ctx->col_cap = 0;
+    int rc = dev_alloc(ctx, &ctx->d_colsum, ints);
+    if (rc != SCHED_OK) return rc;
+    rc = dev_alloc(ctx, &ctx->d_colelig, ints);
+    if (rc != SCHED_OK) return rc;
+    ctx->col_cap = ints;
+  }
+  return SCHED_OK;
+}
+
 extern "C" {
 #pragma GCC visibility push(default)
 
@@ -172,6 +190,7 @@ int sched_init(const sched_config *cfg, const int16_t *h_node_capacity, void *cu
   // replicas that fit on the N largest nodes, N = 0..n_max
   std::vector<int16_t> sorted(h_node_capacity, h_node_capacity + cfg->num_nodes);
   std::sort(sorted.begin(), sorted.end(), [](int16_t a, int16_t b) { return a > b; });
+  ctx->cap_max = std::max<int>(sorted[0], 0);
   std::vector<int32_t> kfit(ctx->ND, 0);
   for (int n = 1; n < ctx->ND; ++n) {
     const int add = (n <= cfg->num_nodes && sorted[n - 1] > 0) ? sorted[n - 1] : 0;
@@ -211,7 +230,8 @@ int sched_destroy(sched_ctx *ctx) {
   void *ptrs[] = {ctx->d_cap, ctx->d_kfit, ctx->d_gmax, ctx->d_amax, ctx->d_rank, ctx->d_order,
                   ctx->d_dflag, ctx->d_pen, ctx->d_partial, ctx->d_ticket, ctx->d_status,
                   ctx->d_popA, ctx->d_popB, ctx->d_fit, ctx->d_tab_goodput, ctx->d_tab_speedup,
-                  ctx->d_rf, ctx->d_best_idx, ctx->d_stage, ctx->d_stage_fit};
+                  ctx->d_rf, ctx->d_best_idx, ctx->d_stage, ctx->d_stage_fit, ctx->d_colsum,
+                  ctx->d_colelig};
   for (void *p : ptrs)
     if (p) cudaFree(p);
   for (auto *v : {&ctx->spans, &ctx->free_spans})

@@ -49,7 +49,9 @@ struct sched_ctx {
   float *d_pen;          // [J] effective penalty factor (1 when none applies)
   double *d_partial;     // [count][chunks] partial sums of the fitness reduction
   unsigned int *d_ticket;  // [count] arrival counters of the fitness reduction
-  size_t partial_cap, ticket_cap, dflag_cap;
+  int32_t *d_colsum, *d_colelig;  // [count][row batches][num_nodes] column partials of the row pass
+  size_t partial_cap, ticket_cap, dflag_cap, col_cap;
+  int cap_max;           // largest node size
   int *d_status;         // device status word
 
   // scratch of schedule_round (allocated on first use)
@@ -184,3 +186,4 @@ int launch_select_best(sched_ctx *ctx, const int16_t *d_pop, const float *d_fitn
                        int16_t *d_best, float *d_best_fitness);
 int ensure_fitness_scratch(sched_ctx *ctx, int32_t count, int chunks);
 int ensure_dflag(sched_ctx *ctx, int32_t count);
+int ensure_colscratch(sched_ctx *ctx, size_t ints);

@@ -302,6 +302,312 @@ __global__ void copy_best_kernel(const int16_t *__restrict__ pop, const int32_t 
     out[i] = src[i];
 }
 
+
+// ---------------------------------------------------------------------------------------
+// Batched row kernel with fused column sums (rows of at most 64 16-byte vectors).
+//
+// A block owns 256 consecutive rows of one candidate, a warp 32 of them.  Each lane draws
+// the crossover / perturbation words of "its" row once (32 Philox calls run side by side
+// instead of one per warp), then the warp walks the 32 rows: one 16-byte load per lane and
+// vector, clamp, row totals by shuffle, store.  Rows that are perturbed or break a row cap
+// detour through shared memory.  While walking, every lane accumulates, for its own
+// columns, the GPUs placed and the number of distributed jobs; the block's column partials
+// go to scratch, so the column pass never re-reads the population.
+// ---------------------------------------------------------------------------------------
+struct Rows2Args {
+  RowsArgs r;
+  int32_t *colsum;   // [count][nbatch][num_nodes] GPUs placed on the node by the batch's rows
+  int32_t *colelig;  // same shape: rows of the batch that are distributed and occupy the node
+  int nbatch;
+};
+
+__device__ __forceinline__ uint4 clamp_vec(uint4 x, uint4 cp) {
+  x.x = __vimin_s16x2_relu(x.x, cp.x);
+  x.y = __vimin_s16x2_relu(x.y, cp.y);
+  x.z = __vimin_s16x2_relu(x.z, cp.z);
+  x.w = __vimin_s16x2_relu(x.w, cp.w);
+  return x;
+}
+
+// K in the low 22 bits, occupied-node count in the high 10 (entries are >= 0 here)
+__device__ __forceinline__ uint32_t row_partial(uint4 x) {
+  const uint32_t k = (x.x & 0xFFFFu) + (x.x >> 16) + (x.y & 0xFFFFu) + (x.y >> 16) +
+                     (x.z & 0xFFFFu) + (x.z >> 16) + (x.w & 0xFFFFu) + (x.w >> 16);
+  const uint32_t o = __vimin_s16x2_relu(x.x, 0x00010001u) + __vimin_s16x2_relu(x.y, 0x00010001u) +
+                     __vimin_s16x2_relu(x.z, 0x00010001u) + __vimin_s16x2_relu(x.w, 0x00010001u);
+  return k | (((o & 0xFFFFu) + (o >> 16)) << 22);
+}
+
+template <int VPL>
+__global__ void __launch_bounds__(256) rows2_kernel(Rows2Args aa) {
+  const RowsArgs &a = aa.r;
+  __shared__ __align__(16) int16_t s_row[8][256 * VPL];   // per-warp detour buffer
+  __shared__ int32_t s_tot[256 * VPL], s_el[256 * VPL];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int cl = blockIdx.y, batch = blockIdx.x;
+  const uint32_t c = a.first_cand + (uint32_t)cl;
+  const int NN = a.num_nodes, J = a.J;
+  const int row_vecs = NN >> 3;
+  for (int i = threadIdx.x; i < NN; i += blockDim.x) { s_tot[i] = 0; s_el[i] = 0; }
+  __syncthreads();
+
+  const int j0 = batch * 256 + warp * 32;
+  const int nrows = min(32, J - j0);          // may be <= 0 for trailing warps
+  // ---- per-lane set-up for row j0 + lane -------------------------------------------------
+  int parent_l = 0;
+  uint32_t flags_l = 0;                       // bit 0 perturb, bit 1 active, bits 2.. replica cap
+  u32x4 mw = {0, 0, 0, 0};
+  if (lane < nrows) {
+    const int j = j0 + lane;
+    const bool act = !a.active || a.active[j];
+    int kc = a.k_cap ? a.k_cap[j] : a.k_max;
+    kc = max(0, min(kc, a.k_max));
+    bool mut = false;
+    if (a.mode == ROWS_GENERATION) {
+      if ((int)c < a.num_elite) {
+        parent_l = a.order[c];
+      } else {
+        const u32x4 s = draw(a.key, 0u, c, a.gen, SLOT_SELECT);
+        const int i0 = bounded(s.x, a.P), i1 = bounded(s.y, a.P);
+        const int i2 = bounded(s.z, a.P), i3 = bounded(s.w, a.P);
+        const int pa = a.rank[i0] <= a.rank[i1] ? i0 : i1;
+        const int pb = a.rank[i2] <= a.rank[i3] ? i2 : i3;
+        const u32x4 x = draw(a.key, (uint32_t)j, c, a.gen, SLOT_XOVER);
+        parent_l = (x.x >> 31) ? pb : pa;
+        mw = draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE);
+        mut = mw.x < a.thr;
+      }
+    } else if (a.mode == ROWS_INIT && c > 0) {
+      mw = draw(a.key, (uint32_t)j, c, GEN_INIT, SLOT_INIT);
+      mut = mw.x < a.thr;
+    }
+    flags_l = (mut ? 1u : 0u) | (act ? 2u : 0u) | ((uint32_t)kc << 2);
+  }
+  // node sizes of this lane's columns, floored at 0
+  uint4 capv[VPL];
+#pragma unroll
+  for (int q = 0; q < VPL; ++q) {
+    const int v = lane + 32 * q;
+    capv[q] = make_uint4(0, 0, 0, 0);
+    if (v < row_vecs) {
+      const uint4 t = __ldg((const uint4 *)a.cap + v);
+      capv[q] = make_uint4(__vimax_s16x2_relu(t.x, 0u), __vimax_s16x2_relu(t.y, 0u),
+                           __vimax_s16x2_relu(t.z, 0u), __vimax_s16x2_relu(t.w, 0u));
+    }
+  }
+  uint4 tot[VPL], el[VPL];
+#pragma unroll
+  for (int q = 0; q < VPL; ++q) { tot[q] = make_uint4(0, 0, 0, 0); el[q] = make_uint4(0, 0, 0, 0); }
+  int16_t *row = s_row[warp];
+
+  for (int r = 0; r < nrows; ++r) {
+    const int j = j0 + r;
+    const int parent = __shfl_sync(0xffffffffu, parent_l, r);
+    const uint32_t flags = __shfl_sync(0xffffffffu, flags_l, r);
+    int16_t *out = a.dst + ((size_t)cl * J + j) * NN;
+    if (!(flags & 2u)) {                      // inactive job: empty row
+#pragma unroll
+      for (int q = 0; q < VPL; ++q)
+        if (lane + 32 * q < row_vecs) ((uint4 *)out)[lane + 32 * q] = make_uint4(0, 0, 0, 0);
+      if (lane == 0) a.dflag[(size_t)cl * J + j] = 0;
+      continue;
+    }
+    const int16_t *src;
+    if (a.mode == ROWS_GENERATION) src = a.src + ((size_t)parent * J + j) * NN;
+    else if (a.mode == ROWS_INIT) src = a.src ? a.src + (size_t)j * NN : nullptr;
+    else src = out;
+    uint4 x[VPL];
+    uint32_t part = 0;
+#pragma unroll
+    for (int q = 0; q < VPL; ++q) {
+      const int v = lane + 32 * q;
+      x[q] = make_uint4(0, 0, 0, 0);
+      if (src && v < row_vecs) x[q] = clamp_vec(__ldg((const uint4 *)src + v), capv[q]);
+      part += row_partial(x[q]);
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+    int K = (int)(part & 0x3FFFFFu), N = (int)(part >> 22);
+    const int kc = (int)(flags >> 2);
+    if ((flags & 1u) || K > kc || N > a.n_max) {
+      // detour: row into shared memory, perturb, apply the row caps, read it back
+#pragma unroll
+      for (int q = 0; q < VPL; ++q)
+        if (lane + 32 * q < row_vecs) ((uint4 *)row)[lane + 32 * q] = x[q];
+      __syncwarp();
+      if (flags & 1u) {
+        const uint32_t m1 = __shfl_sync(0xffffffffu, mw.y, r), m2 = __shfl_sync(0xffffffffu, mw.z, r),
+                       m3 = __shfl_sync(0xffffffffu, mw.w, r);
+        const uint32_t op = bounded(m1, 3u);
+        if (op == 0u) {
+          const int n = (int)bounded(m3, (uint32_t)NN);
+          if (lane == 0) row[n] = (int16_t)min((int)row[n] + 1, max((int)a.cap[n], 0));
+        } else if (N > 0) {
+          const int ns = nth_occupied(row, NN, bounded(m2, (uint32_t)N), lane);
+          if (op == 1u) {
+            if (lane == 0) row[ns] = (int16_t)(row[ns] - 1);
+          } else {
+            const int nd = (int)bounded(m3, (uint32_t)NN);
+            if (nd != ns && lane == 0) {
+              row[nd] = (int16_t)min((int)row[nd] + (int)row[ns], max((int)a.cap[nd], 0));
+              row[ns] = 0;
+            }
+          }
+        }
+        __syncwarp();
+        K = 0; N = 0;
+        for (int n = lane; n < NN; n += 32) { K += row[n]; N += row[n] > 0; }
+        K = warp_sum(K);
+        N = warp_sum(N);
+      }
+      if (K > kc || N > a.n_max) {
+        if (lane == 0) {
+          int excess = K - kc;
+          for (int n = NN - 1; n >= 0 && excess > 0; --n) {
+            const int take = min((int)row[n], excess);
+            row[n] = (int16_t)(row[n] - take);
+            excess -= take;
+          }
+          int occ = 0;
+          for (int n = 0; n < NN; ++n) {
+            if (row[n] > 0) {
+              ++occ;
+              if (occ > a.n_max) row[n] = 0;
+            }
+          }
+          N = min(occ, a.n_max);
+        }
+        N = __shfl_sync(0xffffffffu, N, 0);
+      }
+      __syncwarp();
+#pragma unroll
+      for (int q = 0; q < VPL; ++q)
+        if (lane + 32 * q < row_vecs) x[q] = ((const uint4 *)row)[lane + 32 * q];
+      __syncwarp();
+    }
+    const bool dist = N >= 2;
+#pragma unroll
+    for (int q = 0; q < VPL; ++q) {
+      if (lane + 32 * q < row_vecs) ((uint4 *)out)[lane + 32 * q] = x[q];
+      tot[q].x += x[q].x; tot[q].y += x[q].y; tot[q].z += x[q].z; tot[q].w += x[q].w;
+      if (dist) {
+        el[q].x += __vimin_s16x2_relu(x[q].x, 0x00010001u);
+        el[q].y += __vimin_s16x2_relu(x[q].y, 0x00010001u);
+        el[q].z += __vimin_s16x2_relu(x[q].z, 0x00010001u);
+        el[q].w += __vimin_s16x2_relu(x[q].w, 0x00010001u);
+      }
+    }
+    if (lane == 0) a.dflag[(size_t)cl * J + j] = dist ? 1 : 0;
+  }
+
+  // ---- column partials of the block --------------------------------------------------------
+#pragma unroll
+  for (int q = 0; q < VPL; ++q) {
+    const int v = lane + 32 * q;
+    if (v < row_vecs) {
+      const uint32_t t[4] = {tot[q].x, tot[q].y, tot[q].z, tot[q].w};
+      const uint32_t e[4] = {el[q].x, el[q].y, el[q].z, el[q].w};
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        const int n = v * 8 + w * 2;
+        if (t[w] & 0xFFFFu) atomicAdd(&s_tot[n], (int)(t[w] & 0xFFFFu));
+        if (t[w] >> 16) atomicAdd(&s_tot[n + 1], (int)(t[w] >> 16));
+        if (e[w] & 0xFFFFu) atomicAdd(&s_el[n], (int)(e[w] & 0xFFFFu));
+        if (e[w] >> 16) atomicAdd(&s_el[n + 1], (int)(e[w] >> 16));
+      }
+    }
+  }
+  __syncthreads();
+  const size_t base = ((size_t)cl * aa.nbatch + batch) * NN;
+  for (int i = threadIdx.x; i < NN; i += blockDim.x) {
+    aa.colsum[base + i] = s_tot[i];
+    aa.colelig[base + i] = s_el[i];
+  }
+}
+
+struct ColfixArgs {
+  int16_t *pop;
+  const uint8_t *dflag;
+  const int16_t *cap;
+  const int32_t *colsum, *colelig;
+  int J, num_nodes, nbatch;
+  uint32_t gen, first_cand;
+  RngKey key;
+};
+
+// Column pass on the batch partials: a thread per (candidate, node) adds them up; columns
+// that hold two distributed jobs or exceed the node size are then repaired by the whole
+// warp, one column at a time (same rules as cols_kernel).
+__global__ void __launch_bounds__(128) colfix_kernel(ColfixArgs a) {
+  const int lane = threadIdx.x & 31;
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  const int cl = blockIdx.y;
+  const uint32_t c = a.first_cand + (uint32_t)cl;
+  const int J = a.J, NN = a.num_nodes;
+  int total = 0, nelig = 0, cp = 0;
+  if (n < NN) {
+    for (int b = 0; b < a.nbatch; ++b) {
+      total += a.colsum[((size_t)cl * a.nbatch + b) * NN + n];
+      nelig += a.colelig[((size_t)cl * a.nbatch + b) * NN + n];
+    }
+    cp = max((int)a.cap[n], 0);
+  }
+  unsigned todo = __ballot_sync(0xffffffffu, n < NN && (nelig >= 2 || total > cp));
+  const uint8_t *df = a.dflag + (size_t)cl * J;
+  while (todo) {
+    const int src = __ffs(todo) - 1;
+    todo &= todo - 1;
+    const int nn = __shfl_sync(0xffffffffu, n, src);
+    int tot = __shfl_sync(0xffffffffu, total, src);
+    const int ne = __shfl_sync(0xffffffffu, nelig, src);
+    const int cap_n = __shfl_sync(0xffffffffu, cp, src);
+    int16_t *col = a.pop + (size_t)cl * J * NN + nn;
+    if (ne >= 2) {
+      const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
+      int best = J;
+      for (int j = lane; j < J; j += 32) {
+        if (df[j] && col[(size_t)j * NN] > 0) {
+          int t = j - o;
+          if (t < 0) t += J;
+          best = min(best, t);
+        }
+      }
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, off));
+      int keep = o + best;
+      if (keep >= J) keep -= J;
+      int removed = 0;
+      for (int j = lane; j < J; j += 32) {
+        if (j != keep && df[j]) {
+          const int v = col[(size_t)j * NN];
+          if (v > 0) { col[(size_t)j * NN] = 0; removed += v; }
+        }
+      }
+      tot -= warp_sum(removed);
+    }
+    int excess = tot - cap_n;
+    if (excess > 0) {
+      const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J);
+      for (int t0 = 0; t0 < J && excess > 0; t0 += 32) {
+        const int t = t0 + lane;
+        int j = o + t;
+        if (j >= J) j -= J;
+        const int v = (t < J) ? (int)col[(size_t)j * NN] : 0;
+        int s = v;                                   // inclusive prefix over the 32 jobs
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const int u = __shfl_up_sync(0xffffffffu, s, off);
+          if (lane >= off) s += u;
+        }
+        const int take = min(v, max(excess - (s - v), 0));
+        if (take > 0) col[(size_t)j * NN] = (int16_t)(v - take);
+        excess -= __shfl_sync(0xffffffffu, s, 31);
+      }
+    }
+    __syncwarp();
+  }
+}
+
 int launch_rows(sched_ctx *ctx, RowsArgs &a) {
   const long long warps = (long long)a.count * a.J;
   if (warps == 0) return SCHED_OK;
@@ -343,6 +649,44 @@ int launch_cols(sched_ctx *ctx, int16_t *pop, int count, uint32_t first_cand, ui
   return SCHED_OK;
 }
 
+// Row pass + column pass of `count` candidates.  Rows of a multiple of 8 and at most 512
+// nodes (16-byte vectors, <= 2 per lane) with node sizes <= 2047 take the batched kernels
+// with fused column sums; everything else the general warp-per-row / thread-per-column pair.
+int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint32_t first_cand,
+                     uint32_t round, uint32_t gen) {
+  if (count == 0 || a.J == 0) return SCHED_OK;
+  const int NN = a.num_nodes;
+  const bool aligned = ((((uintptr_t)a.dst | (uintptr_t)a.src) & 15) == 0);
+  const bool fused = (NN % 8 == 0) && NN <= 512 && aligned && ctx->cap_max <= 2047 && count <= 65535;
+  if (!fused) {
+    int rc = launch_rows(ctx, a);
+    if (rc != SCHED_OK) return rc;
+    return launch_cols(ctx, pop, count, first_cand, round, gen);
+  }
+  const int nbatch = (a.J + 255) / 256;
+  int rc = ensure_colscratch(ctx, (size_t)count * nbatch * NN);
+  if (rc != SCHED_OK) return rc;
+  Rows2Args aa;
+  aa.r = a;
+  aa.colsum = ctx->d_colsum; aa.colelig = ctx->d_colelig; aa.nbatch = nbatch;
+  dim3 grid((unsigned)nbatch, (unsigned)count);
+  {
+    TimedLaunch tl_(ctx, KK_ROWS);
+    if (NN <= 256) rows2_kernel<1><<<grid, 256, 0, ctx->stream>>>(aa);
+    else rows2_kernel<2><<<grid, 256, 0, ctx->stream>>>(aa);
+  }
+  SCHED_LAUNCH_CHECK(ctx);
+  ColfixArgs f;
+  f.pop = pop; f.dflag = ctx->d_dflag; f.cap = ctx->d_cap;
+  f.colsum = ctx->d_colsum; f.colelig = ctx->d_colelig;
+  f.J = a.J; f.num_nodes = NN; f.nbatch = nbatch;
+  f.gen = gen; f.first_cand = first_cand; f.key = make_key(ctx->cfg.seed, round);
+  dim3 g2((unsigned)((NN + 127) / 128), (unsigned)count);
+  { TimedLaunch tl_(ctx, KK_COLS); colfix_kernel<<<g2, 128, 0, ctx->stream>>>(f); }
+  SCHED_LAUNCH_CHECK(ctx);
+  return SCHED_OK;
+}
+
 RowsArgs base_rows_args(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active, int count) {
   RowsArgs a;
   const sched_config &c = ctx->cfg;
@@ -365,9 +709,7 @@ int launch_repair(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_activ
   RowsArgs a = base_rows_args(ctx, d_k_cap, d_active, count);
   a.mode = ROWS_REPAIR; a.src = d_pop; a.dst = d_pop;
   a.first_cand = first_candidate; a.gen = generation; a.key = make_key(ctx->cfg.seed, round);
-  rc = launch_rows(ctx, a);
-  if (rc != SCHED_OK) return rc;
-  return launch_cols(ctx, d_pop, count, first_candidate, round, generation);
+  return launch_rows_cols(ctx, a, d_pop, count, first_candidate, round, generation);
 }
 
 int launch_init_population(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active,
@@ -378,9 +720,7 @@ int launch_init_population(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t
   RowsArgs a = base_rows_args(ctx, d_k_cap, d_active, P);
   a.mode = ROWS_INIT; a.src = d_cur; a.dst = d_pop_out;
   a.thr = ctx->cfg.thr_init; a.gen = GEN_INIT; a.key = make_key(ctx->cfg.seed, round);
-  rc = launch_rows(ctx, a);
-  if (rc != SCHED_OK) return rc;
-  return launch_cols(ctx, d_pop_out, P, 0u, round, GEN_INIT);
+  return launch_rows_cols(ctx, a, d_pop_out, P, 0u, round, GEN_INIT);
 }
 
 int launch_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active,
@@ -398,9 +738,7 @@ int launch_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_a
   RowsArgs a = base_rows_args(ctx, d_k_cap, d_active, P);
   a.mode = ROWS_GENERATION; a.src = d_pop_in; a.dst = d_pop_out;
   a.thr = ctx->cfg.thr_mutate; a.gen = generation; a.key = make_key(ctx->cfg.seed, round);
-  rc = launch_rows(ctx, a);
-  if (rc != SCHED_OK) return rc;
-  return launch_cols(ctx, d_pop_out, P, 0u, round, generation);
+  return launch_rows_cols(ctx, a, d_pop_out, P, 0u, round, generation);
 }
 
 int launch_select_best(sched_ctx *ctx, const int16_t *d_pop, const float *d_fitness,
