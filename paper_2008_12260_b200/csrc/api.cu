@@ -201,6 +201,15 @@ int sched_init(const sched_config *cfg, const int16_t *h_node_capacity, void *cu
   int rc;
   if ((rc = dev_alloc(ctx, &ctx->d_cap, ((size_t)cfg->num_nodes + 7) & ~(size_t)7)) != SCHED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_kfit, (size_t)ctx->ND)) != SCHED_OK) return fail(rc);
+  // (K, class) pairs that exist: class 0 (one node) needs K <= largest node; class 1 (several
+  // nodes) needs K >= 2 and K <= the min(K, n_max) largest nodes together
+  std::vector<int32_t> pairs;
+  for (int K = 1; K <= cfg->k_max; ++K) {
+    if (K <= kfit[1]) pairs.push_back(K * 2);
+    if (cfg->n_max >= 2 && K >= 2 && K <= kfit[std::min(K, cfg->n_max)]) pairs.push_back(K * 2 + 1);
+  }
+  ctx->num_pairs = (int)pairs.size();
+  if ((rc = dev_alloc(ctx, &ctx->d_pairs, pairs.size())) != SCHED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_gmax, J * ctx->KD * 2)) != SCHED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_amax, J * ctx->KD * 2)) != SCHED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_rank, P)) != SCHED_OK) return fail(rc);
@@ -212,6 +221,8 @@ int sched_init(const sched_config *cfg, const int16_t *h_node_capacity, void *cu
                       cudaMemcpyHostToDevice, ctx->stream);
   if (e == cudaSuccess)
     e = cudaMemcpyAsync(ctx->d_kfit, kfit.data(), sizeof(int32_t) * ctx->ND, cudaMemcpyHostToDevice, ctx->stream);
+  if (e == cudaSuccess && !pairs.empty())
+    e = cudaMemcpyAsync(ctx->d_pairs, pairs.data(), sizeof(int32_t) * pairs.size(), cudaMemcpyHostToDevice, ctx->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_status, 0, sizeof(int), ctx->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_gmax, 0, sizeof(float) * std::max<size_t>(J * ctx->KD * 2, 1), ctx->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_amax, 0xFF, sizeof(uint16_t) * std::max<size_t>(J * ctx->KD * 2, 1), ctx->stream);
@@ -227,7 +238,7 @@ int sched_init(const sched_config *cfg, const int16_t *h_node_capacity, void *cu
 int sched_destroy(sched_ctx *ctx) {
   if (!ctx) return SCHED_OK;
   cudaStreamSynchronize(ctx->stream);
-  void *ptrs[] = {ctx->d_cap, ctx->d_kfit, ctx->d_gmax, ctx->d_amax, ctx->d_rank, ctx->d_order,
+  void *ptrs[] = {ctx->d_cap, ctx->d_kfit, ctx->d_pairs, ctx->d_gmax, ctx->d_amax, ctx->d_rank, ctx->d_order,
                   ctx->d_dflag, ctx->d_pen, ctx->d_partial, ctx->d_ticket, ctx->d_status,
                   ctx->d_popA, ctx->d_popB, ctx->d_fit, ctx->d_tab_goodput, ctx->d_tab_speedup,
                   ctx->d_rf, ctx->d_best_idx, ctx->d_stage, ctx->d_stage_fit, ctx->d_colsum,
@@ -370,14 +381,21 @@ int schedule_round(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cu
   const float *rf = penalise ? ctx->d_rf : nullptr;
   int16_t *pa = ctx->d_popA, *pb = ctx->d_popB;
   if ((rc = launch_init_population(ctx, d_jobs->k_cap, d_jobs->active, d_cur, round, pa)) != SCHED_OK) return rc;
-  if ((rc = launch_fitness(ctx, pa, ctx->cfg.population, ctx->d_tab_speedup, d_cur, rf, d_jobs->active,
-                           ctx->cfg.p, ctx->d_fit)) != SCHED_OK) return rc;
-  for (int g = 0; g < generations; ++g) {
-    if ((rc = launch_generation(ctx, d_jobs->k_cap, d_jobs->active, pa, ctx->d_fit, pb, round, (uint32_t)g)) != SCHED_OK) return rc;
+  // the first fitness call of the round prepares the per-job penalty factors; the current
+  // allocation does not change within a round, so later generations reuse them
+  ctx->pen_ready = false;
+  rc = launch_fitness(ctx, pa, ctx->cfg.population, ctx->d_tab_speedup, d_cur, rf, d_jobs->active,
+                      ctx->cfg.p, ctx->d_fit);
+  ctx->pen_ready = (rc == SCHED_OK);
+  for (int g = 0; g < generations && rc == SCHED_OK; ++g) {
+    rc = launch_generation(ctx, d_jobs->k_cap, d_jobs->active, pa, ctx->d_fit, pb, round, (uint32_t)g);
+    if (rc != SCHED_OK) break;
     std::swap(pa, pb);
-    if ((rc = launch_fitness(ctx, pa, ctx->cfg.population, ctx->d_tab_speedup, d_cur, rf, d_jobs->active,
-                             ctx->cfg.p, ctx->d_fit)) != SCHED_OK) return rc;
+    rc = launch_fitness(ctx, pa, ctx->cfg.population, ctx->d_tab_speedup, d_cur, rf, d_jobs->active,
+                        ctx->cfg.p, ctx->d_fit);
   }
+  ctx->pen_ready = false;
+  if (rc != SCHED_OK) return rc;
   ctx->d_pop_last = pa;
   return launch_select_best(ctx, pa, ctx->d_fit, d_best, d_best_fitness);
 }

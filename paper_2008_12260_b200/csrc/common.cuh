@@ -41,6 +41,8 @@ struct sched_ctx {
   // device scratch owned by the context
   int16_t *d_cap;        // [num_nodes]
   int32_t *d_kfit;       // [ND] replicas that fit on the N largest nodes
+  int32_t *d_pairs;      // [num_pairs] K * 2 + class of every (K, class) that exists on this cluster
+  int num_pairs;
   float *d_gmax;         // [J][KD][2] compact goodput maxima (class local / node)
   uint16_t *d_amax;      // [J][KD][2]
   int32_t *d_rank;       // [P]
@@ -52,6 +54,7 @@ struct sched_ctx {
   int32_t *d_colsum, *d_colelig;  // [count][row batches][num_nodes] column partials of the row pass
   size_t partial_cap, ticket_cap, dflag_cap, col_cap;
   int cap_max;           // largest node size
+  bool pen_ready;        // d_pen already holds this round's factors (set by schedule_round)
   int *d_status;         // device status word
 
   // scratch of schedule_round (allocated on first use)

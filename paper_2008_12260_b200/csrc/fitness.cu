@@ -211,6 +211,28 @@ __global__ void penalty_prep_kernel(const int16_t *__restrict__ cur, const float
   if (lane == 0) pen[j] = (k > 0) ? rf[j] : 1.f;
 }
 
+// Launch geometry shared by the entry points: the widest vector that divides a row and
+// keeps every row aligned; lanes per row so that a lane owns about four vectors (several
+// loads in flight, few shuffle steps); rows per block of about 1 MB of population, shrunk
+// while the grid would leave SMs idle.
+void fitness_geometry(size_t row_bytes, uintptr_t align_bits, int J, int count, int num_sms, int &W,
+                      int &lpr_log2, int &rows_per_block, int &chunks) {
+  W = 2;
+  if (row_bytes % 16 == 0 && align_bits % 16 == 0) W = 16;
+  else if (row_bytes % 8 == 0 && align_bits % 8 == 0) W = 8;
+  else if (row_bytes % 4 == 0 && align_bits % 4 == 0) W = 4;
+  const int row_vecs = (int)(row_bytes / W);
+  lpr_log2 = 0;
+  while ((4 << lpr_log2) < row_vecs && lpr_log2 < 5) ++lpr_log2;
+  rows_per_block = (int)((1u << 20) / row_bytes);
+  if (rows_per_block < 256) rows_per_block = 256;
+  if (rows_per_block > J) rows_per_block = J > 0 ? J : 1;
+  while (rows_per_block > 256 &&
+         (long long)count * ((J + rows_per_block - 1) / rows_per_block) < 4LL * num_sms)
+    rows_per_block = (rows_per_block + 1) / 2;
+  chunks = J > 0 ? (J + rows_per_block - 1) / rows_per_block : 1;
+}
+
 }  // namespace
 
 int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const float *d_speedup,
@@ -221,7 +243,7 @@ int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const fl
   if (count == 0) return SCHED_OK;
 
   const bool penalise = d_cur && d_rf;
-  if (penalise && J > 0) {
+  if (penalise && J > 0 && !ctx->pen_ready) {
     {
     TimedLaunch tl_(ctx, KK_PENPREP);
     penalty_prep_kernel<<<(J * 32 + 255) / 256, 256, 0, ctx->stream>>>(d_cur, d_rf, J, c.num_nodes,
@@ -230,26 +252,9 @@ int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const fl
     SCHED_LAUNCH_CHECK(ctx);
   }
 
-  // widest vector that divides the row and keeps every row aligned
-  const size_t row_bytes = (size_t)c.num_nodes * 2;
-  const uintptr_t al = (uintptr_t)d_pop | (penalise ? (uintptr_t)d_cur : 0);
-  int W = 2;
-  if (row_bytes % 16 == 0 && al % 16 == 0) W = 16;
-  else if (row_bytes % 8 == 0 && al % 8 == 0) W = 8;
-  else if (row_bytes % 4 == 0 && al % 4 == 0) W = 4;
-  const int row_vecs = (int)(row_bytes / W);
-  int lpr_log2 = 0;
-  while ((1 << lpr_log2) < row_vecs && lpr_log2 < 5) ++lpr_log2;
-
-  // chunk of rows per block: about 1 MB of population, at least 32 rows per warp batch
-  int rows_per_block = (int)((1u << 20) / row_bytes);
-  if (rows_per_block < 256) rows_per_block = 256;
-  if (rows_per_block > J) rows_per_block = J > 0 ? J : 1;
-  // keep enough blocks in flight for small populations
-  while (rows_per_block > 256 && (long long)count * ((J + rows_per_block - 1) / rows_per_block) <
-                                     4LL * ctx->num_sms)
-    rows_per_block = (rows_per_block + 1) / 2;
-  const int chunks = J > 0 ? (J + rows_per_block - 1) / rows_per_block : 1;
+  int W, lpr_log2, rows_per_block, chunks;
+  fitness_geometry((size_t)c.num_nodes * 2, (uintptr_t)d_pop | (penalise ? (uintptr_t)d_cur : 0), J, count,
+                   ctx->num_sms, W, lpr_log2, rows_per_block, chunks);
   int rc = ensure_fitness_scratch(ctx, count, chunks);
   if (rc != SCHED_OK) return rc;
 
@@ -384,22 +389,9 @@ int eval_fitness_noalloc(const int16_t *d_pop, int32_t count, int32_t num_jobs, 
     if (e != cudaSuccess) return noalloc_fail(SCHED_ERR_CUDA, "penalty_prep_kernel launch", e);
   }
 
-  const size_t row_bytes = (size_t)num_nodes * 2;
-  const uintptr_t al = (uintptr_t)d_pop | (penalise ? (uintptr_t)d_cur : 0);
-  int W = 2;
-  if (row_bytes % 16 == 0 && al % 16 == 0) W = 16;
-  else if (row_bytes % 8 == 0 && al % 8 == 0) W = 8;
-  else if (row_bytes % 4 == 0 && al % 4 == 0) W = 4;
-  const int row_vecs = (int)(row_bytes / W);
-  int lpr_log2 = 0;
-  while ((1 << lpr_log2) < row_vecs && lpr_log2 < 5) ++lpr_log2;
-  int rows_per_block = (int)((1u << 20) / row_bytes);
-  if (rows_per_block < 256) rows_per_block = 256;
-  if (rows_per_block > J) rows_per_block = J;
-  while (rows_per_block > 256 &&
-         (long long)count * ((J + rows_per_block - 1) / rows_per_block) < 4LL * g_noalloc_sms[device])
-    rows_per_block = (rows_per_block + 1) / 2;
-  const int chunks = (J + rows_per_block - 1) / rows_per_block;
+  int W, lpr_log2, rows_per_block, chunks;
+  fitness_geometry((size_t)num_nodes * 2, (uintptr_t)d_pop | (penalise ? (uintptr_t)d_cur : 0), J, count,
+                   g_noalloc_sms[device], W, lpr_log2, rows_per_block, chunks);
   if (chunks > NOALLOC_MAX_CHUNKS)
     return noalloc_fail(SCHED_ERR_TOO_LARGE, "eval_fitness_noalloc: internal chunk count exceeds the scratch array");
 

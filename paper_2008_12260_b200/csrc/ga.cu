@@ -46,6 +46,7 @@ struct RowsArgs {
   const uint8_t *active;    // [J] or NULL
   const int32_t *rank;      // [P]   (generation mode)
   const int32_t *order;     // [P]
+  const uint32_t *fitness_bits;  // [P] parents' fitness (generation mode)
   uint8_t *dflag;           // [count][J]
   int mode, P, J, num_nodes, k_max, n_max, num_elite, count;
   uint32_t thr, gen, first_cand;
@@ -351,6 +352,48 @@ __global__ void __launch_bounds__(256) rows2_kernel(Rows2Args aa) {
   for (int i = threadIdx.x; i < NN; i += blockDim.x) { s_tot[i] = 0; s_el[i] = 0; }
   __syncthreads();
 
+  // ---- parents of this candidate (generation mode), found by the block itself -------------
+  // rank(i) = number of candidates ordered before i (fitness descending, index ascending).
+  // An elite child needs the candidate of rank c; any other child the better-ranked of two
+  // random pairs, i.e. the ranks of four candidates only.
+  __shared__ int s_parent[2];
+  __shared__ int s_rank4[4];
+  if (a.mode == ROWS_GENERATION) {
+    const int P = a.P;
+    if ((int)c < a.num_elite) {
+      for (int i = threadIdx.x; i < P; i += blockDim.x) {
+        const uint32_t ki = order_key(a.fitness_bits[i]);
+        int rk = 0;
+        for (int o = 0; o < P; ++o) {
+          const uint32_t ko = order_key(__ldg(a.fitness_bits + o));
+          rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
+        }
+        if (rk == (int)c) s_parent[0] = s_parent[1] = i;
+      }
+    } else {
+      const u32x4 sel = draw(a.key, 0u, c, a.gen, SLOT_SELECT);
+      const int idx[4] = {(int)bounded(sel.x, P), (int)bounded(sel.y, P), (int)bounded(sel.z, P),
+                          (int)bounded(sel.w, P)};
+      if (warp < 4) {
+        const int i = idx[warp];
+        const uint32_t ki = order_key(a.fitness_bits[i]);
+        int rk = 0;
+        for (int o = lane; o < P; o += 32) {
+          const uint32_t ko = order_key(__ldg(a.fitness_bits + o));
+          rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
+        }
+        rk = warp_sum(rk);
+        if (lane == 0) s_rank4[warp] = rk;
+      }
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        s_parent[0] = s_rank4[0] <= s_rank4[1] ? idx[0] : idx[1];
+        s_parent[1] = s_rank4[2] <= s_rank4[3] ? idx[2] : idx[3];
+      }
+    }
+  }
+  __syncthreads();
+
   const int j0 = batch * 256 + warp * 32;
   const int nrows = min(32, J - j0);          // may be <= 0 for trailing warps
   // ---- per-lane set-up for row j0 + lane -------------------------------------------------
@@ -365,15 +408,10 @@ __global__ void __launch_bounds__(256) rows2_kernel(Rows2Args aa) {
     bool mut = false;
     if (a.mode == ROWS_GENERATION) {
       if ((int)c < a.num_elite) {
-        parent_l = a.order[c];
+        parent_l = s_parent[0];
       } else {
-        const u32x4 s = draw(a.key, 0u, c, a.gen, SLOT_SELECT);
-        const int i0 = bounded(s.x, a.P), i1 = bounded(s.y, a.P);
-        const int i2 = bounded(s.z, a.P), i3 = bounded(s.w, a.P);
-        const int pa = a.rank[i0] <= a.rank[i1] ? i0 : i1;
-        const int pb = a.rank[i2] <= a.rank[i3] ? i2 : i3;
         const u32x4 x = draw(a.key, (uint32_t)j, c, a.gen, SLOT_XOVER);
-        parent_l = (x.x >> 31) ? pb : pa;
+        parent_l = (x.x >> 31) ? s_parent[1] : s_parent[0];
         mw = draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE);
         mut = mw.x < a.thr;
       }
@@ -659,6 +697,13 @@ int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint3
   const bool aligned = ((((uintptr_t)a.dst | (uintptr_t)a.src) & 15) == 0);
   const bool fused = (NN % 8 == 0) && NN <= 512 && aligned && ctx->cap_max <= 2047 && count <= 65535;
   if (!fused) {
+    if (a.mode == ROWS_GENERATION) {
+      {
+        TimedLaunch tl_(ctx, KK_RANK);
+        rank_kernel<<<(a.P + 127) / 128, 128, 0, ctx->stream>>>(a.fitness_bits, a.P, ctx->d_rank, ctx->d_order);
+      }
+      SCHED_LAUNCH_CHECK(ctx);
+    }
     int rc = launch_rows(ctx, a);
     if (rc != SCHED_OK) return rc;
     return launch_cols(ctx, pop, count, first_cand, round, gen);
@@ -696,7 +741,7 @@ RowsArgs base_rows_args(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d
   a.k_max = c.k_max; a.n_max = c.n_max; a.num_elite = c.num_elite; a.count = count;
   a.thr = 0; a.gen = 0; a.first_cand = 0;
   a.key = make_key(c.seed, 0);
-  a.src = nullptr; a.dst = nullptr; a.mode = ROWS_REPAIR;
+  a.src = nullptr; a.dst = nullptr; a.mode = ROWS_REPAIR; a.fitness_bits = nullptr;
   return a;
 }
 
@@ -729,14 +774,9 @@ int launch_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_a
   const int P = ctx->cfg.population;
   int rc = ensure_dflag(ctx, P);
   if (rc != SCHED_OK) return rc;
-  {
-  TimedLaunch tl_(ctx, KK_RANK);
-  rank_kernel<<<(P + 127) / 128, 128, 0, ctx->stream>>>((const uint32_t *)d_fitness_in, P,
-                                                         ctx->d_rank, ctx->d_order);
-  }
-  SCHED_LAUNCH_CHECK(ctx);
   RowsArgs a = base_rows_args(ctx, d_k_cap, d_active, P);
   a.mode = ROWS_GENERATION; a.src = d_pop_in; a.dst = d_pop_out;
+  a.fitness_bits = (const uint32_t *)d_fitness_in;
   a.thr = ctx->cfg.thr_mutate; a.gen = generation; a.key = make_key(ctx->cfg.seed, round);
   return launch_rows_cols(ctx, a, d_pop_out, P, 0u, round, generation);
 }

@@ -30,7 +30,7 @@ __device__ __forceinline__ float ex2_approx(float x) {
 __device__ __forceinline__ float overlap_time(float tg, float ts, float gamma, float inv_gamma) {
   if (ts <= 0.f) return tg;
   const float hi = fmaxf(tg, ts), lo = fminf(tg, ts);
-  const float r = lo / hi;
+  const float r = __fdividef(lo, hi);
   const float x = ex2_approx(gamma * lg2_approx(r));
   return hi * ex2_approx(lg2_approx(1.f + x) * inv_gamma);
 }
@@ -47,31 +47,24 @@ __device__ __forceinline__ bool beats(const Best &a, const Best &b) {
 }
 
 // One warp per (job, K, class).  Lane l owns grid indices l, l+32, ... (MQ of them per
-// pass); T_grad, the overlapped time and K*m of each are held in registers while the
-// warp sweeps s.  Goodput is compared as num/den by cross-multiplication:
-//   num = M,  den = T_iter * (phi + M) / (phi + M0)   =>  num/den = THROUGHPUT * EFFICIENCY.
+// pass), held in registers while the warp sweeps s.  Goodput is kept as num/den and
+// compared by cross-multiplication:
+//   num = M = K m (s+1),  den = T_iter * (phi + M) / (phi + M0)  =>  num/den = THROUGHPUT * EFFICIENCY.
 template <int MQ>
 __global__ void __launch_bounds__(256)
 goodput_sweep_kernel(JobPtrs jp, const int32_t *__restrict__ m_grid,
-                     const int32_t *__restrict__ kfit, int J, int k_max, int n_max, int Gm, int Gs,
-                     float *__restrict__ gmax, uint16_t *__restrict__ amax) {
+                     const int32_t *__restrict__ pairs, int npairs, int k_max, int Gm, int Gs,
+                     float one, float zero, float *__restrict__ gmax, uint16_t *__restrict__ amax) {
   const int lane = threadIdx.x & 31;
-  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const long long total = (long long)J * k_max * 2;
-  if (warp >= total) return;
-  const int cls = (int)(warp & 1);
-  const int K = (int)((warp >> 1) % k_max) + 1;
-  const int j = (int)((warp >> 1) / k_max);
+  // blockIdx.x = job; the block's warps walk the list of (K, class) pairs that exist on
+  // this cluster (pairs[] = K * 2 + class, built on the host)
+  const int j = blockIdx.x;
+  const int pi = blockIdx.y * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (pi >= npairs) return;
+  const int pr = pairs[pi];
+  const int cls = pr & 1, K = pr >> 1;
   const int KD = k_max + 1;
   const size_t out = ((size_t)j * KD + K) * 2 + cls;
-
-  bool valid;
-  if (cls == 0) valid = K <= kfit[1];
-  else valid = (n_max >= 2) && (K >= 2) && (K <= kfit[min(K, n_max)]);
-  if (!valid) {
-    if (lane == 0) { gmax[out] = 0.f; amax[out] = 0xFFFFu; }
-    return;
-  }
 
   const float a_g = jp.alpha_grad[j], b_g = jp.beta_grad[j];
   const float gamma = jp.gamma[j], inv_gamma = 1.f / gamma;
@@ -88,37 +81,68 @@ goodput_sweep_kernel(JobPtrs jp, const int32_t *__restrict__ m_grid,
 
   Best best = {0.f, 1.f, 0xFFFFFFFFu};
   for (int base = 0; base < Gm; base += 32 * MQ) {
-    float tg[MQ], tov[MQ], km[MQ], mlo[MQ];
+    // Per grid point m of this lane, with u = s + 1:
+    //   T_iter = ta + u tg,  1/EFFICIENCY = c0 + u kr  (kr = K m / (phi + M0)),
+    //   goodput = K m * u / den(u),  den(u) = (ta + u tg)(c0 + u kr).
+    // den(u)/u is convex in u, so goodput is unimodal in s for a fixed m.  The loop therefore
+    // tracks, per m, the maximiser over ALL s (a chain of its own, no masking); the window
+    // M0 <= K m u <= Mmax is a contiguous range of u, and the masked maximum is at the
+    // unmasked maximiser clamped into that range.
+    float tg[MQ], ta[MQ], kr[MQ], bu[MQ], bd[MQ];
 #pragma unroll
     for (int q = 0; q < MQ; ++q) {
       const int i = base + lane + 32 * q;
-      const bool in = i < Gm;
-      const float mf = in ? (float)m_grid[(size_t)j * Gm + i] : 1.f;
+      const float mf = (i < Gm) ? (float)m_grid[(size_t)j * Gm + i] : 1.f;
       tg[q] = fmaf(b_g, mf, a_g);
-      tov[q] = overlap_time(tg[q], ts, gamma, inv_gamma);
-      km[q] = Kf * mf;
-      mlo[q] = in ? M0 : __int_as_float(0x7f800000);
+      ta[q] = overlap_time(tg[q], ts, gamma, inv_gamma) - tg[q];
+      kr[q] = Kf * mf * rinv;
+      bu[q] = 0.f;
+      bd[q] = 1.f;
     }
-    float bn = 0.f, bd = 1.f;
-    int code = -1;   // s * MQ + q of this pass's best
+    float u = 1.f;
 #pragma unroll 4
-    for (int s = 0; s < Gs; ++s) {
-      const float sf = (float)s, sp1 = (float)(s + 1);
+    for (int s = 0; s < Gs; ++s, u += 1.f) {
 #pragma unroll
       for (int q = 0; q < MQ; ++q) {
-        const float tit = fmaf(sf, tg[q], tov[q]);
-        const float M = km[q] * sp1;
-        const float den = tit * fmaf(M, rinv, c0);
-        const bool better = (M >= mlo[q]) && (M <= Mmax) && (M * bd > bn * den);
-        bn = better ? M : bn;
-        bd = better ? den : bd;
-        code = better ? s * MQ + q : code;
+        const float den = fmaf(u, tg[q], ta[q]) * fmaf(u, kr[q], c0);
+        // if (u * bd > bu * den) { bu = u; bd = den; }   -- u/den > bu/bd
+        // The conditional moves are predicated FMAs (x * 1 + 0 with run-time 1 and 0) so that
+        // they issue on the fp32 pipe; compares and selects share the half-rate integer pipe.
+        asm("{\n"
+            " .reg .pred pb;\n"
+            " .reg .f32 l, r;\n"
+            " mul.f32 l, %2, %1;\n"
+            " mul.f32 r, %0, %3;\n"
+            " setp.gt.f32 pb, l, r;\n"
+            " @pb fma.rn.f32 %0, %2, %4, %5;\n"
+            " @pb fma.rn.f32 %1, %3, %4, %5;\n"
+            "}"
+            : "+f"(bu[q]), "+f"(bd[q])
+            : "f"(u), "f"(den), "f"(one), "f"(zero));
       }
     }
-    if (code >= 0) {
+#pragma unroll
+    for (int q = 0; q < MQ; ++q) {
+      const int i = base + lane + 32 * q;
+      if (i >= Gm) continue;
+      const float km = Kf * (float)m_grid[(size_t)j * Gm + i];
+      // integer range of u with M0 <= km u <= Mmax (products are exact integers below 2^24)
+      // approximate quotients are enough: the four exact product tests below correct an
+      // off-by-one in either direction
+      const float rkm = __frcp_rn(km);
+      float ulo = ceilf(M0 * rkm), uhi = floorf(Mmax * rkm);
+      if (km * (ulo - 1.f) >= M0) ulo -= 1.f;
+      if (km * ulo < M0) ulo += 1.f;
+      if (km * (uhi + 1.f) <= Mmax) uhi += 1.f;
+      if (km * uhi > Mmax) uhi -= 1.f;
+      ulo = fmaxf(ulo, 1.f);
+      uhi = fminf(uhi, (float)Gs);
+      if (ulo > uhi) continue;
+      const float us = fminf(fmaxf(bu[q], ulo), uhi);
       Best b;
-      b.num = bn; b.den = bd;
-      b.tie = ((uint32_t)(code / MQ) << 16) | (uint32_t)(base + lane + 32 * (code % MQ));
+      b.num = km * us;
+      b.den = (us == bu[q]) ? bd[q] : fmaf(us, tg[q], ta[q]) * fmaf(us, kr[q], c0);
+      b.tie = ((uint32_t)(us - 1.f) << 16) | (uint32_t)i;
       if (beats(b, best)) best = b;
     }
   }
@@ -192,20 +216,20 @@ int launch_speedup_table(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodpu
   JobPtrs jp = {jobs->alpha_grad, jobs->beta_grad, jobs->alpha_local, jobs->beta_local,
                 jobs->alpha_node, jobs->beta_node, jobs->gamma, jobs->phi, jobs->m0,
                 jobs->m_max_total};
-  const long long warps = (long long)J * c.k_max * 2;
-  const int block = 256;
-  const long long blocks = (warps * 32 + block - 1) / block;
   const int mq = (c.grid_m + 31) / 32;
+  if (ctx->num_pairs > 0) {
+    dim3 grid((unsigned)J, (unsigned)((ctx->num_pairs + 7) / 8));
 #define SWEEP(MQ)                                                                              \
   TimedLaunch tl_(ctx, KK_SWEEP);                                                              \
-  goodput_sweep_kernel<MQ><<<(unsigned)blocks, block, 0, ctx->stream>>>(                       \
-      jp, jobs->m_grid, ctx->d_kfit, J, c.k_max, c.n_max, c.grid_m, c.grid_s, ctx->d_gmax,    \
-      ctx->d_amax)
-  if (mq <= 1) { SWEEP(1); }
-  else if (mq == 2) { SWEEP(2); }
-  else { SWEEP(4); }
+  goodput_sweep_kernel<MQ><<<grid, 256, 0, ctx->stream>>>(                                     \
+      jp, jobs->m_grid, ctx->d_pairs, ctx->num_pairs, c.k_max, c.grid_m, c.grid_s, 1.f, 0.f,   \
+      ctx->d_gmax, ctx->d_amax)
+    if (mq <= 1) { SWEEP(1); }
+    else if (mq == 2) { SWEEP(2); }
+    else { SWEEP(4); }
 #undef SWEEP
-  SCHED_LAUNCH_CHECK(ctx);
+    SCHED_LAUNCH_CHECK(ctx);
+  }
   const long long entries = (long long)J * ctx->KD * ctx->ND;
   {
   TimedLaunch tl_(ctx, KK_EXPAND);
