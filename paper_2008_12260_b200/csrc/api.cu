@@ -82,6 +82,7 @@ int ensure_round_scratch(sched_ctx *ctx) {
   if ((rc = dev_alloc(ctx, &ctx->d_tab_goodput, tab)) != SCHED_OK) return rc;
   if ((rc = dev_alloc(ctx, &ctx->d_tab_speedup, tab)) != SCHED_OK) return rc;
   if ((rc = dev_alloc(ctx, &ctx->d_rf, (size_t)c.num_jobs)) != SCHED_OK) return rc;
+  if ((rc = dev_alloc(ctx, &ctx->d_summ, (size_t)c.population * c.num_jobs)) != SCHED_OK) return rc;
   ctx->round_ready = true;
   return SCHED_OK;
 }
@@ -138,6 +139,15 @@ int ensure_colscratch(sched_ctx *ctx, size_t ints) {
     int rc = dev_alloc(ctx, &ctx->d_colsum, ints);
     if (rc != SCHED_OK) return rc;
     rc = dev_alloc(ctx, &ctx->d_colelig, ints);
+    if (rc != SCHED_OK) return rc;
+    if (ctx->d_collist) SCHED_CUDA_CHECK(ctx, cudaFree(ctx->d_collist));
+    rc = dev_alloc(ctx, &ctx->d_collist, ints);
+    if (rc != SCHED_OK) return rc;
+    if (ctx->d_occcount) SCHED_CUDA_CHECK(ctx, cudaFree(ctx->d_occcount));
+    if (ctx->d_occlist) SCHED_CUDA_CHECK(ctx, cudaFree(ctx->d_occlist));
+    rc = dev_alloc(ctx, &ctx->d_occcount, ints);
+    if (rc != SCHED_OK) return rc;
+    rc = dev_alloc(ctx, &ctx->d_occlist, ints * 8);
     if (rc != SCHED_OK) return rc;
     ctx->col_cap = ints;
   }
@@ -217,6 +227,7 @@ int sched_init(const sched_config *cfg, const int16_t *h_node_capacity, void *cu
   if ((rc = dev_alloc(ctx, &ctx->d_pen, J)) != SCHED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_status, 1)) != SCHED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_best_idx, 1)) != SCHED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_colcount, 1)) != SCHED_OK) return fail(rc);
   e = cudaMemcpyAsync(ctx->d_cap, h_node_capacity, sizeof(int16_t) * cfg->num_nodes,
                       cudaMemcpyHostToDevice, ctx->stream);
   if (e == cudaSuccess)
@@ -241,7 +252,7 @@ int sched_destroy(sched_ctx *ctx) {
   void *ptrs[] = {ctx->d_cap, ctx->d_kfit, ctx->d_pairs, ctx->d_gmax, ctx->d_amax, ctx->d_rank, ctx->d_order,
                   ctx->d_dflag, ctx->d_pen, ctx->d_partial, ctx->d_ticket, ctx->d_status,
                   ctx->d_popA, ctx->d_popB, ctx->d_fit, ctx->d_tab_goodput, ctx->d_tab_speedup,
-                  ctx->d_rf, ctx->d_best_idx, ctx->d_stage, ctx->d_stage_fit, ctx->d_colsum,
+                  ctx->d_rf, ctx->d_best_idx, ctx->d_stage, ctx->d_stage_fit, ctx->d_colsum, ctx->d_summ, ctx->d_collist, ctx->d_colcount, ctx->d_occcount, ctx->d_occlist,
                   ctx->d_colelig};
   for (void *p : ptrs)
     if (p) cudaFree(p);
@@ -275,7 +286,7 @@ int sched_num_kernel_kinds(void) { return KK_COUNT; }
 const char *sched_kernel_kind_name(int kind) {
   static const char *names[KK_COUNT] = {"goodput_sweep", "speedup_expand", "realloc_factor",
                                         "penalty_prep", "fitness", "rank", "rows", "cols",
-                                        "best_index", "copy_best"};
+                                        "best_index", "copy_best", "colscan"};
   return (kind >= 0 && kind < KK_COUNT) ? names[kind] : "";
 }
 
@@ -380,21 +391,29 @@ int schedule_round(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cu
   if (penalise && (rc = launch_realloc_factor(ctx, d_jobs, ctx->d_rf)) != SCHED_OK) return rc;
   const float *rf = penalise ? ctx->d_rf : nullptr;
   int16_t *pa = ctx->d_popA, *pb = ctx->d_popB;
-  if ((rc = launch_init_population(ctx, d_jobs->k_cap, d_jobs->active, d_cur, round, pa)) != SCHED_OK) return rc;
-  // the first fitness call of the round prepares the per-job penalty factors; the current
-  // allocation does not change within a round, so later generations reuse them
+  // While the round runs, the row/column kernels also keep per-row summaries (K, N, differs
+  // from the current allocation); the in-round fitness reads those instead of the matrices
+  // whenever the batched kernels were used, with bit-identical results.
+  ctx->round_cur = rf ? d_cur : nullptr;
+  ctx->round_summ = ctx->d_summ;
   ctx->pen_ready = false;
-  rc = launch_fitness(ctx, pa, ctx->cfg.population, ctx->d_tab_speedup, d_cur, rf, d_jobs->active,
-                      ctx->cfg.p, ctx->d_fit);
+  rc = launch_init_population(ctx, d_jobs->k_cap, d_jobs->active, d_cur, round, pa);
+  if (rc == SCHED_OK)
+    rc = launch_fitness(ctx, pa, ctx->cfg.population, ctx->d_tab_speedup, d_cur, rf, d_jobs->active,
+                        ctx->cfg.p, ctx->d_fit, ctx->summ_valid ? ctx->d_summ : nullptr);
+  // the per-job penalty factors depend only on the current allocation: prepared once
   ctx->pen_ready = (rc == SCHED_OK);
   for (int g = 0; g < generations && rc == SCHED_OK; ++g) {
     rc = launch_generation(ctx, d_jobs->k_cap, d_jobs->active, pa, ctx->d_fit, pb, round, (uint32_t)g);
     if (rc != SCHED_OK) break;
     std::swap(pa, pb);
     rc = launch_fitness(ctx, pa, ctx->cfg.population, ctx->d_tab_speedup, d_cur, rf, d_jobs->active,
-                        ctx->cfg.p, ctx->d_fit);
+                        ctx->cfg.p, ctx->d_fit, ctx->summ_valid ? ctx->d_summ : nullptr);
   }
   ctx->pen_ready = false;
+  ctx->round_cur = nullptr;
+  ctx->round_summ = nullptr;
+  ctx->summ_valid = false;
   if (rc != SCHED_OK) return rc;
   ctx->d_pop_last = pa;
   return launch_select_best(ctx, pa, ctx->d_fit, d_best, d_best_fitness);

@@ -21,7 +21,7 @@
 // kernel classes, for launch accounting and optional per-kernel timing
 enum KernelKind {
   KK_SWEEP = 0, KK_EXPAND, KK_REALLOC, KK_PENPREP, KK_FITNESS, KK_RANK, KK_ROWS, KK_COLS, KK_BEST,
-  KK_COPY, KK_COUNT
+  KK_COPY, KK_COLSCAN, KK_COUNT
 };
 
 struct TimedSpan {
@@ -51,9 +51,19 @@ struct sched_ctx {
   float *d_pen;          // [J] effective penalty factor (1 when none applies)
   double *d_partial;     // [count][chunks] partial sums of the fitness reduction
   unsigned int *d_ticket;  // [count] arrival counters of the fitness reduction
+  uint32_t *d_collist;   // [count * num_nodes] columns that need repair
+  unsigned int *d_colcount;  // [1]
+  int32_t *d_occcount;   // [count][row batches][num_nodes] occupants recorded per node
+  uint32_t *d_occlist;   // [count][row batches][num_nodes][8]
   int32_t *d_colsum, *d_colelig;  // [count][row batches][num_nodes] column partials of the row pass
   size_t partial_cap, ticket_cap, dflag_cap, col_cap;
   int cap_max;           // largest node size
+  // state of a running schedule_round: the batched row kernel also emits per-row summaries
+  // (K, N, differs-from-current) so that the in-round fitness need not re-read the population
+  const int16_t *round_cur;  // current allocation of the round (NULL outside a round)
+  uint32_t *round_summ;      // d_summ while a round runs, else NULL
+  uint32_t *d_summ;          // [P][J]
+  bool summ_valid;           // the last row/column pass filled d_summ
   bool pen_ready;        // d_pen already holds this round's factors (set by schedule_round)
   int *d_status;         // device status word
 
@@ -177,7 +187,7 @@ int launch_speedup_table(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodpu
 int launch_realloc_factor(sched_ctx *ctx, const sched_jobs *jobs, float *d_out);
 int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const float *d_speedup,
                    const int16_t *d_cur, const float *d_rf, const uint8_t *d_active, float p,
-                   float *d_fitness);
+                   float *d_fitness, const uint32_t *d_summ = nullptr);
 int launch_repair(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active, int16_t *d_pop,
                   int32_t count, uint32_t first_candidate, uint32_t round, uint32_t generation);
 int launch_init_population(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active,

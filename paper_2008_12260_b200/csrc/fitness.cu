@@ -61,6 +61,7 @@ struct FitnessArgs {
   const float *table;
   const float *pen;       // [J] factor applied to changed rows, or NULL
   const uint8_t *active;  // or NULL
+  const uint32_t *summ;   // [count][J] row summaries from the row/column kernels (SUMMARY mode)
   int J, num_nodes, k_max, n_max;
   int lpr_log2;           // lanes per row = 1 << lpr_log2
   int rows_per_block, chunks;
@@ -71,7 +72,10 @@ struct FitnessArgs {
   float *fitness;
 };
 
-template <int W>
+// SUMMARY = true: the per-row (K, N, changed) words come from `summ` instead of a pass over
+// the rows; the walk over rows, the lane that owns each row and every reduction are the same,
+// so both modes produce identical bits.
+template <int W, bool SUMMARY>
 __global__ void __launch_bounds__(256) fitness_kernel(FitnessArgs a) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int cand = blockIdx.y, chunk = blockIdx.x;
@@ -97,6 +101,14 @@ __global__ void __launch_bounds__(256) fitness_kernel(FitnessArgs a) {
   for (int jb = j0 + warp * RPW; jb < j1; jb += nwarps * RPW, ++it) {
     const int j = jb + group;
     const bool live = j < j1;
+    if (SUMMARY) {
+      if (live && sub == (it & (LPR - 1))) {
+        // summary word of the row kernel: K | N << 11 | (entries differing from current) << 22
+        const uint32_t w = a.summ[(size_t)cand * a.J + j];
+        mine = (w & 0x7FFu) | (((w >> 11) & 0x7FFu) << 16) | ((w >> 22) ? 0x80000000u : 0u);
+        myrow = j;
+      }
+    } else {
     int ksum = 0;
     uint32_t npos = 0, diff = 0;
     if (live) {
@@ -129,6 +141,7 @@ __global__ void __launch_bounds__(256) fitness_kernel(FitnessArgs a) {
       // K <= 32*2047 < 2^16, N likewise; keep "changed" in the top bit of the N field
       mine = (packed & 0x7FFFFFFFu) | (changed ? 0x80000000u : 0u);
       myrow = j;
+    }
     }
     const bool flush = ((it + 1) % slots_per_fill == 0) || (jb + nwarps * RPW >= j1);
     if (flush) {
@@ -237,7 +250,7 @@ void fitness_geometry(size_t row_bytes, uintptr_t align_bits, int J, int count, 
 
 int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const float *d_speedup,
                    const int16_t *d_cur, const float *d_rf, const uint8_t *d_active, float p,
-                   float *d_fitness) {
+                   float *d_fitness, const uint32_t *d_summ) {
   const sched_config &c = ctx->cfg;
   const int J = c.num_jobs;
   if (count == 0) return SCHED_OK;
@@ -264,6 +277,7 @@ int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const fl
   a.table = d_speedup;
   a.pen = penalise ? ctx->d_pen : nullptr;
   a.active = d_active;
+  a.summ = d_summ;
   a.J = J; a.num_nodes = c.num_nodes; a.k_max = c.k_max; a.n_max = c.n_max;
   a.lpr_log2 = lpr_log2;
   a.rows_per_block = rows_per_block; a.chunks = chunks;
@@ -282,14 +296,18 @@ int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const fl
     b.partial = ctx->d_partial + (size_t)first * chunks * 2;
     b.ticket = ctx->d_ticket + first;
     b.fitness = d_fitness + first;
+    if (d_summ) b.summ = d_summ + (size_t)first * J;
     dim3 grid((unsigned)chunks, (unsigned)n);
     {
     TimedLaunch tl_(ctx, KK_FITNESS);
     switch (W) {
-      case 16: fitness_kernel<16><<<grid, 256, 0, ctx->stream>>>(b); break;
-      case 8: fitness_kernel<8><<<grid, 256, 0, ctx->stream>>>(b); break;
-      case 4: fitness_kernel<4><<<grid, 256, 0, ctx->stream>>>(b); break;
-      default: fitness_kernel<2><<<grid, 256, 0, ctx->stream>>>(b); break;
+      case 16:
+        if (d_summ) fitness_kernel<16, true><<<grid, 256, 0, ctx->stream>>>(b);
+        else fitness_kernel<16, false><<<grid, 256, 0, ctx->stream>>>(b);
+        break;
+      case 8: fitness_kernel<8, false><<<grid, 256, 0, ctx->stream>>>(b); break;
+      case 4: fitness_kernel<4, false><<<grid, 256, 0, ctx->stream>>>(b); break;
+      default: fitness_kernel<2, false><<<grid, 256, 0, ctx->stream>>>(b); break;
     }
     }
     SCHED_LAUNCH_CHECK(ctx);
@@ -401,6 +419,7 @@ int eval_fitness_noalloc(const int16_t *d_pop, int32_t count, int32_t num_jobs, 
   a.table = d_speedup;
   a.pen = penalise ? scratch->pen : nullptr;
   a.active = d_active;
+  a.summ = nullptr;
   a.J = J; a.num_nodes = num_nodes; a.k_max = k_max; a.n_max = n_max;
   a.lpr_log2 = lpr_log2;
   a.rows_per_block = rows_per_block; a.chunks = chunks;
@@ -412,10 +431,10 @@ int eval_fitness_noalloc(const int16_t *d_pop, int32_t count, int32_t num_jobs, 
   a.fitness = d_fitness;
   dim3 grid((unsigned)chunks, (unsigned)count);
   switch (W) {
-    case 16: fitness_kernel<16><<<grid, 256, 0, stream>>>(a); break;
-    case 8: fitness_kernel<8><<<grid, 256, 0, stream>>>(a); break;
-    case 4: fitness_kernel<4><<<grid, 256, 0, stream>>>(a); break;
-    default: fitness_kernel<2><<<grid, 256, 0, stream>>>(a); break;
+    case 16: fitness_kernel<16, false><<<grid, 256, 0, stream>>>(a); break;
+    case 8: fitness_kernel<8, false><<<grid, 256, 0, stream>>>(a); break;
+    case 4: fitness_kernel<4, false><<<grid, 256, 0, stream>>>(a); break;
+    default: fitness_kernel<2, false><<<grid, 256, 0, stream>>>(a); break;
   }
   e = cudaGetLastError();
   if (e != cudaSuccess) return noalloc_fail(SCHED_ERR_CUDA, "fitness_kernel launch", e);

@@ -48,6 +48,8 @@ struct RowsArgs {
   const int32_t *order;     // [P]
   const uint32_t *fitness_bits;  // [P] parents' fitness (generation mode)
   uint8_t *dflag;           // [count][J]
+  const int16_t *cur;       // [J][N] current allocation for the summaries' "changed" bit, or NULL
+  uint32_t *summ;           // [count][J] row summaries (batched kernels only), or NULL
   int mode, P, J, num_nodes, k_max, n_max, num_elite, count;
   uint32_t thr, gen, first_cand;
   RngKey key;
@@ -315,11 +317,18 @@ __global__ void copy_best_kernel(const int16_t *__restrict__ pop, const int32_t 
 // columns, the GPUs placed and the number of distributed jobs; the block's column partials
 // go to scratch, so the column pass never re-reads the population.
 // ---------------------------------------------------------------------------------------
+// Occupants of a node recorded per (candidate, row batch, node); a node with more occupants in
+// one batch than this falls back to scanning the column.
+constexpr int OCC_SLOTS = 8;
+
 struct Rows2Args {
   RowsArgs r;
   int32_t *colsum;   // [count][nbatch][num_nodes] GPUs placed on the node by the batch's rows
   int32_t *colelig;  // same shape: rows of the batch that are distributed and occupy the node
-  int nbatch;
+  unsigned int *list_count;  // length of the column work list, reset here for the column pass
+  int32_t *occ_count;        // [count][nbatch][num_nodes] rows of the batch that occupy the node
+  uint32_t *occ_list;        // [count][nbatch][num_nodes][OCC_SLOTS] job | GPUs << 20 | distributed << 31
+  int nbatch, lpr_log2;
 };
 
 __device__ __forceinline__ uint4 clamp_vec(uint4 x, uint4 cp) {
@@ -332,32 +341,49 @@ __device__ __forceinline__ uint4 clamp_vec(uint4 x, uint4 cp) {
 
 // K in the low 22 bits, occupied-node count in the high 10 (entries are >= 0 here)
 __device__ __forceinline__ uint32_t row_partial(uint4 x) {
-  const uint32_t k = (x.x & 0xFFFFu) + (x.x >> 16) + (x.y & 0xFFFFu) + (x.y >> 16) +
-                     (x.z & 0xFFFFu) + (x.z >> 16) + (x.w & 0xFFFFu) + (x.w >> 16);
+  int k = __dp2a_lo((int)x.x, 0x0101, 0);
+  k = __dp2a_lo((int)x.y, 0x0101, k);
+  k = __dp2a_lo((int)x.z, 0x0101, k);
+  k = __dp2a_lo((int)x.w, 0x0101, k);
   const uint32_t o = __vimin_s16x2_relu(x.x, 0x00010001u) + __vimin_s16x2_relu(x.y, 0x00010001u) +
                      __vimin_s16x2_relu(x.z, 0x00010001u) + __vimin_s16x2_relu(x.w, 0x00010001u);
-  return k | (((o & 0xFFFFu) + (o >> 16)) << 22);
+  return (uint32_t)k | (((o & 0xFFFFu) + (o >> 16)) << 22);
 }
 
-template <int VPL>
-__global__ void __launch_bounds__(256) rows2_kernel(Rows2Args aa) {
+// VPL = 16-byte vectors per lane; a row is split over LPR = 1 << LPR_LOG2 lanes
+// (LPR * VPL >= row_vecs, FULL when equal), so a warp works on 32 / LPR rows at a time.
+template <int LPR_LOG2, int VPL, bool FULL>
+__global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
   const RowsArgs &a = aa.r;
-  __shared__ __align__(16) int16_t s_row[8][256 * VPL];   // per-warp detour buffer
-  __shared__ int32_t s_tot[256 * VPL], s_el[256 * VPL];
+  constexpr int MAXN = 8 * (1 << LPR_LOG2) * VPL;   // nodes this instantiation can hold
+  constexpr int QCAP = 64;                          // vectors in a warp's occupant queue
+  __shared__ __align__(16) int16_t s_row[8][MAXN];  // per-warp detour buffer
+  __shared__ __align__(16) int16_t s_cap[MAXN];     // node sizes floored at 0
+  __shared__ int32_t s_tot[MAXN], s_el[MAXN], s_cnt[MAXN];
+  __shared__ uint32_t s_occ[MAXN * OCC_SLOTS];
+  __shared__ int s_parent[2];
+  __shared__ int s_rank4[4];
+  // per-warp queue of non-empty vectors waiting to be expanded into occupants
+  __shared__ __align__(16) uint4 s_qvec[8][QCAP];
+  __shared__ uint32_t s_qmeta[8][QCAP];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int cl = blockIdx.y, batch = blockIdx.x;
   const uint32_t c = a.first_cand + (uint32_t)cl;
   const int NN = a.num_nodes, J = a.J;
   const int row_vecs = NN >> 3;
-  for (int i = threadIdx.x; i < NN; i += blockDim.x) { s_tot[i] = 0; s_el[i] = 0; }
-  __syncthreads();
+  constexpr int LPR = 1 << LPR_LOG2, RPI = 32 >> LPR_LOG2;        // lanes per row, rows per iteration
+  const int grp = lane >> LPR_LOG2, sub = lane & (LPR - 1);
+  const unsigned gmask = (LPR == 32) ? 0xffffffffu : (((1u << LPR) - 1u) << (grp * LPR));
+  for (int i = threadIdx.x; i < NN; i += blockDim.x) {
+    s_tot[i] = 0; s_el[i] = 0; s_cnt[i] = 0;
+    s_cap[i] = (int16_t)max((int)a.cap[i], 0);
+  }
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *aa.list_count = 0u;
 
   // ---- parents of this candidate (generation mode), found by the block itself -------------
   // rank(i) = number of candidates ordered before i (fitness descending, index ascending).
   // An elite child needs the candidate of rank c; any other child the better-ranked of two
   // random pairs, i.e. the ranks of four candidates only.
-  __shared__ int s_parent[2];
-  __shared__ int s_rank4[4];
   if (a.mode == ROWS_GENERATION) {
     const int P = a.P;
     if ((int)c < a.num_elite) {
@@ -396,22 +422,19 @@ __global__ void __launch_bounds__(256) rows2_kernel(Rows2Args aa) {
 
   const int j0 = batch * 256 + warp * 32;
   const int nrows = min(32, J - j0);          // may be <= 0 for trailing warps
-  // ---- per-lane set-up for row j0 + lane -------------------------------------------------
-  int parent_l = 0;
-  uint32_t flags_l = 0;                       // bit 0 perturb, bit 1 active, bits 2.. replica cap
+  // ---- per-lane set-up for row j0 + lane: 32 draws side by side -----------------------------
+  uint32_t flags_l = 0;   // bit 0 perturb, bit 1 active, bit 2 row comes from the second parent, bits 3.. replica cap
   u32x4 mw = {0, 0, 0, 0};
   if (lane < nrows) {
     const int j = j0 + lane;
     const bool act = !a.active || a.active[j];
     int kc = a.k_cap ? a.k_cap[j] : a.k_max;
     kc = max(0, min(kc, a.k_max));
-    bool mut = false;
+    bool mut = false, second = false;
     if (a.mode == ROWS_GENERATION) {
-      if ((int)c < a.num_elite) {
-        parent_l = s_parent[0];
-      } else {
+      if ((int)c >= a.num_elite) {
         const u32x4 x = draw(a.key, (uint32_t)j, c, a.gen, SLOT_XOVER);
-        parent_l = (x.x >> 31) ? s_parent[1] : s_parent[0];
+        second = (x.x >> 31) != 0u;
         mw = draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE);
         mut = mw.x < a.thr;
       }
@@ -419,88 +442,125 @@ __global__ void __launch_bounds__(256) rows2_kernel(Rows2Args aa) {
       mw = draw(a.key, (uint32_t)j, c, GEN_INIT, SLOT_INIT);
       mut = mw.x < a.thr;
     }
-    flags_l = (mut ? 1u : 0u) | (act ? 2u : 0u) | ((uint32_t)kc << 2);
+    flags_l = (mut ? 1u : 0u) | (act ? 2u : 0u) | (second ? 4u : 0u) | ((uint32_t)kc << 3);
   }
-  // node sizes of this lane's columns, floored at 0
-  uint4 capv[VPL];
-#pragma unroll
-  for (int q = 0; q < VPL; ++q) {
-    const int v = lane + 32 * q;
-    capv[q] = make_uint4(0, 0, 0, 0);
-    if (v < row_vecs) {
-      const uint4 t = __ldg((const uint4 *)a.cap + v);
-      capv[q] = make_uint4(__vimax_s16x2_relu(t.x, 0u), __vimax_s16x2_relu(t.y, 0u),
-                           __vimax_s16x2_relu(t.z, 0u), __vimax_s16x2_relu(t.w, 0u));
-    }
+
+  // row j0 of the possible sources; per row only the offset r * NN is added
+  const size_t roff0 = (size_t)j0 * NN;
+  const int16_t *src_a = nullptr, *src_b = nullptr;
+  if (a.mode == ROWS_GENERATION) {
+    src_a = a.src + (size_t)s_parent[0] * J * NN + roff0;
+    src_b = a.src + (size_t)s_parent[1] * J * NN + roff0;
+  } else if (a.mode == ROWS_INIT) {
+    src_a = src_b = a.src ? a.src + roff0 : nullptr;
+  } else {
+    src_a = src_b = a.dst + (size_t)cl * J * NN + roff0;
   }
-  uint4 tot[VPL], el[VPL];
-#pragma unroll
-  for (int q = 0; q < VPL; ++q) { tot[q] = make_uint4(0, 0, 0, 0); el[q] = make_uint4(0, 0, 0, 0); }
+  const int16_t *cur0 = a.cur ? a.cur + roff0 : nullptr;
+  int16_t *dst0 = a.dst + (size_t)cl * J * NN + roff0;
   int16_t *row = s_row[warp];
 
-  for (int r = 0; r < nrows; ++r) {
-    const int j = j0 + r;
-    const int parent = __shfl_sync(0xffffffffu, parent_l, r);
-    const uint32_t flags = __shfl_sync(0xffffffffu, flags_l, r);
-    int16_t *out = a.dst + ((size_t)cl * J + j) * NN;
-    if (!(flags & 2u)) {                      // inactive job: empty row
-#pragma unroll
-      for (int q = 0; q < VPL; ++q)
-        if (lane + 32 * q < row_vecs) ((uint4 *)out)[lane + 32 * q] = make_uint4(0, 0, 0, 0);
-      if (lane == 0) a.dflag[(size_t)cl * J + j] = 0;
-      continue;
-    }
-    const int16_t *src;
-    if (a.mode == ROWS_GENERATION) src = a.src + ((size_t)parent * J + j) * NN;
-    else if (a.mode == ROWS_INIT) src = a.src ? a.src + (size_t)j * NN : nullptr;
-    else src = out;
-    uint4 x[VPL];
-    uint32_t part = 0;
+  // Iterations are software-pipelined: the loads of the next RPI rows are issued before the
+  // current ones are processed.
+  uint4 raw[VPL];
+  auto fetch = [&](int r) {   // r = this lane's row within the warp's 32 (may be >= nrows)
+    const uint32_t fl = __shfl_sync(0xffffffffu, flags_l, r & 31);
+    const int16_t *src = (fl & 4u) ? src_b : src_a;
+    const bool on = r < nrows && (fl & 2u) && src;
 #pragma unroll
     for (int q = 0; q < VPL; ++q) {
-      const int v = lane + 32 * q;
-      x[q] = make_uint4(0, 0, 0, 0);
-      if (src && v < row_vecs) x[q] = clamp_vec(__ldg((const uint4 *)src + v), capv[q]);
-      part += row_partial(x[q]);
+      const int v = sub + LPR * q;
+      raw[q] = make_uint4(0, 0, 0, 0);
+      if (on && (FULL || v < row_vecs)) raw[q] = __ldg((const uint4 *)(src + (size_t)r * NN) + v);
     }
+  };
+  if (nrows > 0) fetch(grp);
+  // Expands the queued vectors: entry e = (vector e / 8, half e % 8), one lane per entry.  Per
+  // occupant: add to the node's GPU total and distributed-job count, record it in the
+  // node's occupant list.
+  auto flush_queue = [&](int count) {
+    __syncwarp();
+    for (int e = lane; e < count * 8; e += 32) {
+      const uint32_t val = ((const uint16_t *)s_qvec[warp])[e];
+      if (val) {
+        const uint32_t meta = s_qmeta[warp][e >> 3];
+        const int n = (int)((meta >> 20) & 0x7FFu) * 8 + (e & 7);
+        atomicAdd(&s_tot[n], (int)val);
+        if (meta >> 31) atomicAdd(&s_el[n], 1);
+        const int slot = atomicAdd(&s_cnt[n], 1);
+        if (slot < OCC_SLOTS) s_occ[n * OCC_SLOTS + slot] = (meta & 0xFFFFFu) | (val << 20) | (meta & 0x80000000u);
+      }
+    }
+    __syncwarp();
+  };
+
+  for (int r0 = 0; r0 < nrows; r0 += RPI) {
+    const int r = r0 + grp;                       // this lane's row
+    const bool live = r < nrows;
+    const uint32_t flags = __shfl_sync(0xffffffffu, flags_l, r & 31);
+    const bool act = live && (flags & 2u);
+    uint4 x[VPL];
 #pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+    for (int q = 0; q < VPL; ++q) {
+      const int v = sub + LPR * q;
+      x[q] = make_uint4(0, 0, 0, 0);
+      if (FULL || v < row_vecs) x[q] = clamp_vec(raw[q], ((const uint4 *)s_cap)[v]);
+    }
+    if (r0 + RPI < nrows) fetch(r0 + RPI + grp);
+
+    uint32_t part = 0;
+#pragma unroll
+    for (int q = 0; q < VPL; ++q) part += row_partial(x[q]);
+    part = __reduce_add_sync(gmask, part);
     int K = (int)(part & 0x3FFFFFu), N = (int)(part >> 22);
-    const int kc = (int)(flags >> 2);
-    if ((flags & 1u) || K > kc || N > a.n_max) {
-      // detour: row into shared memory, perturb, apply the row caps, read it back
+    const int kc = (int)(flags >> 3);
+
+    // rows that are perturbed or break a row cap take a detour through shared memory, one
+    // row at a time with the whole warp
+    unsigned need = __ballot_sync(0xffffffffu, act && sub == 0 && ((flags & 1u) || K > kc || N > a.n_max));
+    while (need) {
+      const int leader = __ffs(need) - 1;         // lane `leader` is sub 0 of the row's group
+      need &= need - 1;
+      const int g = leader >> LPR_LOG2;
+      const int rr = r0 + g;
+      const uint32_t rflags = __shfl_sync(0xffffffffu, flags, leader);
+      int rK = __shfl_sync(0xffffffffu, K, leader), rN = __shfl_sync(0xffffffffu, N, leader);
+      const int rkc = (int)(rflags >> 3);
+      if (grp == g) {
 #pragma unroll
-      for (int q = 0; q < VPL; ++q)
-        if (lane + 32 * q < row_vecs) ((uint4 *)row)[lane + 32 * q] = x[q];
+        for (int q = 0; q < VPL; ++q)
+          if (FULL || sub + LPR * q < row_vecs) ((uint4 *)row)[sub + LPR * q] = x[q];
+      }
       __syncwarp();
-      if (flags & 1u) {
-        const uint32_t m1 = __shfl_sync(0xffffffffu, mw.y, r), m2 = __shfl_sync(0xffffffffu, mw.z, r),
-                       m3 = __shfl_sync(0xffffffffu, mw.w, r);
+      if (rflags & 1u) {
+        const uint32_t m1 = __shfl_sync(0xffffffffu, mw.y, rr), m2 = __shfl_sync(0xffffffffu, mw.z, rr),
+                       m3 = __shfl_sync(0xffffffffu, mw.w, rr);
         const uint32_t op = bounded(m1, 3u);
         if (op == 0u) {
           const int n = (int)bounded(m3, (uint32_t)NN);
-          if (lane == 0) row[n] = (int16_t)min((int)row[n] + 1, max((int)a.cap[n], 0));
-        } else if (N > 0) {
-          const int ns = nth_occupied(row, NN, bounded(m2, (uint32_t)N), lane);
+          if (lane == 0) row[n] = (int16_t)min((int)row[n] + 1, (int)s_cap[n]);
+        } else if (rN > 0) {
+          const int ns = nth_occupied(row, NN, bounded(m2, (uint32_t)rN), lane);
           if (op == 1u) {
             if (lane == 0) row[ns] = (int16_t)(row[ns] - 1);
           } else {
             const int nd = (int)bounded(m3, (uint32_t)NN);
             if (nd != ns && lane == 0) {
-              row[nd] = (int16_t)min((int)row[nd] + (int)row[ns], max((int)a.cap[nd], 0));
+              row[nd] = (int16_t)min((int)row[nd] + (int)row[ns], (int)s_cap[nd]);
               row[ns] = 0;
             }
           }
         }
         __syncwarp();
-        K = 0; N = 0;
-        for (int n = lane; n < NN; n += 32) { K += row[n]; N += row[n] > 0; }
-        K = warp_sum(K);
-        N = warp_sum(N);
+        rK = 0; rN = 0;
+        for (int n = lane; n < NN; n += 32) { rK += row[n]; rN += row[n] > 0; }
+        rK = __reduce_add_sync(0xffffffffu, rK);
+        rN = __reduce_add_sync(0xffffffffu, rN);
       }
-      if (K > kc || N > a.n_max) {
+      if (rK > rkc || rN > a.n_max) {
         if (lane == 0) {
-          int excess = K - kc;
+          int excess = rK - rkc;
+          rK = min(rK, rkc);
           for (int n = NN - 1; n >= 0 && excess > 0; --n) {
             const int take = min((int)row[n], excess);
             row[n] = (int16_t)(row[n] - take);
@@ -510,56 +570,79 @@ __global__ void __launch_bounds__(256) rows2_kernel(Rows2Args aa) {
           for (int n = 0; n < NN; ++n) {
             if (row[n] > 0) {
               ++occ;
-              if (occ > a.n_max) row[n] = 0;
+              if (occ > a.n_max) { rK -= row[n]; row[n] = 0; }
             }
           }
-          N = min(occ, a.n_max);
+          rN = min(occ, a.n_max);
         }
-        N = __shfl_sync(0xffffffffu, N, 0);
+        rN = __shfl_sync(0xffffffffu, rN, 0);
+        rK = __shfl_sync(0xffffffffu, rK, 0);
       }
       __syncwarp();
+      if (grp == g) {
 #pragma unroll
-      for (int q = 0; q < VPL; ++q)
-        if (lane + 32 * q < row_vecs) x[q] = ((const uint4 *)row)[lane + 32 * q];
+        for (int q = 0; q < VPL; ++q)
+          if (FULL || sub + LPR * q < row_vecs) x[q] = ((const uint4 *)row)[sub + LPR * q];
+        K = rK;
+        N = rN;
+      }
       __syncwarp();
     }
+
+    // ---- store, column bookkeeping, row summary ---------------------------------------------
     const bool dist = N >= 2;
+    int ndiff = 0;   // entries of this lane that differ from the current allocation
+    int qn = 0;      // vectors queued by the warp in this iteration
+    const int j = j0 + r;
 #pragma unroll
     for (int q = 0; q < VPL; ++q) {
-      if (lane + 32 * q < row_vecs) ((uint4 *)out)[lane + 32 * q] = x[q];
-      tot[q].x += x[q].x; tot[q].y += x[q].y; tot[q].z += x[q].z; tot[q].w += x[q].w;
-      if (dist) {
-        el[q].x += __vimin_s16x2_relu(x[q].x, 0x00010001u);
-        el[q].y += __vimin_s16x2_relu(x[q].y, 0x00010001u);
-        el[q].z += __vimin_s16x2_relu(x[q].z, 0x00010001u);
-        el[q].w += __vimin_s16x2_relu(x[q].w, 0x00010001u);
+      const int v = sub + LPR * q;
+      const bool in = live && (FULL || v < row_vecs);
+      if (in) ((uint4 *)(dst0 + (size_t)r * NN))[v] = x[q];
+      // Occupied nodes are few.  Vectors with any occupant are compacted into a per-warp
+      // queue (ballot + popc, no atomics) and expanded below with one lane per entry.
+      if (qn > QCAP - 32) { flush_queue(qn); qn = 0; }
+      const bool nz = in && (x[q].x | x[q].y | x[q].z | x[q].w) != 0u;
+      const unsigned bal = __ballot_sync(0xffffffffu, nz);
+      if (nz) {
+        const int pos = qn + __popc(bal & ((1u << lane) - 1u));
+        s_qvec[warp][pos] = x[q];
+        s_qmeta[warp][pos] = (uint32_t)j | ((uint32_t)v << 20) | (dist ? 0x80000000u : 0u);   // v < 64
+      }
+      qn += __popc(bal);
+      if (cur0 && in) {
+        const uint4 cx = __ldg((const uint4 *)(cur0 + (size_t)r * NN) + v);
+        const uint4 d = make_uint4(x[q].x ^ cx.x, x[q].y ^ cx.y, x[q].z ^ cx.z, x[q].w ^ cx.w);
+        if ((d.x | d.y | d.z | d.w) != 0u) {
+          // entries on both sides are in [0, 32767], so each half of the xor is a non-negative
+          // int16 and min(half, 1) counts the halves that differ
+          const uint32_t dc = __vimin_s16x2_relu(d.x, 0x00010001u) + __vimin_s16x2_relu(d.y, 0x00010001u) +
+                              __vimin_s16x2_relu(d.z, 0x00010001u) + __vimin_s16x2_relu(d.w, 0x00010001u);
+          ndiff += (int)((dc & 0xFFFFu) + (dc >> 16));
+        }
       }
     }
-    if (lane == 0) a.dflag[(size_t)cl * J + j] = dist ? 1 : 0;
+    flush_queue(qn);
+    qn = 0;
+    if (cur0) ndiff = __reduce_add_sync(gmask, ndiff);
+    if (live && sub == 0) {
+      const bool on = (flags & 2u) != 0u;
+      a.dflag[(size_t)cl * J + j] = (on && dist) ? 1 : 0;
+      // row summary for the fitness: K | N << 11 | (entries that differ from current) << 22
+      if (a.summ)
+        a.summ[(size_t)cl * J + j] = on ? ((uint32_t)K | ((uint32_t)N << 11) | ((uint32_t)ndiff << 22)) : 0u;
+    }
   }
 
-  // ---- column partials of the block --------------------------------------------------------
-#pragma unroll
-  for (int q = 0; q < VPL; ++q) {
-    const int v = lane + 32 * q;
-    if (v < row_vecs) {
-      const uint32_t t[4] = {tot[q].x, tot[q].y, tot[q].z, tot[q].w};
-      const uint32_t e[4] = {el[q].x, el[q].y, el[q].z, el[q].w};
-#pragma unroll
-      for (int w = 0; w < 4; ++w) {
-        const int n = v * 8 + w * 2;
-        if (t[w] & 0xFFFFu) atomicAdd(&s_tot[n], (int)(t[w] & 0xFFFFu));
-        if (t[w] >> 16) atomicAdd(&s_tot[n + 1], (int)(t[w] >> 16));
-        if (e[w] & 0xFFFFu) atomicAdd(&s_el[n], (int)(e[w] & 0xFFFFu));
-        if (e[w] >> 16) atomicAdd(&s_el[n + 1], (int)(e[w] >> 16));
-      }
-    }
-  }
+  // ---- column partials and occupant lists of the block -------------------------------------
   __syncthreads();
   const size_t base = ((size_t)cl * aa.nbatch + batch) * NN;
   for (int i = threadIdx.x; i < NN; i += blockDim.x) {
     aa.colsum[base + i] = s_tot[i];
     aa.colelig[base + i] = s_el[i];
+    aa.occ_count[base + i] = s_cnt[i];
+    const int cnt = min(s_cnt[i], OCC_SLOTS);
+    for (int k = 0; k < cnt; ++k) aa.occ_list[(base + i) * OCC_SLOTS + k] = s_occ[i * OCC_SLOTS + k];
   }
 }
 
@@ -568,46 +651,61 @@ struct ColfixArgs {
   const uint8_t *dflag;
   const int16_t *cap;
   const int32_t *colsum, *colelig;
+  uint32_t *summ;           // [count][J] row summaries to keep in step with the removals, or NULL
+  const int16_t *cur;       // current allocation (for the summaries' differing-entries count), or NULL
+  const int32_t *occ_count; // per (candidate, row batch, node) occupants recorded by the row kernel
+  const uint32_t *occ_list;
+  uint32_t *list;           // work list of (candidate << 13 | node) entries
+  unsigned int *list_count;
   int J, num_nodes, nbatch;
   uint32_t gen, first_cand;
   RngKey key;
 };
 
-// Column pass on the batch partials: a thread per (candidate, node) adds them up; columns
-// that hold two distributed jobs or exceed the node size are then repaired by the whole
-// warp, one column at a time (same rules as cols_kernel).
-__global__ void __launch_bounds__(128) colfix_kernel(ColfixArgs a) {
-  const int lane = threadIdx.x & 31;
-  const int n = blockIdx.x * blockDim.x + threadIdx.x;
-  const int cl = blockIdx.y;
+// A column-pass write A[j][n]: v_old -> v_new keeps row j's summary in step:
+// K += v_new - v_old, N -= 1 if the entry became empty, and the count of entries that
+// differ from the current allocation is adjusted.  The three fields never leave their
+// ranges, so one wrapped 32-bit add does all three.
+__device__ __forceinline__ void summ_update(const ColfixArgs &a, int cl, int j, int n, int v_old, int v_new) {
+  if (!a.summ) return;
+  int d_diff = 0;
+  if (a.cur) {
+    const int cv = a.cur[(size_t)j * a.num_nodes + n];
+    d_diff = (int)(v_new != cv) - (int)(v_old != cv);
+  }
+  const uint32_t delta = (uint32_t)(v_new - v_old) + ((uint32_t)((v_new == 0 && v_old > 0) ? -1 : 0) << 11) +
+                         ((uint32_t)d_diff << 22);
+  atomicAdd(a.summ + (size_t)cl * a.J + j, delta);
+}
+
+// Repair of one column by a whole warp (any J): interference, then capacity, each with a
+// few passes over the column; loads are issued in batches so that they overlap.
+__device__ __noinline__ void repair_column_any(const ColfixArgs &a, int cl, int nn, int tot, int ne, int cap_n, int lane) {
   const uint32_t c = a.first_cand + (uint32_t)cl;
   const int J = a.J, NN = a.num_nodes;
-  int total = 0, nelig = 0, cp = 0;
-  if (n < NN) {
-    for (int b = 0; b < a.nbatch; ++b) {
-      total += a.colsum[((size_t)cl * a.nbatch + b) * NN + n];
-      nelig += a.colelig[((size_t)cl * a.nbatch + b) * NN + n];
-    }
-    cp = max((int)a.cap[n], 0);
-  }
-  unsigned todo = __ballot_sync(0xffffffffu, n < NN && (nelig >= 2 || total > cp));
   const uint8_t *df = a.dflag + (size_t)cl * J;
-  while (todo) {
-    const int src = __ffs(todo) - 1;
-    todo &= todo - 1;
-    const int nn = __shfl_sync(0xffffffffu, n, src);
-    int tot = __shfl_sync(0xffffffffu, total, src);
-    const int ne = __shfl_sync(0xffffffffu, nelig, src);
-    const int cap_n = __shfl_sync(0xffffffffu, cp, src);
+  {
     int16_t *col = a.pop + (size_t)cl * J * NN + nn;
+    // the loops below first issue a batch of independent column loads, then work on them
+    constexpr int U = 8;
     if (ne >= 2) {
       const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
       int best = J;
-      for (int j = lane; j < J; j += 32) {
-        if (df[j] && col[(size_t)j * NN] > 0) {
-          int t = j - o;
-          if (t < 0) t += J;
-          best = min(best, t);
+      for (int jb = 0; jb < J; jb += 32 * U) {
+        int v[U], d[U];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+          const int j = jb + 32 * k + lane;
+          v[k] = (j < J) ? (int)col[(size_t)j * NN] : 0;
+          d[k] = (j < J) ? (int)df[j] : 0;
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+          if (d[k] && v[k] > 0) {
+            int t = jb + 32 * k + lane - o;
+            if (t < 0) t += J;
+            best = min(best, t);
+          }
         }
       }
 #pragma unroll
@@ -615,10 +713,22 @@ __global__ void __launch_bounds__(128) colfix_kernel(ColfixArgs a) {
       int keep = o + best;
       if (keep >= J) keep -= J;
       int removed = 0;
-      for (int j = lane; j < J; j += 32) {
-        if (j != keep && df[j]) {
-          const int v = col[(size_t)j * NN];
-          if (v > 0) { col[(size_t)j * NN] = 0; removed += v; }
+      for (int jb = 0; jb < J; jb += 32 * U) {
+        int v[U], d[U];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+          const int j = jb + 32 * k + lane;
+          v[k] = (j < J) ? (int)col[(size_t)j * NN] : 0;
+          d[k] = (j < J) ? (int)df[j] : 0;
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+          const int j = jb + 32 * k + lane;
+          if (d[k] && v[k] > 0 && j != keep) {
+            col[(size_t)j * NN] = 0;
+            removed += v[k];
+            summ_update(a, cl, j, nn, v[k], 0);
+          }
         }
       }
       tot -= warp_sum(removed);
@@ -626,22 +736,135 @@ __global__ void __launch_bounds__(128) colfix_kernel(ColfixArgs a) {
     int excess = tot - cap_n;
     if (excess > 0) {
       const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J);
-      for (int t0 = 0; t0 < J && excess > 0; t0 += 32) {
-        const int t = t0 + lane;
-        int j = o + t;
-        if (j >= J) j -= J;
-        const int v = (t < J) ? (int)col[(size_t)j * NN] : 0;
-        int s = v;                                   // inclusive prefix over the 32 jobs
+      constexpr int C = 4;   // chunks of 32 jobs loaded together
+      for (int t0 = 0; t0 < J && excess > 0; t0 += 32 * C) {
+        int v[C], jj[C];
 #pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-          const int u = __shfl_up_sync(0xffffffffu, s, off);
-          if (lane >= off) s += u;
+        for (int k = 0; k < C; ++k) {
+          const int t = t0 + 32 * k + lane;
+          int j = o + t;
+          if (j >= J) j -= J;
+          jj[k] = j;
+          v[k] = (t < J) ? (int)col[(size_t)j * NN] : 0;
         }
-        const int take = min(v, max(excess - (s - v), 0));
-        if (take > 0) col[(size_t)j * NN] = (int16_t)(v - take);
-        excess -= __shfl_sync(0xffffffffu, s, 31);
+#pragma unroll
+        for (int k = 0; k < C; ++k) {
+          if (excess <= 0) break;
+          int s = v[k];                                // inclusive prefix over the 32 jobs
+#pragma unroll
+          for (int off = 1; off < 32; off <<= 1) {
+            const int u = __shfl_up_sync(0xffffffffu, s, off);
+            if (lane >= off) s += u;
+          }
+          const int take = min(v[k], max(excess - (s - v[k]), 0));
+          if (take > 0) {
+            col[(size_t)jj[k] * NN] = (int16_t)(v[k] - take);
+            summ_update(a, cl, jj[k], nn, v[k], v[k] - take);
+          }
+          excess -= __shfl_sync(0xffffffffu, s, 31);
+        }
       }
     }
+  }
+}
+
+// Repair of one column from the occupant lists of the row kernel: one occupant per lane, no
+// pass over the column.  Falls back to the column scan when a batch overflowed its slots
+// or the node has more than 32 occupants.
+__device__ void repair_column_list(const ColfixArgs &a, int cl, int nn, int tot, int ne, int cap_n, int lane) {
+  const uint32_t c = a.first_cand + (uint32_t)cl;
+  const int J = a.J, NN = a.num_nodes;
+  uint32_t entry = 0;
+  int have_n = 0;
+  bool overflow = false;
+  for (int b = 0; b < a.nbatch; ++b) {
+    const size_t at = ((size_t)cl * a.nbatch + b) * NN + nn;
+    const int cb = a.occ_count[at];
+    overflow |= cb > OCC_SLOTS;
+    const int take_n = min(cb, OCC_SLOTS);
+    if (lane >= have_n && lane < have_n + take_n) entry = a.occ_list[at * OCC_SLOTS + (lane - have_n)];
+    have_n += take_n;
+  }
+  if (overflow || have_n > 32) {
+    repair_column_any(a, cl, nn, tot, ne, cap_n, lane);
+    return;
+  }
+  const bool have = lane < have_n;
+  const int j = (int)(entry & 0xFFFFFu);
+  int v = have ? (int)((entry >> 20) & 0x7FFu) : 0;
+  const bool dist = have && (entry >> 31);
+  int16_t *col = a.pop + (size_t)cl * J * NN + nn;
+  if (ne >= 2) {
+    const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
+    int t = J;
+    if (dist && v > 0) { t = j - o; if (t < 0) t += J; }
+    int best = t;
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, off));
+    int removed = 0;
+    if (dist && v > 0 && t != best) {
+      col[(size_t)j * NN] = 0;
+      summ_update(a, cl, j, nn, v, 0);
+      removed = v;
+      v = 0;
+    }
+    tot -= warp_sum(removed);
+  }
+  const int excess = tot - cap_n;
+  if (excess > 0) {
+    const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J);
+    int rot = 0x7fffffff;
+    if (have) { rot = j - o; if (rot < 0) rot += J; }
+    int ahead = 0;                       // GPUs of the occupants that come first in rotated order
+#pragma unroll
+    for (int k = 0; k < 32; ++k) {
+      const int rk = __shfl_sync(0xffffffffu, rot, k);
+      const int vk = __shfl_sync(0xffffffffu, v, k);
+      if (rk < rot) ahead += vk;
+    }
+    const int take = have ? min(v, max(excess - ahead, 0)) : 0;
+    if (take > 0) {
+      col[(size_t)j * NN] = (int16_t)(v - take);
+      summ_update(a, cl, j, nn, v, v - take);
+    }
+  }
+}
+
+// Column pass, step 1: a thread per (candidate, node) adds the batch partials up; nodes that
+// hold two distributed jobs or exceed their size are appended to a work list.
+__global__ void __launch_bounds__(128) colscan_kernel(ColfixArgs a) {
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  const int cl = blockIdx.y;
+  const int NN = a.num_nodes;
+  if (n >= NN) return;
+  int total = 0, nelig = 0;
+  for (int b = 0; b < a.nbatch; ++b) {
+    total += a.colsum[((size_t)cl * a.nbatch + b) * NN + n];
+    nelig += a.colelig[((size_t)cl * a.nbatch + b) * NN + n];
+  }
+  if (nelig >= 2 || total > max((int)a.cap[n], 0)) {
+    const unsigned slot = atomicAdd(a.list_count, 1u);
+    a.list[slot] = ((uint32_t)cl << 13) | (uint32_t)n;      // n < 8192, cl < 65536
+  }
+}
+
+// Column pass, step 2: warps take columns from the work list (any order: columns are
+// independent) and repair them.
+__global__ void __launch_bounds__(128, 4) colrepair_kernel(ColfixArgs a) {
+  const int lane = threadIdx.x & 31;
+  const unsigned nwarps = gridDim.x * (blockDim.x >> 5);
+  const unsigned count = *a.list_count;
+  const int NN = a.num_nodes;
+  for (unsigned i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); i < count; i += nwarps) {
+    const uint32_t e = a.list[i];
+    const int cl = (int)(e >> 13), n = (int)(e & 0x1FFFu);
+    int total = 0, nelig = 0;
+    for (int b = 0; b < a.nbatch; ++b) {
+      total += a.colsum[((size_t)cl * a.nbatch + b) * NN + n];
+      nelig += a.colelig[((size_t)cl * a.nbatch + b) * NN + n];
+    }
+    const int cp = max((int)a.cap[n], 0);
+    repair_column_list(a, cl, n, total, nelig, cp, lane);
     __syncwarp();
   }
 }
@@ -694,8 +917,10 @@ int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint3
                      uint32_t round, uint32_t gen) {
   if (count == 0 || a.J == 0) return SCHED_OK;
   const int NN = a.num_nodes;
-  const bool aligned = ((((uintptr_t)a.dst | (uintptr_t)a.src) & 15) == 0);
-  const bool fused = (NN % 8 == 0) && NN <= 512 && aligned && ctx->cap_max <= 2047 && count <= 65535;
+  const bool aligned = ((((uintptr_t)a.dst | (uintptr_t)a.src | (uintptr_t)a.cur) & 15) == 0);
+  const bool fused = (NN % 8 == 0) && NN <= 512 && aligned && ctx->cap_max <= 2047 && count <= 65535 &&
+                     a.J <= (1 << 20);
+  ctx->summ_valid = fused && a.summ != nullptr;
   if (!fused) {
     if (a.mode == ROWS_GENERATION) {
       {
@@ -714,20 +939,45 @@ int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint3
   Rows2Args aa;
   aa.r = a;
   aa.colsum = ctx->d_colsum; aa.colelig = ctx->d_colelig; aa.nbatch = nbatch;
+  aa.list_count = ctx->d_colcount;
+  aa.occ_count = ctx->d_occcount; aa.occ_list = ctx->d_occlist;
   dim3 grid((unsigned)nbatch, (unsigned)count);
   {
     TimedLaunch tl_(ctx, KK_ROWS);
-    if (NN <= 256) rows2_kernel<1><<<grid, 256, 0, ctx->stream>>>(aa);
-    else rows2_kernel<2><<<grid, 256, 0, ctx->stream>>>(aa);
+    // about four vectors per lane: several loads in flight and the per-row overhead shared
+    const int row_vecs = NN / 8;
+    int lpr_log2 = 0;
+    while ((4 << lpr_log2) < row_vecs && lpr_log2 < 5) ++lpr_log2;
+    aa.lpr_log2 = lpr_log2;
+    const int vpl = (row_vecs + (1 << lpr_log2) - 1) >> lpr_log2;
+    const bool full = (vpl << lpr_log2) == row_vecs && (vpl == 1 || vpl == 2 || vpl == 4);
+#define ROWS2(L, V)                                                            \
+  do {                                                                         \
+    if (full) rows2_kernel<L, V, true><<<grid, 256, 0, ctx->stream>>>(aa);     \
+    else rows2_kernel<L, V, false><<<grid, 256, 0, ctx->stream>>>(aa);         \
+  } while (0)
+    if (lpr_log2 == 0) {
+      if (vpl <= 1) ROWS2(0, 1);
+      else if (vpl == 2) ROWS2(0, 2);
+      else ROWS2(0, 4);
+    } else if (lpr_log2 == 1) ROWS2(1, 4);
+    else if (lpr_log2 == 2) ROWS2(2, 4);
+    else if (lpr_log2 == 3) ROWS2(3, 4);
+    else ROWS2(4, 4);
+#undef ROWS2
   }
   SCHED_LAUNCH_CHECK(ctx);
   ColfixArgs f;
   f.pop = pop; f.dflag = ctx->d_dflag; f.cap = ctx->d_cap;
-  f.colsum = ctx->d_colsum; f.colelig = ctx->d_colelig;
+  f.colsum = ctx->d_colsum; f.colelig = ctx->d_colelig; f.summ = a.summ;
   f.J = a.J; f.num_nodes = NN; f.nbatch = nbatch;
   f.gen = gen; f.first_cand = first_cand; f.key = make_key(ctx->cfg.seed, round);
+  f.list = ctx->d_collist; f.list_count = ctx->d_colcount;
+  f.cur = a.cur; f.occ_count = ctx->d_occcount; f.occ_list = ctx->d_occlist;
   dim3 g2((unsigned)((NN + 127) / 128), (unsigned)count);
-  { TimedLaunch tl_(ctx, KK_COLS); colfix_kernel<<<g2, 128, 0, ctx->stream>>>(f); }
+  { TimedLaunch tl_(ctx, KK_COLSCAN); colscan_kernel<<<g2, 128, 0, ctx->stream>>>(f); }
+  SCHED_LAUNCH_CHECK(ctx);
+  { TimedLaunch tl_(ctx, KK_COLS); colrepair_kernel<<<ctx->num_sms * 4, 128, 0, ctx->stream>>>(f); }
   SCHED_LAUNCH_CHECK(ctx);
   return SCHED_OK;
 }
@@ -742,6 +992,7 @@ RowsArgs base_rows_args(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d
   a.thr = 0; a.gen = 0; a.first_cand = 0;
   a.key = make_key(c.seed, 0);
   a.src = nullptr; a.dst = nullptr; a.mode = ROWS_REPAIR; a.fitness_bits = nullptr;
+  a.cur = nullptr; a.summ = nullptr;
   return a;
 }
 
@@ -765,6 +1016,7 @@ int launch_init_population(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t
   RowsArgs a = base_rows_args(ctx, d_k_cap, d_active, P);
   a.mode = ROWS_INIT; a.src = d_cur; a.dst = d_pop_out;
   a.thr = ctx->cfg.thr_init; a.gen = GEN_INIT; a.key = make_key(ctx->cfg.seed, round);
+  a.cur = ctx->round_cur; a.summ = ctx->round_summ;
   return launch_rows_cols(ctx, a, d_pop_out, P, 0u, round, GEN_INIT);
 }
 
@@ -778,6 +1030,7 @@ int launch_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_a
   a.mode = ROWS_GENERATION; a.src = d_pop_in; a.dst = d_pop_out;
   a.fitness_bits = (const uint32_t *)d_fitness_in;
   a.thr = ctx->cfg.thr_mutate; a.gen = generation; a.key = make_key(ctx->cfg.seed, round);
+  a.cur = ctx->round_cur; a.summ = ctx->round_summ;
   return launch_rows_cols(ctx, a, d_pop_out, P, 0u, round, generation);
 }
 
