@@ -186,6 +186,13 @@ int ga_generation(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_pop
 int schedule_round(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cur, uint32_t round,
                    int32_t generations, int16_t *d_best, float *d_best_fitness);
 
+/* schedule_round replays a CUDA graph of the whole round from the third call on that passes
+ * the same pointers and generation count (the second such call captures it); this removes
+ * the per-kernel launch cost that dominates small problems.  Results are identical with
+ * and without graphs.  On by default; not used on the NULL stream or while per-kernel
+ * timing is enabled.  sched_set_graphs(ctx, 0) turns it off. */
+int sched_set_graphs(sched_ctx *ctx, int enable);
+
 /* Same with HOST buffers: copies the job arrays and h_cur to the device, runs the round,
  * copies the result back and waits for it.  Every member of h_jobs is a host pointer. */
 int schedule_round_host(sched_ctx *ctx, const sched_jobs *h_jobs, const int16_t *h_cur,

@@ -78,7 +78,8 @@ int ensure_round_scratch(sched_ctx *ctx) {
   int rc;
   if ((rc = dev_alloc(ctx, &ctx->d_popA, pop)) != SCHED_OK) return rc;
   if ((rc = dev_alloc(ctx, &ctx->d_popB, pop)) != SCHED_OK) return rc;
-  if ((rc = dev_alloc(ctx, &ctx->d_fit, (size_t)c.population)) != SCHED_OK) return rc;
+  if ((rc = dev_alloc(ctx, &ctx->d_fit_buf, 2 * (size_t)c.population)) != SCHED_OK) return rc;
+  ctx->d_fit = ctx->d_fit_buf;
   if ((rc = dev_alloc(ctx, &ctx->d_tab_goodput, tab)) != SCHED_OK) return rc;
   if ((rc = dev_alloc(ctx, &ctx->d_tab_speedup, tab)) != SCHED_OK) return rc;
   if ((rc = dev_alloc(ctx, &ctx->d_rf, (size_t)c.num_jobs)) != SCHED_OK) return rc;
@@ -228,6 +229,8 @@ int sched_init(const sched_config *cfg, const int16_t *h_node_capacity, void *cu
   if ((rc = dev_alloc(ctx, &ctx->d_status, 1)) != SCHED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_best_idx, 1)) != SCHED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_colcount, 1)) != SCHED_OK) return fail(rc);
+  if ((rc = dev_alloc(ctx, &ctx->d_round, 1)) != SCHED_OK) return fail(rc);
+  ctx->graphs_enabled = true;
   e = cudaMemcpyAsync(ctx->d_cap, h_node_capacity, sizeof(int16_t) * cfg->num_nodes,
                       cudaMemcpyHostToDevice, ctx->stream);
   if (e == cudaSuccess)
@@ -251,11 +254,12 @@ int sched_destroy(sched_ctx *ctx) {
   cudaStreamSynchronize(ctx->stream);
   void *ptrs[] = {ctx->d_cap, ctx->d_kfit, ctx->d_pairs, ctx->d_gmax, ctx->d_amax, ctx->d_rank, ctx->d_order,
                   ctx->d_dflag, ctx->d_pen, ctx->d_partial, ctx->d_ticket, ctx->d_status,
-                  ctx->d_popA, ctx->d_popB, ctx->d_fit, ctx->d_tab_goodput, ctx->d_tab_speedup,
-                  ctx->d_rf, ctx->d_best_idx, ctx->d_stage, ctx->d_stage_fit, ctx->d_colsum, ctx->d_summ, ctx->d_collist, ctx->d_colcount, ctx->d_occcount, ctx->d_occlist,
+                  ctx->d_popA, ctx->d_popB, ctx->d_fit_buf, ctx->d_tab_goodput, ctx->d_tab_speedup,
+                  ctx->d_rf, ctx->d_best_idx, ctx->d_stage, ctx->d_stage_fit, ctx->d_colsum, ctx->d_summ, ctx->d_collist, ctx->d_colcount, ctx->d_round, ctx->d_occcount, ctx->d_occlist,
                   ctx->d_colelig};
   for (void *p : ptrs)
     if (p) cudaFree(p);
+  if (ctx->graph_exec) cudaGraphExecDestroy(ctx->graph_exec);
   for (auto *v : {&ctx->spans, &ctx->free_spans})
     for (TimedSpan &t : *v) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
   delete ctx;
@@ -278,6 +282,12 @@ int64_t sched_launch_count(const sched_ctx *ctx) { return ctx ? ctx->launches : 
 int sched_set_kernel_timing(sched_ctx *ctx, int enable) {
   REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "sched_set_kernel_timing: ctx is NULL");
   ctx->timing_on = enable != 0;
+  return SCHED_OK;
+}
+
+int sched_set_graphs(sched_ctx *ctx, int enable) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "sched_set_graphs: ctx is NULL");
+  ctx->graphs_enabled = enable != 0;
   return SCHED_OK;
 }
 
@@ -348,8 +358,10 @@ int repair_population(sched_ctx *ctx, const sched_jobs *d_jobs, int16_t *d_pop, 
   REQUIRE(ctx, (long long)count * ctx->cfg.num_jobs < (1LL << 31), SCHED_ERR_TOO_LARGE,
           "repair_population: count * num_jobs must be below 2^31");
   if (ctx->cfg.num_jobs == 0) return SCHED_OK;
+  int rc = launch_set_round(ctx, round);
+  if (rc != SCHED_OK) return rc;
   return launch_repair(ctx, d_jobs ? d_jobs->k_cap : nullptr, d_jobs ? d_jobs->active : nullptr, d_pop,
-                       count, first_candidate, round, generation);
+                       count, first_candidate, generation);
 }
 
 int init_population(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cur, uint32_t round,
@@ -359,8 +371,10 @@ int init_population(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_c
   REQUIRE(ctx, ((uintptr_t)d_pop_out & 1) == 0 && ((uintptr_t)d_cur & 1) == 0, SCHED_ERR_INVALID_ARG,
           "init_population: a buffer is misaligned");
   if (ctx->cfg.num_jobs == 0) return SCHED_OK;
+  int rc = launch_set_round(ctx, round);
+  if (rc != SCHED_OK) return rc;
   return launch_init_population(ctx, d_jobs ? d_jobs->k_cap : nullptr,
-                                d_jobs ? d_jobs->active : nullptr, d_cur, round, d_pop_out);
+                                d_jobs ? d_jobs->active : nullptr, d_cur, d_pop_out);
 }
 
 int ga_generation(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_pop_in,
@@ -372,9 +386,75 @@ int ga_generation(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_pop
   REQUIRE(ctx, (((uintptr_t)d_pop_in | (uintptr_t)d_pop_out) & 1) == 0 && ((uintptr_t)d_fitness_in & 3) == 0,
           SCHED_ERR_INVALID_ARG, "ga_generation: a buffer is misaligned");
   if (ctx->cfg.num_jobs == 0) return SCHED_OK;
+  int rc = launch_set_round(ctx, round);
+  if (rc != SCHED_OK) return rc;
   return launch_generation(ctx, d_jobs ? d_jobs->k_cap : nullptr, d_jobs ? d_jobs->active : nullptr,
-                           d_pop_in, d_fitness_in, d_pop_out, round, generation);
+                           d_pop_in, d_fitness_in, d_pop_out, generation);
 }
+
+// Everything a round enqueues on the stream (the round number is already in d_round).
+static int round_body(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cur, int32_t generations,
+                      int16_t *d_best, float *d_best_fitness) {
+  int rc;
+  const bool penalise = d_cur && d_jobs->age_sec && d_jobs->num_restarts;
+  if ((rc = launch_speedup_table(ctx, d_jobs, ctx->d_tab_goodput, ctx->d_tab_speedup, nullptr)) != SCHED_OK) return rc;
+  if (penalise && (rc = launch_realloc_factor(ctx, d_jobs, ctx->d_rf)) != SCHED_OK) return rc;
+  const float *rf = penalise ? ctx->d_rf : nullptr;
+  int16_t *pa = ctx->d_popA, *pb = ctx->d_popB;
+  // While the round runs, the row/column kernels also keep per-row summaries (K, N, differs
+  // from the current allocation); the in-round fitness reads those instead of the matrices
+  // whenever the batched kernels were used, with bit-identical results.
+  ctx->round_cur = rf ? d_cur : nullptr;
+  ctx->round_summ = ctx->d_summ;
+  // the per-job penalty factors depend only on the current allocation: prepared once
+  ctx->pen_ready = false;
+  rc = SCHED_OK;
+  if (rf) rc = launch_penalty_prep(ctx, d_cur, rf);
+  ctx->pen_ready = (rc == SCHED_OK) && rf;
+  // problems whose candidates fit one block get row pass, column pass and fitness in one kernel
+  ctx->ff_on = true;
+  ctx->ff_table = ctx->d_tab_speedup;
+  ctx->ff_pen = rf ? ctx->d_pen : nullptr;
+  ctx->ff_active = d_jobs->active;
+  ctx->ff_p = ctx->cfg.p;
+  // parents' fitness is read while children's is written: the two alternate between buffers
+  float *fit_cur = ctx->d_fit_buf, *fit_next = ctx->d_fit_buf + ctx->cfg.population;
+  ctx->ff_out = fit_cur;
+  auto fitness_of = [&](const int16_t *pop, float *out) {
+    if (ctx->fit_done) return (int)SCHED_OK;
+    return launch_fitness(ctx, pop, ctx->cfg.population, ctx->d_tab_speedup, d_cur, rf, d_jobs->active,
+                          ctx->cfg.p, out, ctx->summ_valid ? ctx->d_summ : nullptr);
+  };
+  if (rc == SCHED_OK) rc = launch_init_population(ctx, d_jobs->k_cap, d_jobs->active, d_cur, pa);
+  if (rc == SCHED_OK) rc = fitness_of(pa, fit_cur);
+  for (int g = 0; g < generations && rc == SCHED_OK; ++g) {
+    ctx->ff_out = fit_next;
+    rc = launch_generation(ctx, d_jobs->k_cap, d_jobs->active, pa, fit_cur, pb, (uint32_t)g);
+    if (rc != SCHED_OK) break;
+    std::swap(pa, pb);
+    rc = fitness_of(pa, fit_next);
+    std::swap(fit_cur, fit_next);
+  }
+  ctx->d_fit = fit_cur;
+  ctx->pen_ready = false;
+  ctx->ff_on = false;
+  ctx->fit_done = false;
+  ctx->round_cur = nullptr;
+  ctx->round_summ = nullptr;
+  ctx->summ_valid = false;
+  if (rc != SCHED_OK) return rc;
+  ctx->d_pop_last = pa;
+  return launch_select_best(ctx, pa, ctx->d_fit, d_best, d_best_fitness);
+}
+
+
+// A round is a fixed sequence of kernels whose arguments do not change from round to round
+// when the caller reuses its buffers (the round number lives in device memory).  The second
+// time a round is requested with the same pointers and generation count it is captured
+// into a CUDA graph; later rounds replay the graph, which removes the per-kernel launch
+// cost that dominates small problems.  Graphs are not used while per-kernel timing is on,
+// on the legacy default stream, or after a capture failed.
+static bool same_round_key(const RoundKey &a, const RoundKey &b) { return memcmp(&a, &b, sizeof(RoundKey)) == 0; }
 
 int schedule_round(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cur, uint32_t round,
                    int32_t generations, int16_t *d_best, float *d_best_fitness) {
@@ -385,38 +465,56 @@ int schedule_round(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cu
   REQUIRE(ctx, d_best && d_best_fitness, SCHED_ERR_INVALID_ARG,
           "schedule_round: d_best and d_best_fitness must be non-NULL");
   REQUIRE(ctx, ctx->cfg.num_jobs >= 1, SCHED_ERR_BAD_CONFIG, "schedule_round: needs at least one job");
-  const bool penalise = d_cur && d_jobs->age_sec && d_jobs->num_restarts;
   if ((rc = ensure_round_scratch(ctx)) != SCHED_OK) return rc;
-  if ((rc = launch_speedup_table(ctx, d_jobs, ctx->d_tab_goodput, ctx->d_tab_speedup, nullptr)) != SCHED_OK) return rc;
-  if (penalise && (rc = launch_realloc_factor(ctx, d_jobs, ctx->d_rf)) != SCHED_OK) return rc;
-  const float *rf = penalise ? ctx->d_rf : nullptr;
-  int16_t *pa = ctx->d_popA, *pb = ctx->d_popB;
-  // While the round runs, the row/column kernels also keep per-row summaries (K, N, differs
-  // from the current allocation); the in-round fitness reads those instead of the matrices
-  // whenever the batched kernels were used, with bit-identical results.
-  ctx->round_cur = rf ? d_cur : nullptr;
-  ctx->round_summ = ctx->d_summ;
-  ctx->pen_ready = false;
-  rc = launch_init_population(ctx, d_jobs->k_cap, d_jobs->active, d_cur, round, pa);
-  if (rc == SCHED_OK)
-    rc = launch_fitness(ctx, pa, ctx->cfg.population, ctx->d_tab_speedup, d_cur, rf, d_jobs->active,
-                        ctx->cfg.p, ctx->d_fit, ctx->summ_valid ? ctx->d_summ : nullptr);
-  // the per-job penalty factors depend only on the current allocation: prepared once
-  ctx->pen_ready = (rc == SCHED_OK);
-  for (int g = 0; g < generations && rc == SCHED_OK; ++g) {
-    rc = launch_generation(ctx, d_jobs->k_cap, d_jobs->active, pa, ctx->d_fit, pb, round, (uint32_t)g);
-    if (rc != SCHED_OK) break;
-    std::swap(pa, pb);
-    rc = launch_fitness(ctx, pa, ctx->cfg.population, ctx->d_tab_speedup, d_cur, rf, d_jobs->active,
-                        ctx->cfg.p, ctx->d_fit, ctx->summ_valid ? ctx->d_summ : nullptr);
+  if ((rc = launch_set_round(ctx, round)) != SCHED_OK) return rc;
+
+  RoundKey key;
+  memset(&key, 0, sizeof(key));
+  key.jobs = *d_jobs;
+  key.cur = d_cur; key.best = d_best; key.best_fitness = d_best_fitness; key.generations = generations;
+  const bool graphs_ok = ctx->graphs_enabled && !ctx->timing_on && ctx->stream != nullptr;
+  if (graphs_ok && ctx->graph_exec && same_round_key(key, ctx->graph_key)) {
+    SCHED_CUDA_CHECK(ctx, cudaGraphLaunch(ctx->graph_exec, ctx->stream));
+    ctx->launches += ctx->graph_launches;
+    ctx->d_fit = ctx->graph_fit;
+    ctx->d_pop_last = ctx->graph_pop_last;
+    return SCHED_OK;
   }
-  ctx->pen_ready = false;
-  ctx->round_cur = nullptr;
-  ctx->round_summ = nullptr;
-  ctx->summ_valid = false;
-  if (rc != SCHED_OK) return rc;
-  ctx->d_pop_last = pa;
-  return launch_select_best(ctx, pa, ctx->d_fit, d_best, d_best_fitness);
+  const bool capture = graphs_ok && ctx->seen_valid && same_round_key(key, ctx->seen_key);
+  memcpy(&ctx->seen_key, &key, sizeof(key));
+  ctx->seen_valid = true;
+  if (!capture) return round_body(ctx, d_jobs, d_cur, generations, d_best, d_best_fitness);
+
+  // second request with the same arguments: all scratch exists already, so the body makes no
+  // allocation and can be captured
+  if (ctx->graph_exec) { cudaGraphExecDestroy(ctx->graph_exec); ctx->graph_exec = nullptr; }
+  const int64_t launches_before = ctx->launches;
+  cudaGraph_t graph = nullptr;
+  if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();
+    ctx->graphs_enabled = false;
+    return round_body(ctx, d_jobs, d_cur, generations, d_best, d_best_fitness);
+  }
+  rc = round_body(ctx, d_jobs, d_cur, generations, d_best, d_best_fitness);
+  const cudaError_t ce = cudaStreamEndCapture(ctx->stream, &graph);
+  const int64_t captured = ctx->launches - launches_before;
+  ctx->launches = launches_before;
+  if (rc != SCHED_OK || ce != cudaSuccess || !graph ||
+      cudaGraphInstantiate(&ctx->graph_exec, graph, 0) != cudaSuccess) {
+    cudaGetLastError();
+    if (graph) cudaGraphDestroy(graph);
+    ctx->graph_exec = nullptr;
+    ctx->graphs_enabled = false;   // run plainly from now on
+    return round_body(ctx, d_jobs, d_cur, generations, d_best, d_best_fitness);
+  }
+  cudaGraphDestroy(graph);
+  memcpy(&ctx->graph_key, &key, sizeof(key));
+  ctx->graph_launches = captured;
+  ctx->graph_fit = ctx->d_fit;
+  ctx->graph_pop_last = ctx->d_pop_last;
+  SCHED_CUDA_CHECK(ctx, cudaGraphLaunch(ctx->graph_exec, ctx->stream));
+  ctx->launches += captured;
+  return SCHED_OK;
 }
 
 int sched_get_population(sched_ctx *ctx, int16_t *d_pop_out, float *d_fitness_out) {

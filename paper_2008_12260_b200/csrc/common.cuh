@@ -29,6 +29,15 @@ struct TimedSpan {
   int kind;
 };
 
+// What identifies a round for graph reuse: every pointer it is given and its length.
+struct RoundKey {
+  sched_jobs jobs;
+  const int16_t *cur;
+  int16_t *best;
+  float *best_fitness;
+  int32_t generations;
+};
+
 struct sched_ctx {
   sched_config cfg;
   cudaStream_t stream;
@@ -64,12 +73,21 @@ struct sched_ctx {
   uint32_t *round_summ;      // d_summ while a round runs, else NULL
   uint32_t *d_summ;          // [P][J]
   bool summ_valid;           // the last row/column pass filled d_summ
+  // fitness fused into the generation kernel (single-batch problems): inputs set by
+  // schedule_round, fit_done reports that the last row/column pass also wrote the fitness
+  const float *ff_table, *ff_pen;
+  const uint8_t *ff_active;
+  float ff_p;
+  float *ff_out;
+  bool ff_on, fit_done;
   bool pen_ready;        // d_pen already holds this round's factors (set by schedule_round)
   int *d_status;         // device status word
+  uint32_t *d_round;     // round number read by the operator kernels
 
   // scratch of schedule_round (allocated on first use)
   int16_t *d_popA, *d_popB;
-  float *d_fit;          // [P]
+  float *d_fit;          // [P] fitness of the current population (points into d_fit_buf)
+  float *d_fit_buf;      // [2][P]: parents' and children's fitness alternate between the halves
   float *d_tab_goodput, *d_tab_speedup;
   float *d_rf;           // [J]
   int32_t *d_best_idx;
@@ -81,6 +99,14 @@ struct sched_ctx {
   size_t stage_bytes;
   void *d_stage_fit;     // eval_fitness_host staging
   size_t stage_fit_bytes;
+
+  // CUDA graph of a whole round (see schedule_round)
+  bool graphs_enabled, seen_valid;
+  RoundKey seen_key, graph_key;
+  cudaGraphExec_t graph_exec;
+  int64_t graph_launches;
+  float *graph_fit;
+  int16_t *graph_pop_last;
 
   // optional per-kernel timing with CUDA events on the context's stream
   bool timing_on;
@@ -155,22 +181,24 @@ __host__ __device__ __forceinline__ u32x4 philox4x32_10(u32x4 c, uint32_t k0, ui
 }
 
 // Random stream of the operators: key = (seed_lo ^ seed_hi, round),
-// counter = (idx, candidate, generation, slot).
+// counter = (idx, candidate, generation, slot).  The round number is read from device
+// memory so that a captured CUDA graph of a round can be replayed for any round.
 struct RngKey {
-  uint32_t k0, k1;
+  uint32_t k0;
+  const uint32_t *round_ptr;
 };
 
-__host__ __device__ __forceinline__ RngKey make_key(uint64_t seed, uint32_t round) {
+inline RngKey make_key(uint64_t seed, const uint32_t *d_round) {
   RngKey k;
   k.k0 = (uint32_t)seed ^ (uint32_t)(seed >> 32);
-  k.k1 = round;
+  k.round_ptr = d_round;
   return k;
 }
 
 __device__ __forceinline__ u32x4 draw(RngKey k, uint32_t idx, uint32_t cand, uint32_t gen,
                                       uint32_t slot) {
   u32x4 c = {idx, cand, gen, slot};
-  return philox4x32_10(c, k.k0, k.k1);
+  return philox4x32_10(c, k.k0, __ldg(k.round_ptr));
 }
 
 // floor(w * n / 2^32): an integer in [0, n)
@@ -189,14 +217,16 @@ int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const fl
                    const int16_t *d_cur, const float *d_rf, const uint8_t *d_active, float p,
                    float *d_fitness, const uint32_t *d_summ = nullptr);
 int launch_repair(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active, int16_t *d_pop,
-                  int32_t count, uint32_t first_candidate, uint32_t round, uint32_t generation);
+                  int32_t count, uint32_t first_candidate, uint32_t generation);
 int launch_init_population(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active,
-                           const int16_t *d_cur, uint32_t round, int16_t *d_pop_out);
+                           const int16_t *d_cur, int16_t *d_pop_out);
 int launch_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active,
                       const int16_t *d_pop_in, const float *d_fitness_in, int16_t *d_pop_out,
-                      uint32_t round, uint32_t generation);
+                      uint32_t generation);
+int launch_set_round(sched_ctx *ctx, uint32_t round);
 int launch_select_best(sched_ctx *ctx, const int16_t *d_pop, const float *d_fitness,
                        int16_t *d_best, float *d_best_fitness);
 int ensure_fitness_scratch(sched_ctx *ctx, int32_t count, int chunks);
 int ensure_dflag(sched_ctx *ctx, int32_t count);
+int launch_penalty_prep(sched_ctx *ctx, const int16_t *d_cur, const float *d_rf);
 int ensure_colscratch(sched_ctx *ctx, size_t ints);

@@ -9,10 +9,9 @@
 // candidate's rows; chunk sums go to a scratch array and the last block to arrive adds
 // them in index order, so results are bitwise reproducible.
 #include "common.cuh"
+#include "fitness_common.cuh"
 
 namespace {
-
-enum { MODE_POW = 0, MODE_ARITH = 1, MODE_HARM = 2, MODE_GEO = 3, MODE_SQRT = 4 };
 
 template <int W>
 struct VecLoad;
@@ -90,8 +89,10 @@ __global__ void __launch_bounds__(256) fitness_kernel(FitnessArgs a) {
   const char *cur_base = (const char *)a.cur;
   const size_t row_bytes = (size_t)a.num_nodes * 2;
 
-  double acc = 0.0;
-  int cnt = 0;
+  __shared__ float s_term[FITNESS_MAX_ROWS_PER_BLOCK];
+  TermParams tp;
+  tp.table = a.table; tp.pen = a.pen; tp.active = a.active;
+  tp.k_max = a.k_max; tp.n_max = a.n_max; tp.mode = a.mode; tp.p = a.p; tp.floor_ = a.floor_;
   uint32_t mine = 0;
   int myrow = -1;
   int it = 0;
@@ -145,45 +146,22 @@ __global__ void __launch_bounds__(256) fitness_kernel(FitnessArgs a) {
     }
     const bool flush = ((it + 1) % slots_per_fill == 0) || (jb + nwarps * RPW >= j1);
     if (flush) {
-      if (myrow >= 0 && (!a.active || a.active[myrow])) {
-        const int K = min((int)(mine & 0xFFFFu), a.k_max);
-        const int N = min((int)((mine >> 16) & 0x7FFFu), a.n_max);
-        float x = __ldg(a.table + ((size_t)myrow * KD + K) * ND + N);
-        if (a.pen && (mine >> 31)) x *= a.pen[myrow];
-        x = fmaxf(x, a.floor_);
-        float t;
-        switch (a.mode) {
-          case MODE_ARITH: t = x; break;
-          case MODE_HARM: t = 1.f / x; break;
-          case MODE_GEO: t = logf(x); break;
-          case MODE_SQRT: t = sqrtf(x); break;
-          default: t = powf(x, a.p); break;
-        }
-        acc += (double)t;
-        cnt += 1;
-      }
+      if (myrow >= 0 && (!a.active || a.active[myrow]))
+        s_term[myrow - j0] = fitness_term(tp, myrow, (int)(mine & 0xFFFFu), (int)((mine >> 16) & 0x7FFFu),
+                                          (mine >> 31) != 0u);
       myrow = -1;
     }
   }
 
-  // block reduction in a fixed order
-#pragma unroll
-  for (int off = 16; off >= 1; off >>= 1) {
-    acc += __shfl_xor_sync(0xffffffffu, acc, off);
-    cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
-  }
-  __shared__ double s_acc[8];
-  __shared__ int s_cnt[8];
-  __shared__ bool s_last;
-  if (lane == 0) { s_acc[warp] = acc; s_cnt[warp] = cnt; }
+  // the block's terms, summed in an order that does not depend on how rows were mapped to lanes
   __syncthreads();
+  double t, n;
+  block_term_sum(s_term, j1 - j0, j0, a.active, t, n);
+  __shared__ bool s_last;
   if (threadIdx.x == 0) {
-    double t = 0.0;
-    int n = 0;
-    for (int w = 0; w < nwarps; ++w) { t += s_acc[w]; n += s_cnt[w]; }
     double *dst = a.partial + ((size_t)cand * a.chunks + chunk) * 2;
     dst[0] = t;
-    dst[1] = (double)n;
+    dst[1] = n;
     __threadfence();
     const unsigned prev = atomicAdd(a.ticket + cand, 1u);
     s_last = (prev == (unsigned)a.chunks - 1u);
@@ -192,21 +170,9 @@ __global__ void __launch_bounds__(256) fitness_kernel(FitnessArgs a) {
   if (s_last && threadIdx.x == 0) {
     __threadfence();
     const volatile double *src = a.partial + (size_t)cand * a.chunks * 2;
-    double t = 0.0, n = 0.0;
-    for (int c = 0; c < a.chunks; ++c) { t += src[2 * c]; n += src[2 * c + 1]; }
-    double f;
-    if (n == 0.0) f = 0.0;
-    else {
-      const double mean = t / n;
-      switch (a.mode) {
-        case MODE_ARITH: f = mean; break;
-        case MODE_HARM: f = 1.0 / mean; break;
-        case MODE_GEO: f = exp(mean); break;
-        case MODE_SQRT: f = mean * mean; break;
-        default: f = pow(mean, 1.0 / (double)a.p); break;
-      }
-    }
-    a.fitness[cand] = (float)f;
+    double ts = 0.0, ns = 0.0;
+    for (int c = 0; c < a.chunks; ++c) { ts += src[2 * c]; ns += src[2 * c + 1]; }
+    a.fitness[cand] = fitness_finalise(a.mode, a.p, ts, ns);
     a.ticket[cand] = 0u;   // ready for the next call on this stream
   }
 }
@@ -239,6 +205,7 @@ void fitness_geometry(size_t row_bytes, uintptr_t align_bits, int J, int count, 
   while ((4 << lpr_log2) < row_vecs && lpr_log2 < 5) ++lpr_log2;
   rows_per_block = (int)((1u << 20) / row_bytes);
   if (rows_per_block < 256) rows_per_block = 256;
+  if (rows_per_block > FITNESS_MAX_ROWS_PER_BLOCK) rows_per_block = FITNESS_MAX_ROWS_PER_BLOCK;
   if (rows_per_block > J) rows_per_block = J > 0 ? J : 1;
   while (rows_per_block > 256 &&
          (long long)count * ((J + rows_per_block - 1) / rows_per_block) < 4LL * num_sms)
@@ -247,6 +214,17 @@ void fitness_geometry(size_t row_bytes, uintptr_t align_bits, int J, int count, 
 }
 
 }  // namespace
+
+int launch_penalty_prep(sched_ctx *ctx, const int16_t *d_cur, const float *d_rf) {
+  const int J = ctx->cfg.num_jobs;
+  if (J == 0) return SCHED_OK;
+  {
+    TimedLaunch tl_(ctx, KK_PENPREP);
+    penalty_prep_kernel<<<(J * 32 + 255) / 256, 256, 0, ctx->stream>>>(d_cur, d_rf, J, ctx->cfg.num_nodes, ctx->d_pen);
+  }
+  SCHED_LAUNCH_CHECK(ctx);
+  return SCHED_OK;
+}
 
 int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const float *d_speedup,
                    const int16_t *d_cur, const float *d_rf, const uint8_t *d_active, float p,
@@ -282,8 +260,7 @@ int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const fl
   a.lpr_log2 = lpr_log2;
   a.rows_per_block = rows_per_block; a.chunks = chunks;
   a.p = p; a.floor_ = c.speedup_floor;
-  a.mode = (p == 1.f) ? MODE_ARITH : (p == -1.f) ? MODE_HARM : (p == 0.f) ? MODE_GEO
-           : (p == 0.5f) ? MODE_SQRT : MODE_POW;
+  a.mode = fitness_mode(p);
   a.partial = ctx->d_partial;
   a.ticket = ctx->d_ticket;
   a.fitness = d_fitness;
@@ -424,8 +401,7 @@ int eval_fitness_noalloc(const int16_t *d_pop, int32_t count, int32_t num_jobs, 
   a.lpr_log2 = lpr_log2;
   a.rows_per_block = rows_per_block; a.chunks = chunks;
   a.p = p; a.floor_ = speedup_floor;
-  a.mode = (p == 1.f) ? MODE_ARITH : (p == -1.f) ? MODE_HARM : (p == 0.f) ? MODE_GEO
-           : (p == 0.5f) ? MODE_SQRT : MODE_POW;
+  a.mode = fitness_mode(p);
   a.partial = scratch->partial;
   a.ticket = scratch->ticket;
   a.fitness = d_fitness;

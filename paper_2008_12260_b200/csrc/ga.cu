@@ -8,6 +8,7 @@
 // followed by a column kernel (one thread per (candidate, node): interference and
 // capacity passes over the jobs of that node).
 #include "common.cuh"
+#include "fitness_common.cuh"
 
 namespace {
 
@@ -329,6 +330,11 @@ struct Rows2Args {
   int32_t *occ_count;        // [count][nbatch][num_nodes] rows of the batch that occupy the node
   uint32_t *occ_list;        // [count][nbatch][num_nodes][OCC_SLOTS] job | GPUs << 20 | distributed << 31
   int nbatch, lpr_log2;
+  // Single-batch candidates (J <= 256): the block also does the column pass and the fitness of
+  // its candidate, so a whole generation is one kernel.
+  int fuse;
+  TermParams tp;
+  float *fitness_out;        // [count]
 };
 
 __device__ __forceinline__ uint4 clamp_vec(uint4 x, uint4 cp) {
@@ -350,6 +356,197 @@ __device__ __forceinline__ uint32_t row_partial(uint4 x) {
   return (uint32_t)k | (((o & 0xFFFFu) + (o >> 16)) << 22);
 }
 
+struct ColfixArgs {
+  int16_t *pop;
+  const uint8_t *dflag;
+  const int16_t *cap;
+  const int32_t *colsum, *colelig;
+  uint32_t *summ;           // [count][J] row summaries to keep in step with the removals, or NULL
+  const int16_t *cur;       // current allocation (for the summaries' differing-entries count), or NULL
+  const int32_t *occ_count; // per (candidate, row batch, node) occupants recorded by the row kernel
+  const uint32_t *occ_list;
+  uint32_t *list;           // work list of (candidate << 13 | node) entries
+  unsigned int *list_count;
+  int J, num_nodes, nbatch;
+  uint32_t gen, first_cand;
+  RngKey key;
+};
+
+// A column-pass write A[j][n]: v_old -> v_new keeps row j's summary in step:
+// K += v_new - v_old, N -= 1 if the entry became empty, and the count of entries that
+// differ from the current allocation is adjusted.  The three fields never leave their
+// ranges, so one wrapped 32-bit add does all three.
+__device__ __forceinline__ void summ_update(const ColfixArgs &a, uint32_t *summ_c, int j, int n, int v_old, int v_new) {
+  if (!summ_c) return;
+  int d_diff = 0;
+  if (a.cur) {
+    const int cv = a.cur[(size_t)j * a.num_nodes + n];
+    d_diff = (int)(v_new != cv) - (int)(v_old != cv);
+  }
+  const uint32_t delta = (uint32_t)(v_new - v_old) + ((uint32_t)((v_new == 0 && v_old > 0) ? -1 : 0) << 11) +
+                         ((uint32_t)d_diff << 22);
+  atomicAdd(summ_c + j, delta);
+}
+
+// Repair of one column by a whole warp (any J): interference, then capacity, each with a
+// few passes over the column; loads are issued in batches so that they overlap.
+__device__ __noinline__ void repair_column_any(const ColfixArgs &a, uint32_t *summ_c, int cl, int nn, int tot, int ne,
+                                               int cap_n, int lane) {
+  const uint32_t c = a.first_cand + (uint32_t)cl;
+  const int J = a.J, NN = a.num_nodes;
+  const uint8_t *df = a.dflag + (size_t)cl * J;
+  {
+    int16_t *col = a.pop + (size_t)cl * J * NN + nn;
+    // the loops below first issue a batch of independent column loads, then work on them
+    constexpr int U = 8;
+    if (ne >= 2) {
+      const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
+      int best = J;
+      for (int jb = 0; jb < J; jb += 32 * U) {
+        int v[U], d[U];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+          const int j = jb + 32 * k + lane;
+          v[k] = (j < J) ? (int)col[(size_t)j * NN] : 0;
+          d[k] = (j < J) ? (int)df[j] : 0;
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+          if (d[k] && v[k] > 0) {
+            int t = jb + 32 * k + lane - o;
+            if (t < 0) t += J;
+            best = min(best, t);
+          }
+        }
+      }
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, off));
+      int keep = o + best;
+      if (keep >= J) keep -= J;
+      int removed = 0;
+      for (int jb = 0; jb < J; jb += 32 * U) {
+        int v[U], d[U];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+          const int j = jb + 32 * k + lane;
+          v[k] = (j < J) ? (int)col[(size_t)j * NN] : 0;
+          d[k] = (j < J) ? (int)df[j] : 0;
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+          const int j = jb + 32 * k + lane;
+          if (d[k] && v[k] > 0 && j != keep) {
+            col[(size_t)j * NN] = 0;
+            removed += v[k];
+            summ_update(a, summ_c, j, nn, v[k], 0);
+          }
+        }
+      }
+      tot -= warp_sum(removed);
+    }
+    int excess = tot - cap_n;
+    if (excess > 0) {
+      const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J);
+      constexpr int C = 4;   // chunks of 32 jobs loaded together
+      for (int t0 = 0; t0 < J && excess > 0; t0 += 32 * C) {
+        int v[C], jj[C];
+#pragma unroll
+        for (int k = 0; k < C; ++k) {
+          const int t = t0 + 32 * k + lane;
+          int j = o + t;
+          if (j >= J) j -= J;
+          jj[k] = j;
+          v[k] = (t < J) ? (int)col[(size_t)j * NN] : 0;
+        }
+#pragma unroll
+        for (int k = 0; k < C; ++k) {
+          if (excess <= 0) break;
+          int s = v[k];                                // inclusive prefix over the 32 jobs
+#pragma unroll
+          for (int off = 1; off < 32; off <<= 1) {
+            const int u = __shfl_up_sync(0xffffffffu, s, off);
+            if (lane >= off) s += u;
+          }
+          const int take = min(v[k], max(excess - (s - v[k]), 0));
+          if (take > 0) {
+            col[(size_t)jj[k] * NN] = (int16_t)(v[k] - take);
+            summ_update(a, summ_c, jj[k], nn, v[k], v[k] - take);
+          }
+          excess -= __shfl_sync(0xffffffffu, s, 31);
+        }
+      }
+    }
+  }
+}
+
+// Repair of one column from its occupants, one occupant per lane (entry = job | GPUs << 20 |
+// distributed << 31 in the first have_n lanes): no pass over the column.
+__device__ void repair_column_entries(const ColfixArgs &a, uint32_t *summ_c, int cl, int nn, int tot, int ne,
+                                      int cap_n, int lane, uint32_t entry, int have_n) {
+  const uint32_t c = a.first_cand + (uint32_t)cl;
+  const int J = a.J, NN = a.num_nodes;
+  const bool have = lane < have_n;
+  const int j = (int)(entry & 0xFFFFFu);
+  int v = have ? (int)((entry >> 20) & 0x7FFu) : 0;
+  const bool dist = have && (entry >> 31);
+  int16_t *col = a.pop + (size_t)cl * J * NN + nn;
+  if (ne >= 2) {
+    const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
+    int t = J;
+    if (dist && v > 0) { t = j - o; if (t < 0) t += J; }
+    int best = t;
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, off));
+    int removed = 0;
+    if (dist && v > 0 && t != best) {
+      col[(size_t)j * NN] = 0;
+      summ_update(a, summ_c, j, nn, v, 0);
+      removed = v;
+      v = 0;
+    }
+    tot -= warp_sum(removed);
+  }
+  const int excess = tot - cap_n;
+  if (excess > 0) {
+    const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J);
+    int rot = 0x7fffffff;
+    if (have) { rot = j - o; if (rot < 0) rot += J; }
+    int ahead = 0;                       // GPUs of the occupants that come first in rotated order
+#pragma unroll
+    for (int k = 0; k < 32; ++k) {
+      const int rk = __shfl_sync(0xffffffffu, rot, k);
+      const int vk = __shfl_sync(0xffffffffu, v, k);
+      if (rk < rot) ahead += vk;
+    }
+    const int take = have ? min(v, max(excess - ahead, 0)) : 0;
+    if (take > 0) {
+      col[(size_t)j * NN] = (int16_t)(v - take);
+      summ_update(a, summ_c, j, nn, v, v - take);
+    }
+  }
+}
+
+// Occupants gathered from the per-batch lists the row kernel left in global memory.  Falls
+// back to the column scan when a batch overflowed its slots or the node has more than 32
+// occupants.
+__device__ void repair_column_list(const ColfixArgs &a, int cl, int nn, int tot, int ne, int cap_n, int lane) {
+  const int NN = a.num_nodes;
+  uint32_t *summ_c = a.summ ? a.summ + (size_t)cl * a.J : nullptr;
+  uint32_t entry = 0;
+  int have_n = 0;
+  bool overflow = false;
+  for (int b = 0; b < a.nbatch; ++b) {
+    const size_t at = ((size_t)cl * a.nbatch + b) * NN + nn;
+    const int cb = a.occ_count[at];
+    overflow |= cb > OCC_SLOTS;
+    const int take_n = min(cb, OCC_SLOTS);
+    if (lane >= have_n && lane < have_n + take_n) entry = a.occ_list[at * OCC_SLOTS + (lane - have_n)];
+    have_n += take_n;
+  }
+  if (overflow || have_n > 32) repair_column_any(a, summ_c, cl, nn, tot, ne, cap_n, lane);
+  else repair_column_entries(a, summ_c, cl, nn, tot, ne, cap_n, lane, entry, have_n);
+}
+
 // VPL = 16-byte vectors per lane; a row is split over LPR = 1 << LPR_LOG2 lanes
 // (LPR * VPL >= row_vecs, FULL when equal), so a warp works on 32 / LPR rows at a time.
 template <int LPR_LOG2, int VPL, bool FULL>
@@ -363,6 +560,8 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
   __shared__ uint32_t s_occ[MAXN * OCC_SLOTS];
   __shared__ int s_parent[2];
   __shared__ int s_rank4[4];
+  __shared__ uint32_t s_summ[256];   // row summaries of the block's rows
+  __shared__ float s_term[256];
   // per-warp queue of non-empty vectors waiting to be expanded into occupants
   __shared__ __align__(16) uint4 s_qvec[8][QCAP];
   __shared__ uint32_t s_qmeta[8][QCAP];
@@ -629,13 +828,55 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
       const bool on = (flags & 2u) != 0u;
       a.dflag[(size_t)cl * J + j] = (on && dist) ? 1 : 0;
       // row summary for the fitness: K | N << 11 | (entries that differ from current) << 22
-      if (a.summ)
-        a.summ[(size_t)cl * J + j] = on ? ((uint32_t)K | ((uint32_t)N << 11) | ((uint32_t)ndiff << 22)) : 0u;
+      const uint32_t word = on ? ((uint32_t)K | ((uint32_t)N << 11) | ((uint32_t)ndiff << 22)) : 0u;
+      s_summ[warp * 32 + r] = word;
+      if (a.summ && !aa.fuse) a.summ[(size_t)cl * J + j] = word;
     }
   }
 
-  // ---- column partials and occupant lists of the block -------------------------------------
   __syncthreads();
+  if (aa.fuse) {
+    // ---- the whole candidate lives in this block: column pass and fitness right here ---------
+    ColfixArgs f;
+    f.pop = a.dst; f.dflag = a.dflag; f.cap = a.cap; f.cur = a.cur;
+    f.colsum = nullptr; f.colelig = nullptr; f.summ = nullptr; f.occ_count = nullptr; f.occ_list = nullptr;
+    f.list = nullptr; f.list_count = nullptr;
+    f.J = J; f.num_nodes = NN; f.nbatch = 1; f.gen = a.gen; f.first_cand = a.first_cand; f.key = a.key;
+    for (int nb = warp * 32; nb < NN; nb += 256) {
+      const int n = nb + lane;
+      const int total = (n < NN) ? s_tot[n] : 0, nelig = (n < NN) ? s_el[n] : 0;
+      const int cp = (n < NN) ? (int)s_cap[n] : 0;
+      unsigned todo = __ballot_sync(0xffffffffu, n < NN && (nelig >= 2 || total > cp));
+      while (todo) {
+        const int srcl = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const int nn = nb + srcl;
+        const int tot_n = __shfl_sync(0xffffffffu, total, srcl), ne_n = __shfl_sync(0xffffffffu, nelig, srcl);
+        const int cap_n = __shfl_sync(0xffffffffu, cp, srcl);
+        const int have_n = s_cnt[nn];
+        if (have_n > OCC_SLOTS) {
+          repair_column_any(f, s_summ, cl, nn, tot_n, ne_n, cap_n, lane);
+        } else {
+          const uint32_t entry = (lane < have_n) ? s_occ[nn * OCC_SLOTS + lane] : 0u;
+          repair_column_entries(f, s_summ, cl, nn, tot_n, ne_n, cap_n, lane, entry, have_n);
+        }
+        __syncwarp();
+      }
+    }
+    __syncthreads();
+    for (int j = threadIdx.x; j < J; j += blockDim.x) {
+      if (!aa.tp.active || aa.tp.active[j]) {
+        const uint32_t w = s_summ[j];
+        s_term[j] = fitness_term(aa.tp, j, (int)(w & 0x7FFu), (int)((w >> 11) & 0x7FFu), (w >> 22) != 0u);
+      }
+    }
+    __syncthreads();
+    double tsum, tcount;
+    block_term_sum(s_term, J, 0, aa.tp.active, tsum, tcount);
+    if (threadIdx.x == 0) aa.fitness_out[cl] = fitness_finalise(aa.tp.mode, aa.tp.p, tsum, tcount);
+    return;
+  }
+  // ---- column partials and occupant lists of the block -------------------------------------
   const size_t base = ((size_t)cl * aa.nbatch + batch) * NN;
   for (int i = threadIdx.x; i < NN; i += blockDim.x) {
     aa.colsum[base + i] = s_tot[i];
@@ -643,190 +884,6 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
     aa.occ_count[base + i] = s_cnt[i];
     const int cnt = min(s_cnt[i], OCC_SLOTS);
     for (int k = 0; k < cnt; ++k) aa.occ_list[(base + i) * OCC_SLOTS + k] = s_occ[i * OCC_SLOTS + k];
-  }
-}
-
-struct ColfixArgs {
-  int16_t *pop;
-  const uint8_t *dflag;
-  const int16_t *cap;
-  const int32_t *colsum, *colelig;
-  uint32_t *summ;           // [count][J] row summaries to keep in step with the removals, or NULL
-  const int16_t *cur;       // current allocation (for the summaries' differing-entries count), or NULL
-  const int32_t *occ_count; // per (candidate, row batch, node) occupants recorded by the row kernel
-  const uint32_t *occ_list;
-  uint32_t *list;           // work list of (candidate << 13 | node) entries
-  unsigned int *list_count;
-  int J, num_nodes, nbatch;
-  uint32_t gen, first_cand;
-  RngKey key;
-};
-
-// A column-pass write A[j][n]: v_old -> v_new keeps row j's summary in step:
-// K += v_new - v_old, N -= 1 if the entry became empty, and the count of entries that
-// differ from the current allocation is adjusted.  The three fields never leave their
-// ranges, so one wrapped 32-bit add does all three.
-__device__ __forceinline__ void summ_update(const ColfixArgs &a, int cl, int j, int n, int v_old, int v_new) {
-  if (!a.summ) return;
-  int d_diff = 0;
-  if (a.cur) {
-    const int cv = a.cur[(size_t)j * a.num_nodes + n];
-    d_diff = (int)(v_new != cv) - (int)(v_old != cv);
-  }
-  const uint32_t delta = (uint32_t)(v_new - v_old) + ((uint32_t)((v_new == 0 && v_old > 0) ? -1 : 0) << 11) +
-                         ((uint32_t)d_diff << 22);
-  atomicAdd(a.summ + (size_t)cl * a.J + j, delta);
-}
-
-// Repair of one column by a whole warp (any J): interference, then capacity, each with a
-// few passes over the column; loads are issued in batches so that they overlap.
-__device__ __noinline__ void repair_column_any(const ColfixArgs &a, int cl, int nn, int tot, int ne, int cap_n, int lane) {
-  const uint32_t c = a.first_cand + (uint32_t)cl;
-  const int J = a.J, NN = a.num_nodes;
-  const uint8_t *df = a.dflag + (size_t)cl * J;
-  {
-    int16_t *col = a.pop + (size_t)cl * J * NN + nn;
-    // the loops below first issue a batch of independent column loads, then work on them
-    constexpr int U = 8;
-    if (ne >= 2) {
-      const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
-      int best = J;
-      for (int jb = 0; jb < J; jb += 32 * U) {
-        int v[U], d[U];
-#pragma unroll
-        for (int k = 0; k < U; ++k) {
-          const int j = jb + 32 * k + lane;
-          v[k] = (j < J) ? (int)col[(size_t)j * NN] : 0;
-          d[k] = (j < J) ? (int)df[j] : 0;
-        }
-#pragma unroll
-        for (int k = 0; k < U; ++k) {
-          if (d[k] && v[k] > 0) {
-            int t = jb + 32 * k + lane - o;
-            if (t < 0) t += J;
-            best = min(best, t);
-          }
-        }
-      }
-#pragma unroll
-      for (int off = 16; off >= 1; off >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, off));
-      int keep = o + best;
-      if (keep >= J) keep -= J;
-      int removed = 0;
-      for (int jb = 0; jb < J; jb += 32 * U) {
-        int v[U], d[U];
-#pragma unroll
-        for (int k = 0; k < U; ++k) {
-          const int j = jb + 32 * k + lane;
-          v[k] = (j < J) ? (int)col[(size_t)j * NN] : 0;
-          d[k] = (j < J) ? (int)df[j] : 0;
-        }
-#pragma unroll
-        for (int k = 0; k < U; ++k) {
-          const int j = jb + 32 * k + lane;
-          if (d[k] && v[k] > 0 && j != keep) {
-            col[(size_t)j * NN] = 0;
-            removed += v[k];
-            summ_update(a, cl, j, nn, v[k], 0);
-          }
-        }
-      }
-      tot -= warp_sum(removed);
-    }
-    int excess = tot - cap_n;
-    if (excess > 0) {
-      const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J);
-      constexpr int C = 4;   // chunks of 32 jobs loaded together
-      for (int t0 = 0; t0 < J && excess > 0; t0 += 32 * C) {
-        int v[C], jj[C];
-#pragma unroll
-        for (int k = 0; k < C; ++k) {
-          const int t = t0 + 32 * k + lane;
-          int j = o + t;
-          if (j >= J) j -= J;
-          jj[k] = j;
-          v[k] = (t < J) ? (int)col[(size_t)j * NN] : 0;
-        }
-#pragma unroll
-        for (int k = 0; k < C; ++k) {
-          if (excess <= 0) break;
-          int s = v[k];                                // inclusive prefix over the 32 jobs
-#pragma unroll
-          for (int off = 1; off < 32; off <<= 1) {
-            const int u = __shfl_up_sync(0xffffffffu, s, off);
-            if (lane >= off) s += u;
-          }
-          const int take = min(v[k], max(excess - (s - v[k]), 0));
-          if (take > 0) {
-            col[(size_t)jj[k] * NN] = (int16_t)(v[k] - take);
-            summ_update(a, cl, jj[k], nn, v[k], v[k] - take);
-          }
-          excess -= __shfl_sync(0xffffffffu, s, 31);
-        }
-      }
-    }
-  }
-}
-
-// Repair of one column from the occupant lists of the row kernel: one occupant per lane, no
-// pass over the column.  Falls back to the column scan when a batch overflowed its slots
-// or the node has more than 32 occupants.
-__device__ void repair_column_list(const ColfixArgs &a, int cl, int nn, int tot, int ne, int cap_n, int lane) {
-  const uint32_t c = a.first_cand + (uint32_t)cl;
-  const int J = a.J, NN = a.num_nodes;
-  uint32_t entry = 0;
-  int have_n = 0;
-  bool overflow = false;
-  for (int b = 0; b < a.nbatch; ++b) {
-    const size_t at = ((size_t)cl * a.nbatch + b) * NN + nn;
-    const int cb = a.occ_count[at];
-    overflow |= cb > OCC_SLOTS;
-    const int take_n = min(cb, OCC_SLOTS);
-    if (lane >= have_n && lane < have_n + take_n) entry = a.occ_list[at * OCC_SLOTS + (lane - have_n)];
-    have_n += take_n;
-  }
-  if (overflow || have_n > 32) {
-    repair_column_any(a, cl, nn, tot, ne, cap_n, lane);
-    return;
-  }
-  const bool have = lane < have_n;
-  const int j = (int)(entry & 0xFFFFFu);
-  int v = have ? (int)((entry >> 20) & 0x7FFu) : 0;
-  const bool dist = have && (entry >> 31);
-  int16_t *col = a.pop + (size_t)cl * J * NN + nn;
-  if (ne >= 2) {
-    const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
-    int t = J;
-    if (dist && v > 0) { t = j - o; if (t < 0) t += J; }
-    int best = t;
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, off));
-    int removed = 0;
-    if (dist && v > 0 && t != best) {
-      col[(size_t)j * NN] = 0;
-      summ_update(a, cl, j, nn, v, 0);
-      removed = v;
-      v = 0;
-    }
-    tot -= warp_sum(removed);
-  }
-  const int excess = tot - cap_n;
-  if (excess > 0) {
-    const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J);
-    int rot = 0x7fffffff;
-    if (have) { rot = j - o; if (rot < 0) rot += J; }
-    int ahead = 0;                       // GPUs of the occupants that come first in rotated order
-#pragma unroll
-    for (int k = 0; k < 32; ++k) {
-      const int rk = __shfl_sync(0xffffffffu, rot, k);
-      const int vk = __shfl_sync(0xffffffffu, v, k);
-      if (rk < rot) ahead += vk;
-    }
-    const int take = have ? min(v, max(excess - ahead, 0)) : 0;
-    if (take > 0) {
-      col[(size_t)j * NN] = (int16_t)(v - take);
-      summ_update(a, cl, j, nn, v, v - take);
-    }
   }
 }
 
@@ -890,13 +947,12 @@ int launch_rows(sched_ctx *ctx, RowsArgs &a) {
   return SCHED_OK;
 }
 
-int launch_cols(sched_ctx *ctx, int16_t *pop, int count, uint32_t first_cand, uint32_t round,
-                uint32_t gen) {
+int launch_cols(sched_ctx *ctx, int16_t *pop, int count, uint32_t first_cand, uint32_t gen) {
   if (count == 0 || ctx->cfg.num_jobs == 0) return SCHED_OK;
   ColsArgs a;
   a.pop = pop; a.dflag = ctx->d_dflag; a.cap = ctx->d_cap;
   a.J = ctx->cfg.num_jobs; a.num_nodes = ctx->cfg.num_nodes;
-  a.gen = gen; a.key = make_key(ctx->cfg.seed, round);
+  a.gen = gen; a.key = make_key(ctx->cfg.seed, ctx->d_round);
   for (int first = 0; first < count; first += 65535) {
     const int n = min(65535, count - first);
     a.count = n;
@@ -913,14 +969,14 @@ int launch_cols(sched_ctx *ctx, int16_t *pop, int count, uint32_t first_cand, ui
 // Row pass + column pass of `count` candidates.  Rows of a multiple of 8 and at most 512
 // nodes (16-byte vectors, <= 2 per lane) with node sizes <= 2047 take the batched kernels
 // with fused column sums; everything else the general warp-per-row / thread-per-column pair.
-int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint32_t first_cand,
-                     uint32_t round, uint32_t gen) {
+int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint32_t first_cand, uint32_t gen) {
   if (count == 0 || a.J == 0) return SCHED_OK;
   const int NN = a.num_nodes;
   const bool aligned = ((((uintptr_t)a.dst | (uintptr_t)a.src | (uintptr_t)a.cur) & 15) == 0);
   const bool fused = (NN % 8 == 0) && NN <= 512 && aligned && ctx->cap_max <= 2047 && count <= 65535 &&
                      a.J <= (1 << 20);
   ctx->summ_valid = fused && a.summ != nullptr;
+  ctx->fit_done = false;
   if (!fused) {
     if (a.mode == ROWS_GENERATION) {
       {
@@ -931,7 +987,7 @@ int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint3
     }
     int rc = launch_rows(ctx, a);
     if (rc != SCHED_OK) return rc;
-    return launch_cols(ctx, pop, count, first_cand, round, gen);
+    return launch_cols(ctx, pop, count, first_cand, gen);
   }
   const int nbatch = (a.J + 255) / 256;
   int rc = ensure_colscratch(ctx, (size_t)count * nbatch * NN);
@@ -941,6 +997,12 @@ int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint3
   aa.colsum = ctx->d_colsum; aa.colelig = ctx->d_colelig; aa.nbatch = nbatch;
   aa.list_count = ctx->d_colcount;
   aa.occ_count = ctx->d_occcount; aa.occ_list = ctx->d_occlist;
+  aa.fuse = (nbatch == 1 && ctx->ff_on) ? 1 : 0;
+  aa.tp.table = ctx->ff_table; aa.tp.pen = ctx->ff_pen; aa.tp.active = ctx->ff_active;
+  aa.tp.k_max = ctx->cfg.k_max; aa.tp.n_max = ctx->cfg.n_max; aa.tp.mode = fitness_mode(ctx->ff_p);
+  aa.tp.p = ctx->ff_p; aa.tp.floor_ = ctx->cfg.speedup_floor;
+  aa.fitness_out = ctx->ff_out;
+  ctx->fit_done = aa.fuse != 0;
   dim3 grid((unsigned)nbatch, (unsigned)count);
   {
     TimedLaunch tl_(ctx, KK_ROWS);
@@ -967,11 +1029,12 @@ int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint3
 #undef ROWS2
   }
   SCHED_LAUNCH_CHECK(ctx);
+  if (aa.fuse) return SCHED_OK;   // the block did the column pass and the fitness itself
   ColfixArgs f;
   f.pop = pop; f.dflag = ctx->d_dflag; f.cap = ctx->d_cap;
   f.colsum = ctx->d_colsum; f.colelig = ctx->d_colelig; f.summ = a.summ;
   f.J = a.J; f.num_nodes = NN; f.nbatch = nbatch;
-  f.gen = gen; f.first_cand = first_cand; f.key = make_key(ctx->cfg.seed, round);
+  f.gen = gen; f.first_cand = first_cand; f.key = make_key(ctx->cfg.seed, ctx->d_round);
   f.list = ctx->d_collist; f.list_count = ctx->d_colcount;
   f.cur = a.cur; f.occ_count = ctx->d_occcount; f.occ_list = ctx->d_occlist;
   dim3 g2((unsigned)((NN + 127) / 128), (unsigned)count);
@@ -990,7 +1053,7 @@ RowsArgs base_rows_args(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d
   a.P = c.population; a.J = c.num_jobs; a.num_nodes = c.num_nodes;
   a.k_max = c.k_max; a.n_max = c.n_max; a.num_elite = c.num_elite; a.count = count;
   a.thr = 0; a.gen = 0; a.first_cand = 0;
-  a.key = make_key(c.seed, 0);
+  a.key = make_key(c.seed, ctx->d_round);
   a.src = nullptr; a.dst = nullptr; a.mode = ROWS_REPAIR; a.fitness_bits = nullptr;
   a.cur = nullptr; a.summ = nullptr;
   return a;
@@ -999,39 +1062,47 @@ RowsArgs base_rows_args(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d
 }  // namespace
 
 int launch_repair(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active, int16_t *d_pop,
-                  int32_t count, uint32_t first_candidate, uint32_t round, uint32_t generation) {
+                  int32_t count, uint32_t first_candidate, uint32_t generation) {
   int rc = ensure_dflag(ctx, count);
   if (rc != SCHED_OK) return rc;
   RowsArgs a = base_rows_args(ctx, d_k_cap, d_active, count);
   a.mode = ROWS_REPAIR; a.src = d_pop; a.dst = d_pop;
-  a.first_cand = first_candidate; a.gen = generation; a.key = make_key(ctx->cfg.seed, round);
-  return launch_rows_cols(ctx, a, d_pop, count, first_candidate, round, generation);
+  a.first_cand = first_candidate; a.gen = generation; a.key = make_key(ctx->cfg.seed, ctx->d_round);
+  return launch_rows_cols(ctx, a, d_pop, count, first_candidate, generation);
 }
 
 int launch_init_population(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active,
-                           const int16_t *d_cur, uint32_t round, int16_t *d_pop_out) {
+                           const int16_t *d_cur, int16_t *d_pop_out) {
   const int P = ctx->cfg.population;
   int rc = ensure_dflag(ctx, P);
   if (rc != SCHED_OK) return rc;
   RowsArgs a = base_rows_args(ctx, d_k_cap, d_active, P);
   a.mode = ROWS_INIT; a.src = d_cur; a.dst = d_pop_out;
-  a.thr = ctx->cfg.thr_init; a.gen = GEN_INIT; a.key = make_key(ctx->cfg.seed, round);
+  a.thr = ctx->cfg.thr_init; a.gen = GEN_INIT; a.key = make_key(ctx->cfg.seed, ctx->d_round);
   a.cur = ctx->round_cur; a.summ = ctx->round_summ;
-  return launch_rows_cols(ctx, a, d_pop_out, P, 0u, round, GEN_INIT);
+  return launch_rows_cols(ctx, a, d_pop_out, P, 0u, GEN_INIT);
 }
 
 int launch_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active,
                       const int16_t *d_pop_in, const float *d_fitness_in, int16_t *d_pop_out,
-                      uint32_t round, uint32_t generation) {
+                      uint32_t generation) {
   const int P = ctx->cfg.population;
   int rc = ensure_dflag(ctx, P);
   if (rc != SCHED_OK) return rc;
   RowsArgs a = base_rows_args(ctx, d_k_cap, d_active, P);
   a.mode = ROWS_GENERATION; a.src = d_pop_in; a.dst = d_pop_out;
   a.fitness_bits = (const uint32_t *)d_fitness_in;
-  a.thr = ctx->cfg.thr_mutate; a.gen = generation; a.key = make_key(ctx->cfg.seed, round);
+  a.thr = ctx->cfg.thr_mutate; a.gen = generation; a.key = make_key(ctx->cfg.seed, ctx->d_round);
   a.cur = ctx->round_cur; a.summ = ctx->round_summ;
-  return launch_rows_cols(ctx, a, d_pop_out, P, 0u, round, generation);
+  return launch_rows_cols(ctx, a, d_pop_out, P, 0u, generation);
+}
+
+__global__ void set_round_kernel(uint32_t *dst, uint32_t value) { *dst = value; }
+
+int launch_set_round(sched_ctx *ctx, uint32_t round) {
+  set_round_kernel<<<1, 1, 0, ctx->stream>>>(ctx->d_round, round);
+  SCHED_LAUNCH_CHECK(ctx);
+  return SCHED_OK;
 }
 
 int launch_select_best(sched_ctx *ctx, const int16_t *d_pop, const float *d_fitness,
