@@ -549,7 +549,7 @@ __device__ void repair_column_list(const ColfixArgs &a, int cl, int nn, int tot,
 
 // VPL = 16-byte vectors per lane; a row is split over LPR = 1 << LPR_LOG2 lanes
 // (LPR * VPL >= row_vecs, FULL when equal), so a warp works on 32 / LPR rows at a time.
-template <int LPR_LOG2, int VPL, bool FULL>
+template <int LPR_LOG2, int VPL, bool FULL, bool FUSE>
 __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
   const RowsArgs &a = aa.r;
   constexpr int MAXN = 8 * (1 << LPR_LOG2) * VPL;   // nodes this instantiation can hold
@@ -671,6 +671,10 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
       const int v = sub + LPR * q;
       raw[q] = make_uint4(0, 0, 0, 0);
       if (on && (FULL || v < row_vecs)) raw[q] = __ldg((const uint4 *)(src + (size_t)r * NN) + v);
+      // the matching piece of the current allocation is read late in the iteration: pull it
+      // towards L1 now, without tying up registers
+      if (cur0 && r < nrows && (FULL || v < row_vecs))
+        asm volatile("prefetch.global.L1 [%0];" ::"l"((const uint4 *)(cur0 + (size_t)r * NN) + v));
     }
   };
   if (nrows > 0) fetch(grp);
@@ -829,13 +833,13 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
       a.dflag[(size_t)cl * J + j] = (on && dist) ? 1 : 0;
       // row summary for the fitness: K | N << 11 | (entries that differ from current) << 22
       const uint32_t word = on ? ((uint32_t)K | ((uint32_t)N << 11) | ((uint32_t)ndiff << 22)) : 0u;
-      s_summ[warp * 32 + r] = word;
-      if (a.summ && !aa.fuse) a.summ[(size_t)cl * J + j] = word;
+      if (FUSE) s_summ[warp * 32 + r] = word;
+      if (!FUSE && a.summ) a.summ[(size_t)cl * J + j] = word;
     }
   }
 
   __syncthreads();
-  if (aa.fuse) {
+  if (FUSE) {
     // ---- the whole candidate lives in this block: column pass and fitness right here ---------
     ColfixArgs f;
     f.pop = a.dst; f.dflag = a.dflag; f.cap = a.cap; f.cur = a.cur;
@@ -1015,8 +1019,13 @@ int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint3
     const bool full = (vpl << lpr_log2) == row_vecs && (vpl == 1 || vpl == 2 || vpl == 4);
 #define ROWS2(L, V)                                                            \
   do {                                                                         \
-    if (full) rows2_kernel<L, V, true><<<grid, 256, 0, ctx->stream>>>(aa);     \
-    else rows2_kernel<L, V, false><<<grid, 256, 0, ctx->stream>>>(aa);         \
+    if (aa.fuse) {                                                             \
+      if (full) rows2_kernel<L, V, true, true><<<grid, 256, 0, ctx->stream>>>(aa);    \
+      else rows2_kernel<L, V, false, true><<<grid, 256, 0, ctx->stream>>>(aa);        \
+    } else {                                                                   \
+      if (full) rows2_kernel<L, V, true, false><<<grid, 256, 0, ctx->stream>>>(aa);   \
+      else rows2_kernel<L, V, false, false><<<grid, 256, 0, ctx->stream>>>(aa);       \
+    }                                                                          \
   } while (0)
     if (lpr_log2 == 0) {
       if (vpl <= 1) ROWS2(0, 1);
