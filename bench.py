@@ -40,9 +40,12 @@ FP32_LANES_PER_SM = 128          # CUDA cores per SM (compute capability 10.0)
 OPS_PER_POINT = 10               # fp32 lane-ops counted as useful per (job, K, class, m, s) point
 HBM_FALLBACK_GBS = 6650.0
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
-# captures summarised under profiles/; None = kernel changed since the counters were taken.
-NCU_TRAFFIC_BYTES = {"rows": None, "cols": None, "fitness": None, "fitness_stress": None}
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+# summarised in profiles/kernel_counters.md; None = kernel changed since the counters were taken.
+# "rows": one large-workload generation (234.7 MB read + 242.2 MB written).
+# "fitness_stress": 16 dense stress candidates moved 544.8 + 3.0 MB; every candidate is streamed
+# once, so the figure is scaled by candidates / 16 to the chunk that is timed.
+NCU_TRAFFIC_BYTES = {"rows": 476.9e6, "fitness_stress_per_candidate": 547.8e6 / 16}
 
 
 def measured_peaks():
@@ -344,7 +347,8 @@ def bench_stress(api, torch, dev, stream, hbm_peak, peak_src, args):
     out["roofline"] = {"kernel": "fitness", "bound": "hbm", "achieved": round(best[0], 1), "peak": hbm_peak,
                        "peak_source": "MEASURED_PEAKS.json hbm_gbs" if peak_src == "measured" else "recipe fallback",
                        "unit": "GB/s", "frac": round(best[0] / hbm_peak, 4), "frac_of_8tbs_nominal": round(best[0] / 8000.0, 4),
-                       "traffic": NCU_TRAFFIC_BYTES.get("fitness_stress"),
+                       "traffic": NCU_TRAFFIC_BYTES["fitness_stress_per_candidate"] * chunk,
+                       "traffic_note": "ncu capture of 16 candidates scaled by candidates / 16",
                        "algorithmic_bytes_per_launch": chunk * bytes_per_cand, "note": "slowest of the three exponents"}
     sched.close()
     del pop, table
