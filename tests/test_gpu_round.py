@@ -77,6 +77,43 @@ def test_round_equals_stepwise_calls_and_oracle_fitness(gpu, oracle, cfg):
     s.close()
 
 
+def test_large_config_round_equals_stepwise(gpu, oracle):
+    """The large configuration (batched row kernel, work-list column repair, fitness from row
+    summaries) for three generations: the round must equal the entry points called one by one,
+    whose fitness reads the dense matrices; the final fitness is checked against the oracle on a
+    sample of candidates."""
+    torch, api = gpu
+    cfg = synth.LARGE
+    cl, jobs = setup(cfg)
+    cur = cfg.cur()
+    s, dj, best, bf, pop, fit = _round(gpu, cfg, jobs, cur, 3, rnd=7)
+    dev = "cuda:0"
+    sp = torch.empty(s.table_shape, dtype=torch.float32, device=dev)
+    s.build_speedup_table(dj, None, sp, None)
+    rf = torch.empty(cfg.num_jobs, dtype=torch.float32, device=dev)
+    s.compute_realloc_factor(dj, rf)
+    d_cur = torch.from_numpy(cur).cuda()
+    a = torch.empty((cfg.population, cfg.num_jobs, cfg.num_nodes), dtype=torch.int16, device=dev)
+    b = torch.empty_like(a)
+    f = torch.empty(cfg.population, dtype=torch.float32, device=dev)
+    s.init_population(dj, d_cur, a, round=7)
+    s.eval_fitness(a, sp, f, p=cfg.p, cur=d_cur, realloc_factor=rf, active=dj.tensors["active"])
+    for g in range(3):
+        s.ga_generation(dj, a, f, b, round=7, generation=g)
+        a, b = b, a
+        s.eval_fitness(a, sp, f, p=cfg.p, cur=d_cur, realloc_factor=rf, active=dj.tensors["active"])
+    assert np.array_equal(a.cpu().numpy(), pop)
+    assert np.array_equal(f.cpu().numpy().view(np.uint32), fit.view(np.uint32))
+    sample = [0, 1, 100, 511]
+    ref = oracle.eval_fitness(pop[sample], sp.cpu().numpy().astype(np.float64), cl.k_max, cl.n_max, cfg.p,
+                              cfg.speedup_floor, cur=cur, realloc=rf.cpu().numpy().astype(np.float64),
+                              active=jobs.active)
+    assert_close(fit[sample], ref, what="large round fitness")
+    for c in sample:
+        assert feasible(pop[c], cl.node_capacity, jobs.k_cap, cl.n_max)
+    s.close()
+
+
 def test_round_is_reproducible_and_round_number_matters(gpu):
     cfg = synth.TESTBED
     cl, jobs = setup(cfg)
