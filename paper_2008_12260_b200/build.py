@@ -36,11 +36,34 @@ def _stale() -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB
+    from concurrent.futures import ThreadPoolExecutor
+
     nvcc = os.environ.get("NVCC", "nvcc")
+    objdir = os.path.join(HERE, "_build")
+    os.makedirs(objdir, exist_ok=True)
+    common = [f for f in NVCC_FLAGS if f not in ("--shared", "-cudart", "static")]
+    common += (["-Xptxas", "-v"] if verbose else []) + ["-I", INCLUDE, "-I", CSRC]
+
+    def compile_one(src):
+        obj = os.path.join(objdir, os.path.basename(src) + ".%d.o" % os.getpid())
+        res = subprocess.run([nvcc] + common + ["-c", "-o", obj, src], capture_output=True, text=True)
+        return src, obj, res
+
+    with ThreadPoolExecutor(max_workers=4) as ex:          # one nvcc per translation unit
+        results = list(ex.map(compile_one, sources()))
+    objs = []
+    for src, obj, res in results:
+        if verbose or res.returncode != 0:
+            sys.stderr.write(res.stdout + res.stderr)
+        if res.returncode != 0:
+            raise subprocess.CalledProcessError(res.returncode, "nvcc -c " + src)
+        objs.append(obj)
     tmp = LIB + ".tmp%d" % os.getpid()
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-I", INCLUDE, "-I", CSRC, "-o", tmp] + sources()
-    subprocess.check_call(cmd)
+    subprocess.check_call([nvcc, "--shared", "-cudart", "static", "-gencode", "arch=compute_100a,code=sm_100a",
+                           "-o", tmp] + objs)
     os.replace(tmp, LIB)
+    for obj in objs:
+        os.remove(obj)
     return LIB
 
 
