@@ -100,14 +100,54 @@ goodput_sweep_kernel(JobPtrs jp, const int32_t *__restrict__ m_grid,
       bd[q] = 1.f;
     }
     float u = 1.f;
-#pragma unroll 4
-    for (int s = 0; s < Gs; ++s, u += 1.f) {
+    if (MQ >= 2) {
+      // two grid points per instruction: sm_100's packed fp32 FMA / MUL work on register
+      // pairs and halve the issue slots of the arithmetic (same roundings as the scalar ops)
+      constexpr int H = MQ >= 2 ? MQ / 2 : 1;
+      float2 tg2[H], ta2[H], kr2[H], bu2[H], bd2[H];
 #pragma unroll
-      for (int q = 0; q < MQ; ++q) {
-        const float den = fmaf(u, tg[q], ta[q]) * fmaf(u, kr[q], c0);
+      for (int h = 0; h < H; ++h) {
+        tg2[h] = make_float2(tg[2 * h], tg[2 * h + (MQ >= 2)]);
+        ta2[h] = make_float2(ta[2 * h], ta[2 * h + (MQ >= 2)]);
+        kr2[h] = make_float2(kr[2 * h], kr[2 * h + (MQ >= 2)]);
+        bu2[h] = make_float2(0.f, 0.f);
+        bd2[h] = make_float2(1.f, 1.f);
+      }
+      const float2 c02 = make_float2(c0, c0);
+#pragma unroll 4
+      for (int s = 0; s < Gs; ++s, u += 1.f) {
+        const float2 u2 = make_float2(u, u);
+#pragma unroll
+        for (int h = 0; h < H; ++h) {
+          const float2 den2 = __fmul2_rn(__ffma2_rn(u2, tg2[h], ta2[h]), __ffma2_rn(u2, kr2[h], c02));
+          const float2 l2 = __fmul2_rn(u2, bd2[h]);
+          const float2 r2 = __fmul2_rn(bu2[h], den2);
+          // per half: if (l > r) { bu = u; bd = den; } with the moves as predicated FMAs
+          // (x * 1 + 0, run-time 1 and 0): compares and selects share the half-rate integer
+          // pipe, and this form measured faster than plain selects
+          asm("{\n"
+              " .reg .pred pa, pb;\n"
+              " setp.gt.f32 pa, %4, %6;\n"
+              " setp.gt.f32 pb, %5, %7;\n"
+              " @pa fma.rn.f32 %0, %8, %11, %12;\n"
+              " @pa fma.rn.f32 %2, %9, %11, %12;\n"
+              " @pb fma.rn.f32 %1, %8, %11, %12;\n"
+              " @pb fma.rn.f32 %3, %10, %11, %12;\n"
+              "}"
+              : "+f"(bu2[h].x), "+f"(bu2[h].y), "+f"(bd2[h].x), "+f"(bd2[h].y)
+              : "f"(l2.x), "f"(l2.y), "f"(r2.x), "f"(r2.y), "f"(u), "f"(den2.x), "f"(den2.y), "f"(one), "f"(zero));
+        }
+      }
+#pragma unroll
+      for (int h = 0; h < H; ++h) {
+        bu[2 * h] = bu2[h].x; bd[2 * h] = bd2[h].x;
+        bu[2 * h + (MQ >= 2)] = bu2[h].y; bd[2 * h + (MQ >= 2)] = bd2[h].y;
+      }
+    } else {
+#pragma unroll 4
+      for (int s = 0; s < Gs; ++s, u += 1.f) {
+        const float den = fmaf(u, tg[0], ta[0]) * fmaf(u, kr[0], c0);
         // if (u * bd > bu * den) { bu = u; bd = den; }   -- u/den > bu/bd
-        // The conditional moves are predicated FMAs (x * 1 + 0 with run-time 1 and 0) so that
-        // they issue on the fp32 pipe; compares and selects share the half-rate integer pipe.
         asm("{\n"
             " .reg .pred pb;\n"
             " .reg .f32 l, r;\n"
@@ -117,7 +157,7 @@ goodput_sweep_kernel(JobPtrs jp, const int32_t *__restrict__ m_grid,
             " @pb fma.rn.f32 %0, %2, %4, %5;\n"
             " @pb fma.rn.f32 %1, %3, %4, %5;\n"
             "}"
-            : "+f"(bu[q]), "+f"(bd[q])
+            : "+f"(bu[0]), "+f"(bd[0])
             : "f"(u), "f"(den), "f"(one), "f"(zero));
       }
     }
