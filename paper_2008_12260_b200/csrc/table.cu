@@ -5,6 +5,8 @@
 // whether one or several nodes are occupied (Eq. 9), so the sweep runs once per
 // (job, K, class) with class in {local, node}; a second kernel broadcasts the class
 // results along the N axis of the [J][K][N] tables and divides by the fair-share entry.
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace {
@@ -207,32 +209,35 @@ __device__ __forceinline__ bool kn_valid(int K, int N, int k_max, int n_max,
 }
 
 // Broadcast the class results along N and divide by the fair-share goodput (Eq. 15).
+// Block = a 32-wide stripe of N of one job's slab (blockIdx.z = job); its 8 thread rows walk K.
 __global__ void __launch_bounds__(256)
 speedup_expand_kernel(const float *__restrict__ gmax, const uint16_t *__restrict__ amax,
                       const int32_t *__restrict__ kfit, const int32_t *__restrict__ fair_k,
-                      const int32_t *__restrict__ fair_n, int J, int k_max, int n_max,
+                      const int32_t *__restrict__ fair_n, int j_first, int k_max, int n_max,
                       float *__restrict__ goodput, float *__restrict__ speedup,
                       uint16_t *__restrict__ argmax) {
   const int KD = k_max + 1, ND = n_max + 1;
-  const long long total = (long long)J * KD * ND;
-  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= total) return;
-  const int N = (int)(e % ND);
-  const int K = (int)((e / ND) % KD);
-  const int j = (int)(e / ((long long)ND * KD));
-  float g = 0.f;
-  uint16_t a = 0xFFFFu;
-  if (kn_valid(K, N, k_max, n_max, kfit)) {
-    const size_t src = ((size_t)j * KD + K) * 2 + (N >= 2 ? 1 : 0);
-    g = gmax[src];
-    a = amax[src];
-  }
+  const int N = blockIdx.x * 32 + threadIdx.x;
+  const int j = j_first + blockIdx.z;
+  if (N >= ND) return;
   const int kf = fair_k[j], nf = fair_n[j];
   float denom = 0.f;
   if (kn_valid(kf, nf, k_max, n_max, kfit)) denom = gmax[((size_t)j * KD + kf) * 2 + (nf >= 2 ? 1 : 0)];
-  if (goodput) goodput[e] = g;
-  if (argmax) argmax[e] = a;
-  speedup[e] = denom > 0.f ? g / denom : 0.f;
+  const int kfitN = (N >= 1 && N <= n_max) ? kfit[N] : -1;
+#pragma unroll 4
+  for (int K = threadIdx.y; K < KD; K += 8) {
+    const size_t e = ((size_t)j * KD + K) * ND + N;
+    float g = 0.f;
+    uint16_t a = 0xFFFFu;
+    if (K >= N && K <= kfitN && N >= 1) {
+      const size_t src = ((size_t)j * KD + K) * 2 + (N >= 2 ? 1 : 0);
+      g = gmax[src];
+      a = amax[src];
+    }
+    if (goodput) goodput[e] = g;
+    if (argmax) argmax[e] = a;
+    speedup[e] = denom > 0.f ? g / denom : 0.f;
+  }
 }
 
 // REALLOC_FACTOR_j(delta) = (T_j - R_j delta) / (T_j + delta), clamped to [0, 1].
@@ -270,14 +275,16 @@ int launch_speedup_table(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodpu
 #undef SWEEP
     SCHED_LAUNCH_CHECK(ctx);
   }
-  const long long entries = (long long)J * ctx->KD * ctx->ND;
-  {
-  TimedLaunch tl_(ctx, KK_EXPAND);
-  speedup_expand_kernel<<<(unsigned)((entries + 255) / 256), 256, 0, ctx->stream>>>(
-      ctx->d_gmax, ctx->d_amax, ctx->d_kfit, jobs->fair_k, jobs->fair_n, J, c.k_max, c.n_max,
-      d_goodput, d_speedup, d_argmax);
+  for (int j0 = 0; j0 < J; j0 += 65535) {      // grid.z is limited to 65535 jobs per launch
+    dim3 grid((unsigned)((ctx->ND + 31) / 32), 1u, (unsigned)std::min(65535, J - j0));
+    {
+      TimedLaunch tl_(ctx, KK_EXPAND);
+      speedup_expand_kernel<<<grid, dim3(32, 8), 0, ctx->stream>>>(ctx->d_gmax, ctx->d_amax, ctx->d_kfit,
+                                                                   jobs->fair_k, jobs->fair_n, j0, c.k_max, c.n_max,
+                                                                   d_goodput, d_speedup, d_argmax);
+    }
+    SCHED_LAUNCH_CHECK(ctx);
   }
-  SCHED_LAUNCH_CHECK(ctx);
   return SCHED_OK;
 }
 
