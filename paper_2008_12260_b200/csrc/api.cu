@@ -83,7 +83,7 @@ int ensure_round_scratch(sched_ctx *ctx) {
   if ((rc = dev_alloc(ctx, &ctx->d_tab_goodput, tab)) != SCHED_OK) return rc;
   if ((rc = dev_alloc(ctx, &ctx->d_tab_speedup, tab)) != SCHED_OK) return rc;
   if ((rc = dev_alloc(ctx, &ctx->d_rf, (size_t)c.num_jobs)) != SCHED_OK) return rc;
-  if ((rc = dev_alloc(ctx, &ctx->d_summ, (size_t)c.population * c.num_jobs)) != SCHED_OK) return rc;
+  if ((rc = dev_alloc(ctx, &ctx->d_summ, 2 * (size_t)c.population * c.num_jobs)) != SCHED_OK) return rc;
   ctx->round_ready = true;
   return SCHED_OK;
 }
@@ -406,6 +406,8 @@ static int round_body(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d
   // whenever the batched kernels were used, with bit-identical results.
   ctx->round_cur = rf ? d_cur : nullptr;
   ctx->round_summ = ctx->d_summ;
+  ctx->round_summ_in = nullptr;
+  uint32_t *summ_other = ctx->d_summ + (size_t)ctx->cfg.population * ctx->cfg.num_jobs;
   // the per-job penalty factors depend only on the current allocation: prepared once
   ctx->pen_ready = false;
   rc = SCHED_OK;
@@ -423,12 +425,15 @@ static int round_body(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d
   auto fitness_of = [&](const int16_t *pop, float *out) {
     if (ctx->fit_done) return (int)SCHED_OK;
     return launch_fitness(ctx, pop, ctx->cfg.population, ctx->d_tab_speedup, d_cur, rf, d_jobs->active,
-                          ctx->cfg.p, out, ctx->summ_valid ? ctx->d_summ : nullptr);
+                          ctx->cfg.p, out, ctx->summ_valid ? ctx->round_summ : nullptr);
   };
   if (rc == SCHED_OK) rc = launch_init_population(ctx, d_jobs->k_cap, d_jobs->active, d_cur, pa);
   if (rc == SCHED_OK) rc = fitness_of(pa, fit_cur);
   for (int g = 0; g < generations && rc == SCHED_OK; ++g) {
     ctx->ff_out = fit_next;
+    // children's summaries go to the other half; the parents' feed the unperturbed rows
+    ctx->round_summ_in = ctx->summ_valid ? ctx->round_summ : nullptr;
+    std::swap(ctx->round_summ, summ_other);
     rc = launch_generation(ctx, d_jobs->k_cap, d_jobs->active, pa, fit_cur, pb, (uint32_t)g);
     if (rc != SCHED_OK) break;
     std::swap(pa, pb);
@@ -441,6 +446,7 @@ static int round_body(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d
   ctx->fit_done = false;
   ctx->round_cur = nullptr;
   ctx->round_summ = nullptr;
+  ctx->round_summ_in = nullptr;
   ctx->summ_valid = false;
   if (rc != SCHED_OK) return rc;
   ctx->d_pop_last = pa;

@@ -70,8 +70,9 @@ struct sched_ctx {
   // state of a running schedule_round: the batched row kernel also emits per-row summaries
   // (K, N, differs-from-current) so that the in-round fitness need not re-read the population
   const int16_t *round_cur;  // current allocation of the round (NULL outside a round)
-  uint32_t *round_summ;      // d_summ while a round runs, else NULL
-  uint32_t *d_summ;          // [P][J]
+  uint32_t *round_summ;      // where the running round's row pass writes its summaries, else NULL
+  const uint32_t *round_summ_in;  // summaries of the parent population (the other half), or NULL
+  uint32_t *d_summ;          // [2][P][J]: parents' and children's summaries alternate
   bool summ_valid;           // the last row/column pass filled d_summ
   // fitness fused into the generation kernel (single-batch problems): inputs set by
   // schedule_round, fit_done reports that the last row/column pass also wrote the fitness

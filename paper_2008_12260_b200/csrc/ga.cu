@@ -51,6 +51,7 @@ struct RowsArgs {
   uint8_t *dflag;           // [count][J]
   const int16_t *cur;       // [J][N] current allocation for the summaries' "changed" bit, or NULL
   uint32_t *summ;           // [count][J] row summaries (batched kernels only), or NULL
+  const uint32_t *summ_in;  // [P][J] summaries of the parents (generation mode), or NULL
   int mode, P, J, num_nodes, k_max, n_max, num_elite, count;
   uint32_t thr, gen, first_cand;
   RngKey key;
@@ -661,11 +662,20 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
 
   // Iterations are software-pipelined: the loads of the next RPI rows are issued before the
   // current ones are processed.
+  // An unperturbed child row is a verbatim copy of a parent's row, whose summary (K, N, entries
+  // differing from the current allocation; kept exact by the column pass) is already known:
+  // such rows skip the row totals and the comparison with the current allocation.
+  const bool inherit = !FUSE && a.mode == ROWS_GENERATION && a.summ_in != nullptr;
+  const uint32_t *sin_a = inherit ? a.summ_in + (size_t)s_parent[0] * J + j0 : nullptr;
+  const uint32_t *sin_b = inherit ? a.summ_in + (size_t)s_parent[1] * J + j0 : nullptr;
   uint4 raw[VPL];
+  uint32_t pword = 0;
   auto fetch = [&](int r) {   // r = this lane's row within the warp's 32 (may be >= nrows)
     const uint32_t fl = __shfl_sync(0xffffffffu, flags_l, r & 31);
     const int16_t *src = (fl & 4u) ? src_b : src_a;
     const bool on = r < nrows && (fl & 2u) && src;
+    const bool copy = inherit && !(fl & 1u);
+    if (copy && on && sub == 0) pword = __ldg(((fl & 4u) ? sin_b : sin_a) + r);
 #pragma unroll
     for (int q = 0; q < VPL; ++q) {
       const int v = sub + LPR * q;
@@ -673,7 +683,7 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
       if (on && (FULL || v < row_vecs)) raw[q] = __ldg((const uint4 *)(src + (size_t)r * NN) + v);
       // the matching piece of the current allocation is read late in the iteration: pull it
       // towards L1 now, without tying up registers
-      if (cur0 && r < nrows && (FULL || v < row_vecs))
+      if (cur0 && !copy && r < nrows && (FULL || v < row_vecs))
         asm volatile("prefetch.global.L1 [%0];" ::"l"((const uint4 *)(cur0 + (size_t)r * NN) + v));
     }
   };
@@ -709,18 +719,26 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
       x[q] = make_uint4(0, 0, 0, 0);
       if (FULL || v < row_vecs) x[q] = clamp_vec(raw[q], ((const uint4 *)s_cap)[v]);
     }
+    const bool copy = inherit && act && !(flags & 1u);       // uniform within the row's lanes
+    const uint32_t pw = __shfl_sync(0xffffffffu, pword, grp << LPR_LOG2);
     if (r0 + RPI < nrows) fetch(r0 + RPI + grp);
 
-    uint32_t part = 0;
+    const bool compute = __any_sync(0xffffffffu, live && !copy);   // some row of this iteration needs totals
+    int K = 0, N = 0;
+    if (compute) {
+      uint32_t part = 0;
 #pragma unroll
-    for (int q = 0; q < VPL; ++q) part += row_partial(x[q]);
-    part = __reduce_add_sync(gmask, part);
-    int K = (int)(part & 0x3FFFFFu), N = (int)(part >> 22);
+      for (int q = 0; q < VPL; ++q) part += row_partial(x[q]);
+      part = __reduce_add_sync(gmask, part);
+      K = (int)(part & 0x3FFFFFu);
+      N = (int)(part >> 22);
+    }
+    if (copy) { K = (int)(pw & 0x7FFu); N = (int)((pw >> 11) & 0x7FFu); }
     const int kc = (int)(flags >> 3);
 
     // rows that are perturbed or break a row cap take a detour through shared memory, one
     // row at a time with the whole warp
-    unsigned need = __ballot_sync(0xffffffffu, act && sub == 0 && ((flags & 1u) || K > kc || N > a.n_max));
+    unsigned need = __ballot_sync(0xffffffffu, act && !copy && sub == 0 && ((flags & 1u) || K > kc || N > a.n_max));
     while (need) {
       const int leader = __ffs(need) - 1;         // lane `leader` is sub 0 of the row's group
       need &= need - 1;
@@ -813,7 +831,7 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
         s_qmeta[warp][pos] = (uint32_t)j | ((uint32_t)v << 20) | (dist ? 0x80000000u : 0u);   // v < 64
       }
       qn += __popc(bal);
-      if (cur0 && in) {
+      if (cur0 && in && !copy) {
         const uint4 cx = __ldg((const uint4 *)(cur0 + (size_t)r * NN) + v);
         const uint4 d = make_uint4(x[q].x ^ cx.x, x[q].y ^ cx.y, x[q].z ^ cx.z, x[q].w ^ cx.w);
         if ((d.x | d.y | d.z | d.w) != 0u) {
@@ -827,7 +845,8 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
     }
     flush_queue(qn);
     qn = 0;
-    if (cur0) ndiff = __reduce_add_sync(gmask, ndiff);
+    if (cur0 && compute) ndiff = __reduce_add_sync(gmask, ndiff);
+    if (copy) ndiff = (int)(pw >> 22);
     if (live && sub == 0) {
       const bool on = (flags & 2u) != 0u;
       a.dflag[(size_t)cl * J + j] = (on && dist) ? 1 : 0;
@@ -1064,7 +1083,7 @@ RowsArgs base_rows_args(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d
   a.thr = 0; a.gen = 0; a.first_cand = 0;
   a.key = make_key(c.seed, ctx->d_round);
   a.src = nullptr; a.dst = nullptr; a.mode = ROWS_REPAIR; a.fitness_bits = nullptr;
-  a.cur = nullptr; a.summ = nullptr;
+  a.cur = nullptr; a.summ = nullptr; a.summ_in = nullptr;
   return a;
 }
 
@@ -1102,7 +1121,7 @@ int launch_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_a
   a.mode = ROWS_GENERATION; a.src = d_pop_in; a.dst = d_pop_out;
   a.fitness_bits = (const uint32_t *)d_fitness_in;
   a.thr = ctx->cfg.thr_mutate; a.gen = generation; a.key = make_key(ctx->cfg.seed, ctx->d_round);
-  a.cur = ctx->round_cur; a.summ = ctx->round_summ;
+  a.cur = ctx->round_cur; a.summ = ctx->round_summ; a.summ_in = ctx->round_summ_in;
   return launch_rows_cols(ctx, a, d_pop_out, P, 0u, generation);
 }
 
