@@ -129,6 +129,13 @@ int ensure_dflag(sched_ctx *ctx, int32_t count) {
 }
 
 int ensure_colscratch(sched_ctx *ctx, size_t ints) {
+  const size_t tickets = (size_t)65536;   // one per candidate of a launch
+  if (!ctx->d_rowticket) {
+    int rc = dev_alloc(ctx, &ctx->d_rowticket, tickets);
+    if (rc != SCHED_OK) return rc;
+    SCHED_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->d_rowticket, 0, tickets * sizeof(unsigned int), ctx->stream));
+    ctx->rowticket_cap = tickets;
+  }
   if (ints > ctx->col_cap) {
     if (ctx->d_colsum || ctx->d_colelig) {
       SCHED_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
@@ -255,7 +262,7 @@ int sched_destroy(sched_ctx *ctx) {
   void *ptrs[] = {ctx->d_cap, ctx->d_kfit, ctx->d_pairs, ctx->d_gmax, ctx->d_amax, ctx->d_rank, ctx->d_order,
                   ctx->d_dflag, ctx->d_pen, ctx->d_partial, ctx->d_ticket, ctx->d_status,
                   ctx->d_popA, ctx->d_popB, ctx->d_fit_buf, ctx->d_tab_goodput, ctx->d_tab_speedup,
-                  ctx->d_rf, ctx->d_best_idx, ctx->d_stage, ctx->d_stage_fit, ctx->d_colsum, ctx->d_summ, ctx->d_collist, ctx->d_colcount, ctx->d_round, ctx->d_occcount, ctx->d_occlist,
+                  ctx->d_rf, ctx->d_best_idx, ctx->d_stage, ctx->d_stage_fit, ctx->d_colsum, ctx->d_summ, ctx->d_collist, ctx->d_colcount, ctx->d_rowticket, ctx->d_round, ctx->d_occcount, ctx->d_occlist,
                   ctx->d_colelig};
   for (void *p : ptrs)
     if (p) cudaFree(p);

@@ -62,6 +62,8 @@ struct sched_ctx {
   unsigned int *d_ticket;  // [count] arrival counters of the fitness reduction
   uint32_t *d_collist;   // [count * num_nodes] columns that need repair
   unsigned int *d_colcount;  // [1]
+  unsigned int *d_rowticket; // [count] finished row blocks per candidate (kept at zero between kernels)
+  size_t rowticket_cap;
   int32_t *d_occcount;   // [count][row batches][num_nodes] occupants recorded per node
   uint32_t *d_occlist;   // [count][row batches][num_nodes][8]
   int32_t *d_colsum, *d_colelig;  // [count][row batches][num_nodes] column partials of the row pass

@@ -71,10 +71,35 @@ struct FitnessArgs {
   float *fitness;
 };
 
-// SUMMARY = true: the per-row (K, N, changed) words come from `summ` instead of a pass over
-// the rows; the walk over rows, the lane that owns each row and every reduction are the same,
-// so both modes produce identical bits.
-template <int W, bool SUMMARY>
+// End of a block's work: its terms are added in a fixed order, the chunk sum goes to scratch,
+// and the last block of the candidate to arrive adds the chunk sums in index order and
+// writes the power mean.
+__device__ __forceinline__ void block_finish(const FitnessArgs &a, int cand, int chunk, int j0, int j1,
+                                             const float *s_term) {
+  __syncthreads();
+  double t, n;
+  block_term_sum(s_term, j1 - j0, j0, a.active, t, n);
+  __shared__ bool s_last;
+  if (threadIdx.x == 0) {
+    double *dst = a.partial + ((size_t)cand * a.chunks + chunk) * 2;
+    dst[0] = t;
+    dst[1] = n;
+    __threadfence();
+    const unsigned prev = atomicAdd(a.ticket + cand, 1u);
+    s_last = (prev == (unsigned)a.chunks - 1u);
+  }
+  __syncthreads();
+  if (s_last && threadIdx.x == 0) {
+    __threadfence();
+    const volatile double *src = a.partial + (size_t)cand * a.chunks * 2;
+    double ts = 0.0, ns = 0.0;
+    for (int c = 0; c < a.chunks; ++c) { ts += src[2 * c]; ns += src[2 * c + 1]; }
+    a.fitness[cand] = fitness_finalise(a.mode, a.p, ts, ns);
+    a.ticket[cand] = 0u;   // ready for the next call on this stream
+  }
+}
+
+template <int W>
 __global__ void __launch_bounds__(256) fitness_kernel(FitnessArgs a) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int cand = blockIdx.y, chunk = blockIdx.x;
@@ -102,14 +127,6 @@ __global__ void __launch_bounds__(256) fitness_kernel(FitnessArgs a) {
   for (int jb = j0 + warp * RPW; jb < j1; jb += nwarps * RPW, ++it) {
     const int j = jb + group;
     const bool live = j < j1;
-    if (SUMMARY) {
-      if (live && sub == (it & (LPR - 1))) {
-        // summary word of the row kernel: K | N << 11 | (entries differing from current) << 22
-        const uint32_t w = a.summ[(size_t)cand * a.J + j];
-        mine = (w & 0x7FFu) | (((w >> 11) & 0x7FFu) << 16) | ((w >> 22) ? 0x80000000u : 0u);
-        myrow = j;
-      }
-    } else {
     int ksum = 0;
     uint32_t npos = 0, diff = 0;
     if (live) {
@@ -143,7 +160,6 @@ __global__ void __launch_bounds__(256) fitness_kernel(FitnessArgs a) {
       mine = (packed & 0x7FFFFFFFu) | (changed ? 0x80000000u : 0u);
       myrow = j;
     }
-    }
     const bool flush = ((it + 1) % slots_per_fill == 0) || (jb + nwarps * RPW >= j1);
     if (flush) {
       if (myrow >= 0 && (!a.active || a.active[myrow]))
@@ -153,28 +169,27 @@ __global__ void __launch_bounds__(256) fitness_kernel(FitnessArgs a) {
     }
   }
 
-  // the block's terms, summed in an order that does not depend on how rows were mapped to lanes
-  __syncthreads();
-  double t, n;
-  block_term_sum(s_term, j1 - j0, j0, a.active, t, n);
-  __shared__ bool s_last;
-  if (threadIdx.x == 0) {
-    double *dst = a.partial + ((size_t)cand * a.chunks + chunk) * 2;
-    dst[0] = t;
-    dst[1] = n;
-    __threadfence();
-    const unsigned prev = atomicAdd(a.ticket + cand, 1u);
-    s_last = (prev == (unsigned)a.chunks - 1u);
+  block_finish(a, cand, chunk, j0, j1, s_term);
+}
+
+// Fitness from the row summaries the row / column kernels keep (K | N << 11 | entries
+// differing from the current allocation << 22): no pass over the matrices.  Same chunks, same
+// terms and the same fixed-order sums as fitness_kernel, hence identical bits.
+__global__ void __launch_bounds__(256) fitness_summary_kernel(FitnessArgs a) {
+  __shared__ float s_term[FITNESS_MAX_ROWS_PER_BLOCK];
+  const int cand = blockIdx.y, chunk = blockIdx.x;
+  const int j0 = chunk * a.rows_per_block;
+  const int j1 = min(a.J, j0 + a.rows_per_block);
+  TermParams tp;
+  tp.table = a.table; tp.pen = a.pen; tp.active = a.active;
+  tp.k_max = a.k_max; tp.n_max = a.n_max; tp.mode = a.mode; tp.p = a.p; tp.floor_ = a.floor_;
+  for (int j = j0 + threadIdx.x; j < j1; j += blockDim.x) {
+    if (!a.active || a.active[j]) {
+      const uint32_t w = a.summ[(size_t)cand * a.J + j];
+      s_term[j - j0] = fitness_term(tp, j, (int)(w & 0x7FFu), (int)((w >> 11) & 0x7FFu), (w >> 22) != 0u);
+    }
   }
-  __syncthreads();
-  if (s_last && threadIdx.x == 0) {
-    __threadfence();
-    const volatile double *src = a.partial + (size_t)cand * a.chunks * 2;
-    double ts = 0.0, ns = 0.0;
-    for (int c = 0; c < a.chunks; ++c) { ts += src[2 * c]; ns += src[2 * c + 1]; }
-    a.fitness[cand] = fitness_finalise(a.mode, a.p, ts, ns);
-    a.ticket[cand] = 0u;   // ready for the next call on this stream
-  }
+  block_finish(a, cand, chunk, j0, j1, s_term);
 }
 
 // Effective penalty per job: the re-allocation factor when the job currently holds GPUs,
@@ -277,14 +292,13 @@ int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const fl
     dim3 grid((unsigned)chunks, (unsigned)n);
     {
     TimedLaunch tl_(ctx, KK_FITNESS);
+    if (d_summ) fitness_summary_kernel<<<grid, 256, 0, ctx->stream>>>(b);
+    else
     switch (W) {
-      case 16:
-        if (d_summ) fitness_kernel<16, true><<<grid, 256, 0, ctx->stream>>>(b);
-        else fitness_kernel<16, false><<<grid, 256, 0, ctx->stream>>>(b);
-        break;
-      case 8: fitness_kernel<8, false><<<grid, 256, 0, ctx->stream>>>(b); break;
-      case 4: fitness_kernel<4, false><<<grid, 256, 0, ctx->stream>>>(b); break;
-      default: fitness_kernel<2, false><<<grid, 256, 0, ctx->stream>>>(b); break;
+      case 16: fitness_kernel<16><<<grid, 256, 0, ctx->stream>>>(b); break;
+      case 8: fitness_kernel<8><<<grid, 256, 0, ctx->stream>>>(b); break;
+      case 4: fitness_kernel<4><<<grid, 256, 0, ctx->stream>>>(b); break;
+      default: fitness_kernel<2><<<grid, 256, 0, ctx->stream>>>(b); break;
     }
     }
     SCHED_LAUNCH_CHECK(ctx);
@@ -407,10 +421,10 @@ int eval_fitness_noalloc(const int16_t *d_pop, int32_t count, int32_t num_jobs, 
   a.fitness = d_fitness;
   dim3 grid((unsigned)chunks, (unsigned)count);
   switch (W) {
-    case 16: fitness_kernel<16, false><<<grid, 256, 0, stream>>>(a); break;
-    case 8: fitness_kernel<8, false><<<grid, 256, 0, stream>>>(a); break;
-    case 4: fitness_kernel<4, false><<<grid, 256, 0, stream>>>(a); break;
-    default: fitness_kernel<2, false><<<grid, 256, 0, stream>>>(a); break;
+    case 16: fitness_kernel<16><<<grid, 256, 0, stream>>>(a); break;
+    case 8: fitness_kernel<8><<<grid, 256, 0, stream>>>(a); break;
+    case 4: fitness_kernel<4><<<grid, 256, 0, stream>>>(a); break;
+    default: fitness_kernel<2><<<grid, 256, 0, stream>>>(a); break;
   }
   e = cudaGetLastError();
   if (e != cudaSuccess) return noalloc_fail(SCHED_ERR_CUDA, "fitness_kernel launch", e);

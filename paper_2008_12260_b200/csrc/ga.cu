@@ -327,7 +327,9 @@ struct Rows2Args {
   RowsArgs r;
   int32_t *colsum;   // [count][nbatch][num_nodes] GPUs placed on the node by the batch's rows
   int32_t *colelig;  // same shape: rows of the batch that are distributed and occupy the node
-  unsigned int *list_count;  // length of the column work list, reset here for the column pass
+  unsigned int *list_count;  // length of the column work list (zeroed before this kernel)
+  uint32_t *list;            // the work list: (candidate << 13 | node) of nodes that need repair
+  unsigned int *cand_ticket; // [count] blocks of the candidate that have finished (self-resetting)
   int32_t *occ_count;        // [count][nbatch][num_nodes] rows of the batch that occupy the node
   uint32_t *occ_list;        // [count][nbatch][num_nodes][OCC_SLOTS] job | GPUs << 20 | distributed << 31
   int nbatch, lpr_log2;
@@ -578,7 +580,6 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
     s_tot[i] = 0; s_el[i] = 0; s_cnt[i] = 0;
     s_cap[i] = (int16_t)max((int)a.cap[i], 0);
   }
-  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *aa.list_count = 0u;
 
   // ---- parents of this candidate (generation mode), found by the block itself -------------
   // rank(i) = number of candidates ordered before i (fitness descending, index ascending).
@@ -908,27 +909,34 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
     const int cnt = min(s_cnt[i], OCC_SLOTS);
     for (int k = 0; k < cnt; ++k) aa.occ_list[(base + i) * OCC_SLOTS + k] = s_occ[i * OCC_SLOTS + k];
   }
+  // The last block of the candidate to get here adds the batch partials per node and appends
+  // the nodes that hold two distributed jobs or exceed their size to the work list.
+  __shared__ bool s_last_block;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned prev = atomicAdd(aa.cand_ticket + cl, 1u);
+    s_last_block = (prev == (unsigned)aa.nbatch - 1u);
+    if (s_last_block) aa.cand_ticket[cl] = 0u;
+  }
+  __syncthreads();
+  if (s_last_block) {
+    __threadfence();
+    for (int n = threadIdx.x; n < NN; n += blockDim.x) {
+      int total = 0, nelig = 0;
+      for (int b = 0; b < aa.nbatch; ++b) {
+        total += __ldcg(aa.colsum + ((size_t)cl * aa.nbatch + b) * NN + n);
+        nelig += __ldcg(aa.colelig + ((size_t)cl * aa.nbatch + b) * NN + n);
+      }
+      if (nelig >= 2 || total > (int)s_cap[n]) {
+        const unsigned slot = atomicAdd(aa.list_count, 1u);
+        aa.list[slot] = ((uint32_t)cl << 13) | (uint32_t)n;      // n < 8192, cl < 65536
+      }
+    }
+  }
 }
 
-// Column pass, step 1: a thread per (candidate, node) adds the batch partials up; nodes that
-// hold two distributed jobs or exceed their size are appended to a work list.
-__global__ void __launch_bounds__(128) colscan_kernel(ColfixArgs a) {
-  const int n = blockIdx.x * blockDim.x + threadIdx.x;
-  const int cl = blockIdx.y;
-  const int NN = a.num_nodes;
-  if (n >= NN) return;
-  int total = 0, nelig = 0;
-  for (int b = 0; b < a.nbatch; ++b) {
-    total += a.colsum[((size_t)cl * a.nbatch + b) * NN + n];
-    nelig += a.colelig[((size_t)cl * a.nbatch + b) * NN + n];
-  }
-  if (nelig >= 2 || total > max((int)a.cap[n], 0)) {
-    const unsigned slot = atomicAdd(a.list_count, 1u);
-    a.list[slot] = ((uint32_t)cl << 13) | (uint32_t)n;      // n < 8192, cl < 65536
-  }
-}
-
-// Column pass, step 2: warps take columns from the work list (any order: columns are
+// Column pass: warps take nodes from the work list the row kernel built (any order: columns are
 // independent) and repair them.
 __global__ void __launch_bounds__(128, 4) colrepair_kernel(ColfixArgs a) {
   const int lane = threadIdx.x & 31;
@@ -1018,7 +1026,7 @@ int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint3
   Rows2Args aa;
   aa.r = a;
   aa.colsum = ctx->d_colsum; aa.colelig = ctx->d_colelig; aa.nbatch = nbatch;
-  aa.list_count = ctx->d_colcount;
+  aa.list_count = ctx->d_colcount; aa.list = ctx->d_collist; aa.cand_ticket = ctx->d_rowticket;
   aa.occ_count = ctx->d_occcount; aa.occ_list = ctx->d_occlist;
   aa.fuse = (nbatch == 1 && ctx->ff_on) ? 1 : 0;
   aa.tp.table = ctx->ff_table; aa.tp.pen = ctx->ff_pen; aa.tp.active = ctx->ff_active;
@@ -1027,6 +1035,7 @@ int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint3
   aa.fitness_out = ctx->ff_out;
   ctx->fit_done = aa.fuse != 0;
   dim3 grid((unsigned)nbatch, (unsigned)count);
+  SCHED_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->d_colcount, 0, sizeof(unsigned int), ctx->stream));
   {
     TimedLaunch tl_(ctx, KK_ROWS);
     // about four vectors per lane: several loads in flight and the per-row overhead shared
@@ -1065,9 +1074,6 @@ int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint3
   f.gen = gen; f.first_cand = first_cand; f.key = make_key(ctx->cfg.seed, ctx->d_round);
   f.list = ctx->d_collist; f.list_count = ctx->d_colcount;
   f.cur = a.cur; f.occ_count = ctx->d_occcount; f.occ_list = ctx->d_occlist;
-  dim3 g2((unsigned)((NN + 127) / 128), (unsigned)count);
-  { TimedLaunch tl_(ctx, KK_COLSCAN); colscan_kernel<<<g2, 128, 0, ctx->stream>>>(f); }
-  SCHED_LAUNCH_CHECK(ctx);
   { TimedLaunch tl_(ctx, KK_COLS); colrepair_kernel<<<ctx->num_sms * 4, 128, 0, ctx->stream>>>(f); }
   SCHED_LAUNCH_CHECK(ctx);
   return SCHED_OK;
