@@ -50,6 +50,7 @@ int dev_alloc(sched_ctx *ctx, T **p, size_t n) {
   *p = nullptr;
   if (n == 0) n = 1;
   SCHED_CUDA_CHECK(ctx, cudaMalloc((void **)p, n * sizeof(T)));
+  ctx->scratch_epoch++;
   return SCHED_OK;
 }
 
@@ -486,6 +487,10 @@ int schedule_round(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cu
   key.jobs = *d_jobs;
   key.cur = d_cur; key.best = d_best; key.best_fitness = d_best_fitness; key.generations = generations;
   const bool graphs_ok = ctx->graphs_enabled && !ctx->timing_on && ctx->stream != nullptr;
+  if (ctx->graph_exec && ctx->graph_epoch != ctx->scratch_epoch) {   // scratch moved: pointers in the graph are stale
+    cudaGraphExecDestroy(ctx->graph_exec);
+    ctx->graph_exec = nullptr;
+  }
   if (graphs_ok && ctx->graph_exec && same_round_key(key, ctx->graph_key)) {
     SCHED_CUDA_CHECK(ctx, cudaGraphLaunch(ctx->graph_exec, ctx->stream));
     ctx->launches += ctx->graph_launches;
@@ -502,6 +507,7 @@ int schedule_round(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cu
   // allocation and can be captured
   if (ctx->graph_exec) { cudaGraphExecDestroy(ctx->graph_exec); ctx->graph_exec = nullptr; }
   const int64_t launches_before = ctx->launches;
+  const uint64_t epoch_before = ctx->scratch_epoch;
   cudaGraph_t graph = nullptr;
   if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
     cudaGetLastError();
@@ -512,7 +518,7 @@ int schedule_round(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cu
   const cudaError_t ce = cudaStreamEndCapture(ctx->stream, &graph);
   const int64_t captured = ctx->launches - launches_before;
   ctx->launches = launches_before;
-  if (rc != SCHED_OK || ce != cudaSuccess || !graph ||
+  if (rc != SCHED_OK || ce != cudaSuccess || !graph || ctx->scratch_epoch != epoch_before ||
       cudaGraphInstantiate(&ctx->graph_exec, graph, 0) != cudaSuccess) {
     cudaGetLastError();
     if (graph) cudaGraphDestroy(graph);
@@ -522,6 +528,7 @@ int schedule_round(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cu
   }
   cudaGraphDestroy(graph);
   memcpy(&ctx->graph_key, &key, sizeof(key));
+  ctx->graph_epoch = ctx->scratch_epoch;
   ctx->graph_launches = captured;
   ctx->graph_fit = ctx->d_fit;
   ctx->graph_pop_last = ctx->d_pop_last;

@@ -105,6 +105,8 @@ struct sched_ctx {
 
   // CUDA graph of a whole round (see schedule_round)
   bool graphs_enabled, seen_valid;
+  uint64_t scratch_epoch;   // bumped whenever a scratch buffer is reallocated: a captured graph
+  uint64_t graph_epoch;     // holds raw pointers and is only valid for the epoch it was captured in
   RoundKey seen_key, graph_key;
   cudaGraphExec_t graph_exec;
   int64_t graph_launches;

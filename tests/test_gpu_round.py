@@ -197,6 +197,37 @@ def test_graph_replay_gives_the_same_rounds(gpu):
     assert len({r[1] for r in outs[True][0]}) > 1    # the round number reaches the kernels
 
 
+def test_graph_survives_scratch_reallocation(gpu):
+    """A captured round holds raw scratch pointers; a later call that makes the context grow
+    its scratch must not leave a stale graph behind."""
+    torch, api = gpu
+    cfg = synth.TESTBED
+    cl, jobs = setup(cfg)
+    s = api.scheduler_for(cfg, stream=torch.cuda.Stream().cuda_stream)
+    dj = api.DeviceJobs(jobs, "cuda:0", torch)
+    d_cur = torch.from_numpy(cfg.cur()).cuda()
+    best = torch.empty((cfg.num_jobs, cfg.num_nodes), dtype=torch.int16, device="cuda:0")
+    bf = torch.zeros(1, dtype=torch.float32, device="cuda:0")
+    torch.cuda.synchronize()
+    ref = []
+    for rnd in range(4):
+        s.schedule_round(dj, d_cur, best, bf, round=rnd, generations=6)
+        s.sync_status()
+        ref.append((best.cpu().numpy().copy(), float(bf.item())))
+    # a much larger fitness call and a larger repair call reallocate the context's scratch
+    big = torch.zeros((cfg.population * 8, cfg.num_jobs, cfg.num_nodes), dtype=torch.int16, device="cuda:0")
+    table = torch.ones(s.table_shape, dtype=torch.float32, device="cuda:0")
+    fit = torch.empty(big.shape[0], dtype=torch.float32, device="cuda:0")
+    s.eval_fitness(big, table, fit, p=1.0)
+    s.repair_population(None, big, round=0, generation=0)
+    s.sync_status()
+    for rnd in range(4):
+        s.schedule_round(dj, d_cur, best, bf, round=rnd, generations=6)
+        s.sync_status()
+        assert np.array_equal(best.cpu().numpy(), ref[rnd][0]) and float(bf.item()) == ref[rnd][1]
+    s.close()
+
+
 def test_argument_errors(gpu):
     torch, api = gpu
     cfg = synth.TINY
