@@ -378,6 +378,17 @@ def bench_trace(api, torch, stream):
            "kernel_launches_per_round": (sched.launch_count() - l0) / len(fits),
            "mean_best_fitness": float(np.mean(fits[10:])), "mean_gpus_allocated": float(np.mean(used[10:])),
            "note": "launch- and latency-bound (population 150 KB): a roofline fraction is not meaningful here"}
+    # the same trace with training progress coupled to the allocations (jobs advance at the goodput
+    # the round's own tables predict, 30 s restart delay): completion times depend on the scheduler
+    pr = trace.ProgressReplay()
+    t0 = time.perf_counter()
+    pfits = trace.replay_progress(sched, pr, torch)
+    torch.cuda.synchronize()
+    pdt = time.perf_counter() - t0
+    jct = pr.completion_times()
+    out["progress_coupled"] = {"rounds_per_sec": len(pfits) / pdt, "jobs_finished": int(jct.size),
+                               "avg_jct_hours": float(jct.mean() / 3600.0) if jct.size else None,
+                               "p99_jct_hours": float(np.percentile(jct, 99) / 3600.0) if jct.size else None}
     sched.close()
     return out
 

@@ -203,6 +203,12 @@ int schedule_round_host(sched_ctx *ctx, const sched_jobs *h_jobs, const int16_t 
  * (either may be NULL).  d_pop_out: int16 [P][J][num_nodes], d_fitness_out: fp32 [P]. */
 int sched_get_population(sched_ctx *ctx, int16_t *d_pop_out, float *d_fitness_out);
 
+/* Copies the goodput and speedup tables built by the last schedule_round (Eq. 13, 15) into
+ * caller buffers, fp32 [J][k_max+1][n_max+1] each, either may be NULL.  goodput[j][K][N] is
+ * the predicted goodput of job j at its best (m, s) on that allocation: what a simulator
+ * needs to advance the job's training progress. */
+int sched_get_round_tables(sched_ctx *ctx, float *d_goodput_out, float *d_speedup_out);
+
 /* Pointer to the fp32 [J][k_max+1][n_max+1] speedup table built by the last schedule_round
  * (context scratch, device memory), or NULL before the first round. */
 const float *sched_round_speedup_table(const sched_ctx *ctx);

@@ -20,7 +20,7 @@ EXPORTS = (
     "sched_init", "sched_destroy", "sched_last_error", "sched_sync_status", "sched_launch_count",
     "build_speedup_table", "compute_realloc_factor", "eval_fitness", "repair_population",
     "init_population", "ga_generation", "schedule_round", "schedule_round_host",
-    "sched_get_population", "sched_round_speedup_table", "eval_fitness_host",
+    "sched_get_population", "sched_get_round_tables", "sched_round_speedup_table", "eval_fitness_host",
     "sched_set_kernel_timing", "sched_num_kernel_kinds", "sched_kernel_kind_name",
     "sched_read_kernel_timing", "sched_set_graphs", "eval_fitness_noalloc", "eval_fitness_noalloc_last_error",
 )
@@ -74,6 +74,7 @@ def load_library(path: str = LIB_PATH):
     lib.schedule_round.argtypes = [vp, C.POINTER(SchedJobs), vp, u32, i32, vp, vp]
     lib.schedule_round_host.argtypes = [vp, C.POINTER(SchedJobs), vp, u32, i32, vp, vp]
     lib.sched_get_population.argtypes = [vp, vp, vp]
+    lib.sched_get_round_tables.argtypes = [vp, vp, vp]
     lib.sched_round_speedup_table.argtypes = [vp]
     lib.sched_round_speedup_table.restype = vp
     lib.eval_fitness_host.argtypes = [vp, vp, i32, vp, vp, vp, vp, f32, vp]
@@ -254,6 +255,9 @@ class Scheduler:
 
     def get_population(self, pop_out=None, fitness_out=None):
         self._check(_lib.sched_get_population(self._ctx, _ptr(pop_out), _ptr(fitness_out)))
+
+    def get_round_tables(self, goodput_out=None, speedup_out=None):
+        self._check(_lib.sched_get_round_tables(self._ctx, _ptr(goodput_out), _ptr(speedup_out)))
 
     def eval_fitness_host(self, pop, speedup, fitness, *, p, cur=None, realloc_factor=None, active=None):
         self._check(_lib.eval_fitness_host(self._ctx, _ptr(pop), pop.shape[0], _ptr(speedup), _ptr(cur),

@@ -551,6 +551,17 @@ int sched_get_population(sched_ctx *ctx, int16_t *d_pop_out, float *d_fitness_ou
   return SCHED_OK;
 }
 
+int sched_get_round_tables(sched_ctx *ctx, float *d_goodput_out, float *d_speedup_out) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "sched_get_round_tables: ctx is NULL");
+  REQUIRE(ctx, ctx->round_ready && ctx->d_pop_last, SCHED_ERR_INVALID_ARG, "sched_get_round_tables: no round has run yet");
+  const size_t bytes = sizeof(float) * (size_t)ctx->cfg.num_jobs * ctx->KD * ctx->ND;
+  if (d_goodput_out)
+    SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(d_goodput_out, ctx->d_tab_goodput, bytes, cudaMemcpyDeviceToDevice, ctx->stream));
+  if (d_speedup_out)
+    SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(d_speedup_out, ctx->d_tab_speedup, bytes, cudaMemcpyDeviceToDevice, ctx->stream));
+  return SCHED_OK;
+}
+
 const float *sched_round_speedup_table(const sched_ctx *ctx) {
   return (ctx && ctx->round_ready) ? ctx->d_tab_speedup : nullptr;
 }

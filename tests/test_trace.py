@@ -74,3 +74,66 @@ def test_trace_rounds_on_gpu(oracle):
     fits3, used3 = trace.replay(s, tr, torch, rounds=40, first_round=30)
     assert fits2 == fits3 and used2 == used3
     s.close()
+
+
+def test_progress_bookkeeping():
+    """Progress-coupled replay, host side only: work is fixed on a job's first round, progress
+    integrates goodput over 60 s minus the restart delay, completion time is interpolated."""
+    from paper_2008_12260_b200 import trace
+    tr = trace.ProgressReplay()
+    k = 40
+    jobs, cur = tr.round_inputs(k)
+    act = np.nonzero(jobs.active)[0]
+    assert act.size >= 2
+    a, b = int(act[0]), int(act[1])
+    best = cur.copy()
+    best[a, 0] = 2                       # job a (pending) starts: allocation changed -> 30 s delay
+    g_kn = np.zeros(tr.cfg.num_jobs); g_1 = np.ones(tr.cfg.num_jobs)
+    g_kn[a] = 3.0
+    tr.advance(k, jobs, cur, best, g_kn, g_1)
+    assert tr.work[a] == pytest.approx(tr.life[a] * 1.0) and np.isinf(tr.work[~(jobs.active > 0)]).all()
+    assert tr.done[a] == pytest.approx(3.0 * 30.0) and tr.done[b] == 0.0
+    # unchanged allocation next round: full 60 s
+    jobs2, cur2 = tr.round_inputs(k + 1)
+    assert np.array_equal(cur2[a], best[a])
+    tr.advance(k + 1, jobs2, cur2, cur2.copy(), g_kn, g_1)
+    assert tr.done[a] == pytest.approx(3.0 * 90.0)
+    assert jobs2.phi[a] > tr.phi0[a] * 0.999           # phi follows the work done
+    # finishing: give job a all its remaining work in half an interval
+    rem = tr.work[a] - tr.done[a]
+    g_kn[a] = rem / 30.0
+    jobs3, cur3 = tr.round_inputs(k + 2)
+    tr.advance(k + 2, jobs3, cur3, cur3.copy(), g_kn, g_1)
+    assert tr.finish[a] == pytest.approx((k + 2) * 60.0 + 30.0)
+    assert not tr.cur[a].any()
+    jobs4, _ = tr.round_inputs(k + 3)
+    assert jobs4.active[a] == 0
+    assert tr.completion_times().size == 1
+
+
+@pytest.mark.gpu
+def test_progress_replay_on_gpu(oracle):
+    import torch
+    from paper_2008_12260_b200 import api, trace
+
+    tr = trace.ProgressReplay(generations=20)
+    cfg, cl = tr.cfg, tr.cluster
+    s = api.scheduler_for(cfg, stream=torch.cuda.Stream().cuda_stream)
+    seen = []
+
+    def check(k, jobs, cur, best, fit, g_kn):
+        if k % 15 == 3 and jobs.active.any():
+            gp, _, _ = oracle.build_speedup_table(jobs, cl.node_capacity, cl.k_max, cl.n_max, cfg.grid_s,
+                                                  want_argmax=False)
+            K = np.minimum(best.sum(1), cl.k_max); N = np.minimum((best > 0).sum(1), cl.n_max)
+            ref = gp[np.arange(cfg.num_jobs), K, N]
+            on = jobs.active > 0
+            np.testing.assert_allclose(g_kn[on], ref[on], rtol=REL_TOL, atol=0)
+            seen.append(k)
+
+    fits = trace.replay_progress(s, tr, torch, rounds=120, on_round=check)
+    assert len(seen) >= 6
+    jct = tr.completion_times()
+    assert jct.size >= 3 and np.all(jct > 0) and np.all(np.isfinite(jct))
+    assert np.all(tr.done[~np.isnan(tr.finish)] >= tr.work[~np.isnan(tr.finish)] * (1 - 1e-12))
+    s.close()
