@@ -141,6 +141,16 @@ int build_speedup_table(sched_ctx *ctx, const sched_jobs *d_jobs, float *d_goodp
  * (Sec. 4.2), with delta = cfg.delta_sec.  d_out: fp32 [J].  Uses age_sec, num_restarts. */
 int compute_realloc_factor(sched_ctx *ctx, const sched_jobs *d_jobs, float *d_out);
 
+/* Goodput-driven auto-scaling rule (Sec. 5.3, "Cloud auto-scaling").  For a job that holds
+ * d_cur_nodes[j] whole nodes of gpus_per_node GPUs, with g(n) = goodput[j][n G][n] and the
+ * ideal n G goodput[j][1][1] of perfect scalability: if g(cur) > U * ideal(cur) the target is
+ * the largest n > cur (n <= n_max, n G <= k_max) with g(n) >= L * ideal(n), or cur if there
+ * is none; otherwise the target is cur (the rule never scales down).  The paper uses
+ * U = 2/3, L = 1/2.  d_goodput: fp32 [J][k_max+1][n_max+1] from build_speedup_table;
+ * d_cur_nodes, d_target_nodes: int32 [J].  Jobs with cur < 1 or beyond the table keep cur. */
+int autoscale_targets(sched_ctx *ctx, const float *d_goodput, const int32_t *d_cur_nodes, int32_t gpus_per_node,
+                      float U, float L, int32_t *d_target_nodes);
+
 /* Fitness of `count` candidates (Eq. 14).  d_pop: int16 [count][J][num_nodes].  For each
  * active job the speedup is read at (K, N) = (sum of the row, entries > 0), clamped to
  * the table; if d_cur (int16 [J][num_nodes]) and d_realloc_factor (fp32 [J]) are both

@@ -264,3 +264,14 @@ def schedule_round(jobs, node_capacity, k_max, n_max, grid_s, P, p, delta, floor
     if rc != 0:
         raise ValueError("oracle_schedule_round: bad arguments")
     return best, bf.value
+
+
+def autoscale_targets(goodput_f32, k_max, n_max, gpus_per_node, cur_nodes, U, L):
+    g = _c(goodput_f32, np.float32)
+    cn = _c(cur_nodes, np.int32)
+    out = np.empty(cn.shape[0], dtype=np.int32)
+    rc = lib().oracle_autoscale_targets(cn.shape[0], int(k_max), int(n_max), int(gpus_per_node), _p(g), _p(cn),
+                                        C.c_float(U), C.c_float(L), _p(out))
+    if rc != 0:
+        raise ValueError("oracle_autoscale_targets: bad arguments")
+    return out

@@ -566,6 +566,38 @@ int oracle_schedule_round(int P, int J, int num_nodes, const int16_t *cap, int k
     return ORACLE_OK;
 }
 
+/* Goodput-driven auto-scaling (Sec. 5.3, cloud auto-scaling): a job on n whole nodes of G GPUs
+ * is scaled up when its goodput per GPU exceeds the fraction U of the single-GPU goodput
+ * ("ideal" = perfect scalability), to the largest node count whose goodput is still at
+ * least the fraction L of ideal; otherwise it keeps its nodes.  The comparisons are made in
+ * fp32, in this order of operations, on the fp32 table: they decide integers. */
+int oracle_autoscale_targets(int J, int k_max, int n_max, int gpus_per_node, const float *goodput,
+                             const int32_t *cur_nodes, float U, float L, int32_t *target_nodes) {
+  if (J < 0 || gpus_per_node < 1 || !goodput || !cur_nodes || !target_nodes) return ORACLE_ERR_ARG;
+  const int KD = k_max + 1, ND = n_max + 1;
+  for (int j = 0; j < J; ++j) {
+    const float *g = goodput + (size_t)j * KD * ND;
+    const float g1 = g[1 * ND + 1];
+    int n = cur_nodes[j];
+    int limit = n_max;
+    if (limit * gpus_per_node > k_max) limit = k_max / gpus_per_node;
+    int target = n;
+    if (n >= 1 && n <= limit && g1 > 0.0f) {
+      const float k = (float)(n * gpus_per_node);
+      const float ideal_u = (float)((float)(U * k) * g1);
+      if (g[(n * gpus_per_node) * ND + n] > ideal_u) {
+        for (int t = n + 1; t <= limit; ++t) {
+          const float kt = (float)(t * gpus_per_node);
+          const float ideal_l = (float)((float)(L * kt) * g1);
+          if (g[(t * gpus_per_node) * ND + t] >= ideal_l) target = t;
+        }
+      }
+    }
+    target_nodes[j] = target;
+  }
+  return ORACLE_OK;
+}
+
 int oracle_num_threads(void) {
     int n = 1;
 #ifdef _OPENMP

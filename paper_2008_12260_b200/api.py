@@ -18,7 +18,7 @@ ERRORS = {-1: "INVALID_ARG", -2: "BAD_CONFIG", -3: "CUDA", -4: "TIMEOUT", -5: "N
 
 EXPORTS = (
     "sched_init", "sched_destroy", "sched_last_error", "sched_sync_status", "sched_launch_count",
-    "build_speedup_table", "compute_realloc_factor", "eval_fitness", "repair_population",
+    "build_speedup_table", "compute_realloc_factor", "autoscale_targets", "eval_fitness", "repair_population",
     "init_population", "ga_generation", "schedule_round", "schedule_round_host",
     "sched_get_population", "sched_get_round_tables", "sched_round_speedup_table", "eval_fitness_host",
     "sched_set_kernel_timing", "sched_num_kernel_kinds", "sched_kernel_kind_name",
@@ -67,6 +67,7 @@ def load_library(path: str = LIB_PATH):
     lib.sched_launch_count.restype = C.c_int64
     lib.build_speedup_table.argtypes = [vp, C.POINTER(SchedJobs), vp, vp, vp]
     lib.compute_realloc_factor.argtypes = [vp, C.POINTER(SchedJobs), vp]
+    lib.autoscale_targets.argtypes = [vp, vp, vp, i32, f32, f32, vp]
     lib.eval_fitness.argtypes = [vp, vp, i32, vp, vp, vp, vp, f32, vp]
     lib.repair_population.argtypes = [vp, C.POINTER(SchedJobs), vp, i32, u32, u32, u32]
     lib.init_population.argtypes = [vp, C.POINTER(SchedJobs), vp, u32, vp]
@@ -224,6 +225,10 @@ class Scheduler:
 
     def compute_realloc_factor(self, jobs, out):
         self._check(_lib.compute_realloc_factor(self._ctx, C.byref(jobs.struct), _ptr(out)))
+
+    def autoscale_targets(self, goodput, cur_nodes, target_nodes, *, gpus_per_node, U=2.0 / 3.0, L=0.5):
+        self._check(_lib.autoscale_targets(self._ctx, _ptr(goodput), _ptr(cur_nodes), gpus_per_node, U, L,
+                                           _ptr(target_nodes)))
 
     def eval_fitness(self, pop, speedup, fitness, *, p, cur=None, realloc_factor=None, active=None,
                      count=None):

@@ -341,6 +341,16 @@ int compute_realloc_factor(sched_ctx *ctx, const sched_jobs *d_jobs, float *d_ou
   return launch_realloc_factor(ctx, d_jobs, d_out);
 }
 
+int autoscale_targets(sched_ctx *ctx, const float *d_goodput, const int32_t *d_cur_nodes, int32_t gpus_per_node,
+                      float U, float L, int32_t *d_target_nodes) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "autoscale_targets: ctx is NULL");
+  REQUIRE(ctx, d_goodput && d_cur_nodes && d_target_nodes, SCHED_ERR_INVALID_ARG,
+          "autoscale_targets: d_goodput, d_cur_nodes and d_target_nodes must be non-NULL");
+  REQUIRE(ctx, gpus_per_node >= 1 && U == U && L == L, SCHED_ERR_INVALID_ARG,
+          "autoscale_targets: gpus_per_node must be >= 1, U and L not NaN");
+  return launch_autoscale(ctx, d_goodput, d_cur_nodes, gpus_per_node, U, L, d_target_nodes);
+}
+
 int eval_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const float *d_speedup,
                  const int16_t *d_cur, const float *d_realloc_factor, const uint8_t *d_active,
                  float p, float *d_fitness) {

@@ -218,6 +218,8 @@ __device__ __forceinline__ uint32_t order_key(uint32_t bits) {
 int launch_speedup_table(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodput, float *d_speedup,
                          uint16_t *d_argmax);
 int launch_realloc_factor(sched_ctx *ctx, const sched_jobs *jobs, float *d_out);
+int launch_autoscale(sched_ctx *ctx, const float *d_goodput, const int32_t *d_cur_nodes, int gpn, float U, float L,
+                     int32_t *d_target_nodes);
 int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const float *d_speedup,
                    const int16_t *d_cur, const float *d_rf, const uint8_t *d_active, float p,
                    float *d_fitness, const uint32_t *d_summ = nullptr);

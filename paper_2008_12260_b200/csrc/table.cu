@@ -251,7 +251,42 @@ __global__ void realloc_factor_kernel(const float *__restrict__ age, const int32
   out[j] = fminf(f, 1.f);
 }
 
+// Goodput-driven auto-scaling rule (Sec. 5.3): one thread per job.  All products are
+// rounded one by one (no contraction): the comparisons decide integers.
+__global__ void autoscale_kernel(const float *__restrict__ goodput, const int32_t *__restrict__ cur_nodes,
+                                 int J, int k_max, int n_max, int gpn, float U, float L,
+                                 int32_t *__restrict__ target_nodes) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= J) return;
+  const int KD = k_max + 1, ND = n_max + 1;
+  const float *g = goodput + (size_t)j * KD * ND;
+  const float g1 = g[ND + 1];
+  const int n = cur_nodes[j];
+  const int limit = min(n_max, k_max / gpn);
+  int target = n;
+  if (n >= 1 && n <= limit && g1 > 0.f) {
+    const float ideal_u = __fmul_rn(__fmul_rn(U, (float)(n * gpn)), g1);
+    if (g[(size_t)(n * gpn) * ND + n] > ideal_u) {
+      for (int t = n + 1; t <= limit; ++t) {
+        const float ideal_l = __fmul_rn(__fmul_rn(L, (float)(t * gpn)), g1);
+        if (g[(size_t)(t * gpn) * ND + t] >= ideal_l) target = t;
+      }
+    }
+  }
+  target_nodes[j] = target;
+}
+
 }  // namespace
+
+int launch_autoscale(sched_ctx *ctx, const float *d_goodput, const int32_t *d_cur_nodes, int gpn, float U, float L,
+                     int32_t *d_target_nodes) {
+  const int J = ctx->cfg.num_jobs;
+  if (J == 0) return SCHED_OK;
+  autoscale_kernel<<<(J + 127) / 128, 128, 0, ctx->stream>>>(d_goodput, d_cur_nodes, J, ctx->cfg.k_max,
+                                                             ctx->cfg.n_max, gpn, U, L, d_target_nodes);
+  SCHED_LAUNCH_CHECK(ctx);
+  return SCHED_OK;
+}
 
 int launch_speedup_table(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodput, float *d_speedup,
                          uint16_t *d_argmax) {
