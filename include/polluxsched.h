@@ -137,6 +137,19 @@ int sched_read_kernel_timing(sched_ctx *ctx, float *h_ms_total, int64_t *h_launc
 int build_speedup_table(sched_ctx *ctx, const sched_jobs *d_jobs, float *d_goodput,
                         float *d_speedup, uint16_t *d_argmax);
 
+/* Speedup tables with the (m, s) sub-procedure as the paper words it (Sec. 4.3) instead of a
+ * fixed grid: d_m_samples (int32 [J][num_samples]) holds candidate total batch sizes M; for
+ * each, per_gpu = ceil(M / K), s = ceil(per_gpu / m_max_gpu[j]) - 1 is the smallest number of
+ * accumulation steps whose per-GPU batch m = ceil(per_gpu / (s + 1)) fits the limit, the
+ * batch run is M' = K m (s + 1) and must satisfy M0 <= M' <= m_max_total; the best goodput
+ * over the candidates is tabulated (ties: smallest candidate index; argmax = candidate
+ * index).  Jobs with d_adaptive[j] == 0 (d_adaptive nullable = all adaptive) are the
+ * non-adaptive jobs of Sec. 4.2: the single candidate M = M0 with EFFICIENCY fixed to 1.
+ * Outputs, validity of (K, N) and normalisation as build_speedup_table; m_grid is not used. */
+int build_speedup_table_msample(sched_ctx *ctx, const sched_jobs *d_jobs, const int32_t *d_m_samples,
+                                int32_t num_samples, const int32_t *d_m_max_gpu, const uint8_t *d_adaptive,
+                                float *d_goodput, float *d_speedup, uint16_t *d_argmax);
+
 /* REALLOC_FACTOR_j(delta) = (T_j - R_j delta) / (T_j + delta) clamped to [0, 1]
  * (Sec. 4.2), with delta = cfg.delta_sec.  d_out: fp32 [J].  Uses age_sec, num_restarts. */
 int compute_realloc_factor(sched_ctx *ctx, const sched_jobs *d_jobs, float *d_out);

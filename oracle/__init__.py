@@ -275,3 +275,27 @@ def autoscale_targets(goodput_f32, k_max, n_max, gpus_per_node, cur_nodes, U, L)
     if rc != 0:
         raise ValueError("oracle_autoscale_targets: bad arguments")
     return out
+
+
+def build_speedup_table_msample(jobs, node_capacity, k_max, n_max, m_samples, m_max_gpu, adaptive=None,
+                                want_argmax=True):
+    """Tables from the paper's total-batch sampling search (Sec. 4.3) and, for jobs with
+    adaptive == 0, the fixed-batch rule of Sec. 4.2."""
+    cap = _c(node_capacity, np.int16)
+    fa = _job_args(jobs)
+    ms = _c(m_samples, np.int32)
+    mm = _c(m_max_gpu, np.int32)
+    ad = _c(adaptive, np.uint8)
+    fk = _c(jobs.fair_k, np.int32)
+    fn = _c(jobs.fair_n, np.int32)
+    J, G = ms.shape
+    shape = (J, k_max + 1, n_max + 1)
+    gp = np.zeros(shape, dtype=np.float64)
+    sp = np.zeros(shape, dtype=np.float64)
+    am = np.zeros(shape, dtype=np.uint16) if want_argmax else None
+    rc = lib().oracle_build_speedup_table_msample(
+        J, cap.shape[0], _p(cap), int(k_max), int(n_max), int(G), *[_p(a) for a in fa], _p(ms), _p(mm), _p(ad),
+        _p(fk), _p(fn), _p(gp), _p(sp), _p(am))
+    if rc != 0:
+        raise ValueError("oracle_build_speedup_table_msample: bad arguments")
+    return gp, sp, am

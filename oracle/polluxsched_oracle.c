@@ -207,6 +207,67 @@ int oracle_build_speedup_table(int J, int num_nodes, const int16_t *cap, int k_m
     return ORACLE_OK;
 }
 
+/* The (m, s) sub-procedure as the paper words it (Sec. 4.3): sample candidate total batch
+ * sizes M, for each take the smallest s such that the per-GPU batch fits the limit m_max,
+ * and keep the configuration with the highest goodput.  Read here (the printed
+ * "m = ceil(M / s)" cannot hold for s = 0) as: per_gpu = ceil(M / K);
+ * s = ceil(per_gpu / m_max) - 1; m = ceil(per_gpu / (s + 1)); the batch actually run is
+ * M' = K m (s + 1) >= M and must satisfy M0 <= M' <= M_max.  A non-adaptive job (Sec. 4.2,
+ * "supporting non-adaptive jobs") has the single candidate M = M0 and EFFICIENCY fixed to 1.
+ * Table layout, validity of (K, N), normalisation and ties (smallest sample index) as in
+ * oracle_build_speedup_table; argmax = sample index. */
+int oracle_build_speedup_table_msample(int J, int num_nodes, const int16_t *cap, int k_max, int n_max,
+                                       int num_samples, const float *alpha_grad, const float *beta_grad,
+                                       const float *alpha_local, const float *beta_local,
+                                       const float *alpha_node, const float *beta_node, const float *gamma,
+                                       const float *phi, const float *m0, const float *m_max_total,
+                                       const int32_t *m_samples, const int32_t *m_max_gpu,
+                                       const uint8_t *adaptive, const int32_t *fair_k, const int32_t *fair_n,
+                                       double *goodput, double *speedup, uint16_t *argmax) {
+  if (J < 0 || k_max < 1 || n_max < 1 || num_samples < 1) return ORACLE_ERR_ARG;
+  const int KD = k_max + 1, ND = n_max + 1;
+  int64_t *kfit = (int64_t *)malloc(sizeof(int64_t) * (size_t)ND);
+  max_k_per_n(num_nodes, cap, n_max, kfit);
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int j = 0; j < J; ++j) {
+    double *gj = goodput + (size_t)j * KD * ND;
+    double *sj = speedup + (size_t)j * KD * ND;
+    uint16_t *aj = argmax ? argmax + (size_t)j * KD * ND : NULL;
+    const int adapt = adaptive ? adaptive[j] != 0 : 1;
+    const int ns = adapt ? num_samples : 1;
+    for (int K = 0; K < KD; ++K) {
+      for (int N = 0; N < ND; ++N) {
+        double best = 0.0;
+        int best_i = -1;
+        if (N >= 1 && K >= N && (int64_t)K <= kfit[N] && m_max_gpu[j] >= 1) {
+          for (int i = 0; i < ns; ++i) {
+            const int64_t M = adapt ? (int64_t)m_samples[(size_t)j * num_samples + i] : (int64_t)m0[j];
+            if (M < 1) continue;
+            const int64_t per_gpu = (M + K - 1) / K;
+            const int64_t s = (per_gpu + m_max_gpu[j] - 1) / m_max_gpu[j] - 1;
+            const int64_t m = (per_gpu + s) / (s + 1);
+            const double Mrun = (double)K * (double)m * (double)(s + 1);
+            if (Mrun < m0[j] || Mrun > m_max_total[j]) continue;
+            const double tg = oracle_t_grad(alpha_grad[j], beta_grad[j], (double)m);
+            const double ts = oracle_t_sync(alpha_local[j], beta_local[j], alpha_node[j], beta_node[j], K, N);
+            const double ti = oracle_t_iter(tg, ts, gamma[j], (int)s);
+            const double eff = adapt ? oracle_efficiency(phi[j], m0[j], Mrun) : 1.0;
+            const double g = (Mrun / ti) * eff;
+            if (best_i < 0 || g > best) { best = g; best_i = i; }
+          }
+        }
+        gj[K * ND + N] = best_i >= 0 ? best : 0.0;
+        if (aj) aj[K * ND + N] = best_i >= 0 ? (uint16_t)best_i : 0xFFFFu;
+      }
+    }
+    const int kf = fair_k[j], nf = fair_n[j];
+    const double denom = (kf >= 0 && kf < KD && nf >= 0 && nf < ND) ? gj[kf * ND + nf] : 0.0;
+    for (int e = 0; e < KD * ND; ++e) sj[e] = denom > 0.0 ? gj[e] / denom : 0.0;
+  }
+  free(kfit);
+  return ORACLE_OK;
+}
+
 /* REALLOC_FACTOR_j(delta) = (T_j - R_j delta) / (T_j + delta), kept inside [0, 1]
  * (Sec. 4.2, re-allocation penalty). */
 void oracle_realloc_factor(int J, const float *age_sec, const int32_t *num_restarts, double delta,

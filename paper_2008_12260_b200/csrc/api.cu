@@ -334,6 +334,22 @@ int build_speedup_table(sched_ctx *ctx, const sched_jobs *d_jobs, float *d_goodp
   return launch_speedup_table(ctx, d_jobs, d_goodput, d_speedup, d_argmax);
 }
 
+int build_speedup_table_msample(sched_ctx *ctx, const sched_jobs *d_jobs, const int32_t *d_m_samples,
+                                int32_t num_samples, const int32_t *d_m_max_gpu, const uint8_t *d_adaptive,
+                                float *d_goodput, float *d_speedup, uint16_t *d_argmax) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "build_speedup_table_msample: ctx is NULL");
+  REQUIRE(ctx, d_jobs && d_jobs->alpha_grad && d_jobs->beta_grad && d_jobs->alpha_local && d_jobs->beta_local &&
+                   d_jobs->alpha_node && d_jobs->beta_node && d_jobs->gamma && d_jobs->phi && d_jobs->m0 &&
+                   d_jobs->m_max_total && d_jobs->fair_k && d_jobs->fair_n,
+          SCHED_ERR_INVALID_ARG, "build_speedup_table_msample: a goodput-model array, fair_k or fair_n is NULL");
+  REQUIRE(ctx, d_m_samples && d_m_max_gpu && d_speedup, SCHED_ERR_INVALID_ARG,
+          "build_speedup_table_msample: d_m_samples, d_m_max_gpu and d_speedup must be non-NULL");
+  REQUIRE(ctx, num_samples >= 1 && num_samples <= 65535, SCHED_ERR_INVALID_ARG,
+          "build_speedup_table_msample: num_samples must be in [1, 65535]");
+  return launch_speedup_table_msample(ctx, d_jobs, d_m_samples, num_samples, d_m_max_gpu, d_adaptive, d_goodput,
+                                      d_speedup, d_argmax);
+}
+
 int compute_realloc_factor(sched_ctx *ctx, const sched_jobs *d_jobs, float *d_out) {
   REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "compute_realloc_factor: ctx is NULL");
   REQUIRE(ctx, d_jobs && d_jobs->age_sec && d_jobs->num_restarts && d_out, SCHED_ERR_INVALID_ARG,

@@ -217,6 +217,9 @@ __device__ __forceinline__ uint32_t order_key(uint32_t bits) {
 // kernels' launchers (defined in table.cu / fitness.cu / ga.cu)
 int launch_speedup_table(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodput, float *d_speedup,
                          uint16_t *d_argmax);
+int launch_speedup_table_msample(sched_ctx *ctx, const sched_jobs *jobs, const int32_t *d_m_samples, int G,
+                                 const int32_t *d_m_max_gpu, const uint8_t *d_adaptive, float *d_goodput,
+                                 float *d_speedup, uint16_t *d_argmax);
 int launch_realloc_factor(sched_ctx *ctx, const sched_jobs *jobs, float *d_out);
 int launch_autoscale(sched_ctx *ctx, const float *d_goodput, const int32_t *d_cur_nodes, int gpn, float U, float L,
                      int32_t *d_target_nodes);

@@ -203,6 +203,71 @@ goodput_sweep_kernel(JobPtrs jp, const int32_t *__restrict__ m_grid,
   }
 }
 
+// The (m, s) search as the paper words it (Sec. 4.3): candidate total batch sizes M are given;
+// per candidate, per_gpu = ceil(M / K), s = ceil(per_gpu / m_max) - 1 (the fewest accumulation
+// steps that fit the per-GPU limit), m = ceil(per_gpu / (s + 1)), and the batch actually run
+// is M' = K m (s + 1), feasible when M0 <= M' <= M_max.  A non-adaptive job has the single
+// candidate M0 and EFFICIENCY fixed to 1 (Sec. 4.2).  One warp per (job, K, class), lanes over
+// the candidates; all feasibility decisions are integer.
+__global__ void __launch_bounds__(256)
+msample_sweep_kernel(JobPtrs jp, const int32_t *__restrict__ m_samples, const int32_t *__restrict__ m_max_gpu,
+                     const uint8_t *__restrict__ adaptive, const int32_t *__restrict__ pairs, int npairs,
+                     int k_max, int G, float *__restrict__ gmax, uint16_t *__restrict__ amax) {
+  const int lane = threadIdx.x & 31;
+  const int j = blockIdx.x;
+  const int pi = blockIdx.y * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (pi >= npairs) return;
+  const int pr = pairs[pi];
+  const int cls = pr & 1, K = pr >> 1;
+  const size_t out = ((size_t)j * (k_max + 1) + K) * 2 + cls;
+  const float a_g = jp.alpha_grad[j], b_g = jp.beta_grad[j];
+  const float gamma = jp.gamma[j], inv_gamma = 1.f / gamma;
+  const float phi = jp.phi[j], M0 = jp.m0[j], Mmax = jp.m_max_total[j];
+  const bool adapt = !adaptive || adaptive[j];
+  const int mmax = m_max_gpu[j];
+  float ts = 0.f;
+  if (K >= 2) {
+    const float a = cls ? jp.alpha_node[j] : jp.alpha_local[j];
+    const float b = cls ? jp.beta_node[j] : jp.beta_local[j];
+    ts = fmaf(b, (float)(K - 2), a);
+  }
+  const float rinv = adapt ? 1.f / (phi + M0) : 0.f;   // (c0 + M rinv) = 1 / EFFICIENCY; 1 when fixed
+  const float c0 = adapt ? phi * rinv : 1.f;
+  Best best = {0.f, 1.f, 0xFFFFFFFFu};
+  const int ns = adapt ? G : 1;
+  if (mmax >= 1) {
+    for (int i = lane; i < ns; i += 32) {
+      const long long M = adapt ? (long long)m_samples[(size_t)j * G + i] : (long long)M0;
+      if (M < 1) continue;
+      const long long per_gpu = (M + K - 1) / K;
+      const long long s = (per_gpu + mmax - 1) / mmax - 1;
+      const long long m = (per_gpu + s) / (s + 1);
+      const float Mrun = (float)((long long)K * m * (s + 1));
+      if (Mrun < M0 || Mrun > Mmax) continue;
+      const float tg = fmaf(b_g, (float)m, a_g);
+      const float tit = fmaf((float)s, tg, overlap_time(tg, ts, gamma, inv_gamma));
+      Best b;
+      b.num = Mrun;
+      b.den = tit * fmaf(Mrun, rinv, c0);
+      b.tie = (uint32_t)i;
+      if (beats(b, best)) best = b;
+    }
+  }
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    Best o;
+    o.num = __shfl_xor_sync(0xffffffffu, best.num, off);
+    o.den = __shfl_xor_sync(0xffffffffu, best.den, off);
+    o.tie = __shfl_xor_sync(0xffffffffu, best.tie, off);
+    if (beats(o, best)) best = o;
+  }
+  if (lane == 0) {
+    const bool found = best.num > 0.f;
+    gmax[out] = found ? best.num / best.den : 0.f;
+    amax[out] = found ? (uint16_t)best.tie : (uint16_t)0xFFFFu;
+  }
+}
+
 __device__ __forceinline__ bool kn_valid(int K, int N, int k_max, int n_max,
                                          const int32_t *__restrict__ kfit) {
   return N >= 1 && N <= n_max && K >= N && K <= k_max && K <= kfit[N];
@@ -288,6 +353,23 @@ int launch_autoscale(sched_ctx *ctx, const float *d_goodput, const int32_t *d_cu
   return SCHED_OK;
 }
 
+static int launch_expand(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodput, float *d_speedup,
+                         uint16_t *d_argmax) {
+  const sched_config &c = ctx->cfg;
+  const int J = c.num_jobs;
+  for (int j0 = 0; j0 < J; j0 += 65535) {      // grid.z is limited to 65535 jobs per launch
+    dim3 grid((unsigned)((ctx->ND + 31) / 32), 1u, (unsigned)std::min(65535, J - j0));
+    {
+      TimedLaunch tl_(ctx, KK_EXPAND);
+      speedup_expand_kernel<<<grid, dim3(32, 8), 0, ctx->stream>>>(ctx->d_gmax, ctx->d_amax, ctx->d_kfit,
+                                                                   jobs->fair_k, jobs->fair_n, j0, c.k_max, c.n_max,
+                                                                   d_goodput, d_speedup, d_argmax);
+    }
+    SCHED_LAUNCH_CHECK(ctx);
+  }
+  return SCHED_OK;
+}
+
 int launch_speedup_table(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodput, float *d_speedup,
                          uint16_t *d_argmax) {
   const sched_config &c = ctx->cfg;
@@ -310,17 +392,28 @@ int launch_speedup_table(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodpu
 #undef SWEEP
     SCHED_LAUNCH_CHECK(ctx);
   }
-  for (int j0 = 0; j0 < J; j0 += 65535) {      // grid.z is limited to 65535 jobs per launch
-    dim3 grid((unsigned)((ctx->ND + 31) / 32), 1u, (unsigned)std::min(65535, J - j0));
+  return launch_expand(ctx, jobs, d_goodput, d_speedup, d_argmax);
+}
+
+int launch_speedup_table_msample(sched_ctx *ctx, const sched_jobs *jobs, const int32_t *d_m_samples, int G,
+                                 const int32_t *d_m_max_gpu, const uint8_t *d_adaptive, float *d_goodput,
+                                 float *d_speedup, uint16_t *d_argmax) {
+  const sched_config &c = ctx->cfg;
+  const int J = c.num_jobs;
+  if (J == 0) return SCHED_OK;
+  JobPtrs jp = {jobs->alpha_grad, jobs->beta_grad, jobs->alpha_local, jobs->beta_local,
+                jobs->alpha_node, jobs->beta_node, jobs->gamma, jobs->phi, jobs->m0,
+                jobs->m_max_total};
+  if (ctx->num_pairs > 0) {
+    dim3 grid((unsigned)J, (unsigned)((ctx->num_pairs + 7) / 8));
     {
-      TimedLaunch tl_(ctx, KK_EXPAND);
-      speedup_expand_kernel<<<grid, dim3(32, 8), 0, ctx->stream>>>(ctx->d_gmax, ctx->d_amax, ctx->d_kfit,
-                                                                   jobs->fair_k, jobs->fair_n, j0, c.k_max, c.n_max,
-                                                                   d_goodput, d_speedup, d_argmax);
+      TimedLaunch tl_(ctx, KK_SWEEP);
+      msample_sweep_kernel<<<grid, 256, 0, ctx->stream>>>(jp, d_m_samples, d_m_max_gpu, d_adaptive, ctx->d_pairs,
+                                                          ctx->num_pairs, c.k_max, G, ctx->d_gmax, ctx->d_amax);
     }
     SCHED_LAUNCH_CHECK(ctx);
   }
-  return SCHED_OK;
+  return launch_expand(ctx, jobs, d_goodput, d_speedup, d_argmax);
 }
 
 int launch_realloc_factor(sched_ctx *ctx, const sched_jobs *jobs, float *d_out) {

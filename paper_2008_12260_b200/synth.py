@@ -105,6 +105,19 @@ def make_m_grid(m_max_gpu: np.ndarray, grid_m: int) -> np.ndarray:
     return out
 
 
+def make_m_samples(m0: np.ndarray, m_max_total: np.ndarray, num_samples: int) -> np.ndarray:
+    """Candidate total batch sizes per job: `num_samples` integers log-spaced from M0 to M_max
+    (inputs of the total-batch sampling search; built once on the host)."""
+    J = int(m0.shape[0])
+    out = np.empty((J, num_samples), dtype=np.int32)
+    for j in range(J):
+        lo, hi = math.log(float(m0[j])), math.log(float(m_max_total[j]))
+        for i in range(num_samples):
+            v = math.exp(lo + (hi - lo) * (i / (num_samples - 1) if num_samples > 1 else 0.0))
+            out[j, i] = min(max(int(math.floor(v + 0.5)), int(m0[j])), int(m_max_total[j]))
+    return out
+
+
 def draw_jobs(num_jobs: int, seed: int, grid_m: int, grid_s: int, k_max: int,
               phi_hi: float = 1e5, with_history: bool = False) -> Jobs:
     """Draw job parameters in a fixed order from PCG64(seed).
