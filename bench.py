@@ -294,6 +294,17 @@ def bench_table(api, torch, dev, stream, cfg, cl, jobs, sm_max_mhz, clocks):
         flush.fill_(1)                      # L2 flush between iterations
         sched.build_speedup_table(dj, gp, sp, am)
     t = sched.read_kernel_timing()
+    # the total-batch sampling search of Sec. 4.3 on the same jobs (128 candidates per job)
+    ms = torch.from_numpy(synth.make_m_samples(jobs.m0, jobs.m_max_total, 128)).to(dev)
+    mm = torch.from_numpy(jobs.m_max_gpu).to(dev)
+    for _ in range(3):
+        sched.build_speedup_table_msample(dj, ms, mm, gp, sp, am)
+    sched.read_kernel_timing()
+    for _ in range(reps):
+        flush.fill_(1)
+        sched.build_speedup_table_msample(dj, ms, mm, gp, sp, am)
+    t2 = sched.read_kernel_timing()
+    msample_ms = t2["goodput_sweep"][0] / reps
     sched.close()
     sweep_ms = t["goodput_sweep"][0] / reps
     expand_ms = t["speedup_expand"][0] / reps
@@ -306,6 +317,9 @@ def bench_table(api, torch, dev, stream, cfg, cl, jobs, sm_max_mhz, clocks):
         "expand_us": round(expand_ms * 1e3, 2),
         "evals_per_sec": points / ((sweep_ms + expand_ms) * 1e-3),
         "evals_per_sec_sweep_only": points / (sweep_ms * 1e-3),
+        "msample_search": {"candidates_per_job": 128, "sweep_us": round(msample_ms * 1e3, 2),
+                           "evals_per_sec": float(cfg.num_jobs) * distinct_classes(cl) * 128 / (msample_ms * 1e-3),
+                           "note": "integer (m, s) derivation + 3 MUFU per candidate; latency-sized at this size"},
         "roofline": {"kernel": "goodput_sweep", "bound": "alu", "achieved": achieved / 1e12, "peak": peak / 1e12,
                      "unit": "T lane-op/s", "frac": achieved / peak,
                      "peak_source": "%d SMs x %d fp32 lanes x %.0f MHz (max SM clock)" % (num_sms, FP32_LANES_PER_SM, sm_max_mhz),
