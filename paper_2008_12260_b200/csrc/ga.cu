@@ -1035,7 +1035,7 @@ int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint3
   aa.fitness_out = ctx->ff_out;
   ctx->fit_done = aa.fuse != 0;
   dim3 grid((unsigned)nbatch, (unsigned)count);
-  SCHED_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->d_colcount, 0, sizeof(unsigned int), ctx->stream));
+  if (!aa.fuse) SCHED_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->d_colcount, 0, sizeof(unsigned int), ctx->stream));
   {
     TimedLaunch tl_(ctx, KK_ROWS);
     // about four vectors per lane: several loads in flight and the per-row overhead shared

@@ -239,9 +239,18 @@ msample_sweep_kernel(JobPtrs jp, const int32_t *__restrict__ m_samples, const in
     for (int i = lane; i < ns; i += 32) {
       const long long M = adapt ? (long long)m_samples[(size_t)j * G + i] : (long long)M0;
       if (M < 1) continue;
-      const long long per_gpu = (M + K - 1) / K;
-      const long long s = (per_gpu + mmax - 1) / mmax - 1;
-      const long long m = (per_gpu + s) / (s + 1);
+      long long s, m;
+      if (M <= (1ll << 30)) {          // 32-bit divisions (the usual case) are several times cheaper
+        const unsigned Mu = (unsigned)M, Ku = (unsigned)K, mu = (unsigned)mmax;
+        const unsigned per_gpu = (Mu + Ku - 1u) / Ku;
+        const unsigned su = (per_gpu + mu - 1u) / mu - 1u;
+        s = su;
+        m = (per_gpu + su) / (su + 1u);
+      } else {
+        const long long per_gpu = (M + K - 1) / K;
+        s = (per_gpu + mmax - 1) / mmax - 1;
+        m = (per_gpu + s) / (s + 1);
+      }
       const float Mrun = (float)((long long)K * m * (s + 1));
       if (Mrun < M0 || Mrun > Mmax) continue;
       const float tg = fmaf(b_g, (float)m, a_g);
