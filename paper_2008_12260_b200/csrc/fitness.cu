@@ -19,7 +19,7 @@ template <>
 struct VecLoad<16> {
   static __device__ __forceinline__ uint4 ld(const void *p) {
     uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+    asm("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
   }
@@ -132,17 +132,28 @@ __global__ void __launch_bounds__(256) fitness_kernel(FitnessArgs a) {
     if (live) {
       const char *row = cand_base + (size_t)j * row_bytes;
       const char *crow = cur_base ? cur_base + (size_t)j * row_bytes : nullptr;
-#pragma unroll 4
-      for (int v = sub; v < row_vecs; v += LPR) {
-        const uint4 x = VecLoad<W>::ld(row + (size_t)v * W);
-        if ((x.x | x.y | x.z | x.w) != 0u) {
-          summarise_word(x.x, ksum, npos);
-          if (W >= 8) summarise_word(x.y, ksum, npos);
-          if (W >= 16) { summarise_word(x.z, ksum, npos); summarise_word(x.w, ksum, npos); }
+      // batches of up to 8 vectors per lane: all loads of a batch are issued before any is used
+      constexpr int B = 8;
+      for (int v0 = sub; v0 < row_vecs; v0 += LPR * B) {
+        uint4 x[B];
+#pragma unroll
+        for (int k = 0; k < B; ++k) {
+          const int v = v0 + k * LPR;
+          x[k] = make_uint4(0u, 0u, 0u, 0u);
+          if (v < row_vecs) x[k] = VecLoad<W>::ld(row + (size_t)v * W);
         }
-        if (crow) {
-          const uint4 c = VecLoad<W>::ld_cached(crow + (size_t)v * W);
-          diff |= (x.x ^ c.x) | (x.y ^ c.y) | (x.z ^ c.z) | (x.w ^ c.w);
+#pragma unroll
+        for (int k = 0; k < B; ++k) {
+          const int v = v0 + k * LPR;
+          if ((x[k].x | x[k].y | x[k].z | x[k].w) != 0u) {
+            summarise_word(x[k].x, ksum, npos);
+            if (W >= 8) summarise_word(x[k].y, ksum, npos);
+            if (W >= 16) { summarise_word(x[k].z, ksum, npos); summarise_word(x[k].w, ksum, npos); }
+          }
+          if (crow && v < row_vecs) {
+            const uint4 c = VecLoad<W>::ld_cached(crow + (size_t)v * W);
+            diff |= (x[k].x ^ c.x) | (x[k].y ^ c.y) | (x[k].z ^ c.z) | (x[k].w ^ c.w);
+          }
         }
       }
     }
