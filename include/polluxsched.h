@@ -150,6 +150,22 @@ int build_speedup_table_msample(sched_ctx *ctx, const sched_jobs *d_jobs, const 
                                 int32_t num_samples, const int32_t *d_m_max_gpu, const uint8_t *d_adaptive,
                                 float *d_goodput, float *d_speedup, uint16_t *d_argmax);
 
+/* Batched fit of the throughput-model parameters (Sec. 4.1, online model fitting).  For each
+ * of num_jobs jobs (independent of cfg.num_jobs) the observations offset[j] .. offset[j+1] of
+ * (K, N, m, s, T_iter) are fitted by theta = (alpha_grad, beta_grad, alpha_local, beta_local,
+ * alpha_node, beta_node, gamma) minimising the root mean squared logarithmic error
+ * sqrt(mean((ln(1 + T_pred) - ln(1 + T_obs))^2)) with T_pred from Eq. 11, subject to
+ * alpha, beta >= 0 and 1 <= gamma <= 10, starting from d_theta0 (fp32 [num_jobs][7], clamped
+ * into the bounds).  Bit i of d_frozen[j] (nullable) holds parameter i at its starting value:
+ * the paper's prior-driven exploration keeps unexplored synchronisation parameters at 0
+ * this way.  At most max_iters damped Gauss-Newton steps per job.  Outputs: d_theta_out fp32
+ * [num_jobs][7], d_loss_out fp32 [num_jobs] (the error reached; 0 for a job without
+ * observations, whose theta is returned unchanged).  The minimiser found is a local one. */
+int fit_throughput_model(sched_ctx *ctx, int32_t num_jobs, const int32_t *d_obs_offset, const int32_t *d_obs_k,
+                         const int32_t *d_obs_n, const int32_t *d_obs_m, const int32_t *d_obs_s,
+                         const float *d_obs_t, const float *d_theta0, const uint8_t *d_frozen, int32_t max_iters,
+                         float *d_theta_out, float *d_loss_out);
+
 /* REALLOC_FACTOR_j(delta) = (T_j - R_j delta) / (T_j + delta) clamped to [0, 1]
  * (Sec. 4.2), with delta = cfg.delta_sec.  d_out: fp32 [J].  Uses age_sec, num_restarts. */
 int compute_realloc_factor(sched_ctx *ctx, const sched_jobs *d_jobs, float *d_out);

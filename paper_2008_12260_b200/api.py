@@ -18,7 +18,7 @@ ERRORS = {-1: "INVALID_ARG", -2: "BAD_CONFIG", -3: "CUDA", -4: "TIMEOUT", -5: "N
 
 EXPORTS = (
     "sched_init", "sched_destroy", "sched_last_error", "sched_sync_status", "sched_launch_count",
-    "build_speedup_table", "build_speedup_table_msample", "compute_realloc_factor", "autoscale_targets", "eval_fitness", "repair_population",
+    "build_speedup_table", "build_speedup_table_msample", "fit_throughput_model", "compute_realloc_factor", "autoscale_targets", "eval_fitness", "repair_population",
     "init_population", "ga_generation", "schedule_round", "schedule_round_host",
     "sched_get_population", "sched_get_round_tables", "sched_round_speedup_table", "eval_fitness_host",
     "sched_set_kernel_timing", "sched_num_kernel_kinds", "sched_kernel_kind_name",
@@ -67,6 +67,7 @@ def load_library(path: str = LIB_PATH):
     lib.sched_launch_count.restype = C.c_int64
     lib.build_speedup_table.argtypes = [vp, C.POINTER(SchedJobs), vp, vp, vp]
     lib.build_speedup_table_msample.argtypes = [vp, C.POINTER(SchedJobs), vp, i32, vp, vp, vp, vp, vp]
+    lib.fit_throughput_model.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp]
     lib.compute_realloc_factor.argtypes = [vp, C.POINTER(SchedJobs), vp]
     lib.autoscale_targets.argtypes = [vp, vp, vp, i32, f32, f32, vp]
     lib.eval_fitness.argtypes = [vp, vp, i32, vp, vp, vp, vp, f32, vp]
@@ -228,6 +229,11 @@ class Scheduler:
         self._check(_lib.build_speedup_table_msample(self._ctx, C.byref(jobs.struct), _ptr(m_samples),
                                                      m_samples.shape[1], _ptr(m_max_gpu), _ptr(adaptive),
                                                      _ptr(goodput), _ptr(speedup), _ptr(argmax)))
+
+    def fit_throughput_model(self, offset, k, n, m, s, t, theta0, theta_out, loss_out, *, frozen=None, max_iters=100):
+        self._check(_lib.fit_throughput_model(self._ctx, theta0.shape[0], _ptr(offset), _ptr(k), _ptr(n), _ptr(m),
+                                              _ptr(s), _ptr(t), _ptr(theta0), _ptr(frozen), max_iters,
+                                              _ptr(theta_out), _ptr(loss_out)))
 
     def compute_realloc_factor(self, jobs, out):
         self._check(_lib.compute_realloc_factor(self._ctx, C.byref(jobs.struct), _ptr(out)))

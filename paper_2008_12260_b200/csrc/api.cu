@@ -304,7 +304,7 @@ int sched_num_kernel_kinds(void) { return KK_COUNT; }
 const char *sched_kernel_kind_name(int kind) {
   static const char *names[KK_COUNT] = {"goodput_sweep", "speedup_expand", "realloc_factor",
                                         "penalty_prep", "fitness", "rank", "rows", "cols",
-                                        "best_index", "copy_best", "colscan"};
+                                        "best_index", "copy_best", "colscan", "fit_theta"};
   return (kind >= 0 && kind < KK_COUNT) ? names[kind] : "";
 }
 
@@ -348,6 +348,20 @@ int build_speedup_table_msample(sched_ctx *ctx, const sched_jobs *d_jobs, const 
           "build_speedup_table_msample: num_samples must be in [1, 65535]");
   return launch_speedup_table_msample(ctx, d_jobs, d_m_samples, num_samples, d_m_max_gpu, d_adaptive, d_goodput,
                                       d_speedup, d_argmax);
+}
+
+int fit_throughput_model(sched_ctx *ctx, int32_t num_jobs, const int32_t *d_obs_offset, const int32_t *d_obs_k,
+                         const int32_t *d_obs_n, const int32_t *d_obs_m, const int32_t *d_obs_s,
+                         const float *d_obs_t, const float *d_theta0, const uint8_t *d_frozen, int32_t max_iters,
+                         float *d_theta_out, float *d_loss_out) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "fit_throughput_model: ctx is NULL");
+  REQUIRE(ctx, num_jobs >= 0 && max_iters >= 0, SCHED_ERR_INVALID_ARG,
+          "fit_throughput_model: num_jobs and max_iters must be >= 0");
+  REQUIRE(ctx, num_jobs == 0 || (d_obs_offset && d_obs_k && d_obs_n && d_obs_m && d_obs_s && d_obs_t && d_theta0 &&
+                                 d_theta_out && d_loss_out),
+          SCHED_ERR_INVALID_ARG, "fit_throughput_model: an observation array, d_theta0 or an output is NULL");
+  return launch_fit(ctx, num_jobs, d_obs_offset, d_obs_k, d_obs_n, d_obs_m, d_obs_s, d_obs_t, d_theta0, d_frozen,
+                    max_iters, d_theta_out, d_loss_out);
 }
 
 int compute_realloc_factor(sched_ctx *ctx, const sched_jobs *d_jobs, float *d_out) {

@@ -21,7 +21,7 @@
 // kernel classes, for launch accounting and optional per-kernel timing
 enum KernelKind {
   KK_SWEEP = 0, KK_EXPAND, KK_REALLOC, KK_PENPREP, KK_FITNESS, KK_RANK, KK_ROWS, KK_COLS, KK_BEST,
-  KK_COPY, KK_COLSCAN, KK_COUNT
+  KK_COPY, KK_COLSCAN, KK_FIT, KK_COUNT
 };
 
 struct TimedSpan {
@@ -234,6 +234,9 @@ int launch_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_a
                       const int16_t *d_pop_in, const float *d_fitness_in, int16_t *d_pop_out,
                       uint32_t generation);
 int launch_set_round(sched_ctx *ctx, uint32_t round);
+int launch_fit(sched_ctx *ctx, int32_t num_jobs, const int32_t *d_offset, const int32_t *d_k, const int32_t *d_n,
+               const int32_t *d_m, const int32_t *d_s, const float *d_t, const float *d_theta0,
+               const uint8_t *d_frozen, int32_t max_iters, float *d_theta_out, float *d_loss_out);
 int launch_select_best(sched_ctx *ctx, const int16_t *d_pop, const float *d_fitness,
                        int16_t *d_best, float *d_best_fitness);
 int ensure_fitness_scratch(sched_ctx *ctx, int32_t count, int chunks);

@@ -161,6 +161,26 @@ def draw_jobs(num_jobs: int, seed: int, grid_m: int, grid_s: int, k_max: int,
     )
 
 
+def draw_observations(jobs: "Jobs", per_job, seed: int, gpus_per_node: int = 4, noise: float = 0.02):
+    """Profiled iteration times for fitting: per job a list of (K, N, m, s, T_iter) tuples at
+    random allocations and batch sizes.  The times are passed in by the caller-supplied
+    function of the test or benchmark (this module holds no model arithmetic): here only the
+    configurations are drawn.  Returns (offset [J+1], K, N, m, s, noise factors)."""
+    g = np.random.Generator(np.random.PCG64(seed))
+    J = jobs.num_jobs
+    counts = np.full(J, per_job, dtype=np.int64) if np.isscalar(per_job) else np.asarray(per_job, dtype=np.int64)
+    offset = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    total = int(offset[-1])
+    K = g.integers(1, 17, total).astype(np.int32)
+    spread = g.integers(1, 5, total)
+    N = np.where(K == 1, 1, np.minimum(np.maximum(spread, -(-K // gpus_per_node)), K)).astype(np.int32)
+    job_of = np.repeat(np.arange(J), counts)
+    m = (1 + g.integers(0, 1 << 30, total) % np.maximum(jobs.m_max_gpu[job_of], 1)).astype(np.int32)
+    s = g.integers(0, 4, total).astype(np.int32)
+    factor = np.exp(g.normal(0.0, noise, total))
+    return offset, K, N, m, s, factor
+
+
 def random_feasible_allocation(cluster: Cluster, num_jobs: int, seed: int,
                                k_hi: int = 8, active: np.ndarray | None = None) -> np.ndarray:
     """A random allocation matrix that satisfies node capacity and interference avoidance.
