@@ -377,7 +377,7 @@ def bench_fit(api, torch, dev, stream):
     from oracle import fit as ofit
 
     J, per_job = 1024, 64
-    jobs = synth.draw_jobs(J, 7, 8, 4, 16)
+    jobs = synth.draw_jobs(J, 7, 8, 8, 16)
     offset, K, N, m, s, factor = synth.draw_observations(jobs, per_job, 8)
     true = np.stack([jobs.alpha_grad, jobs.beta_grad, jobs.alpha_local, jobs.beta_local, jobs.alpha_node,
                      jobs.beta_node, jobs.gamma], axis=1).astype(np.float64)
