@@ -42,10 +42,10 @@ HBM_FALLBACK_GBS = 6650.0
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
 # summarised in profiles/kernel_counters.md; None = kernel changed since the counters were taken.
-# "rows": one large-workload generation (234.7 MB read + 242.2 MB written).
+# "rows": one large-workload generation (237.1 MB read + 257.1 MB written).
 # "fitness_stress": 16 dense stress candidates moved 544.8 + 3.0 MB; every candidate is streamed
-# once, so the figure is scaled by candidates / 16 to the chunk that is timed.
-NCU_TRAFFIC_BYTES = {"rows": 476.9e6, "fitness_stress_per_candidate": 547.8e6 / 16}
+# once, so the figure is scaled by candidates / 16 to the chunk that is timed (544.8 + 3.5 MB).
+NCU_TRAFFIC_BYTES = {"rows": 494.2e6, "fitness_stress_per_candidate": 548.3e6 / 16}
 
 
 def measured_peaks():
