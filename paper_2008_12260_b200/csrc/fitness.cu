@@ -132,27 +132,48 @@ __global__ void __launch_bounds__(256) fitness_kernel(FitnessArgs a) {
     if (live) {
       const char *row = cand_base + (size_t)j * row_bytes;
       const char *crow = cur_base ? cur_base + (size_t)j * row_bytes : nullptr;
-      // batches of up to 8 vectors per lane: all loads of a batch are issued before any is used
-      constexpr int B = 8;
-      for (int v0 = sub; v0 < row_vecs; v0 += LPR * B) {
-        uint4 x[B];
+      // batches of vectors per lane: all loads of a batch are issued before any is used
+      if (!crow) {
+        constexpr int B = 8;
+        for (int v0 = sub; v0 < row_vecs; v0 += LPR * B) {
+          uint4 x[B];
 #pragma unroll
-        for (int k = 0; k < B; ++k) {
-          const int v = v0 + k * LPR;
-          x[k] = make_uint4(0u, 0u, 0u, 0u);
-          if (v < row_vecs) x[k] = VecLoad<W>::ld(row + (size_t)v * W);
-        }
-#pragma unroll
-        for (int k = 0; k < B; ++k) {
-          const int v = v0 + k * LPR;
-          if ((x[k].x | x[k].y | x[k].z | x[k].w) != 0u) {
-            summarise_word(x[k].x, ksum, npos);
-            if (W >= 8) summarise_word(x[k].y, ksum, npos);
-            if (W >= 16) { summarise_word(x[k].z, ksum, npos); summarise_word(x[k].w, ksum, npos); }
+          for (int k = 0; k < B; ++k) {
+            const int v = v0 + k * LPR;
+            x[k] = make_uint4(0u, 0u, 0u, 0u);
+            if (v < row_vecs) x[k] = VecLoad<W>::ld(row + (size_t)v * W);
           }
-          if (crow && v < row_vecs) {
-            const uint4 c = VecLoad<W>::ld_cached(crow + (size_t)v * W);
-            diff |= (x[k].x ^ c.x) | (x[k].y ^ c.y) | (x[k].z ^ c.z) | (x[k].w ^ c.w);
+#pragma unroll
+          for (int k = 0; k < B; ++k) {
+            if ((x[k].x | x[k].y | x[k].z | x[k].w) != 0u) {
+              summarise_word(x[k].x, ksum, npos);
+              if (W >= 8) summarise_word(x[k].y, ksum, npos);
+              if (W >= 16) { summarise_word(x[k].z, ksum, npos); summarise_word(x[k].w, ksum, npos); }
+            }
+          }
+        }
+      } else {
+        constexpr int B = 4;   // the current allocation's vectors travel with the candidate's
+        for (int v0 = sub; v0 < row_vecs; v0 += LPR * B) {
+          uint4 x[B], c[B];
+#pragma unroll
+          for (int k = 0; k < B; ++k) {
+            const int v = v0 + k * LPR;
+            x[k] = make_uint4(0u, 0u, 0u, 0u);
+            c[k] = make_uint4(0u, 0u, 0u, 0u);
+            if (v < row_vecs) {
+              x[k] = VecLoad<W>::ld(row + (size_t)v * W);
+              c[k] = VecLoad<W>::ld_cached(crow + (size_t)v * W);
+            }
+          }
+#pragma unroll
+          for (int k = 0; k < B; ++k) {
+            if ((x[k].x | x[k].y | x[k].z | x[k].w) != 0u) {
+              summarise_word(x[k].x, ksum, npos);
+              if (W >= 8) summarise_word(x[k].y, ksum, npos);
+              if (W >= 16) { summarise_word(x[k].z, ksum, npos); summarise_word(x[k].w, ksum, npos); }
+            }
+            diff |= (x[k].x ^ c[k].x) | (x[k].y ^ c[k].y) | (x[k].z ^ c[k].z) | (x[k].w ^ c[k].w);
           }
         }
       }
