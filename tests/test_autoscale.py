@@ -16,6 +16,13 @@ def test_hand_cases(oracle):
     assert oracle.autoscale_targets(g, 8, 2, 4, [2], 0.1, 0.1).tolist() == [2]       # already at the limit
     assert oracle.autoscale_targets(g, 8, 2, 4, [0], 0.1, 0.1).tolist() == [0]       # no nodes: untouched
     assert oracle.autoscale_targets(g, 8, 2, 4, [7], 0.1, 0.1).tolist() == [7]       # outside the table
+    # n_max = 3 nodes of 4 GPUs would need 12 > k_max = 8 GPUs: the search stops at 2 nodes.
+    # (A second job with large entries follows, so that a read past row k_max would show.)
+    g = np.zeros((2, 9, 4), np.float32)
+    g[0, 1, 1] = 1.0; g[0, 4, 1] = 3.5; g[0, 8, 2] = 4.0
+    g[1] = 100.0
+    assert oracle.autoscale_targets(g, 8, 3, 4, [1, 0], 2 / 3, 0.5).tolist() == [2, 0]
+    assert oracle.autoscale_targets(g, 8, 3, 4, [3, 0], 0.1, 0.1).tolist() == [3, 0]
 
 
 def test_properties_on_model_tables(oracle):

@@ -190,6 +190,10 @@ def test_selection_and_crossover_statistics(oracle):
     assert chi2 < 70.0                                           # 31 dof
     assert np.corrcoef(wins, expect)[0, 1] > 0.9
     assert abs(np.mean(from_b) - 0.5) < 0.03
+    # A fair coin per row over J = 40 rows leaves the minority parent about 0.44 of them
+    # (0.5 - E|Binomial(40, 1/2)/40 - 1/2|); a coin biased to 3/4 would leave it 0.25.
+    minority = np.minimum(from_b, 1.0 - np.asarray(from_b))
+    assert 0.41 < minority.mean() < 0.47
 
 
 def test_mutation_statistics(oracle):
