@@ -77,8 +77,15 @@ int ensure_round_scratch(sched_ctx *ctx) {
   const size_t pop = (size_t)c.population * c.num_jobs * c.num_nodes;
   const size_t tab = (size_t)c.num_jobs * ctx->KD * ctx->ND;
   int rc;
-  if ((rc = dev_alloc(ctx, &ctx->d_popA, pop)) != SCHED_OK) return rc;
-  if ((rc = dev_alloc(ctx, &ctx->d_popB, pop)) != SCHED_OK) return rc;
+  // Large problems keep the round's population in the row store, whose pool starts with the
+  // dense initial population; if it cannot be allocated the round runs on dense matrices.
+  if (rowstore_eligible(ctx, nullptr) && !ctx->rs_off) {
+    if (rowstore_ensure(ctx) != SCHED_OK) ctx->rs_off = true;
+  }
+  if (!ctx->rs_ready) {
+    if ((rc = dev_alloc(ctx, &ctx->d_popA, pop)) != SCHED_OK) return rc;
+    if ((rc = dev_alloc(ctx, &ctx->d_popB, pop)) != SCHED_OK) return rc;
+  }
   if ((rc = dev_alloc(ctx, &ctx->d_fit_buf, 2 * (size_t)c.population)) != SCHED_OK) return rc;
   ctx->d_fit = ctx->d_fit_buf;
   if ((rc = dev_alloc(ctx, &ctx->d_tab_goodput, tab)) != SCHED_OK) return rc;
@@ -264,7 +271,7 @@ int sched_destroy(sched_ctx *ctx) {
                   ctx->d_dflag, ctx->d_pen, ctx->d_partial, ctx->d_ticket, ctx->d_status,
                   ctx->d_popA, ctx->d_popB, ctx->d_fit_buf, ctx->d_tab_goodput, ctx->d_tab_speedup,
                   ctx->d_rf, ctx->d_best_idx, ctx->d_stage, ctx->d_stage_fit, ctx->d_colsum, ctx->d_summ, ctx->d_collist, ctx->d_colcount, ctx->d_rowticket, ctx->d_round, ctx->d_occcount, ctx->d_occlist,
-                  ctx->d_colelig};
+                  ctx->d_colelig, ctx->rs_pool, ctx->rs_rec, ctx->rs_summ, ctx->rs_ptr, ctx->rs_state};
   for (void *p : ptrs)
     if (p) cudaFree(p);
   if (ctx->graph_exec) cudaGraphExecDestroy(ctx->graph_exec);
@@ -304,7 +311,8 @@ int sched_num_kernel_kinds(void) { return KK_COUNT; }
 const char *sched_kernel_kind_name(int kind) {
   static const char *names[KK_COUNT] = {"goodput_sweep", "speedup_expand", "realloc_factor",
                                         "penalty_prep", "fitness", "rank", "rows", "cols",
-                                        "best_index", "copy_best", "colscan", "fit_theta"};
+                                        "best_index", "copy_best", "colscan", "fit_theta",
+                                        "generation_store", "store_build", "store_compact", "store_gather"};
   return (kind >= 0 && kind < KK_COUNT) ? names[kind] : "";
 }
 
@@ -475,9 +483,30 @@ static int round_body(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d
     return launch_fitness(ctx, pop, ctx->cfg.population, ctx->d_tab_speedup, d_cur, rf, d_jobs->active,
                           ctx->cfg.p, out, ctx->summ_valid ? ctx->round_summ : nullptr);
   };
+  const bool store = ctx->rs_ready;
+  if (store) pa = ctx->rs_pool;   // the dense initial population is the first P * J slots of the pool
   if (rc == SCHED_OK) rc = launch_init_population(ctx, d_jobs->k_cap, d_jobs->active, d_cur, pa);
   if (rc == SCHED_OK) rc = fitness_of(pa, fit_cur);
-  for (int g = 0; g < generations && rc == SCHED_OK; ++g) {
+  int parity = 0;
+  if (store && generations > 0) {
+    // From here on candidates are arrays of row indices: one kernel per generation does the
+    // operators, the repair and the fitness; every few generations a check moves the live rows
+    // to the other half of the pool if the half in use could run out.
+    if (rc == SCHED_OK) rc = rowstore_build(ctx, d_jobs->active, ctx->round_cur);
+    int phase = 0;
+    for (int g = 0; g < generations && rc == SCHED_OK; ++g) {
+      if (g > 0 && g % ctx->rs_check_every == 0) {
+        rc = rowstore_compact(ctx, parity, phase);
+        phase ^= 1;
+        if (rc != SCHED_OK) break;
+      }
+      rc = rowstore_generation(ctx, d_jobs->k_cap, d_jobs->active, ctx->round_cur, rf ? ctx->d_pen : nullptr,
+                               fit_cur, fit_next, parity, phase, (uint32_t)g);
+      parity ^= 1;
+      std::swap(fit_cur, fit_next);
+    }
+  }
+  for (int g = 0; g < generations && rc == SCHED_OK && !store; ++g) {
     ctx->ff_out = fit_next;
     // children's summaries go to the other half; the parents' feed the unperturbed rows
     ctx->round_summ_in = ctx->summ_valid ? ctx->round_summ : nullptr;
@@ -498,6 +527,12 @@ static int round_body(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d
   ctx->summ_valid = false;
   if (rc != SCHED_OK) return rc;
   ctx->d_pop_last = pa;
+  ctx->rs_ptr_last = nullptr;
+  if (store && generations > 0) {
+    ctx->rs_ptr_last = ctx->rs_ptr + (size_t)parity * ctx->cfg.population * ctx->cfg.num_jobs;
+    if ((rc = launch_select_best(ctx, nullptr, ctx->d_fit, nullptr, d_best_fitness)) != SCHED_OK) return rc;
+    return rowstore_gather(ctx, ctx->rs_ptr_last, 0, 1, ctx->d_best_idx, d_best);
+  }
   return launch_select_best(ctx, pa, ctx->d_fit, d_best, d_best_fitness);
 }
 
@@ -536,6 +571,7 @@ int schedule_round(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cu
     ctx->launches += ctx->graph_launches;
     ctx->d_fit = ctx->graph_fit;
     ctx->d_pop_last = ctx->graph_pop_last;
+    ctx->rs_ptr_last = ctx->graph_ptr_last;
     return SCHED_OK;
   }
   const bool capture = graphs_ok && ctx->seen_valid && same_round_key(key, ctx->seen_key);
@@ -572,6 +608,7 @@ int schedule_round(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cu
   ctx->graph_launches = captured;
   ctx->graph_fit = ctx->d_fit;
   ctx->graph_pop_last = ctx->d_pop_last;
+  ctx->graph_ptr_last = ctx->rs_ptr_last;
   SCHED_CUDA_CHECK(ctx, cudaGraphLaunch(ctx->graph_exec, ctx->stream));
   ctx->launches += captured;
   return SCHED_OK;
@@ -581,7 +618,10 @@ int sched_get_population(sched_ctx *ctx, int16_t *d_pop_out, float *d_fitness_ou
   REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "sched_get_population: ctx is NULL");
   REQUIRE(ctx, ctx->d_pop_last, SCHED_ERR_INVALID_ARG, "sched_get_population: no round has run yet");
   const sched_config &c = ctx->cfg;
-  if (d_pop_out)
+  if (d_pop_out && ctx->rs_ptr_last) {
+    int rc = rowstore_gather(ctx, ctx->rs_ptr_last, 0, c.population, nullptr, d_pop_out);
+    if (rc != SCHED_OK) return rc;
+  } else if (d_pop_out)
     SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(d_pop_out, ctx->d_pop_last,
                                           sizeof(int16_t) * (size_t)c.population * c.num_jobs * c.num_nodes,
                                           cudaMemcpyDeviceToDevice, ctx->stream));

@@ -21,7 +21,7 @@
 // kernel classes, for launch accounting and optional per-kernel timing
 enum KernelKind {
   KK_SWEEP = 0, KK_EXPAND, KK_REALLOC, KK_PENPREP, KK_FITNESS, KK_RANK, KK_ROWS, KK_COLS, KK_BEST,
-  KK_COPY, KK_COLSCAN, KK_FIT, KK_COUNT
+  KK_COPY, KK_COLSCAN, KK_FIT, KK_GENSTORE, KK_STORE_BUILD, KK_STORE_COMPACT, KK_STORE_GATHER, KK_COUNT
 };
 
 struct TimedSpan {
@@ -97,6 +97,19 @@ struct sched_ctx {
   int16_t *d_pop_last;   // points at d_popA or d_popB after a round
   bool round_ready;
 
+  // Row store of a running round (large problems): rows live once in a pool and candidates
+  // hold row indices, so a child row that equals its parent's costs one index.
+  int16_t *rs_pool;        // [2 * rs_half_cap + 1][num_nodes] row contents (last slot: the empty row)
+  uint32_t *rs_rec;        // [slots][8] occupied nodes of the row: node | GPUs << 12, or an overflow mark
+  uint32_t *rs_summ;       // [slots] K | N << 11 | (entries differing from the current allocation) << 22
+  uint32_t *rs_ptr;        // [2][P][J] row index per (candidate, job): parents and children alternate
+  unsigned int *rs_state;  // [2][2] {next free slot, half in use}; the two copies alternate at each compaction check
+  size_t rs_half_cap;      // slots per half of the pool
+  int rs_check_every;      // generations between compaction checks
+  bool rs_ready;           // the buffers above exist
+  bool rs_off;             // the store could not be allocated: rounds run on dense matrices
+  const uint32_t *rs_ptr_last;  // indices of the last round's final population, or NULL when it is dense
+
   // staging for the *_host entry points (allocated on first use)
   void *d_stage;         // job arrays + cur + best
   size_t stage_bytes;
@@ -112,6 +125,7 @@ struct sched_ctx {
   int64_t graph_launches;
   float *graph_fit;
   int16_t *graph_pop_last;
+  const uint32_t *graph_ptr_last;
 
   // optional per-kernel timing with CUDA events on the context's stream
   bool timing_on;
@@ -214,7 +228,25 @@ __device__ __forceinline__ uint32_t order_key(uint32_t bits) {
   return bits ^ ((bits >> 31) ? 0xFFFFFFFFu : 0x80000000u);
 }
 
-// kernels' launchers (defined in table.cu / fitness.cu / ga.cu)
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+  return v;
+}
+
+// node index of the t-th occupied entry (ascending) of a row held in shared memory
+__device__ __forceinline__ int nth_occupied(const int16_t *row, int num_nodes, uint32_t t, int lane) {
+  for (int base = 0; base < num_nodes; base += 32) {
+    const int n = base + lane;
+    const unsigned m = __ballot_sync(0xffffffffu, n < num_nodes && row[n] > 0);
+    const uint32_t c = __popc(m);
+    if (t < c) return base + (int)__fns(m, 0, (int)t + 1);
+    t -= c;
+  }
+  return -1;
+}
+
+// kernels' launchers (defined in table.cu / fitness.cu / ga.cu / rowstore.cu)
 int launch_speedup_table(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodput, float *d_speedup,
                          uint16_t *d_argmax);
 int launch_speedup_table_msample(sched_ctx *ctx, const sched_jobs *jobs, const int32_t *d_m_samples, int G,
@@ -243,3 +275,14 @@ int ensure_fitness_scratch(sched_ctx *ctx, int32_t count, int chunks);
 int ensure_dflag(sched_ctx *ctx, int32_t count);
 int launch_penalty_prep(sched_ctx *ctx, const int16_t *d_cur, const float *d_rf);
 int ensure_colscratch(sched_ctx *ctx, size_t ints);
+void fitness_chunking(const sched_ctx *ctx, int32_t count, int &rows_per_block, int &chunks);
+// row store (rowstore.cu)
+bool rowstore_eligible(const sched_ctx *ctx, const int16_t *d_cur);
+int rowstore_ensure(sched_ctx *ctx);
+int rowstore_build(sched_ctx *ctx, const uint8_t *d_active, const int16_t *d_cur);
+int rowstore_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active, const int16_t *d_cur,
+                        const float *d_pen, const float *d_fitness_in, float *d_fitness_out, int parity,
+                        int state_phase, uint32_t generation);
+int rowstore_compact(sched_ctx *ctx, int parity, int state_phase);
+int rowstore_gather(sched_ctx *ctx, const uint32_t *d_ptr, int first_candidate, int count, const int32_t *d_index,
+                    int16_t *d_out);

@@ -262,6 +262,13 @@ void fitness_geometry(size_t row_bytes, uintptr_t align_bits, int J, int count, 
 
 }  // namespace
 
+// Rows per block and blocks per candidate that launch_fitness uses for `count` candidates.
+void fitness_chunking(const sched_ctx *ctx, int32_t count, int &rows_per_block, int &chunks) {
+  int W, lpr_log2;
+  fitness_geometry((size_t)ctx->cfg.num_nodes * 2, 0, ctx->cfg.num_jobs, count, ctx->num_sms, W, lpr_log2,
+                   rows_per_block, chunks);
+}
+
 int launch_penalty_prep(sched_ctx *ctx, const int16_t *d_cur, const float *d_rf) {
   const int J = ctx->cfg.num_jobs;
   if (J == 0) return SCHED_OK;

@@ -57,24 +57,6 @@ struct RowsArgs {
   RngKey key;
 };
 
-__device__ __forceinline__ int warp_sum(int v) {
-#pragma unroll
-  for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-  return v;
-}
-
-// node index of the t-th occupied entry (ascending) of a row held in shared memory
-__device__ __forceinline__ int nth_occupied(const int16_t *row, int num_nodes, uint32_t t, int lane) {
-  for (int base = 0; base < num_nodes; base += 32) {
-    const int n = base + lane;
-    const unsigned m = __ballot_sync(0xffffffffu, n < num_nodes && row[n] > 0);
-    const uint32_t c = __popc(m);
-    if (t < c) return base + (int)__fns(m, 0, (int)t + 1);
-    t -= c;
-  }
-  return -1;
-}
-
 __global__ void __launch_bounds__(256) rows_kernel(RowsArgs a) {
   extern __shared__ __align__(16) int16_t s_rows[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -1149,7 +1131,7 @@ int launch_select_best(sched_ctx *ctx, const int16_t *d_pop, const float *d_fitn
   }
   SCHED_LAUNCH_CHECK(ctx);
   const size_t elems = (size_t)ctx->cfg.num_jobs * ctx->cfg.num_nodes;
-  if (elems == 0) return SCHED_OK;
+  if (elems == 0 || !d_pop) return SCHED_OK;   // no dense population: the caller gathers the rows
   const int blocks = (int)((elems + 256 * 8 - 1) / (256 * 8));
   {
   TimedLaunch tl_(ctx, KK_COPY);

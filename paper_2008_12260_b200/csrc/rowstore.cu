@@ -1,0 +1,826 @@
+// Row store: the population of a running scheduling round kept as shared rows (Sec. 4.3).
+//
+// A generation copies almost every child row verbatim from one of two parents; only the
+// perturbed rows and the few rows the repair touches are new.  Here a row's contents live
+// once in a pool and a candidate is an array of row indices.  Next to each stored row sit
+// its summary (K, N, entries that differ from the current allocation) and a short record of
+// its occupied nodes, so a generation reads 44 bytes per unchanged row instead of the row,
+// and writes 4.  New rows are appended to the pool (copy on write); when a half of the pool
+// runs low the live rows are copied to the other half.
+//
+// One block evolves one candidate per generation: parent selection, row-wise crossover,
+// perturbation, per-row caps, interference and capacity repair, and the candidate's fitness.
+// The operators, their random draws and the order of the fitness sums are the same as in
+// the dense kernels, so both paths produce identical populations and fitness bits.
+#include "common.cuh"
+#include "fitness_common.cuh"
+
+namespace {
+
+constexpr int REC_WORDS = 8;                  // occupied nodes a record can hold
+constexpr uint32_t REC_OVERFLOW = 0xFFFFFFFFu;  // first word of a record whose row has more
+constexpr int OCC = 16;                       // occupants listed per node inside a block
+constexpr int GEN_THREADS = 256;
+constexpr int GEN_WARPS = GEN_THREADS / 32;
+constexpr int STORE_MAX_JOBS = 8192;          // job index must fit 13 bits of an occupant entry
+
+struct StoreView {
+  int16_t *pool;
+  uint32_t *rec, *summ;
+  unsigned long long half_cap;
+  uint32_t zero_slot;
+};
+
+// K, N, entries differing from `cur_row` (NULL: none) and the occupant record of a row held
+// in shared memory.  All lanes return the same K, N, ndiff; rec_out (shared, REC_WORDS) is
+// complete after the trailing __syncwarp().
+__device__ __forceinline__ void summarise_row(const int16_t *row, int NN, const int16_t *cur_row, int lane,
+                                              int &K, int &N, int &ndiff, uint32_t *rec_out) {
+  int k = 0, nd = 0, cnt = 0;
+  for (int base = 0; base < NN; base += 32) {
+    const int n = base + lane;
+    const int v = (n < NN) ? (int)row[n] : 0;
+    if (cur_row && n < NN) nd += (v != (int)__ldg(cur_row + n)) ? 1 : 0;
+    k += v;
+    const unsigned m = __ballot_sync(0xffffffffu, v > 0);
+    const int pos = cnt + __popc(m & ((1u << lane) - 1u));
+    if (v > 0 && pos < REC_WORDS) rec_out[pos] = (uint32_t)n | ((uint32_t)v << 12);
+    cnt += __popc(m);
+  }
+  K = warp_sum(k);
+  ndiff = warp_sum(nd);
+  N = cnt;
+  __syncwarp();
+  if (cnt > REC_WORDS) {
+    if (lane == 0) rec_out[0] = REC_OVERFLOW;
+  } else if (lane >= cnt && lane < REC_WORDS) {
+    rec_out[lane] = 0u;
+  }
+  __syncwarp();
+}
+
+__device__ __forceinline__ uint32_t pack_summary(int K, int N, int ndiff) {
+  return (uint32_t)K | ((uint32_t)N << 11) | ((uint32_t)ndiff << 22);
+}
+
+// ---------------------------------------------------------------------------------------
+// Build: the dense initial population (rows c * J + j at the start of the pool) gets its
+// records and summaries; candidate c, job j points at slot c * J + j.
+// ---------------------------------------------------------------------------------------
+struct BuildArgs {
+  StoreView st;
+  uint32_t *ptr;            // [P][J]
+  unsigned int *state;      // {next free slot, half}
+  const uint8_t *active;
+  const int16_t *cur;       // or NULL
+  int P, J, NN;
+};
+
+__global__ void __launch_bounds__(256) rowstore_build_kernel(BuildArgs a) {
+  __shared__ __align__(16) int16_t s_row[8][512];
+  __shared__ uint32_t s_rec[8][REC_WORDS];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const long long rows = (long long)a.P * a.J;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    a.state[0] = (unsigned int)rows;
+    a.state[1] = 0u;
+  }
+  // the empty row: contents, record and summary all zero
+  if (blockIdx.x == 0) {
+    for (int n = threadIdx.x; n < a.NN; n += blockDim.x) a.st.pool[(size_t)a.st.zero_slot * a.NN + n] = 0;
+    if (threadIdx.x < REC_WORDS) a.st.rec[(size_t)a.st.zero_slot * REC_WORDS + threadIdx.x] = 0u;
+    if (threadIdx.x == 0) a.st.summ[a.st.zero_slot] = 0u;
+  }
+  for (long long r = (long long)blockIdx.x * 8 + warp; r < rows; r += (long long)gridDim.x * 8) {
+    const int j = (int)(r % a.J);
+    const uint4 *src = (const uint4 *)(a.st.pool + (size_t)r * a.NN);
+    for (int v = lane; v < (a.NN >> 3); v += 32) ((uint4 *)s_row[warp])[v] = src[v];
+    __syncwarp();
+    int K, N, nd;
+    summarise_row(s_row[warp], a.NN, a.cur ? a.cur + (size_t)j * a.NN : nullptr, lane, K, N, nd, s_rec[warp]);
+    const bool on = !a.active || a.active[j];
+    if (lane < REC_WORDS) a.st.rec[(size_t)r * REC_WORDS + lane] = s_rec[warp][lane];
+    if (lane == 0) {
+      a.st.summ[r] = on ? pack_summary(K, N, nd) : 0u;
+      a.ptr[r] = (uint32_t)r;
+    }
+    __syncwarp();
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Compaction check: when the half in use could run out within the next `gens_ahead`
+// generations (each may append up to P * J rows), every live row moves to the other half,
+// in candidate order, and the indices are rewritten.  The state is read from one copy and
+// written to the other, so no block sees it change under it.
+// ---------------------------------------------------------------------------------------
+struct CompactArgs {
+  StoreView st;
+  uint32_t *ptr;            // [P][J] indices of the current population (rewritten)
+  const unsigned int *state_in;
+  unsigned int *state_out;
+  int P, J, NN, gens_ahead;
+};
+
+__global__ void __launch_bounds__(256) rowstore_compact_kernel(CompactArgs a) {
+  const unsigned long long rows = (unsigned long long)a.P * a.J;
+  const unsigned int used = a.state_in[0], half = a.state_in[1];
+  const unsigned long long limit = (unsigned long long)(half + 1u) * a.st.half_cap;
+  const bool move = (unsigned long long)used + (unsigned long long)a.gens_ahead * rows > limit;
+  if (!move) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) { a.state_out[0] = used; a.state_out[1] = half; }
+    return;
+  }
+  const unsigned int new_half = 1u - half;
+  const unsigned long long base = (unsigned long long)new_half * a.st.half_cap;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    a.state_out[0] = (unsigned int)(base + rows);
+    a.state_out[1] = new_half;
+  }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int row_vecs = a.NN >> 3;
+  for (unsigned long long r = (unsigned long long)blockIdx.x * 8 + warp; r < rows; r += (unsigned long long)gridDim.x * 8) {
+    const uint32_t slot = a.ptr[r];
+    if (slot == a.st.zero_slot) continue;
+    const size_t dst = (size_t)(base + r);
+    const uint4 *s4 = (const uint4 *)(a.st.pool + (size_t)slot * a.NN);
+    uint4 *d4 = (uint4 *)(a.st.pool + dst * a.NN);
+    for (int v = lane; v < row_vecs; v += 32) d4[v] = s4[v];
+    if (lane < REC_WORDS) a.st.rec[dst * REC_WORDS + lane] = a.st.rec[(size_t)slot * REC_WORDS + lane];
+    if (lane == 0) {
+      a.st.summ[dst] = a.st.summ[slot];
+      a.ptr[r] = (uint32_t)dst;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Gather: dense rows of `count` candidates (first_candidate .., or the single candidate
+// *index when index is not NULL) from their indices.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+rowstore_gather_kernel(StoreView st, const uint32_t *__restrict__ ptr, int first_candidate, long long rows,
+                       const int32_t *__restrict__ index, int J, int NN, int16_t *__restrict__ out) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const long long first = (long long)(index ? *index : first_candidate) * J;
+  const int row_vecs = NN >> 3;
+  const bool aligned = ((uintptr_t)out & 15) == 0;
+  for (long long r = (long long)blockIdx.x * 8 + warp; r < rows; r += (long long)gridDim.x * 8) {
+    const uint32_t slot = ptr[first + r];
+    if (aligned) {
+      const uint4 *s4 = (const uint4 *)(st.pool + (size_t)slot * NN);
+      uint4 *d4 = (uint4 *)(out + (size_t)r * NN);
+      for (int v = lane; v < row_vecs; v += 32) d4[v] = s4[v];
+    } else {
+      for (int n = lane; n < NN; n += 32) out[(size_t)r * NN + n] = st.pool[(size_t)slot * NN + n];
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// One generation of one candidate per block.
+// ---------------------------------------------------------------------------------------
+struct GenArgs {
+  StoreView st;
+  const uint32_t *ptr_in;   // [P][J] parents
+  uint32_t *ptr_out;        // [P][J] children
+  unsigned int *state;      // {next free slot, half}
+  const int16_t *cap;       // [NN]
+  const int32_t *k_cap;     // [J] or NULL
+  const uint8_t *active;    // [J] or NULL
+  const uint32_t *fitness_bits;  // [P] parents' fitness
+  const int16_t *cur;       // [J][NN] or NULL
+  int P, J, NN, k_max, n_max, num_elite;
+  uint32_t thr, gen;
+  RngKey key;
+  TermParams tp;
+  int rows_per_chunk, chunks;   // the dense fitness kernel's chunking, reproduced for identical sums
+  float *fitness_out;       // [P]
+  int *status;
+};
+
+// what the per-node repair decides for the occupant held by this lane (entry = job | GPUs << 13
+// | distributed << 31 in the first have_n lanes): the GPUs the job keeps on the node
+__device__ __forceinline__ int decide_entries(const GenArgs &a, uint32_t c, int nn, int tot, int ne, int cap_n,
+                                              int lane, uint32_t entry, int have_n) {
+  const int J = a.J;
+  const bool have = lane < have_n;
+  const int j = (int)(entry & 0x1FFFu);
+  int v = have ? (int)((entry >> 13) & 0x7FFu) : 0;
+  const bool dist = have && (entry >> 31);
+  if (ne >= 2) {
+    const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
+    int t = J;
+    if (dist && v > 0) { t = j - o; if (t < 0) t += J; }
+    int best = t;
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, off));
+    int removed = 0;
+    if (dist && v > 0 && t != best) { removed = v; v = 0; }
+    tot -= warp_sum(removed);
+  }
+  const int excess = tot - cap_n;
+  if (excess > 0) {
+    const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J);
+    int rot = 0x7fffffff;
+    if (have) { rot = j - o; if (rot < 0) rot += J; }
+    int ahead = 0;                       // GPUs of the occupants that come first in rotated order
+#pragma unroll
+    for (int k = 0; k < 32; ++k) {
+      const int rk = __shfl_sync(0xffffffffu, rot, k);
+      const int vk = __shfl_sync(0xffffffffu, v, k);
+      if (rk < rot) ahead += vk;
+    }
+    if (have) v -= min(v, max(excess - ahead, 0));
+  }
+  return v;
+}
+
+// Shared-memory carve-up of the generation kernel (sizes in bytes, 16-byte aligned pieces).
+struct GenSmem {
+  size_t slot, summ, term_mark, tot, el, cnt, viol, occ, occnew_row, mut, ovf, mod, cap, rec, total;
+};
+
+__host__ __device__ inline GenSmem gen_smem_layout(int J, int NN) {
+  GenSmem L;
+  size_t off = 0;
+#define TAKE(field, bytes) do { L.field = off; off += ((size_t)(bytes) + 15) & ~(size_t)15; } while (0)
+  TAKE(slot, (size_t)J * 4);
+  TAKE(summ, (size_t)J * 4);
+  TAKE(term_mark, (size_t)J * 4);              // marks during the repair, terms afterwards
+  TAKE(tot, (size_t)NN * 4);
+  TAKE(el, (size_t)NN * 4);
+  TAKE(cnt, (size_t)NN * 4);
+  TAKE(viol, (size_t)NN);
+  TAKE(occ, (size_t)NN * OCC * 4);
+  // decided GPU counts of the listed occupants; the same bytes serve as the warps' row buffers
+  // before the column pass and after it
+  const size_t occnew = (size_t)NN * OCC * 2, rowbuf = (size_t)GEN_WARPS * NN * 2;
+  TAKE(occnew_row, occnew > rowbuf ? occnew : rowbuf);
+  TAKE(mut, (size_t)J * 2);
+  TAKE(ovf, (size_t)J * 2);
+  TAKE(mod, (size_t)J * 2);
+  TAKE(cap, (size_t)NN * 2);
+  TAKE(rec, (size_t)GEN_WARPS * REC_WORDS * 4);
+#undef TAKE
+  L.total = off;
+  return L;
+}
+
+// Column value of job j on node nn as the capacity pass must see it: zero when the
+// interference pass removes it.
+__device__ __forceinline__ int column_value(const GenArgs &a, const uint32_t *s_slot, const uint32_t *s_summ, int j,
+                                            int nn, int keep, bool intf, bool &dist) {
+  const int v = (int)a.st.pool[(size_t)s_slot[j] * a.NN + nn];
+  dist = ((s_summ[j] >> 11) & 0x7FFu) >= 2u;
+  if (intf && dist && v > 0 && j != keep) return 0;
+  return v;
+}
+
+// Repair of a node whose occupants did not fit the block's list: passes over the whole
+// column through the row indices.  APPLY false: only marks the rows that will change.
+template <bool APPLY, typename MarkFn>
+__device__ void repair_column_scan(const GenArgs &a, uint32_t c, const uint32_t *s_slot, const uint32_t *s_summ,
+                                   int nn, int tot, int ne, int cap_n, int lane, MarkFn mark) {
+  const int J = a.J, NN = a.NN;
+  int keep = -1;
+  const bool intf = ne >= 2;
+  if (intf) {
+    const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
+    int best = J;
+    for (int j = lane; j < J; j += 32) {
+      const int v = (int)a.st.pool[(size_t)s_slot[j] * NN + nn];
+      if (v > 0 && ((s_summ[j] >> 11) & 0x7FFu) >= 2u) {
+        int t = j - o;
+        if (t < 0) t += J;
+        best = min(best, t);
+      }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, off));
+    keep = o + best;
+    if (keep >= J) keep -= J;
+    int removed = 0;
+    for (int j = lane; j < J; j += 32) {
+      const int v = (int)a.st.pool[(size_t)s_slot[j] * NN + nn];
+      if (v > 0 && ((s_summ[j] >> 11) & 0x7FFu) >= 2u && j != keep) removed += v;
+    }
+    tot -= warp_sum(removed);
+  }
+  int excess = tot - cap_n;
+  // the capacity pass walks every job once in rotated order; jobs removed by the interference
+  // pass count as empty there and are written (or marked) on the way
+  const int o = (excess > 0) ? (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J) : 0;
+  for (int t0 = 0; t0 < J; t0 += 32) {
+    const int t = t0 + lane;
+    int j = o + t;
+    if (j >= J) j -= J;
+    int v_old = 0, v_eff = 0;
+    if (t < J) {
+      bool dist;
+      v_old = (int)a.st.pool[(size_t)s_slot[j] * NN + nn];
+      v_eff = column_value(a, s_slot, s_summ, j, nn, keep, intf, dist);
+    }
+    int s = v_eff;                                // inclusive prefix over the 32 jobs
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int u = __shfl_up_sync(0xffffffffu, s, off);
+      if (lane >= off) s += u;
+    }
+    const int take = (excess > 0) ? min(v_eff, max(excess - (s - v_eff), 0)) : 0;
+    const int v_new = v_eff - take;
+    if (t < J && v_new != v_old) {
+      if (APPLY) a.st.pool[(size_t)s_slot[j] * NN + nn] = (int16_t)v_new;
+      else mark(j);
+    }
+    excess -= __shfl_sync(0xffffffffu, s, 31);
+  }
+}
+
+__global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArgs a) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int J = a.J, NN = a.NN, P = a.P;
+  const GenSmem L = gen_smem_layout(J, NN);
+  uint32_t *s_slot = (uint32_t *)(smem + L.slot);
+  uint32_t *s_summ = (uint32_t *)(smem + L.summ);
+  int *s_mark = (int *)(smem + L.term_mark);       // bit 0: changed by the column pass, bit 1: row is new
+  float *s_term = (float *)(smem + L.term_mark);
+  int *s_tot = (int *)(smem + L.tot), *s_el = (int *)(smem + L.el), *s_cnt = (int *)(smem + L.cnt);
+  uint8_t *s_viol = (uint8_t *)(smem + L.viol);
+  uint32_t *s_occ = (uint32_t *)(smem + L.occ);
+  uint16_t *s_occnew = (uint16_t *)(smem + L.occnew_row);
+  int16_t *s_rowbuf = (int16_t *)(smem + L.occnew_row);
+  uint16_t *s_mut = (uint16_t *)(smem + L.mut), *s_ovf = (uint16_t *)(smem + L.ovf), *s_mod = (uint16_t *)(smem + L.mod);
+  int16_t *s_cap = (int16_t *)(smem + L.cap);
+  uint32_t *s_rec = (uint32_t *)(smem + L.rec);
+  __shared__ int s_nmut, s_novf, s_nmod, s_ncow, s_fail;
+  __shared__ unsigned int s_base_mut, s_base_cow;
+  __shared__ int s_parent[2], s_rank4[4];
+  __shared__ double s_acc[GEN_WARPS];
+  __shared__ int s_acn[GEN_WARPS];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t c = blockIdx.x;
+  const bool elite = (int)c < a.num_elite;
+
+  for (int i = tid; i < NN; i += GEN_THREADS) {
+    s_tot[i] = 0; s_el[i] = 0; s_cnt[i] = 0; s_viol[i] = 0;
+    s_cap[i] = (int16_t)max((int)a.cap[i], 0);
+  }
+  for (int i = tid; i < J; i += GEN_THREADS) s_mark[i] = 0;
+  if (tid == 0) { s_nmut = 0; s_novf = 0; s_nmod = 0; s_ncow = 0; s_fail = 0; }
+
+  // ---- parents: the candidate of rank c for an elite child, else the better-ranked of two
+  // random pairs (rank = candidates ordered before, fitness descending, index ascending) ----
+  if (elite) {
+    for (int i = tid; i < P; i += GEN_THREADS) {
+      const uint32_t ki = order_key(a.fitness_bits[i]);
+      int rk = 0;
+      for (int o = 0; o < P; ++o) {
+        const uint32_t ko = order_key(__ldg(a.fitness_bits + o));
+        rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
+      }
+      if (rk == (int)c) s_parent[0] = s_parent[1] = i;
+    }
+  } else {
+    const u32x4 sel = draw(a.key, 0u, c, a.gen, SLOT_SELECT);
+    const int idx[4] = {(int)bounded(sel.x, P), (int)bounded(sel.y, P), (int)bounded(sel.z, P), (int)bounded(sel.w, P)};
+    if (warp < 4) {
+      const int i = idx[warp];
+      const uint32_t ki = order_key(a.fitness_bits[i]);
+      int rk = 0;
+      for (int o = lane; o < P; o += 32) {
+        const uint32_t ko = order_key(__ldg(a.fitness_bits + o));
+        rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
+      }
+      rk = warp_sum(rk);
+      if (lane == 0) s_rank4[warp] = rk;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      s_parent[0] = s_rank4[0] <= s_rank4[1] ? idx[0] : idx[1];
+      s_parent[1] = s_rank4[2] <= s_rank4[3] ? idx[2] : idx[3];
+    }
+  }
+  __syncthreads();
+
+  // occupant (job j holds g GPUs on node n) into the node's totals and list
+  auto add_occupant = [&](int j, int n, int g, bool dist) {
+    atomicAdd(&s_tot[n], g);
+    if (dist) atomicAdd(&s_el[n], 1);
+    const int k = atomicAdd(&s_cnt[n], 1);
+    if (k < OCC) s_occ[n * OCC + k] = (uint32_t)j | ((uint32_t)g << 13) | (dist ? 0x80000000u : 0u);
+  };
+
+  // ---- rows, one thread each: the child row is the chosen parent's row -----------------------
+  const uint32_t *pin_a = a.ptr_in + (size_t)s_parent[0] * J, *pin_b = a.ptr_in + (size_t)s_parent[1] * J;
+  for (int j = tid; j < J; j += GEN_THREADS) {
+    if (a.active && !a.active[j]) {
+      s_slot[j] = a.st.zero_slot;
+      s_summ[j] = 0u;
+      continue;
+    }
+    bool second = false, mut = false;
+    if (!elite) {
+      second = (draw(a.key, (uint32_t)j, c, a.gen, SLOT_XOVER).x >> 31) != 0u;
+      mut = draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE).x < a.thr;
+    }
+    const uint32_t slot = second ? pin_b[j] : pin_a[j];
+    s_slot[j] = slot;
+    const uint32_t w = a.st.summ[slot];
+    s_summ[j] = w;
+    if (mut) {
+      s_mut[atomicAdd(&s_nmut, 1)] = (uint16_t)j;
+      continue;
+    }
+    const uint4 r0 = *(const uint4 *)(a.st.rec + (size_t)slot * REC_WORDS);
+    if (r0.x == REC_OVERFLOW) {
+      s_ovf[atomicAdd(&s_novf, 1)] = (uint16_t)j;
+      continue;
+    }
+    if (r0.x == 0u) continue;
+    const bool dist = ((w >> 11) & 0x7FFu) >= 2u;
+    const uint4 r1 = *(const uint4 *)(a.st.rec + (size_t)slot * REC_WORDS + 4);
+    const uint32_t e[REC_WORDS] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+#pragma unroll
+    for (int k = 0; k < REC_WORDS; ++k)
+      if (e[k]) add_occupant(j, (int)(e[k] & 0xFFFu), (int)((e[k] >> 12) & 0x7FFu), dist);
+  }
+  __syncthreads();
+  if (tid == 0 && s_nmut > 0) {
+    const unsigned int base = atomicAdd(a.state, (unsigned int)s_nmut);
+    const unsigned long long limit = (unsigned long long)(a.state[1] + 1u) * a.st.half_cap;
+    s_base_mut = base;
+    if ((unsigned long long)base + (unsigned long long)s_nmut > limit) { s_fail = 1; atomicExch(a.status, SCHED_ERR_TOO_LARGE); }
+  }
+  __syncthreads();
+
+  // ---- perturbed rows, one warp each: new row in a fresh slot ---------------------------------
+  int16_t *row = s_rowbuf + (size_t)warp * NN;
+  uint32_t *recw = s_rec + warp * REC_WORDS;
+  const int row_vecs = NN >> 3;
+  if (!s_fail) {
+    for (int i = warp; i < s_nmut; i += GEN_WARPS) {
+      const int j = (int)s_mut[i];
+      const uint32_t old = s_slot[j], w = s_summ[j];
+      const uint4 *s4 = (const uint4 *)(a.st.pool + (size_t)old * NN);
+      for (int v = lane; v < row_vecs; v += 32) ((uint4 *)row)[v] = s4[v];
+      __syncwarp();
+      int rK = (int)(w & 0x7FFu), rN = (int)((w >> 11) & 0x7FFu);
+      const u32x4 mw = draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE);
+      const uint32_t op = bounded(mw.y, 3u);
+      if (op == 0u) {
+        const int n = (int)bounded(mw.w, (uint32_t)NN);
+        if (lane == 0) row[n] = (int16_t)min((int)row[n] + 1, (int)s_cap[n]);
+      } else if (rN > 0) {
+        const int ns = nth_occupied(row, NN, bounded(mw.z, (uint32_t)rN), lane);
+        if (op == 1u) {
+          if (lane == 0) row[ns] = (int16_t)(row[ns] - 1);
+        } else {
+          const int nd = (int)bounded(mw.w, (uint32_t)NN);
+          if (nd != ns && lane == 0) {
+            row[nd] = (int16_t)min((int)row[nd] + (int)row[ns], (int)s_cap[nd]);
+            row[ns] = 0;
+          }
+        }
+      }
+      __syncwarp();
+      rK = 0; rN = 0;
+      for (int n = lane; n < NN; n += 32) { rK += row[n]; rN += row[n] > 0; }
+      rK = warp_sum(rK);
+      rN = warp_sum(rN);
+      // per-row caps: replicas above the job's cap leave from the highest node index down, then
+      // occupied nodes beyond n_max are cleared from the highest index down
+      int kc = a.k_cap ? a.k_cap[j] : a.k_max;
+      kc = max(0, min(kc, a.k_max));
+      if (rK > kc || rN > a.n_max) {
+        if (lane == 0) {
+          int excess = rK - kc;
+          for (int n = NN - 1; n >= 0 && excess > 0; --n) {
+            const int take = min((int)row[n], excess);
+            row[n] = (int16_t)(row[n] - take);
+            excess -= take;
+          }
+          int occ = 0;
+          for (int n = 0; n < NN; ++n) {
+            if (row[n] > 0) {
+              ++occ;
+              if (occ > a.n_max) row[n] = 0;
+            }
+          }
+        }
+        __syncwarp();
+      }
+      int K, N, nd;
+      summarise_row(row, NN, a.cur ? a.cur + (size_t)j * NN : nullptr, lane, K, N, nd, recw);
+      const uint32_t slot = s_base_mut + (uint32_t)i;
+      uint4 *d4 = (uint4 *)(a.st.pool + (size_t)slot * NN);
+      for (int v = lane; v < row_vecs; v += 32) d4[v] = ((const uint4 *)row)[v];
+      if (lane < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + lane] = recw[lane];
+      const uint32_t word = pack_summary(K, N, nd);
+      if (lane == 0) {
+        a.st.summ[slot] = word;
+        s_slot[j] = slot;
+        s_summ[j] = word;
+        s_mark[j] = 2;
+      }
+      const bool dist = N >= 2;
+      for (int n = lane; n < NN; n += 32)
+        if (row[n] > 0) add_occupant(j, n, (int)row[n], dist);
+      __syncwarp();
+    }
+  }
+  // rows with more occupied nodes than a record holds: occupants from the row itself
+  for (int i = warp; i < s_novf; i += GEN_WARPS) {
+    const int j = (int)s_ovf[i];
+    const int16_t *src = a.st.pool + (size_t)s_slot[j] * NN;
+    const bool dist = ((s_summ[j] >> 11) & 0x7FFu) >= 2u;
+    for (int n = lane; n < NN; n += 32) {
+      const int v = (int)src[n];
+      if (v > 0) add_occupant(j, n, v, dist);
+    }
+  }
+  __syncthreads();
+
+  // ---- column pass, decisions: which occupants of the violating nodes change ------------------
+  auto mark_row = [&](int j) {
+    if ((atomicOr(&s_mark[j], 1) & 1) == 0) s_mod[atomicAdd(&s_nmod, 1)] = (uint16_t)j;
+  };
+  for (int nb = warp * 32; nb < NN; nb += GEN_WARPS * 32) {
+    const int n = nb + lane;
+    const int total = (n < NN) ? s_tot[n] : 0, nelig = (n < NN) ? s_el[n] : 0;
+    const int cp = (n < NN) ? (int)s_cap[n] : 0;
+    unsigned todo = __ballot_sync(0xffffffffu, n < NN && (nelig >= 2 || total > cp));
+    while (todo) {
+      const int srcl = __ffs(todo) - 1;
+      todo &= todo - 1;
+      const int nn = nb + srcl;
+      const int tot_n = __shfl_sync(0xffffffffu, total, srcl), ne_n = __shfl_sync(0xffffffffu, nelig, srcl);
+      const int cap_n = __shfl_sync(0xffffffffu, cp, srcl);
+      const int have_n = s_cnt[nn];
+      if (have_n > OCC) {
+        if (lane == 0) s_viol[nn] = 2;
+        repair_column_scan<false>(a, c, s_slot, s_summ, nn, tot_n, ne_n, cap_n, lane, mark_row);
+      } else {
+        const uint32_t entry = (lane < have_n) ? s_occ[nn * OCC + lane] : 0u;
+        const int v_new = decide_entries(a, c, nn, tot_n, ne_n, cap_n, lane, entry, have_n);
+        if (lane < have_n) {
+          s_occnew[nn * OCC + lane] = (uint16_t)v_new;
+          if (v_new != (int)((entry >> 13) & 0x7FFu)) mark_row((int)(entry & 0x1FFFu));
+        }
+        if (lane == 0) s_viol[nn] = 1;
+      }
+      __syncwarp();
+    }
+  }
+  __syncthreads();
+
+  // ---- rows the column pass changes get a slot of their own unless they are new already -------
+  const int nmod = s_nmod;
+  for (int i = tid; i < nmod; i += GEN_THREADS) {
+    const int j = (int)s_mod[i];
+    s_ovf[i] = (s_mark[j] & 2) ? (uint16_t)0xFFFFu : (uint16_t)atomicAdd(&s_ncow, 1);
+  }
+  __syncthreads();
+  if (tid == 0 && s_ncow > 0) {
+    const unsigned int base = atomicAdd(a.state, (unsigned int)s_ncow);
+    const unsigned long long limit = (unsigned long long)(a.state[1] + 1u) * a.st.half_cap;
+    s_base_cow = base;
+    if ((unsigned long long)base + (unsigned long long)s_ncow > limit) { s_fail = 1; atomicExch(a.status, SCHED_ERR_TOO_LARGE); }
+  }
+  __syncthreads();
+  if (!s_fail) {
+    for (int i = warp; i < nmod; i += GEN_WARPS) {
+      const uint32_t k = s_ovf[i];
+      if (k == 0xFFFFu) continue;
+      const int j = (int)s_mod[i];
+      const uint32_t slot = s_base_cow + k;
+      const uint4 *s4 = (const uint4 *)(a.st.pool + (size_t)s_slot[j] * NN);
+      uint4 *d4 = (uint4 *)(a.st.pool + (size_t)slot * NN);
+      for (int v = lane; v < row_vecs; v += 32) d4[v] = s4[v];
+      __syncwarp();
+      if (lane == 0) s_slot[j] = slot;
+    }
+  }
+  __syncthreads();
+
+  // ---- column pass, writes --------------------------------------------------------------------
+  if (!s_fail && nmod > 0) {
+    for (int i = tid; i < NN * OCC; i += GEN_THREADS) {
+      const int n = i / OCC, k = i - n * OCC;
+      if (s_viol[n] != 1 || k >= s_cnt[n]) continue;
+      const uint32_t entry = s_occ[i];
+      const int v_new = (int)s_occnew[i];
+      if (v_new != (int)((entry >> 13) & 0x7FFu))
+        a.st.pool[(size_t)s_slot[entry & 0x1FFFu] * NN + n] = (int16_t)v_new;
+    }
+    for (int nn = warp; nn < NN; nn += GEN_WARPS) {
+      if (s_viol[nn] != 2) continue;
+      repair_column_scan<true>(a, c, s_slot, s_summ, nn, s_tot[nn], s_el[nn], (int)s_cap[nn], lane, [](int) {});
+    }
+  }
+  __syncthreads();
+
+  // ---- changed rows: summary and record from the row as it now stands -------------------------
+  if (!s_fail) {
+    for (int i = warp; i < nmod; i += GEN_WARPS) {
+      const int j = (int)s_mod[i];
+      const uint32_t slot = s_slot[j];
+      const volatile int16_t *src = a.st.pool + (size_t)slot * NN;   // written in this kernel: no read-only path
+      for (int n = lane; n < NN; n += 32) row[n] = src[n];
+      __syncwarp();
+      int K, N, nd;
+      summarise_row(row, NN, a.cur ? a.cur + (size_t)j * NN : nullptr, lane, K, N, nd, recw);
+      if (lane < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + lane] = recw[lane];
+      const uint32_t word = pack_summary(K, N, nd);
+      if (lane == 0) {
+        a.st.summ[slot] = word;
+        s_summ[j] = word;
+      }
+      __syncwarp();
+    }
+  }
+  __syncthreads();
+
+  // ---- children's indices out, fitness of the candidate (Eq. 14) ------------------------------
+  uint32_t *pout = a.ptr_out + (size_t)c * J;
+  for (int j = tid; j < J; j += GEN_THREADS) {
+    pout[j] = s_slot[j];
+    if (!a.tp.active || a.tp.active[j]) {
+      const uint32_t w = s_summ[j];
+      s_term[j] = fitness_term(a.tp, j, (int)(w & 0x7FFu), (int)((w >> 11) & 0x7FFu), (w >> 22) != 0u);
+    }
+  }
+  __syncthreads();
+  // sums in the order of the dense fitness kernel: per chunk of rows, thread t adds rows t,
+  // t + 256, ... in double, a shuffle tree per warp, the warps in index order; then the chunks
+  // in index order
+  double ts = 0.0, ns = 0.0;
+  for (int ch = 0; ch < a.chunks; ++ch) {
+    const int j0 = ch * a.rows_per_chunk, j1 = min(J, j0 + a.rows_per_chunk);
+    double acc = 0.0;
+    int cnt = 0;
+    for (int j = j0 + tid; j < j1; j += GEN_THREADS) {
+      if (!a.tp.active || a.tp.active[j]) { acc += (double)s_term[j]; cnt += 1; }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+      acc += __shfl_xor_sync(0xffffffffu, acc, off);
+      cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
+    }
+    if (lane == 0) { s_acc[warp] = acc; s_acn[warp] = cnt; }
+    __syncthreads();
+    if (tid == 0) {
+      double t = 0.0;
+      int n = 0;
+      for (int w = 0; w < GEN_WARPS; ++w) { t += s_acc[w]; n += s_acn[w]; }
+      ts += t;
+      ns += (double)n;
+    }
+    __syncthreads();
+  }
+  if (tid == 0) a.fitness_out[c] = fitness_finalise(a.tp.mode, a.tp.p, ts, ns);
+}
+
+StoreView store_view(const sched_ctx *ctx) {
+  StoreView v;
+  v.pool = ctx->rs_pool; v.rec = ctx->rs_rec; v.summ = ctx->rs_summ;
+  v.half_cap = ctx->rs_half_cap;
+  v.zero_slot = (uint32_t)(2 * ctx->rs_half_cap);
+  return v;
+}
+
+}  // namespace
+
+// The row store serves rounds whose candidates span several row batches of the dense
+// kernels (J > 256; smaller problems run a generation as one dense kernel already), with
+// rows of whole 16-byte vectors and sizes that fit the packed fields.
+bool rowstore_eligible(const sched_ctx *ctx, const int16_t *) {
+  const sched_config &c = ctx->cfg;
+  if (c.num_jobs <= 256 || c.num_jobs > STORE_MAX_JOBS) return false;
+  if (c.num_nodes % 8 != 0 || c.num_nodes > 512 || ctx->cap_max > 2047) return false;
+  if (c.k_max > 2047 || c.n_max > 2047) return false;
+  const unsigned long long rows = (unsigned long long)c.population * c.num_jobs;
+  if (12ull * rows >= (1ull << 32)) return false;   // slot indices are 32-bit
+  if (gen_smem_layout(c.num_jobs, c.num_nodes).total > 200 * 1024) return false;
+  // at least three populations' worth of slots per half; beyond 8 GiB of pool the dense path runs
+  const unsigned long long row_bytes = (unsigned long long)c.num_nodes * 2 + REC_WORDS * 4 + 4;
+  return 6ull * rows * row_bytes <= (8ull << 30);
+}
+
+int rowstore_ensure(sched_ctx *ctx) {
+  if (ctx->rs_ready) return SCHED_OK;
+  const sched_config &c = ctx->cfg;
+  const unsigned long long rows = (unsigned long long)c.population * c.num_jobs;
+  const unsigned long long row_bytes = (unsigned long long)c.num_nodes * 2 + REC_WORDS * 4 + 4;
+  // half = (1 + gens between checks + slack) populations; shrink until the pool fits 8 GiB
+  int check = 2, slack = 2;
+  while (2ull * (1 + check + slack) * rows * row_bytes > (8ull << 30) && (check > 1 || slack > 1)) {
+    if (slack > 1) --slack; else --check;
+  }
+  ctx->rs_check_every = check;
+  ctx->rs_half_cap = (size_t)((1 + check + slack) * rows);
+  const size_t slots = 2 * ctx->rs_half_cap + 1;
+  cudaError_t e = cudaMalloc((void **)&ctx->rs_pool, slots * c.num_nodes * sizeof(int16_t));
+  if (e == cudaSuccess) e = cudaMalloc((void **)&ctx->rs_rec, slots * REC_WORDS * sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMalloc((void **)&ctx->rs_summ, slots * sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMalloc((void **)&ctx->rs_ptr, 2 * (size_t)rows * sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMalloc((void **)&ctx->rs_state, 4 * sizeof(unsigned int));
+  if (e == cudaSuccess) {
+    const size_t smem = gen_smem_layout(c.num_jobs, c.num_nodes).total;
+    if (smem > 48 * 1024)
+      e = cudaFuncSetAttribute(generation_store_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  }
+  if (e != cudaSuccess) {
+    set_error(ctx, "row store allocation failed: %s", cudaGetErrorString(e));
+    for (void *p : {(void *)ctx->rs_pool, (void *)ctx->rs_rec, (void *)ctx->rs_summ, (void *)ctx->rs_ptr, (void *)ctx->rs_state})
+      if (p) cudaFree(p);
+    ctx->rs_pool = nullptr; ctx->rs_rec = nullptr; ctx->rs_summ = nullptr; ctx->rs_ptr = nullptr; ctx->rs_state = nullptr;
+    cudaGetLastError();
+    return SCHED_ERR_CUDA;
+  }
+  ctx->scratch_epoch++;
+  ctx->rs_ready = true;
+  return SCHED_OK;
+}
+
+int rowstore_build(sched_ctx *ctx, const uint8_t *d_active, const int16_t *d_cur) {
+  const sched_config &c = ctx->cfg;
+  BuildArgs a;
+  a.st = store_view(ctx);
+  a.ptr = ctx->rs_ptr;
+  a.state = ctx->rs_state;
+  a.active = d_active; a.cur = d_cur;
+  a.P = c.population; a.J = c.num_jobs; a.NN = c.num_nodes;
+  {
+    TimedLaunch tl_(ctx, KK_STORE_BUILD);
+    rowstore_build_kernel<<<ctx->num_sms * 8, 256, 0, ctx->stream>>>(a);
+  }
+  SCHED_LAUNCH_CHECK(ctx);
+  return SCHED_OK;
+}
+
+int rowstore_compact(sched_ctx *ctx, int parity, int state_phase) {
+  const sched_config &c = ctx->cfg;
+  CompactArgs a;
+  a.st = store_view(ctx);
+  a.ptr = ctx->rs_ptr + (size_t)parity * c.population * c.num_jobs;
+  a.state_in = ctx->rs_state + 2 * state_phase;
+  a.state_out = ctx->rs_state + 2 * (state_phase ^ 1);
+  a.P = c.population; a.J = c.num_jobs; a.NN = c.num_nodes;
+  a.gens_ahead = ctx->rs_check_every;
+  {
+    TimedLaunch tl_(ctx, KK_STORE_COMPACT);
+    rowstore_compact_kernel<<<ctx->num_sms * 8, 256, 0, ctx->stream>>>(a);
+  }
+  SCHED_LAUNCH_CHECK(ctx);
+  return SCHED_OK;
+}
+
+int rowstore_gather(sched_ctx *ctx, const uint32_t *d_ptr, int first_candidate, int count, const int32_t *d_index,
+                    int16_t *d_out) {
+  const sched_config &c = ctx->cfg;
+  const long long rows = (long long)count * c.num_jobs;
+  if (rows == 0) return SCHED_OK;
+  const long long want = (rows + 7) / 8;
+  const int blocks = (int)(want < (long long)ctx->num_sms * 8 ? want : (long long)ctx->num_sms * 8);
+  {
+    TimedLaunch tl_(ctx, KK_STORE_GATHER);
+    rowstore_gather_kernel<<<blocks, 256, 0, ctx->stream>>>(store_view(ctx), d_ptr, first_candidate, rows, d_index,
+                                                           c.num_jobs, c.num_nodes, d_out);
+  }
+  SCHED_LAUNCH_CHECK(ctx);
+  return SCHED_OK;
+}
+
+int rowstore_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active, const int16_t *d_cur,
+                        const float *d_pen, const float *d_fitness_in, float *d_fitness_out, int parity,
+                        int state_phase, uint32_t generation) {
+  const sched_config &c = ctx->cfg;
+  const size_t rows = (size_t)c.population * c.num_jobs;
+  GenArgs a;
+  a.st = store_view(ctx);
+  a.ptr_in = ctx->rs_ptr + (size_t)parity * rows;
+  a.ptr_out = ctx->rs_ptr + (size_t)(parity ^ 1) * rows;
+  a.state = ctx->rs_state + 2 * state_phase;
+  a.cap = ctx->d_cap; a.k_cap = d_k_cap; a.active = d_active;
+  a.fitness_bits = (const uint32_t *)d_fitness_in;
+  a.cur = d_cur;
+  a.P = c.population; a.J = c.num_jobs; a.NN = c.num_nodes;
+  a.k_max = c.k_max; a.n_max = c.n_max; a.num_elite = c.num_elite;
+  a.thr = c.thr_mutate; a.gen = generation;
+  a.key = make_key(c.seed, ctx->d_round);
+  a.tp.table = ctx->d_tab_speedup; a.tp.pen = d_pen; a.tp.active = d_active;
+  a.tp.k_max = c.k_max; a.tp.n_max = c.n_max; a.tp.mode = fitness_mode(c.p); a.tp.p = c.p;
+  a.tp.floor_ = c.speedup_floor;
+  fitness_chunking(ctx, c.population, a.rows_per_chunk, a.chunks);
+  a.fitness_out = d_fitness_out;
+  a.status = ctx->d_status;
+  const size_t smem = gen_smem_layout(c.num_jobs, c.num_nodes).total;
+  {
+    TimedLaunch tl_(ctx, KK_GENSTORE);
+    generation_store_kernel<<<c.population, GEN_THREADS, smem, ctx->stream>>>(a);
+  }
+  SCHED_LAUNCH_CHECK(ctx);
+  return SCHED_OK;
+}
