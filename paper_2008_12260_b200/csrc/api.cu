@@ -271,7 +271,7 @@ int sched_destroy(sched_ctx *ctx) {
                   ctx->d_dflag, ctx->d_pen, ctx->d_partial, ctx->d_ticket, ctx->d_status,
                   ctx->d_popA, ctx->d_popB, ctx->d_fit_buf, ctx->d_tab_goodput, ctx->d_tab_speedup,
                   ctx->d_rf, ctx->d_best_idx, ctx->d_stage, ctx->d_stage_fit, ctx->d_colsum, ctx->d_summ, ctx->d_collist, ctx->d_colcount, ctx->d_rowticket, ctx->d_round, ctx->d_occcount, ctx->d_occlist,
-                  ctx->d_colelig, ctx->rs_pool, ctx->rs_rec, ctx->rs_summ, ctx->rs_ptr, ctx->rs_state};
+                  ctx->d_colelig, ctx->rs_pool, ctx->rs_rec, ctx->rs_ptr, ctx->rs_state};
   for (void *p : ptrs)
     if (p) cudaFree(p);
   if (ctx->graph_exec) cudaGraphExecDestroy(ctx->graph_exec);
@@ -492,7 +492,7 @@ static int round_body(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d
     // From here on candidates are arrays of row indices: one kernel per generation does the
     // operators, the repair and the fitness; every few generations a check moves the live rows
     // to the other half of the pool if the half in use could run out.
-    if (rc == SCHED_OK) rc = rowstore_build(ctx, d_jobs->active, ctx->round_cur);
+    if (rc == SCHED_OK) rc = rowstore_build(ctx, d_jobs->active, ctx->round_cur, rf ? ctx->d_pen : nullptr);
     int phase = 0;
     for (int g = 0; g < generations && rc == SCHED_OK; ++g) {
       if (g > 0 && g % ctx->rs_check_every == 0) {

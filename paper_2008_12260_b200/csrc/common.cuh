@@ -100,8 +100,8 @@ struct sched_ctx {
   // Row store of a running round (large problems): rows live once in a pool and candidates
   // hold row indices, so a child row that equals its parent's costs one index.
   int16_t *rs_pool;        // [2 * rs_half_cap + 1][num_nodes] row contents (last slot: the empty row)
-  uint32_t *rs_rec;        // [slots][8] occupied nodes of the row: node | GPUs << 12, or an overflow mark
-  uint32_t *rs_summ;       // [slots] K | N << 11 | (entries differing from the current allocation) << 22
+  uint32_t *rs_rec;        // [slots][8] up to 7 occupied nodes of the row (node | GPUs << 12, or an overflow
+                           // mark), then K | N << 11 | (entries differing from the current allocation) << 22
   uint32_t *rs_ptr;        // [2][P][J] row index per (candidate, job): parents and children alternate
   unsigned int *rs_state;  // [2][2] {next free slot, half in use}; the two copies alternate at each compaction check
   size_t rs_half_cap;      // slots per half of the pool
@@ -228,11 +228,7 @@ __device__ __forceinline__ uint32_t order_key(uint32_t bits) {
   return bits ^ ((bits >> 31) ? 0xFFFFFFFFu : 0x80000000u);
 }
 
-__device__ __forceinline__ int warp_sum(int v) {
-#pragma unroll
-  for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-  return v;
-}
+__device__ __forceinline__ int warp_sum(int v) { return __reduce_add_sync(0xffffffffu, v); }
 
 // node index of the t-th occupied entry (ascending) of a row held in shared memory
 __device__ __forceinline__ int nth_occupied(const int16_t *row, int num_nodes, uint32_t t, int lane) {
@@ -279,7 +275,7 @@ void fitness_chunking(const sched_ctx *ctx, int32_t count, int &rows_per_block, 
 // row store (rowstore.cu)
 bool rowstore_eligible(const sched_ctx *ctx, const int16_t *d_cur);
 int rowstore_ensure(sched_ctx *ctx);
-int rowstore_build(sched_ctx *ctx, const uint8_t *d_active, const int16_t *d_cur);
+int rowstore_build(sched_ctx *ctx, const uint8_t *d_active, const int16_t *d_cur, const float *d_pen);
 int rowstore_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active, const int16_t *d_cur,
                         const float *d_pen, const float *d_fitness_in, float *d_fitness_out, int parity,
                         int state_phase, uint32_t generation);

@@ -20,12 +20,16 @@ struct TermParams {
   float p, floor_;
 };
 
-// x_j^p of one row (SPEEDUP looked up at (K, N), re-allocation penalty, floor), in the form
-// that the mode sums: x, 1/x, ln x, sqrt x or x^p.
-__device__ __forceinline__ float fitness_term(const TermParams &tp, int j, int K, int N, bool changed) {
+// Table position of SPEEDUP_j at (K, N), both clamped into the table.
+__device__ __forceinline__ size_t fitness_table_index(const TermParams &tp, int j, int K, int N) {
   K = min(K, tp.k_max);
   N = min(N, tp.n_max);
-  float x = __ldg(tp.table + ((size_t)j * (tp.k_max + 1) + K) * (tp.n_max + 1) + N);
+  return ((size_t)j * (tp.k_max + 1) + K) * (tp.n_max + 1) + N;
+}
+
+// x_j^p from the looked-up speedup x: re-allocation penalty, floor, and the form that the
+// mode sums (x, 1/x, ln x, sqrt x or x^p).
+__device__ __forceinline__ float fitness_term_of(const TermParams &tp, int j, float x, bool changed) {
   if (tp.pen && changed) x *= tp.pen[j];
   x = fmaxf(x, tp.floor_);
   switch (tp.mode) {
@@ -35,6 +39,11 @@ __device__ __forceinline__ float fitness_term(const TermParams &tp, int j, int K
     case MODE_SQRT: return sqrtf(x);
     default: return powf(x, tp.p);
   }
+}
+
+// x_j^p of one row (SPEEDUP looked up at (K, N), re-allocation penalty, floor).
+__device__ __forceinline__ float fitness_term(const TermParams &tp, int j, int K, int N, bool changed) {
+  return fitness_term_of(tp, j, __ldg(tp.table + fitness_table_index(tp, j, K, N)), changed);
 }
 
 // Sum and count of the terms s_term[0 .. nrows) of the active rows j_first + i, in a fixed

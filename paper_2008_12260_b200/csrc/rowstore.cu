@@ -3,9 +3,10 @@
 // A generation copies almost every child row verbatim from one of two parents; only the
 // perturbed rows and the few rows the repair touches are new.  Here a row's contents live
 // once in a pool and a candidate is an array of row indices.  Next to each stored row sit
-// its summary (K, N, entries that differ from the current allocation) and a short record of
-// its occupied nodes, so a generation reads 44 bytes per unchanged row instead of the row,
-// and writes 4.  New rows are appended to the pool (copy on write); when a half of the pool
+// a 32-byte record: up to six occupied nodes, the row's summary (K, N, entries that differ
+// from the current allocation) and its term of the fitness sum (a stored row always serves
+// the same job, so the term is fixed for the round).  A generation reads 36 bytes per
+// unchanged row instead of the row, and writes 4.  New rows are appended to the pool (copy on write); when a half of the pool
 // runs low the live rows are copied to the other half.
 //
 // One block evolves one candidate per generation: parent selection, row-wise crossover,
@@ -17,47 +18,71 @@
 
 namespace {
 
-constexpr int REC_WORDS = 8;                  // occupied nodes a record can hold
+constexpr int REC_WORDS = 8;                  // words of a record: REC_ENTRIES occupants, the row's fitness term, its summary
+constexpr int REC_ENTRIES = 6;                // occupied nodes a record can hold
+constexpr int REC_TERM = 6, REC_SUMM = 7;     // positions of the term (float bits) and the summary
 constexpr uint32_t REC_OVERFLOW = 0xFFFFFFFFu;  // first word of a record whose row has more
 constexpr int OCC = 16;                       // occupants listed per node inside a block
 constexpr int GEN_THREADS = 256;
 constexpr int GEN_WARPS = GEN_THREADS / 32;
 constexpr int STORE_MAX_JOBS = 8192;          // job index must fit 13 bits of an occupant entry
+constexpr int COW_RESERVE = 24;               // slots a block takes up front for rows the column pass changes
 
 struct StoreView {
   int16_t *pool;
-  uint32_t *rec, *summ;
+  uint32_t *rec;
   unsigned long long half_cap;
   uint32_t zero_slot;
 };
 
-// K, N, entries differing from `cur_row` (NULL: none) and the occupant record of a row held
-// in shared memory.  All lanes return the same K, N, ndiff; rec_out (shared, REC_WORDS) is
-// complete after the trailing __syncwarp().
+// K, N, entries differing from `cur_row` (NULL: none) and the occupant entries of a row; both
+// rows are held in shared memory.  All lanes return the same K, N, ndiff; rec_out (shared, REC_WORDS: the
+// entries, the summary word is the caller's) is complete after the trailing __syncwarp().
 __device__ __forceinline__ void summarise_row(const int16_t *row, int NN, const int16_t *cur_row, int lane,
                                               int &K, int &N, int &ndiff, uint32_t *rec_out) {
   int k = 0, nd = 0, cnt = 0;
   for (int base = 0; base < NN; base += 32) {
     const int n = base + lane;
     const int v = (n < NN) ? (int)row[n] : 0;
-    if (cur_row && n < NN) nd += (v != (int)__ldg(cur_row + n)) ? 1 : 0;
+    if (cur_row && n < NN) nd += (v != (int)cur_row[n]) ? 1 : 0;
     k += v;
     const unsigned m = __ballot_sync(0xffffffffu, v > 0);
     const int pos = cnt + __popc(m & ((1u << lane) - 1u));
-    if (v > 0 && pos < REC_WORDS) rec_out[pos] = (uint32_t)n | ((uint32_t)v << 12);
+    if (v > 0 && pos < REC_ENTRIES) rec_out[pos] = (uint32_t)n | ((uint32_t)v << 12);
     cnt += __popc(m);
   }
   K = warp_sum(k);
   ndiff = warp_sum(nd);
   N = cnt;
   __syncwarp();
-  if (cnt > REC_WORDS) {
+  if (cnt > REC_ENTRIES) {
     if (lane == 0) rec_out[0] = REC_OVERFLOW;
-  } else if (lane >= cnt && lane < REC_WORDS) {
+  } else if (lane >= cnt && lane < REC_ENTRIES) {
     rec_out[lane] = 0u;
   }
   __syncwarp();
 }
+
+// A row of NN entries from global to shared memory, 16 bytes per lane and step when the
+// source allows; `cg` reads through to L2 (for rows written earlier in the same kernel).
+template <bool CG>
+__device__ __forceinline__ void load_row(int16_t *dst, const int16_t *src, int NN, int lane) {
+  if (((uintptr_t)src & 15) == 0) {
+    for (int v = lane; v < (NN >> 3); v += 32)
+      ((uint4 *)dst)[v] = CG ? __ldcg((const uint4 *)src + v) : *((const uint4 *)src + v);
+  } else {
+    for (int n = lane; n < NN; n += 32) dst[n] = CG ? __ldcg(src + n) : src[n];
+  }
+}
+
+// one 32-byte record with a single request
+__device__ __forceinline__ void load_record(uint32_t (&r)[REC_WORDS], const uint32_t *p) {
+  asm volatile("ld.global.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "l"(p) : "memory");
+}
+
+__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 __device__ __forceinline__ uint32_t pack_summary(int K, int N, int ndiff) {
   return (uint32_t)K | ((uint32_t)N << 11) | ((uint32_t)ndiff << 22);
@@ -73,11 +98,13 @@ struct BuildArgs {
   unsigned int *state;      // {next free slot, half}
   const uint8_t *active;
   const int16_t *cur;       // or NULL
+  TermParams tp;
   int P, J, NN;
 };
 
 __global__ void __launch_bounds__(256) rowstore_build_kernel(BuildArgs a) {
   __shared__ __align__(16) int16_t s_row[8][512];
+  __shared__ __align__(16) int16_t s_cur[8][512];
   __shared__ uint32_t s_rec[8][REC_WORDS];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const long long rows = (long long)a.P * a.J;
@@ -89,28 +116,34 @@ __global__ void __launch_bounds__(256) rowstore_build_kernel(BuildArgs a) {
   if (blockIdx.x == 0) {
     for (int n = threadIdx.x; n < a.NN; n += blockDim.x) a.st.pool[(size_t)a.st.zero_slot * a.NN + n] = 0;
     if (threadIdx.x < REC_WORDS) a.st.rec[(size_t)a.st.zero_slot * REC_WORDS + threadIdx.x] = 0u;
-    if (threadIdx.x == 0) a.st.summ[a.st.zero_slot] = 0u;
   }
   for (long long r = (long long)blockIdx.x * 8 + warp; r < rows; r += (long long)gridDim.x * 8) {
     const int j = (int)(r % a.J);
-    const uint4 *src = (const uint4 *)(a.st.pool + (size_t)r * a.NN);
-    for (int v = lane; v < (a.NN >> 3); v += 32) ((uint4 *)s_row[warp])[v] = src[v];
+    load_row<false>(s_row[warp], a.st.pool + (size_t)r * a.NN, a.NN, lane);
+    if (a.cur) load_row<false>(s_cur[warp], a.cur + (size_t)j * a.NN, a.NN, lane);
     __syncwarp();
     int K, N, nd;
-    summarise_row(s_row[warp], a.NN, a.cur ? a.cur + (size_t)j * a.NN : nullptr, lane, K, N, nd, s_rec[warp]);
+    summarise_row(s_row[warp], a.NN, a.cur ? s_cur[warp] : nullptr, lane, K, N, nd, s_rec[warp]);
     const bool on = !a.active || a.active[j];
-    if (lane < REC_WORDS) a.st.rec[(size_t)r * REC_WORDS + lane] = s_rec[warp][lane];
     if (lane == 0) {
-      a.st.summ[r] = on ? pack_summary(K, N, nd) : 0u;
+      s_rec[warp][REC_SUMM] = on ? pack_summary(K, N, nd) : 0u;
+      s_rec[warp][REC_TERM] = on ? __float_as_uint(fitness_term(a.tp, j, K, N, nd != 0)) : 0u;
       a.ptr[r] = (uint32_t)r;
     }
+    __syncwarp();
+    if (lane < REC_WORDS) a.st.rec[(size_t)r * REC_WORDS + lane] = s_rec[warp][lane];
     __syncwarp();
   }
 }
 
+// most slots one generation can take: every row new, plus every block's reserve
+__host__ __device__ inline unsigned long long store_worst_case(int P, int J) {
+  return (unsigned long long)P * J + (unsigned long long)P * COW_RESERVE;
+}
+
 // ---------------------------------------------------------------------------------------
 // Compaction check: when the half in use could run out within the next `gens_ahead`
-// generations (each may append up to P * J rows), every live row moves to the other half,
+// generations (each may take up to store_worst_case slots), every live row moves to the other half,
 // in candidate order, and the indices are rewritten.  The state is read from one copy and
 // written to the other, so no block sees it change under it.
 // ---------------------------------------------------------------------------------------
@@ -126,7 +159,7 @@ __global__ void __launch_bounds__(256) rowstore_compact_kernel(CompactArgs a) {
   const unsigned long long rows = (unsigned long long)a.P * a.J;
   const unsigned int used = a.state_in[0], half = a.state_in[1];
   const unsigned long long limit = (unsigned long long)(half + 1u) * a.st.half_cap;
-  const bool move = (unsigned long long)used + (unsigned long long)a.gens_ahead * rows > limit;
+  const bool move = (unsigned long long)used + (unsigned long long)a.gens_ahead * store_worst_case(a.P, a.J) > limit;
   if (!move) {
     if (blockIdx.x == 0 && threadIdx.x == 0) { a.state_out[0] = used; a.state_out[1] = half; }
     return;
@@ -147,10 +180,7 @@ __global__ void __launch_bounds__(256) rowstore_compact_kernel(CompactArgs a) {
     uint4 *d4 = (uint4 *)(a.st.pool + dst * a.NN);
     for (int v = lane; v < row_vecs; v += 32) d4[v] = s4[v];
     if (lane < REC_WORDS) a.st.rec[dst * REC_WORDS + lane] = a.st.rec[(size_t)slot * REC_WORDS + lane];
-    if (lane == 0) {
-      a.st.summ[dst] = a.st.summ[slot];
-      a.ptr[r] = (uint32_t)dst;
-    }
+    if (lane == 0) a.ptr[r] = (uint32_t)dst;
   }
 }
 
@@ -225,8 +255,7 @@ __device__ __forceinline__ int decide_entries(const GenArgs &a, uint32_t c, int 
     int rot = 0x7fffffff;
     if (have) { rot = j - o; if (rot < 0) rot += J; }
     int ahead = 0;                       // GPUs of the occupants that come first in rotated order
-#pragma unroll
-    for (int k = 0; k < 32; ++k) {
+    for (int k = 0; k < have_n; ++k) {
       const int rk = __shfl_sync(0xffffffffu, rot, k);
       const int vk = __shfl_sync(0xffffffffu, v, k);
       if (rk < rot) ahead += vk;
@@ -238,7 +267,7 @@ __device__ __forceinline__ int decide_entries(const GenArgs &a, uint32_t c, int 
 
 // Shared-memory carve-up of the generation kernel (sizes in bytes, 16-byte aligned pieces).
 struct GenSmem {
-  size_t slot, summ, term_mark, tot, el, cnt, viol, occ, occnew_row, mut, ovf, mod, cap, rec, total;
+  size_t slot, summ, term, mark, tot, el, cnt, viol, occ, occnew_row, mut, ovf, mod, cap, rec, total;
 };
 
 __host__ __device__ inline GenSmem gen_smem_layout(int J, int NN) {
@@ -247,15 +276,16 @@ __host__ __device__ inline GenSmem gen_smem_layout(int J, int NN) {
 #define TAKE(field, bytes) do { L.field = off; off += ((size_t)(bytes) + 15) & ~(size_t)15; } while (0)
   TAKE(slot, (size_t)J * 4);
   TAKE(summ, (size_t)J * 4);
-  TAKE(term_mark, (size_t)J * 4);              // marks during the repair, terms afterwards
+  TAKE(term, (size_t)J * 4);
+  TAKE(mark, (size_t)J * 4);
   TAKE(tot, (size_t)NN * 4);
   TAKE(el, (size_t)NN * 4);
   TAKE(cnt, (size_t)NN * 4);
   TAKE(viol, (size_t)NN);
   TAKE(occ, (size_t)NN * OCC * 4);
   // decided GPU counts of the listed occupants; the same bytes serve as the warps' row buffers
-  // before the column pass and after it
-  const size_t occnew = (size_t)NN * OCC * 2, rowbuf = (size_t)GEN_WARPS * NN * 2;
+  // (a row and its counterpart in the current allocation) before the column pass and after it
+  const size_t occnew = (size_t)NN * OCC * 2, rowbuf = (size_t)2 * GEN_WARPS * NN * 2;
   TAKE(occnew_row, occnew > rowbuf ? occnew : rowbuf);
   TAKE(mut, (size_t)J * 2);
   TAKE(ovf, (size_t)J * 2);
@@ -343,8 +373,8 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   const GenSmem L = gen_smem_layout(J, NN);
   uint32_t *s_slot = (uint32_t *)(smem + L.slot);
   uint32_t *s_summ = (uint32_t *)(smem + L.summ);
-  int *s_mark = (int *)(smem + L.term_mark);       // bit 0: changed by the column pass, bit 1: row is new
-  float *s_term = (float *)(smem + L.term_mark);
+  int *s_mark = (int *)(smem + L.mark);            // bit 0: changed by the column pass, bit 1: row is new
+  float *s_term = (float *)(smem + L.term);
   int *s_tot = (int *)(smem + L.tot), *s_el = (int *)(smem + L.el), *s_cnt = (int *)(smem + L.cnt);
   uint8_t *s_viol = (uint8_t *)(smem + L.viol);
   uint32_t *s_occ = (uint32_t *)(smem + L.occ);
@@ -363,25 +393,33 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   const uint32_t c = blockIdx.x;
   const bool elite = (int)c < a.num_elite;
 
-  for (int i = tid; i < NN; i += GEN_THREADS) {
-    s_tot[i] = 0; s_el[i] = 0; s_cnt[i] = 0; s_viol[i] = 0;
-    s_cap[i] = (int16_t)max((int)a.cap[i], 0);
-  }
-  for (int i = tid; i < J; i += GEN_THREADS) s_mark[i] = 0;
-  if (tid == 0) { s_nmut = 0; s_novf = 0; s_nmod = 0; s_ncow = 0; s_fail = 0; }
-
   // ---- parents: the candidate of rank c for an elite child, else the better-ranked of two
   // random pairs (rank = candidates ordered before, fitness descending, index ascending) ----
   if (elite) {
-    for (int i = tid; i < P; i += GEN_THREADS) {
-      const uint32_t ki = order_key(a.fitness_bits[i]);
-      int rk = 0;
-      for (int o = 0; o < P; ++o) {
-        const uint32_t ko = order_key(__ldg(a.fitness_bits + o));
-        rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
+    // The candidate of rank c: composite keys (fitness key, then lower index first) are unique,
+    // so c + 1 rounds of "largest key below the previous one" find it; one barrier per round.
+    __shared__ unsigned long long s_wmax[2][GEN_WARPS];
+    unsigned long long prev = ~0ull;
+    for (int t = 0; t <= (int)c; ++t) {
+      unsigned long long best = 0ull;
+      for (int i = tid; i < P; i += GEN_THREADS) {
+        const unsigned long long key = ((unsigned long long)order_key(__ldg(a.fitness_bits + i)) << 32) |
+                                       (unsigned long long)(0xFFFFFFFFu - (uint32_t)i);
+        if (key < prev && key > best) best = key;
       }
-      if (rk == (int)c) s_parent[0] = s_parent[1] = i;
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xffffffffu, best, off);
+        best = o > best ? o : best;
+      }
+      if (lane == 0) s_wmax[t & 1][warp] = best;
+      __syncthreads();
+      best = 0ull;
+#pragma unroll
+      for (int w = 0; w < GEN_WARPS; ++w) best = s_wmax[t & 1][w] > best ? s_wmax[t & 1][w] : best;
+      prev = best;
     }
+    if (tid == 0) s_parent[0] = s_parent[1] = (int)(0xFFFFFFFFu - (uint32_t)(prev & 0xFFFFFFFFull));
   } else {
     const u32x4 sel = draw(a.key, 0u, c, a.gen, SLOT_SELECT);
     const int idx[4] = {(int)bounded(sel.x, P), (int)bounded(sel.y, P), (int)bounded(sel.z, P), (int)bounded(sel.w, P)};
@@ -404,6 +442,14 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   }
   __syncthreads();
 
+  for (int i = tid; i < NN; i += GEN_THREADS) {
+    s_tot[i] = 0; s_el[i] = 0; s_cnt[i] = 0; s_viol[i] = 0;
+    s_cap[i] = (int16_t)max((int)a.cap[i], 0);
+  }
+  for (int i = tid; i < J; i += GEN_THREADS) s_mark[i] = 0;
+  if (tid == 0) { s_nmut = 0; s_novf = 0; s_nmod = 0; s_ncow = 0; s_fail = 0; }
+  __syncthreads();
+
   // occupant (job j holds g GPUs on node n) into the node's totals and list
   auto add_occupant = [&](int j, int n, int g, bool dist) {
     atomicAdd(&s_tot[n], g);
@@ -413,58 +459,92 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   };
 
   // ---- rows, one thread each: the child row is the chosen parent's row -----------------------
-  const uint32_t *pin_a = a.ptr_in + (size_t)s_parent[0] * J, *pin_b = a.ptr_in + (size_t)s_parent[1] * J;
-  for (int j = tid; j < J; j += GEN_THREADS) {
-    if (a.active && !a.active[j]) {
-      s_slot[j] = a.st.zero_slot;
-      s_summ[j] = 0u;
-      continue;
+  // First every row's draws (which parent; perturbed or not).  The count of perturbed rows is
+  // then known and the block takes its slots - those plus a reserve for the rows the column
+  // pass will change - with one atomic whose answer is not needed before the rows are done.
+  uint32_t secbits = 0, mutbits = 0;   // bit r: this thread's r-th row (j = tid + r * GEN_THREADS)
+  if (!elite) {
+    int r = 0;
+    for (int j = tid; j < J; j += GEN_THREADS, ++r) {
+      if (a.active && !a.active[j]) continue;
+      if (draw(a.key, (uint32_t)j, c, a.gen, SLOT_XOVER).x >> 31) secbits |= 1u << r;
+      if (draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE).x < a.thr) {
+        mutbits |= 1u << r;
+        s_mut[atomicAdd(&s_nmut, 1)] = (uint16_t)j;
+      }
     }
-    bool second = false, mut = false;
-    if (!elite) {
-      second = (draw(a.key, (uint32_t)j, c, a.gen, SLOT_XOVER).x >> 31) != 0u;
-      mut = draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE).x < a.thr;
-    }
-    const uint32_t slot = second ? pin_b[j] : pin_a[j];
-    s_slot[j] = slot;
-    const uint32_t w = a.st.summ[slot];
-    s_summ[j] = w;
-    if (mut) {
-      s_mut[atomicAdd(&s_nmut, 1)] = (uint16_t)j;
-      continue;
-    }
-    const uint4 r0 = *(const uint4 *)(a.st.rec + (size_t)slot * REC_WORDS);
-    if (r0.x == REC_OVERFLOW) {
-      s_ovf[atomicAdd(&s_novf, 1)] = (uint16_t)j;
-      continue;
-    }
-    if (r0.x == 0u) continue;
-    const bool dist = ((w >> 11) & 0x7FFu) >= 2u;
-    const uint4 r1 = *(const uint4 *)(a.st.rec + (size_t)slot * REC_WORDS + 4);
-    const uint32_t e[REC_WORDS] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
-#pragma unroll
-    for (int k = 0; k < REC_WORDS; ++k)
-      if (e[k]) add_occupant(j, (int)(e[k] & 0xFFFu), (int)((e[k] >> 12) & 0x7FFu), dist);
   }
   __syncthreads();
-  if (tid == 0 && s_nmut > 0) {
-    const unsigned int base = atomicAdd(a.state, (unsigned int)s_nmut);
+  unsigned int base_reg = 0;
+  if (tid == 0) base_reg = atomicAdd(a.state, (unsigned int)(s_nmut + COW_RESERVE));
+
+  // Then RB rows per thread at a time, so that their dependent loads (index -> record) travel
+  // together.
+  const uint32_t *pin_a = a.ptr_in + (size_t)s_parent[0] * J, *pin_b = a.ptr_in + (size_t)s_parent[1] * J;
+  constexpr int RB = 4;
+  for (int jb = tid, rb = 0; jb < J; jb += GEN_THREADS * RB, rb += RB) {
+    uint32_t slot[RB];
+    bool on[RB], mut[RB];
+#pragma unroll
+    for (int r = 0; r < RB; ++r) {
+      const int j = jb + r * GEN_THREADS;
+      on[r] = j < J && (!a.active || a.active[j]);
+      mut[r] = ((mutbits >> (rb + r)) & 1u) != 0u;
+      slot[r] = on[r] ? (((secbits >> (rb + r)) & 1u) ? pin_b[j] : pin_a[j]) : a.st.zero_slot;
+    }
+    uint32_t rec[RB][REC_WORDS];
+#pragma unroll
+    for (int r = 0; r < RB; ++r) load_record(rec[r], a.st.rec + (size_t)slot[r] * REC_WORDS);
+#pragma unroll
+    for (int r = 0; r < RB; ++r) {
+      const int j = jb + r * GEN_THREADS;
+      if (j >= J) continue;
+      const uint32_t w = on[r] ? rec[r][REC_SUMM] : 0u;
+      s_slot[j] = slot[r];
+      s_summ[j] = w;
+      if (!on[r] || mut[r]) continue;
+      s_term[j] = __uint_as_float(rec[r][REC_TERM]);
+      if (rec[r][0] == REC_OVERFLOW) {
+        s_ovf[atomicAdd(&s_novf, 1)] = (uint16_t)j;
+        continue;
+      }
+      const bool dist = ((w >> 11) & 0x7FFu) >= 2u;
+#pragma unroll
+      for (int k = 0; k < REC_ENTRIES; ++k) {
+        const uint32_t e = rec[r][k];
+        if (e) add_occupant(j, (int)(e & 0xFFFu), (int)((e >> 12) & 0x7FFu), dist);
+      }
+    }
+  }
+  if (tid == 0) {
     const unsigned long long limit = (unsigned long long)(a.state[1] + 1u) * a.st.half_cap;
-    s_base_mut = base;
-    if ((unsigned long long)base + (unsigned long long)s_nmut > limit) { s_fail = 1; atomicExch(a.status, SCHED_ERR_TOO_LARGE); }
+    s_base_mut = base_reg;
+    s_base_cow = base_reg + (unsigned int)s_nmut;
+    if ((unsigned long long)base_reg + (unsigned long long)(s_nmut + COW_RESERVE) > limit) {
+      s_fail = 1;
+      atomicExch(a.status, SCHED_ERR_TOO_LARGE);
+    }
   }
   __syncthreads();
 
   // ---- perturbed rows, one warp each: new row in a fresh slot ---------------------------------
-  int16_t *row = s_rowbuf + (size_t)warp * NN;
+  int16_t *row = s_rowbuf + (size_t)warp * NN;                  // this warp's row
+  int16_t *crow = s_rowbuf + (size_t)(GEN_WARPS + warp) * NN;   // and its counterpart in the current allocation
   uint32_t *recw = s_rec + warp * REC_WORDS;
   const int row_vecs = NN >> 3;
   if (!s_fail) {
+    // the warp's rows and their counterparts in the current allocation are asked for up front
+    for (int i = warp; i < s_nmut; i += GEN_WARPS) {
+      const int j = (int)s_mut[i];
+      if (lane * 64 < NN) prefetch_l2(a.st.pool + (size_t)s_slot[j] * NN + lane * 64);
+      if (a.cur && lane * 64 < NN) prefetch_l2(a.cur + (size_t)j * NN + lane * 64);
+    }
     for (int i = warp; i < s_nmut; i += GEN_WARPS) {
       const int j = (int)s_mut[i];
       const uint32_t old = s_slot[j], w = s_summ[j];
-      const uint4 *s4 = (const uint4 *)(a.st.pool + (size_t)old * NN);
-      for (int v = lane; v < row_vecs; v += 32) ((uint4 *)row)[v] = s4[v];
+      load_row<false>(row, a.st.pool + (size_t)old * NN, NN, lane);
+      if (a.cur) load_row<false>(crow, a.cur + (size_t)j * NN, NN, lane);
+      const int kc_in = a.k_cap ? a.k_cap[j] : a.k_max;
       __syncwarp();
       int rK = (int)(w & 0x7FFu), rN = (int)((w >> 11) & 0x7FFu);
       const u32x4 mw = draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE);
@@ -491,8 +571,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       rN = warp_sum(rN);
       // per-row caps: replicas above the job's cap leave from the highest node index down, then
       // occupied nodes beyond n_max are cleared from the highest index down
-      int kc = a.k_cap ? a.k_cap[j] : a.k_max;
-      kc = max(0, min(kc, a.k_max));
+      const int kc = max(0, min(kc_in, a.k_max));
       if (rK > kc || rN > a.n_max) {
         if (lane == 0) {
           int excess = rK - kc;
@@ -512,18 +591,20 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         __syncwarp();
       }
       int K, N, nd;
-      summarise_row(row, NN, a.cur ? a.cur + (size_t)j * NN : nullptr, lane, K, N, nd, recw);
+      summarise_row(row, NN, a.cur ? crow : nullptr, lane, K, N, nd, recw);
       const uint32_t slot = s_base_mut + (uint32_t)i;
       uint4 *d4 = (uint4 *)(a.st.pool + (size_t)slot * NN);
       for (int v = lane; v < row_vecs; v += 32) d4[v] = ((const uint4 *)row)[v];
-      if (lane < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + lane] = recw[lane];
       const uint32_t word = pack_summary(K, N, nd);
       if (lane == 0) {
-        a.st.summ[slot] = word;
+        recw[REC_SUMM] = word;
+        recw[REC_TERM] = 0u;   // filled in with the other new rows' terms at the end
         s_slot[j] = slot;
         s_summ[j] = word;
         s_mark[j] = 2;
       }
+      __syncwarp();
+      if (lane < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + lane] = recw[lane];
       const bool dist = N >= 2;
       for (int n = lane; n < NN; n += 32)
         if (row[n] > 0) add_occupant(j, n, (int)row[n], dist);
@@ -579,10 +660,15 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   const int nmod = s_nmod;
   for (int i = tid; i < nmod; i += GEN_THREADS) {
     const int j = (int)s_mod[i];
-    s_ovf[i] = (s_mark[j] & 2) ? (uint16_t)0xFFFFu : (uint16_t)atomicAdd(&s_ncow, 1);
+    const bool own = (s_mark[j] & 2) != 0;
+    s_ovf[i] = own ? (uint16_t)0xFFFFu : (uint16_t)atomicAdd(&s_ncow, 1);
+    if (!own)
+      for (int b = 0; b * 64 < NN; ++b) prefetch_l2(a.st.pool + (size_t)s_slot[j] * NN + b * 64);
+    if (a.cur)
+      for (int b = 0; b * 64 < NN; ++b) prefetch_l2(a.cur + (size_t)j * NN + b * 64);
   }
   __syncthreads();
-  if (tid == 0 && s_ncow > 0) {
+  if (tid == 0 && s_ncow > COW_RESERVE) {   // more than the reserve: a run of slots of their own
     const unsigned int base = atomicAdd(a.state, (unsigned int)s_ncow);
     const unsigned long long limit = (unsigned long long)(a.state[1] + 1u) * a.st.half_cap;
     s_base_cow = base;
@@ -626,30 +712,35 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
     for (int i = warp; i < nmod; i += GEN_WARPS) {
       const int j = (int)s_mod[i];
       const uint32_t slot = s_slot[j];
-      const volatile int16_t *src = a.st.pool + (size_t)slot * NN;   // written in this kernel: no read-only path
-      for (int n = lane; n < NN; n += 32) row[n] = src[n];
+      load_row<true>(row, a.st.pool + (size_t)slot * NN, NN, lane);   // written in this kernel: read through to L2
+      if (a.cur) load_row<false>(crow, a.cur + (size_t)j * NN, NN, lane);
       __syncwarp();
       int K, N, nd;
-      summarise_row(row, NN, a.cur ? a.cur + (size_t)j * NN : nullptr, lane, K, N, nd, recw);
-      if (lane < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + lane] = recw[lane];
+      summarise_row(row, NN, a.cur ? crow : nullptr, lane, K, N, nd, recw);
       const uint32_t word = pack_summary(K, N, nd);
       if (lane == 0) {
-        a.st.summ[slot] = word;
+        recw[REC_SUMM] = word;
+        recw[REC_TERM] = 0u;
         s_summ[j] = word;
       }
+      __syncwarp();
+      if (lane < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + lane] = recw[lane];
       __syncwarp();
     }
   }
   __syncthreads();
 
-  // ---- children's indices out, fitness of the candidate (Eq. 14) ------------------------------
+  // ---- children's indices out, fitness of the candidate (Eq. 14) from the rows' terms ----------
   uint32_t *pout = a.ptr_out + (size_t)c * J;
-  for (int j = tid; j < J; j += GEN_THREADS) {
-    pout[j] = s_slot[j];
-    if (!a.tp.active || a.tp.active[j]) {
-      const uint32_t w = s_summ[j];
-      s_term[j] = fitness_term(a.tp, j, (int)(w & 0x7FFu), (int)((w >> 11) & 0x7FFu), (w >> 22) != 0u);
-    }
+  for (int j = tid; j < J; j += GEN_THREADS) pout[j] = s_slot[j];
+  // terms of the rows that are new in this generation (the others got theirs with their record)
+  const int nmut = s_nmut;
+  for (int i = tid; i < nmut + nmod; i += GEN_THREADS) {
+    const int j = (int)(i < nmut ? s_mut[i] : s_mod[i - nmut]);
+    const uint32_t w = s_summ[j];
+    const float term = fitness_term(a.tp, j, (int)(w & 0x7FFu), (int)((w >> 11) & 0x7FFu), (w >> 22) != 0u);
+    s_term[j] = term;
+    if (!s_fail) a.st.rec[(size_t)s_slot[j] * REC_WORDS + REC_TERM] = __float_as_uint(term);
   }
   __syncthreads();
   // sums in the order of the dense fitness kernel: per chunk of rows, thread t adds rows t,
@@ -684,7 +775,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
 
 StoreView store_view(const sched_ctx *ctx) {
   StoreView v;
-  v.pool = ctx->rs_pool; v.rec = ctx->rs_rec; v.summ = ctx->rs_summ;
+  v.pool = ctx->rs_pool; v.rec = ctx->rs_rec;
   v.half_cap = ctx->rs_half_cap;
   v.zero_slot = (uint32_t)(2 * ctx->rs_half_cap);
   return v;
@@ -701,29 +792,32 @@ bool rowstore_eligible(const sched_ctx *ctx, const int16_t *) {
   if (c.num_nodes % 8 != 0 || c.num_nodes > 512 || ctx->cap_max > 2047) return false;
   if (c.k_max > 2047 || c.n_max > 2047) return false;
   const unsigned long long rows = (unsigned long long)c.population * c.num_jobs;
-  if (12ull * rows >= (1ull << 32)) return false;   // slot indices are 32-bit
+  const unsigned long long worst = store_worst_case(c.population, c.num_jobs);
+  if (2ull * rows + 11ull * worst >= (1ull << 32)) return false;   // slot indices are 32-bit
   if (gen_smem_layout(c.num_jobs, c.num_nodes).total > 200 * 1024) return false;
-  // at least three populations' worth of slots per half; beyond 8 GiB of pool the dense path runs
-  const unsigned long long row_bytes = (unsigned long long)c.num_nodes * 2 + REC_WORDS * 4 + 4;
-  return 6ull * rows * row_bytes <= (8ull << 30);
+  // a half holds the population plus at least two generations' worst case; beyond 8 GiB of pool
+  // the dense path runs
+  const unsigned long long row_bytes = (unsigned long long)c.num_nodes * 2 + REC_WORDS * 4;
+  return 2ull * (rows + 2ull * worst) * row_bytes <= (8ull << 30);
 }
 
 int rowstore_ensure(sched_ctx *ctx) {
   if (ctx->rs_ready) return SCHED_OK;
   const sched_config &c = ctx->cfg;
   const unsigned long long rows = (unsigned long long)c.population * c.num_jobs;
-  const unsigned long long row_bytes = (unsigned long long)c.num_nodes * 2 + REC_WORDS * 4 + 4;
-  // half = (1 + gens between checks + slack) populations; shrink until the pool fits 8 GiB
+  const unsigned long long row_bytes = (unsigned long long)c.num_nodes * 2 + REC_WORDS * 4;
+  // half = the population + (gens between checks + slack) generations' worst case; shrink until
+  // the pool fits 8 GiB
   int check = 2, slack = 2;
-  while (2ull * (1 + check + slack) * rows * row_bytes > (8ull << 30) && (check > 1 || slack > 1)) {
+  const unsigned long long worst = store_worst_case(c.population, c.num_jobs);
+  while (2ull * (rows + (check + slack) * worst) * row_bytes > (8ull << 30) && (check > 1 || slack > 1)) {
     if (slack > 1) --slack; else --check;
   }
   ctx->rs_check_every = check;
-  ctx->rs_half_cap = (size_t)((1 + check + slack) * rows);
+  ctx->rs_half_cap = (size_t)(rows + (check + slack) * worst);
   const size_t slots = 2 * ctx->rs_half_cap + 1;
   cudaError_t e = cudaMalloc((void **)&ctx->rs_pool, slots * c.num_nodes * sizeof(int16_t));
   if (e == cudaSuccess) e = cudaMalloc((void **)&ctx->rs_rec, slots * REC_WORDS * sizeof(uint32_t));
-  if (e == cudaSuccess) e = cudaMalloc((void **)&ctx->rs_summ, slots * sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaMalloc((void **)&ctx->rs_ptr, 2 * (size_t)rows * sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaMalloc((void **)&ctx->rs_state, 4 * sizeof(unsigned int));
   if (e == cudaSuccess) {
@@ -733,9 +827,9 @@ int rowstore_ensure(sched_ctx *ctx) {
   }
   if (e != cudaSuccess) {
     set_error(ctx, "row store allocation failed: %s", cudaGetErrorString(e));
-    for (void *p : {(void *)ctx->rs_pool, (void *)ctx->rs_rec, (void *)ctx->rs_summ, (void *)ctx->rs_ptr, (void *)ctx->rs_state})
+    for (void *p : {(void *)ctx->rs_pool, (void *)ctx->rs_rec, (void *)ctx->rs_ptr, (void *)ctx->rs_state})
       if (p) cudaFree(p);
-    ctx->rs_pool = nullptr; ctx->rs_rec = nullptr; ctx->rs_summ = nullptr; ctx->rs_ptr = nullptr; ctx->rs_state = nullptr;
+    ctx->rs_pool = nullptr; ctx->rs_rec = nullptr; ctx->rs_ptr = nullptr; ctx->rs_state = nullptr;
     cudaGetLastError();
     return SCHED_ERR_CUDA;
   }
@@ -744,13 +838,16 @@ int rowstore_ensure(sched_ctx *ctx) {
   return SCHED_OK;
 }
 
-int rowstore_build(sched_ctx *ctx, const uint8_t *d_active, const int16_t *d_cur) {
+int rowstore_build(sched_ctx *ctx, const uint8_t *d_active, const int16_t *d_cur, const float *d_pen) {
   const sched_config &c = ctx->cfg;
   BuildArgs a;
   a.st = store_view(ctx);
   a.ptr = ctx->rs_ptr;
   a.state = ctx->rs_state;
   a.active = d_active; a.cur = d_cur;
+  a.tp.table = ctx->d_tab_speedup; a.tp.pen = d_pen; a.tp.active = d_active;
+  a.tp.k_max = c.k_max; a.tp.n_max = c.n_max; a.tp.mode = fitness_mode(c.p); a.tp.p = c.p;
+  a.tp.floor_ = c.speedup_floor;
   a.P = c.population; a.J = c.num_jobs; a.NN = c.num_nodes;
   {
     TimedLaunch tl_(ctx, KK_STORE_BUILD);

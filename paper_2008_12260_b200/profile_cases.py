@@ -2,7 +2,8 @@
 
     python -m paper_2008_12260_b200.profile_cases fitness_stress   # 16 stress candidates (537 MB)
     python -m paper_2008_12260_b200.profile_cases table_large      # 1024-job speedup table
-    python -m paper_2008_12260_b200.profile_cases round_large      # large round, 2 generations
+    python -m paper_2008_12260_b200.profile_cases round_large [G]  # large round, G generations (default 2)
+    python -m paper_2008_12260_b200.profile_cases generation_large # dense ga_generation, large shape
 
 Each case holds well under a few GB on the device, launches its kernel a handful of
 times and exits; inputs are larger than L2 wherever DRAM traffic is the point.
@@ -25,7 +26,7 @@ def _large(api, synth, torch):
     return cfg, cl, jobs, s, api.DeviceJobs(jobs, "cuda", torch)
 
 
-def main(case: str, reps: int = 3):
+def main(case: str, reps: int = 3, generations: int = 2):
     import torch
     from . import api, synth
 
@@ -54,13 +55,26 @@ def main(case: str, reps: int = 3):
         cur = torch.from_numpy(cfg.cur()).cuda()
         best = torch.empty((cfg.num_jobs, cfg.num_nodes), dtype=torch.int16, device="cuda")
         bf = torch.zeros(1, dtype=torch.float32, device="cuda")
-        s.schedule_round(dj, cur, best, bf, round=0, generations=2)
+        s.schedule_round(dj, cur, best, bf, round=0, generations=generations)
         s.sync_status()
         print("round_large", float(bf.item()))
+    elif case == "generation_large":
+        cfg, cl, jobs, s, dj = _large(api, synth, torch)
+        shape = (cfg.population, cfg.num_jobs, cfg.num_nodes)
+        a = torch.empty(shape, dtype=torch.int16, device="cuda")
+        b = torch.empty_like(a)
+        fit = torch.rand(cfg.population, dtype=torch.float32, device="cuda")
+        s.init_population(dj, torch.from_numpy(cfg.cur()).cuda(), a, round=0)
+        for g in range(reps):
+            s.ga_generation(dj, a, fit, b, round=0, generation=g)
+            a, b = b, a
+        s.sync_status()
+        print("generation_large", int(a.sum().item()))
     else:
         raise SystemExit("unknown case %r" % case)
     s.close()
 
 
 if __name__ == "__main__":
-    main(sys.argv[1] if len(sys.argv) > 1 else "fitness_stress")
+    main(sys.argv[1] if len(sys.argv) > 1 else "fitness_stress",
+         generations=int(sys.argv[2]) if len(sys.argv) > 2 else 2)
