@@ -267,7 +267,7 @@ __device__ __forceinline__ int decide_entries(const GenArgs &a, uint32_t c, int 
 
 // Shared-memory carve-up of the generation kernel (sizes in bytes, 16-byte aligned pieces).
 struct GenSmem {
-  size_t slot, summ, term, mark, tot, el, cnt, viol, occ, occnew_row, mut, ovf, mod, cap, rec, total;
+  size_t slot, summ, term, mark, acc, viol, occ, rowbuf, mut, ovf, mod, cap, rec, total;
 };
 
 __host__ __device__ inline GenSmem gen_smem_layout(int J, int NN) {
@@ -278,15 +278,11 @@ __host__ __device__ inline GenSmem gen_smem_layout(int J, int NN) {
   TAKE(summ, (size_t)J * 4);
   TAKE(term, (size_t)J * 4);
   TAKE(mark, (size_t)J * 4);
-  TAKE(tot, (size_t)NN * 4);
-  TAKE(el, (size_t)NN * 4);
-  TAKE(cnt, (size_t)NN * 4);
+  TAKE(acc, (size_t)NN * 8);
   TAKE(viol, (size_t)NN);
   TAKE(occ, (size_t)NN * OCC * 4);
-  // decided GPU counts of the listed occupants; the same bytes serve as the warps' row buffers
-  // (a row and its counterpart in the current allocation) before the column pass and after it
-  const size_t occnew = (size_t)NN * OCC * 2, rowbuf = (size_t)2 * GEN_WARPS * NN * 2;
-  TAKE(occnew_row, occnew > rowbuf ? occnew : rowbuf);
+  // per warp: a row and its counterpart in the current allocation
+  TAKE(rowbuf, (size_t)2 * GEN_WARPS * NN * 2);
   TAKE(mut, (size_t)J * 2);
   TAKE(ovf, (size_t)J * 2);
   TAKE(mod, (size_t)J * 2);
@@ -375,15 +371,15 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   uint32_t *s_summ = (uint32_t *)(smem + L.summ);
   int *s_mark = (int *)(smem + L.mark);            // bit 0: changed by the column pass, bit 1: row is new
   float *s_term = (float *)(smem + L.term);
-  int *s_tot = (int *)(smem + L.tot), *s_el = (int *)(smem + L.el), *s_cnt = (int *)(smem + L.cnt);
+  // per node: GPUs placed (bits 0..31), distributed jobs on it (32..47), occupants (48..63)
+  unsigned long long *s_node = (unsigned long long *)(smem + L.acc);
   uint8_t *s_viol = (uint8_t *)(smem + L.viol);
   uint32_t *s_occ = (uint32_t *)(smem + L.occ);
-  uint16_t *s_occnew = (uint16_t *)(smem + L.occnew_row);
-  int16_t *s_rowbuf = (int16_t *)(smem + L.occnew_row);
+  int16_t *s_rowbuf = (int16_t *)(smem + L.rowbuf);
   uint16_t *s_mut = (uint16_t *)(smem + L.mut), *s_ovf = (uint16_t *)(smem + L.ovf), *s_mod = (uint16_t *)(smem + L.mod);
   int16_t *s_cap = (int16_t *)(smem + L.cap);
   uint32_t *s_rec = (uint32_t *)(smem + L.rec);
-  __shared__ int s_nmut, s_novf, s_nmod, s_ncow, s_fail;
+  __shared__ int s_nmut, s_novf, s_nmod, s_ncow, s_fail, s_anyscan;
   __shared__ unsigned int s_base_mut, s_base_cow;
   __shared__ int s_parent[2], s_rank4[4];
   __shared__ double s_acc[GEN_WARPS];
@@ -443,18 +439,18 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   __syncthreads();
 
   for (int i = tid; i < NN; i += GEN_THREADS) {
-    s_tot[i] = 0; s_el[i] = 0; s_cnt[i] = 0; s_viol[i] = 0;
+    s_node[i] = 0ull; s_viol[i] = 0;
     s_cap[i] = (int16_t)max((int)a.cap[i], 0);
   }
   for (int i = tid; i < J; i += GEN_THREADS) s_mark[i] = 0;
-  if (tid == 0) { s_nmut = 0; s_novf = 0; s_nmod = 0; s_ncow = 0; s_fail = 0; }
+  if (tid == 0) { s_nmut = 0; s_novf = 0; s_nmod = 0; s_ncow = 0; s_fail = 0; s_anyscan = 0; }
   __syncthreads();
 
   // occupant (job j holds g GPUs on node n) into the node's totals and list
   auto add_occupant = [&](int j, int n, int g, bool dist) {
-    atomicAdd(&s_tot[n], g);
-    if (dist) atomicAdd(&s_el[n], 1);
-    const int k = atomicAdd(&s_cnt[n], 1);
+    const unsigned long long old =
+        atomicAdd(&s_node[n], (unsigned long long)(unsigned)g | (dist ? (1ull << 32) : 0ull) | (1ull << 48));
+    const int k = (int)(old >> 48);
     if (k < OCC) s_occ[n * OCC + k] = (uint32_t)j | ((uint32_t)g << 13) | (dist ? 0x80000000u : 0u);
   };
 
@@ -625,11 +621,18 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
 
   // ---- column pass, decisions: which occupants of the violating nodes change ------------------
   auto mark_row = [&](int j) {
-    if ((atomicOr(&s_mark[j], 1) & 1) == 0) s_mod[atomicAdd(&s_nmod, 1)] = (uint16_t)j;
+    if ((atomicOr(&s_mark[j], 1) & 1) == 0) {
+      s_mod[atomicAdd(&s_nmod, 1)] = (uint16_t)j;
+      for (int b = 0; b * 64 < NN; ++b) {   // the row and its counterpart will be read next
+        prefetch_l2(a.st.pool + (size_t)s_slot[j] * NN + b * 64);
+        if (a.cur) prefetch_l2(a.cur + (size_t)j * NN + b * 64);
+      }
+    }
   };
   for (int nb = warp * 32; nb < NN; nb += GEN_WARPS * 32) {
     const int n = nb + lane;
-    const int total = (n < NN) ? s_tot[n] : 0, nelig = (n < NN) ? s_el[n] : 0;
+    const unsigned long long acc = (n < NN) ? s_node[n] : 0ull;
+    const int total = (int)(uint32_t)acc, nelig = (int)((acc >> 32) & 0xFFFFu), count = (int)(acc >> 48);
     const int cp = (n < NN) ? (int)s_cap[n] : 0;
     unsigned todo = __ballot_sync(0xffffffffu, n < NN && (nelig >= 2 || total > cp));
     while (todo) {
@@ -638,16 +641,18 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       const int nn = nb + srcl;
       const int tot_n = __shfl_sync(0xffffffffu, total, srcl), ne_n = __shfl_sync(0xffffffffu, nelig, srcl);
       const int cap_n = __shfl_sync(0xffffffffu, cp, srcl);
-      const int have_n = s_cnt[nn];
+      const int have_n = __shfl_sync(0xffffffffu, count, srcl);
       if (have_n > OCC) {
-        if (lane == 0) s_viol[nn] = 2;
+        if (lane == 0) { s_viol[nn] = 2; s_anyscan = 1; }
         repair_column_scan<false>(a, c, s_slot, s_summ, nn, tot_n, ne_n, cap_n, lane, mark_row);
       } else {
         const uint32_t entry = (lane < have_n) ? s_occ[nn * OCC + lane] : 0u;
         const int v_new = decide_entries(a, c, nn, tot_n, ne_n, cap_n, lane, entry, have_n);
         if (lane < have_n) {
-          s_occnew[nn * OCC + lane] = (uint16_t)v_new;
-          if (v_new != (int)((entry >> 13) & 0x7FFu)) mark_row((int)(entry & 0x1FFFu));
+          // the entry now carries the decision: GPUs kept, and bit 24 when that is a change
+          const bool changed = v_new != (int)((entry >> 13) & 0x7FFu);
+          s_occ[nn * OCC + lane] = (entry & 0x80001FFFu) | ((uint32_t)v_new << 13) | (changed ? (1u << 24) : 0u);
+          if (changed) mark_row((int)(entry & 0x1FFFu));
         }
         if (lane == 0) s_viol[nn] = 1;
       }
@@ -656,79 +661,130 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   }
   __syncthreads();
 
-  // ---- rows the column pass changes get a slot of their own unless they are new already -------
+  // ---- rows the column pass changes -----------------------------------------------------------
+  // Usual case (every violating node's occupants were listed): one warp per changed row takes
+  // the row, applies the decisions of its nodes, and writes it with its record - to a slot of
+  // its own unless the row is new in this generation already.
   const int nmod = s_nmod;
-  for (int i = tid; i < nmod; i += GEN_THREADS) {
-    const int j = (int)s_mod[i];
-    const bool own = (s_mark[j] & 2) != 0;
-    s_ovf[i] = own ? (uint16_t)0xFFFFu : (uint16_t)atomicAdd(&s_ncow, 1);
-    if (!own)
-      for (int b = 0; b * 64 < NN; ++b) prefetch_l2(a.st.pool + (size_t)s_slot[j] * NN + b * 64);
-    if (a.cur)
-      for (int b = 0; b * 64 < NN; ++b) prefetch_l2(a.cur + (size_t)j * NN + b * 64);
-  }
-  __syncthreads();
-  if (tid == 0 && s_ncow > COW_RESERVE) {   // more than the reserve: a run of slots of their own
-    const unsigned int base = atomicAdd(a.state, (unsigned int)s_ncow);
-    const unsigned long long limit = (unsigned long long)(a.state[1] + 1u) * a.st.half_cap;
-    s_base_cow = base;
-    if ((unsigned long long)base + (unsigned long long)s_ncow > limit) { s_fail = 1; atomicExch(a.status, SCHED_ERR_TOO_LARGE); }
-  }
-  __syncthreads();
-  if (!s_fail) {
-    for (int i = warp; i < nmod; i += GEN_WARPS) {
-      const uint32_t k = s_ovf[i];
-      if (k == 0xFFFFu) continue;
-      const int j = (int)s_mod[i];
-      const uint32_t slot = s_base_cow + k;
-      const uint4 *s4 = (const uint4 *)(a.st.pool + (size_t)s_slot[j] * NN);
-      uint4 *d4 = (uint4 *)(a.st.pool + (size_t)slot * NN);
-      for (int v = lane; v < row_vecs; v += 32) d4[v] = s4[v];
-      __syncwarp();
-      if (lane == 0) s_slot[j] = slot;
-    }
-  }
-  __syncthreads();
-
-  // ---- column pass, writes --------------------------------------------------------------------
-  if (!s_fail && nmod > 0) {
-    for (int i = tid; i < NN * OCC; i += GEN_THREADS) {
-      const int n = i / OCC, k = i - n * OCC;
-      if (s_viol[n] != 1 || k >= s_cnt[n]) continue;
-      const uint32_t entry = s_occ[i];
-      const int v_new = (int)s_occnew[i];
-      if (v_new != (int)((entry >> 13) & 0x7FFu))
-        a.st.pool[(size_t)s_slot[entry & 0x1FFFu] * NN + n] = (int16_t)v_new;
-    }
-    for (int nn = warp; nn < NN; nn += GEN_WARPS) {
-      if (s_viol[nn] != 2) continue;
-      repair_column_scan<true>(a, c, s_slot, s_summ, nn, s_tot[nn], s_el[nn], (int)s_cap[nn], lane, [](int) {});
-    }
-  }
-  __syncthreads();
-
-  // ---- changed rows: summary and record from the row as it now stands -------------------------
-  if (!s_fail) {
-    for (int i = warp; i < nmod; i += GEN_WARPS) {
-      const int j = (int)s_mod[i];
-      const uint32_t slot = s_slot[j];
-      load_row<true>(row, a.st.pool + (size_t)slot * NN, NN, lane);   // written in this kernel: read through to L2
-      if (a.cur) load_row<false>(crow, a.cur + (size_t)j * NN, NN, lane);
-      __syncwarp();
-      int K, N, nd;
-      summarise_row(row, NN, a.cur ? crow : nullptr, lane, K, N, nd, recw);
-      const uint32_t word = pack_summary(K, N, nd);
-      if (lane == 0) {
-        recw[REC_SUMM] = word;
-        recw[REC_TERM] = 0u;
-        s_summ[j] = word;
+  if (!s_anyscan) {
+    if (nmod > COW_RESERVE) {   // more than the reserve: a run of slots of their own
+      if (tid == 0) {
+        const unsigned int base = atomicAdd(a.state, (unsigned int)nmod);
+        const unsigned long long limit = (unsigned long long)(a.state[1] + 1u) * a.st.half_cap;
+        s_base_cow = base;
+        if ((unsigned long long)base + (unsigned long long)nmod > limit) { s_fail = 1; atomicExch(a.status, SCHED_ERR_TOO_LARGE); }
       }
-      __syncwarp();
-      if (lane < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + lane] = recw[lane];
-      __syncwarp();
+      __syncthreads();
     }
+    if (!s_fail) {
+      for (int i = warp; i < nmod; i += GEN_WARPS) {
+        const int j = (int)s_mod[i];
+        const bool own = (s_mark[j] & 2) != 0;
+        const uint32_t src = s_slot[j];
+        load_row<true>(row, a.st.pool + (size_t)src * NN, NN, lane);   // may have been written in this kernel
+        if (a.cur) load_row<false>(crow, a.cur + (size_t)j * NN, NN, lane);
+        __syncwarp();
+        for (int n = lane; n < NN; n += 32) {
+          if (row[n] > 0 && s_viol[n] == 1) {
+            const int cnt = (int)(s_node[n] >> 48);
+            for (int k = 0; k < cnt; ++k) {
+              if ((int)(s_occ[n * OCC + k] & 0x1FFFu) == j) {
+                row[n] = (int16_t)((s_occ[n * OCC + k] >> 13) & 0x7FFu);
+                break;
+              }
+            }
+          }
+        }
+        __syncwarp();
+        int K, N, nd;
+        summarise_row(row, NN, a.cur ? crow : nullptr, lane, K, N, nd, recw);
+        const uint32_t dst = own ? src : s_base_cow + (uint32_t)i;
+        uint4 *d4 = (uint4 *)(a.st.pool + (size_t)dst * NN);
+        for (int v = lane; v < row_vecs; v += 32) d4[v] = ((const uint4 *)row)[v];
+        const uint32_t word = pack_summary(K, N, nd);
+        if (lane == 0) {
+          recw[REC_SUMM] = word;
+          recw[REC_TERM] = 0u;
+          s_slot[j] = dst;
+          s_summ[j] = word;
+        }
+        __syncwarp();
+        if (lane < REC_WORDS) a.st.rec[(size_t)dst * REC_WORDS + lane] = recw[lane];
+        __syncwarp();
+      }
+    }
+    __syncthreads();
+  } else {
+    // Some node had more occupants than the block lists: its column is scanned through the
+    // row indices, so the rows are first copied, then written in place, then summarised.
+      for (int i = tid; i < nmod; i += GEN_THREADS) {
+      const int j = (int)s_mod[i];
+      const bool own = (s_mark[j] & 2) != 0;
+      s_ovf[i] = own ? (uint16_t)0xFFFFu : (uint16_t)atomicAdd(&s_ncow, 1);
+    }
+    __syncthreads();
+    if (tid == 0 && s_ncow > COW_RESERVE) {   // more than the reserve: a run of slots of their own
+      const unsigned int base = atomicAdd(a.state, (unsigned int)s_ncow);
+      const unsigned long long limit = (unsigned long long)(a.state[1] + 1u) * a.st.half_cap;
+      s_base_cow = base;
+      if ((unsigned long long)base + (unsigned long long)s_ncow > limit) { s_fail = 1; atomicExch(a.status, SCHED_ERR_TOO_LARGE); }
+    }
+    __syncthreads();
+    if (!s_fail) {
+      for (int i = warp; i < nmod; i += GEN_WARPS) {
+        const uint32_t k = s_ovf[i];
+        if (k == 0xFFFFu) continue;
+        const int j = (int)s_mod[i];
+        const uint32_t slot = s_base_cow + k;
+        const uint4 *s4 = (const uint4 *)(a.st.pool + (size_t)s_slot[j] * NN);
+        uint4 *d4 = (uint4 *)(a.st.pool + (size_t)slot * NN);
+        for (int v = lane; v < row_vecs; v += 32) d4[v] = s4[v];
+        __syncwarp();
+        if (lane == 0) s_slot[j] = slot;
+      }
+    }
+    __syncthreads();
+
+    // column pass, writes
+    if (!s_fail && nmod > 0) {
+      for (int i = tid; i < NN * OCC; i += GEN_THREADS) {
+        const int n = i / OCC, k = i - n * OCC;
+        if (s_viol[n] != 1 || k >= (int)(s_node[n] >> 48)) continue;
+        const uint32_t entry = s_occ[i];
+        if ((entry >> 24) & 1u)
+          a.st.pool[(size_t)s_slot[entry & 0x1FFFu] * NN + n] = (int16_t)((entry >> 13) & 0x7FFu);
+      }
+      for (int nn = warp; nn < NN; nn += GEN_WARPS) {
+        if (s_viol[nn] != 2) continue;
+        repair_column_scan<true>(a, c, s_slot, s_summ, nn, (int)(uint32_t)s_node[nn], (int)((s_node[nn] >> 32) & 0xFFFFu),
+                                 (int)s_cap[nn], lane, [](int) {});
+      }
+    }
+    __syncthreads();
+
+    // changed rows: summary and record from the row as it now stands
+    if (!s_fail) {
+      for (int i = warp; i < nmod; i += GEN_WARPS) {
+        const int j = (int)s_mod[i];
+        const uint32_t slot = s_slot[j];
+        load_row<true>(row, a.st.pool + (size_t)slot * NN, NN, lane);   // written in this kernel: read through to L2
+        if (a.cur) load_row<false>(crow, a.cur + (size_t)j * NN, NN, lane);
+        __syncwarp();
+        int K, N, nd;
+        summarise_row(row, NN, a.cur ? crow : nullptr, lane, K, N, nd, recw);
+        const uint32_t word = pack_summary(K, N, nd);
+        if (lane == 0) {
+          recw[REC_SUMM] = word;
+          recw[REC_TERM] = 0u;
+          s_summ[j] = word;
+        }
+        __syncwarp();
+        if (lane < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + lane] = recw[lane];
+        __syncwarp();
+      }
+    }
+    __syncthreads();
   }
-  __syncthreads();
 
   // ---- children's indices out, fitness of the candidate (Eq. 14) from the rows' terms ----------
   uint32_t *pout = a.ptr_out + (size_t)c * J;
