@@ -35,32 +35,107 @@ struct StoreView {
   uint32_t zero_slot;
 };
 
+// ---- a row as 16-byte pieces of 8 entries (entries of stored rows are in [0, 2047]) -----------
+__device__ __forceinline__ uint32_t piece_mask(uint4 x) {   // bit h: entry h of the piece is occupied
+  return ((x.x & 0xFFFFu) ? 1u : 0u) | ((x.x >> 16) ? 2u : 0u) | ((x.y & 0xFFFFu) ? 4u : 0u) | ((x.y >> 16) ? 8u : 0u) |
+         ((x.z & 0xFFFFu) ? 16u : 0u) | ((x.z >> 16) ? 32u : 0u) | ((x.w & 0xFFFFu) ? 64u : 0u) | ((x.w >> 16) ? 128u : 0u);
+}
+__device__ __forceinline__ int piece_sum(uint4 x) {
+  int k = __dp2a_lo((int)x.x, 0x0101, 0);
+  k = __dp2a_lo((int)x.y, 0x0101, k);
+  k = __dp2a_lo((int)x.z, 0x0101, k);
+  return __dp2a_lo((int)x.w, 0x0101, k);
+}
+__device__ __forceinline__ int piece_entry(uint4 x, int h) {
+  const uint32_t w = (h < 2) ? x.x : (h < 4) ? x.y : (h < 6) ? x.z : x.w;
+  return (int)((w >> ((h & 1) * 16)) & 0xFFFFu);
+}
+__device__ __forceinline__ int piece_diff(uint4 x, uint4 c) {   // entries that differ
+  // each half of the xor is a non-negative int16, so min(half, 1) counts the halves that differ
+  const uint32_t d = __vimin_s16x2_relu(x.x ^ c.x, 0x00010001u) + __vimin_s16x2_relu(x.y ^ c.y, 0x00010001u) +
+                     __vimin_s16x2_relu(x.z ^ c.z, 0x00010001u) + __vimin_s16x2_relu(x.w ^ c.w, 0x00010001u);
+  return (int)((d & 0xFFFFu) + (d >> 16));
+}
+
+// The pieces of a row in shared memory that this lane looks after (pieces lane and lane + 32;
+// rows have at most 64), their occupancy masks, and where this lane's occupants come in node
+// order: first[q] = occupants before piece q of this lane, total = occupied nodes of the row.
+struct RowPieces {
+  uint4 x[2];
+  uint32_t mask[2];
+  int first[2], total;
+};
+
+__device__ __forceinline__ RowPieces row_pieces(const int16_t *row, int NN, int lane) {
+  RowPieces p;
+  const int row_vecs = NN >> 3;
+#pragma unroll
+  for (int q = 0; q < 2; ++q) {
+    const int v = lane + 32 * q;
+    p.x[q] = make_uint4(0u, 0u, 0u, 0u);
+    if (v < row_vecs) p.x[q] = ((const uint4 *)row)[v];
+    p.mask[q] = piece_mask(p.x[q]);
+  }
+  const uint32_t cnt = (uint32_t)__popc(p.mask[0]) | ((uint32_t)__popc(p.mask[1]) << 16);
+  uint32_t incl = cnt;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t u = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += u;
+  }
+  const uint32_t all = __shfl_sync(0xffffffffu, incl, 31), ex = incl - cnt;
+  p.first[0] = (int)(ex & 0xFFFFu);
+  p.first[1] = (int)(all & 0xFFFFu) + (int)(ex >> 16);
+  p.total = (int)(all & 0xFFFFu) + (int)(all >> 16);
+  return p;
+}
+
 // K, N, entries differing from `cur_row` (NULL: none) and the occupant entries of a row; both
-// rows are held in shared memory.  All lanes return the same K, N, ndiff; rec_out (shared, REC_WORDS: the
-// entries, the summary word is the caller's) is complete after the trailing __syncwarp().
+// rows are held in shared memory (16-byte aligned, a multiple of 8 entries).  All lanes return
+// the same K, N, ndiff; rec_out (shared, REC_WORDS: the entries, the other words are the
+// caller's) is complete after the trailing __syncwarp().
 __device__ __forceinline__ void summarise_row(const int16_t *row, int NN, const int16_t *cur_row, int lane,
                                               int &K, int &N, int &ndiff, uint32_t *rec_out) {
-  int k = 0, nd = 0, cnt = 0;
-  for (int base = 0; base < NN; base += 32) {
-    const int n = base + lane;
-    const int v = (n < NN) ? (int)row[n] : 0;
-    if (cur_row && n < NN) nd += (v != (int)cur_row[n]) ? 1 : 0;
-    k += v;
-    const unsigned m = __ballot_sync(0xffffffffu, v > 0);
-    const int pos = cnt + __popc(m & ((1u << lane) - 1u));
-    if (v > 0 && pos < REC_ENTRIES) rec_out[pos] = (uint32_t)n | ((uint32_t)v << 12);
-    cnt += __popc(m);
+  const RowPieces p = row_pieces(row, NN, lane);
+  const int row_vecs = NN >> 3;
+  int k = 0, nd = 0;
+#pragma unroll
+  for (int q = 0; q < 2; ++q) {
+    const int v = lane + 32 * q;
+    k += piece_sum(p.x[q]);
+    if (cur_row && v < row_vecs) nd += piece_diff(p.x[q], ((const uint4 *)cur_row)[v]);
+    int pos = p.first[q];
+    uint32_t m = p.mask[q];
+    while (m && pos < REC_ENTRIES) {
+      const int h = __ffs(m) - 1;
+      m &= m - 1;
+      rec_out[pos++] = (uint32_t)(8 * v + h) | ((uint32_t)piece_entry(p.x[q], h) << 12);
+    }
   }
   K = warp_sum(k);
   ndiff = warp_sum(nd);
-  N = cnt;
+  N = p.total;
   __syncwarp();
-  if (cnt > REC_ENTRIES) {
+  if (N > REC_ENTRIES) {
     if (lane == 0) rec_out[0] = REC_OVERFLOW;
-  } else if (lane >= cnt && lane < REC_ENTRIES) {
+  } else if (lane >= N && lane < REC_ENTRIES) {
     rec_out[lane] = 0u;
   }
   __syncwarp();
+}
+
+// node index of the t-th occupied entry (ascending) of a row held in shared memory; t < N
+__device__ __forceinline__ int nth_occupied_row(const int16_t *row, int NN, uint32_t t, int lane) {
+  const RowPieces p = row_pieces(row, NN, lane);
+  int node = -1;
+#pragma unroll
+  for (int q = 0; q < 2; ++q) {
+    const int c = __popc(p.mask[q]);
+    if ((int)t >= p.first[q] && (int)t < p.first[q] + c)
+      node = 8 * (lane + 32 * q) + (int)__fns(p.mask[q], 0, (int)t - p.first[q] + 1);
+  }
+  const unsigned who = __ballot_sync(0xffffffffu, node >= 0);
+  return __shfl_sync(0xffffffffu, node, who ? __ffs(who) - 1 : 0);
 }
 
 // A row of NN entries from global to shared memory, 16 bytes per lane and step when the
@@ -454,6 +529,22 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
     if (k < OCC) s_occ[n * OCC + k] = (uint32_t)j | ((uint32_t)g << 13) | (dist ? 0x80000000u : 0u);
   };
 
+  // all occupants of a row held in shared memory (whole warp)
+  auto add_row_occupants = [&](int j, const int16_t *r, bool dist) {
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const int v = lane + 32 * q;
+      if (v >= (NN >> 3)) continue;
+      const uint4 x = ((const uint4 *)r)[v];
+      uint32_t m = piece_mask(x);
+      while (m) {
+        const int h = __ffs(m) - 1;
+        m &= m - 1;
+        add_occupant(j, 8 * v + h, piece_entry(x, h), dist);
+      }
+    }
+  };
+
   // ---- rows, one thread each: the child row is the chosen parent's row -----------------------
   // First every row's draws (which parent; perturbed or not).  The count of perturbed rows is
   // then known and the block takes its slots - those plus a reserve for the rows the column
@@ -542,14 +633,14 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       if (a.cur) load_row<false>(crow, a.cur + (size_t)j * NN, NN, lane);
       const int kc_in = a.k_cap ? a.k_cap[j] : a.k_max;
       __syncwarp();
-      int rK = (int)(w & 0x7FFu), rN = (int)((w >> 11) & 0x7FFu);
+      const int rN = (int)((w >> 11) & 0x7FFu);
       const u32x4 mw = draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE);
       const uint32_t op = bounded(mw.y, 3u);
       if (op == 0u) {
         const int n = (int)bounded(mw.w, (uint32_t)NN);
         if (lane == 0) row[n] = (int16_t)min((int)row[n] + 1, (int)s_cap[n]);
       } else if (rN > 0) {
-        const int ns = nth_occupied(row, NN, bounded(mw.z, (uint32_t)rN), lane);
+        const int ns = nth_occupied_row(row, NN, bounded(mw.z, (uint32_t)rN), lane);
         if (op == 1u) {
           if (lane == 0) row[ns] = (int16_t)(row[ns] - 1);
         } else {
@@ -561,16 +652,14 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         }
       }
       __syncwarp();
-      rK = 0; rN = 0;
-      for (int n = lane; n < NN; n += 32) { rK += row[n]; rN += row[n] > 0; }
-      rK = warp_sum(rK);
-      rN = warp_sum(rN);
+      int K, N, nd;
+      summarise_row(row, NN, a.cur ? crow : nullptr, lane, K, N, nd, recw);
       // per-row caps: replicas above the job's cap leave from the highest node index down, then
       // occupied nodes beyond n_max are cleared from the highest index down
       const int kc = max(0, min(kc_in, a.k_max));
-      if (rK > kc || rN > a.n_max) {
+      if (K > kc || N > a.n_max) {
         if (lane == 0) {
-          int excess = rK - kc;
+          int excess = K - kc;
           for (int n = NN - 1; n >= 0 && excess > 0; --n) {
             const int take = min((int)row[n], excess);
             row[n] = (int16_t)(row[n] - take);
@@ -585,9 +674,8 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
           }
         }
         __syncwarp();
+        summarise_row(row, NN, a.cur ? crow : nullptr, lane, K, N, nd, recw);
       }
-      int K, N, nd;
-      summarise_row(row, NN, a.cur ? crow : nullptr, lane, K, N, nd, recw);
       const uint32_t slot = s_base_mut + (uint32_t)i;
       uint4 *d4 = (uint4 *)(a.st.pool + (size_t)slot * NN);
       for (int v = lane; v < row_vecs; v += 32) d4[v] = ((const uint4 *)row)[v];
@@ -601,21 +689,17 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       }
       __syncwarp();
       if (lane < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + lane] = recw[lane];
-      const bool dist = N >= 2;
-      for (int n = lane; n < NN; n += 32)
-        if (row[n] > 0) add_occupant(j, n, (int)row[n], dist);
+      add_row_occupants(j, row, N >= 2);
       __syncwarp();
     }
   }
   // rows with more occupied nodes than a record holds: occupants from the row itself
   for (int i = warp; i < s_novf; i += GEN_WARPS) {
     const int j = (int)s_ovf[i];
-    const int16_t *src = a.st.pool + (size_t)s_slot[j] * NN;
-    const bool dist = ((s_summ[j] >> 11) & 0x7FFu) >= 2u;
-    for (int n = lane; n < NN; n += 32) {
-      const int v = (int)src[n];
-      if (v > 0) add_occupant(j, n, v, dist);
-    }
+    load_row<false>(row, a.st.pool + (size_t)s_slot[j] * NN, NN, lane);
+    __syncwarp();
+    add_row_occupants(j, row, ((s_summ[j] >> 11) & 0x7FFu) >= 2u);
+    __syncwarp();
   }
   __syncthreads();
 
@@ -684,12 +768,20 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         load_row<true>(row, a.st.pool + (size_t)src * NN, NN, lane);   // may have been written in this kernel
         if (a.cur) load_row<false>(crow, a.cur + (size_t)j * NN, NN, lane);
         __syncwarp();
-        for (int n = lane; n < NN; n += 32) {
-          if (row[n] > 0 && s_viol[n] == 1) {
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const int v = lane + 32 * q;
+          if (v >= row_vecs) continue;
+          uint32_t m = piece_mask(((const uint4 *)row)[v]);
+          while (m) {
+            const int n = 8 * v + __ffs(m) - 1;
+            m &= m - 1;
+            if (s_viol[n] != 1) continue;
             const int cnt = (int)(s_node[n] >> 48);
             for (int k = 0; k < cnt; ++k) {
-              if ((int)(s_occ[n * OCC + k] & 0x1FFFu) == j) {
-                row[n] = (int16_t)((s_occ[n * OCC + k] >> 13) & 0x7FFu);
+              const uint32_t e = s_occ[n * OCC + k];
+              if ((int)(e & 0x1FFFu) == j) {
+                if ((e >> 24) & 1u) row[n] = (int16_t)((e >> 13) & 0x7FFu);
                 break;
               }
             }
