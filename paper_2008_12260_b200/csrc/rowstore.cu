@@ -25,6 +25,7 @@ constexpr uint32_t REC_OVERFLOW = 0xFFFFFFFFu;  // first word of a record whose 
 constexpr int OCC = 16;                       // occupants listed per node inside a block
 constexpr int GEN_THREADS = 256;
 constexpr int GEN_WARPS = GEN_THREADS / 32;
+constexpr int GEN_GROUPS = GEN_THREADS / 16;  // rows worked on at a time by a block
 constexpr int STORE_MAX_JOBS = 8192;          // job index must fit 13 bits of an occupant entry
 constexpr int COW_RESERVE = 24;               // slots a block takes up front for rows the column pass changes
 
@@ -57,54 +58,98 @@ __device__ __forceinline__ int piece_diff(uint4 x, uint4 c) {   // entries that 
   return (int)((d & 0xFFFFu) + (d >> 16));
 }
 
-// The pieces of a row in shared memory that this lane looks after (pieces lane and lane + 32;
-// rows have at most 64), their occupancy masks, and where this lane's occupants come in node
-// order: first[q] = occupants before piece q of this lane, total = occupied nodes of the row.
-struct RowPieces {
-  uint4 x[2];
-  uint32_t mask[2];
-  int first[2], total;
+// Rows are worked on by groups of 16 lanes (two rows per warp at a time).  A lane looks after
+// the ROW_PPL-or-fewer consecutive pieces [sub * ppl, sub * ppl + ppl) of its group's row, so
+// lane order is node order.
+constexpr int GROUP = 16;
+constexpr int ROW_PPL = 4;   // rows have at most 64 pieces
+
+struct Grp {
+  int sub;         // lane within the group
+  unsigned mask;   // the group's lanes
+  int row_vecs;    // pieces of a row
+  int ppl;         // pieces per lane
 };
 
-__device__ __forceinline__ RowPieces row_pieces(const int16_t *row, int NN, int lane) {
+__device__ __forceinline__ Grp make_group(int lane, int NN) {
+  Grp g;
+  g.sub = lane & (GROUP - 1);
+  g.mask = 0xFFFFu << (lane & GROUP);
+  g.row_vecs = NN >> 3;
+  g.ppl = (g.row_vecs + GROUP - 1) / GROUP;
+  return g;
+}
+
+__device__ __forceinline__ int group_sum(const Grp &g, int v) { return __reduce_add_sync(g.mask, v); }
+
+// 16 bytes of a row in global memory (any alignment of the row's start); `cg` reads through to
+// L2, for rows written earlier in the same kernel
+template <bool CG>
+__device__ __forceinline__ uint4 load_piece(const int16_t *src, int v) {
+  if (((uintptr_t)src & 15) == 0) return CG ? __ldcg((const uint4 *)src + v) : *((const uint4 *)src + v);
+  uint32_t w[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t lo = (uint16_t)(CG ? __ldcg(src + 8 * v + 2 * k) : src[8 * v + 2 * k]);
+    const uint32_t hi = (uint16_t)(CG ? __ldcg(src + 8 * v + 2 * k + 1) : src[8 * v + 2 * k + 1]);
+    w[k] = lo | (hi << 16);
+  }
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// a row from global to shared memory by one group (coalesced: piece sub, sub + 16, ...)
+template <bool CG>
+__device__ __forceinline__ void load_row(const Grp &g, int16_t *dst, const int16_t *src) {
+  for (int v = g.sub; v < g.row_vecs; v += GROUP) ((uint4 *)dst)[v] = load_piece<CG>(src, v);
+}
+
+__device__ __forceinline__ void store_row(const Grp &g, int16_t *dst, const int16_t *src_shared) {
+  for (int v = g.sub; v < g.row_vecs; v += GROUP) ((uint4 *)dst)[v] = ((const uint4 *)src_shared)[v];
+}
+
+// This lane's pieces of a row in shared memory, their occupancy masks, and where the lane's
+// occupants come in node order: `first` = occupants in lower lanes, `total` = the row's N.
+struct RowPieces {
+  uint4 x[ROW_PPL];
+  uint32_t mask[ROW_PPL];
+  int first, total;
+};
+
+__device__ __forceinline__ RowPieces row_pieces(const Grp &g, const int16_t *row) {
   RowPieces p;
-  const int row_vecs = NN >> 3;
+  int cnt = 0;
 #pragma unroll
-  for (int q = 0; q < 2; ++q) {
-    const int v = lane + 32 * q;
+  for (int q = 0; q < ROW_PPL; ++q) {
+    const int v = g.sub * g.ppl + q;
     p.x[q] = make_uint4(0u, 0u, 0u, 0u);
-    if (v < row_vecs) p.x[q] = ((const uint4 *)row)[v];
+    if (q < g.ppl && v < g.row_vecs) p.x[q] = ((const uint4 *)row)[v];
     p.mask[q] = piece_mask(p.x[q]);
+    cnt += __popc(p.mask[q]);
   }
-  const uint32_t cnt = (uint32_t)__popc(p.mask[0]) | ((uint32_t)__popc(p.mask[1]) << 16);
-  uint32_t incl = cnt;
+  int incl = cnt;
 #pragma unroll
-  for (int off = 1; off < 32; off <<= 1) {
-    const uint32_t u = __shfl_up_sync(0xffffffffu, incl, off);
-    if (lane >= off) incl += u;
+  for (int off = 1; off < GROUP; off <<= 1) {
+    const int u = __shfl_up_sync(g.mask, incl, off, GROUP);
+    if (g.sub >= off) incl += u;
   }
-  const uint32_t all = __shfl_sync(0xffffffffu, incl, 31), ex = incl - cnt;
-  p.first[0] = (int)(ex & 0xFFFFu);
-  p.first[1] = (int)(all & 0xFFFFu) + (int)(ex >> 16);
-  p.total = (int)(all & 0xFFFFu) + (int)(all >> 16);
+  p.total = __shfl_sync(g.mask, incl, GROUP - 1, GROUP);
+  p.first = incl - cnt;
   return p;
 }
 
-// K, N, entries differing from `cur_row` (NULL: none) and the occupant entries of a row; both
-// rows are held in shared memory (16-byte aligned, a multiple of 8 entries).  All lanes return
-// the same K, N, ndiff; rec_out (shared, REC_WORDS: the entries, the other words are the
-// caller's) is complete after the trailing __syncwarp().
-__device__ __forceinline__ void summarise_row(const int16_t *row, int NN, const int16_t *cur_row, int lane,
-                                              int &K, int &N, int &ndiff, uint32_t *rec_out) {
-  const RowPieces p = row_pieces(row, NN, lane);
-  const int row_vecs = NN >> 3;
-  int k = 0, nd = 0;
+// K, N, entries differing from the current allocation's row (`cur_row` in global memory, NULL:
+// none) and the occupant entries of a row held in shared memory.  All lanes of the group
+// return the same K, N, ndiff; rec_out (shared, REC_WORDS: the entries, the other words are the
+// caller's) is complete after the trailing __syncwarp(group).
+__device__ __forceinline__ RowPieces summarise_row(const Grp &g, const int16_t *row, const int16_t *cur_row,
+                                                   int &K, int &N, int &ndiff, uint32_t *rec_out) {
+  const RowPieces p = row_pieces(g, row);
+  int k = 0, nd = 0, pos = p.first;
 #pragma unroll
-  for (int q = 0; q < 2; ++q) {
-    const int v = lane + 32 * q;
+  for (int q = 0; q < ROW_PPL; ++q) {
+    const int v = g.sub * g.ppl + q;
     k += piece_sum(p.x[q]);
-    if (cur_row && v < row_vecs) nd += piece_diff(p.x[q], ((const uint4 *)cur_row)[v]);
-    int pos = p.first[q];
+    if (cur_row && q < g.ppl && v < g.row_vecs) nd += piece_diff(p.x[q], load_piece<false>(cur_row, v));
     uint32_t m = p.mask[q];
     while (m && pos < REC_ENTRIES) {
       const int h = __ffs(m) - 1;
@@ -112,42 +157,32 @@ __device__ __forceinline__ void summarise_row(const int16_t *row, int NN, const 
       rec_out[pos++] = (uint32_t)(8 * v + h) | ((uint32_t)piece_entry(p.x[q], h) << 12);
     }
   }
-  K = warp_sum(k);
-  ndiff = warp_sum(nd);
+  K = group_sum(g, k);
+  ndiff = group_sum(g, nd);
   N = p.total;
-  __syncwarp();
+  __syncwarp(g.mask);
   if (N > REC_ENTRIES) {
-    if (lane == 0) rec_out[0] = REC_OVERFLOW;
-  } else if (lane >= N && lane < REC_ENTRIES) {
-    rec_out[lane] = 0u;
+    if (g.sub == 0) rec_out[0] = REC_OVERFLOW;
+  } else if (g.sub >= N && g.sub < REC_ENTRIES) {
+    rec_out[g.sub] = 0u;
   }
-  __syncwarp();
+  __syncwarp(g.mask);
+  return p;
 }
 
 // node index of the t-th occupied entry (ascending) of a row held in shared memory; t < N
-__device__ __forceinline__ int nth_occupied_row(const int16_t *row, int NN, uint32_t t, int lane) {
-  const RowPieces p = row_pieces(row, NN, lane);
-  int node = -1;
+__device__ __forceinline__ int nth_occupied_row(const Grp &g, const int16_t *row, uint32_t t) {
+  const RowPieces p = row_pieces(g, row);
+  int node = -1, before = p.first;
 #pragma unroll
-  for (int q = 0; q < 2; ++q) {
+  for (int q = 0; q < ROW_PPL; ++q) {
     const int c = __popc(p.mask[q]);
-    if ((int)t >= p.first[q] && (int)t < p.first[q] + c)
-      node = 8 * (lane + 32 * q) + (int)__fns(p.mask[q], 0, (int)t - p.first[q] + 1);
+    if ((int)t >= before && (int)t < before + c)
+      node = 8 * (g.sub * g.ppl + q) + (int)__fns(p.mask[q], 0, (int)t - before + 1);
+    before += c;
   }
-  const unsigned who = __ballot_sync(0xffffffffu, node >= 0);
-  return __shfl_sync(0xffffffffu, node, who ? __ffs(who) - 1 : 0);
-}
-
-// A row of NN entries from global to shared memory, 16 bytes per lane and step when the
-// source allows; `cg` reads through to L2 (for rows written earlier in the same kernel).
-template <bool CG>
-__device__ __forceinline__ void load_row(int16_t *dst, const int16_t *src, int NN, int lane) {
-  if (((uintptr_t)src & 15) == 0) {
-    for (int v = lane; v < (NN >> 3); v += 32)
-      ((uint4 *)dst)[v] = CG ? __ldcg((const uint4 *)src + v) : *((const uint4 *)src + v);
-  } else {
-    for (int n = lane; n < NN; n += 32) dst[n] = CG ? __ldcg(src + n) : src[n];
-  }
+  const unsigned who = __ballot_sync(g.mask, node >= 0);
+  return __shfl_sync(g.mask, node, who ? __ffs(who) - 1 : (__ffs(g.mask) - 1));
 }
 
 // one 32-byte record with a single request
@@ -178,36 +213,35 @@ struct BuildArgs {
 };
 
 __global__ void __launch_bounds__(256) rowstore_build_kernel(BuildArgs a) {
-  __shared__ __align__(16) int16_t s_row[8][512];
-  __shared__ __align__(16) int16_t s_cur[8][512];
-  __shared__ uint32_t s_rec[8][REC_WORDS];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __shared__ __align__(16) int16_t s_row[16][512];
+  __shared__ uint32_t s_rec[16][REC_WORDS];
+  const int lane = threadIdx.x & 31, grp = threadIdx.x >> 4;   // 16 groups of 16 lanes, a row each
+  const Grp g = make_group(lane, a.NN);
   const long long rows = (long long)a.P * a.J;
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     a.state[0] = (unsigned int)rows;
     a.state[1] = 0u;
   }
-  // the empty row: contents, record and summary all zero
+  // the empty row: contents and record all zero
   if (blockIdx.x == 0) {
     for (int n = threadIdx.x; n < a.NN; n += blockDim.x) a.st.pool[(size_t)a.st.zero_slot * a.NN + n] = 0;
     if (threadIdx.x < REC_WORDS) a.st.rec[(size_t)a.st.zero_slot * REC_WORDS + threadIdx.x] = 0u;
   }
-  for (long long r = (long long)blockIdx.x * 8 + warp; r < rows; r += (long long)gridDim.x * 8) {
+  for (long long r = (long long)blockIdx.x * 16 + grp; r < rows; r += (long long)gridDim.x * 16) {
     const int j = (int)(r % a.J);
-    load_row<false>(s_row[warp], a.st.pool + (size_t)r * a.NN, a.NN, lane);
-    if (a.cur) load_row<false>(s_cur[warp], a.cur + (size_t)j * a.NN, a.NN, lane);
-    __syncwarp();
+    load_row<false>(g, s_row[grp], a.st.pool + (size_t)r * a.NN);
+    __syncwarp(g.mask);
     int K, N, nd;
-    summarise_row(s_row[warp], a.NN, a.cur ? s_cur[warp] : nullptr, lane, K, N, nd, s_rec[warp]);
+    summarise_row(g, s_row[grp], a.cur ? a.cur + (size_t)j * a.NN : nullptr, K, N, nd, s_rec[grp]);
     const bool on = !a.active || a.active[j];
-    if (lane == 0) {
-      s_rec[warp][REC_SUMM] = on ? pack_summary(K, N, nd) : 0u;
-      s_rec[warp][REC_TERM] = on ? __float_as_uint(fitness_term(a.tp, j, K, N, nd != 0)) : 0u;
+    if (g.sub == 0) {
+      s_rec[grp][REC_SUMM] = on ? pack_summary(K, N, nd) : 0u;
+      s_rec[grp][REC_TERM] = on ? __float_as_uint(fitness_term(a.tp, j, K, N, nd != 0)) : 0u;
       a.ptr[r] = (uint32_t)r;
     }
-    __syncwarp();
-    if (lane < REC_WORDS) a.st.rec[(size_t)r * REC_WORDS + lane] = s_rec[warp][lane];
-    __syncwarp();
+    __syncwarp(g.mask);
+    if (g.sub < REC_WORDS) a.st.rec[(size_t)r * REC_WORDS + g.sub] = s_rec[grp][g.sub];
+    __syncwarp(g.mask);
   }
 }
 
@@ -356,13 +390,13 @@ __host__ __device__ inline GenSmem gen_smem_layout(int J, int NN) {
   TAKE(acc, (size_t)NN * 8);
   TAKE(viol, (size_t)NN);
   TAKE(occ, (size_t)NN * OCC * 4);
-  // per warp: a row and its counterpart in the current allocation
-  TAKE(rowbuf, (size_t)2 * GEN_WARPS * NN * 2);
+  // a row per group of 16 lanes
+  TAKE(rowbuf, (size_t)GEN_GROUPS * NN * 2);
   TAKE(mut, (size_t)J * 2);
   TAKE(ovf, (size_t)J * 2);
   TAKE(mod, (size_t)J * 2);
   TAKE(cap, (size_t)NN * 2);
-  TAKE(rec, (size_t)GEN_WARPS * REC_WORDS * 4);
+  TAKE(rec, (size_t)GEN_GROUPS * REC_WORDS * 4);
 #undef TAKE
   L.total = off;
   return L;
@@ -523,24 +557,21 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
 
   // occupant (job j holds g GPUs on node n) into the node's totals and list
   auto add_occupant = [&](int j, int n, int g, bool dist) {
-    const unsigned long long old =
-        atomicAdd(&s_node[n], (unsigned long long)(unsigned)g | (dist ? (1ull << 32) : 0ull) | (1ull << 48));
-    const int k = (int)(old >> 48);
+    uint32_t *w = (uint32_t *)&s_node[n];   // two 32-bit adds: the low word's answer is not needed
+    atomicAdd(&w[0], (uint32_t)g);
+    const int k = (int)(atomicAdd(&w[1], (dist ? 1u : 0u) | (1u << 16)) >> 16);
     if (k < OCC) s_occ[n * OCC + k] = (uint32_t)j | ((uint32_t)g << 13) | (dist ? 0x80000000u : 0u);
   };
 
-  // all occupants of a row held in shared memory (whole warp)
-  auto add_row_occupants = [&](int j, const int16_t *r, bool dist) {
+  // the occupants in this lane's pieces of a row
+  auto add_row_occupants = [&](const Grp &g, int j, const RowPieces &p, bool dist) {
 #pragma unroll
-    for (int q = 0; q < 2; ++q) {
-      const int v = lane + 32 * q;
-      if (v >= (NN >> 3)) continue;
-      const uint4 x = ((const uint4 *)r)[v];
-      uint32_t m = piece_mask(x);
+    for (int q = 0; q < ROW_PPL; ++q) {
+      uint32_t m = p.mask[q];
       while (m) {
         const int h = __ffs(m) - 1;
         m &= m - 1;
-        add_occupant(j, 8 * v + h, piece_entry(x, h), dist);
+        add_occupant(j, 8 * (g.sub * g.ppl + q) + h, piece_entry(p.x[q], h), dist);
       }
     }
   };
@@ -614,51 +645,46 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   }
   __syncthreads();
 
-  // ---- perturbed rows, one warp each: new row in a fresh slot ---------------------------------
-  int16_t *row = s_rowbuf + (size_t)warp * NN;                  // this warp's row
-  int16_t *crow = s_rowbuf + (size_t)(GEN_WARPS + warp) * NN;   // and its counterpart in the current allocation
-  uint32_t *recw = s_rec + warp * REC_WORDS;
-  const int row_vecs = NN >> 3;
+  // ---- perturbed rows, one group of 16 lanes each: new row in a fresh slot --------------------
+  const Grp g = make_group(lane, NN);
+  const int grp = tid >> 4;
+  int16_t *row = s_rowbuf + (size_t)grp * NN;   // this group's row
+  uint32_t *recw = s_rec + grp * REC_WORDS;
   if (!s_fail) {
-    // the warp's rows and their counterparts in the current allocation are asked for up front
-    for (int i = warp; i < s_nmut; i += GEN_WARPS) {
-      const int j = (int)s_mut[i];
-      if (lane * 64 < NN) prefetch_l2(a.st.pool + (size_t)s_slot[j] * NN + lane * 64);
-      if (a.cur && lane * 64 < NN) prefetch_l2(a.cur + (size_t)j * NN + lane * 64);
-    }
-    for (int i = warp; i < s_nmut; i += GEN_WARPS) {
+    for (int i = grp; i < s_nmut; i += GEN_GROUPS) {
       const int j = (int)s_mut[i];
       const uint32_t old = s_slot[j], w = s_summ[j];
-      load_row<false>(row, a.st.pool + (size_t)old * NN, NN, lane);
-      if (a.cur) load_row<false>(crow, a.cur + (size_t)j * NN, NN, lane);
+      load_row<false>(g, row, a.st.pool + (size_t)old * NN);
+      const int16_t *cur_row = a.cur ? a.cur + (size_t)j * NN : nullptr;
+      if (cur_row) prefetch_l2(cur_row + g.sub * 8 * g.ppl);
       const int kc_in = a.k_cap ? a.k_cap[j] : a.k_max;
-      __syncwarp();
+      __syncwarp(g.mask);
       const int rN = (int)((w >> 11) & 0x7FFu);
       const u32x4 mw = draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE);
       const uint32_t op = bounded(mw.y, 3u);
       if (op == 0u) {
         const int n = (int)bounded(mw.w, (uint32_t)NN);
-        if (lane == 0) row[n] = (int16_t)min((int)row[n] + 1, (int)s_cap[n]);
+        if (g.sub == 0) row[n] = (int16_t)min((int)row[n] + 1, (int)s_cap[n]);
       } else if (rN > 0) {
-        const int ns = nth_occupied_row(row, NN, bounded(mw.z, (uint32_t)rN), lane);
+        const int ns = nth_occupied_row(g, row, bounded(mw.z, (uint32_t)rN));
         if (op == 1u) {
-          if (lane == 0) row[ns] = (int16_t)(row[ns] - 1);
+          if (g.sub == 0) row[ns] = (int16_t)(row[ns] - 1);
         } else {
           const int nd = (int)bounded(mw.w, (uint32_t)NN);
-          if (nd != ns && lane == 0) {
+          if (nd != ns && g.sub == 0) {
             row[nd] = (int16_t)min((int)row[nd] + (int)row[ns], (int)s_cap[nd]);
             row[ns] = 0;
           }
         }
       }
-      __syncwarp();
+      __syncwarp(g.mask);
       int K, N, nd;
-      summarise_row(row, NN, a.cur ? crow : nullptr, lane, K, N, nd, recw);
+      RowPieces p = summarise_row(g, row, cur_row, K, N, nd, recw);
       // per-row caps: replicas above the job's cap leave from the highest node index down, then
       // occupied nodes beyond n_max are cleared from the highest index down
       const int kc = max(0, min(kc_in, a.k_max));
       if (K > kc || N > a.n_max) {
-        if (lane == 0) {
+        if (g.sub == 0) {
           int excess = K - kc;
           for (int n = NN - 1; n >= 0 && excess > 0; --n) {
             const int take = min((int)row[n], excess);
@@ -673,33 +699,33 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
             }
           }
         }
-        __syncwarp();
-        summarise_row(row, NN, a.cur ? crow : nullptr, lane, K, N, nd, recw);
+        __syncwarp(g.mask);
+        p = summarise_row(g, row, cur_row, K, N, nd, recw);
       }
       const uint32_t slot = s_base_mut + (uint32_t)i;
-      uint4 *d4 = (uint4 *)(a.st.pool + (size_t)slot * NN);
-      for (int v = lane; v < row_vecs; v += 32) d4[v] = ((const uint4 *)row)[v];
+      store_row(g, a.st.pool + (size_t)slot * NN, row);
       const uint32_t word = pack_summary(K, N, nd);
-      if (lane == 0) {
+      if (g.sub == 0) {
         recw[REC_SUMM] = word;
         recw[REC_TERM] = 0u;   // filled in with the other new rows' terms at the end
         s_slot[j] = slot;
         s_summ[j] = word;
         s_mark[j] = 2;
       }
-      __syncwarp();
-      if (lane < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + lane] = recw[lane];
-      add_row_occupants(j, row, N >= 2);
-      __syncwarp();
+      __syncwarp(g.mask);
+      if (g.sub < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + g.sub] = recw[g.sub];
+      add_row_occupants(g, j, p, N >= 2);
+      __syncwarp(g.mask);
     }
   }
   // rows with more occupied nodes than a record holds: occupants from the row itself
-  for (int i = warp; i < s_novf; i += GEN_WARPS) {
+  for (int i = grp; i < s_novf; i += GEN_GROUPS) {
     const int j = (int)s_ovf[i];
-    load_row<false>(row, a.st.pool + (size_t)s_slot[j] * NN, NN, lane);
-    __syncwarp();
-    add_row_occupants(j, row, ((s_summ[j] >> 11) & 0x7FFu) >= 2u);
-    __syncwarp();
+    load_row<false>(g, row, a.st.pool + (size_t)s_slot[j] * NN);
+    __syncwarp(g.mask);
+    const RowPieces p = row_pieces(g, row);
+    add_row_occupants(g, j, p, ((s_summ[j] >> 11) & 0x7FFu) >= 2u);
+    __syncwarp(g.mask);
   }
   __syncthreads();
 
@@ -746,7 +772,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   __syncthreads();
 
   // ---- rows the column pass changes -----------------------------------------------------------
-  // Usual case (every violating node's occupants were listed): one warp per changed row takes
+  // Usual case (every violating node's occupants were listed): one group per changed row takes
   // the row, applies the decisions of its nodes, and writes it with its record - to a slot of
   // its own unless the row is new in this generation already.
   const int nmod = s_nmod;
@@ -761,48 +787,47 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       __syncthreads();
     }
     if (!s_fail) {
-      for (int i = warp; i < nmod; i += GEN_WARPS) {
+      for (int i = grp; i < nmod; i += GEN_GROUPS) {
         const int j = (int)s_mod[i];
         const bool own = (s_mark[j] & 2) != 0;
         const uint32_t src = s_slot[j];
-        load_row<true>(row, a.st.pool + (size_t)src * NN, NN, lane);   // may have been written in this kernel
-        if (a.cur) load_row<false>(crow, a.cur + (size_t)j * NN, NN, lane);
-        __syncwarp();
+        load_row<true>(g, row, a.st.pool + (size_t)src * NN);   // may have been written in this kernel
+        __syncwarp(g.mask);
+        {
+          const RowPieces p = row_pieces(g, row);
 #pragma unroll
-        for (int q = 0; q < 2; ++q) {
-          const int v = lane + 32 * q;
-          if (v >= row_vecs) continue;
-          uint32_t m = piece_mask(((const uint4 *)row)[v]);
-          while (m) {
-            const int n = 8 * v + __ffs(m) - 1;
-            m &= m - 1;
-            if (s_viol[n] != 1) continue;
-            const int cnt = (int)(s_node[n] >> 48);
-            for (int k = 0; k < cnt; ++k) {
-              const uint32_t e = s_occ[n * OCC + k];
-              if ((int)(e & 0x1FFFu) == j) {
-                if ((e >> 24) & 1u) row[n] = (int16_t)((e >> 13) & 0x7FFu);
-                break;
+          for (int q = 0; q < ROW_PPL; ++q) {
+            uint32_t m = p.mask[q];
+            while (m) {
+              const int n = 8 * (g.sub * g.ppl + q) + __ffs(m) - 1;
+              m &= m - 1;
+              if (s_viol[n] != 1) continue;
+              const int cnt = (int)(s_node[n] >> 48);
+              for (int k = 0; k < cnt; ++k) {
+                const uint32_t e = s_occ[n * OCC + k];
+                if ((int)(e & 0x1FFFu) == j) {
+                  if ((e >> 24) & 1u) row[n] = (int16_t)((e >> 13) & 0x7FFu);
+                  break;
+                }
               }
             }
           }
         }
-        __syncwarp();
+        __syncwarp(g.mask);
         int K, N, nd;
-        summarise_row(row, NN, a.cur ? crow : nullptr, lane, K, N, nd, recw);
+        summarise_row(g, row, a.cur ? a.cur + (size_t)j * NN : nullptr, K, N, nd, recw);
         const uint32_t dst = own ? src : s_base_cow + (uint32_t)i;
-        uint4 *d4 = (uint4 *)(a.st.pool + (size_t)dst * NN);
-        for (int v = lane; v < row_vecs; v += 32) d4[v] = ((const uint4 *)row)[v];
+        store_row(g, a.st.pool + (size_t)dst * NN, row);
         const uint32_t word = pack_summary(K, N, nd);
-        if (lane == 0) {
+        if (g.sub == 0) {
           recw[REC_SUMM] = word;
           recw[REC_TERM] = 0u;
           s_slot[j] = dst;
           s_summ[j] = word;
         }
-        __syncwarp();
-        if (lane < REC_WORDS) a.st.rec[(size_t)dst * REC_WORDS + lane] = recw[lane];
-        __syncwarp();
+        __syncwarp(g.mask);
+        if (g.sub < REC_WORDS) a.st.rec[(size_t)dst * REC_WORDS + g.sub] = recw[g.sub];
+        __syncwarp(g.mask);
       }
     }
     __syncthreads();
@@ -823,16 +848,16 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
     }
     __syncthreads();
     if (!s_fail) {
-      for (int i = warp; i < nmod; i += GEN_WARPS) {
+      for (int i = grp; i < nmod; i += GEN_GROUPS) {
         const uint32_t k = s_ovf[i];
         if (k == 0xFFFFu) continue;
         const int j = (int)s_mod[i];
         const uint32_t slot = s_base_cow + k;
-        const uint4 *s4 = (const uint4 *)(a.st.pool + (size_t)s_slot[j] * NN);
-        uint4 *d4 = (uint4 *)(a.st.pool + (size_t)slot * NN);
-        for (int v = lane; v < row_vecs; v += 32) d4[v] = s4[v];
-        __syncwarp();
-        if (lane == 0) s_slot[j] = slot;
+        load_row<true>(g, row, a.st.pool + (size_t)s_slot[j] * NN);
+        __syncwarp(g.mask);
+        store_row(g, a.st.pool + (size_t)slot * NN, row);
+        __syncwarp(g.mask);
+        if (g.sub == 0) s_slot[j] = slot;
       }
     }
     __syncthreads();
@@ -856,23 +881,22 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
 
     // changed rows: summary and record from the row as it now stands
     if (!s_fail) {
-      for (int i = warp; i < nmod; i += GEN_WARPS) {
+      for (int i = grp; i < nmod; i += GEN_GROUPS) {
         const int j = (int)s_mod[i];
         const uint32_t slot = s_slot[j];
-        load_row<true>(row, a.st.pool + (size_t)slot * NN, NN, lane);   // written in this kernel: read through to L2
-        if (a.cur) load_row<false>(crow, a.cur + (size_t)j * NN, NN, lane);
-        __syncwarp();
+        load_row<true>(g, row, a.st.pool + (size_t)slot * NN);   // written in this kernel: read through to L2
+        __syncwarp(g.mask);
         int K, N, nd;
-        summarise_row(row, NN, a.cur ? crow : nullptr, lane, K, N, nd, recw);
+        summarise_row(g, row, a.cur ? a.cur + (size_t)j * NN : nullptr, K, N, nd, recw);
         const uint32_t word = pack_summary(K, N, nd);
-        if (lane == 0) {
+        if (g.sub == 0) {
           recw[REC_SUMM] = word;
           recw[REC_TERM] = 0u;
           s_summ[j] = word;
         }
-        __syncwarp();
-        if (lane < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + lane] = recw[lane];
-        __syncwarp();
+        __syncwarp(g.mask);
+        if (g.sub < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + g.sub] = recw[g.sub];
+        __syncwarp(g.mask);
       }
     }
     __syncthreads();
