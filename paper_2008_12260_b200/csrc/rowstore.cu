@@ -27,7 +27,7 @@ constexpr int GEN_THREADS = 256;
 constexpr int GEN_WARPS = GEN_THREADS / 32;
 constexpr int GEN_GROUPS = GEN_THREADS / 16;  // rows worked on at a time by a block
 constexpr int STORE_MAX_JOBS = 8192;          // job index must fit 13 bits of an occupant entry
-constexpr int COW_RESERVE = 24;               // slots a block takes up front for rows the column pass changes
+constexpr int COW_RESERVE = 16;               // slots a block takes up front for rows the column pass changes
 
 struct StoreView {
   int16_t *pool;
@@ -528,12 +528,20 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   } else {
     const u32x4 sel = draw(a.key, 0u, c, a.gen, SLOT_SELECT);
     const int idx[4] = {(int)bounded(sel.x, P), (int)bounded(sel.y, P), (int)bounded(sel.z, P), (int)bounded(sel.w, P)};
+    // the ranks of the four drawn candidates, a warp each; the keys are first staged in the (still
+    // unused) dynamic shared memory when they fit, so that every key is fetched once
+    uint32_t *s_keys = (uint32_t *)smem;
+    const bool staged = (size_t)P * 4 <= L.total;
+    if (staged) {
+      for (int i = tid; i < P; i += GEN_THREADS) s_keys[i] = order_key(__ldg(a.fitness_bits + i));
+      __syncthreads();
+    }
     if (warp < 4) {
       const int i = idx[warp];
-      const uint32_t ki = order_key(a.fitness_bits[i]);
+      const uint32_t ki = staged ? s_keys[i] : order_key(a.fitness_bits[i]);
       int rk = 0;
       for (int o = lane; o < P; o += 32) {
-        const uint32_t ko = order_key(__ldg(a.fitness_bits + o));
+        const uint32_t ko = staged ? s_keys[o] : order_key(__ldg(a.fitness_bits + o));
         rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
       }
       rk = warp_sum(rk);
@@ -965,7 +973,7 @@ bool rowstore_eligible(const sched_ctx *ctx, const int16_t *) {
   if (c.k_max > 2047 || c.n_max > 2047) return false;
   const unsigned long long rows = (unsigned long long)c.population * c.num_jobs;
   const unsigned long long worst = store_worst_case(c.population, c.num_jobs);
-  if (2ull * rows + 11ull * worst >= (1ull << 32)) return false;   // slot indices are 32-bit
+  if (2ull * rows + 17ull * worst >= (1ull << 32)) return false;   // slot indices are 32-bit
   if (gen_smem_layout(c.num_jobs, c.num_nodes).total > 200 * 1024) return false;
   // a half holds the population plus at least two generations' worst case; beyond 8 GiB of pool
   // the dense path runs
@@ -980,7 +988,7 @@ int rowstore_ensure(sched_ctx *ctx) {
   const unsigned long long row_bytes = (unsigned long long)c.num_nodes * 2 + REC_WORDS * 4;
   // half = the population + (gens between checks + slack) generations' worst case; shrink until
   // the pool fits 8 GiB
-  int check = 2, slack = 2;
+  int check = 4, slack = 4;
   const unsigned long long worst = store_worst_case(c.population, c.num_jobs);
   while (2ull * (rows + (check + slack) * worst) * row_bytes > (8ull << 30) && (check > 1 || slack > 1)) {
     if (slack > 1) --slack; else --check;
