@@ -221,7 +221,14 @@ int ga_generation(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_pop
  * fitness, `generations` x (ga_generation, eval_fitness), then the best candidate of the
  * last population.  d_cur: int16 [J][num_nodes] or NULL.  d_best: int16 [J][num_nodes],
  * d_best_fitness: fp32 [1].  Population and table buffers are context scratch allocated
- * on the first call. */
+ * on the first call.  Problems with more than 256 jobs (rows of whole 16-byte pieces, at
+ * most 512 nodes and 8192 jobs) keep the population of the round as shared rows - row
+ * indices per candidate into a pool of rows, copy on write - instead of dense matrices;
+ * the results are the same bit for bit, the scratch is larger (a pool of up to 8 GiB, sized
+ * at 2 x (1 + 8 worst-case generations) populations when that fits), and a pool overflow
+ * (not expected: the pool is compacted before it can run out) would be reported as device
+ * status SCHED_ERR_TOO_LARGE by sched_sync_status.  If the pool cannot be allocated the
+ * round runs on dense matrices. */
 int schedule_round(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cur, uint32_t round,
                    int32_t generations, int16_t *d_best, float *d_best_fitness);
 
