@@ -137,11 +137,29 @@ __device__ __forceinline__ RowPieces row_pieces(const Grp &g, const int16_t *row
   return p;
 }
 
-// K, N, entries differing from the current allocation's row (`cur_row` in global memory, NULL:
-// none) and the occupant entries of a row held in shared memory.  All lanes of the group
+// K, N, entries differing from the current allocation's row (`cur`: its pieces, if any) and the
+// occupant entries of a row held in shared memory.  All lanes of the group
 // return the same K, N, ndiff; rec_out (shared, REC_WORDS: the entries, the other words are the
 // caller's) is complete after the trailing __syncwarp(group).
-__device__ __forceinline__ RowPieces summarise_row(const Grp &g, const int16_t *row, const int16_t *cur_row,
+struct CurPieces {
+  uint4 x[ROW_PPL];
+  bool have;
+};
+
+// this lane's pieces of the current allocation's row (NULL: none), fetched ahead of their use
+__device__ __forceinline__ CurPieces cur_pieces(const Grp &g, const int16_t *cur_row) {
+  CurPieces c;
+  c.have = cur_row != nullptr;
+#pragma unroll
+  for (int q = 0; q < ROW_PPL; ++q) {
+    const int v = g.sub * g.ppl + q;
+    c.x[q] = make_uint4(0u, 0u, 0u, 0u);
+    if (c.have && q < g.ppl && v < g.row_vecs) c.x[q] = load_piece<false>(cur_row, v);
+  }
+  return c;
+}
+
+__device__ __forceinline__ RowPieces summarise_row(const Grp &g, const int16_t *row, const CurPieces &cur,
                                                    int &K, int &N, int &ndiff, uint32_t *rec_out) {
   const RowPieces p = row_pieces(g, row);
   int k = 0, nd = 0, pos = p.first;
@@ -149,7 +167,7 @@ __device__ __forceinline__ RowPieces summarise_row(const Grp &g, const int16_t *
   for (int q = 0; q < ROW_PPL; ++q) {
     const int v = g.sub * g.ppl + q;
     k += piece_sum(p.x[q]);
-    if (cur_row && q < g.ppl && v < g.row_vecs) nd += piece_diff(p.x[q], load_piece<false>(cur_row, v));
+    if (cur.have && q < g.ppl && v < g.row_vecs) nd += piece_diff(p.x[q], cur.x[q]);
     uint32_t m = p.mask[q];
     while (m && pos < REC_ENTRIES) {
       const int h = __ffs(m) - 1;
@@ -230,9 +248,10 @@ __global__ void __launch_bounds__(256) rowstore_build_kernel(BuildArgs a) {
   for (long long r = (long long)blockIdx.x * 16 + grp; r < rows; r += (long long)gridDim.x * 16) {
     const int j = (int)(r % a.J);
     load_row<false>(g, s_row[grp], a.st.pool + (size_t)r * a.NN);
+    const CurPieces cur = cur_pieces(g, a.cur ? a.cur + (size_t)j * a.NN : nullptr);
     __syncwarp(g.mask);
     int K, N, nd;
-    summarise_row(g, s_row[grp], a.cur ? a.cur + (size_t)j * a.NN : nullptr, K, N, nd, s_rec[grp]);
+    summarise_row(g, s_row[grp], cur, K, N, nd, s_rec[grp]);
     const bool on = !a.active || a.active[j];
     if (g.sub == 0) {
       s_rec[grp][REC_SUMM] = on ? pack_summary(K, N, nd) : 0u;
@@ -338,12 +357,12 @@ struct GenArgs {
   int *status;
 };
 
-// what the per-node repair decides for the occupant held by this lane (entry = job | GPUs << 13
-// | distributed << 31 in the first have_n lanes): the GPUs the job keeps on the node
-__device__ __forceinline__ int decide_entries(const GenArgs &a, uint32_t c, int nn, int tot, int ne, int cap_n,
-                                              int lane, uint32_t entry, int have_n) {
+// what the per-node repair decides for the occupant held by this lane of a group (entry = job |
+// GPUs << 13 | distributed << 31 in the first have_n <= 16 lanes): the GPUs the job keeps on the node
+__device__ __forceinline__ int decide_entries(const GenArgs &a, const Grp &g, uint32_t c, int nn, int tot, int ne,
+                                              int cap_n, uint32_t entry, int have_n) {
   const int J = a.J;
-  const bool have = lane < have_n;
+  const bool have = g.sub < have_n;
   const int j = (int)(entry & 0x1FFFu);
   int v = have ? (int)((entry >> 13) & 0x7FFu) : 0;
   const bool dist = have && (entry >> 31);
@@ -353,10 +372,10 @@ __device__ __forceinline__ int decide_entries(const GenArgs &a, uint32_t c, int 
     if (dist && v > 0) { t = j - o; if (t < 0) t += J; }
     int best = t;
 #pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, off));
+    for (int off = GROUP / 2; off >= 1; off >>= 1) best = min(best, __shfl_xor_sync(g.mask, best, off, GROUP));
     int removed = 0;
     if (dist && v > 0 && t != best) { removed = v; v = 0; }
-    tot -= warp_sum(removed);
+    tot -= group_sum(g, removed);
   }
   const int excess = tot - cap_n;
   if (excess > 0) {
@@ -365,8 +384,8 @@ __device__ __forceinline__ int decide_entries(const GenArgs &a, uint32_t c, int 
     if (have) { rot = j - o; if (rot < 0) rot += J; }
     int ahead = 0;                       // GPUs of the occupants that come first in rotated order
     for (int k = 0; k < have_n; ++k) {
-      const int rk = __shfl_sync(0xffffffffu, rot, k);
-      const int vk = __shfl_sync(0xffffffffu, v, k);
+      const int rk = __shfl_sync(g.mask, rot, k, GROUP);
+      const int vk = __shfl_sync(g.mask, v, k, GROUP);
       if (rk < rot) ahead += vk;
     }
     if (have) v -= min(v, max(excess - ahead, 0));
@@ -376,7 +395,7 @@ __device__ __forceinline__ int decide_entries(const GenArgs &a, uint32_t c, int 
 
 // Shared-memory carve-up of the generation kernel (sizes in bytes, 16-byte aligned pieces).
 struct GenSmem {
-  size_t slot, summ, term, mark, acc, viol, occ, rowbuf, mut, ovf, mod, cap, rec, total;
+  size_t slot, summ, term, mark, acc, viol, viollist, occ, rowbuf, mut, ovf, mod, cap, rec, total;
 };
 
 __host__ __device__ inline GenSmem gen_smem_layout(int J, int NN) {
@@ -389,6 +408,7 @@ __host__ __device__ inline GenSmem gen_smem_layout(int J, int NN) {
   TAKE(mark, (size_t)J * 4);
   TAKE(acc, (size_t)NN * 8);
   TAKE(viol, (size_t)NN);
+  TAKE(viollist, (size_t)NN * 2);
   TAKE(occ, (size_t)NN * OCC * 4);
   // a row per group of 16 lanes
   TAKE(rowbuf, (size_t)GEN_GROUPS * NN * 2);
@@ -483,12 +503,13 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   // per node: GPUs placed (bits 0..31), distributed jobs on it (32..47), occupants (48..63)
   unsigned long long *s_node = (unsigned long long *)(smem + L.acc);
   uint8_t *s_viol = (uint8_t *)(smem + L.viol);
+  uint16_t *s_viollist = (uint16_t *)(smem + L.viollist);
   uint32_t *s_occ = (uint32_t *)(smem + L.occ);
   int16_t *s_rowbuf = (int16_t *)(smem + L.rowbuf);
   uint16_t *s_mut = (uint16_t *)(smem + L.mut), *s_ovf = (uint16_t *)(smem + L.ovf), *s_mod = (uint16_t *)(smem + L.mod);
   int16_t *s_cap = (int16_t *)(smem + L.cap);
   uint32_t *s_rec = (uint32_t *)(smem + L.rec);
-  __shared__ int s_nmut, s_novf, s_nmod, s_ncow, s_fail, s_anyscan;
+  __shared__ int s_nmut, s_novf, s_nmod, s_ncow, s_fail, s_anyscan, s_nviol;
   __shared__ unsigned int s_base_mut, s_base_cow;
   __shared__ int s_parent[2], s_rank4[4];
   __shared__ double s_acc[GEN_WARPS];
@@ -560,7 +581,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
     s_cap[i] = (int16_t)max((int)a.cap[i], 0);
   }
   for (int i = tid; i < J; i += GEN_THREADS) s_mark[i] = 0;
-  if (tid == 0) { s_nmut = 0; s_novf = 0; s_nmod = 0; s_ncow = 0; s_fail = 0; s_anyscan = 0; }
+  if (tid == 0) { s_nmut = 0; s_novf = 0; s_nmod = 0; s_ncow = 0; s_fail = 0; s_anyscan = 0; s_nviol = 0; }
   __syncthreads();
 
   // occupant (job j holds g GPUs on node n) into the node's totals and list
@@ -663,8 +684,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       const int j = (int)s_mut[i];
       const uint32_t old = s_slot[j], w = s_summ[j];
       load_row<false>(g, row, a.st.pool + (size_t)old * NN);
-      const int16_t *cur_row = a.cur ? a.cur + (size_t)j * NN : nullptr;
-      if (cur_row) prefetch_l2(cur_row + g.sub * 8 * g.ppl);
+      const CurPieces cur = cur_pieces(g, a.cur ? a.cur + (size_t)j * NN : nullptr);
       const int kc_in = a.k_cap ? a.k_cap[j] : a.k_max;
       __syncwarp(g.mask);
       const int rN = (int)((w >> 11) & 0x7FFu);
@@ -687,7 +707,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       }
       __syncwarp(g.mask);
       int K, N, nd;
-      RowPieces p = summarise_row(g, row, cur_row, K, N, nd, recw);
+      RowPieces p = summarise_row(g, row, cur, K, N, nd, recw);
       // per-row caps: replicas above the job's cap leave from the highest node index down, then
       // occupied nodes beyond n_max are cleared from the highest index down
       const int kc = max(0, min(kc_in, a.k_max));
@@ -708,7 +728,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
           }
         }
         __syncwarp(g.mask);
-        p = summarise_row(g, row, cur_row, K, N, nd, recw);
+        p = summarise_row(g, row, cur, K, N, nd, recw);
       }
       const uint32_t slot = s_base_mut + (uint32_t)i;
       store_row(g, a.st.pool + (size_t)slot * NN, row);
@@ -747,37 +767,43 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       }
     }
   };
-  for (int nb = warp * 32; nb < NN; nb += GEN_WARPS * 32) {
-    const int n = nb + lane;
-    const unsigned long long acc = (n < NN) ? s_node[n] : 0ull;
-    const int total = (int)(uint32_t)acc, nelig = (int)((acc >> 32) & 0xFFFFu), count = (int)(acc >> 48);
-    const int cp = (n < NN) ? (int)s_cap[n] : 0;
-    unsigned todo = __ballot_sync(0xffffffffu, n < NN && (nelig >= 2 || total > cp));
-    while (todo) {
-      const int srcl = __ffs(todo) - 1;
-      todo &= todo - 1;
-      const int nn = nb + srcl;
-      const int tot_n = __shfl_sync(0xffffffffu, total, srcl), ne_n = __shfl_sync(0xffffffffu, nelig, srcl);
-      const int cap_n = __shfl_sync(0xffffffffu, cp, srcl);
-      const int have_n = __shfl_sync(0xffffffffu, count, srcl);
-      if (have_n > OCC) {
-        if (lane == 0) { s_viol[nn] = 2; s_anyscan = 1; }
-        repair_column_scan<false>(a, c, s_slot, s_summ, nn, tot_n, ne_n, cap_n, lane, mark_row);
-      } else {
-        const uint32_t entry = (lane < have_n) ? s_occ[nn * OCC + lane] : 0u;
-        const int v_new = decide_entries(a, c, nn, tot_n, ne_n, cap_n, lane, entry, have_n);
-        if (lane < have_n) {
-          // the entry now carries the decision: GPUs kept, and bit 24 when that is a change
-          const bool changed = v_new != (int)((entry >> 13) & 0x7FFu);
-          s_occ[nn * OCC + lane] = (entry & 0x80001FFFu) | ((uint32_t)v_new << 13) | (changed ? (1u << 24) : 0u);
-          if (changed) mark_row((int)(entry & 0x1FFFu));
-        }
-        if (lane == 0) s_viol[nn] = 1;
-      }
-      __syncwarp();
-    }
+  // nodes that hold two distributed jobs or more GPUs than they have
+  for (int n = tid; n < NN; n += GEN_THREADS) {
+    const unsigned long long acc = s_node[n];
+    if ((int)((acc >> 32) & 0xFFFFu) >= 2 || (int)(uint32_t)acc > (int)s_cap[n]) s_viollist[atomicAdd(&s_nviol, 1)] = (uint16_t)n;
   }
   __syncthreads();
+  const int nviol = s_nviol;
+  for (int i = grp; i < nviol; i += GEN_GROUPS) {   // a group of 16 lanes per listed node
+    const int nn = (int)s_viollist[i];
+    const unsigned long long acc = s_node[nn];
+    const int have_n = (int)(acc >> 48);
+    if (have_n > OCC) {   // more occupants than the list holds: left to the column scan below
+      if (g.sub == 0) { s_viol[nn] = 2; s_anyscan = 1; }
+      continue;
+    }
+    const uint32_t entry = (g.sub < have_n) ? s_occ[nn * OCC + g.sub] : 0u;
+    const int v_new = decide_entries(a, g, c, nn, (int)(uint32_t)acc, (int)((acc >> 32) & 0xFFFFu), (int)s_cap[nn], entry, have_n);
+    if (g.sub < have_n) {
+      // the entry now carries the decision: GPUs kept, and bit 24 when that is a change
+      const bool changed = v_new != (int)((entry >> 13) & 0x7FFu);
+      s_occ[nn * OCC + g.sub] = (entry & 0x80001FFFu) | ((uint32_t)v_new << 13) | (changed ? (1u << 24) : 0u);
+      if (changed) mark_row((int)(entry & 0x1FFFu));
+    }
+    if (g.sub == 0) s_viol[nn] = 1;
+    __syncwarp(g.mask);
+  }
+  __syncthreads();
+  if (s_anyscan) {
+    for (int i = warp; i < nviol; i += GEN_WARPS) {   // a warp per node whose column must be scanned
+      const int nn = (int)s_viollist[i];
+      if (s_viol[nn] != 2) continue;
+      const unsigned long long acc = s_node[nn];
+      repair_column_scan<false>(a, c, s_slot, s_summ, nn, (int)(uint32_t)acc, (int)((acc >> 32) & 0xFFFFu), (int)s_cap[nn],
+                                lane, mark_row);
+    }
+    __syncthreads();
+  }
 
   // ---- rows the column pass changes -----------------------------------------------------------
   // Usual case (every violating node's occupants were listed): one group per changed row takes
@@ -800,6 +826,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         const bool own = (s_mark[j] & 2) != 0;
         const uint32_t src = s_slot[j];
         load_row<true>(g, row, a.st.pool + (size_t)src * NN);   // may have been written in this kernel
+        const CurPieces cur = cur_pieces(g, a.cur ? a.cur + (size_t)j * NN : nullptr);
         __syncwarp(g.mask);
         {
           const RowPieces p = row_pieces(g, row);
@@ -823,7 +850,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         }
         __syncwarp(g.mask);
         int K, N, nd;
-        summarise_row(g, row, a.cur ? a.cur + (size_t)j * NN : nullptr, K, N, nd, recw);
+        summarise_row(g, row, cur, K, N, nd, recw);
         const uint32_t dst = own ? src : s_base_cow + (uint32_t)i;
         store_row(g, a.st.pool + (size_t)dst * NN, row);
         const uint32_t word = pack_summary(K, N, nd);
@@ -893,9 +920,10 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         const int j = (int)s_mod[i];
         const uint32_t slot = s_slot[j];
         load_row<true>(g, row, a.st.pool + (size_t)slot * NN);   // written in this kernel: read through to L2
+        const CurPieces cur = cur_pieces(g, a.cur ? a.cur + (size_t)j * NN : nullptr);
         __syncwarp(g.mask);
         int K, N, nd;
-        summarise_row(g, row, a.cur ? a.cur + (size_t)j * NN : nullptr, K, N, nd, recw);
+        summarise_row(g, row, cur, K, N, nd, recw);
         const uint32_t word = pack_summary(K, N, nd);
         if (g.sub == 0) {
           recw[REC_SUMM] = word;
