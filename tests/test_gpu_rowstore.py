@@ -25,6 +25,12 @@ CASES = [
                  init_prob=0.9, with_history=True, random_cur=False),
     # no current allocation, inactive jobs, ragged job count
     synth.Config("store-plain", 16, 8, 257, 14, 16, 8, 20, 6, num_elite=1, mutate_prob=0.1),
+    # the widest rows the store takes (512 nodes: four 16-byte pieces per lane of a row's group)
+    synth.Config("store-512-nodes", 512, 2, 600, 15, 16, 8, 12, 10, num_elite=2, mutate_prob=0.2,
+                 init_prob=0.3, with_history=True, random_cur=True),
+    # rows whose pieces do not fill the lanes evenly (17 pieces), many jobs per candidate
+    synth.Config("store-ragged-pieces", 136, 4, 1100, 16, 16, 8, 10, 8, num_elite=1, mutate_prob=0.15,
+                 init_prob=0.3, with_history=True, random_cur=True),
 ]
 
 
