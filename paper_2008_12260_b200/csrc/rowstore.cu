@@ -6,8 +6,8 @@
 // a 32-byte record: up to six occupied nodes, the row's summary (K, N, entries that differ
 // from the current allocation) and its term of the fitness sum (a stored row always serves
 // the same job, so the term is fixed for the round).  A generation reads 36 bytes per
-// unchanged row instead of the row, and writes 4.  New rows are appended to the pool (copy on write); when a half of the pool
-// runs low the live rows are copied to the other half.
+// unchanged row instead of the row, and writes 4.  New rows are appended to the pool (copy
+// on write); when a half of the pool runs low the live rows are copied to the other half.
 //
 // One block evolves one candidate per generation: parent selection, row-wise crossover,
 // perturbation, per-row caps, interference and capacity repair, and the candidate's fitness.

@@ -2,6 +2,8 @@
 into a row pool, copy on write).  Such a round must equal, bit for bit, the same round made
 of the dense entry points called one by one, which the other tests pin to the oracle; the
 last generation is also checked against the oracle directly (teacher-forced)."""
+import dataclasses
+
 import numpy as np
 import pytest
 
@@ -31,6 +33,8 @@ CASES = [
     # rows whose pieces do not fill the lanes evenly (17 pieces), many jobs per candidate
     synth.Config("store-ragged-pieces", 136, 4, 1100, 16, 16, 8, 10, 8, num_elite=1, mutate_prob=0.15,
                  init_prob=0.3, with_history=True, random_cur=True),
+    # the large workload itself (the configuration the benchmark times), ten generations
+    dataclasses.replace(synth.LARGE, name="store-large", generations=10),
 ]
 
 
