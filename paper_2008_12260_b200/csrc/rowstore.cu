@@ -59,16 +59,15 @@ __device__ __forceinline__ int piece_diff(uint4 x, uint4 c) {   // entries that 
 }
 
 // Rows are worked on by groups of 16 lanes (two rows per warp at a time).  A lane looks after
-// the ROW_PPL-or-fewer consecutive pieces [sub * ppl, sub * ppl + ppl) of its group's row, so
-// lane order is node order.
+// the PPL consecutive pieces [sub * PPL, sub * PPL + PPL) of its group's row, so lane order is
+// node order.  PPL (1, 2 or 4: rows have at most 64 pieces) is a template parameter of
+// everything that walks a row, so that short rows do not pay for the pieces they lack.
 constexpr int GROUP = 16;
-constexpr int ROW_PPL = 4;   // rows have at most 64 pieces
 
 struct Grp {
   int sub;         // lane within the group
   unsigned mask;   // the group's lanes
   int row_vecs;    // pieces of a row
-  int ppl;         // pieces per lane
 };
 
 __device__ __forceinline__ Grp make_group(int lane, int NN) {
@@ -76,7 +75,6 @@ __device__ __forceinline__ Grp make_group(int lane, int NN) {
   g.sub = lane & (GROUP - 1);
   g.mask = 0xFFFFu << (lane & GROUP);
   g.row_vecs = NN >> 3;
-  g.ppl = (g.row_vecs + GROUP - 1) / GROUP;
   return g;
 }
 
@@ -109,20 +107,22 @@ __device__ __forceinline__ void store_row(const Grp &g, int16_t *dst, const int1
 
 // This lane's pieces of a row in shared memory, their occupancy masks, and where the lane's
 // occupants come in node order: `first` = occupants in lower lanes, `total` = the row's N.
+template <int PPL>
 struct RowPieces {
-  uint4 x[ROW_PPL];
-  uint32_t mask[ROW_PPL];
+  uint4 x[PPL];
+  uint32_t mask[PPL];
   int first, total;
 };
 
-__device__ __forceinline__ RowPieces row_pieces(const Grp &g, const int16_t *row) {
-  RowPieces p;
+template <int PPL>
+__device__ __forceinline__ RowPieces<PPL> row_pieces(const Grp &g, const int16_t *row) {
+  RowPieces<PPL> p;
   int cnt = 0;
 #pragma unroll
-  for (int q = 0; q < ROW_PPL; ++q) {
-    const int v = g.sub * g.ppl + q;
+  for (int q = 0; q < PPL; ++q) {
+    const int v = g.sub * PPL + q;
     p.x[q] = make_uint4(0u, 0u, 0u, 0u);
-    if (q < g.ppl && v < g.row_vecs) p.x[q] = ((const uint4 *)row)[v];
+    if (v < g.row_vecs) p.x[q] = ((const uint4 *)row)[v];
     p.mask[q] = piece_mask(p.x[q]);
     cnt += __popc(p.mask[q]);
   }
@@ -141,33 +141,36 @@ __device__ __forceinline__ RowPieces row_pieces(const Grp &g, const int16_t *row
 // occupant entries of a row held in shared memory.  All lanes of the group
 // return the same K, N, ndiff; rec_out (shared, REC_WORDS: the entries, the other words are the
 // caller's) is complete after the trailing __syncwarp(group).
+template <int PPL>
 struct CurPieces {
-  uint4 x[ROW_PPL];
+  uint4 x[PPL];
   bool have;
 };
 
 // this lane's pieces of the current allocation's row (NULL: none), fetched ahead of their use
-__device__ __forceinline__ CurPieces cur_pieces(const Grp &g, const int16_t *cur_row) {
-  CurPieces c;
+template <int PPL>
+__device__ __forceinline__ CurPieces<PPL> cur_pieces(const Grp &g, const int16_t *cur_row) {
+  CurPieces<PPL> c;
   c.have = cur_row != nullptr;
 #pragma unroll
-  for (int q = 0; q < ROW_PPL; ++q) {
-    const int v = g.sub * g.ppl + q;
+  for (int q = 0; q < PPL; ++q) {
+    const int v = g.sub * PPL + q;
     c.x[q] = make_uint4(0u, 0u, 0u, 0u);
-    if (c.have && q < g.ppl && v < g.row_vecs) c.x[q] = load_piece<false>(cur_row, v);
+    if (c.have && v < g.row_vecs) c.x[q] = load_piece<false>(cur_row, v);
   }
   return c;
 }
 
-__device__ __forceinline__ RowPieces summarise_row(const Grp &g, const int16_t *row, const CurPieces &cur,
-                                                   int &K, int &N, int &ndiff, uint32_t *rec_out) {
-  const RowPieces p = row_pieces(g, row);
+template <int PPL>
+__device__ __forceinline__ RowPieces<PPL> summarise_row(const Grp &g, const int16_t *row, const CurPieces<PPL> &cur,
+                                                        int &K, int &N, int &ndiff, uint32_t *rec_out) {
+  const RowPieces<PPL> p = row_pieces<PPL>(g, row);
   int k = 0, nd = 0, pos = p.first;
 #pragma unroll
-  for (int q = 0; q < ROW_PPL; ++q) {
-    const int v = g.sub * g.ppl + q;
+  for (int q = 0; q < PPL; ++q) {
+    const int v = g.sub * PPL + q;
     k += piece_sum(p.x[q]);
-    if (cur.have && q < g.ppl && v < g.row_vecs) nd += piece_diff(p.x[q], cur.x[q]);
+    if (cur.have && v < g.row_vecs) nd += piece_diff(p.x[q], cur.x[q]);
     uint32_t m = p.mask[q];
     while (m && pos < REC_ENTRIES) {
       const int h = __ffs(m) - 1;
@@ -189,14 +192,15 @@ __device__ __forceinline__ RowPieces summarise_row(const Grp &g, const int16_t *
 }
 
 // node index of the t-th occupied entry (ascending) of a row held in shared memory; t < N
+template <int PPL>
 __device__ __forceinline__ int nth_occupied_row(const Grp &g, const int16_t *row, uint32_t t) {
-  const RowPieces p = row_pieces(g, row);
+  const RowPieces<PPL> p = row_pieces<PPL>(g, row);
   int node = -1, before = p.first;
 #pragma unroll
-  for (int q = 0; q < ROW_PPL; ++q) {
+  for (int q = 0; q < PPL; ++q) {
     const int c = __popc(p.mask[q]);
     if ((int)t >= before && (int)t < before + c)
-      node = 8 * (g.sub * g.ppl + q) + (int)__fns(p.mask[q], 0, (int)t - before + 1);
+      node = 8 * (g.sub * PPL + q) + (int)__fns(p.mask[q], 0, (int)t - before + 1);
     before += c;
   }
   const unsigned who = __ballot_sync(g.mask, node >= 0);
@@ -230,6 +234,7 @@ struct BuildArgs {
   int P, J, NN;
 };
 
+template <int PPL>
 __global__ void __launch_bounds__(256) rowstore_build_kernel(BuildArgs a) {
   __shared__ __align__(16) int16_t s_row[16][512];
   __shared__ uint32_t s_rec[16][REC_WORDS];
@@ -248,10 +253,10 @@ __global__ void __launch_bounds__(256) rowstore_build_kernel(BuildArgs a) {
   for (long long r = (long long)blockIdx.x * 16 + grp; r < rows; r += (long long)gridDim.x * 16) {
     const int j = (int)(r % a.J);
     load_row<false>(g, s_row[grp], a.st.pool + (size_t)r * a.NN);
-    const CurPieces cur = cur_pieces(g, a.cur ? a.cur + (size_t)j * a.NN : nullptr);
+    const CurPieces<PPL> cur = cur_pieces<PPL>(g, a.cur ? a.cur + (size_t)j * a.NN : nullptr);
     __syncwarp(g.mask);
     int K, N, nd;
-    summarise_row(g, s_row[grp], cur, K, N, nd, s_rec[grp]);
+    summarise_row<PPL>(g, s_row[grp], cur, K, N, nd, s_rec[grp]);
     const bool on = !a.active || a.active[j];
     if (g.sub == 0) {
       s_rec[grp][REC_SUMM] = on ? pack_summary(K, N, nd) : 0u;
@@ -492,6 +497,7 @@ __device__ void repair_column_scan(const GenArgs &a, uint32_t c, const uint32_t 
   }
 }
 
+template <int PPL>
 __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArgs a) {
   extern __shared__ __align__(16) unsigned char smem[];
   const int J = a.J, NN = a.NN, P = a.P;
@@ -593,14 +599,14 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   };
 
   // the occupants in this lane's pieces of a row
-  auto add_row_occupants = [&](const Grp &g, int j, const RowPieces &p, bool dist) {
+  auto add_row_occupants = [&](const Grp &g, int j, const RowPieces<PPL> &p, bool dist) {
 #pragma unroll
-    for (int q = 0; q < ROW_PPL; ++q) {
+    for (int q = 0; q < PPL; ++q) {
       uint32_t m = p.mask[q];
       while (m) {
         const int h = __ffs(m) - 1;
         m &= m - 1;
-        add_occupant(j, 8 * (g.sub * g.ppl + q) + h, piece_entry(p.x[q], h), dist);
+        add_occupant(j, 8 * (g.sub * PPL + q) + h, piece_entry(p.x[q], h), dist);
       }
     }
   };
@@ -684,7 +690,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       const int j = (int)s_mut[i];
       const uint32_t old = s_slot[j], w = s_summ[j];
       load_row<false>(g, row, a.st.pool + (size_t)old * NN);
-      const CurPieces cur = cur_pieces(g, a.cur ? a.cur + (size_t)j * NN : nullptr);
+      const CurPieces<PPL> cur = cur_pieces<PPL>(g, a.cur ? a.cur + (size_t)j * NN : nullptr);
       const int kc_in = a.k_cap ? a.k_cap[j] : a.k_max;
       __syncwarp(g.mask);
       const int rN = (int)((w >> 11) & 0x7FFu);
@@ -694,7 +700,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         const int n = (int)bounded(mw.w, (uint32_t)NN);
         if (g.sub == 0) row[n] = (int16_t)min((int)row[n] + 1, (int)s_cap[n]);
       } else if (rN > 0) {
-        const int ns = nth_occupied_row(g, row, bounded(mw.z, (uint32_t)rN));
+        const int ns = nth_occupied_row<PPL>(g, row, bounded(mw.z, (uint32_t)rN));
         if (op == 1u) {
           if (g.sub == 0) row[ns] = (int16_t)(row[ns] - 1);
         } else {
@@ -707,7 +713,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       }
       __syncwarp(g.mask);
       int K, N, nd;
-      RowPieces p = summarise_row(g, row, cur, K, N, nd, recw);
+      RowPieces<PPL> p = summarise_row<PPL>(g, row, cur, K, N, nd, recw);
       // per-row caps: replicas above the job's cap leave from the highest node index down, then
       // occupied nodes beyond n_max are cleared from the highest index down
       const int kc = max(0, min(kc_in, a.k_max));
@@ -728,7 +734,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
           }
         }
         __syncwarp(g.mask);
-        p = summarise_row(g, row, cur, K, N, nd, recw);
+        p = summarise_row<PPL>(g, row, cur, K, N, nd, recw);
       }
       const uint32_t slot = s_base_mut + (uint32_t)i;
       store_row(g, a.st.pool + (size_t)slot * NN, row);
@@ -751,7 +757,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
     const int j = (int)s_ovf[i];
     load_row<false>(g, row, a.st.pool + (size_t)s_slot[j] * NN);
     __syncwarp(g.mask);
-    const RowPieces p = row_pieces(g, row);
+    const RowPieces<PPL> p = row_pieces<PPL>(g, row);
     add_row_occupants(g, j, p, ((s_summ[j] >> 11) & 0x7FFu) >= 2u);
     __syncwarp(g.mask);
   }
@@ -826,15 +832,15 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         const bool own = (s_mark[j] & 2) != 0;
         const uint32_t src = s_slot[j];
         load_row<true>(g, row, a.st.pool + (size_t)src * NN);   // may have been written in this kernel
-        const CurPieces cur = cur_pieces(g, a.cur ? a.cur + (size_t)j * NN : nullptr);
+        const CurPieces<PPL> cur = cur_pieces<PPL>(g, a.cur ? a.cur + (size_t)j * NN : nullptr);
         __syncwarp(g.mask);
         {
-          const RowPieces p = row_pieces(g, row);
+          const RowPieces<PPL> p = row_pieces<PPL>(g, row);
 #pragma unroll
-          for (int q = 0; q < ROW_PPL; ++q) {
+          for (int q = 0; q < PPL; ++q) {
             uint32_t m = p.mask[q];
             while (m) {
-              const int n = 8 * (g.sub * g.ppl + q) + __ffs(m) - 1;
+              const int n = 8 * (g.sub * PPL + q) + __ffs(m) - 1;
               m &= m - 1;
               if (s_viol[n] != 1) continue;
               const int cnt = (int)(s_node[n] >> 48);
@@ -850,7 +856,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         }
         __syncwarp(g.mask);
         int K, N, nd;
-        summarise_row(g, row, cur, K, N, nd, recw);
+        summarise_row<PPL>(g, row, cur, K, N, nd, recw);
         const uint32_t dst = own ? src : s_base_cow + (uint32_t)i;
         store_row(g, a.st.pool + (size_t)dst * NN, row);
         const uint32_t word = pack_summary(K, N, nd);
@@ -920,10 +926,10 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         const int j = (int)s_mod[i];
         const uint32_t slot = s_slot[j];
         load_row<true>(g, row, a.st.pool + (size_t)slot * NN);   // written in this kernel: read through to L2
-        const CurPieces cur = cur_pieces(g, a.cur ? a.cur + (size_t)j * NN : nullptr);
+        const CurPieces<PPL> cur = cur_pieces<PPL>(g, a.cur ? a.cur + (size_t)j * NN : nullptr);
         __syncwarp(g.mask);
         int K, N, nd;
-        summarise_row(g, row, cur, K, N, nd, recw);
+        summarise_row<PPL>(g, row, cur, K, N, nd, recw);
         const uint32_t word = pack_summary(K, N, nd);
         if (g.sub == 0) {
           recw[REC_SUMM] = word;
@@ -981,6 +987,12 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   if (tid == 0) a.fitness_out[c] = fitness_finalise(a.tp.mode, a.tp.p, ts, ns);
 }
 
+// pieces per lane of a row's group: 1, 2 or 4 (a lane's pieces beyond the row's end are empty)
+int store_pieces_per_lane(int num_nodes) {
+  const int need = ((num_nodes >> 3) + GROUP - 1) / GROUP;
+  return need <= 1 ? 1 : need == 2 ? 2 : 4;
+}
+
 StoreView store_view(const sched_ctx *ctx) {
   StoreView v;
   v.pool = ctx->rs_pool; v.rec = ctx->rs_rec;
@@ -1031,7 +1043,9 @@ int rowstore_ensure(sched_ctx *ctx) {
   if (e == cudaSuccess) {
     const size_t smem = gen_smem_layout(c.num_jobs, c.num_nodes).total;
     if (smem > 48 * 1024)
-      e = cudaFuncSetAttribute(generation_store_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    for (int k = 0; k < 3 && e == cudaSuccess; ++k)
+      e = cudaFuncSetAttribute(k == 0 ? generation_store_kernel<1> : k == 1 ? generation_store_kernel<2> : generation_store_kernel<4>,
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   }
   if (e != cudaSuccess) {
     set_error(ctx, "row store allocation failed: %s", cudaGetErrorString(e));
@@ -1059,7 +1073,10 @@ int rowstore_build(sched_ctx *ctx, const uint8_t *d_active, const int16_t *d_cur
   a.P = c.population; a.J = c.num_jobs; a.NN = c.num_nodes;
   {
     TimedLaunch tl_(ctx, KK_STORE_BUILD);
-    rowstore_build_kernel<<<ctx->num_sms * 8, 256, 0, ctx->stream>>>(a);
+    const int ppl = store_pieces_per_lane(c.num_nodes);
+    if (ppl == 1) rowstore_build_kernel<1><<<ctx->num_sms * 8, 256, 0, ctx->stream>>>(a);
+    else if (ppl == 2) rowstore_build_kernel<2><<<ctx->num_sms * 8, 256, 0, ctx->stream>>>(a);
+    else rowstore_build_kernel<4><<<ctx->num_sms * 8, 256, 0, ctx->stream>>>(a);
   }
   SCHED_LAUNCH_CHECK(ctx);
   return SCHED_OK;
@@ -1124,7 +1141,10 @@ int rowstore_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d
   const size_t smem = gen_smem_layout(c.num_jobs, c.num_nodes).total;
   {
     TimedLaunch tl_(ctx, KK_GENSTORE);
-    generation_store_kernel<<<c.population, GEN_THREADS, smem, ctx->stream>>>(a);
+    const int ppl = store_pieces_per_lane(c.num_nodes);
+    if (ppl == 1) generation_store_kernel<1><<<c.population, GEN_THREADS, smem, ctx->stream>>>(a);
+    else if (ppl == 2) generation_store_kernel<2><<<c.population, GEN_THREADS, smem, ctx->stream>>>(a);
+    else generation_store_kernel<4><<<c.population, GEN_THREADS, smem, ctx->stream>>>(a);
   }
   SCHED_LAUNCH_CHECK(ctx);
   return SCHED_OK;
