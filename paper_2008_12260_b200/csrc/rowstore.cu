@@ -38,8 +38,11 @@ struct StoreView {
 
 // ---- a row as 16-byte pieces of 8 entries (entries of stored rows are in [0, 2047]) -----------
 __device__ __forceinline__ uint32_t piece_mask(uint4 x) {   // bit h: entry h of the piece is occupied
-  return ((x.x & 0xFFFFu) ? 1u : 0u) | ((x.x >> 16) ? 2u : 0u) | ((x.y & 0xFFFFu) ? 4u : 0u) | ((x.y >> 16) ? 8u : 0u) |
-         ((x.z & 0xFFFFu) ? 16u : 0u) | ((x.z >> 16) ? 32u : 0u) | ((x.w & 0xFFFFu) ? 64u : 0u) | ((x.w >> 16) ? 128u : 0u);
+  // per word: min(half, 1) for both halves (entries are non-negative), folded to two bits
+  const uint32_t a = __vimin_s16x2_relu(x.x, 0x00010001u), b = __vimin_s16x2_relu(x.y, 0x00010001u);
+  const uint32_t c = __vimin_s16x2_relu(x.z, 0x00010001u), d = __vimin_s16x2_relu(x.w, 0x00010001u);
+  const uint32_t lo = a | (b << 2) | (c << 4) | (d << 6);   // bits 0,2,4,6: low halves; 16,18,20,22: high halves
+  return (lo | (lo >> 15)) & 0xFFu;
 }
 __device__ __forceinline__ int piece_sum(uint4 x) {
   int k = __dp2a_lo((int)x.x, 0x0101, 0);
