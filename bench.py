@@ -45,9 +45,9 @@ HBM_FALLBACK_GBS = 6650.0
 # "rows": one dense large-workload generation (237.1 MB read + 257.1 MB written).
 # "fitness_stress": 16 dense stress candidates moved 544.8 + 3.0 MB; every candidate is streamed
 # once, so the figure is scaled by candidates / 16 to the chunk that is timed (544.8 + 3.5 MB).
-# "generation_store": one row-store generation of the large workload (13.3 MB read in generation 8;
+# "generation_store": one row-store generation of the large workload (12.7 MB read in generation 9;
 # generations 2..12 of a round read 19.5 .. 11.5 MB as L2 warms up).
-NCU_TRAFFIC_BYTES = {"rows": 494.2e6, "fitness_stress_per_candidate": 548.3e6 / 16, "generation_store": 13.3e6}
+NCU_TRAFFIC_BYTES = {"rows": 494.2e6, "fitness_stress_per_candidate": 548.3e6 / 16, "generation_store": 12.7e6}
 
 
 def measured_peaks():
