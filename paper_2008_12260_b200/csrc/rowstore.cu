@@ -140,10 +140,7 @@ __device__ __forceinline__ RowPieces<PPL> row_pieces(const Grp &g, const int16_t
   return p;
 }
 
-// K, N, entries differing from the current allocation's row (`cur`: its pieces, if any) and the
-// occupant entries of a row held in shared memory.  All lanes of the group
-// return the same K, N, ndiff; rec_out (shared, REC_WORDS: the entries, the other words are the
-// caller's) is complete after the trailing __syncwarp(group).
+// this lane's pieces of the matching row of the current allocation, if there is one
 template <int PPL>
 struct CurPieces {
   uint4 x[PPL];
@@ -164,6 +161,10 @@ __device__ __forceinline__ CurPieces<PPL> cur_pieces(const Grp &g, const int16_t
   return c;
 }
 
+// K, N, entries differing from the current allocation's row (`cur`: its pieces, if any) and the
+// occupant entries of a row held in shared memory.  All lanes of the group return the same K, N,
+// ndiff; rec_out (shared, REC_WORDS: the entries, the other words are the caller's) is complete
+// after the trailing __syncwarp(group).
 template <int PPL>
 __device__ __forceinline__ RowPieces<PPL> summarise_row(const Grp &g, const int16_t *row, const CurPieces<PPL> &cur,
                                                         int &K, int &N, int &ndiff, uint32_t *rec_out) {
