@@ -251,7 +251,12 @@ def run_ours(args):
                     "algorithmic_bytes_per_launch": dom["algorithmic_bytes"], "avg_launch_us": dom["avg_us"],
                     "note": "one block evolves one candidate per launch on L2-resident records: latency- and "
                             "issue-bound, not DRAM-bound (the dense operator kernel, which is, is reported under "
-                            "dense_generation)" if dom["kernel"] == "generation_store" else None}
+                            "dense_generation)" if dom["kernel"] == "generation_store" else None,
+                    # from the committed ncu summary of this kernel (not measured in this run)
+                    "ncu_counters": {"issue_active_pct": 34.7, "dram_pct_of_peak": 3.8, "l2_hit_pct": 48.2,
+                                     "warp_instructions": 12.6e6, "stall_barrier_per_issue": 4.2,
+                                     "stall_long_scoreboard_per_issue": 4.5}
+                    if dom["kernel"] == "generation_store" else None}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
