@@ -918,6 +918,281 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
   }
 }
 
+// ---------------------------------------------------------------------------------------
+// Small problems (at most 256 jobs, at most 32 nodes): one block per candidate, one THREAD
+// per row.  A row is 16 to 64 bytes, so a thread reads its parent's row with one to four
+// vector loads, keeps it in its own line of shared memory, perturbs and caps it there, and
+// adds its occupants to per-node lists; warps then repair the violating nodes from the
+// lists (or from the rows in shared memory when a list overflows), the threads write their
+// rows out and the block sums the fitness.  Same operators, draws and sums as the kernels
+// above: identical populations and fitness bits, with far fewer dependent steps.
+// ---------------------------------------------------------------------------------------
+constexpr int SMALL_MAX_NODES = 32;
+constexpr int SMALL_OCC = 32;   // occupants listed per node: one lane each in the repair
+
+__global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
+  const RowsArgs &a = aa.r;
+  __shared__ __align__(16) int16_t s_rows[256][SMALL_MAX_NODES];   // child rows, a line per job
+  __shared__ __align__(16) int16_t s_cap[SMALL_MAX_NODES];
+  __shared__ uint32_t s_tot[SMALL_MAX_NODES], s_cnt[SMALL_MAX_NODES];  // GPUs placed; distributed jobs | occupants << 16
+  __shared__ uint32_t s_occ[SMALL_MAX_NODES][SMALL_OCC];               // job | GPUs << 13 | distributed << 31
+  __shared__ uint32_t s_summ[256];
+  __shared__ uint8_t s_dirty[256];
+  __shared__ float s_term[256];
+  __shared__ int s_parent[2], s_rank4[4];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int cl = blockIdx.x;
+  const uint32_t c = a.first_cand + (uint32_t)cl;
+  const int NN = a.num_nodes, J = a.J, P = a.P;
+  const int row_vecs = NN >> 3;
+  const bool elite = (int)c < a.num_elite;
+
+  if (tid < NN) {
+    s_cap[tid] = (int16_t)max((int)a.cap[tid], 0);
+    s_tot[tid] = 0u;
+    s_cnt[tid] = 0u;
+  }
+  // ---- parents (rank = candidates ordered before, fitness descending, index ascending) --------
+  if (elite) {
+    for (int i = tid; i < P; i += blockDim.x) {
+      const uint32_t ki = order_key(a.fitness_bits[i]);
+      int rk = 0;
+      for (int o = 0; o < P; ++o) {
+        const uint32_t ko = order_key(__ldg(a.fitness_bits + o));
+        rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
+      }
+      if (rk == (int)c) s_parent[0] = s_parent[1] = i;
+    }
+  } else {
+    const u32x4 sel = draw(a.key, 0u, c, a.gen, SLOT_SELECT);
+    const int idx[4] = {(int)bounded(sel.x, P), (int)bounded(sel.y, P), (int)bounded(sel.z, P), (int)bounded(sel.w, P)};
+    if (warp < 4) {
+      const int i = idx[warp];
+      const uint32_t ki = order_key(a.fitness_bits[i]);
+      int rk = 0;
+      for (int o = lane; o < P; o += 32) {
+        const uint32_t ko = order_key(__ldg(a.fitness_bits + o));
+        rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
+      }
+      rk = warp_sum(rk);
+      if (lane == 0) s_rank4[warp] = rk;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      s_parent[0] = s_rank4[0] <= s_rank4[1] ? idx[0] : idx[1];
+      s_parent[1] = s_rank4[2] <= s_rank4[3] ? idx[2] : idx[3];
+    }
+  }
+  __syncthreads();
+
+  // ---- rows: thread j builds row j of the child ----------------------------------------------
+  const int j = tid;
+  int16_t *row = s_rows[tid];
+  int K = 0, N = 0, ndiff = 0;
+  bool on = false;
+  if (j < J) {
+    on = !a.active || a.active[j];
+    bool second = false, mut = false;
+    u32x4 mw = {0, 0, 0, 0};
+    if (on && !elite) {
+      second = (draw(a.key, (uint32_t)j, c, a.gen, SLOT_XOVER).x >> 31) != 0u;
+      mw = draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE);
+      mut = mw.x < a.thr;
+    }
+    const uint4 *src = (const uint4 *)(a.src + ((size_t)s_parent[second ? 1 : 0] * J + j) * NN);
+    uint4 cur4[SMALL_MAX_NODES / 8];
+#pragma unroll
+    for (int v = 0; v < SMALL_MAX_NODES / 8; ++v) {
+      uint4 x = make_uint4(0u, 0u, 0u, 0u);
+      cur4[v] = make_uint4(0u, 0u, 0u, 0u);
+      if (v < row_vecs) {
+        if (on) x = clamp_vec(__ldg(src + v), ((const uint4 *)s_cap)[v]);   // entries into [0, node size]
+        if (a.cur) cur4[v] = __ldg((const uint4 *)(a.cur + (size_t)j * NN) + v);
+        ((uint4 *)row)[v] = x;
+      }
+    }
+    if (on) {
+      for (int n = 0; n < NN; ++n) { K += row[n]; N += row[n] > 0; }
+      if (mut) {
+        const uint32_t op = bounded(mw.y, 3u);
+        if (op == 0u) {
+          const int n = (int)bounded(mw.w, (uint32_t)NN);
+          row[n] = (int16_t)min((int)row[n] + 1, (int)s_cap[n]);
+        } else if (N > 0) {
+          int t = (int)bounded(mw.z, (uint32_t)N), ns = 0;
+          for (int n = 0; n < NN; ++n) {
+            if (row[n] > 0 && t-- == 0) { ns = n; break; }
+          }
+          if (op == 1u) {
+            row[ns] = (int16_t)(row[ns] - 1);
+          } else {
+            const int nd = (int)bounded(mw.w, (uint32_t)NN);
+            if (nd != ns) {
+              row[nd] = (int16_t)min((int)row[nd] + (int)row[ns], (int)s_cap[nd]);
+              row[ns] = 0;
+            }
+          }
+        }
+        K = 0; N = 0;
+        for (int n = 0; n < NN; ++n) { K += row[n]; N += row[n] > 0; }
+      }
+      // per-row caps: replicas above the job's cap leave from the highest node index down, then
+      // occupied nodes beyond n_max are cleared from the highest index down
+      int kc = a.k_cap ? a.k_cap[j] : a.k_max;
+      kc = max(0, min(kc, a.k_max));
+      if (K > kc || N > a.n_max) {
+        int excess = K - kc;
+        for (int n = NN - 1; n >= 0 && excess > 0; --n) {
+          const int take = min((int)row[n], excess);
+          row[n] = (int16_t)(row[n] - take);
+          excess -= take;
+        }
+        int occ = 0;
+        K = 0;
+        for (int n = 0; n < NN; ++n) {
+          if (row[n] > 0) {
+            ++occ;
+            if (occ > a.n_max) row[n] = 0;
+          }
+          K += row[n];
+        }
+        N = min(occ, a.n_max);
+      }
+      // occupants into the nodes' totals and lists; entries differing from the current allocation
+      const bool dist = N >= 2;
+      for (int n = 0; n < NN; ++n) {
+        const int v = row[n];
+        if (a.cur) ndiff += (v != (int)((const int16_t *)cur4)[n]) ? 1 : 0;
+        if (v > 0) {
+          atomicAdd(&s_tot[n], (uint32_t)v);
+          const uint32_t k = atomicAdd(&s_cnt[n], (dist ? 1u : 0u) | (1u << 16)) >> 16;
+          if (k < SMALL_OCC) s_occ[n][k] = (uint32_t)j | ((uint32_t)v << 13) | (dist ? 0x80000000u : 0u);
+        }
+      }
+    }
+    s_summ[j] = on ? ((uint32_t)K | ((uint32_t)N << 11) | ((uint32_t)ndiff << 22)) : 0u;
+    s_dirty[j] = 0;
+  }
+  __syncthreads();
+
+  // ---- repair, a warp per violating node -------------------------------------------------------
+  for (int nn = warp; nn < NN; nn += 8) {
+    int tot = (int)s_tot[nn];
+    const int ne = (int)(s_cnt[nn] & 0xFFFFu), have_n = (int)(s_cnt[nn] >> 16), cap_n = (int)s_cap[nn];
+    if (ne < 2 && tot <= cap_n) continue;
+    if (have_n <= SMALL_OCC) {
+      // one occupant per lane
+      const bool have = lane < have_n;
+      const uint32_t entry = have ? s_occ[nn][lane] : 0u;
+      const int jj = (int)(entry & 0x1FFFu);
+      const int v_old = have ? (int)((entry >> 13) & 0x7FFu) : 0;
+      int v = v_old;
+      const bool dist = have && (entry >> 31);
+      if (ne >= 2) {
+        const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
+        int t = J;
+        if (dist && v > 0) { t = jj - o; if (t < 0) t += J; }
+        int best = t;
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, off));
+        int removed = 0;
+        if (dist && v > 0 && t != best) { removed = v; v = 0; }
+        tot -= warp_sum(removed);
+      }
+      const int excess = tot - cap_n;
+      if (excess > 0) {
+        const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J);
+        int rot = 0x7fffffff;
+        if (have) { rot = jj - o; if (rot < 0) rot += J; }
+        int ahead = 0;                       // GPUs of the occupants that come first in rotated order
+        for (int k = 0; k < have_n; ++k) {
+          const int rk = __shfl_sync(0xffffffffu, rot, k);
+          const int vk = __shfl_sync(0xffffffffu, v, k);
+          if (rk < rot) ahead += vk;
+        }
+        if (have) v -= min(v, max(excess - ahead, 0));
+      }
+      if (have && v != v_old) {
+        s_rows[jj][nn] = (int16_t)v;
+        s_dirty[jj] = 1;
+      }
+    } else {
+      // more occupants than the list holds: the column of the rows in shared memory
+      int keep = -1;
+      const bool intf = ne >= 2;
+      if (intf) {
+        const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
+        int best = J;
+        for (int jj = lane; jj < J; jj += 32) {
+          if (s_rows[jj][nn] > 0 && ((s_summ[jj] >> 11) & 0x7FFu) >= 2u) {
+            int t = jj - o;
+            if (t < 0) t += J;
+            best = min(best, t);
+          }
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, off));
+        keep = o + best;
+        if (keep >= J) keep -= J;
+        int removed = 0;
+        for (int jj = lane; jj < J; jj += 32) {
+          const int v = s_rows[jj][nn];
+          if (v > 0 && ((s_summ[jj] >> 11) & 0x7FFu) >= 2u && jj != keep) removed += v;
+        }
+        tot -= warp_sum(removed);
+      }
+      int excess = tot - cap_n;
+      const int o = (excess > 0) ? (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J) : 0;
+      for (int t0 = 0; t0 < J; t0 += 32) {
+        const int t = t0 + lane;
+        int jj = o + t;
+        if (jj >= J) jj -= J;
+        int v_old = 0, v_eff = 0;
+        if (t < J) {
+          v_old = s_rows[jj][nn];
+          const bool dist = ((s_summ[jj] >> 11) & 0x7FFu) >= 2u;
+          v_eff = (intf && dist && v_old > 0 && jj != keep) ? 0 : v_old;
+        }
+        int sfx = v_eff;                              // inclusive prefix over the 32 jobs
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const int u = __shfl_up_sync(0xffffffffu, sfx, off);
+          if (lane >= off) sfx += u;
+        }
+        const int take = (excess > 0) ? min(v_eff, max(excess - (sfx - v_eff), 0)) : 0;
+        const int v_new = v_eff - take;
+        if (t < J && v_new != v_old) {
+          s_rows[jj][nn] = (int16_t)v_new;
+          s_dirty[jj] = 1;
+        }
+        excess -= __shfl_sync(0xffffffffu, sfx, 31);
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---- rows out, fitness -----------------------------------------------------------------------
+  if (j < J) {
+    if (s_dirty[j]) {
+      K = 0; N = 0; ndiff = 0;
+      const int16_t *cur_row = a.cur ? a.cur + (size_t)j * NN : nullptr;
+      for (int n = 0; n < NN; ++n) {
+        const int v = row[n];
+        K += v;
+        N += v > 0;
+        if (cur_row) ndiff += (v != (int)__ldg(cur_row + n)) ? 1 : 0;
+      }
+    }
+    uint4 *dst = (uint4 *)(a.dst + ((size_t)cl * J + j) * NN);
+    for (int v = 0; v < row_vecs; ++v) dst[v] = ((const uint4 *)row)[v];
+    if (on && (!aa.tp.active || aa.tp.active[j])) s_term[j] = fitness_term(aa.tp, j, K, N, ndiff != 0);
+  }
+  __syncthreads();
+  double tsum, tcount;
+  block_term_sum(s_term, J, 0, aa.tp.active, tsum, tcount);
+  if (tid == 0) aa.fitness_out[cl] = fitness_finalise(aa.tp.mode, aa.tp.p, tsum, tcount);
+}
+
 // Column pass: warps take nodes from the work list the row kernel built (any order: columns are
 // independent) and repair them.
 __global__ void __launch_bounds__(128, 4) colrepair_kernel(ColfixArgs a) {
@@ -1017,6 +1292,15 @@ int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint3
   aa.fitness_out = ctx->ff_out;
   ctx->fit_done = aa.fuse != 0;
   dim3 grid((unsigned)nbatch, (unsigned)count);
+  if (aa.fuse && a.mode == ROWS_GENERATION && NN <= SMALL_MAX_NODES && a.J <= 8192) {
+    // small problem inside a round: thread-per-row kernel, fitness included
+    {
+      TimedLaunch tl_(ctx, KK_ROWS);
+      generation_small_kernel<<<(unsigned)count, 256, 0, ctx->stream>>>(aa);
+    }
+    SCHED_LAUNCH_CHECK(ctx);
+    return SCHED_OK;
+  }
   if (!aa.fuse) SCHED_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->d_colcount, 0, sizeof(unsigned int), ctx->stream));
   {
     TimedLaunch tl_(ctx, KK_ROWS);
