@@ -947,18 +947,53 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
   const int row_vecs = NN >> 3;
   const bool elite = (int)c < a.num_elite;
 
+  // Everything that does not depend on the parents is asked for first, so that the waits overlap:
+  // the job's flags and caps, the fitness keys (staged in shared memory), and the row's draws.
+  const int j = tid;
+  bool on = false;
+  int kc = a.k_max;
+  if (j < J) {
+    on = !a.active || a.active[j];
+    if (a.k_cap) kc = a.k_cap[j];
+  }
+  __shared__ __align__(16) uint32_t s_keys[256];
+  const bool staged = P <= 256;
+  if (staged && tid < P) s_keys[tid] = order_key(__ldg(a.fitness_bits + tid));
   if (tid < NN) {
     s_cap[tid] = (int16_t)max((int)a.cap[tid], 0);
     s_tot[tid] = 0u;
     s_cnt[tid] = 0u;
   }
+  bool second = false, mut = false;
+  u32x4 mw = {0, 0, 0, 0};
+  if (on && !elite) {
+    second = (draw(a.key, (uint32_t)j, c, a.gen, SLOT_XOVER).x >> 31) != 0u;
+    mw = draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE);
+    mut = mw.x < a.thr;
+  }
+  uint4 cur4[SMALL_MAX_NODES / 8];
+#pragma unroll
+  for (int v = 0; v < SMALL_MAX_NODES / 8; ++v) {
+    cur4[v] = make_uint4(0u, 0u, 0u, 0u);
+    if (a.cur && j < J && v < row_vecs) cur4[v] = __ldg((const uint4 *)(a.cur + (size_t)j * NN) + v);
+  }
+  __syncthreads();
   // ---- parents (rank = candidates ordered before, fitness descending, index ascending) --------
   if (elite) {
     for (int i = tid; i < P; i += blockDim.x) {
-      const uint32_t ki = order_key(a.fitness_bits[i]);
-      int rk = 0;
-      for (int o = 0; o < P; ++o) {
-        const uint32_t ko = order_key(__ldg(a.fitness_bits + o));
+      const uint32_t ki = staged ? s_keys[i] : order_key(a.fitness_bits[i]);
+      int rk = 0, o = 0;
+      if (staged) {
+        for (; o + 4 <= P; o += 4) {   // four staged keys per step
+          const uint4 k4 = *(const uint4 *)(s_keys + o);
+          rk += (k4.x > ki || (k4.x == ki && o < i)) ? 1 : 0;
+          rk += (k4.y > ki || (k4.y == ki && o + 1 < i)) ? 1 : 0;
+          rk += (k4.z > ki || (k4.z == ki && o + 2 < i)) ? 1 : 0;
+          rk += (k4.w > ki || (k4.w == ki && o + 3 < i)) ? 1 : 0;
+        }
+      }
+      for (; o < P; ++o) {
+        const uint32_t ko = staged ? s_keys[o] : order_key(__ldg(a.fitness_bits + o));
         rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
       }
       if (rk == (int)c) s_parent[0] = s_parent[1] = i;
@@ -968,10 +1003,10 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
     const int idx[4] = {(int)bounded(sel.x, P), (int)bounded(sel.y, P), (int)bounded(sel.z, P), (int)bounded(sel.w, P)};
     if (warp < 4) {
       const int i = idx[warp];
-      const uint32_t ki = order_key(a.fitness_bits[i]);
+      const uint32_t ki = staged ? s_keys[i] : order_key(a.fitness_bits[i]);
       int rk = 0;
       for (int o = lane; o < P; o += 32) {
-        const uint32_t ko = order_key(__ldg(a.fitness_bits + o));
+        const uint32_t ko = staged ? s_keys[o] : order_key(__ldg(a.fitness_bits + o));
         rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
       }
       rk = warp_sum(rk);
@@ -986,33 +1021,27 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
   __syncthreads();
 
   // ---- rows: thread j builds row j of the child ----------------------------------------------
-  const int j = tid;
+  // K and N of the row in this thread's line of shared memory, from its 16-byte pieces
+  auto row_totals = [&](const int16_t *r, int &k_out, int &n_out) {
+    uint32_t part = 0;
+    for (int v = 0; v < row_vecs; ++v) part += row_partial(((const uint4 *)r)[v]);
+    k_out = (int)(part & 0x3FFFFFu);
+    n_out = (int)(part >> 22);
+  };
   int16_t *row = s_rows[tid];
   int K = 0, N = 0, ndiff = 0;
-  bool on = false;
   if (j < J) {
-    on = !a.active || a.active[j];
-    bool second = false, mut = false;
-    u32x4 mw = {0, 0, 0, 0};
-    if (on && !elite) {
-      second = (draw(a.key, (uint32_t)j, c, a.gen, SLOT_XOVER).x >> 31) != 0u;
-      mw = draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE);
-      mut = mw.x < a.thr;
-    }
     const uint4 *src = (const uint4 *)(a.src + ((size_t)s_parent[second ? 1 : 0] * J + j) * NN);
-    uint4 cur4[SMALL_MAX_NODES / 8];
 #pragma unroll
     for (int v = 0; v < SMALL_MAX_NODES / 8; ++v) {
       uint4 x = make_uint4(0u, 0u, 0u, 0u);
-      cur4[v] = make_uint4(0u, 0u, 0u, 0u);
       if (v < row_vecs) {
         if (on) x = clamp_vec(__ldg(src + v), ((const uint4 *)s_cap)[v]);   // entries into [0, node size]
-        if (a.cur) cur4[v] = __ldg((const uint4 *)(a.cur + (size_t)j * NN) + v);
         ((uint4 *)row)[v] = x;
       }
     }
     if (on) {
-      for (int n = 0; n < NN; ++n) { K += row[n]; N += row[n] > 0; }
+      row_totals(row, K, N);
       if (mut) {
         const uint32_t op = bounded(mw.y, 3u);
         if (op == 0u) {
@@ -1033,12 +1062,10 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
             }
           }
         }
-        K = 0; N = 0;
-        for (int n = 0; n < NN; ++n) { K += row[n]; N += row[n] > 0; }
+        row_totals(row, K, N);
       }
       // per-row caps: replicas above the job's cap leave from the highest node index down, then
       // occupied nodes beyond n_max are cleared from the highest index down
-      int kc = a.k_cap ? a.k_cap[j] : a.k_max;
       kc = max(0, min(kc, a.k_max));
       if (K > kc || N > a.n_max) {
         int excess = K - kc;
@@ -1060,13 +1087,26 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
       }
       // occupants into the nodes' totals and lists; entries differing from the current allocation
       const bool dist = N >= 2;
-      for (int n = 0; n < NN; ++n) {
-        const int v = row[n];
-        if (a.cur) ndiff += (v != (int)((const int16_t *)cur4)[n]) ? 1 : 0;
-        if (v > 0) {
-          atomicAdd(&s_tot[n], (uint32_t)v);
-          const uint32_t k = atomicAdd(&s_cnt[n], (dist ? 1u : 0u) | (1u << 16)) >> 16;
-          if (k < SMALL_OCC) s_occ[n][k] = (uint32_t)j | ((uint32_t)v << 13) | (dist ? 0x80000000u : 0u);
+#pragma unroll
+      for (int v = 0; v < SMALL_MAX_NODES / 8; ++v) {
+        if (v >= row_vecs) break;
+        const uint4 x = ((const uint4 *)row)[v];
+        if (a.cur) {
+          // each half of the xor is a non-negative int16, so min(half, 1) counts the halves that differ
+          const uint32_t d = __vimin_s16x2_relu(x.x ^ cur4[v].x, 0x00010001u) + __vimin_s16x2_relu(x.y ^ cur4[v].y, 0x00010001u) +
+                             __vimin_s16x2_relu(x.z ^ cur4[v].z, 0x00010001u) + __vimin_s16x2_relu(x.w ^ cur4[v].w, 0x00010001u);
+          ndiff += (int)((d & 0xFFFFu) + (d >> 16));
+        }
+        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int h = 0; h < 8; ++h) {
+          const int g = (int)((w[h >> 1] >> ((h & 1) * 16)) & 0xFFFFu);
+          if (g > 0) {
+            const int n = 8 * v + h;
+            atomicAdd(&s_tot[n], (uint32_t)g);
+            const uint32_t k = atomicAdd(&s_cnt[n], (dist ? 1u : 0u) | (1u << 16)) >> 16;
+            if (k < SMALL_OCC) s_occ[n][k] = (uint32_t)j | ((uint32_t)g << 13) | (dist ? 0x80000000u : 0u);
+          }
         }
       }
     }
@@ -1174,13 +1214,17 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
   // ---- rows out, fitness -----------------------------------------------------------------------
   if (j < J) {
     if (s_dirty[j]) {
-      K = 0; N = 0; ndiff = 0;
-      const int16_t *cur_row = a.cur ? a.cur + (size_t)j * NN : nullptr;
-      for (int n = 0; n < NN; ++n) {
-        const int v = row[n];
-        K += v;
-        N += v > 0;
-        if (cur_row) ndiff += (v != (int)__ldg(cur_row + n)) ? 1 : 0;
+      row_totals(row, K, N);
+      ndiff = 0;
+      if (a.cur) {
+#pragma unroll
+        for (int v = 0; v < SMALL_MAX_NODES / 8; ++v) {
+          if (v >= row_vecs) break;
+          const uint4 x = ((const uint4 *)row)[v];
+          const uint32_t d = __vimin_s16x2_relu(x.x ^ cur4[v].x, 0x00010001u) + __vimin_s16x2_relu(x.y ^ cur4[v].y, 0x00010001u) +
+                             __vimin_s16x2_relu(x.z ^ cur4[v].z, 0x00010001u) + __vimin_s16x2_relu(x.w ^ cur4[v].w, 0x00010001u);
+          ndiff += (int)((d & 0xFFFFu) + (d >> 16));
+        }
       }
     }
     uint4 *dst = (uint4 *)(a.dst + ((size_t)cl * J + j) * NN);
