@@ -947,6 +947,10 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
   const int row_vecs = NN >> 3;
   const bool elite = (int)c < a.num_elite;
 
+  // The next generation's grid may be set up while this one runs (programmatic dependent launch):
+  // its blocks do their own parent-independent prologue and then wait, below, for this grid to
+  // finish.  Nothing this kernel writes to global memory is written before its own wait.
+  asm volatile("griddepcontrol.launch_dependents;");
   // Everything that does not depend on the parents is asked for first, so that the waits overlap:
   // the job's flags and caps, the fitness keys (staged in shared memory), and the row's draws.
   const int j = tid;
@@ -958,7 +962,6 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
   }
   __shared__ __align__(16) uint32_t s_keys[256];
   const bool staged = P <= 256;
-  if (staged && tid < P) s_keys[tid] = order_key(__ldg(a.fitness_bits + tid));
   if (tid < NN) {
     s_cap[tid] = (int16_t)max((int)a.cap[tid], 0);
     s_tot[tid] = 0u;
@@ -977,11 +980,14 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
     cur4[v] = make_uint4(0u, 0u, 0u, 0u);
     if (a.cur && j < J && v < row_vecs) cur4[v] = __ldg((const uint4 *)(a.cur + (size_t)j * NN) + v);
   }
+  // from here on the parents' population and fitness are read: the grid that wrote them must be done
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (staged && tid < P) s_keys[tid] = order_key(__ldcg(a.fitness_bits + tid));
   __syncthreads();
   // ---- parents (rank = candidates ordered before, fitness descending, index ascending) --------
   if (elite) {
     for (int i = tid; i < P; i += blockDim.x) {
-      const uint32_t ki = staged ? s_keys[i] : order_key(a.fitness_bits[i]);
+      const uint32_t ki = staged ? s_keys[i] : order_key(__ldcg(a.fitness_bits + i));
       int rk = 0, o = 0;
       if (staged) {
         for (; o + 4 <= P; o += 4) {   // four staged keys per step
@@ -993,7 +999,7 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
         }
       }
       for (; o < P; ++o) {
-        const uint32_t ko = staged ? s_keys[o] : order_key(__ldg(a.fitness_bits + o));
+        const uint32_t ko = staged ? s_keys[o] : order_key(__ldcg(a.fitness_bits + o));
         rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
       }
       if (rk == (int)c) s_parent[0] = s_parent[1] = i;
@@ -1003,10 +1009,10 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
     const int idx[4] = {(int)bounded(sel.x, P), (int)bounded(sel.y, P), (int)bounded(sel.z, P), (int)bounded(sel.w, P)};
     if (warp < 4) {
       const int i = idx[warp];
-      const uint32_t ki = staged ? s_keys[i] : order_key(a.fitness_bits[i]);
+      const uint32_t ki = staged ? s_keys[i] : order_key(__ldcg(a.fitness_bits + i));
       int rk = 0;
       for (int o = lane; o < P; o += 32) {
-        const uint32_t ko = staged ? s_keys[o] : order_key(__ldg(a.fitness_bits + o));
+        const uint32_t ko = staged ? s_keys[o] : order_key(__ldcg(a.fitness_bits + o));
         rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
       }
       rk = warp_sum(rk);
@@ -1036,7 +1042,7 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
     for (int v = 0; v < SMALL_MAX_NODES / 8; ++v) {
       uint4 x = make_uint4(0u, 0u, 0u, 0u);
       if (v < row_vecs) {
-        if (on) x = clamp_vec(__ldg(src + v), ((const uint4 *)s_cap)[v]);   // entries into [0, node size]
+        if (on) x = clamp_vec(__ldcg(src + v), ((const uint4 *)s_cap)[v]);   // entries into [0, node size]
         ((uint4 *)row)[v] = x;
       }
     }
@@ -1340,7 +1346,21 @@ int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint3
     // small problem inside a round: thread-per-row kernel, fitness included
     {
       TimedLaunch tl_(ctx, KK_ROWS);
-      generation_small_kernel<<<(unsigned)count, 256, 0, ctx->stream>>>(aa);
+      // launched so that it may overlap the tail of the kernel before it (see the kernel's top)
+      cudaLaunchConfig_t lc = {};
+      lc.gridDim = dim3((unsigned)count);
+      lc.blockDim = dim3(256);
+      lc.dynamicSmemBytes = 0;
+      lc.stream = ctx->stream;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = 1;
+      lc.attrs = attr;
+      lc.numAttrs = 1;
+      if (cudaLaunchKernelEx(&lc, generation_small_kernel, aa) != cudaSuccess) {
+        cudaGetLastError();
+        generation_small_kernel<<<(unsigned)count, 256, 0, ctx->stream>>>(aa);
+      }
     }
     SCHED_LAUNCH_CHECK(ctx);
     return SCHED_OK;
