@@ -274,6 +274,7 @@ int sched_destroy(sched_ctx *ctx) {
                   ctx->d_colelig, ctx->rs_pool, ctx->rs_rec, ctx->rs_ptr, ctx->rs_state};
   for (void *p : ptrs)
     if (p) cudaFree(p);
+  if (ctx->h_stage) cudaFreeHost(ctx->h_stage);
   if (ctx->graph_exec) cudaGraphExecDestroy(ctx->graph_exec);
   for (auto *v : {&ctx->spans, &ctx->free_spans})
     for (TimedSpan &t : *v) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
@@ -675,10 +676,22 @@ int schedule_round_host(sched_ctx *ctx, const sched_jobs *h_jobs, const int16_t 
   }
   char *base = (char *)ctx->d_stage;
   size_t off = 0;
+  // Small problems: the inputs are first gathered in a pinned buffer laid out like the device
+  // one and go up in a single copy (launching 18 small copies costs more than the bytes do).
+  const size_t input_bytes = need - 2 * align256(mat) - 256 + align256(mat);   // everything up to and including cur
+  const bool gather = input_bytes <= (256u << 10);
+  if (gather && input_bytes > ctx->h_stage_bytes) {
+    if (ctx->h_stage) { cudaFreeHost(ctx->h_stage); ctx->h_stage = nullptr; ctx->h_stage_bytes = 0; }
+    if (cudaMallocHost(&ctx->h_stage, input_bytes) == cudaSuccess) ctx->h_stage_bytes = input_bytes;
+    else { cudaGetLastError(); ctx->h_stage = nullptr; }
+  }
+  char *hbase = (gather && ctx->h_stage) ? (char *)ctx->h_stage : nullptr;
   auto up = [&](const void *h, size_t bytes, size_t slot) -> const void * {
     void *d = base + off;
+    char *hs = hbase ? hbase + off : nullptr;
     off += slot;
     if (!h) return nullptr;
+    if (hs) { memcpy(hs, h, bytes); return d; }
     if (cudaMemcpyAsync(d, h, bytes, cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess) return (const void *)-1;
     return d;
   };
@@ -704,6 +717,7 @@ int schedule_round_host(sched_ctx *ctx, const sched_jobs *h_jobs, const int16_t 
   bad |= dj.m_grid == (const void *)-1 || dj.k_cap == (const void *)-1 || dj.fair_k == (const void *)-1 ||
          dj.fair_n == (const void *)-1 || dj.age_sec == (const void *)-1 ||
          dj.num_restarts == (const void *)-1 || dj.active == (const void *)-1 || d_cur == (const void *)-1;
+  if (hbase && cudaMemcpyAsync(base, hbase, off, cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess) bad = true;
   REQUIRE(ctx, !bad, SCHED_ERR_CUDA, "schedule_round_host: a host-to-device copy failed: %s",
           cudaGetErrorString(cudaGetLastError()));
   int16_t *d_best = (int16_t *)(base + off);

@@ -113,6 +113,8 @@ struct sched_ctx {
   // staging for the *_host entry points (allocated on first use)
   void *d_stage;         // job arrays + cur + best
   size_t stage_bytes;
+  void *h_stage;         // pinned mirror of the inputs' part of d_stage (small problems: one copy instead of 18)
+  size_t h_stage_bytes;
   void *d_stage_fit;     // eval_fitness_host staging
   size_t stage_fit_bytes;
 
