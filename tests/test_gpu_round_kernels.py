@@ -1,7 +1,9 @@
-"""Rounds of problems with more than 256 jobs keep their population as shared rows (indices
-into a row pool, copy on write).  Such a round must equal, bit for bit, the same round made
-of the dense entry points called one by one, which the other tests pin to the oracle; the
-last generation is also checked against the oracle directly (teacher-forced)."""
+"""Inside a round the generations run on specialised kernels: problems with more than 256 jobs
+keep their population as shared rows (indices into a row pool, copy on write), problems with
+at most 256 jobs and 32 nodes use a thread-per-row kernel.  Either way the round must equal,
+bit for bit, the same round made of the dense entry points called one by one, which the other
+tests pin to the oracle; the last generation is also checked against the oracle directly
+(teacher-forced)."""
 import dataclasses
 
 import numpy as np
@@ -35,6 +37,14 @@ CASES = [
                  init_prob=0.3, with_history=True, random_cur=True),
     # the large workload itself (the configuration the benchmark times), ten generations
     dataclasses.replace(synth.LARGE, name="store-large", generations=10),
+    # thread-per-row kernel: more jobs on a node than its list holds (column scan in shared memory)
+    synth.Config("small-crowded-nodes", 8, 128, 256, 17, 16, 8, 24, 30, num_elite=2, mutate_prob=0.3,
+                 init_prob=0.9, with_history=True, random_cur=True),
+    # thread-per-row kernel: the widest rows it takes (32 nodes), row caps at work, inactive jobs
+    synth.Config("small-32-nodes", 32, 4, 120, 18, 16, 8, 20, 15, num_elite=3, mutate_prob=0.6,
+                 init_prob=0.6, with_history=True, random_cur=True),
+    # thread-per-row kernel: three 16-byte pieces per row, no current allocation
+    synth.Config("small-24-nodes", 24, 2, 90, 19, 16, 8, 16, 10, num_elite=1, mutate_prob=0.4, init_prob=0.4),
 ]
 
 
@@ -75,7 +85,7 @@ def _stepwise(torch, s, dj, cfg, d_cur, rnd, gens, penalise):
 def test_store_round_equals_dense_stepwise_round(gpu, oracle, cfg):
     torch, api = gpu
     cl, jobs = setup(cfg)
-    if cfg.name == "store-plain":
+    if cfg.name in ("store-plain", "small-32-nodes"):
         jobs.active[::7] = 0
         jobs = setup_fair(jobs, cl)
     if cfg.name == "store-wide-rows":      # six jobs share the cluster, so their rows can spread
@@ -105,6 +115,8 @@ def test_store_round_equals_dense_stepwise_round(gpu, oracle, cfg):
         assert feasible(pop[c], cl.node_capacity, jobs.k_cap, cl.n_max)
     if cfg.name == "store-crowded-nodes":
         assert (pop > 0).sum(axis=1).max() > 16      # more jobs on a node than a block lists
+    if cfg.name == "small-crowded-nodes":
+        assert (pop > 0).sum(axis=1).max() > 32
     if cfg.name == "store-wide-rows":
         assert (pop > 0).sum(axis=2).max() > 8       # rows wider than a record
 
