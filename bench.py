@@ -284,6 +284,7 @@ def run_ours(args):
         line["dense_generation"] = bench_dense_generation(api, torch, dev, stream, cfg, cl, jobs, cur, hbm_peak, peak_src)
         line["goodput_model"] = bench_table(api, torch, dev, stream, cfg, cl, jobs, sm_max_mhz, clocks)
         line["stress_fitness"] = bench_stress(api, torch, dev, stream, hbm_peak, peak_src, args)
+        line["testbed_round"] = bench_testbed(api, torch, dev, stream)
         line["trace_replay"] = bench_trace(api, torch, stream)
         line["theta_fit"] = bench_fit(api, torch, dev, stream)
         line["cpu_baseline"] = oracle_sample(cfg, cl, jobs, cur)
@@ -460,6 +461,41 @@ def bench_fit(api, torch, dev, stream):
             "median_rmsle": float(np.median(lg)), "oracle_lbfgsb_sec_per_job": cpu_s,
             "oracle_median_rmsle_8_jobs": float(np.median(ref)),
             "note": "fp64 damped Gauss-Newton, one warp per job; the paper reports 0.2 s per fit on a CPU core"}
+
+
+def bench_testbed(api, torch, dev, stream):
+    """schedule_round on the testbed-scale workload (16 nodes x 4 GPUs, 48 jobs, grid 64 x 16,
+    population 100, 100 generations, re-allocation penalty against a random current allocation):
+    the size of the paper's own cluster.  Launch- and latency-bound; rounds replay as graphs."""
+    cfg = synth.TESTBED
+    cl = cfg.cluster()
+    jobs = cfg.jobs()
+    fk, fn = api.fair_share(cl.node_capacity, cfg.num_jobs, cl.k_max)
+    jobs.fair_k = np.full(cfg.num_jobs, fk, np.int32)
+    jobs.fair_n = np.full(cfg.num_jobs, fn, np.int32)
+    sched = api.scheduler_for(cfg, stream=stream.cuda_stream)
+    dj = api.DeviceJobs(jobs, dev, torch)
+    d_cur = torch.from_numpy(cfg.cur()).to(dev)
+    best = torch.empty((cfg.num_jobs, cfg.num_nodes), dtype=torch.int16, device=dev)
+    bf = torch.zeros(1, dtype=torch.float32, device=dev)
+    for r in range(5):
+        sched.schedule_round(dj, d_cur, best, bf, round=r, generations=cfg.generations)
+    sched.sync_status()
+    n = 200
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for r in range(n):
+        sched.schedule_round(dj, d_cur, best, bf, round=10 + r, generations=cfg.generations)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / n
+    sched.close()
+    return {"workload": "testbed: 16 nodes x 4 GPUs, 48 jobs, grid 64x16, population 100, 100 generations, p=-1",
+            "ms_per_round": ms, "rounds_per_sec": 1e3 / ms,
+            "candidates_per_sec": cfg.population * (cfg.generations + 1) / (ms * 1e-3),
+            "us_per_generation": 1e3 * ms / cfg.generations,
+            "note": "one 100-block kernel per generation (thread per row): latency-bound, no roofline; "
+                    "the paper reports about 1 s per round on one CPU core at this cluster size"}
 
 
 def bench_trace(api, torch, stream):
