@@ -3,10 +3,14 @@
 // avoidance (Sec. 4.2).  Integer work only; all randomness comes from the counter-based
 // stream, so every output is a pure function of the inputs.
 //
-// Structure: a row kernel (one warp per (candidate, job) row: build the child row in
-// shared memory, perturb, apply the per-row caps, write it and a "spans >= 2 nodes" flag)
-// followed by a column kernel (one thread per (candidate, node): interference and
-// capacity passes over the jobs of that node).
+// Three implementations of the same operators on dense matrices, chosen by shape:
+//  * rows_kernel + cols_kernel (+ rank_kernel): the general pair - a warp per (candidate, job)
+//    row through shared memory, then a thread per (candidate, node) column;
+//  * rows2_kernel + colrepair_kernel: rows of whole 16-byte vectors and at most 512 nodes -
+//    batched rows with fused column sums and occupant lists, a work list of violating nodes;
+//    for at most 256 jobs the row kernel also does the column pass and the fitness (FUSE);
+//  * generation_small_kernel: at most 256 jobs and 32 nodes inside a round - a thread per row.
+// Rounds of more than 256 jobs do not use dense matrices for their generations at all (rowstore.cu).
 #include "common.cuh"
 #include "fitness_common.cuh"
 
