@@ -988,6 +988,10 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (staged && tid < P) s_keys[tid] = order_key(__ldcg(a.fitness_bits + tid));
   __syncthreads();
+  const bool early = !elite && row_vecs <= 2;
+  uint4 cand[2][2] = {{make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)},
+                      {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)}};
+  int pair0 = -1;
   // ---- parents (rank = candidates ordered before, fitness descending, index ascending) --------
   if (elite) {
     for (int i = tid; i < P; i += blockDim.x) {
@@ -1011,6 +1015,16 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
   } else {
     const u32x4 sel = draw(a.key, 0u, c, a.gen, SLOT_SELECT);
     const int idx[4] = {(int)bounded(sel.x, P), (int)bounded(sel.y, P), (int)bounded(sel.z, P), (int)bounded(sel.w, P)};
+    // short rows: this thread's row of both candidates of its pair is fetched while the ranks
+    // are being worked out
+    if (early && j < J && on) {
+      pair0 = idx[second ? 2 : 0];
+      const uint4 *r0 = (const uint4 *)(a.src + ((size_t)pair0 * J + j) * NN);
+      const uint4 *r1 = (const uint4 *)(a.src + ((size_t)idx[second ? 3 : 1] * J + j) * NN);
+      cand[0][0] = __ldcg(r0);
+      cand[1][0] = __ldcg(r1);
+      if (row_vecs > 1) { cand[0][1] = __ldcg(r0 + 1); cand[1][1] = __ldcg(r1 + 1); }
+    }
     if (warp < 4) {
       const int i = idx[warp];
       const uint32_t ki = staged ? s_keys[i] : order_key(__ldcg(a.fitness_bits + i));
@@ -1041,12 +1055,17 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
   int16_t *row = s_rows[tid];
   int K = 0, N = 0, ndiff = 0;
   if (j < J) {
-    const uint4 *src = (const uint4 *)(a.src + ((size_t)s_parent[second ? 1 : 0] * J + j) * NN);
+    const int parent = s_parent[second ? 1 : 0];
+    const uint4 *src = (const uint4 *)(a.src + ((size_t)parent * J + j) * NN);
+    const int which = (parent == pair0) ? 0 : 1;   // when the row was fetched early
 #pragma unroll
     for (int v = 0; v < SMALL_MAX_NODES / 8; ++v) {
       uint4 x = make_uint4(0u, 0u, 0u, 0u);
       if (v < row_vecs) {
-        if (on) x = clamp_vec(__ldcg(src + v), ((const uint4 *)s_cap)[v]);   // entries into [0, node size]
+        if (on) {
+          const uint4 raw = (early && v < 2) ? (which == 0 ? cand[0][v] : cand[1][v]) : __ldcg(src + v);
+          x = clamp_vec(raw, ((const uint4 *)s_cap)[v]);   // entries into [0, node size]
+        }
         ((uint4 *)row)[v] = x;
       }
     }
