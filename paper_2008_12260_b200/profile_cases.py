@@ -4,6 +4,7 @@
     python -m paper_2008_12260_b200.profile_cases table_large      # 1024-job speedup table
     python -m paper_2008_12260_b200.profile_cases round_large [G]  # large round, G generations (default 2)
     python -m paper_2008_12260_b200.profile_cases generation_large # dense ga_generation, large shape
+    python -m paper_2008_12260_b200.profile_cases round_testbed [G] # testbed-scale round, G generations
 
 Each case holds well under a few GB on the device, launches its kernel a handful of
 times and exits; inputs are larger than L2 wherever DRAM traffic is the point.
@@ -58,6 +59,21 @@ def main(case: str, reps: int = 3, generations: int = 2):
         s.schedule_round(dj, cur, best, bf, round=0, generations=generations)
         s.sync_status()
         print("round_large", float(bf.item()))
+    elif case == "round_testbed":
+        cfg = synth.TESTBED
+        cl = cfg.cluster()
+        jobs = cfg.jobs()
+        fk, fn = api.fair_share(cl.node_capacity, cfg.num_jobs, cl.k_max)
+        jobs.fair_k = np.full(cfg.num_jobs, fk, np.int32)
+        jobs.fair_n = np.full(cfg.num_jobs, fn, np.int32)
+        s = api.scheduler_for(cfg, stream=torch.cuda.current_stream().cuda_stream)
+        dj = api.DeviceJobs(jobs, "cuda", torch)
+        cur = torch.from_numpy(cfg.cur()).cuda()
+        best = torch.empty((cfg.num_jobs, cfg.num_nodes), dtype=torch.int16, device="cuda")
+        bf = torch.zeros(1, dtype=torch.float32, device="cuda")
+        s.schedule_round(dj, cur, best, bf, round=0, generations=generations)
+        s.sync_status()
+        print("round_testbed", float(bf.item()))
     elif case == "generation_large":
         cfg, cl, jobs, s, dj = _large(api, synth, torch)
         shape = (cfg.population, cfg.num_jobs, cfg.num_nodes)
