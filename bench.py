@@ -252,6 +252,13 @@ def run_ours(args):
                     "note": "one block evolves one candidate per launch on L2-resident records: latency- and "
                             "issue-bound, not DRAM-bound (the dense operator kernel, which is, is reported under "
                             "dense_generation)" if dom["kernel"] == "generation_store" else None,
+                    # what the same generation costs on dense matrices (parents read, children written, the
+                    # repair's row and column passes: about four population sweeps): the bytes this kernel
+                    # exists to avoid.  Reported for scale only; it is NOT the kernel's traffic.
+                    "dense_equivalent": {"bytes_per_launch": 4 * pop_bytes,
+                                         "floor_us_at_hbm_peak": round(4 * pop_bytes / (hbm_peak * 1e9) * 1e6, 1),
+                                         "this_kernel_us": dom["avg_us"]}
+                    if dom["kernel"] == "generation_store" else None,
                     # from the committed ncu summary of this kernel (not measured in this run)
                     "ncu_counters": {"issue_active_pct": 34.7, "dram_pct_of_peak": 3.8, "l2_hit_pct": 48.2,
                                      "warp_instructions": 12.6e6, "stall_barrier_per_issue": 4.2,
