@@ -27,10 +27,10 @@ __device__ __forceinline__ size_t fitness_table_index(const TermParams &tp, int 
   return ((size_t)j * (tp.k_max + 1) + K) * (tp.n_max + 1) + N;
 }
 
-// x_j^p from the looked-up speedup x: re-allocation penalty, floor, and the form that the
-// mode sums (x, 1/x, ln x, sqrt x or x^p).
-__device__ __forceinline__ float fitness_term_of(const TermParams &tp, int j, float x, bool changed) {
-  if (tp.pen && changed) x *= tp.pen[j];
+// x_j^p from the looked-up speedup x and the job's penalty factor (used when the row changed):
+// re-allocation penalty, floor, and the form that the mode sums (x, 1/x, ln x, sqrt x or x^p).
+__device__ __forceinline__ float fitness_term_with(const TermParams &tp, float x, float pen, bool changed) {
+  if (tp.pen && changed) x *= pen;
   x = fmaxf(x, tp.floor_);
   switch (tp.mode) {
     case MODE_ARITH: return x;
@@ -39,6 +39,10 @@ __device__ __forceinline__ float fitness_term_of(const TermParams &tp, int j, fl
     case MODE_SQRT: return sqrtf(x);
     default: return powf(x, tp.p);
   }
+}
+
+__device__ __forceinline__ float fitness_term_of(const TermParams &tp, int j, float x, bool changed) {
+  return fitness_term_with(tp, x, (tp.pen && changed) ? tp.pen[j] : 1.f, changed);
 }
 
 // x_j^p of one row (SPEEDUP looked up at (K, N), re-allocation penalty, floor).

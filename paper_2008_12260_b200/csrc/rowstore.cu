@@ -741,18 +741,28 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         p = summarise_row<PPL>(g, row, cur, K, N, nd, recw);
       }
       const uint32_t slot = s_base_mut + (uint32_t)i;
+      // the row's speedup (and penalty factor) are asked for now and used at the end of the step
+      float x_sp = 0.f, x_pen = 1.f;
+      if (g.sub == 0) {
+        x_sp = __ldg(a.tp.table + fitness_table_index(a.tp, j, K, N));
+        if (a.tp.pen && nd != 0) x_pen = __ldg(a.tp.pen + j);
+      }
       store_row(g, a.st.pool + (size_t)slot * NN, row);
       const uint32_t word = pack_summary(K, N, nd);
       if (g.sub == 0) {
         recw[REC_SUMM] = word;
-        recw[REC_TERM] = 0u;   // filled in with the other new rows' terms at the end
         s_slot[j] = slot;
         s_summ[j] = word;
         s_mark[j] = 2;
       }
+      add_row_occupants(g, j, p, N >= 2);
+      if (g.sub == 0) {
+        const float term = fitness_term_with(a.tp, x_sp, x_pen, nd != 0);
+        s_term[j] = term;
+        recw[REC_TERM] = __float_as_uint(term);
+      }
       __syncwarp(g.mask);
       if (g.sub < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + g.sub] = recw[g.sub];
-      add_row_occupants(g, j, p, N >= 2);
       __syncwarp(g.mask);
     }
   }
@@ -862,13 +872,20 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         int K, N, nd;
         summarise_row<PPL>(g, row, cur, K, N, nd, recw);
         const uint32_t dst = own ? src : s_base_cow + (uint32_t)i;
+        float x_sp = 0.f, x_pen = 1.f;
+        if (g.sub == 0) {
+          x_sp = __ldg(a.tp.table + fitness_table_index(a.tp, j, K, N));
+          if (a.tp.pen && nd != 0) x_pen = __ldg(a.tp.pen + j);
+        }
         store_row(g, a.st.pool + (size_t)dst * NN, row);
         const uint32_t word = pack_summary(K, N, nd);
         if (g.sub == 0) {
+          const float term = fitness_term_with(a.tp, x_sp, x_pen, nd != 0);
           recw[REC_SUMM] = word;
-          recw[REC_TERM] = 0u;
+          recw[REC_TERM] = __float_as_uint(term);
           s_slot[j] = dst;
           s_summ[j] = word;
+          s_term[j] = term;
         }
         __syncwarp(g.mask);
         if (g.sub < REC_WORDS) a.st.rec[(size_t)dst * REC_WORDS + g.sub] = recw[g.sub];
@@ -936,9 +953,11 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         summarise_row<PPL>(g, row, cur, K, N, nd, recw);
         const uint32_t word = pack_summary(K, N, nd);
         if (g.sub == 0) {
+          const float term = fitness_term(a.tp, j, K, N, nd != 0);
           recw[REC_SUMM] = word;
-          recw[REC_TERM] = 0u;
+          recw[REC_TERM] = __float_as_uint(term);
           s_summ[j] = word;
+          s_term[j] = term;
         }
         __syncwarp(g.mask);
         if (g.sub < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + g.sub] = recw[g.sub];
@@ -951,16 +970,6 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   // ---- children's indices out, fitness of the candidate (Eq. 14) from the rows' terms ----------
   uint32_t *pout = a.ptr_out + (size_t)c * J;
   for (int j = tid; j < J; j += GEN_THREADS) pout[j] = s_slot[j];
-  // terms of the rows that are new in this generation (the others got theirs with their record)
-  const int nmut = s_nmut;
-  for (int i = tid; i < nmut + nmod; i += GEN_THREADS) {
-    const int j = (int)(i < nmut ? s_mut[i] : s_mod[i - nmut]);
-    const uint32_t w = s_summ[j];
-    const float term = fitness_term(a.tp, j, (int)(w & 0x7FFu), (int)((w >> 11) & 0x7FFu), (w >> 22) != 0u);
-    s_term[j] = term;
-    if (!s_fail) a.st.rec[(size_t)s_slot[j] * REC_WORDS + REC_TERM] = __float_as_uint(term);
-  }
-  __syncthreads();
   // sums in the order of the dense fitness kernel: per chunk of rows, thread t adds rows t,
   // t + 256, ... in double, a shuffle tree per warp, the warps in index order; then the chunks
   // in index order
