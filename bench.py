@@ -45,9 +45,9 @@ HBM_FALLBACK_GBS = 6650.0
 # "rows": one dense large-workload generation (237.1 MB read + 257.1 MB written).
 # "fitness_stress": 16 dense stress candidates moved 544.8 + 3.0 MB; every candidate is streamed
 # once, so the figure is scaled by candidates / 16 to the chunk that is timed (544.8 + 3.5 MB).
-# "generation_store": one row-store generation of the large workload (12.7 MB read in generation 9;
+# "generation_store": one row-store generation of the large workload (12.8 MB read in generation 8;
 # generations 2..12 of a round read 19.5 .. 11.5 MB as L2 warms up).
-NCU_TRAFFIC_BYTES = {"rows": 494.2e6, "fitness_stress_per_candidate": 548.3e6 / 16, "generation_store": 12.7e6}
+NCU_TRAFFIC_BYTES = {"rows": 494.2e6, "fitness_stress_per_candidate": 548.3e6 / 16, "generation_store": 12.8e6}
 
 
 def measured_peaks():
@@ -260,9 +260,9 @@ def run_ours(args):
                                          "this_kernel_us": dom["avg_us"]}
                     if dom["kernel"] == "generation_store" else None,
                     # from the committed ncu summary of this kernel (not measured in this run)
-                    "ncu_counters": {"issue_active_pct": 34.7, "dram_pct_of_peak": 3.8, "l2_hit_pct": 48.2,
-                                     "warp_instructions": 12.6e6, "stall_barrier_per_issue": 4.2,
-                                     "stall_long_scoreboard_per_issue": 4.5}
+                    "ncu_counters": {"issue_active_pct": 35.8, "dram_pct_of_peak": 3.8, "l2_hit_pct": 47.7,
+                                     "warp_instructions": 13.0e6, "stall_barrier_per_issue": 3.7,
+                                     "stall_long_scoreboard_per_issue": 4.4}
                     if dom["kernel"] == "generation_store" else None}
 
     line = {
