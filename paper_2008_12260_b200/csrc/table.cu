@@ -283,7 +283,9 @@ __device__ __forceinline__ bool kn_valid(int K, int N, int k_max, int n_max,
 }
 
 // Broadcast the class results along N and divide by the fair-share goodput (Eq. 15).
-// Block = a 32-wide stripe of N of one job's slab (blockIdx.z = job); its 8 thread rows walk K.
+// Block = one job's slab of (k_max + 1) x (n_max + 1) entries, walked in memory order (thread
+// t takes entries t, t + 256, ...; its (K, N) advance without divisions), so every store is
+// coalesced whatever the slab's width.
 __global__ void __launch_bounds__(256)
 speedup_expand_kernel(const float *__restrict__ gmax, const uint16_t *__restrict__ amax,
                       const int32_t *__restrict__ kfit, const int32_t *__restrict__ fair_k,
@@ -291,26 +293,28 @@ speedup_expand_kernel(const float *__restrict__ gmax, const uint16_t *__restrict
                       float *__restrict__ goodput, float *__restrict__ speedup,
                       uint16_t *__restrict__ argmax) {
   const int KD = k_max + 1, ND = n_max + 1;
-  const int N = blockIdx.x * 32 + threadIdx.x;
-  const int j = j_first + blockIdx.z;
-  if (N >= ND) return;
+  const int j = j_first + blockIdx.x;
   const int kf = fair_k[j], nf = fair_n[j];
   float denom = 0.f;
   if (kn_valid(kf, nf, k_max, n_max, kfit)) denom = gmax[((size_t)j * KD + kf) * 2 + (nf >= 2 ? 1 : 0)];
-  const int kfitN = (N >= 1 && N <= n_max) ? kfit[N] : -1;
-#pragma unroll 4
-  for (int K = threadIdx.y; K < KD; K += 8) {
-    const size_t e = ((size_t)j * KD + K) * ND + N;
+  const int entries = KD * ND;
+  const int step_k = (int)blockDim.x / ND, step_n = (int)blockDim.x % ND;
+  int K = (int)threadIdx.x / ND, N = (int)threadIdx.x % ND;
+  const size_t slab = (size_t)j * entries;
+  for (int e = threadIdx.x; e < entries; e += blockDim.x) {
     float g = 0.f;
     uint16_t a = 0xFFFFu;
-    if (K >= N && K <= kfitN && N >= 1) {
+    if (N >= 1 && K >= N && K <= __ldg(kfit + N)) {
       const size_t src = ((size_t)j * KD + K) * 2 + (N >= 2 ? 1 : 0);
       g = gmax[src];
       a = amax[src];
     }
-    if (goodput) goodput[e] = g;
-    if (argmax) argmax[e] = a;
-    speedup[e] = denom > 0.f ? g / denom : 0.f;
+    if (goodput) goodput[slab + e] = g;
+    if (argmax) argmax[slab + e] = a;
+    speedup[slab + e] = denom > 0.f ? g / denom : 0.f;
+    K += step_k;
+    N += step_n;
+    if (N >= ND) { N -= ND; ++K; }
   }
 }
 
@@ -366,11 +370,11 @@ static int launch_expand(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodpu
                          uint16_t *d_argmax) {
   const sched_config &c = ctx->cfg;
   const int J = c.num_jobs;
-  for (int j0 = 0; j0 < J; j0 += 65535) {      // grid.z is limited to 65535 jobs per launch
-    dim3 grid((unsigned)((ctx->ND + 31) / 32), 1u, (unsigned)std::min(65535, J - j0));
+  for (int j0 = 0; j0 < J; j0 += 65535) {      // at most 65535 jobs per launch
+    const unsigned grid = (unsigned)std::min(65535, J - j0);
     {
       TimedLaunch tl_(ctx, KK_EXPAND);
-      speedup_expand_kernel<<<grid, dim3(32, 8), 0, ctx->stream>>>(ctx->d_gmax, ctx->d_amax, ctx->d_kfit,
+      speedup_expand_kernel<<<grid, 256, 0, ctx->stream>>>(ctx->d_gmax, ctx->d_amax, ctx->d_kfit,
                                                                    jobs->fair_k, jobs->fair_n, j0, c.k_max, c.n_max,
                                                                    d_goodput, d_speedup, d_argmax);
     }
