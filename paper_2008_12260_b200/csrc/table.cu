@@ -300,18 +300,24 @@ speedup_expand_kernel(const float *__restrict__ gmax, const uint16_t *__restrict
   const int entries = KD * ND;
   const int step_k = (int)blockDim.x / ND, step_n = (int)blockDim.x % ND;
   int K = (int)threadIdx.x / ND, N = (int)threadIdx.x % ND;
-  const size_t slab = (size_t)j * entries;
+  // the job's own pieces of every array, so that the loop indexes with 32-bit offsets
+  const float *gj = gmax + (size_t)j * KD * 2;
+  const uint16_t *aj = amax + (size_t)j * KD * 2;
+  float *gout = goodput ? goodput + (size_t)j * entries : nullptr;
+  uint16_t *aout = argmax ? argmax + (size_t)j * entries : nullptr;
+  float *sout = speedup + (size_t)j * entries;
   for (int e = threadIdx.x; e < entries; e += blockDim.x) {
-    float g = 0.f;
+    float g = 0.f, sp = 0.f;
     uint16_t a = 0xFFFFu;
     if (N >= 1 && K >= N && K <= __ldg(kfit + N)) {
-      const size_t src = ((size_t)j * KD + K) * 2 + (N >= 2 ? 1 : 0);
-      g = gmax[src];
-      a = amax[src];
+      const int src = K * 2 + (N >= 2 ? 1 : 0);
+      g = gj[src];
+      a = aj[src];
+      if (denom > 0.f) sp = g / denom;   // empty entries stay 0 without a division
     }
-    if (goodput) goodput[slab + e] = g;
-    if (argmax) argmax[slab + e] = a;
-    speedup[slab + e] = denom > 0.f ? g / denom : 0.f;
+    if (gout) gout[e] = g;
+    if (aout) aout[e] = a;
+    sout[e] = sp;
     K += step_k;
     N += step_n;
     if (N >= ND) { N -= ND; ++K; }
