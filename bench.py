@@ -115,12 +115,13 @@ class ClockSampler:
         return out
 
 
-def large_inputs(rank: int):
+def large_inputs(rank: int, fair_share):
+    """Inputs of the large workload; `fair_share` is the arm's own (K_f, N_f) routine: the
+    library's for the CUDA arm, the oracle's for the reference arm."""
     cfg = synth.LARGE
     cl = cfg.cluster()
     jobs = synth.draw_jobs(cfg.num_jobs, cfg.seed + 1000 * rank, cfg.grid_m, cfg.grid_s, cl.k_max,
                            phi_hi=cfg.phi_hi, with_history=True)
-    from paper_2008_12260_b200.api import fair_share
     fk, fn = fair_share(cl.node_capacity, cfg.num_jobs, cl.k_max)
     jobs.fair_k = np.full(cfg.num_jobs, fk, np.int32)
     jobs.fair_n = np.full(cfg.num_jobs, fn, np.int32)
@@ -153,7 +154,7 @@ def run_ours(args):
     torch.cuda.set_stream(stream)
     hbm_peak, peak_src, sm_max_mhz = measured_peaks()
 
-    cfg, cl, jobs, cur = large_inputs(rank)
+    cfg, cl, jobs, cur = large_inputs(rank, api.fair_share)
     G, P, J, NN = cfg.generations, cfg.population, cfg.num_jobs, cfg.num_nodes
     sched = api.scheduler_for(cfg, stream=stream.cuda_stream)
     dj = api.DeviceJobs(jobs, dev, torch)
@@ -582,7 +583,9 @@ def run_reference(args):
     rank, _, world = pdist.env_world()
     if rank != 0:
         return
-    cfg, cl, jobs, cur = large_inputs(0)
+    import oracle
+
+    cfg, cl, jobs, cur = large_inputs(0, oracle.fair_share)
     samples = []
     for i in range(args.warmup + args.steps):
         s = oracle_sample(cfg, cl, jobs, cur, table_jobs=4, gens=1)

@@ -40,8 +40,9 @@ extern "C" {
 #define SCHED_ERR_INVALID_ARG (-1) /* null pointer, negative size, misaligned buffer   */
 #define SCHED_ERR_BAD_CONFIG (-2)  /* a sched_config field outside its documented range */
 #define SCHED_ERR_CUDA (-3)        /* a CUDA runtime call failed                        */
-#define SCHED_ERR_TIMEOUT (-4)     /* a bounded device-side wait ran out                */
-#define SCHED_ERR_NOT_FINITE (-5)  /* reserved                                          */
+#define SCHED_ERR_TIMEOUT (-4)     /* a bounded device-side wait ran out (reserved: no
+                                      kernel of this version waits on another)          */
+#define SCHED_ERR_NOT_FINITE (-5)  /* a host input array holds a NaN or an infinity     */
 #define SCHED_ERR_TOO_LARGE (-6)   /* a size exceeds a documented fixed maximum         */
 
 /* Limits checked by sched_init. */
@@ -97,6 +98,18 @@ typedef struct {
 int sched_init(const sched_config *cfg, const int16_t *h_node_capacity, void *cuda_stream,
                sched_ctx **out);
 
+/* The fair allocation a_f of Eq. 15, "an exclusive 1/J share of the cluster", as a (K, N)
+ * pair: fair_k = clamp(total GPUs / num_active, 1, k_max) (integer division; the whole
+ * cluster when num_active <= 0), placed on as few nodes as possible, fair_n =
+ * ceil(fair_k / largest node).  The paper leaves open what the share is when the quotient
+ * is fractional or below one GPU; this is the reading the tables are normalised with.
+ * Host-only helper, needs no context and no GPU: h_node_capacity is a HOST array
+ * [num_nodes] (negative entries count as 0); the results are what sched_jobs.fair_k /
+ * fair_n expect for every job.  Errors: INVALID_ARG (NULL pointer, num_nodes < 1,
+ * k_max < 1), BAD_CONFIG (the cluster has no GPU). */
+int sched_fair_share(const int16_t *h_node_capacity, int32_t num_nodes, int32_t num_active, int32_t k_max,
+                     int32_t *fair_k, int32_t *fair_n);
+
 /* Frees the context and its scratch.  NULL is accepted. */
 int sched_destroy(sched_ctx *ctx);
 
@@ -105,7 +118,8 @@ int sched_destroy(sched_ctx *ctx);
 const char *sched_last_error(const sched_ctx *ctx);
 
 /* Waits for the stream and returns the device-side status word (SCHED_OK unless a
- * kernel recorded an error such as an exhausted bounded wait). */
+ * kernel recorded an error, e.g. SCHED_ERR_TOO_LARGE when the row pool of a round ran
+ * out).  A recorded error is reported once: reading it clears the word. */
 int sched_sync_status(sched_ctx *ctx);
 
 /* Number of kernels this context has launched so far (for accounting in benchmarks). */
@@ -240,7 +254,14 @@ int schedule_round(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cu
 int sched_set_graphs(sched_ctx *ctx, int enable);
 
 /* Same with HOST buffers: copies the job arrays and h_cur to the device, runs the round,
- * copies the result back and waits for it.  Every member of h_jobs is a host pointer. */
+ * copies the result back and waits for it.  Every member of h_jobs is a host pointer.
+ * Because the arrays are on the host they are validated first: SCHED_ERR_NOT_FINITE when a
+ * goodput-model parameter or age_sec is NaN or infinite;
+ * SCHED_ERR_INVALID_ARG when alpha or beta is negative, gamma < 1, phi < 0, M0 < 1,
+ * m_max_total < M0, a batch size of m_grid is < 1, age_sec or num_restarts is negative, or
+ * an entry of h_cur is negative (Eq. 8-11 and Sec. 4.2 give these ranges).  The device
+ * status word is read back with the result: a device-side error of the round (see
+ * schedule_round) is this call's return value. */
 int schedule_round_host(sched_ctx *ctx, const sched_jobs *h_jobs, const int16_t *h_cur,
                         uint32_t round, int32_t generations, int16_t *h_best,
                         float *h_best_fitness);
@@ -260,7 +281,9 @@ int sched_get_round_tables(sched_ctx *ctx, float *d_goodput_out, float *d_speedu
 const float *sched_round_speedup_table(const sched_ctx *ctx);
 
 /* Fitness with HOST buffers (population, table, optional cur / factors / active mask are
- * copied in, fitness copied out, the call waits).  Staging buffers are context scratch. */
+ * copied in, fitness copied out, the call waits).  Staging buffers are context scratch.
+ * Validated first: SCHED_ERR_NOT_FINITE when h_speedup or h_realloc_factor holds a NaN or an
+ * infinity; SCHED_ERR_INVALID_ARG when a speedup is negative or a factor lies outside [0, 1]. */
 int eval_fitness_host(sched_ctx *ctx, const int16_t *h_pop, int32_t count, const float *h_speedup,
                       const int16_t *h_cur, const float *h_realloc_factor,
                       const uint8_t *h_active, float p, float *h_fitness);

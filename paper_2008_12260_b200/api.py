@@ -17,7 +17,7 @@ SCHED_OK = 0
 ERRORS = {-1: "INVALID_ARG", -2: "BAD_CONFIG", -3: "CUDA", -4: "TIMEOUT", -5: "NOT_FINITE", -6: "TOO_LARGE"}
 
 EXPORTS = (
-    "sched_init", "sched_destroy", "sched_last_error", "sched_sync_status", "sched_launch_count",
+    "sched_init", "sched_fair_share", "sched_destroy", "sched_last_error", "sched_sync_status", "sched_launch_count",
     "build_speedup_table", "build_speedup_table_msample", "fit_throughput_model", "compute_realloc_factor", "autoscale_targets", "eval_fitness", "repair_population",
     "init_population", "ga_generation", "schedule_round", "schedule_round_host",
     "sched_get_population", "sched_get_round_tables", "sched_round_speedup_table", "eval_fitness_host",
@@ -60,6 +60,7 @@ def load_library(path: str = LIB_PATH):
     vp, i32, u32, f32 = C.c_void_p, C.c_int32, C.c_uint32, C.c_float
     lib.sched_init.argtypes = [C.POINTER(SchedConfig), vp, vp, C.POINTER(vp)]
     lib.sched_destroy.argtypes = [vp]
+    lib.sched_fair_share.argtypes = [vp, i32, i32, i32, C.POINTER(i32), C.POINTER(i32)]
     lib.sched_last_error.argtypes = [vp]
     lib.sched_last_error.restype = C.c_char_p
     lib.sched_sync_status.argtypes = [vp]
@@ -111,16 +112,13 @@ def _ptr(t):
 
 
 def fair_share(node_capacity, num_active: int, k_max: int):
-    """(K_f, N_f) of the fair allocation a_f of Eq. 15, an exclusive 1/J share of the
-    cluster: K_f = clamp(total GPUs // active jobs, 1, k_max), placed on as few nodes as
-    possible, N_f = ceil(K_f / largest node).  Host-side input preparation."""
-    cap = np.maximum(np.asarray(node_capacity, dtype=np.int64), 0)
-    big = int(cap.max())
-    if big <= 0:
-        raise ValueError("cluster has no GPUs")
-    k = int(cap.sum()) // num_active if num_active > 0 else int(cap.sum())
-    k = min(max(k, 1), int(k_max))
-    return k, -(-k // big)
+    """(K_f, N_f) of the fair allocation a_f of Eq. 15 from sched_fair_share (host-only)."""
+    cap = np.ascontiguousarray(node_capacity, dtype=np.int16)
+    fk, fn = C.c_int32(0), C.c_int32(0)
+    rc = _lib.sched_fair_share(cap.ctypes.data, cap.shape[0], int(num_active), int(k_max), C.byref(fk), C.byref(fn))
+    if rc != SCHED_OK:
+        raise SchedError(rc, _lib.sched_last_error(None).decode())
+    return fk.value, fn.value
 
 
 class DeviceJobs:

@@ -264,6 +264,26 @@ int sched_init(const sched_config *cfg, const int16_t *h_node_capacity, void *cu
   return SCHED_OK;
 }
 
+int sched_fair_share(const int16_t *h_node_capacity, int32_t num_nodes, int32_t num_active, int32_t k_max,
+                     int32_t *fair_k, int32_t *fair_n) {
+  REQUIRE(nullptr, h_node_capacity && fair_k && fair_n, SCHED_ERR_INVALID_ARG,
+          "sched_fair_share: h_node_capacity, fair_k and fair_n must be non-NULL");
+  REQUIRE(nullptr, num_nodes >= 1 && k_max >= 1, SCHED_ERR_INVALID_ARG,
+          "sched_fair_share: num_nodes and k_max must be positive");
+  long long total = 0, largest = 0;
+  for (int32_t n = 0; n < num_nodes; ++n) {
+    const long long g = h_node_capacity[n] > 0 ? h_node_capacity[n] : 0;
+    total += g;
+    largest = std::max(largest, g);
+  }
+  REQUIRE(nullptr, largest > 0, SCHED_ERR_BAD_CONFIG, "sched_fair_share: the cluster has no GPU");
+  long long k = num_active > 0 ? total / num_active : total;
+  k = std::min<long long>(std::max<long long>(k, 1), k_max);
+  *fair_k = (int32_t)k;
+  *fair_n = (int32_t)((k + largest - 1) / largest);
+  return SCHED_OK;
+}
+
 int sched_destroy(sched_ctx *ctx) {
   if (!ctx) return SCHED_OK;
   cudaStreamSynchronize(ctx->stream);
@@ -289,7 +309,10 @@ int sched_sync_status(sched_ctx *ctx) {
   int status = 0;
   SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(&status, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
   SCHED_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
-  if (status != SCHED_OK) set_error(ctx, "a kernel recorded device status %d", status);
+  if (status != SCHED_OK) {
+    set_error(ctx, "a kernel recorded device status %d", status);
+    cudaMemsetAsync(ctx->d_status, 0, sizeof(int), ctx->stream);   // reported once; the context stays usable
+  }
   return status;
 }
 
@@ -651,6 +674,59 @@ const float *sched_round_speedup_table(const sched_ctx *ctx) {
 
 static size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
+// Host-side checks of arrays that arrive in host memory.  first_bad: index of the first entry
+// that is NaN / infinite (kind 1) or below `lo` / above `hi` (kind 2), or -1.
+static long long first_bad(const float *a, size_t n, float lo, float hi, int &kind) {
+  for (size_t i = 0; i < n; ++i) {
+    const float v = a[i];
+    if (!(v - v == 0.f)) { kind = 1; return (long long)i; }       // NaN or +-inf
+    if (v < lo || v > hi) { kind = 2; return (long long)i; }
+  }
+  return -1;
+}
+
+#define CHECK_HOST_F32(ctx, who, name, ptr, n, lo, hi)                                              \
+  do {                                                                                              \
+    int kind__ = 0;                                                                                 \
+    const long long at__ = (ptr) ? first_bad((ptr), (n), (lo), (hi), kind__) : -1;                  \
+    if (at__ >= 0) {                                                                                \
+      set_error(ctx, "%s: %s[%lld] = %g is %s", who, name, at__, (double)(ptr)[at__],               \
+                kind__ == 1 ? "not finite" : "outside its range");                                  \
+      return kind__ == 1 ? SCHED_ERR_NOT_FINITE : SCHED_ERR_INVALID_ARG;                            \
+    }                                                                                               \
+  } while (0)
+
+static int validate_host_jobs(sched_ctx *ctx, const sched_jobs *h, const int16_t *h_cur) {
+  const sched_config &c = ctx->cfg;
+  const size_t J = (size_t)c.num_jobs;
+  const float big = 3.0e38f;
+  const char *who = "schedule_round_host";
+  CHECK_HOST_F32(ctx, who, "alpha_grad", h->alpha_grad, J, 0.f, big);
+  CHECK_HOST_F32(ctx, who, "beta_grad", h->beta_grad, J, 0.f, big);
+  CHECK_HOST_F32(ctx, who, "alpha_local", h->alpha_local, J, 0.f, big);
+  CHECK_HOST_F32(ctx, who, "beta_local", h->beta_local, J, 0.f, big);
+  CHECK_HOST_F32(ctx, who, "alpha_node", h->alpha_node, J, 0.f, big);
+  CHECK_HOST_F32(ctx, who, "beta_node", h->beta_node, J, 0.f, big);
+  CHECK_HOST_F32(ctx, who, "gamma", h->gamma, J, 1.f, big);
+  CHECK_HOST_F32(ctx, who, "phi", h->phi, J, 0.f, big);
+  CHECK_HOST_F32(ctx, who, "m0", h->m0, J, 1.f, big);
+  CHECK_HOST_F32(ctx, who, "m_max_total", h->m_max_total, J, 1.f, big);
+  CHECK_HOST_F32(ctx, who, "age_sec", h->age_sec, J, 0.f, big);
+  for (size_t j = 0; j < J; ++j) {
+    REQUIRE(ctx, h->m_max_total[j] >= h->m0[j], SCHED_ERR_INVALID_ARG,
+            "schedule_round_host: m_max_total[%zu] = %g is below m0 = %g", j, (double)h->m_max_total[j], (double)h->m0[j]);
+    REQUIRE(ctx, !h->num_restarts || h->num_restarts[j] >= 0, SCHED_ERR_INVALID_ARG,
+            "schedule_round_host: num_restarts[%zu] is negative", j);
+  }
+  for (size_t i = 0; i < J * (size_t)c.grid_m; ++i)
+    REQUIRE(ctx, h->m_grid[i] >= 1, SCHED_ERR_INVALID_ARG, "schedule_round_host: m_grid[%zu] = %d is below 1", i,
+            (int)h->m_grid[i]);
+  if (h_cur)
+    for (size_t i = 0; i < J * (size_t)c.num_nodes; ++i)
+      REQUIRE(ctx, h_cur[i] >= 0, SCHED_ERR_INVALID_ARG, "schedule_round_host: h_cur[%zu] is negative", i);
+  return SCHED_OK;
+}
+
 int schedule_round_host(sched_ctx *ctx, const sched_jobs *h_jobs, const int16_t *h_cur, uint32_t round,
                         int32_t generations, int16_t *h_best, float *h_best_fitness) {
   REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "schedule_round_host: ctx is NULL");
@@ -658,6 +734,7 @@ int schedule_round_host(sched_ctx *ctx, const sched_jobs *h_jobs, const int16_t 
   if (rc != SCHED_OK) return rc;
   REQUIRE(ctx, h_best && h_best_fitness, SCHED_ERR_INVALID_ARG,
           "schedule_round_host: h_best and h_best_fitness must be non-NULL");
+  if ((rc = validate_host_jobs(ctx, h_jobs, h_cur)) != SCHED_OK) return rc;
   const sched_config &c = ctx->cfg;
   const size_t J = (size_t)c.num_jobs, mat = J * c.num_nodes * sizeof(int16_t);
   // layout of the staging buffer: 10 fp32 arrays, m_grid, k_cap, fair_k, fair_n, age,
@@ -727,8 +804,14 @@ int schedule_round_host(sched_ctx *ctx, const sched_jobs *h_jobs, const int16_t 
   if (rc != SCHED_OK) return rc;
   SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(h_best, d_best, mat, cudaMemcpyDeviceToHost, ctx->stream));
   SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(h_best_fitness, d_bf, sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
+  int status = SCHED_OK;   // the call waits anyway: a device-side error of the round is its result
+  SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(&status, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
   SCHED_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
-  return SCHED_OK;
+  if (status != SCHED_OK) {
+    set_error(ctx, "schedule_round_host: a kernel recorded device status %d", status);
+    cudaMemsetAsync(ctx->d_status, 0, sizeof(int), ctx->stream);
+  }
+  return status;
 }
 
 int eval_fitness_host(sched_ctx *ctx, const int16_t *h_pop, int32_t count, const float *h_speedup,
@@ -740,6 +823,8 @@ int eval_fitness_host(sched_ctx *ctx, const int16_t *h_pop, int32_t count, const
   if (count == 0) return SCHED_OK;
   const sched_config &c = ctx->cfg;
   const size_t J = (size_t)c.num_jobs, mat = J * c.num_nodes * sizeof(int16_t);
+  CHECK_HOST_F32(ctx, "eval_fitness_host", "h_speedup", h_speedup, J * ctx->KD * ctx->ND, 0.f, 3.0e38f);
+  CHECK_HOST_F32(ctx, "eval_fitness_host", "h_realloc_factor", h_realloc_factor, J, 0.f, 1.f);
   const size_t pop_b = align256(mat * count), tab_b = align256(J * ctx->KD * ctx->ND * 4);
   const size_t need = pop_b + tab_b + align256(mat) + align256(J * 4) + align256(J) + align256((size_t)count * 4);
   if (need > ctx->stage_fit_bytes) {

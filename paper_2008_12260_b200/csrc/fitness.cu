@@ -354,10 +354,15 @@ namespace {
 
 constexpr int NOALLOC_MAX_COUNT = SCHED_NOALLOC_MAX_COUNT;
 constexpr int NOALLOC_MAX_JOBS = SCHED_NOALLOC_MAX_JOBS;
-constexpr int NOALLOC_MAX_CHUNKS = NOALLOC_MAX_JOBS / 256;   // a block covers at least 256 rows
+// Chunk sums are stored flat, candidate-major: (candidate * chunks + chunk) * 2.  The geometry
+// gives at most NOALLOC_MAX_JOBS / 256 chunks per candidate unless it halves the rows of a block
+// to fill the GPU, which it only does while count * chunks < 4 * SMs: a halving at most doubles
+// the chunks, so count * chunks then stays below 8 * SMs.  Either way count * chunks fits
+// NOALLOC_MAX_PARTIALS for every size within the documented limits (checked again per call).
+constexpr size_t NOALLOC_MAX_PARTIALS = (size_t)NOALLOC_MAX_COUNT * (NOALLOC_MAX_JOBS / 256);
 
 struct NoAllocScratch {
-  double partial[(size_t)NOALLOC_MAX_COUNT * NOALLOC_MAX_CHUNKS * 2];
+  double partial[NOALLOC_MAX_PARTIALS * 2];
   unsigned int ticket[NOALLOC_MAX_COUNT];
   float pen[NOALLOC_MAX_JOBS];
 };
@@ -440,8 +445,8 @@ int eval_fitness_noalloc(const int16_t *d_pop, int32_t count, int32_t num_jobs, 
   int W, lpr_log2, rows_per_block, chunks;
   fitness_geometry((size_t)num_nodes * 2, (uintptr_t)d_pop | (penalise ? (uintptr_t)d_cur : 0), J, count,
                    g_noalloc_sms[device], W, lpr_log2, rows_per_block, chunks);
-  if (chunks > NOALLOC_MAX_CHUNKS)
-    return noalloc_fail(SCHED_ERR_TOO_LARGE, "eval_fitness_noalloc: internal chunk count exceeds the scratch array");
+  if ((size_t)count * (size_t)chunks > NOALLOC_MAX_PARTIALS)   // cannot happen within the limits above
+    return noalloc_fail(SCHED_ERR_TOO_LARGE, "eval_fitness_noalloc: chunk sums exceed the scratch array");
 
   FitnessArgs a;
   a.pop = d_pop;

@@ -128,7 +128,7 @@ def test_store_round_equals_dense_stepwise_round(gpu, oracle, cfg):
     rf_ref = oracle.realloc_factor(jobs.age_sec, jobs.num_restarts, cfg.delta_sec) if penalise else None
     fit_ref = oracle.eval_fitness(pop, sp.astype(np.float64), cl.k_max, cl.n_max, cfg.p, cfg.speedup_floor,
                                   cur=cur, realloc=rf_ref, active=jobs.active)
-    assert_close(fit, fit_ref, rel=3 * REL_TOL, what="fitness of the final population")
+    assert_close(fit, fit_ref, what="fitness of the final population")
     s.close()
 
 

@@ -50,7 +50,7 @@ def test_large_config_sampled_jobs(gpu, oracle):
     cfg = synth.LARGE
     cl, jobs = setup(cfg)
     gp, sp, am = _gpu_table(gpu, cl, jobs, cfg.grid_s)
-    idx = np.array([0, 1, 17, 255, 256, 511, 777, 1000, 1023])
+    idx = np.unique(np.concatenate([np.arange(0, 1024, 16), [1, 17, 255, 256, 511, 777, 1000, 1023]]))   # 71 jobs
     sub = jobs.take(idx)
     gp_r, sp_r, am_r = oracle.build_speedup_table(sub, cl.node_capacity, cl.k_max, cl.n_max, cfg.grid_s)
     check_table(oracle, sub, cfg.grid_s, gp[idx], sp[idx], am[idx], gp_r, sp_r, am_r)

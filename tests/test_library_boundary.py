@@ -82,3 +82,35 @@ def test_fair_share_helper_matches_oracle(oracle):
         n_act = int(rng.integers(0, 300))
         k_max = min(int(cap.sum()), 64)
         assert api.fair_share(cap, n_act, k_max) == oracle.fair_share(cap, n_act, k_max)
+
+
+def test_fair_share_raw_abi_errors(lib):
+    fk, fn = ctypes.c_int32(-7), ctypes.c_int32(-7)
+    cap = np.array([4, 0, 8, -3], np.int16)
+    f = lib.sched_fair_share
+    f.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                  ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
+    assert f(cap.ctypes.data, 4, 5, 64, ctypes.byref(fk), ctypes.byref(fn)) == 0
+    assert (fk.value, fn.value) == (2, 1)            # 12 GPUs over 5 jobs; the negative node counts as empty
+    assert f(cap.ctypes.data, 4, 1, 64, ctypes.byref(fk), ctypes.byref(fn)) == 0
+    assert (fk.value, fn.value) == (12, 2)           # ceil(12 / largest node 8)
+    assert f(cap.ctypes.data, 4, 1, 5, ctypes.byref(fk), ctypes.byref(fn)) == 0 and fk.value == 5
+    assert f(cap.ctypes.data, 4, 100, 64, ctypes.byref(fk), ctypes.byref(fn)) == 0 and (fk.value, fn.value) == (1, 1)
+    assert f(None, 4, 5, 64, ctypes.byref(fk), ctypes.byref(fn)) == -1
+    assert f(cap.ctypes.data, 0, 5, 64, ctypes.byref(fk), ctypes.byref(fn)) == -1
+    assert f(cap.ctypes.data, 4, 5, 0, ctypes.byref(fk), ctypes.byref(fn)) == -1
+    empty = np.zeros(3, np.int16)
+    assert f(empty.ctypes.data, 3, 5, 64, ctypes.byref(fk), ctypes.byref(fn)) == -2
+
+
+def test_reference_arm_inputs_do_not_load_the_product_library():
+    """bench.py --impl reference times the oracle; preparing its inputs must not even import the
+    binding (which would dlopen the CUDA library)."""
+    import subprocess
+    import sys
+    code = ("import sys; sys.argv=['bench.py']; import bench, oracle; "
+            "bench.large_inputs(0, oracle.fair_share); "
+            "assert 'paper_2008_12260_b200.api' not in sys.modules; "
+            "assert 'libpolluxsched' not in open('/proc/self/maps').read(); print('ok')")
+    out = subprocess.run([sys.executable, "-c", code], cwd=ROOT, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0 and "ok" in out.stdout, out.stderr
