@@ -211,14 +211,14 @@ __device__ __forceinline__ int nth_occupied_row(const Grp &g, const int16_t *row
   return __shfl_sync(g.mask, node, who ? __ffs(who) - 1 : (__ffs(g.mask) - 1));
 }
 
-// one 32-byte record with a single request
+// One 32-byte record with a single request, read from L2: records may have been written by the
+// previous kernel, which can still be running when this one starts (programmatic dependent
+// launch), so a line cached in this SM's L1 before that write must not serve the load.
 __device__ __forceinline__ void load_record(uint32_t (&r)[REC_WORDS], const uint32_t *p) {
-  asm volatile("ld.global.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+  asm volatile("ld.global.cg.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
                : "l"(p) : "memory");
 }
-
-__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 __device__ __forceinline__ uint32_t pack_summary(int K, int N, int ndiff) {
   return (uint32_t)K | ((uint32_t)N << 11) | ((uint32_t)ndiff << 22);
@@ -273,7 +273,8 @@ __global__ void __launch_bounds__(256) rowstore_build_kernel(BuildArgs a) {
   }
 }
 
-// most slots one generation can take: every row new, plus every block's reserve
+// most slots one generation can take: every row new (a row gets at most one slot per generation:
+// perturbed, or copied when the column pass first changes it), plus every block's reserve
 __host__ __device__ inline unsigned long long store_worst_case(int P, int J) {
   return (unsigned long long)P * J + (unsigned long long)P * COW_RESERVE;
 }
@@ -313,10 +314,13 @@ __global__ void __launch_bounds__(256) rowstore_compact_kernel(CompactArgs a) {
     const uint32_t slot = a.ptr[r];
     if (slot == a.st.zero_slot) continue;
     const size_t dst = (size_t)(base + r);
-    const uint4 *s4 = (const uint4 *)(a.st.pool + (size_t)slot * a.NN);
-    uint4 *d4 = (uint4 *)(a.st.pool + dst * a.NN);
-    for (int v = lane; v < row_vecs; v += 32) d4[v] = s4[v];
-    if (lane < REC_WORDS) a.st.rec[dst * REC_WORDS + lane] = a.st.rec[(size_t)slot * REC_WORDS + lane];
+    const uint32_t w = (lane < REC_WORDS) ? a.st.rec[(size_t)slot * REC_WORDS + lane] : 0u;
+    if (__shfl_sync(0xffffffffu, w, 0) == REC_OVERFLOW) {   // the record does not hold the row: its contents move too
+      const uint4 *s4 = (const uint4 *)(a.st.pool + (size_t)slot * a.NN);
+      uint4 *d4 = (uint4 *)(a.st.pool + dst * a.NN);
+      for (int v = lane; v < row_vecs; v += 32) d4[v] = s4[v];
+    }
+    if (lane < REC_WORDS) a.st.rec[dst * REC_WORDS + lane] = w;
     if (lane == 0) a.ptr[r] = (uint32_t)dst;
   }
 }
@@ -334,12 +338,40 @@ rowstore_gather_kernel(StoreView st, const uint32_t *__restrict__ ptr, int first
   const bool aligned = ((uintptr_t)out & 15) == 0;
   for (long long r = (long long)blockIdx.x * 8 + warp; r < rows; r += (long long)gridDim.x * 8) {
     const uint32_t slot = ptr[first + r];
-    if (aligned) {
-      const uint4 *s4 = (const uint4 *)(st.pool + (size_t)slot * NN);
-      uint4 *d4 = (uint4 *)(out + (size_t)r * NN);
-      for (int v = lane; v < row_vecs; v += 32) d4[v] = s4[v];
-    } else {
-      for (int n = lane; n < NN; n += 32) out[(size_t)r * NN + n] = st.pool[(size_t)slot * NN + n];
+    // every lane reads the row's record (one address: a broadcast)
+    const uint4 lo = *((const uint4 *)(st.rec + (size_t)slot * REC_WORDS));
+    const uint4 hi = *((const uint4 *)(st.rec + (size_t)slot * REC_WORDS) + 1);
+    if (lo.x == REC_OVERFLOW) {          // more occupied nodes than a record holds: the contents are in the pool
+      if (aligned) {
+        const uint4 *s4 = (const uint4 *)(st.pool + (size_t)slot * NN);
+        uint4 *d4 = (uint4 *)(out + (size_t)r * NN);
+        for (int v = lane; v < row_vecs; v += 32) d4[v] = s4[v];
+      } else {
+        for (int n = lane; n < NN; n += 32) out[(size_t)r * NN + n] = st.pool[(size_t)slot * NN + n];
+      }
+      continue;
+    }
+    const uint32_t e[REC_ENTRIES] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y};
+    for (int v = lane; v < row_vecs; v += 32) {   // the row laid out from the record, a piece per lane
+      uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+      for (int k = 0; k < REC_ENTRIES; ++k) {
+        const int node = (int)(e[k] & 0xFFFu);
+        if (e[k] && (node >> 3) == v) {
+          const uint32_t val = ((e[k] >> 12) & 0x7FFu) << ((node & 1) * 16);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) w[q] |= (((node & 7) >> 1) == q) ? val : 0u;
+        }
+      }
+      if (aligned) {
+        ((uint4 *)(out + (size_t)r * NN))[v] = make_uint4(w[0], w[1], w[2], w[3]);
+      } else {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          out[(size_t)r * NN + 8 * v + 2 * q] = (int16_t)(w[q] & 0xFFFFu);
+          out[(size_t)r * NN + 8 * v + 2 * q + 1] = (int16_t)(w[q] >> 16);
+        }
+      }
     }
   }
 }
@@ -349,7 +381,7 @@ rowstore_gather_kernel(StoreView st, const uint32_t *__restrict__ ptr, int first
 // ---------------------------------------------------------------------------------------
 struct GenArgs {
   StoreView st;
-  const uint32_t *ptr_in;   // [P][J] parents
+  const uint32_t *ptr_in;   // [P][J] parents ([J] for the initial population: the current allocation's rows)
   uint32_t *ptr_out;        // [P][J] children
   unsigned int *state;      // {next free slot, half}
   const int16_t *cap;       // [NN]
@@ -358,7 +390,8 @@ struct GenArgs {
   const uint32_t *fitness_bits;  // [P] parents' fitness
   const int16_t *cur;       // [J][NN] or NULL
   int P, J, NN, k_max, n_max, num_elite;
-  uint32_t thr, gen;
+  uint32_t thr, gen;        // perturbation threshold; generation number of the draws
+  uint32_t init_src;        // initial population: slot of job 0's row before the row caps (perturbation source)
   RngKey key;
   TermParams tp;
   int rows_per_chunk, chunks;   // the dense fitness kernel's chunking, reproduced for identical sums
@@ -366,17 +399,211 @@ struct GenArgs {
   int *status;
 };
 
+// ---- a row as the list of its occupied nodes, which is what a record holds ---------------------
+// e[0 .. n) = node | GPUs << 12 in ascending node order, K = GPUs in the row, nd = entries that
+// differ from the current allocation's row.  One entry more than a record holds, so that a
+// perturbation may add a node before the row caps take one away again.  Few rows of a generation
+// are edited, each by one thread, so the helpers are plain loops (kept rolled: the kernel's
+// instruction footprint matters more than their speed) over eight words of shared memory that
+// belong to the thread.
+constexpr int LIST_MAX = REC_ENTRIES + 1;
+constexpr int LIST_WORDS = LIST_MAX + 1;
+
+struct RowList {
+  uint32_t *e;          // LIST_WORDS words of the thread's own
+  int n, K, nd;
+  // up to two entries changed by the perturbation whose effect on nd is still to be worked out
+  // (their current-allocation values are fetched together, with the row's speedup, once K and N
+  // are known)
+  int pn, pnode0, pold0, pnew0, pnode1, pold1, pnew1;
+};
+
+__device__ __forceinline__ int ent_node(uint32_t e) { return (int)(e & 0xFFFu); }
+__device__ __forceinline__ int ent_gpus(uint32_t e) { return (int)((e >> 12) & 0x7FFu); }
+
+// fitness term of a row of job j from its summary: speedup looked up at (K, N), penalty when the
+// row differs from the current allocation, floor, and the form that the mode sums (one copy of
+// this code for all its users)
+__device__ __noinline__ float row_term_from(bool has_pen, int mode, float p, float floor_, float x_sp, float x_pen,
+                                            bool changed) {
+  TermParams tp;
+  tp.table = nullptr; tp.pen = nullptr; tp.active = nullptr;
+  tp.k_max = 0; tp.n_max = 0; tp.mode = mode; tp.p = p; tp.floor_ = floor_;
+  // the re-allocation penalty is applied here, the rest (floor, the form the mode sums) is shared
+  return fitness_term_with(tp, (has_pen && changed) ? x_sp * x_pen : x_sp, 1.f, false);
+}
+
+__device__ __forceinline__ float row_term_of(const float *table, const float *pen, int k_max, int n_max, int mode, float p,
+                                             float floor_, int j, int K, int N, int nd) {
+  TermParams tp;
+  tp.k_max = k_max; tp.n_max = n_max;
+  const float x_sp = __ldg(table + fitness_table_index(tp, j, K, N));
+  const float x_pen = (pen && nd != 0) ? __ldg(pen + j) : 1.f;
+  return row_term_from(pen != nullptr, mode, p, floor_, x_sp, x_pen, nd != 0);
+}
+
+// one call of the random stream (one copy of the ten rounds for all users in this file)
+__device__ __noinline__ u32x4 draw_call(uint32_t k0, uint32_t k1, uint32_t idx, uint32_t cand, uint32_t gen, uint32_t slot) {
+  const u32x4 c = {idx, cand, gen, slot};
+  return philox4x32_10(c, k0, k1);
+}
+
+// GPUs of the row on `node` (0 when the node is not occupied) and where its entry is or belongs
+__device__ __forceinline__ int list_find(const RowList &r, int node, int &pos, bool &found) {
+  int v = 0;
+  pos = 0;
+  found = false;
+#pragma unroll 1
+  for (int k = 0; k < r.n; ++k) {
+    const int nk = ent_node(r.e[k]);
+    if (nk < node) pos = k + 1;
+    if (nk == node) { found = true; v = ent_gpus(r.e[k]); }
+  }
+  return v;
+}
+
+// change in the count of entries that differ from the current allocation when A[j][node] goes
+// from v_old to v_new
+__device__ __forceinline__ int diff_delta(const int16_t *cur, int NN, int j, int node, int v_old, int v_new) {
+  if (!cur) return 0;
+  const int cv = (int)__ldg(cur + (size_t)j * NN + node);
+  return (int)(v_new != cv) - (int)(v_old != cv);
+}
+
+// A[j][node] = v_new on the list form of row j (nd is brought up to date later, see RowList)
+__device__ __forceinline__ void list_put(RowList &r, int node, int v_new) {
+  int pos;
+  bool found;
+  const int v_old = list_find(r, node, pos, found);
+  if (v_new == v_old) return;
+  if (r.pn == 0) { r.pnode0 = node; r.pold0 = v_old; r.pnew0 = v_new; }
+  else { r.pnode1 = node; r.pold1 = v_old; r.pnew1 = v_new; }
+  r.pn += 1;
+  r.K += v_new - v_old;
+  const uint32_t ent = (uint32_t)node | ((uint32_t)v_new << 12);
+  if (found && v_new > 0) {
+    r.e[pos] = ent;
+  } else if (found) {            // the entry goes: the ones above it move down
+#pragma unroll 1
+    for (int k = pos; k + 1 < r.n; ++k) r.e[k] = r.e[k + 1];
+    r.n -= 1;
+    r.e[r.n] = 0u;
+  } else if (r.n < LIST_MAX) {   // a new entry: the ones above its place move up
+#pragma unroll 1
+    for (int k = r.n; k > pos; --k) r.e[k] = r.e[k - 1];
+    r.e[pos] = ent;
+    r.n += 1;
+  }
+}
+
+// the perturbation of a row (grow / shrink / relocate, chosen by the row's draw `mw`)
+__device__ __forceinline__ void list_perturb(int NN, RowList &r, const u32x4 &mw, const int16_t *s_cap) {
+  const uint32_t op = bounded(mw.y, 3u);
+  int pos;
+  bool found;
+  int node0 = -1, val0 = 0, node1 = -1, val1 = 0;   // up to two entries change
+  if (op == 0u) {
+    node0 = (int)bounded(mw.w, (uint32_t)NN);
+    val0 = min(list_find(r, node0, pos, found) + 1, (int)s_cap[node0]);
+  } else if (r.n > 0) {
+    const uint32_t ent = r.e[bounded(mw.z, (uint32_t)r.n)];
+    const int ns = ent_node(ent), vs = ent_gpus(ent);
+    if (op == 1u) {
+      node0 = ns;
+      val0 = vs - 1;
+    } else {
+      const int nd = (int)bounded(mw.w, (uint32_t)NN);
+      if (nd != ns) {
+        node0 = nd;
+        val0 = min(list_find(r, nd, pos, found) + vs, (int)s_cap[nd]);
+        node1 = ns;
+        val1 = 0;
+      }
+    }
+  }
+#pragma unroll 1
+  for (int q = 0; q < 2; ++q) {
+    const int node = q ? node1 : node0, val = q ? val1 : val0;
+    if (node >= 0) list_put(r, node, val);
+  }
+}
+
+// per-row caps: replicas above kc leave from the highest node index down, then occupied nodes
+// beyond n_max are cleared from the highest index down
+__device__ __forceinline__ void list_caps(const int16_t *cur, int NN, int n_max, RowList &r, int j, int kc) {
+  if (r.K > kc) {
+    int excess = r.K - kc;
+#pragma unroll 1
+    for (int k = r.n - 1; k >= 0 && excess > 0; --k) {
+      const int node = ent_node(r.e[k]), v = ent_gpus(r.e[k]);
+      const int take = min(v, excess);
+      excess -= take;
+      r.nd += diff_delta(cur, NN, j, node, v, v - take);
+      if (v - take > 0) r.e[k] = (uint32_t)node | ((uint32_t)(v - take) << 12);
+      else { r.e[k] = 0u; r.n = k; }      // everything above it has gone already
+    }
+    r.K = kc;
+  }
+#pragma unroll 1
+  for (int k = r.n - 1; k >= n_max; --k) {
+    const int node = ent_node(r.e[k]), v = ent_gpus(r.e[k]);
+    r.K -= v;
+    r.nd += diff_delta(cur, NN, j, node, v, 0);
+    r.e[k] = 0u;
+    r.n = k;
+  }
+}
+
+__device__ __forceinline__ void list_from_record(RowList &r, uint32_t *words, uint4 lo, uint4 hi) {
+  r.e = words;
+  r.pnode0 = r.pold0 = r.pnew0 = r.pnode1 = r.pold1 = r.pnew1 = 0;
+  r.e[0] = lo.x; r.e[1] = lo.y; r.e[2] = lo.z; r.e[3] = lo.w; r.e[4] = hi.x; r.e[5] = hi.y; r.e[6] = 0u; r.e[7] = 0u;
+  r.K = (int)(hi.w & 0x7FFu);
+  r.n = (int)((hi.w >> 11) & 0x7FFu);
+  r.nd = (int)(hi.w >> 22);
+  r.pn = 0;
+}
+
+// a record written by one thread: two 16-byte stores
+__device__ __forceinline__ void store_record(uint32_t *rec, const RowList &r, float term, uint32_t word) {
+  ((uint4 *)rec)[0] = make_uint4(r.e[0], r.e[1], r.e[2], r.e[3]);
+  ((uint4 *)rec)[1] = make_uint4(r.e[4], r.e[5], __float_as_uint(term), word);
+}
+
+__device__ __forceinline__ uint4 piece_with(uint4 x, int h, int val) {   // entry h of the piece set to val
+  const uint32_t sh = (uint32_t)(h & 1) * 16u, m = 0xFFFFu << sh, v = ((uint32_t)val & 0xFFFFu) << sh;
+  if (h < 2) x.x = (x.x & ~m) | v;
+  else if (h < 4) x.y = (x.y & ~m) | v;
+  else if (h < 6) x.z = (x.z & ~m) | v;
+  else x.w = (x.w & ~m) | v;
+  return x;
+}
+
+// GPUs that the row stored in `slot` holds on node nn: from its record, or from its contents when
+// the record does not hold the row (read from L2: the row may be new in this kernel)
+__device__ __noinline__ int row_value_at(const uint32_t *rec, const int16_t *pool, int NN, uint32_t slot, int nn) {
+  const uint4 lo = __ldcg((const uint4 *)(rec + (size_t)slot * REC_WORDS));
+  if (lo.x == REC_OVERFLOW) return (int)__ldcg(pool + (size_t)slot * NN + nn);
+  const uint4 hi = __ldcg((const uint4 *)(rec + (size_t)slot * REC_WORDS) + 1);
+  const uint32_t e[REC_ENTRIES] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y};
+  int v = 0;
+#pragma unroll
+  for (int k = 0; k < REC_ENTRIES; ++k)
+    if (e[k] && ent_node(e[k]) == nn) v = ent_gpus(e[k]);
+  return v;
+}
+
 // what the per-node repair decides for the occupant held by this lane of a group (entry = job |
 // GPUs << 13 | distributed << 31 in the first have_n <= 16 lanes): the GPUs the job keeps on the node
-__device__ __forceinline__ int decide_entries(const GenArgs &a, const Grp &g, uint32_t c, int nn, int tot, int ne,
-                                              int cap_n, uint32_t entry, int have_n) {
+__device__ __forceinline__ int decide_entries(const GenArgs &a, uint32_t rkey, const Grp &g, uint32_t c, int nn, int tot,
+                                              int ne, int cap_n, uint32_t entry, int have_n) {
   const int J = a.J;
   const bool have = g.sub < have_n;
   const int j = (int)(entry & 0x1FFFu);
   int v = have ? (int)((entry >> 13) & 0x7FFu) : 0;
   const bool dist = have && (entry >> 31);
   if (ne >= 2) {
-    const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
+    const int o = (int)bounded(draw_call(a.key.k0, rkey, (uint32_t)nn, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
     int t = J;
     if (dist && v > 0) { t = j - o; if (t < 0) t += J; }
     int best = t;
@@ -388,7 +615,7 @@ __device__ __forceinline__ int decide_entries(const GenArgs &a, const Grp &g, ui
   }
   const int excess = tot - cap_n;
   if (excess > 0) {
-    const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J);
+    const int o = (int)bounded(draw_call(a.key.k0, rkey, (uint32_t)nn, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J);
     int rot = 0x7fffffff;
     if (have) { rot = j - o; if (rot < 0) rot += J; }
     int ahead = 0;                       // GPUs of the occupants that come first in rotated order
@@ -402,144 +629,198 @@ __device__ __forceinline__ int decide_entries(const GenArgs &a, const Grp &g, ui
   return v;
 }
 
+// perturbed rows of a block whose draw (and replica cap) is kept from the prologue; further ones
+// draw again when their turn comes
+constexpr int MUT_STASH = 128;
+
 // Shared-memory carve-up of the generation kernel (sizes in bytes, 16-byte aligned pieces).
 struct GenSmem {
-  size_t slot, summ, term, mark, acc, viol, viollist, occ, rowbuf, mut, ovf, mod, cap, rec, total;
+  size_t slot, term, mark, acc, viol, occ, rowbuf, mut, ovf, slow, mod, cap, rec, sums, stash, total;
 };
+
+// most chunks the fitness chunking can cut J rows into (a block of the dense kernel covers at
+// least 129 rows unless the whole candidate is smaller)
+__host__ __device__ inline int gen_max_chunks(int J) { return J / 129 + 2; }
 
 __host__ __device__ inline GenSmem gen_smem_layout(int J, int NN) {
   GenSmem L;
   size_t off = 0;
 #define TAKE(field, bytes) do { L.field = off; off += ((size_t)(bytes) + 15) & ~(size_t)15; } while (0)
   TAKE(slot, (size_t)J * 4);
-  TAKE(summ, (size_t)J * 4);
   TAKE(term, (size_t)J * 4);
   TAKE(mark, (size_t)J * 4);
   TAKE(acc, (size_t)NN * 8);
   TAKE(viol, (size_t)NN);
-  TAKE(viollist, (size_t)NN * 2);
   TAKE(occ, (size_t)NN * OCC * 4);
-  // a row per group of 16 lanes
-  TAKE(rowbuf, (size_t)GEN_GROUPS * NN * 2);
+  // a row per group of 16 lanes; at other times eight words per thread for the list form of a row
+  TAKE(rowbuf, (size_t)GEN_GROUPS * NN * 2 > (size_t)GEN_THREADS * LIST_WORDS * 4 ? (size_t)GEN_GROUPS * NN * 2
+                                                                                     : (size_t)GEN_THREADS * LIST_WORDS * 4);
   TAKE(mut, (size_t)J * 2);
   TAKE(ovf, (size_t)J * 2);
+  TAKE(slow, (size_t)J * 2);
   TAKE(mod, (size_t)J * 2);
   TAKE(cap, (size_t)NN * 2);
   TAKE(rec, (size_t)GEN_GROUPS * REC_WORDS * 4);
+  TAKE(sums, (size_t)gen_max_chunks(J) * GEN_WARPS * 12);
+  TAKE(stash, (size_t)MUT_STASH * 16);
 #undef TAKE
   L.total = off;
   return L;
 }
 
-// Column value of job j on node nn as the capacity pass must see it: zero when the
-// interference pass removes it.
-__device__ __forceinline__ int column_value(const GenArgs &a, const uint32_t *s_slot, const uint32_t *s_summ, int j,
-                                            int nn, int keep, bool intf, bool &dist) {
-  const int v = (int)a.st.pool[(size_t)s_slot[j] * a.NN + nn];
-  dist = ((s_summ[j] >> 11) & 0x7FFu) >= 2u;
-  if (intf && dist && v > 0 && j != keep) return 0;
-  return v;
+// flags of a row inside a block (s_mark); bits 4.. hold the row's place among the perturbed rows
+constexpr int MARK_CHANGED = 1;   // the column pass changes the row
+constexpr int MARK_OWN = 2;       // the row's slot was made in this generation (rewritten in place)
+constexpr int MARK_DIST = 4;      // the row spanned two nodes or more after the row pass (interference snapshot)
+
+// block-wide minimum / exclusive prefix sum of one int per thread (s_red: GEN_WARPS + 1 ints);
+// both end with a barrier, so s_red can be reused at once
+__device__ __forceinline__ int block_min(int v, int *s_red) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) v = min(v, __shfl_xor_sync(0xffffffffu, v, off));
+  if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  int r = s_red[0];
+#pragma unroll
+  for (int w = 1; w < GEN_WARPS; ++w) r = min(r, s_red[w]);
+  __syncthreads();
+  return r;
 }
 
-// Repair of a node whose occupants did not fit the block's list: passes over the whole
-// column through the row indices.  APPLY false: only marks the rows that will change.
-template <bool APPLY, typename MarkFn>
-__device__ void repair_column_scan(const GenArgs &a, uint32_t c, const uint32_t *s_slot, const uint32_t *s_summ,
-                                   int nn, int tot, int ne, int cap_n, int lane, MarkFn mark) {
-  const int J = a.J, NN = a.NN;
-  int keep = -1;
-  const bool intf = ne >= 2;
-  if (intf) {
-    const int o = (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
-    int best = J;
-    for (int j = lane; j < J; j += 32) {
-      const int v = (int)a.st.pool[(size_t)s_slot[j] * NN + nn];
-      if (v > 0 && ((s_summ[j] >> 11) & 0x7FFu) >= 2u) {
-        int t = j - o;
-        if (t < 0) t += J;
-        best = min(best, t);
-      }
-    }
+__device__ __forceinline__ int block_exscan(int v, int *s_red, int &total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
 #pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, off));
-    keep = o + best;
-    if (keep >= J) keep -= J;
-    int removed = 0;
-    for (int j = lane; j < J; j += 32) {
-      const int v = (int)a.st.pool[(size_t)s_slot[j] * NN + nn];
-      if (v > 0 && ((s_summ[j] >> 11) & 0x7FFu) >= 2u && j != keep) removed += v;
-    }
-    tot -= warp_sum(removed);
+  for (int off = 1; off < 32; off <<= 1) {
+    const int u = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += u;
   }
-  int excess = tot - cap_n;
-  // the capacity pass walks every job once in rotated order; jobs removed by the interference
-  // pass count as empty there and are written (or marked) on the way
-  const int o = (excess > 0) ? (int)bounded(draw(a.key, (uint32_t)nn, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J) : 0;
-  for (int t0 = 0; t0 < J; t0 += 32) {
-    const int t = t0 + lane;
-    int j = o + t;
-    if (j >= J) j -= J;
-    int v_old = 0, v_eff = 0;
-    if (t < J) {
-      bool dist;
-      v_old = (int)a.st.pool[(size_t)s_slot[j] * NN + nn];
-      v_eff = column_value(a, s_slot, s_summ, j, nn, keep, intf, dist);
-    }
-    int s = v_eff;                                // inclusive prefix over the 32 jobs
+  if (lane == 31) s_red[warp] = incl;
+  __syncthreads();
+  int before = 0;
+  total = 0;
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-      const int u = __shfl_up_sync(0xffffffffu, s, off);
-      if (lane >= off) s += u;
-    }
-    const int take = (excess > 0) ? min(v_eff, max(excess - (s - v_eff), 0)) : 0;
-    const int v_new = v_eff - take;
-    if (t < J && v_new != v_old) {
-      if (APPLY) a.st.pool[(size_t)s_slot[j] * NN + nn] = (int16_t)v_new;
-      else mark(j);
-    }
-    excess -= __shfl_sync(0xffffffffu, s, 31);
+  for (int w = 0; w < GEN_WARPS; ++w) {
+    const int t = s_red[w];
+    if (w < warp) before += t;
+    total += t;
   }
+  __syncthreads();
+  return before + incl - v;
 }
 
-template <int PPL>
+template <int PPL, bool INIT>
 __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArgs a) {
   extern __shared__ __align__(16) unsigned char smem[];
   const int J = a.J, NN = a.NN, P = a.P;
   const GenSmem L = gen_smem_layout(J, NN);
   uint32_t *s_slot = (uint32_t *)(smem + L.slot);
-  uint32_t *s_summ = (uint32_t *)(smem + L.summ);
-  int *s_mark = (int *)(smem + L.mark);            // bit 0: changed by the column pass, bit 1: row is new
+  int *s_mark = (int *)(smem + L.mark);
   float *s_term = (float *)(smem + L.term);
   // per node: GPUs placed (bits 0..31), distributed jobs on it (32..47), occupants (48..63)
   unsigned long long *s_node = (unsigned long long *)(smem + L.acc);
-  uint8_t *s_viol = (uint8_t *)(smem + L.viol);
-  uint16_t *s_viollist = (uint16_t *)(smem + L.viollist);
+  uint8_t *s_viol = (uint8_t *)(smem + L.viol);       // 1: decided from the node's list, 2: column walked
   uint32_t *s_occ = (uint32_t *)(smem + L.occ);
   int16_t *s_rowbuf = (int16_t *)(smem + L.rowbuf);
-  uint16_t *s_mut = (uint16_t *)(smem + L.mut), *s_ovf = (uint16_t *)(smem + L.ovf), *s_mod = (uint16_t *)(smem + L.mod);
+  uint16_t *s_mut = (uint16_t *)(smem + L.mut), *s_ovf = (uint16_t *)(smem + L.ovf), *s_slow = (uint16_t *)(smem + L.slow);
+  uint16_t *s_mod = (uint16_t *)(smem + L.mod);
   int16_t *s_cap = (int16_t *)(smem + L.cap);
   uint32_t *s_rec = (uint32_t *)(smem + L.rec);
-  __shared__ int s_nmut, s_novf, s_nmod, s_ncow, s_fail, s_anyscan, s_nviol;
-  __shared__ unsigned int s_base_mut, s_base_cow;
-  __shared__ int s_parent[2], s_rank4[4];
-  __shared__ double s_acc[GEN_WARPS];
-  __shared__ int s_acn[GEN_WARPS];
+  double *s_csum = (double *)(smem + L.sums);
+  int *s_ccnt = (int *)(smem + L.sums + (size_t)gen_max_chunks(J) * GEN_WARPS * 8);
+  uint4 *s_stash = (uint4 *)(smem + L.stash);         // per perturbed row: draw words y, z, w and the replica cap
+  __shared__ int s_nmut, s_novf, s_nslow, s_nmod, s_nneed, s_ncow, s_fail, s_anyscan, s_po;
+  __shared__ unsigned int s_base_mut, s_base_cow, s_base_cow2;
+  __shared__ int s_parent, s_rank4[4], s_red[GEN_WARPS + 1];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t *my_list = (uint32_t *)s_rowbuf + tid * LIST_WORDS;
   const uint32_t c = blockIdx.x;
-  const bool elite = (int)c < a.num_elite;
+  // children that are plain copies: the best-ranked parents of a generation, the current allocation
+  // itself in the initial population
+  const bool elite = INIT ? (c == 0u) : ((int)c < a.num_elite);
+  const uint32_t mut_slot = INIT ? SLOT_INIT : SLOT_MUTATE;
+
+  // The next kernel of the stream may start while this one runs (programmatic dependent launch):
+  // a following generation does its own prologue below and then waits for this grid to finish.
+  asm volatile("griddepcontrol.launch_dependents;");
+
+  // ---- prologue: nothing in it reads what the previous kernel writes, nothing is written to
+  // global memory -----------------------------------------------------------------------------
+  const uint32_t rkey = __ldg(a.key.round_ptr);
+#pragma unroll 1
+  for (int i = tid; i < NN; i += GEN_THREADS) {
+    s_node[i] = 0ull; s_viol[i] = 0;
+    s_cap[i] = (int16_t)max((int)a.cap[i], 0);
+  }
+#pragma unroll 1
+  for (int i = tid; i < J; i += GEN_THREADS) s_mark[i] = 0;
+  if (tid == 0) { s_nmut = 0; s_novf = 0; s_nslow = 0; s_nmod = 0; s_nneed = 0; s_ncow = 0; s_fail = 0; s_anyscan = 0; }
+  __syncthreads();
+  // every row's draws: which parent, perturbed or not; the perturbed rows are numbered
+  uint32_t secbits = 0, mutbits = 0;   // bit r: this thread's r-th row (j = tid + r * GEN_THREADS)
+  if (!elite) {
+    int r = 0;
+#pragma unroll 1
+    for (int j = tid; j < J; j += GEN_THREADS, ++r) {
+      if (a.active && !a.active[j]) continue;
+      const bool sec = !INIT && (draw_call(a.key.k0, rkey, (uint32_t)j, c, a.gen, SLOT_XOVER).x >> 31);
+      if (sec) secbits |= 1u << r;
+      const u32x4 mw = draw_call(a.key.k0, rkey, (uint32_t)j, c, a.gen, mut_slot);
+      if (mw.x < a.thr) {
+        mutbits |= 1u << r;
+        const int i = atomicAdd(&s_nmut, 1);
+        s_mut[i] = (uint16_t)(j | (sec ? 0x8000 : 0));          // j < 8192
+        if (i < MUT_STASH)
+          s_stash[i] = make_uint4(mw.y, mw.z, mw.w, (uint32_t)max(0, min(a.k_cap ? a.k_cap[j] : a.k_max, a.k_max)));
+      }
+    }
+  }
+  int idx[4] = {0, 0, 0, 0};
+  if (!INIT && !elite) {
+    const u32x4 sel = draw_call(a.key.k0, rkey, 0u, c, a.gen, SLOT_SELECT);
+    idx[0] = (int)bounded(sel.x, P); idx[1] = (int)bounded(sel.y, P);
+    idx[2] = (int)bounded(sel.z, P); idx[3] = (int)bounded(sel.w, P);
+  }
+  __syncthreads();
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  // ---- slots for the new rows: the perturbed ones plus a reserve for the rows the column pass
+  // changes; one atomic, asked for now and needed once the parents are known -------------------
+  unsigned int base_reg = 0, half_reg = 0;
+  const int nmut = s_nmut;
+  if (tid == GEN_THREADS - 1) {          // a thread of a warp that has no rank to work out
+    half_reg = __ldcg(a.state + 1);
+    base_reg = atomicAdd(a.state, (unsigned int)(nmut + COW_RESERVE));
+  }
 
   // ---- parents: the candidate of rank c for an elite child, else the better-ranked of two
   // random pairs (rank = candidates ordered before, fitness descending, index ascending) ----
-  if (elite) {
+  if (INIT) {
+    // every candidate descends from the current allocation
+  } else if (elite) {
     // The candidate of rank c: composite keys (fitness key, then lower index first) are unique,
     // so c + 1 rounds of "largest key below the previous one" find it; one barrier per round.
+    // Each thread keeps its first candidates' keys in registers.
     __shared__ unsigned long long s_wmax[2][GEN_WARPS];
+    constexpr int KEEP = 4;
+    unsigned long long mine[KEEP];
+#pragma unroll
+    for (int q = 0; q < KEEP; ++q) {
+      const int i = tid + q * GEN_THREADS;
+      mine[q] = (i < P) ? (((unsigned long long)order_key(__ldcg(a.fitness_bits + i)) << 32) |
+                           (unsigned long long)(0xFFFFFFFFu - (uint32_t)i)) : 0ull;
+    }
     unsigned long long prev = ~0ull;
+#pragma unroll 1
     for (int t = 0; t <= (int)c; ++t) {
       unsigned long long best = 0ull;
-      for (int i = tid; i < P; i += GEN_THREADS) {
-        const unsigned long long key = ((unsigned long long)order_key(__ldg(a.fitness_bits + i)) << 32) |
+#pragma unroll
+      for (int q = 0; q < KEEP; ++q)
+        if (mine[q] < prev && mine[q] > best) best = mine[q];
+#pragma unroll 1
+      for (int i = tid + KEEP * GEN_THREADS; i < P; i += GEN_THREADS) {
+        const unsigned long long key = ((unsigned long long)order_key(__ldcg(a.fitness_bits + i)) << 32) |
                                        (unsigned long long)(0xFFFFFFFFu - (uint32_t)i);
         if (key < prev && key > best) best = key;
       }
@@ -555,44 +836,47 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       for (int w = 0; w < GEN_WARPS; ++w) best = s_wmax[t & 1][w] > best ? s_wmax[t & 1][w] : best;
       prev = best;
     }
-    if (tid == 0) s_parent[0] = s_parent[1] = (int)(0xFFFFFFFFu - (uint32_t)(prev & 0xFFFFFFFFull));
-  } else {
-    const u32x4 sel = draw(a.key, 0u, c, a.gen, SLOT_SELECT);
-    const int idx[4] = {(int)bounded(sel.x, P), (int)bounded(sel.y, P), (int)bounded(sel.z, P), (int)bounded(sel.w, P)};
-    // the ranks of the four drawn candidates, a warp each; the keys are first staged in the (still
-    // unused) dynamic shared memory when they fit, so that every key is fetched once
-    uint32_t *s_keys = (uint32_t *)smem;
-    const bool staged = (size_t)P * 4 <= L.total;
-    if (staged) {
-      for (int i = tid; i < P; i += GEN_THREADS) s_keys[i] = order_key(__ldg(a.fitness_bits + i));
-      __syncthreads();
-    }
-    if (warp < 4) {
-      const int i = idx[warp];
-      const uint32_t ki = staged ? s_keys[i] : order_key(a.fitness_bits[i]);
-      int rk = 0;
-      for (int o = lane; o < P; o += 32) {
-        const uint32_t ko = staged ? s_keys[o] : order_key(__ldg(a.fitness_bits + o));
-        rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
+    if (tid == 0) s_parent = (int)(0xFFFFFFFFu - (uint32_t)(prev & 0xFFFFFFFFull));
+  } else if (warp < 4) {
+    // the ranks of the four drawn candidates, a warp each: every lane fetches its share of the keys
+    // (all loads in flight together) and counts those ordered before the warp's candidate
+    const int i = warp == 0 ? idx[0] : warp == 1 ? idx[1] : warp == 2 ? idx[2] : idx[3];
+    const uint32_t ki = order_key(__ldcg(a.fitness_bits + i));
+    int rk = 0;
+#pragma unroll 1
+    for (int o0 = lane; o0 < P; o0 += 32 * 8) {
+      uint32_t kk[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) kk[q] = (o0 + 32 * q < P) ? __ldcg(a.fitness_bits + o0 + 32 * q) : 0u;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const int o = o0 + 32 * q;
+        const uint32_t ko = order_key(kk[q]);
+        rk += (o < P && (ko > ki || (ko == ki && o < i))) ? 1 : 0;
       }
-      rk = warp_sum(rk);
-      if (lane == 0) s_rank4[warp] = rk;
     }
-    __syncthreads();
-    if (tid == 0) {
-      s_parent[0] = s_rank4[0] <= s_rank4[1] ? idx[0] : idx[1];
-      s_parent[1] = s_rank4[2] <= s_rank4[3] ? idx[2] : idx[3];
+    rk = warp_sum(rk);
+    if (lane == 0) s_rank4[warp] = rk;
+  }
+  if (tid == GEN_THREADS - 1) {
+    const unsigned long long limit = (unsigned long long)(half_reg + 1u) * a.st.half_cap;
+    s_base_mut = base_reg;
+    s_base_cow = base_reg + (unsigned int)nmut;
+    if ((unsigned long long)base_reg + (unsigned long long)(nmut + COW_RESERVE) > limit) {
+      s_fail = 1;
+      atomicExch(a.status, SCHED_ERR_TOO_LARGE);
     }
   }
   __syncthreads();
-
-  for (int i = tid; i < NN; i += GEN_THREADS) {
-    s_node[i] = 0ull; s_viol[i] = 0;
-    s_cap[i] = (int16_t)max((int)a.cap[i], 0);
+  const bool fail = s_fail != 0;          // no slots: perturbed rows stay as their parents', nothing is repaired
+  int par_a = 0, par_b = 0;
+  if (!INIT) {
+    if (elite) { par_a = par_b = s_parent; }
+    else {
+      par_a = s_rank4[0] <= s_rank4[1] ? idx[0] : idx[1];
+      par_b = s_rank4[2] <= s_rank4[3] ? idx[2] : idx[3];
+    }
   }
-  for (int i = tid; i < J; i += GEN_THREADS) s_mark[i] = 0;
-  if (tid == 0) { s_nmut = 0; s_novf = 0; s_nmod = 0; s_ncow = 0; s_fail = 0; s_anyscan = 0; s_nviol = 0; }
-  __syncthreads();
 
   // occupant (job j holds g GPUs on node n) into the node's totals and list
   auto add_occupant = [&](int j, int n, int g, bool dist) {
@@ -601,7 +885,6 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
     const int k = (int)(atomicAdd(&w[1], (dist ? 1u : 0u) | (1u << 16)) >> 16);
     if (k < OCC) s_occ[n * OCC + k] = (uint32_t)j | ((uint32_t)g << 13) | (dist ? 0x80000000u : 0u);
   };
-
   // the occupants in this lane's pieces of a row
   auto add_row_occupants = [&](const Grp &g, int j, const RowPieces<PPL> &p, bool dist) {
 #pragma unroll
@@ -616,29 +899,22 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   };
 
   // ---- rows, one thread each: the child row is the chosen parent's row -----------------------
-  // First every row's draws (which parent; perturbed or not).  The count of perturbed rows is
-  // then known and the block takes its slots - those plus a reserve for the rows the column
-  // pass will change - with one atomic whose answer is not needed before the rows are done.
-  uint32_t secbits = 0, mutbits = 0;   // bit r: this thread's r-th row (j = tid + r * GEN_THREADS)
-  if (!elite) {
-    int r = 0;
-    for (int j = tid; j < J; j += GEN_THREADS, ++r) {
-      if (a.active && !a.active[j]) continue;
-      if (draw(a.key, (uint32_t)j, c, a.gen, SLOT_XOVER).x >> 31) secbits |= 1u << r;
-      if (draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE).x < a.thr) {
-        mutbits |= 1u << r;
-        s_mut[atomicAdd(&s_nmut, 1)] = (uint16_t)j;
-      }
-    }
+  // RB rows per thread at a time, so that their dependent loads (index -> record) travel together.
+  // Perturbed rows are dealt out separately (row i of the block's list goes to lane i / 8 of warp
+  // i % 8); the loads of a thread's first perturbed row travel with those of its unperturbed rows.
+  const uint32_t *pin_a = a.ptr_in + (INIT ? (size_t)0 : (size_t)par_a * J);
+  const uint32_t *pin_b = a.ptr_in + (INIT ? (size_t)0 : (size_t)par_b * J);
+  const int mine_first = lane * GEN_WARPS + warp;
+  bool pre_loaded = mine_first < nmut;
+  uint32_t pre_slot = 0;
+  uint4 pre_lo = make_uint4(0u, 0u, 0u, 0u), pre_hi = pre_lo;
+  if (pre_loaded) {
+    const uint32_t mj = s_mut[mine_first];
+    const int j = (int)(mj & 0x1FFFu);
+    pre_slot = (INIT && !fail) ? a.init_src + (uint32_t)j : ((mj >> 15) ? __ldcg(pin_b + j) : __ldcg(pin_a + j));
   }
-  __syncthreads();
-  unsigned int base_reg = 0;
-  if (tid == 0) base_reg = atomicAdd(a.state, (unsigned int)(s_nmut + COW_RESERVE));
-
-  // Then RB rows per thread at a time, so that their dependent loads (index -> record) travel
-  // together.
-  const uint32_t *pin_a = a.ptr_in + (size_t)s_parent[0] * J, *pin_b = a.ptr_in + (size_t)s_parent[1] * J;
   constexpr int RB = 4;
+#pragma unroll 1
   for (int jb = tid, rb = 0; jb < J; jb += GEN_THREADS * RB, rb += RB) {
     uint32_t slot[RB];
     bool on[RB], mut[RB];
@@ -647,58 +923,138 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       const int j = jb + r * GEN_THREADS;
       on[r] = j < J && (!a.active || a.active[j]);
       mut[r] = ((mutbits >> (rb + r)) & 1u) != 0u;
-      slot[r] = on[r] ? (((secbits >> (rb + r)) & 1u) ? pin_b[j] : pin_a[j]) : a.st.zero_slot;
+      slot[r] = a.st.zero_slot;
+      if (on[r]) {
+        if (INIT && mut[r]) slot[r] = a.init_src + (uint32_t)j;   // perturbation starts before the row caps
+        else slot[r] = ((secbits >> (rb + r)) & 1u) ? __ldcg(pin_b + j) : __ldcg(pin_a + j);
+      }
     }
     uint32_t rec[RB][REC_WORDS];
 #pragma unroll
     for (int r = 0; r < RB; ++r) load_record(rec[r], a.st.rec + (size_t)slot[r] * REC_WORDS);
+    if (rb == 0 && pre_loaded) {
+      pre_lo = __ldcg((const uint4 *)(a.st.rec + (size_t)pre_slot * REC_WORDS));
+      pre_hi = __ldcg((const uint4 *)(a.st.rec + (size_t)pre_slot * REC_WORDS) + 1);
+    }
 #pragma unroll
     for (int r = 0; r < RB; ++r) {
       const int j = jb + r * GEN_THREADS;
-      if (j >= J) continue;
+      if (j >= J || mut[r]) continue;
       const uint32_t w = on[r] ? rec[r][REC_SUMM] : 0u;
       s_slot[j] = slot[r];
-      s_summ[j] = w;
-      if (!on[r] || mut[r]) continue;
+      if (!on[r]) continue;
       s_term[j] = __uint_as_float(rec[r][REC_TERM]);
+      const bool dist = ((w >> 11) & 0x7FFu) >= 2u;
+      if (dist) s_mark[j] = MARK_DIST;
       if (rec[r][0] == REC_OVERFLOW) {
         s_ovf[atomicAdd(&s_novf, 1)] = (uint16_t)j;
         continue;
       }
-      const bool dist = ((w >> 11) & 0x7FFu) >= 2u;
 #pragma unroll
       for (int k = 0; k < REC_ENTRIES; ++k) {
         const uint32_t e = rec[r][k];
-        if (e) add_occupant(j, (int)(e & 0xFFFu), (int)((e >> 12) & 0x7FFu), dist);
+        if (e) add_occupant(j, ent_node(e), ent_gpus(e), dist);
       }
     }
   }
-  if (tid == 0) {
-    const unsigned long long limit = (unsigned long long)(a.state[1] + 1u) * a.st.half_cap;
-    s_base_mut = base_reg;
-    s_base_cow = base_reg + (unsigned int)s_nmut;
-    if ((unsigned long long)base_reg + (unsigned long long)(s_nmut + COW_RESERVE) > limit) {
-      s_fail = 1;
-      atomicExch(a.status, SCHED_ERR_TOO_LARGE);
+  // ---- perturbed rows, one thread each -----------------------------------------------------------
+  // The row is worked out on the list of occupied nodes its record holds and gets a record of
+  // its own; only a row with more occupied nodes than a record holds needs its contents (left to
+  // a group of lanes below).
+#pragma unroll 1
+  for (int i = mine_first; i < nmut; i += GEN_THREADS) {
+    const uint32_t mj = s_mut[i];
+    const int j = (int)(mj & 0x1FFFu);
+    uint32_t src = pre_slot;
+    uint4 lo = pre_lo, hi = pre_hi;
+    if (!pre_loaded) {
+      src = (INIT && !fail) ? a.init_src + (uint32_t)j : ((mj >> 15) ? __ldcg(pin_b + j) : __ldcg(pin_a + j));
+      lo = __ldcg((const uint4 *)(a.st.rec + (size_t)src * REC_WORDS));
+      hi = __ldcg((const uint4 *)(a.st.rec + (size_t)src * REC_WORDS) + 1);
     }
+    pre_loaded = false;
+    s_slot[j] = src;
+    s_mark[j] = i << 4;
+    bool slow = lo.x == REC_OVERFLOW;
+    if (fail) {
+      // as an unperturbed row
+      s_term[j] = __uint_as_float(hi.z);
+      RowList rl;
+      list_from_record(rl, my_list, lo, hi);
+      if (slow) { s_ovf[atomicAdd(&s_novf, 1)] = (uint16_t)j; if (rl.n >= 2) s_mark[j] = MARK_DIST; continue; }
+      if (rl.n >= 2) s_mark[j] = MARK_DIST;
+#pragma unroll 1
+      for (int k = 0; k < rl.n; ++k) add_occupant(j, ent_node(rl.e[k]), ent_gpus(rl.e[k]), rl.n >= 2);
+      continue;
+    }
+    if (!slow) {
+      RowList rl;
+      list_from_record(rl, my_list, lo, hi);
+      u32x4 mw;
+      int kc;
+      if (i < MUT_STASH) {
+        const uint4 st = s_stash[i];
+        mw.x = 0u; mw.y = st.x; mw.z = st.y; mw.w = st.z;
+        kc = (int)st.w;
+      } else {
+        mw = draw_call(a.key.k0, rkey, (uint32_t)j, c, a.gen, mut_slot);
+        kc = max(0, min(a.k_cap ? a.k_cap[j] : a.k_max, a.k_max));
+      }
+      list_perturb(NN, rl, mw, s_cap);
+      list_caps(a.cur, NN, a.n_max, rl, j, kc);
+      slow = rl.n > REC_ENTRIES;
+      if (!slow) {
+        // K and N are final: the speedup, the penalty factor and the current allocation's values on
+        // the nodes the perturbation touched are fetched together
+        const float x_sp = __ldg(a.tp.table + fitness_table_index(a.tp, j, rl.K, rl.n));
+        const float x_pen = a.tp.pen ? __ldg(a.tp.pen + j) : 1.f;
+        int cv0 = 0, cv1 = 0;
+        if (a.cur && rl.pn > 0) cv0 = (int)__ldg(a.cur + (size_t)j * NN + rl.pnode0);
+        if (a.cur && rl.pn > 1) cv1 = (int)__ldg(a.cur + (size_t)j * NN + rl.pnode1);
+        if (a.cur && rl.pn > 0) rl.nd += (int)(rl.pnew0 != cv0) - (int)(rl.pold0 != cv0);
+        if (a.cur && rl.pn > 1) rl.nd += (int)(rl.pnew1 != cv1) - (int)(rl.pold1 != cv1);
+        const uint32_t nslot = s_base_mut + (uint32_t)i;
+        const uint32_t word = pack_summary(rl.K, rl.n, rl.nd);
+        const float term = row_term_from(a.tp.pen != nullptr, a.tp.mode, a.tp.p, a.tp.floor_, x_sp, x_pen, rl.nd != 0);
+        store_record(a.st.rec + (size_t)nslot * REC_WORDS, rl, term, word);
+        s_slot[j] = nslot;
+        s_term[j] = term;
+        s_mark[j] = MARK_OWN | (rl.n >= 2 ? MARK_DIST : 0);
+#pragma unroll 1
+        for (int k = 0; k < rl.n; ++k) add_occupant(j, ent_node(rl.e[k]), ent_gpus(rl.e[k]), rl.n >= 2);
+      }
+    }
+    if (slow) s_slow[atomicAdd(&s_nslow, 1)] = (uint16_t)j;   // s_slot[j] is the source row, s_mark[j] >> 4 its number
   }
   __syncthreads();
 
-  // ---- perturbed rows, one group of 16 lanes each: new row in a fresh slot --------------------
+  // ---- the few rows that need their contents: a group of 16 lanes each --------------------------
   const Grp g = make_group(lane, NN);
   const int grp = tid >> 4;
   int16_t *row = s_rowbuf + (size_t)grp * NN;   // this group's row
   uint32_t *recw = s_rec + grp * REC_WORDS;
-  if (!s_fail) {
-    for (int i = grp; i < s_nmut; i += GEN_GROUPS) {
-      const int j = (int)s_mut[i];
-      const uint32_t old = s_slot[j], w = s_summ[j];
-      load_row<false>(g, row, a.st.pool + (size_t)old * NN);
+  if (s_nslow | s_novf) {
+    // perturbed rows whose record does not hold them (before or after): contents from the pool, or
+    // laid out from the record; perturbed, capped and summarised as a row; the contents are
+    // written out only if the new record cannot hold the row either
+#pragma unroll 1
+    for (int i = grp; i < s_nslow; i += GEN_GROUPS) {
+      const int j = (int)s_slow[i];
+      const uint32_t old = s_slot[j];
+      if (g.sub < REC_WORDS) recw[g.sub] = __ldcg(a.st.rec + (size_t)old * REC_WORDS + g.sub);
       const CurPieces<PPL> cur = cur_pieces<PPL>(g, a.cur ? a.cur + (size_t)j * NN : nullptr);
       const int kc_in = a.k_cap ? a.k_cap[j] : a.k_max;
       __syncwarp(g.mask);
-      const int rN = (int)((w >> 11) & 0x7FFu);
-      const u32x4 mw = draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE);
+      const int rN = (int)((recw[REC_SUMM] >> 11) & 0x7FFu);
+      if (recw[0] == REC_OVERFLOW) {
+        load_row<true>(g, row, a.st.pool + (size_t)old * NN);
+      } else {
+        for (int v = g.sub; v < g.row_vecs; v += GROUP) ((uint4 *)row)[v] = make_uint4(0u, 0u, 0u, 0u);
+        __syncwarp(g.mask);
+        if (g.sub < REC_ENTRIES && recw[g.sub]) row[ent_node(recw[g.sub])] = (int16_t)ent_gpus(recw[g.sub]);
+      }
+      __syncwarp(g.mask);
+      const u32x4 mw = draw_call(a.key.k0, rkey, (uint32_t)j, c, a.gen, mut_slot);
       const uint32_t op = bounded(mw.y, 3u);
       if (op == 0u) {
         const int n = (int)bounded(mw.w, (uint32_t)NN);
@@ -718,8 +1074,6 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       __syncwarp(g.mask);
       int K, N, nd;
       RowPieces<PPL> p = summarise_row<PPL>(g, row, cur, K, N, nd, recw);
-      // per-row caps: replicas above the job's cap leave from the highest node index down, then
-      // occupied nodes beyond n_max are cleared from the highest index down
       const int kc = max(0, min(kc_in, a.k_max));
       if (K > kc || N > a.n_max) {
         if (g.sub == 0) {
@@ -740,244 +1094,297 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         __syncwarp(g.mask);
         p = summarise_row<PPL>(g, row, cur, K, N, nd, recw);
       }
-      const uint32_t slot = s_base_mut + (uint32_t)i;
-      // the row's speedup (and penalty factor) are asked for now and used at the end of the step
-      float x_sp = 0.f, x_pen = 1.f;
-      if (g.sub == 0) {
-        x_sp = __ldg(a.tp.table + fitness_table_index(a.tp, j, K, N));
-        if (a.tp.pen && nd != 0) x_pen = __ldg(a.tp.pen + j);
-      }
-      store_row(g, a.st.pool + (size_t)slot * NN, row);
+      const uint32_t slot = s_base_mut + (uint32_t)(s_mark[j] >> 4);
+      float term = 0.f;
+      if (g.sub == 0)
+        term = row_term_of(a.tp.table, a.tp.pen, a.tp.k_max, a.tp.n_max, a.tp.mode, a.tp.p, a.tp.floor_, j, K, N, nd);
+      if (N > REC_ENTRIES) store_row(g, a.st.pool + (size_t)slot * NN, row);
       const uint32_t word = pack_summary(K, N, nd);
+      __syncwarp(g.mask);
       if (g.sub == 0) {
         recw[REC_SUMM] = word;
+        recw[REC_TERM] = __float_as_uint(term);
         s_slot[j] = slot;
-        s_summ[j] = word;
-        s_mark[j] = 2;
+        s_term[j] = term;
+        s_mark[j] = MARK_OWN | (N >= 2 ? MARK_DIST : 0);
       }
       add_row_occupants(g, j, p, N >= 2);
-      if (g.sub == 0) {
-        const float term = fitness_term_with(a.tp, x_sp, x_pen, nd != 0);
-        s_term[j] = term;
-        recw[REC_TERM] = __float_as_uint(term);
-      }
       __syncwarp(g.mask);
       if (g.sub < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + g.sub] = recw[g.sub];
       __syncwarp(g.mask);
     }
-  }
-  // rows with more occupied nodes than a record holds: occupants from the row itself
-  for (int i = grp; i < s_novf; i += GEN_GROUPS) {
-    const int j = (int)s_ovf[i];
-    load_row<false>(g, row, a.st.pool + (size_t)s_slot[j] * NN);
-    __syncwarp(g.mask);
-    const RowPieces<PPL> p = row_pieces<PPL>(g, row);
-    add_row_occupants(g, j, p, ((s_summ[j] >> 11) & 0x7FFu) >= 2u);
-    __syncwarp(g.mask);
-  }
-  __syncthreads();
-
-  // ---- column pass, decisions: which occupants of the violating nodes change ------------------
-  auto mark_row = [&](int j) {
-    if ((atomicOr(&s_mark[j], 1) & 1) == 0) {
-      s_mod[atomicAdd(&s_nmod, 1)] = (uint16_t)j;
-      for (int b = 0; b * 64 < NN; ++b) {   // the row and its counterpart will be read next
-        prefetch_l2(a.st.pool + (size_t)s_slot[j] * NN + b * 64);
-        if (a.cur) prefetch_l2(a.cur + (size_t)j * NN + b * 64);
-      }
-    }
-  };
-  // nodes that hold two distributed jobs or more GPUs than they have
-  for (int n = tid; n < NN; n += GEN_THREADS) {
-    const unsigned long long acc = s_node[n];
-    if ((int)((acc >> 32) & 0xFFFFu) >= 2 || (int)(uint32_t)acc > (int)s_cap[n]) s_viollist[atomicAdd(&s_nviol, 1)] = (uint16_t)n;
-  }
-  __syncthreads();
-  const int nviol = s_nviol;
-  for (int i = grp; i < nviol; i += GEN_GROUPS) {   // a group of 16 lanes per listed node
-    const int nn = (int)s_viollist[i];
-    const unsigned long long acc = s_node[nn];
-    const int have_n = (int)(acc >> 48);
-    if (have_n > OCC) {   // more occupants than the list holds: left to the column scan below
-      if (g.sub == 0) { s_viol[nn] = 2; s_anyscan = 1; }
-      continue;
-    }
-    const uint32_t entry = (g.sub < have_n) ? s_occ[nn * OCC + g.sub] : 0u;
-    const int v_new = decide_entries(a, g, c, nn, (int)(uint32_t)acc, (int)((acc >> 32) & 0xFFFFu), (int)s_cap[nn], entry, have_n);
-    if (g.sub < have_n) {
-      // the entry now carries the decision: GPUs kept, and bit 24 when that is a change
-      const bool changed = v_new != (int)((entry >> 13) & 0x7FFu);
-      s_occ[nn * OCC + g.sub] = (entry & 0x80001FFFu) | ((uint32_t)v_new << 13) | (changed ? (1u << 24) : 0u);
-      if (changed) mark_row((int)(entry & 0x1FFFu));
-    }
-    if (g.sub == 0) s_viol[nn] = 1;
-    __syncwarp(g.mask);
-  }
-  __syncthreads();
-  if (s_anyscan) {
-    for (int i = warp; i < nviol; i += GEN_WARPS) {   // a warp per node whose column must be scanned
-      const int nn = (int)s_viollist[i];
-      if (s_viol[nn] != 2) continue;
-      const unsigned long long acc = s_node[nn];
-      repair_column_scan<false>(a, c, s_slot, s_summ, nn, (int)(uint32_t)acc, (int)((acc >> 32) & 0xFFFFu), (int)s_cap[nn],
-                                lane, mark_row);
+    // unperturbed rows with more occupied nodes than a record holds: occupants from the contents
+#pragma unroll 1
+    for (int i = grp; i < s_novf; i += GEN_GROUPS) {
+      const int j = (int)s_ovf[i];
+      load_row<true>(g, row, a.st.pool + (size_t)s_slot[j] * NN);
+      __syncwarp(g.mask);
+      const RowPieces<PPL> p = row_pieces<PPL>(g, row);
+      add_row_occupants(g, j, p, (s_mark[j] & MARK_DIST) != 0);
+      __syncwarp(g.mask);
     }
     __syncthreads();
   }
 
-  // ---- rows the column pass changes -----------------------------------------------------------
-  // Usual case (every violating node's occupants were listed): one group per changed row takes
-  // the row, applies the decisions of its nodes, and writes it with its record - to a slot of
-  // its own unless the row is new in this generation already.
-  const int nmod = s_nmod;
-  if (!s_anyscan) {
-    if (nmod > COW_RESERVE) {   // more than the reserve: a run of slots of their own
+  // ---- column pass, decisions: which occupants of the violating nodes change ------------------
+  // a warp looks at 32 nodes at a time, a lane each; its two groups of 16 lanes then decide the
+  // nodes that hold two distributed jobs or more GPUs than they have
+  if (!fail) {
+#pragma unroll 1
+    for (int nbase = warp * 32; nbase < NN; nbase += GEN_THREADS) {
+      const int n_l = nbase + lane;
+      bool bad = false;
+      if (n_l < NN) {
+        const unsigned long long acc_l = s_node[n_l];
+        bad = (int)((acc_l >> 32) & 0xFFFFu) >= 2 || (int)(uint32_t)acc_l > (int)s_cap[n_l];
+      }
+      unsigned todo = __ballot_sync(0xffffffffu, bad);
+#pragma unroll 1
+      while (todo) {
+      // the two lowest set bits: one node per group (the second group may have none)
+      const int b0 = __ffs(todo) - 1;
+      todo &= todo - 1;
+      int b1 = -1;
+      if (todo) { b1 = __ffs(todo) - 1; todo &= todo - 1; }
+      const int bsel = (lane & GROUP) ? b1 : b0;
+      if (bsel >= 0) {
+      const int nn = nbase + bsel;
+      const unsigned long long acc = s_node[nn];
+      const int have_n = (int)(acc >> 48);
+      if (have_n > OCC) {   // more occupants than the list holds: the column is walked below
+        if (g.sub == 0) { s_viol[nn] = 2; s_anyscan = 1; }
+      } else {
+      const uint32_t entry = (g.sub < have_n) ? s_occ[nn * OCC + g.sub] : 0u;
+      const int v_new = decide_entries(a, rkey, g, c, nn, (int)(uint32_t)acc, (int)((acc >> 32) & 0xFFFFu), (int)s_cap[nn], entry, have_n);
+      if (g.sub < have_n) {
+        // the entry now carries the decision: GPUs kept, and bit 24 when that is a change
+        const bool changed = v_new != (int)((entry >> 13) & 0x7FFu);
+        s_occ[nn * OCC + g.sub] = (entry & 0x80001FFFu) | ((uint32_t)v_new << 13) | (changed ? (1u << 24) : 0u);
+        if (changed) {
+          const int j = (int)(entry & 0x1FFFu);
+          const int before = atomicOr(&s_mark[j], MARK_CHANGED);
+          if ((before & MARK_CHANGED) == 0) {
+            s_mod[atomicAdd(&s_nmod, 1)] = (uint16_t)j;
+            if ((before & MARK_OWN) == 0) atomicAdd(&s_nneed, 1);   // will want a slot of its own
+          }
+        }
+      }
+      if (g.sub == 0) s_viol[nn] = 1;
+      }
+      }
+      __syncwarp();
+      }
+    }
+    __syncthreads();
+
+    // ---- rows the column pass changes: rewritten by one thread each ----------------------------
+    // The row keeps on each occupied node what the node's decision says (only_node < 0: looked up
+    // in the lists of the decided nodes; else: only_value on that node).  The list of occupied
+    // nodes is edited and stored as a new record - in a slot of its own (copy on write) unless the
+    // row is new in this generation already; a row that only exists as contents is copied and
+    // patched piece by piece.
+    const int nmod = s_nmod;
+    const bool scan = s_anyscan != 0;
+    const int nneed = s_nneed;
+    if (nneed > COW_RESERVE) {   // more rows to copy than the reserve: a further run of slots for the block
       if (tid == 0) {
-        const unsigned int base = atomicAdd(a.state, (unsigned int)nmod);
-        const unsigned long long limit = (unsigned long long)(a.state[1] + 1u) * a.st.half_cap;
-        s_base_cow = base;
-        if ((unsigned long long)base + (unsigned long long)nmod > limit) { s_fail = 1; atomicExch(a.status, SCHED_ERR_TOO_LARGE); }
+        const unsigned int base = atomicAdd(a.state, (unsigned int)(nneed - COW_RESERVE));
+        const unsigned long long limit = (unsigned long long)(__ldcg(a.state + 1) + 1u) * a.st.half_cap;
+        s_base_cow2 = base;
+        if ((unsigned long long)base + (unsigned long long)(nneed - COW_RESERVE) > limit) {
+          s_fail = 1;
+          atomicExch(a.status, SCHED_ERR_TOO_LARGE);
+        }
       }
       __syncthreads();
     }
-    if (!s_fail) {
-      for (int i = grp; i < nmod; i += GEN_GROUPS) {
-        const int j = (int)s_mod[i];
-        const bool own = (s_mark[j] & 2) != 0;
-        const uint32_t src = s_slot[j];
-        load_row<true>(g, row, a.st.pool + (size_t)src * NN);   // may have been written in this kernel
-        const CurPieces<PPL> cur = cur_pieces<PPL>(g, a.cur ? a.cur + (size_t)j * NN : nullptr);
-        __syncwarp(g.mask);
-        {
-          const RowPieces<PPL> p = row_pieces<PPL>(g, row);
+    const bool fail2 = s_fail != 0;
+    auto rewrite_row = [&](int j, int only_node, int only_value) {
+      const uint32_t src = s_slot[j];
+      const bool own = (s_mark[j] & MARK_OWN) != 0;
+      const uint4 lo = __ldcg((const uint4 *)(a.st.rec + (size_t)src * REC_WORDS));
+      const uint4 hi = __ldcg((const uint4 *)(a.st.rec + (size_t)src * REC_WORDS) + 1);
+      uint32_t dst = src;
+      if (!own) {   // a slot from the block's reserve, beyond it one by one
+        const int k = atomicAdd(&s_ncow, 1);
+        if (k < COW_RESERVE) {
+          dst = s_base_cow + (uint32_t)k;
+        } else if (k < nneed) {
+          dst = s_base_cow2 + (uint32_t)(k - COW_RESERVE);
+        } else {
+          dst = atomicAdd(a.state, 1u);
+          const unsigned long long limit = (unsigned long long)(__ldcg(a.state + 1) + 1u) * a.st.half_cap;
+          if ((unsigned long long)dst + 1ull > limit) { atomicExch(a.status, SCHED_ERR_TOO_LARGE); return; }
+        }
+      }
+      auto new_value = [&](int node, int v) -> int {
+        if (only_node >= 0) return node == only_node ? only_value : v;
+        if (s_viol[node] != 1) return v;
+        const int cnt = (int)(s_node[node] >> 48);
+#pragma unroll 1
+        for (int k = 0; k < cnt; ++k) {
+          const uint32_t e = s_occ[node * OCC + k];
+          if ((int)(e & 0x1FFFu) == j) return ((e >> 24) & 1u) ? (int)((e >> 13) & 0x7FFu) : v;
+        }
+        return v;
+      };
+      RowList rl;
+      list_from_record(rl, my_list, lo, hi);
+      if (lo.x != REC_OVERFLOW) {
+        int m = 0;                      // entries kept so far
+#pragma unroll 1
+        for (int k = 0; k < rl.n; ++k) {
+          const int node = ent_node(rl.e[k]), v = ent_gpus(rl.e[k]);
+          const int v_new = new_value(node, v);
+          if (v_new != v) {
+            rl.nd += diff_delta(a.cur, NN, j, node, v, v_new);
+            rl.K += v_new - v;
+          }
+          rl.e[k] = 0u;
+          if (v_new > 0) rl.e[m++] = (uint32_t)node | ((uint32_t)v_new << 12);
+        }
+        rl.n = m;
+      } else {
+        // contents only: pieces pass through this thread, patched on the way; the occupied nodes
+        // that remain are listed, so that a row that now fits a record becomes one again
+        const int16_t *from = a.st.pool + (size_t)src * NN;
+        int16_t *to = a.st.pool + (size_t)dst * NN;
+        int kept = 0;                   // occupied nodes that remain
 #pragma unroll
-          for (int q = 0; q < PPL; ++q) {
-            uint32_t m = p.mask[q];
-            while (m) {
-              const int n = 8 * (g.sub * PPL + q) + __ffs(m) - 1;
-              m &= m - 1;
-              if (s_viol[n] != 1) continue;
-              const int cnt = (int)(s_node[n] >> 48);
-              for (int k = 0; k < cnt; ++k) {
-                const uint32_t e = s_occ[n * OCC + k];
-                if ((int)(e & 0x1FFFu) == j) {
-                  if ((e >> 24) & 1u) row[n] = (int16_t)((e >> 13) & 0x7FFu);
-                  break;
-                }
-              }
+        for (int k = 0; k <= LIST_MAX; ++k) rl.e[k] = 0u;
+#pragma unroll 1
+        for (int v = 0; v < (NN >> 3); ++v) {
+          uint4 x = load_piece<true>(from, v);
+          const uint4 x0 = x;
+          uint32_t m = piece_mask(x);
+          while (m) {
+            const int h = __ffs(m) - 1;
+            m &= m - 1;
+            const int node = 8 * v + h, val = piece_entry(x, h);
+            const int v_new = new_value(node, val);
+            if (v_new != val) {
+              rl.nd += diff_delta(a.cur, NN, j, node, val, v_new);
+              rl.K += v_new - val;
+              rl.n -= (v_new == 0) ? 1 : 0;
+              x = piece_with(x, h, v_new);
+            }
+            if (v_new > 0) {
+              if (kept < REC_ENTRIES) rl.e[kept] = (uint32_t)node | ((uint32_t)v_new << 12);
+              ++kept;
             }
           }
+          if (!own || x.x != x0.x || x.y != x0.y || x.z != x0.z || x.w != x0.w) ((uint4 *)to)[v] = x;
         }
-        __syncwarp(g.mask);
-        int K, N, nd;
-        summarise_row<PPL>(g, row, cur, K, N, nd, recw);
-        const uint32_t dst = own ? src : s_base_cow + (uint32_t)i;
-        float x_sp = 0.f, x_pen = 1.f;
-        if (g.sub == 0) {
-          x_sp = __ldg(a.tp.table + fitness_table_index(a.tp, j, K, N));
-          if (a.tp.pen && nd != 0) x_pen = __ldg(a.tp.pen + j);
+        if (kept > REC_ENTRIES) {       // still more occupied nodes than a record holds
+          rl.e[0] = REC_OVERFLOW;
+#pragma unroll
+          for (int k = 1; k < LIST_MAX; ++k) rl.e[k] = 0u;
         }
-        store_row(g, a.st.pool + (size_t)dst * NN, row);
-        const uint32_t word = pack_summary(K, N, nd);
-        if (g.sub == 0) {
-          const float term = fitness_term_with(a.tp, x_sp, x_pen, nd != 0);
-          recw[REC_SUMM] = word;
-          recw[REC_TERM] = __float_as_uint(term);
-          s_slot[j] = dst;
-          s_summ[j] = word;
-          s_term[j] = term;
-        }
-        __syncwarp(g.mask);
-        if (g.sub < REC_WORDS) a.st.rec[(size_t)dst * REC_WORDS + g.sub] = recw[g.sub];
-        __syncwarp(g.mask);
       }
-    }
-    __syncthreads();
-  } else {
-    // Some node had more occupants than the block lists: its column is scanned through the
-    // row indices, so the rows are first copied, then written in place, then summarised.
-      for (int i = tid; i < nmod; i += GEN_THREADS) {
-      const int j = (int)s_mod[i];
-      const bool own = (s_mark[j] & 2) != 0;
-      s_ovf[i] = own ? (uint16_t)0xFFFFu : (uint16_t)atomicAdd(&s_ncow, 1);
-    }
-    __syncthreads();
-    if (tid == 0 && s_ncow > COW_RESERVE) {   // more than the reserve: a run of slots of their own
-      const unsigned int base = atomicAdd(a.state, (unsigned int)s_ncow);
-      const unsigned long long limit = (unsigned long long)(a.state[1] + 1u) * a.st.half_cap;
-      s_base_cow = base;
-      if ((unsigned long long)base + (unsigned long long)s_ncow > limit) { s_fail = 1; atomicExch(a.status, SCHED_ERR_TOO_LARGE); }
-    }
-    __syncthreads();
-    if (!s_fail) {
-      for (int i = grp; i < nmod; i += GEN_GROUPS) {
-        const uint32_t k = s_ovf[i];
-        if (k == 0xFFFFu) continue;
-        const int j = (int)s_mod[i];
-        const uint32_t slot = s_base_cow + k;
-        load_row<true>(g, row, a.st.pool + (size_t)s_slot[j] * NN);
-        __syncwarp(g.mask);
-        store_row(g, a.st.pool + (size_t)slot * NN, row);
-        __syncwarp(g.mask);
-        if (g.sub == 0) s_slot[j] = slot;
-      }
-    }
-    __syncthreads();
-
-    // column pass, writes
-    if (!s_fail && nmod > 0) {
-      for (int i = tid; i < NN * OCC; i += GEN_THREADS) {
-        const int n = i / OCC, k = i - n * OCC;
-        if (s_viol[n] != 1 || k >= (int)(s_node[n] >> 48)) continue;
-        const uint32_t entry = s_occ[i];
-        if ((entry >> 24) & 1u)
-          a.st.pool[(size_t)s_slot[entry & 0x1FFFu] * NN + n] = (int16_t)((entry >> 13) & 0x7FFu);
-      }
-      for (int nn = warp; nn < NN; nn += GEN_WARPS) {
+      const uint32_t word = pack_summary(rl.K, rl.n, rl.nd);
+      const float term = row_term_of(a.tp.table, a.tp.pen, a.tp.k_max, a.tp.n_max, a.tp.mode, a.tp.p, a.tp.floor_, j,
+                                     rl.K, rl.n, rl.nd);
+      store_record(a.st.rec + (size_t)dst * REC_WORDS, rl, term, word);
+      s_slot[j] = dst;
+      s_term[j] = term;
+      s_mark[j] |= MARK_OWN;
+    };
+    // Thread work for the two uses of rewrite_row, gathered so that the code exists once: first the
+    // rows the listed nodes changed (row i of the list to lane i / 8 of warp i % 8), then, node by
+    // node, the rows of the columns that had to be walked.
+    const int rpt = (J + GEN_THREADS - 1) / GEN_THREADS;
+    const int j_lo = min(J, tid * rpt), j_hi = min(J, j_lo + rpt);
+    // ---- nodes with more occupants than a list holds: the whole block walks the column -------
+    // Thread t looks after the consecutive rows [t * rpt, (t + 1) * rpt); a row's GPUs on the node
+    // come from its record (or its contents).  Interference: the first distributed occupant in
+    // rotated job order stays.  Capacity: a block-wide prefix sum in job order gives every row the
+    // GPUs that come before it in rotated order.
+#pragma unroll 1
+    for (int step = -1; step < (scan ? NN : 0) && !fail2; ++step) {
+      int nn = -1, keep = -1, excess = 0, o2 = 0, p_o = 0, total = 0, running = 0;
+      if (step >= 0) {
+        if (step == 0) __syncthreads();          // the listed rewrites are done
+        nn = step;
         if (s_viol[nn] != 2) continue;
-        repair_column_scan<true>(a, c, s_slot, s_summ, nn, (int)(uint32_t)s_node[nn], (int)((s_node[nn] >> 32) & 0xFFFFu),
-                                 (int)s_cap[nn], lane, [](int) {});
-      }
-    }
-    __syncthreads();
-
-    // changed rows: summary and record from the row as it now stands
-    if (!s_fail) {
-      for (int i = grp; i < nmod; i += GEN_GROUPS) {
-        const int j = (int)s_mod[i];
-        const uint32_t slot = s_slot[j];
-        load_row<true>(g, row, a.st.pool + (size_t)slot * NN);   // written in this kernel: read through to L2
-        const CurPieces<PPL> cur = cur_pieces<PPL>(g, a.cur ? a.cur + (size_t)j * NN : nullptr);
-        __syncwarp(g.mask);
-        int K, N, nd;
-        summarise_row<PPL>(g, row, cur, K, N, nd, recw);
-        const uint32_t word = pack_summary(K, N, nd);
-        if (g.sub == 0) {
-          const float term = fitness_term(a.tp, j, K, N, nd != 0);
-          recw[REC_SUMM] = word;
-          recw[REC_TERM] = __float_as_uint(term);
-          s_summ[j] = word;
-          s_term[j] = term;
+        const unsigned long long acc = s_node[nn];
+        const int ne = (int)((acc >> 32) & 0xFFFFu), cap_n = (int)s_cap[nn];
+        if (ne >= 2) {
+          const int o = (int)bounded(draw_call(a.key.k0, rkey, (uint32_t)nn, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
+          int best = J;
+#pragma unroll 1
+          for (int j = j_lo; j < j_hi; ++j) {
+            if ((s_mark[j] & MARK_DIST) && row_value_at(a.st.rec, a.st.pool, NN, s_slot[j], nn) > 0) {
+              int t = j - o;
+              if (t < 0) t += J;
+              best = min(best, t);
+            }
+          }
+          best = block_min(best, s_red);
+          keep = o + best;
+          if (keep >= J) keep -= J;
         }
-        __syncwarp(g.mask);
-        if (g.sub < REC_WORDS) a.st.rec[(size_t)slot * REC_WORDS + g.sub] = recw[g.sub];
-        __syncwarp(g.mask);
+        int mine = 0;
+#pragma unroll 1
+        for (int j = j_lo; j < j_hi; ++j) {
+          const int v = row_value_at(a.st.rec, a.st.pool, NN, s_slot[j], nn);
+          mine += (keep >= 0 && (s_mark[j] & MARK_DIST) && v > 0 && j != keep) ? 0 : v;
+        }
+        running = block_exscan(mine, s_red, total);
+        excess = total - cap_n;
+        if (excess > 0) {
+          o2 = (int)bounded(draw_call(a.key.k0, rkey, (uint32_t)nn, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J);
+          if (o2 >= j_lo && o2 < j_hi) {      // GPUs of the rows before row o2 in job order
+            int p = running;
+#pragma unroll 1
+            for (int j = j_lo; j < o2; ++j) {
+              const int v = row_value_at(a.st.rec, a.st.pool, NN, s_slot[j], nn);
+              p += (keep >= 0 && (s_mark[j] & MARK_DIST) && v > 0 && j != keep) ? 0 : v;
+            }
+            s_po = p;
+          }
+          __syncthreads();
+          p_o = s_po;
+        }
       }
+      // the rows this thread rewrites in this step
+      const int first = (step < 0) ? mine_first : j_lo;
+      const int last = (step < 0) ? nmod : j_hi;
+      const int stride = (step < 0) ? GEN_THREADS : 1;
+#pragma unroll 1
+      for (int i = first; i < last; i += stride) {
+        if (step < 0) {
+          rewrite_row((int)s_mod[i], -1, 0);
+          continue;
+        }
+        const int j = i;
+        const int v = row_value_at(a.st.rec, a.st.pool, NN, s_slot[j], nn);
+        const int v_eff = (keep >= 0 && (s_mark[j] & MARK_DIST) && v > 0 && j != keep) ? 0 : v;
+        int take = 0;
+        if (excess > 0) {
+          const int ahead = (j >= o2) ? running - p_o : total - p_o + running;
+          take = min(v_eff, max(excess - ahead, 0));
+        }
+        running += v_eff;
+        if (v_eff - take != v) rewrite_row(j, nn, v_eff - take);
+      }
+      if (step >= 0) __syncthreads();   // the rewritten rows are read again for the next such node
     }
-    __syncthreads();
   }
+  __syncthreads();
 
   // ---- children's indices out, fitness of the candidate (Eq. 14) from the rows' terms ----------
   uint32_t *pout = a.ptr_out + (size_t)c * J;
+#pragma unroll 1
   for (int j = tid; j < J; j += GEN_THREADS) pout[j] = s_slot[j];
   // sums in the order of the dense fitness kernel: per chunk of rows, thread t adds rows t,
   // t + 256, ... in double, a shuffle tree per warp, the warps in index order; then the chunks
   // in index order
-  double ts = 0.0, ns = 0.0;
+#pragma unroll 1
   for (int ch = 0; ch < a.chunks; ++ch) {
     const int j0 = ch * a.rows_per_chunk, j1 = min(J, j0 + a.rows_per_chunk);
     double acc = 0.0;
     int cnt = 0;
+#pragma unroll 1
     for (int j = j0 + tid; j < j1; j += GEN_THREADS) {
       if (!a.tp.active || a.tp.active[j]) { acc += (double)s_term[j]; cnt += 1; }
     }
@@ -986,18 +1393,21 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       acc += __shfl_xor_sync(0xffffffffu, acc, off);
       cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
     }
-    if (lane == 0) { s_acc[warp] = acc; s_acn[warp] = cnt; }
-    __syncthreads();
-    if (tid == 0) {
+    if (lane == 0) { s_csum[ch * GEN_WARPS + warp] = acc; s_ccnt[ch * GEN_WARPS + warp] = cnt; }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    double ts = 0.0, ns = 0.0;
+#pragma unroll 1
+    for (int ch = 0; ch < a.chunks; ++ch) {
       double t = 0.0;
       int n = 0;
-      for (int w = 0; w < GEN_WARPS; ++w) { t += s_acc[w]; n += s_acn[w]; }
+      for (int w = 0; w < GEN_WARPS; ++w) { t += s_csum[ch * GEN_WARPS + w]; n += s_ccnt[ch * GEN_WARPS + w]; }
       ts += t;
       ns += (double)n;
     }
-    __syncthreads();
+    a.fitness_out[c] = fitness_finalise(a.tp.mode, a.tp.p, ts, ns);
   }
-  if (tid == 0) a.fitness_out[c] = fitness_finalise(a.tp.mode, a.tp.p, ts, ns);
 }
 
 // pieces per lane of a row's group: 1, 2 or 4 (a lane's pieces beyond the row's end are empty)
@@ -1057,7 +1467,8 @@ int rowstore_ensure(sched_ctx *ctx) {
     const size_t smem = gen_smem_layout(c.num_jobs, c.num_nodes).total;
     if (smem > 48 * 1024)
     for (int k = 0; k < 3 && e == cudaSuccess; ++k)
-      e = cudaFuncSetAttribute(k == 0 ? generation_store_kernel<1> : k == 1 ? generation_store_kernel<2> : generation_store_kernel<4>,
+      e = cudaFuncSetAttribute(k == 0 ? generation_store_kernel<1, false> : k == 1 ? generation_store_kernel<2, false>
+                                                                                  : generation_store_kernel<4, false>,
                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   }
   if (e != cudaSuccess) {
@@ -1143,7 +1554,7 @@ int rowstore_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d
   a.cur = d_cur;
   a.P = c.population; a.J = c.num_jobs; a.NN = c.num_nodes;
   a.k_max = c.k_max; a.n_max = c.n_max; a.num_elite = c.num_elite;
-  a.thr = c.thr_mutate; a.gen = generation;
+  a.thr = c.thr_mutate; a.gen = generation; a.init_src = 0u;
   a.key = make_key(c.seed, ctx->d_round);
   a.tp.table = ctx->d_tab_speedup; a.tp.pen = d_pen; a.tp.active = d_active;
   a.tp.k_max = c.k_max; a.tp.n_max = c.n_max; a.tp.mode = fitness_mode(c.p); a.tp.p = c.p;
@@ -1154,10 +1565,25 @@ int rowstore_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d
   const size_t smem = gen_smem_layout(c.num_jobs, c.num_nodes).total;
   {
     TimedLaunch tl_(ctx, KK_GENSTORE);
+    // launched so that it may start while the previous kernel of the stream still runs: the kernel
+    // does its draws first and waits for that kernel before it reads anything it wrote
     const int ppl = store_pieces_per_lane(c.num_nodes);
-    if (ppl == 1) generation_store_kernel<1><<<c.population, GEN_THREADS, smem, ctx->stream>>>(a);
-    else if (ppl == 2) generation_store_kernel<2><<<c.population, GEN_THREADS, smem, ctx->stream>>>(a);
-    else generation_store_kernel<4><<<c.population, GEN_THREADS, smem, ctx->stream>>>(a);
+    void (*kernel)(GenArgs) = ppl == 1 ? generation_store_kernel<1, false>
+                              : ppl == 2 ? generation_store_kernel<2, false> : generation_store_kernel<4, false>;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3((unsigned)c.population);
+    lc.blockDim = dim3(GEN_THREADS);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = ctx->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    if (cudaLaunchKernelEx(&lc, kernel, a) != cudaSuccess) {
+      cudaGetLastError();
+      kernel<<<c.population, GEN_THREADS, smem, ctx->stream>>>(a);
+    }
   }
   SCHED_LAUNCH_CHECK(ctx);
   return SCHED_OK;
