@@ -238,13 +238,24 @@ int ga_generation(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_pop
  * on the first call.  Problems with more than 256 jobs (rows of whole 16-byte pieces, at
  * most 512 nodes and 8192 jobs) keep the population of the round as shared rows - row
  * indices per candidate into a pool of rows, copy on write - instead of dense matrices;
- * the results are the same bit for bit, the scratch is larger (a pool of up to 8 GiB, sized
- * at 2 x (1 + 8 worst-case generations) populations when that fits), and a pool overflow
+ * the results are the same bit for bit, the scratch is larger (see sched_set_store_budget),
+ * and a pool overflow
  * (not expected: the pool is compacted before it can run out) would be reported as device
  * status SCHED_ERR_TOO_LARGE by sched_sync_status.  If the pool cannot be allocated the
  * round runs on dense matrices. */
 int schedule_round(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cur, uint32_t round,
                    int32_t generations, int16_t *d_best, float *d_best_fitness);
+
+/* Memory the shared-row pool of schedule_round may take (rows + records; default 12 GiB), to be
+ * set before the first schedule_round of the context.  The pool is sized at twice (the
+ * population + as many worst-case generations as the budget allows, at most 24); with less
+ * room the live rows move between the halves more often (same results, more time), and when
+ * not even two worst-case generations fit, rounds run on dense matrices.  The paper has no
+ * counterpart: a deployment knob.  sched_store_moves: how often the rows have moved since the
+ * context was made (waits for the stream; 0 when rounds run on dense matrices, -1 on a CUDA
+ * error). */
+int sched_set_store_budget(sched_ctx *ctx, uint64_t bytes);
+int64_t sched_store_moves(sched_ctx *ctx);
 
 /* schedule_round replays a CUDA graph of the whole round from the third call on that passes
  * the same pointers and generation count (the second such call captures it); this removes

@@ -22,7 +22,7 @@ EXPORTS = (
     "init_population", "ga_generation", "schedule_round", "schedule_round_host",
     "sched_get_population", "sched_get_round_tables", "sched_round_speedup_table", "eval_fitness_host",
     "sched_set_kernel_timing", "sched_num_kernel_kinds", "sched_kernel_kind_name",
-    "sched_read_kernel_timing", "sched_set_graphs", "eval_fitness_noalloc", "eval_fitness_noalloc_last_error",
+    "sched_read_kernel_timing", "sched_set_graphs", "sched_set_store_budget", "sched_store_moves", "eval_fitness_noalloc", "eval_fitness_noalloc_last_error",
 )
 
 
@@ -84,6 +84,9 @@ def load_library(path: str = LIB_PATH):
     lib.eval_fitness_host.argtypes = [vp, vp, i32, vp, vp, vp, vp, f32, vp]
     lib.sched_set_kernel_timing.argtypes = [vp, i32]
     lib.sched_set_graphs.argtypes = [vp, i32]
+    lib.sched_set_store_budget.argtypes = [vp, C.c_uint64]
+    lib.sched_store_moves.argtypes = [vp]
+    lib.sched_store_moves.restype = C.c_int64
     lib.sched_num_kernel_kinds.argtypes = []
     lib.sched_kernel_kind_name.argtypes = [i32]
     lib.sched_kernel_kind_name.restype = C.c_char_p
@@ -209,6 +212,12 @@ class Scheduler:
 
     def set_graphs(self, enable: bool):
         self._check(_lib.sched_set_graphs(self._ctx, 1 if enable else 0))
+
+    def set_store_budget(self, nbytes: int):
+        self._check(_lib.sched_set_store_budget(self._ctx, int(nbytes)))
+
+    def store_moves(self) -> int:
+        return int(_lib.sched_store_moves(self._ctx))
 
     def read_kernel_timing(self):
         """{kernel class: (total ms, timed launches)} since the previous read-out"""

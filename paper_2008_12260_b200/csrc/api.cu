@@ -246,6 +246,7 @@ int sched_init(const sched_config *cfg, const int16_t *h_node_capacity, void *cu
   if ((rc = dev_alloc(ctx, &ctx->d_colcount, 1)) != SCHED_OK) return fail(rc);
   if ((rc = dev_alloc(ctx, &ctx->d_round, 1)) != SCHED_OK) return fail(rc);
   ctx->graphs_enabled = true;
+  ctx->rs_budget = 12ull << 30;
   e = cudaMemcpyAsync(ctx->d_cap, h_node_capacity, sizeof(int16_t) * cfg->num_nodes,
                       cudaMemcpyHostToDevice, ctx->stream);
   if (e == cudaSuccess)
@@ -328,6 +329,25 @@ int sched_set_graphs(sched_ctx *ctx, int enable) {
   REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "sched_set_graphs: ctx is NULL");
   ctx->graphs_enabled = enable != 0;
   return SCHED_OK;
+}
+
+int sched_set_store_budget(sched_ctx *ctx, uint64_t bytes) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "sched_set_store_budget: ctx is NULL");
+  REQUIRE(ctx, !ctx->round_ready, SCHED_ERR_INVALID_ARG,
+          "sched_set_store_budget: the round scratch exists already (call before the first schedule_round)");
+  ctx->rs_budget = bytes;
+  return SCHED_OK;
+}
+
+int64_t sched_store_moves(sched_ctx *ctx) {
+  if (!ctx || !ctx->rs_ready) return 0;
+  unsigned int moves = 0;
+  if (cudaMemcpyAsync(&moves, ctx->rs_state + 4, sizeof(moves), cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess ||
+      cudaStreamSynchronize(ctx->stream) != cudaSuccess) {
+    cudaGetLastError();
+    return -1;
+  }
+  return (int64_t)moves;
 }
 
 int sched_num_kernel_kinds(void) { return KK_COUNT; }
@@ -507,17 +527,22 @@ static int round_body(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d
     return launch_fitness(ctx, pop, ctx->cfg.population, ctx->d_tab_speedup, d_cur, rf, d_jobs->active,
                           ctx->cfg.p, out, ctx->summ_valid ? ctx->round_summ : nullptr);
   };
-  const bool store = ctx->rs_ready;
-  if (store) pa = ctx->rs_pool;   // the dense initial population is the first P * J slots of the pool
-  if (rc == SCHED_OK) rc = launch_init_population(ctx, d_jobs->k_cap, d_jobs->active, d_cur, pa);
-  if (rc == SCHED_OK) rc = fitness_of(pa, fit_cur);
+  const bool store = ctx->rs_ready && generations > 0;
   int parity = 0;
-  if (store && generations > 0) {
-    // From here on candidates are arrays of row indices: one kernel per generation does the
-    // operators, the repair and the fitness; every few generations a check moves the live rows
-    // to the other half of the pool if the half in use could run out.
-    if (rc == SCHED_OK) rc = rowstore_build(ctx, d_jobs->active, ctx->round_cur, rf ? ctx->d_pen : nullptr);
+  if (store) {
+    // The round runs on the row store: candidates are arrays of row indices.  The current
+    // allocation's rows go in first; the initial population is then made like any generation (its
+    // single parent is the current allocation), by the kernel that also does the operators, the
+    // repair and the fitness; every few generations a check moves the live rows to the other half
+    // of the pool if the half in use could run out.
+    pa = ctx->rs_pool;
+    if (rc == SCHED_OK) rc = rowstore_build_current(ctx, d_jobs->k_cap, d_jobs->active, d_cur, ctx->round_cur,
+                                                    rf ? ctx->d_pen : nullptr);
     int phase = 0;
+    if (rc == SCHED_OK)
+      rc = rowstore_generation(ctx, d_jobs->k_cap, d_jobs->active, ctx->round_cur, rf ? ctx->d_pen : nullptr, fit_next,
+                               fit_cur, 0, phase, GEN_INIT);
+    parity = 1;
     for (int g = 0; g < generations && rc == SCHED_OK; ++g) {
       if (g > 0 && g % ctx->rs_check_every == 0) {
         rc = rowstore_compact(ctx, parity, phase);
@@ -529,6 +554,10 @@ static int round_body(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d
       parity ^= 1;
       std::swap(fit_cur, fit_next);
     }
+  } else {
+    if (ctx->rs_ready) pa = ctx->rs_pool;   // no generations: the dense initial population sits at the start of the pool
+    if (rc == SCHED_OK) rc = launch_init_population(ctx, d_jobs->k_cap, d_jobs->active, d_cur, pa);
+    if (rc == SCHED_OK) rc = fitness_of(pa, fit_cur);
   }
   for (int g = 0; g < generations && rc == SCHED_OK && !store; ++g) {
     ctx->ff_out = fit_next;
@@ -552,7 +581,7 @@ static int round_body(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d
   if (rc != SCHED_OK) return rc;
   ctx->d_pop_last = pa;
   ctx->rs_ptr_last = nullptr;
-  if (store && generations > 0) {
+  if (store) {
     ctx->rs_ptr_last = ctx->rs_ptr + (size_t)parity * ctx->cfg.population * ctx->cfg.num_jobs;
     if ((rc = launch_select_best(ctx, nullptr, ctx->d_fit, nullptr, d_best_fitness)) != SCHED_OK) return rc;
     return rowstore_gather(ctx, ctx->rs_ptr_last, 0, 1, ctx->d_best_idx, d_best);

@@ -103,7 +103,9 @@ struct sched_ctx {
   uint32_t *rs_rec;        // [slots][8] up to 7 occupied nodes of the row (node | GPUs << 12, or an overflow
                            // mark), then K | N << 11 | (entries differing from the current allocation) << 22
   uint32_t *rs_ptr;        // [2][P][J] row index per (candidate, job): parents and children alternate
-  unsigned int *rs_state;  // [2][2] {next free slot, half in use}; the two copies alternate at each compaction check
+  unsigned int *rs_state;  // [2][2] {next free slot, half in use}; the two copies alternate at each compaction check;
+                           // [4]: times the rows have moved to the other half
+  unsigned long long rs_budget;  // bytes the pool (rows + records) may take
   size_t rs_half_cap;      // slots per half of the pool
   int rs_check_every;      // generations between compaction checks
   bool rs_ready;           // the buffers above exist
@@ -277,7 +279,8 @@ void fitness_chunking(const sched_ctx *ctx, int32_t count, int &rows_per_block, 
 // row store (rowstore.cu)
 bool rowstore_eligible(const sched_ctx *ctx, const int16_t *d_cur);
 int rowstore_ensure(sched_ctx *ctx);
-int rowstore_build(sched_ctx *ctx, const uint8_t *d_active, const int16_t *d_cur, const float *d_pen);
+int rowstore_build_current(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active, const int16_t *d_seed,
+                           const int16_t *d_cur, const float *d_pen);
 int rowstore_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active, const int16_t *d_cur,
                         const float *d_pen, const float *d_fitness_in, float *d_fitness_out, int parity,
                         int state_phase, uint32_t generation);

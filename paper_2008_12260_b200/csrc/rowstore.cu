@@ -225,51 +225,92 @@ __device__ __forceinline__ uint32_t pack_summary(int K, int N, int ndiff) {
 }
 
 // ---------------------------------------------------------------------------------------
-// Build: the dense initial population (rows c * J + j at the start of the pool) gets its
-// records and summaries; candidate c, job j points at slot c * J + j.
+// Start of a round on the store: the current allocation's rows become slots 0 .. 2J - 1.
+// Slot j holds job j's row as an unperturbed child of the initial population has it (entries
+// forced into [0, node size], then the row caps); slot J + j holds it before the row caps, which
+// is what a perturbed child starts from.  The initial population itself is then made by the
+// generation kernel with this single "parent".
 // ---------------------------------------------------------------------------------------
-struct BuildArgs {
+struct BuildCurArgs {
   StoreView st;
-  uint32_t *ptr;            // [P][J]
+  uint32_t *ptr;            // [J] the parent's row indices
   unsigned int *state;      // {next free slot, half}
   const uint8_t *active;
-  const int16_t *cur;       // or NULL
+  const int16_t *seed;      // [J][NN] current allocation the population starts from, or NULL (empty cluster)
+  const int16_t *cur;       // [J][NN] current allocation the summaries compare with, or NULL
+  const int16_t *cap;
+  const int32_t *k_cap;
   TermParams tp;
-  int P, J, NN;
+  int J, NN, k_max, n_max;
 };
 
 template <int PPL>
-__global__ void __launch_bounds__(256) rowstore_build_kernel(BuildArgs a) {
+__global__ void __launch_bounds__(256) rowstore_build_cur_kernel(BuildCurArgs a) {
   __shared__ __align__(16) int16_t s_row[16][512];
   __shared__ uint32_t s_rec[16][REC_WORDS];
-  const int lane = threadIdx.x & 31, grp = threadIdx.x >> 4;   // 16 groups of 16 lanes, a row each
+  const int lane = threadIdx.x & 31, grp = threadIdx.x >> 4;
   const Grp g = make_group(lane, a.NN);
-  const long long rows = (long long)a.P * a.J;
   if (blockIdx.x == 0 && threadIdx.x == 0) {
-    a.state[0] = (unsigned int)rows;
+    a.state[0] = 2u * (unsigned int)a.J;
     a.state[1] = 0u;
   }
-  // the empty row: contents and record all zero
-  if (blockIdx.x == 0) {
+  if (blockIdx.x == 0) {    // the empty row: contents and record all zero
     for (int n = threadIdx.x; n < a.NN; n += blockDim.x) a.st.pool[(size_t)a.st.zero_slot * a.NN + n] = 0;
     if (threadIdx.x < REC_WORDS) a.st.rec[(size_t)a.st.zero_slot * REC_WORDS + threadIdx.x] = 0u;
   }
-  for (long long r = (long long)blockIdx.x * 16 + grp; r < rows; r += (long long)gridDim.x * 16) {
-    const int j = (int)(r % a.J);
-    load_row<false>(g, s_row[grp], a.st.pool + (size_t)r * a.NN);
+  for (int j = blockIdx.x * 16 + grp; j < a.J; j += gridDim.x * 16) {
+    const bool on = !a.active || a.active[j];
+    if (g.sub == 0) a.ptr[j] = on ? (uint32_t)j : a.st.zero_slot;
+    if (!on) continue;                                  // (uniform within the group)
+    for (int v = g.sub; v < g.row_vecs; v += GROUP) {
+      uint4 x = make_uint4(0u, 0u, 0u, 0u);
+      if (a.seed) {
+        x = load_piece<false>(a.seed + (size_t)j * a.NN, v);
+        const uint4 cp = *((const uint4 *)a.cap + v);
+        x.x = __vimin_s16x2_relu(x.x, __vimax_s16x2_relu(cp.x, 0u));
+        x.y = __vimin_s16x2_relu(x.y, __vimax_s16x2_relu(cp.y, 0u));
+        x.z = __vimin_s16x2_relu(x.z, __vimax_s16x2_relu(cp.z, 0u));
+        x.w = __vimin_s16x2_relu(x.w, __vimax_s16x2_relu(cp.w, 0u));
+      }
+      ((uint4 *)s_row[grp])[v] = x;
+    }
     const CurPieces<PPL> cur = cur_pieces<PPL>(g, a.cur ? a.cur + (size_t)j * a.NN : nullptr);
     __syncwarp(g.mask);
-    int K, N, nd;
-    summarise_row<PPL>(g, s_row[grp], cur, K, N, nd, s_rec[grp]);
-    const bool on = !a.active || a.active[j];
-    if (g.sub == 0) {
-      s_rec[grp][REC_SUMM] = on ? pack_summary(K, N, nd) : 0u;
-      s_rec[grp][REC_TERM] = on ? __float_as_uint(fitness_term(a.tp, j, K, N, nd != 0)) : 0u;
-      a.ptr[r] = (uint32_t)r;
+    const int kc = max(0, min(a.k_cap ? a.k_cap[j] : a.k_max, a.k_max));
+    for (int pass = 0; pass < 2; ++pass) {              // before the row caps (slot J + j), after them (slot j)
+      int K, N, nd;
+      summarise_row<PPL>(g, s_row[grp], cur, K, N, nd, s_rec[grp]);
+      const size_t slot = pass == 0 ? (size_t)a.J + j : (size_t)j;
+      if (g.sub == 0) {
+        s_rec[grp][REC_SUMM] = pack_summary(K, N, nd);
+        s_rec[grp][REC_TERM] = __float_as_uint(fitness_term(a.tp, j, K, N, nd != 0));
+      }
+      if (N > REC_ENTRIES) store_row(g, a.st.pool + slot * a.NN, s_row[grp]);
+      __syncwarp(g.mask);
+      if (g.sub < REC_WORDS) a.st.rec[slot * REC_WORDS + g.sub] = s_rec[grp][g.sub];
+      __syncwarp(g.mask);
+      if (pass == 0 && (K > kc || N > a.n_max)) {
+        // replicas above the job's cap leave from the highest node index down, then occupied nodes
+        // beyond n_max are cleared from the highest index down
+        if (g.sub == 0) {
+          int16_t *row = s_row[grp];
+          int excess = K - kc;
+          for (int n = a.NN - 1; n >= 0 && excess > 0; --n) {
+            const int take = min((int)row[n], excess);
+            row[n] = (int16_t)(row[n] - take);
+            excess -= take;
+          }
+          int occ = 0;
+          for (int n = 0; n < a.NN; ++n) {
+            if (row[n] > 0) {
+              ++occ;
+              if (occ > a.n_max) row[n] = 0;
+            }
+          }
+        }
+        __syncwarp(g.mask);
+      }
     }
-    __syncwarp(g.mask);
-    if (g.sub < REC_WORDS) a.st.rec[(size_t)r * REC_WORDS + g.sub] = s_rec[grp][g.sub];
-    __syncwarp(g.mask);
   }
 }
 
@@ -290,6 +331,7 @@ struct CompactArgs {
   uint32_t *ptr;            // [P][J] indices of the current population (rewritten)
   const unsigned int *state_in;
   unsigned int *state_out;
+  unsigned int *moves;      // times the rows have moved (since the context was made)
   int P, J, NN, gens_ahead;
 };
 
@@ -307,6 +349,7 @@ __global__ void __launch_bounds__(256) rowstore_compact_kernel(CompactArgs a) {
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     a.state_out[0] = (unsigned int)(base + rows);
     a.state_out[1] = new_half;
+    atomicAdd(a.moves, 1u);
   }
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int row_vecs = a.NN >> 3;
@@ -1426,6 +1469,29 @@ StoreView store_view(const sched_ctx *ctx) {
 
 }  // namespace
 
+// Pool budget (default 12 GiB, sched_set_store_budget) of rows and records; the rows' part is
+// address space more than traffic: a row's contents are only written when its record cannot hold
+// it.  Returns how many generations' worst case a half can take on top of the population, at
+// most 24.
+// rows a half holds before any generation: the population, or the current allocation's two rows
+// per job that a round starts from
+static unsigned long long store_base_rows(const sched_config &c) {
+  const unsigned long long rows = (unsigned long long)c.population * c.num_jobs;
+  return rows > 2ull * c.num_jobs ? rows : 2ull * c.num_jobs;
+}
+
+static int store_units(const sched_config &c, unsigned long long budget) {
+  const unsigned long long rows = store_base_rows(c);
+  const unsigned long long worst = store_worst_case(c.population, c.num_jobs);
+  const unsigned long long row_bytes = (unsigned long long)c.num_nodes * 2 + REC_WORDS * 4;
+  const unsigned long long half_rows = budget / 2 / row_bytes;
+  const unsigned long long index_rows = ((1ull << 32) - 2) / 2;      // slot indices are 32-bit
+  const unsigned long long room = half_rows < index_rows ? half_rows : index_rows;
+  if (room <= rows) return 0;
+  const unsigned long long units = (room - rows) / worst;
+  return (int)(units < 24 ? units : 24);
+}
+
 // The row store serves rounds whose candidates span several row batches of the dense
 // kernels (J > 256; smaller problems run a generation as one dense kernel already), with
 // rows of whole 16-byte vectors and sizes that fit the packed fields.
@@ -1434,42 +1500,40 @@ bool rowstore_eligible(const sched_ctx *ctx, const int16_t *) {
   if (c.num_jobs <= 256 || c.num_jobs > STORE_MAX_JOBS) return false;
   if (c.num_nodes % 8 != 0 || c.num_nodes > 512 || ctx->cap_max > 2047) return false;
   if (c.k_max > 2047 || c.n_max > 2047) return false;
-  const unsigned long long rows = (unsigned long long)c.population * c.num_jobs;
-  const unsigned long long worst = store_worst_case(c.population, c.num_jobs);
-  if (2ull * rows + 17ull * worst >= (1ull << 32)) return false;   // slot indices are 32-bit
   if (gen_smem_layout(c.num_jobs, c.num_nodes).total > 200 * 1024) return false;
-  // a half holds the population plus at least two generations' worst case; beyond 8 GiB of pool
-  // the dense path runs
-  const unsigned long long row_bytes = (unsigned long long)c.num_nodes * 2 + REC_WORDS * 4;
-  return 2ull * (rows + 2ull * worst) * row_bytes <= (8ull << 30);
+  // a half holds the population plus at least two generations' worst case; if that does not fit
+  // the pool's budget (or 32-bit slot indices) the dense path runs
+  return store_units(c, ctx->rs_budget) >= 2;
 }
 
 int rowstore_ensure(sched_ctx *ctx) {
   if (ctx->rs_ready) return SCHED_OK;
   const sched_config &c = ctx->cfg;
   const unsigned long long rows = (unsigned long long)c.population * c.num_jobs;
-  const unsigned long long row_bytes = (unsigned long long)c.num_nodes * 2 + REC_WORDS * 4;
-  // half = the population + (gens between checks + slack) generations' worst case; shrink until
-  // the pool fits 8 GiB
-  int check = 4, slack = 4;
+  // half = the population + `units` generations' worst case.  The check runs every `check`
+  // generations and moves the rows once fewer than `check` units are left, i.e. after the other
+  // units - check have been used up: real generations take a few percent of the worst case, so
+  // a wide margin means a move is rare and a long interval means few check launches.
+  const int units = store_units(c, ctx->rs_budget);
+  const int check = units / 2 < 1 ? 1 : units / 2 > 12 ? 12 : units / 2;
   const unsigned long long worst = store_worst_case(c.population, c.num_jobs);
-  while (2ull * (rows + (check + slack) * worst) * row_bytes > (8ull << 30) && (check > 1 || slack > 1)) {
-    if (slack > 1) --slack; else --check;
-  }
   ctx->rs_check_every = check;
-  ctx->rs_half_cap = (size_t)(rows + (check + slack) * worst);
+  ctx->rs_half_cap = (size_t)(store_base_rows(c) + (unsigned long long)units * worst);
   const size_t slots = 2 * ctx->rs_half_cap + 1;
   cudaError_t e = cudaMalloc((void **)&ctx->rs_pool, slots * c.num_nodes * sizeof(int16_t));
   if (e == cudaSuccess) e = cudaMalloc((void **)&ctx->rs_rec, slots * REC_WORDS * sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaMalloc((void **)&ctx->rs_ptr, 2 * (size_t)rows * sizeof(uint32_t));
-  if (e == cudaSuccess) e = cudaMalloc((void **)&ctx->rs_state, 4 * sizeof(unsigned int));
+  if (e == cudaSuccess) e = cudaMalloc((void **)&ctx->rs_state, 5 * sizeof(unsigned int));
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->rs_state, 0, 5 * sizeof(unsigned int), ctx->stream);
   if (e == cudaSuccess) {
     const size_t smem = gen_smem_layout(c.num_jobs, c.num_nodes).total;
     if (smem > 48 * 1024)
-    for (int k = 0; k < 3 && e == cudaSuccess; ++k)
-      e = cudaFuncSetAttribute(k == 0 ? generation_store_kernel<1, false> : k == 1 ? generation_store_kernel<2, false>
-                                                                                  : generation_store_kernel<4, false>,
-                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    for (int k = 0; k < 6 && e == cudaSuccess; ++k) {
+      void (*kernel)(GenArgs) = k == 0 ? generation_store_kernel<1, false> : k == 1 ? generation_store_kernel<2, false>
+                                : k == 2 ? generation_store_kernel<4, false> : k == 3 ? generation_store_kernel<1, true>
+                                : k == 4 ? generation_store_kernel<2, true> : generation_store_kernel<4, true>;
+      e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    }
   }
   if (e != cudaSuccess) {
     set_error(ctx, "row store allocation failed: %s", cudaGetErrorString(e));
@@ -1484,23 +1548,25 @@ int rowstore_ensure(sched_ctx *ctx) {
   return SCHED_OK;
 }
 
-int rowstore_build(sched_ctx *ctx, const uint8_t *d_active, const int16_t *d_cur, const float *d_pen) {
+int rowstore_build_current(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active, const int16_t *d_seed,
+                           const int16_t *d_cur, const float *d_pen) {
   const sched_config &c = ctx->cfg;
-  BuildArgs a;
+  BuildCurArgs a;
   a.st = store_view(ctx);
   a.ptr = ctx->rs_ptr;
   a.state = ctx->rs_state;
-  a.active = d_active; a.cur = d_cur;
+  a.active = d_active; a.seed = d_seed; a.cur = d_cur; a.cap = ctx->d_cap; a.k_cap = d_k_cap;
   a.tp.table = ctx->d_tab_speedup; a.tp.pen = d_pen; a.tp.active = d_active;
   a.tp.k_max = c.k_max; a.tp.n_max = c.n_max; a.tp.mode = fitness_mode(c.p); a.tp.p = c.p;
   a.tp.floor_ = c.speedup_floor;
-  a.P = c.population; a.J = c.num_jobs; a.NN = c.num_nodes;
+  a.J = c.num_jobs; a.NN = c.num_nodes; a.k_max = c.k_max; a.n_max = c.n_max;
   {
     TimedLaunch tl_(ctx, KK_STORE_BUILD);
     const int ppl = store_pieces_per_lane(c.num_nodes);
-    if (ppl == 1) rowstore_build_kernel<1><<<ctx->num_sms * 8, 256, 0, ctx->stream>>>(a);
-    else if (ppl == 2) rowstore_build_kernel<2><<<ctx->num_sms * 8, 256, 0, ctx->stream>>>(a);
-    else rowstore_build_kernel<4><<<ctx->num_sms * 8, 256, 0, ctx->stream>>>(a);
+    const int blocks = (c.num_jobs + 15) / 16;
+    if (ppl == 1) rowstore_build_cur_kernel<1><<<blocks, 256, 0, ctx->stream>>>(a);
+    else if (ppl == 2) rowstore_build_cur_kernel<2><<<blocks, 256, 0, ctx->stream>>>(a);
+    else rowstore_build_cur_kernel<4><<<blocks, 256, 0, ctx->stream>>>(a);
   }
   SCHED_LAUNCH_CHECK(ctx);
   return SCHED_OK;
@@ -1513,6 +1579,7 @@ int rowstore_compact(sched_ctx *ctx, int parity, int state_phase) {
   a.ptr = ctx->rs_ptr + (size_t)parity * c.population * c.num_jobs;
   a.state_in = ctx->rs_state + 2 * state_phase;
   a.state_out = ctx->rs_state + 2 * (state_phase ^ 1);
+  a.moves = ctx->rs_state + 4;
   a.P = c.population; a.J = c.num_jobs; a.NN = c.num_nodes;
   a.gens_ahead = ctx->rs_check_every;
   {
@@ -1539,9 +1606,12 @@ int rowstore_gather(sched_ctx *ctx, const uint32_t *d_ptr, int first_candidate, 
   return SCHED_OK;
 }
 
+// generation == GEN_INIT: the initial population, made from the rows rowstore_build_current left
+// (children are the current allocation perturbed with thr_init; they go to index set `parity ^ 1`)
 int rowstore_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active, const int16_t *d_cur,
                         const float *d_pen, const float *d_fitness_in, float *d_fitness_out, int parity,
                         int state_phase, uint32_t generation) {
+  const bool init = generation == GEN_INIT;
   const sched_config &c = ctx->cfg;
   const size_t rows = (size_t)c.population * c.num_jobs;
   GenArgs a;
@@ -1554,7 +1624,7 @@ int rowstore_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d
   a.cur = d_cur;
   a.P = c.population; a.J = c.num_jobs; a.NN = c.num_nodes;
   a.k_max = c.k_max; a.n_max = c.n_max; a.num_elite = c.num_elite;
-  a.thr = c.thr_mutate; a.gen = generation; a.init_src = 0u;
+  a.thr = init ? c.thr_init : c.thr_mutate; a.gen = generation; a.init_src = (uint32_t)c.num_jobs;
   a.key = make_key(c.seed, ctx->d_round);
   a.tp.table = ctx->d_tab_speedup; a.tp.pen = d_pen; a.tp.active = d_active;
   a.tp.k_max = c.k_max; a.tp.n_max = c.n_max; a.tp.mode = fitness_mode(c.p); a.tp.p = c.p;
@@ -1568,8 +1638,10 @@ int rowstore_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d
     // launched so that it may start while the previous kernel of the stream still runs: the kernel
     // does its draws first and waits for that kernel before it reads anything it wrote
     const int ppl = store_pieces_per_lane(c.num_nodes);
-    void (*kernel)(GenArgs) = ppl == 1 ? generation_store_kernel<1, false>
-                              : ppl == 2 ? generation_store_kernel<2, false> : generation_store_kernel<4, false>;
+    void (*kernel)(GenArgs) = init ? (ppl == 1 ? generation_store_kernel<1, true>
+                                      : ppl == 2 ? generation_store_kernel<2, true> : generation_store_kernel<4, true>)
+                                   : (ppl == 1 ? generation_store_kernel<1, false>
+                                      : ppl == 2 ? generation_store_kernel<2, false> : generation_store_kernel<4, false>);
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3((unsigned)c.population);
     lc.blockDim = dim3(GEN_THREADS);

@@ -95,6 +95,11 @@ def test_store_round_equals_dense_stepwise_round(gpu, oracle, cfg):
     penalise = cur is not None
     rnd = 3
     s = api.scheduler_for(cfg, stream=torch.cuda.current_stream().cuda_stream)
+    if cfg.name == "store-compaction":
+        # a pool with room for two worst-case generations per half: the rows have to move every
+        # other generation or so
+        rows, worst = cfg.population * cfg.num_jobs, cfg.population * (cfg.num_jobs + 16)
+        s.set_store_budget(2 * (cfg.num_nodes * 2 + 32) * (rows + 2 * worst + 64))
     dj = api.DeviceJobs(jobs, "cuda:0", torch)
     d_cur = None if cur is None else torch.from_numpy(cur).cuda()
     best = torch.full((cfg.num_jobs, cfg.num_nodes), -1, dtype=torch.int16, device="cuda:0")
@@ -113,6 +118,10 @@ def test_store_round_equals_dense_stepwise_round(gpu, oracle, cfg):
     assert np.array_equal(best.cpu().numpy(), pop[i]) and float(bf.item()) == fit[i]
     for c in range(cfg.population):
         assert feasible(pop[c], cl.node_capacity, jobs.k_cap, cl.n_max)
+    if cfg.name == "store-compaction":
+        assert s.store_moves() >= 3
+    elif cfg.name.startswith("store-"):
+        assert s.store_moves() == 0
     if cfg.name == "store-crowded-nodes":
         assert (pop > 0).sum(axis=1).max() > 16      # more jobs on a node than a block lists
     if cfg.name == "small-crowded-nodes":
