@@ -299,3 +299,70 @@ def build_speedup_table_msample(jobs, node_capacity, k_max, n_max, m_samples, m_
     if rc != 0:
         raise ValueError("oracle_build_speedup_table_msample: bad arguments")
     return gp, sp, am
+
+
+def set_threads(n: int):
+    """Threads of the oracle's parallel loops (1 = single core; 0 = all)."""
+    lib().oracle_set_threads(int(n))
+
+
+def t_sync_rack(alpha_local, beta_local, alpha_node, beta_node, alpha_rack, beta_rack, K, N, R):
+    f = lib().oracle_t_sync_rack
+    f.restype = C.c_double
+    f.argtypes = [C.c_double] * 6 + [C.c_int] * 3
+    return float(f(alpha_local, beta_local, alpha_node, beta_node, alpha_rack, beta_rack, K, N, R))
+
+
+def goodput_rack(alpha_grad, beta_grad, alpha_local, beta_local, alpha_node, beta_node, alpha_rack, beta_rack,
+                 gamma, phi, m0, m_max_total, K, N, R, m, s):
+    """Returns (goodput, feasible) with the three-class T_sync."""
+    f = lib().oracle_goodput_rack
+    f.restype = C.c_double
+    f.argtypes = [C.c_double] * 12 + [C.c_int] * 5 + [C.c_void_p]
+    ok = C.c_int(0)
+    g = f(alpha_grad, beta_grad, alpha_local, beta_local, alpha_node, beta_node, alpha_rack, beta_rack, gamma, phi,
+          m0, m_max_total, K, N, R, m, s, C.byref(ok))
+    return float(g), bool(ok.value)
+
+
+def build_speedup_table_rack(jobs, node_capacity, k_max, n_max, grid_s, want_argmax=True):
+    """Third-class tables (allocations that span racks); jobs also carries alpha_rack, beta_rack."""
+    cap = _c(node_capacity, np.int16)
+    fa = _job_args(jobs)
+    ar = _c(jobs.alpha_rack, np.float32)
+    br = _c(jobs.beta_rack, np.float32)
+    mg = _c(jobs.m_grid, np.int32)
+    fk = _c(jobs.fair_k, np.int32)
+    fn = _c(jobs.fair_n, np.int32)
+    J, Gm = mg.shape
+    shape = (J, k_max + 1, n_max + 1)
+    gp = np.zeros(shape, dtype=np.float64)
+    sp = np.zeros(shape, dtype=np.float64)
+    am = np.zeros(shape, dtype=np.uint16) if want_argmax else None
+    rc = lib().oracle_build_speedup_table_rack(
+        J, cap.shape[0], _p(cap), int(k_max), int(n_max), int(Gm), int(grid_s),
+        *[_p(a) for a in fa[:6]], _p(ar), _p(br), *[_p(a) for a in fa[6:]], _p(mg), _p(fk), _p(fn), _p(gp), _p(sp),
+        _p(am))
+    if rc != 0:
+        raise ValueError("oracle_build_speedup_table_rack: bad arguments")
+    return gp, sp, am
+
+
+def eval_fitness_racks(pop, speedup, speedup_rack, node_rack, k_max, n_max, p, floor, cur=None, realloc=None,
+                       active=None):
+    pop = _c(pop, np.int16)
+    P, J, N = pop.shape
+    sp = _c(speedup, np.float64)
+    spr = _c(speedup_rack, np.float64)
+    assert sp.shape == (J, k_max + 1, n_max + 1) and spr.shape == sp.shape
+    rack = _c(node_rack, np.int16)
+    assert rack.shape == (N,)
+    cur = _c(cur, np.int16)
+    rf = _c(realloc, np.float64)
+    act = _c(active, np.uint8)
+    out = np.empty(P, dtype=np.float64)
+    rc = lib().oracle_eval_fitness_racks(P, J, N, int(k_max), int(n_max), _p(pop), _p(sp), _p(spr), _p(rack), _p(cur),
+                                         _p(rf), _p(act), C.c_double(p), C.c_double(floor), _p(out))
+    if rc != 0:
+        raise ValueError("oracle_eval_fitness_racks: bad arguments")
+    return out

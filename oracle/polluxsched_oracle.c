@@ -670,3 +670,167 @@ int oracle_num_threads(void) {
 #endif
     return n;
 }
+
+/* ------------------------------------------------------------------------- */
+/* Rack-level locality                                                        */
+/* ------------------------------------------------------------------------- */
+
+/* T_sync with the extension the paper names right after Eq. 9 ("a third pair of
+ * parameters" for rack-level locality).  Read as three placement classes: all replicas on
+ * one node -> local pair; several nodes of one rack -> node pair; nodes of two or more racks
+ * (R >= 2 racks occupied) -> rack pair.  Linear in K - 2 like the other two. */
+double oracle_t_sync_rack(double alpha_local, double beta_local, double alpha_node, double beta_node,
+                          double alpha_rack, double beta_rack, int K, int N, int R) {
+    if (K <= 1) return 0.0;
+    if (N == 1) return alpha_local + beta_local * (double)(K - 2);
+    if (R <= 1) return alpha_node + beta_node * (double)(K - 2);
+    return alpha_rack + beta_rack * (double)(K - 2);
+}
+
+/* GOODPUT of Eq. 4/7 with the three-class T_sync. */
+double oracle_goodput_rack(double alpha_grad, double beta_grad, double alpha_local, double beta_local,
+                           double alpha_node, double beta_node, double alpha_rack, double beta_rack,
+                           double gamma, double phi, double m0, double m_max_total, int K, int N, int R,
+                           int m, int s, int *feasible) {
+    double M = (double)K * (double)m * (double)(s + 1);
+    int ok = (K >= 1 && N >= 1 && N <= K && R >= 1 && R <= N && M >= m0 && M <= m_max_total);
+    if (feasible) *feasible = ok;
+    if (!ok) return 0.0;
+    double tg = oracle_t_grad(alpha_grad, beta_grad, (double)m);
+    double ts = oracle_t_sync_rack(alpha_local, beta_local, alpha_node, beta_node, alpha_rack, beta_rack, K, N, R);
+    double ti = oracle_t_iter(tg, ts, gamma, s);
+    return (M / ti) * oracle_efficiency(phi, m0, M);
+}
+
+/* The table of the third class: entry (K, N), N >= 2, is the best goodput over the grid of an
+ * allocation of K replicas on N nodes that lie in two or more racks, and its ratio to the same
+ * fair-share goodput as the two-class table uses (Eq. 15; the fair share is packed on as few
+ * nodes as possible, hence inside one rack).  Validity of (K, N) and ties as in
+ * oracle_build_speedup_table; entries with N < 2 are 0 / 0xFFFF. */
+int oracle_build_speedup_table_rack(int J, int num_nodes, const int16_t *cap, int k_max, int n_max,
+                                    int grid_m, int grid_s, const float *alpha_grad,
+                                    const float *beta_grad, const float *alpha_local,
+                                    const float *beta_local, const float *alpha_node,
+                                    const float *beta_node, const float *alpha_rack,
+                                    const float *beta_rack, const float *gamma, const float *phi,
+                                    const float *m0, const float *m_max_total, const int32_t *m_grid,
+                                    const int32_t *fair_k, const int32_t *fair_n, double *goodput,
+                                    double *speedup, uint16_t *argmax) {
+    if (J < 0 || k_max < 1 || n_max < 1 || grid_m < 1 || grid_s < 1) return ORACLE_ERR_ARG;
+    const int KD = k_max + 1, ND = n_max + 1;
+    int64_t *kfit = (int64_t *)malloc(sizeof(int64_t) * (size_t)ND);
+    max_k_per_n(num_nodes, cap, n_max, kfit);
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int j = 0; j < J; ++j) {
+        double *gj = goodput + (size_t)j * KD * ND;
+        double *sj = speedup + (size_t)j * KD * ND;
+        uint16_t *aj = argmax ? argmax + (size_t)j * KD * ND : NULL;
+        for (int K = 0; K < KD; ++K) {
+            for (int N = 0; N < ND; ++N) {
+                double best = 0.0;
+                int best_s = -1, best_i = -1;
+                int valid = (N >= 2 && K >= N && (int64_t)K <= kfit[N]);
+                if (valid) {
+                    for (int i = 0; i < grid_m; ++i) {
+                        for (int s = 0; s < grid_s; ++s) {
+                            int ok = 0;
+                            double g = oracle_goodput_rack(alpha_grad[j], beta_grad[j], alpha_local[j], beta_local[j],
+                                                           alpha_node[j], beta_node[j], alpha_rack[j], beta_rack[j],
+                                                           gamma[j], phi[j], m0[j], m_max_total[j], K, N, 2,
+                                                           m_grid[(size_t)j * grid_m + i], s, &ok);
+                            if (!ok) continue;
+                            int better = (best_i < 0) || (g > best) ||
+                                         (g == best && (s < best_s || (s == best_s && i < best_i)));
+                            if (better) { best = g; best_s = s; best_i = i; }
+                        }
+                    }
+                }
+                gj[K * ND + N] = (best_i >= 0) ? best : 0.0;
+                if (aj) aj[K * ND + N] = (best_i >= 0) ? (uint16_t)(best_i * grid_s + best_s) : 0xFFFFu;
+            }
+        }
+        /* the fair-share goodput: one rack, so the local or the node pair */
+        int kf = fair_k[j], nf = fair_n[j];
+        double denom = 0.0;
+        if (nf >= 1 && nf <= n_max && kf >= nf && kf <= k_max && (int64_t)kf <= kfit[nf]) {
+            for (int i = 0; i < grid_m; ++i) {
+                for (int s = 0; s < grid_s; ++s) {
+                    int ok = 0;
+                    double g = oracle_goodput_rack(alpha_grad[j], beta_grad[j], alpha_local[j], beta_local[j],
+                                                   alpha_node[j], beta_node[j], alpha_rack[j], beta_rack[j], gamma[j],
+                                                   phi[j], m0[j], m_max_total[j], kf, nf, 1,
+                                                   m_grid[(size_t)j * grid_m + i], s, &ok);
+                    if (ok && g > denom) denom = g;
+                }
+            }
+        }
+        for (int e = 0; e < KD * ND; ++e) sj[e] = (denom > 0.0) ? gj[e] / denom : 0.0;
+    }
+    free(kfit);
+    return ORACLE_OK;
+}
+
+/* Eq. 14 with rack-level locality: as oracle_eval_fitness, but a row whose occupied nodes lie in
+ * two or more racks (node_rack[n] = rack of node n) takes its speedup from the third-class
+ * table. */
+int oracle_eval_fitness_racks(int P, int J, int num_nodes, int k_max, int n_max, const int16_t *pop,
+                              const double *speedup, const double *speedup_rack, const int16_t *node_rack,
+                              const int16_t *cur, const double *realloc_factor, const uint8_t *active, double p,
+                              double floor_, double *fitness) {
+    if (P < 0 || J < 0 || num_nodes < 1 || !pop || !speedup || !speedup_rack || !node_rack || !fitness)
+        return ORACLE_ERR_ARG;
+    const int KD = k_max + 1, ND = n_max + 1;
+#pragma omp parallel for schedule(static)
+    for (int c = 0; c < P; ++c) {
+        double acc = 0.0;
+        int64_t count = 0;
+        for (int j = 0; j < J; ++j) {
+            if (active && !active[j]) continue;
+            const int16_t *row = pop + ((size_t)c * J + j) * num_nodes;
+            int64_t K = 0, N = 0, Kcur = 0;
+            int changed = 0, first_rack = -1, several_racks = 0;
+            for (int n = 0; n < num_nodes; ++n) {
+                K += row[n];
+                N += (row[n] > 0);
+                if (row[n] > 0) {
+                    if (first_rack < 0) first_rack = node_rack[n];
+                    else if (node_rack[n] != first_rack) several_racks = 1;
+                }
+                if (cur) {
+                    Kcur += cur[(size_t)j * num_nodes + n];
+                    changed |= (row[n] != cur[(size_t)j * num_nodes + n]);
+                }
+            }
+            if (K < 0) K = 0;
+            if (K > k_max) K = k_max;
+            if (N > n_max) N = n_max;
+            const double *table = several_racks ? speedup_rack : speedup;
+            double x = table[((size_t)j * KD + K) * ND + N];
+            if (cur && realloc_factor && changed && Kcur > 0) x *= realloc_factor[j];
+            if (x < floor_) x = floor_;
+            if (p == 0.0) acc += log(x);
+            else if (p == 1.0) acc += x;
+            else if (p == -1.0) acc += 1.0 / x;
+            else acc += pow(x, p);
+            ++count;
+        }
+        double f;
+        if (count == 0) f = 0.0;
+        else if (p == 0.0) f = exp(acc / (double)count);
+        else if (p == 1.0) f = acc / (double)count;
+        else if (p == -1.0) f = (double)count / acc;
+        else f = pow(acc / (double)count, 1.0 / p);
+        fitness[c] = f;
+    }
+    return ORACLE_OK;
+}
+
+/* Threads the parallel loops above use from now on (1: the single-core figure the paper's
+ * scheduler is quoted on); 0 restores the default. */
+void oracle_set_threads(int n) {
+#ifdef _OPENMP
+    omp_set_num_threads(n > 0 ? n : omp_get_num_procs());
+#else
+    (void)n;
+#endif
+}
