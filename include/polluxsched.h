@@ -164,6 +164,33 @@ int build_speedup_table_msample(sched_ctx *ctx, const sched_jobs *d_jobs, const 
                                 int32_t num_samples, const int32_t *d_m_max_gpu, const uint8_t *d_adaptive,
                                 float *d_goodput, float *d_speedup, uint16_t *d_argmax);
 
+/* Rack-level locality: "our model for T_sync can be extended to account for rack-level locality
+ * by adding a third pair of parameters" (the sentence after Eq. 9).  Read as three placement
+ * classes: all replicas on one node -> local pair; several nodes of one rack -> node pair;
+ * nodes of two or more racks -> rack pair, T_sync = alpha_rack + beta_rack (K - 2).
+ *
+ * sched_set_racks gives the context the rack of every node (h_node_rack: HOST int16
+ * [num_nodes], rack ids >= 0; NULL: one rack again) and the rack pair (DEVICE fp32 [J] each,
+ * caller-owned, must stay valid while the context uses them; NULL = the node pair).  To be
+ * called before the first schedule_round.  With racks set, schedule_round builds the
+ * third-class table as well and evaluates every candidate with eval_fitness_racks; such rounds
+ * run on dense matrices (the shared-row representation is not used).
+ *
+ * build_speedup_table_rack: tables of the third class.  Entry (K, N) with N >= 2 (valid as in
+ * build_speedup_table) is the best goodput over the grid with the rack pair, and its ratio to
+ * the SAME fair-share goodput as the two-class table (the fair share is packed on as few nodes
+ * as possible, so inside one rack); entries with N < 2 are 0 / 0xFFFF.  Outputs as
+ * build_speedup_table; d_goodput and d_argmax may be NULL.
+ *
+ * eval_fitness_racks: eval_fitness, but a row whose occupied nodes lie in two or more racks
+ * reads d_speedup_rack instead of d_speedup.  Needs sched_set_racks. */
+int sched_set_racks(sched_ctx *ctx, const int16_t *h_node_rack, const float *d_alpha_rack, const float *d_beta_rack);
+int build_speedup_table_rack(sched_ctx *ctx, const sched_jobs *d_jobs, const float *d_alpha_rack,
+                             const float *d_beta_rack, float *d_goodput, float *d_speedup, uint16_t *d_argmax);
+int eval_fitness_racks(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const float *d_speedup,
+                       const float *d_speedup_rack, const int16_t *d_cur, const float *d_realloc_factor,
+                       const uint8_t *d_active, float p, float *d_fitness);
+
 /* Batched fit of the throughput-model parameters (Sec. 4.1, online model fitting).  For each
  * of num_jobs jobs (independent of cfg.num_jobs) the observations offset[j] .. offset[j+1] of
  * (K, N, m, s, T_iter) are fitted by theta = (alpha_grad, beta_grad, alpha_local, beta_local,

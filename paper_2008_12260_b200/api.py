@@ -18,7 +18,7 @@ ERRORS = {-1: "INVALID_ARG", -2: "BAD_CONFIG", -3: "CUDA", -4: "TIMEOUT", -5: "N
 
 EXPORTS = (
     "sched_init", "sched_fair_share", "sched_destroy", "sched_last_error", "sched_sync_status", "sched_launch_count",
-    "build_speedup_table", "build_speedup_table_msample", "fit_throughput_model", "compute_realloc_factor", "autoscale_targets", "eval_fitness", "repair_population",
+    "build_speedup_table", "build_speedup_table_msample", "sched_set_racks", "build_speedup_table_rack", "eval_fitness_racks", "fit_throughput_model", "compute_realloc_factor", "autoscale_targets", "eval_fitness", "repair_population",
     "init_population", "ga_generation", "schedule_round", "schedule_round_host",
     "sched_get_population", "sched_get_round_tables", "sched_round_speedup_table", "eval_fitness_host",
     "sched_set_kernel_timing", "sched_num_kernel_kinds", "sched_kernel_kind_name",
@@ -68,6 +68,9 @@ def load_library(path: str = LIB_PATH):
     lib.sched_launch_count.restype = C.c_int64
     lib.build_speedup_table.argtypes = [vp, C.POINTER(SchedJobs), vp, vp, vp]
     lib.build_speedup_table_msample.argtypes = [vp, C.POINTER(SchedJobs), vp, i32, vp, vp, vp, vp, vp]
+    lib.sched_set_racks.argtypes = [vp, vp, vp, vp]
+    lib.build_speedup_table_rack.argtypes = [vp, C.POINTER(SchedJobs), vp, vp, vp, vp, vp]
+    lib.eval_fitness_racks.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, f32, vp]
     lib.fit_throughput_model.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp]
     lib.compute_realloc_factor.argtypes = [vp, C.POINTER(SchedJobs), vp]
     lib.autoscale_targets.argtypes = [vp, vp, vp, i32, f32, f32, vp]
@@ -236,6 +239,21 @@ class Scheduler:
         self._check(_lib.build_speedup_table_msample(self._ctx, C.byref(jobs.struct), _ptr(m_samples),
                                                      m_samples.shape[1], _ptr(m_max_gpu), _ptr(adaptive),
                                                      _ptr(goodput), _ptr(speedup), _ptr(argmax)))
+
+    def set_racks(self, node_rack, alpha_rack=None, beta_rack=None):
+        rack = None if node_rack is None else np.ascontiguousarray(node_rack, dtype=np.int16)
+        self._racks = (alpha_rack, beta_rack)          # keep the device arrays alive
+        self._check(_lib.sched_set_racks(self._ctx, _ptr(rack), _ptr(alpha_rack), _ptr(beta_rack)))
+
+    def build_speedup_table_rack(self, jobs, alpha_rack, beta_rack, goodput, speedup, argmax=None):
+        self._check(_lib.build_speedup_table_rack(self._ctx, C.byref(jobs.struct), _ptr(alpha_rack), _ptr(beta_rack),
+                                                  _ptr(goodput), _ptr(speedup), _ptr(argmax)))
+
+    def eval_fitness_racks(self, pop, speedup, speedup_rack, fitness, *, p, cur=None, realloc_factor=None, active=None,
+                           count=None):
+        n = pop.shape[0] if count is None else count
+        self._check(_lib.eval_fitness_racks(self._ctx, _ptr(pop), n, _ptr(speedup), _ptr(speedup_rack), _ptr(cur),
+                                            _ptr(realloc_factor), _ptr(active), p, _ptr(fitness)))
 
     def fit_throughput_model(self, offset, k, n, m, s, t, theta0, theta_out, loss_out, *, frozen=None, max_iters=100):
         self._check(_lib.fit_throughput_model(self._ctx, theta0.shape[0], _ptr(offset), _ptr(k), _ptr(n), _ptr(m),

@@ -79,7 +79,7 @@ int ensure_round_scratch(sched_ctx *ctx) {
   int rc;
   // Large problems keep the round's population in the row store, whose pool starts with the
   // dense initial population; if it cannot be allocated the round runs on dense matrices.
-  if (rowstore_eligible(ctx, nullptr) && !ctx->rs_off) {
+  if (rowstore_eligible(ctx, nullptr) && !ctx->rs_off && !ctx->d_rack) {
     if (rowstore_ensure(ctx) != SCHED_OK) ctx->rs_off = true;
   }
   if (!ctx->rs_ready) {
@@ -90,6 +90,7 @@ int ensure_round_scratch(sched_ctx *ctx) {
   ctx->d_fit = ctx->d_fit_buf;
   if ((rc = dev_alloc(ctx, &ctx->d_tab_goodput, tab)) != SCHED_OK) return rc;
   if ((rc = dev_alloc(ctx, &ctx->d_tab_speedup, tab)) != SCHED_OK) return rc;
+  if (ctx->d_rack && (rc = dev_alloc(ctx, &ctx->d_tab_speedup_rack, tab)) != SCHED_OK) return rc;
   if ((rc = dev_alloc(ctx, &ctx->d_rf, (size_t)c.num_jobs)) != SCHED_OK) return rc;
   if ((rc = dev_alloc(ctx, &ctx->d_summ, 2 * (size_t)c.population * c.num_jobs)) != SCHED_OK) return rc;
   ctx->round_ready = true;
@@ -292,7 +293,8 @@ int sched_destroy(sched_ctx *ctx) {
                   ctx->d_dflag, ctx->d_pen, ctx->d_partial, ctx->d_ticket, ctx->d_status,
                   ctx->d_popA, ctx->d_popB, ctx->d_fit_buf, ctx->d_tab_goodput, ctx->d_tab_speedup,
                   ctx->d_rf, ctx->d_best_idx, ctx->d_stage, ctx->d_stage_fit, ctx->d_colsum, ctx->d_summ, ctx->d_collist, ctx->d_colcount, ctx->d_rowticket, ctx->d_round, ctx->d_occcount, ctx->d_occlist,
-                  ctx->d_colelig, ctx->rs_pool, ctx->rs_rec, ctx->rs_ptr, ctx->rs_state};
+                  ctx->d_colelig, ctx->rs_pool, ctx->rs_rec, ctx->rs_ptr, ctx->rs_state, ctx->d_gmax_rack,
+                  ctx->d_amax_rack, ctx->d_rack, ctx->d_tab_speedup_rack};
   for (void *p : ptrs)
     if (p) cudaFree(p);
   if (ctx->h_stage) cudaFreeHost(ctx->h_stage);
@@ -348,6 +350,61 @@ int64_t sched_store_moves(sched_ctx *ctx) {
     return -1;
   }
   return (int64_t)moves;
+}
+
+int sched_set_racks(sched_ctx *ctx, const int16_t *h_node_rack, const float *d_alpha_rack, const float *d_beta_rack) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "sched_set_racks: ctx is NULL");
+  REQUIRE(ctx, !ctx->round_ready, SCHED_ERR_INVALID_ARG,
+          "sched_set_racks: the round scratch exists already (call before the first schedule_round)");
+  if (!h_node_rack) {
+    if (ctx->d_rack) {
+      SCHED_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
+      SCHED_CUDA_CHECK(ctx, cudaFree(ctx->d_rack));
+    }
+    ctx->d_rack = nullptr;
+    ctx->d_alpha_rack = ctx->d_beta_rack = nullptr;
+    return SCHED_OK;
+  }
+  for (int n = 0; n < ctx->cfg.num_nodes; ++n)
+    REQUIRE(ctx, h_node_rack[n] >= 0, SCHED_ERR_INVALID_ARG, "sched_set_racks: node %d has a negative rack", n);
+  if (!ctx->d_rack) {
+    int rc = dev_alloc(ctx, &ctx->d_rack, (size_t)ctx->cfg.num_nodes);
+    if (rc != SCHED_OK) return rc;
+  }
+  SCHED_CUDA_CHECK(ctx, cudaMemcpyAsync(ctx->d_rack, h_node_rack, sizeof(int16_t) * ctx->cfg.num_nodes,
+                                        cudaMemcpyHostToDevice, ctx->stream));
+  SCHED_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));   // the host array may go away
+  ctx->d_alpha_rack = d_alpha_rack;
+  ctx->d_beta_rack = d_beta_rack;
+  return SCHED_OK;
+}
+
+int build_speedup_table_rack(sched_ctx *ctx, const sched_jobs *d_jobs, const float *d_alpha_rack,
+                             const float *d_beta_rack, float *d_goodput, float *d_speedup, uint16_t *d_argmax) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "build_speedup_table_rack: ctx is NULL");
+  int rc = check_table_jobs(ctx, d_jobs);
+  if (rc != SCHED_OK) return rc;
+  REQUIRE(ctx, d_alpha_rack && d_beta_rack && d_speedup, SCHED_ERR_INVALID_ARG,
+          "build_speedup_table_rack: d_alpha_rack, d_beta_rack and d_speedup must be non-NULL");
+  return launch_speedup_table_rack(ctx, d_jobs, d_alpha_rack, d_beta_rack, d_goodput, d_speedup, d_argmax);
+}
+
+int eval_fitness_racks(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const float *d_speedup,
+                       const float *d_speedup_rack, const int16_t *d_cur, const float *d_realloc_factor,
+                       const uint8_t *d_active, float p, float *d_fitness) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "eval_fitness_racks: ctx is NULL");
+  REQUIRE(ctx, ctx->d_rack, SCHED_ERR_INVALID_ARG, "eval_fitness_racks: no racks set (sched_set_racks)");
+  REQUIRE(ctx, count >= 0, SCHED_ERR_INVALID_ARG, "eval_fitness_racks: count is negative");
+  REQUIRE(ctx, count == 0 || (d_pop && d_speedup && d_speedup_rack && d_fitness), SCHED_ERR_INVALID_ARG,
+          "eval_fitness_racks: d_pop, d_speedup, d_speedup_rack and d_fitness must be non-NULL");
+  REQUIRE(ctx, p == p, SCHED_ERR_INVALID_ARG, "eval_fitness_racks: p is NaN");
+  REQUIRE(ctx, ((uintptr_t)d_pop & 1) == 0 && ((uintptr_t)d_cur & 1) == 0 && ((uintptr_t)d_speedup & 3) == 0 &&
+                   ((uintptr_t)d_speedup_rack & 3) == 0 && ((uintptr_t)d_fitness & 3) == 0,
+          SCHED_ERR_INVALID_ARG, "eval_fitness_racks: a buffer is not aligned to its element size");
+  REQUIRE(ctx, (long long)count * ctx->cfg.num_jobs < (1LL << 31), SCHED_ERR_TOO_LARGE,
+          "eval_fitness_racks: count * num_jobs must be below 2^31");
+  return launch_fitness_racks(ctx, d_pop, count, d_speedup, d_speedup_rack, d_cur, d_realloc_factor, d_active, p,
+                              d_fitness);
 }
 
 int sched_num_kernel_kinds(void) { return KK_COUNT; }
@@ -498,6 +555,15 @@ static int round_body(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d
   int rc;
   const bool penalise = d_cur && d_jobs->age_sec && d_jobs->num_restarts;
   if ((rc = launch_speedup_table(ctx, d_jobs, ctx->d_tab_goodput, ctx->d_tab_speedup, nullptr)) != SCHED_OK) return rc;
+  // Rack-level locality: a second table for allocations that span racks; the round then runs on
+  // dense matrices with the fitness read from them (the row summaries carry no rack count).
+  const bool racks = ctx->d_rack != nullptr;
+  if (racks) {
+    const float *ar = ctx->d_alpha_rack ? ctx->d_alpha_rack : d_jobs->alpha_node;
+    const float *br = ctx->d_beta_rack ? ctx->d_beta_rack : d_jobs->beta_node;
+    if ((rc = launch_speedup_table_rack(ctx, d_jobs, ar, br, nullptr, ctx->d_tab_speedup_rack, nullptr)) != SCHED_OK)
+      return rc;
+  }
   if (penalise && (rc = launch_realloc_factor(ctx, d_jobs, ctx->d_rf)) != SCHED_OK) return rc;
   const float *rf = penalise ? ctx->d_rf : nullptr;
   int16_t *pa = ctx->d_popA, *pb = ctx->d_popB;
@@ -505,7 +571,7 @@ static int round_body(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d
   // from the current allocation); the in-round fitness reads those instead of the matrices
   // whenever the batched kernels were used, with bit-identical results.
   ctx->round_cur = rf ? d_cur : nullptr;
-  ctx->round_summ = ctx->d_summ;
+  ctx->round_summ = racks ? nullptr : ctx->d_summ;
   ctx->round_summ_in = nullptr;
   uint32_t *summ_other = ctx->d_summ + (size_t)ctx->cfg.population * ctx->cfg.num_jobs;
   // the per-job penalty factors depend only on the current allocation: prepared once
@@ -514,7 +580,7 @@ static int round_body(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d
   if (rf) rc = launch_penalty_prep(ctx, d_cur, rf);
   ctx->pen_ready = (rc == SCHED_OK) && rf;
   // problems whose candidates fit one block get row pass, column pass and fitness in one kernel
-  ctx->ff_on = true;
+  ctx->ff_on = !racks;
   ctx->ff_table = ctx->d_tab_speedup;
   ctx->ff_pen = rf ? ctx->d_pen : nullptr;
   ctx->ff_active = d_jobs->active;
@@ -524,6 +590,9 @@ static int round_body(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d
   ctx->ff_out = fit_cur;
   auto fitness_of = [&](const int16_t *pop, float *out) {
     if (ctx->fit_done) return (int)SCHED_OK;
+    if (racks)
+      return launch_fitness_racks(ctx, pop, ctx->cfg.population, ctx->d_tab_speedup, ctx->d_tab_speedup_rack, d_cur, rf,
+                                  d_jobs->active, ctx->cfg.p, out);
     return launch_fitness(ctx, pop, ctx->cfg.population, ctx->d_tab_speedup, d_cur, rf, d_jobs->active,
                           ctx->cfg.p, out, ctx->summ_valid ? ctx->round_summ : nullptr);
   };
@@ -563,7 +632,7 @@ static int round_body(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d
     ctx->ff_out = fit_next;
     // children's summaries go to the other half; the parents' feed the unperturbed rows
     ctx->round_summ_in = ctx->summ_valid ? ctx->round_summ : nullptr;
-    std::swap(ctx->round_summ, summ_other);
+    if (!racks) std::swap(ctx->round_summ, summ_other);
     rc = launch_generation(ctx, d_jobs->k_cap, d_jobs->active, pa, fit_cur, pb, (uint32_t)g);
     if (rc != SCHED_OK) break;
     std::swap(pa, pb);

@@ -54,6 +54,12 @@ struct sched_ctx {
   int num_pairs;
   float *d_gmax;         // [J][KD][2] compact goodput maxima (class local / node)
   uint16_t *d_amax;      // [J][KD][2]
+  float *d_gmax_rack;    // [J][KD][2] the same with the rack pair in the node pair's place (allocated on first use)
+  uint16_t *d_amax_rack;
+  // rack-level locality (sched_set_racks): rack of every node, the third synchronisation pair
+  int16_t *d_rack;       // [num_nodes] or NULL when the cluster is not split into racks
+  const float *d_alpha_rack, *d_beta_rack;   // caller-owned device arrays [J]
+  float *d_tab_speedup_rack;                 // [J][KD][ND] rack-class table of a running round
   int32_t *d_rank;       // [P]
   int32_t *d_order;      // [P] inverse of rank
   uint8_t *d_dflag;      // [P][J] "row spans >= 2 nodes" after the row pass
@@ -249,6 +255,11 @@ __device__ __forceinline__ int nth_occupied(const int16_t *row, int num_nodes, u
 // kernels' launchers (defined in table.cu / fitness.cu / ga.cu / rowstore.cu)
 int launch_speedup_table(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodput, float *d_speedup,
                          uint16_t *d_argmax);
+int launch_speedup_table_rack(sched_ctx *ctx, const sched_jobs *jobs, const float *d_alpha_rack,
+                              const float *d_beta_rack, float *d_goodput, float *d_speedup, uint16_t *d_argmax);
+int launch_fitness_racks(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const float *d_speedup,
+                         const float *d_speedup_rack, const int16_t *d_cur, const float *d_rf,
+                         const uint8_t *d_active, float p, float *d_fitness);
 int launch_speedup_table_msample(sched_ctx *ctx, const sched_jobs *jobs, const int32_t *d_m_samples, int G,
                                  const int32_t *d_m_max_gpu, const uint8_t *d_adaptive, float *d_goodput,
                                  float *d_speedup, uint16_t *d_argmax);

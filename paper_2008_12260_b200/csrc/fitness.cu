@@ -224,6 +224,54 @@ __global__ void __launch_bounds__(256) fitness_summary_kernel(FitnessArgs a) {
   block_finish(a, cand, chunk, j0, j1, s_term);
 }
 
+// Eq. 14 with rack-level locality: a row whose occupied nodes lie in two or more racks takes its
+// speedup from the rack-class table.  A plain warp-per-row pass (this variant is not the
+// streaming kernel above); same chunks and the same fixed-order sums.
+__global__ void __launch_bounds__(256)
+fitness_racks_kernel(FitnessArgs a, const float *__restrict__ table_rack, const int16_t *__restrict__ rack) {
+  __shared__ float s_term[FITNESS_MAX_ROWS_PER_BLOCK];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const int cand = blockIdx.y, chunk = blockIdx.x;
+  const int j0 = chunk * a.rows_per_block;
+  const int j1 = min(a.J, j0 + a.rows_per_block);
+  TermParams tp;
+  tp.table = a.table; tp.pen = a.pen; tp.active = a.active;
+  tp.k_max = a.k_max; tp.n_max = a.n_max; tp.mode = a.mode; tp.p = a.p; tp.floor_ = a.floor_;
+  for (int j = j0 + warp; j < j1; j += nwarps) {
+    if (a.active && !a.active[j]) continue;
+    const int16_t *row = a.pop + ((size_t)cand * a.J + j) * a.num_nodes;
+    const int16_t *crow = a.cur ? a.cur + (size_t)j * a.num_nodes : nullptr;
+    long long K = 0;
+    int N = 0, rmin = 0x7fffffff, rmax = -1, diff = 0;
+    for (int n = lane; n < a.num_nodes; n += 32) {
+      const int v = row[n];
+      K += v;
+      if (v > 0) {
+        ++N;
+        const int r = rack[n];
+        rmin = min(rmin, r);
+        rmax = max(rmax, r);
+      }
+      if (crow) diff |= (v != (int)crow[n]) ? 1 : 0;
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+      K += __shfl_xor_sync(0xffffffffu, K, off);
+      N += __shfl_xor_sync(0xffffffffu, N, off);
+      rmin = min(rmin, __shfl_xor_sync(0xffffffffu, rmin, off));
+      rmax = max(rmax, __shfl_xor_sync(0xffffffffu, rmax, off));
+      diff |= __shfl_xor_sync(0xffffffffu, diff, off);
+    }
+    if (lane == 0) {
+      const int Kc = (int)max(0ll, min(K, (long long)a.k_max));
+      const bool several = N >= 1 && rmin != rmax;
+      const float x = __ldg((several ? table_rack : a.table) + fitness_table_index(tp, j, Kc, N));
+      s_term[j - j0] = fitness_term_of(tp, j, x, diff != 0);
+    }
+  }
+  block_finish(a, cand, chunk, j0, j1, s_term);
+}
+
 // Effective penalty per job: the re-allocation factor when the job currently holds GPUs,
 // else 1 (pending jobs are never penalised).  One warp per job.
 __global__ void penalty_prep_kernel(const int16_t *__restrict__ cur, const float *__restrict__ rf,
@@ -339,6 +387,53 @@ int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const fl
       case 4: fitness_kernel<4><<<grid, 256, 0, ctx->stream>>>(b); break;
       default: fitness_kernel<2><<<grid, 256, 0, ctx->stream>>>(b); break;
     }
+    }
+    SCHED_LAUNCH_CHECK(ctx);
+  }
+  return SCHED_OK;
+}
+
+int launch_fitness_racks(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const float *d_speedup,
+                         const float *d_speedup_rack, const int16_t *d_cur, const float *d_rf,
+                         const uint8_t *d_active, float p, float *d_fitness) {
+  const sched_config &c = ctx->cfg;
+  const int J = c.num_jobs;
+  if (count == 0) return SCHED_OK;
+  const bool penalise = d_cur && d_rf;
+  if (penalise && J > 0 && !ctx->pen_ready) {
+    int rc = launch_penalty_prep(ctx, d_cur, d_rf);
+    if (rc != SCHED_OK) return rc;
+  }
+  int W, lpr_log2, rows_per_block, chunks;
+  fitness_geometry((size_t)c.num_nodes * 2, 0, J, count, ctx->num_sms, W, lpr_log2, rows_per_block, chunks);
+  int rc = ensure_fitness_scratch(ctx, count, chunks);
+  if (rc != SCHED_OK) return rc;
+  FitnessArgs a;
+  a.pop = d_pop;
+  a.cur = penalise ? d_cur : nullptr;
+  a.table = d_speedup;
+  a.pen = penalise ? ctx->d_pen : nullptr;
+  a.active = d_active;
+  a.summ = nullptr;
+  a.J = J; a.num_nodes = c.num_nodes; a.k_max = c.k_max; a.n_max = c.n_max;
+  a.lpr_log2 = 0;
+  a.rows_per_block = rows_per_block; a.chunks = chunks;
+  a.p = p; a.floor_ = c.speedup_floor;
+  a.mode = fitness_mode(p);
+  a.partial = ctx->d_partial;
+  a.ticket = ctx->d_ticket;
+  a.fitness = d_fitness;
+  for (int32_t first = 0; first < count; first += 65535) {
+    const int32_t n = (count - first < 65535) ? (count - first) : 65535;
+    FitnessArgs b = a;
+    b.pop = d_pop + (size_t)first * J * c.num_nodes;
+    b.partial = ctx->d_partial + (size_t)first * chunks * 2;
+    b.ticket = ctx->d_ticket + first;
+    b.fitness = d_fitness + first;
+    dim3 grid((unsigned)chunks, (unsigned)n);
+    {
+      TimedLaunch tl_(ctx, KK_FITNESS);
+      fitness_racks_kernel<<<grid, 256, 0, ctx->stream>>>(b, d_speedup_rack, ctx->d_rack);
     }
     SCHED_LAUNCH_CHECK(ctx);
   }

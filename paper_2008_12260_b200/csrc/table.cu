@@ -286,8 +286,12 @@ __device__ __forceinline__ bool kn_valid(int K, int N, int k_max, int n_max,
 // Block = one job's slab of (k_max + 1) x (n_max + 1) entries, walked in memory order (thread
 // t takes entries t, t + 256, ...; its (K, N) advance without divisions), so every store is
 // coalesced whatever the slab's width.
+// gden: the class results that hold the fair-share goodput (the two-class sweep's; the table of
+// the rack class is normalised by the same goodput); min_n: entries with fewer nodes stay empty
+// (1 for the two-class table, 2 for the rack class, which always takes the second class of gmax).
 __global__ void __launch_bounds__(256)
 speedup_expand_kernel(const float *__restrict__ gmax, const uint16_t *__restrict__ amax,
+                      const float *__restrict__ gden, int min_n,
                       const int32_t *__restrict__ kfit, const int32_t *__restrict__ fair_k,
                       const int32_t *__restrict__ fair_n, int j_first, int k_max, int n_max,
                       float *__restrict__ goodput, float *__restrict__ speedup,
@@ -296,7 +300,7 @@ speedup_expand_kernel(const float *__restrict__ gmax, const uint16_t *__restrict
   const int j = j_first + blockIdx.x;
   const int kf = fair_k[j], nf = fair_n[j];
   float denom = 0.f;
-  if (kn_valid(kf, nf, k_max, n_max, kfit)) denom = gmax[((size_t)j * KD + kf) * 2 + (nf >= 2 ? 1 : 0)];
+  if (kn_valid(kf, nf, k_max, n_max, kfit)) denom = gden[((size_t)j * KD + kf) * 2 + (nf >= 2 ? 1 : 0)];
   const int entries = KD * ND;
   const int step_k = (int)blockDim.x / ND, step_n = (int)blockDim.x % ND;
   int K = (int)threadIdx.x / ND, N = (int)threadIdx.x % ND;
@@ -309,7 +313,7 @@ speedup_expand_kernel(const float *__restrict__ gmax, const uint16_t *__restrict
   for (int e = threadIdx.x; e < entries; e += blockDim.x) {
     float g = 0.f, sp = 0.f;
     uint16_t a = 0xFFFFu;
-    if (N >= 1 && K >= N && K <= __ldg(kfit + N)) {
+    if (N >= min_n && K >= N && K <= __ldg(kfit + N)) {
       const int src = K * 2 + (N >= 2 ? 1 : 0);
       g = gj[src];
       a = aj[src];
@@ -373,16 +377,17 @@ int launch_autoscale(sched_ctx *ctx, const float *d_goodput, const int32_t *d_cu
 }
 
 static int launch_expand(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodput, float *d_speedup,
-                         uint16_t *d_argmax) {
+                         uint16_t *d_argmax, bool rack_class = false) {
   const sched_config &c = ctx->cfg;
   const int J = c.num_jobs;
   for (int j0 = 0; j0 < J; j0 += 65535) {      // at most 65535 jobs per launch
     const unsigned grid = (unsigned)std::min(65535, J - j0);
     {
       TimedLaunch tl_(ctx, KK_EXPAND);
-      speedup_expand_kernel<<<grid, 256, 0, ctx->stream>>>(ctx->d_gmax, ctx->d_amax, ctx->d_kfit,
-                                                                   jobs->fair_k, jobs->fair_n, j0, c.k_max, c.n_max,
-                                                                   d_goodput, d_speedup, d_argmax);
+      speedup_expand_kernel<<<grid, 256, 0, ctx->stream>>>(rack_class ? ctx->d_gmax_rack : ctx->d_gmax,
+                                                           rack_class ? ctx->d_amax_rack : ctx->d_amax, ctx->d_gmax,
+                                                           rack_class ? 2 : 1, ctx->d_kfit, jobs->fair_k, jobs->fair_n,
+                                                           j0, c.k_max, c.n_max, d_goodput, d_speedup, d_argmax);
     }
     SCHED_LAUNCH_CHECK(ctx);
   }
@@ -412,6 +417,45 @@ int launch_speedup_table(sched_ctx *ctx, const sched_jobs *jobs, float *d_goodpu
     SCHED_LAUNCH_CHECK(ctx);
   }
   return launch_expand(ctx, jobs, d_goodput, d_speedup, d_argmax);
+}
+
+// Tables of the rack class (allocations whose nodes lie in two or more racks): the sweep of the
+// node class with the rack pair in the node pair's place; needs the two-class sweep's results in
+// d_gmax for the fair-share goodput, so that sweep runs first.
+int launch_speedup_table_rack(sched_ctx *ctx, const sched_jobs *jobs, const float *d_alpha_rack,
+                              const float *d_beta_rack, float *d_goodput, float *d_speedup, uint16_t *d_argmax) {
+  const sched_config &c = ctx->cfg;
+  const int J = c.num_jobs;
+  if (J == 0) return SCHED_OK;
+  const size_t n = (size_t)J * ctx->KD * 2;
+  if (!ctx->d_gmax_rack) {
+    SCHED_CUDA_CHECK(ctx, cudaMalloc((void **)&ctx->d_gmax_rack, sizeof(float) * n));
+    SCHED_CUDA_CHECK(ctx, cudaMalloc((void **)&ctx->d_amax_rack, sizeof(uint16_t) * n));
+    ctx->scratch_epoch++;
+  }
+  SCHED_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->d_gmax_rack, 0, sizeof(float) * n, ctx->stream));
+  SCHED_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->d_amax_rack, 0xFF, sizeof(uint16_t) * n, ctx->stream));
+  const int mq = (c.grid_m + 31) / 32;
+  if (ctx->num_pairs > 0) {
+    dim3 grid((unsigned)J, (unsigned)((ctx->num_pairs + 7) / 8));
+    for (int pass = 0; pass < 2; ++pass) {
+      JobPtrs jp = {jobs->alpha_grad, jobs->beta_grad, jobs->alpha_local, jobs->beta_local,
+                    pass ? d_alpha_rack : jobs->alpha_node, pass ? d_beta_rack : jobs->beta_node, jobs->gamma,
+                    jobs->phi, jobs->m0, jobs->m_max_total};
+      float *gm = pass ? ctx->d_gmax_rack : ctx->d_gmax;
+      uint16_t *am = pass ? ctx->d_amax_rack : ctx->d_amax;
+#define SWEEP(MQ)                                                                              \
+  TimedLaunch tl_(ctx, KK_SWEEP);                                                              \
+  goodput_sweep_kernel<MQ><<<grid, 256, 0, ctx->stream>>>(                                     \
+      jp, jobs->m_grid, ctx->d_pairs, ctx->num_pairs, c.k_max, c.grid_m, c.grid_s, 1.f, 0.f, gm, am)
+      if (mq <= 1) { SWEEP(1); }
+      else if (mq == 2) { SWEEP(2); }
+      else { SWEEP(4); }
+#undef SWEEP
+      SCHED_LAUNCH_CHECK(ctx);
+    }
+  }
+  return launch_expand(ctx, jobs, d_goodput, d_speedup, d_argmax, true);
 }
 
 int launch_speedup_table_msample(sched_ctx *ctx, const sched_jobs *jobs, const int32_t *d_m_samples, int G,

@@ -76,6 +76,8 @@ class Jobs:
     active: np.ndarray        # uint8
     fair_k: np.ndarray = field(default=None)  # int32, filled by the caller
     fair_n: np.ndarray = field(default=None)
+    alpha_rack: np.ndarray = field(default=None)  # fp32, third synchronisation pair (rack-level locality), optional
+    beta_rack: np.ndarray = field(default=None)
 
     @property
     def num_jobs(self) -> int:
@@ -366,3 +368,18 @@ def trace_arrivals(num_jobs: int = 160, seed: int = 4, horizon_sec: float = 8 * 
     life = np.exp(g.uniform(np.log(lo[cats]), np.log(hi[cats])))
     names = ["S", "M", "L", "XL"]
     return [TraceJob(float(arrive[i]), float(life[i]), names[int(cats[i])]) for i in range(num_jobs)]
+
+
+def rack_of_nodes(num_nodes: int, nodes_per_rack: int) -> np.ndarray:
+    """Rack id of every node: consecutive nodes share a rack (int16 [num_nodes])."""
+    return (np.arange(num_nodes) // max(int(nodes_per_rack), 1)).astype(np.int16)
+
+
+def draw_rack_pair(jobs: Jobs, seed: int, lo: float = 1.5, hi: float = 3.0):
+    """Third synchronisation pair for allocations that span racks: the node pair times an
+    independent factor U[lo, hi] each (crossing racks is slower than crossing nodes, as crossing
+    nodes is slower than staying on one).  Returns (alpha_rack, beta_rack), fp32 [J]."""
+    g = np.random.Generator(np.random.PCG64(seed))
+    fa = g.uniform(lo, hi, jobs.num_jobs)
+    fb = g.uniform(lo, hi, jobs.num_jobs)
+    return (jobs.alpha_node * fa).astype(np.float32), (jobs.beta_node * fb).astype(np.float32)
