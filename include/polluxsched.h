@@ -137,6 +137,17 @@ int sched_num_kernel_kinds(void);
 const char *sched_kernel_kind_name(int kind);
 int sched_read_kernel_timing(sched_ctx *ctx, float *h_ms_total, int64_t *h_launches);
 
+/* Machine peaks measured in place (the paper has no counterpart; for benchmarks, so that a
+ * roofline fraction is taken against the clocks of the moment): the rate of independent fp32
+ * FMA chains in lane-operations per second (an FMA counts once; bounds the goodput sweep), the
+ * rate of special-function operations (lg2 / ex2 chains; the sweep's co-limit), and the
+ * bandwidth of a read-only stream of 16-byte loads over d_buffer (DEVICE, 16-byte aligned,
+ * `bytes` long, only read; NULL skips it and reports 0; bounds the dense fitness kernel).
+ * Each figure is the mean of `reps` launches after one warm-up, timed with CUDA events on the
+ * context's stream; the call waits.  Outputs are HOST doubles. */
+int sched_measure_peaks(sched_ctx *ctx, const void *d_buffer, uint64_t bytes, int32_t reps,
+                        double *h_fp32_lane_ops_per_s, double *h_mufu_ops_per_s, double *h_read_bytes_per_s);
+
 /* Speedup tables (Eq. 13 and 15).  For every job and every (K, N) with 1 <= N <= n_max,
  * N <= K <= k_max and K no larger than the N largest nodes together:
  *   goodput[j][K][N] = max over the grid {m_grid[j][i]} x {s} of GOODPUT(a, m, s) (Eq. 4)

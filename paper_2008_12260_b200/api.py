@@ -11,7 +11,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libpolluxsched.so")
+# POLLUXSCHED_LIB selects another build of the library (e.g. libpolluxsched_checked.so)
+LIB_PATH = os.environ.get("POLLUXSCHED_LIB") or os.path.join(_HERE, "libpolluxsched.so")
 
 SCHED_OK = 0
 ERRORS = {-1: "INVALID_ARG", -2: "BAD_CONFIG", -3: "CUDA", -4: "TIMEOUT", -5: "NOT_FINITE", -6: "TOO_LARGE"}
@@ -22,7 +23,7 @@ EXPORTS = (
     "init_population", "ga_generation", "schedule_round", "schedule_round_host",
     "sched_get_population", "sched_get_round_tables", "sched_round_speedup_table", "eval_fitness_host",
     "sched_set_kernel_timing", "sched_num_kernel_kinds", "sched_kernel_kind_name",
-    "sched_read_kernel_timing", "sched_set_graphs", "sched_set_store_budget", "sched_store_moves", "eval_fitness_noalloc", "eval_fitness_noalloc_last_error",
+    "sched_read_kernel_timing", "sched_measure_peaks", "sched_set_graphs", "sched_set_store_budget", "sched_store_moves", "eval_fitness_noalloc", "eval_fitness_noalloc_last_error",
 )
 
 
@@ -87,6 +88,8 @@ def load_library(path: str = LIB_PATH):
     lib.eval_fitness_host.argtypes = [vp, vp, i32, vp, vp, vp, vp, f32, vp]
     lib.sched_set_kernel_timing.argtypes = [vp, i32]
     lib.sched_set_graphs.argtypes = [vp, i32]
+    lib.sched_measure_peaks.argtypes = [vp, vp, C.c_uint64, i32, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                        C.POINTER(C.c_double)]
     lib.sched_set_store_budget.argtypes = [vp, C.c_uint64]
     lib.sched_store_moves.argtypes = [vp]
     lib.sched_store_moves.restype = C.c_int64
@@ -215,6 +218,13 @@ class Scheduler:
 
     def set_graphs(self, enable: bool):
         self._check(_lib.sched_set_graphs(self._ctx, 1 if enable else 0))
+
+    def measure_peaks(self, buffer=None, reps: int = 5):
+        """(fp32 lane-ops/s, special-function ops/s, read-only stream bytes/s over `buffer`)"""
+        a, b, c = C.c_double(0), C.c_double(0), C.c_double(0)
+        nbytes = 0 if buffer is None else buffer.numel() * buffer.element_size()
+        self._check(_lib.sched_measure_peaks(self._ctx, _ptr(buffer), nbytes, reps, C.byref(a), C.byref(b), C.byref(c)))
+        return a.value, b.value, c.value
 
     def set_store_budget(self, nbytes: int):
         self._check(_lib.sched_set_store_budget(self._ctx, int(nbytes)))

@@ -1,6 +1,11 @@
 """Builds libpolluxsched.so in-tree with nvcc for sm_100a (cross-compiles without a GPU).
 
-    python -m paper_2008_12260_b200.build [--force] [--verbose]
+    python -m paper_2008_12260_b200.build [--force] [--verbose] [--checked]
+
+--checked builds libpolluxsched_checked.so instead: the same library compiled with
+-DSCHED_CHECKED, in which kernels range-test the indices they compute from data and report a
+violation through the context's status word (see csrc/common.cuh).  Select it at run time with
+the environment variable POLLUXSCHED_LIB.
 """
 from __future__ import annotations
 
@@ -14,6 +19,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(HERE, "libpolluxsched.so")
+LIB_CHECKED = os.path.join(HERE, "libpolluxsched_checked.so")
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
@@ -25,17 +31,18 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+def _stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(INCLUDE, "*.h"))
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not _stale():
-        return LIB
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    lib = LIB_CHECKED if checked else LIB
+    if not force and not _stale(lib):
+        return lib
     from concurrent.futures import ThreadPoolExecutor
 
     nvcc = os.environ.get("NVCC", "nvcc")
@@ -43,9 +50,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(objdir, exist_ok=True)
     common = [f for f in NVCC_FLAGS if f not in ("--shared", "-cudart", "static")]
     common += (["-Xptxas", "-v"] if verbose else []) + ["-I", INCLUDE, "-I", CSRC]
+    common += ["-DSCHED_CHECKED"] if checked else []
 
     def compile_one(src):
-        obj = os.path.join(objdir, os.path.basename(src) + ".%d.o" % os.getpid())
+        obj = os.path.join(objdir, os.path.basename(src) + ".%d%s.o" % (os.getpid(), "c" if checked else ""))
         res = subprocess.run([nvcc] + common + ["-c", "-o", obj, src], capture_output=True, text=True)
         return src, obj, res
 
@@ -58,14 +66,14 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if res.returncode != 0:
             raise subprocess.CalledProcessError(res.returncode, "nvcc -c " + src)
         objs.append(obj)
-    tmp = LIB + ".tmp%d" % os.getpid()
+    tmp = lib + ".tmp%d" % os.getpid()
     subprocess.check_call([nvcc, "--shared", "-cudart", "static", "-gencode", "arch=compute_100a,code=sm_100a",
                            "-o", tmp] + objs)
-    os.replace(tmp, LIB)
+    os.replace(tmp, lib)
     for obj in objs:
         os.remove(obj)
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, checked="--checked" in sys.argv))

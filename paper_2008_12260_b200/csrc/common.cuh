@@ -179,6 +179,28 @@ extern char g_init_error[256];
   } while (0)
 
 // ---------------------------------------------------------------------------------------
+// Checked build (-DSCHED_CHECKED, `python -m paper_2008_12260_b200.build --checked`): indices
+// that kernels compute from data (row slots, node numbers, list positions) are range-tested
+// before they are used; a violation records one of the codes below in the context's status word
+// (first one wins, read by sched_sync_status) and the access is skipped.  Nothing traps.  In the
+// normal build the test compiles away.
+// ---------------------------------------------------------------------------------------
+#define SCHED_CHK_SLOT (-101)     /* a row slot beyond the pool                           */
+#define SCHED_CHK_NODE (-102)     /* a node (or job) number beyond the cluster (the jobs)  */
+#define SCHED_CHK_LIST (-103)     /* a position beyond a block's work list                 */
+#define SCHED_CHK_ENTRY (-104)    /* a position beyond a row's list of occupied nodes      */
+
+__device__ __forceinline__ bool sched_index_ok(int *status, bool ok, int code) {
+#ifdef SCHED_CHECKED
+  if (!ok) atomicCAS(status, 0, code);
+  return ok;
+#else
+  (void)status; (void)code; (void)ok;
+  return true;
+#endif
+}
+
+// ---------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies; the key is
 // advanced by the Weyl constants before every round except the first.
 // ---------------------------------------------------------------------------------------
@@ -189,14 +211,10 @@ struct u32x4 {
 __host__ __device__ __forceinline__ u32x4 philox4x32_10(u32x4 c, uint32_t k0, uint32_t k1) {
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
-#ifdef __CUDA_ARCH__
-    const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
-    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
-#else
+    // one 32 x 32 -> 64 bit multiply per product (a single wide multiply-add on the device)
     const uint64_t p0 = (uint64_t)0xD2511F53u * c.x, p1 = (uint64_t)0xCD9E8D57u * c.z;
     const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
     const uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
-#endif
     u32x4 n;
     n.x = hi1 ^ c.y ^ k0;
     n.y = lo1;

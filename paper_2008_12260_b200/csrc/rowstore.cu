@@ -33,7 +33,8 @@ struct StoreView {
   int16_t *pool;
   uint32_t *rec;
   unsigned long long half_cap;
-  uint32_t zero_slot;
+  uint32_t zero_slot;       // also the largest valid slot
+  int *status;              // the context's status word (checked build)
 };
 
 // ---- a row as 16-byte pieces of 8 entries (entries of stored rows are in [0, 2047]) -----------
@@ -357,6 +358,7 @@ __global__ void __launch_bounds__(256) rowstore_compact_kernel(CompactArgs a) {
     const uint32_t slot = a.ptr[r];
     if (slot == a.st.zero_slot) continue;
     const size_t dst = (size_t)(base + r);
+    if (!sched_index_ok(a.st.status, slot < a.st.zero_slot && dst < a.st.zero_slot, SCHED_CHK_SLOT)) continue;
     const uint32_t w = (lane < REC_WORDS) ? a.st.rec[(size_t)slot * REC_WORDS + lane] : 0u;
     if (__shfl_sync(0xffffffffu, w, 0) == REC_OVERFLOW) {   // the record does not hold the row: its contents move too
       const uint4 *s4 = (const uint4 *)(a.st.pool + (size_t)slot * a.NN);
@@ -380,7 +382,8 @@ rowstore_gather_kernel(StoreView st, const uint32_t *__restrict__ ptr, int first
   const int row_vecs = NN >> 3;
   const bool aligned = ((uintptr_t)out & 15) == 0;
   for (long long r = (long long)blockIdx.x * 8 + warp; r < rows; r += (long long)gridDim.x * 8) {
-    const uint32_t slot = ptr[first + r];
+    uint32_t slot = ptr[first + r];
+    if (!sched_index_ok(st.status, slot <= st.zero_slot, SCHED_CHK_SLOT)) slot = st.zero_slot;
     // every lane reads the row's record (one address: a broadcast)
     const uint4 lo = *((const uint4 *)(st.rec + (size_t)slot * REC_WORDS));
     const uint4 hi = *((const uint4 *)(st.rec + (size_t)slot * REC_WORDS) + 1);
@@ -514,11 +517,12 @@ __device__ __forceinline__ int diff_delta(const int16_t *cur, int NN, int j, int
 }
 
 // A[j][node] = v_new on the list form of row j (nd is brought up to date later, see RowList)
-__device__ __forceinline__ void list_put(RowList &r, int node, int v_new) {
+__device__ __forceinline__ void list_put(int *status, RowList &r, int node, int v_new) {
   int pos;
   bool found;
   const int v_old = list_find(r, node, pos, found);
   if (v_new == v_old) return;
+  if (!sched_index_ok(status, r.n >= 0 && r.n <= LIST_MAX && pos >= 0 && pos <= r.n && r.pn < 2, SCHED_CHK_ENTRY)) return;
   if (r.pn == 0) { r.pnode0 = node; r.pold0 = v_old; r.pnew0 = v_new; }
   else { r.pnode1 = node; r.pold1 = v_old; r.pnew1 = v_new; }
   r.pn += 1;
@@ -540,7 +544,8 @@ __device__ __forceinline__ void list_put(RowList &r, int node, int v_new) {
 }
 
 // the perturbation of a row (grow / shrink / relocate, chosen by the row's draw `mw`)
-__device__ __forceinline__ void list_perturb(int NN, RowList &r, const u32x4 &mw, const int16_t *s_cap) {
+__device__ __forceinline__ void list_perturb(int *status, int NN, RowList &r, const u32x4 &mw, const int16_t *s_cap) {
+  if (!sched_index_ok(status, r.n >= 0 && r.n <= REC_ENTRIES, SCHED_CHK_ENTRY)) return;
   const uint32_t op = bounded(mw.y, 3u);
   int pos;
   bool found;
@@ -567,7 +572,7 @@ __device__ __forceinline__ void list_perturb(int NN, RowList &r, const u32x4 &mw
 #pragma unroll 1
   for (int q = 0; q < 2; ++q) {
     const int node = q ? node1 : node0, val = q ? val1 : val0;
-    if (node >= 0) list_put(r, node, val);
+    if (node >= 0) list_put(status, r, node, val);
   }
 }
 
@@ -813,6 +818,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       if (mw.x < a.thr) {
         mutbits |= 1u << r;
         const int i = atomicAdd(&s_nmut, 1);
+        if (!sched_index_ok(a.status, i < J, SCHED_CHK_LIST)) continue;
         s_mut[i] = (uint16_t)(j | (sec ? 0x8000 : 0));          // j < 8192
         if (i < MUT_STASH)
           s_stash[i] = make_uint4(mw.y, mw.z, mw.w, (uint32_t)max(0, min(a.k_cap ? a.k_cap[j] : a.k_max, a.k_max)));
@@ -923,6 +929,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
 
   // occupant (job j holds g GPUs on node n) into the node's totals and list
   auto add_occupant = [&](int j, int n, int g, bool dist) {
+    if (!sched_index_ok(a.status, n >= 0 && n < NN && j >= 0 && j < J, SCHED_CHK_NODE)) return;
     uint32_t *w = (uint32_t *)&s_node[n];   // two 32-bit adds: the low word's answer is not needed
     atomicAdd(&w[0], (uint32_t)g);
     const int k = (int)(atomicAdd(&w[1], (dist ? 1u : 0u) | (1u << 16)) >> 16);
@@ -974,8 +981,12 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
     }
     uint32_t rec[RB][REC_WORDS];
 #pragma unroll
-    for (int r = 0; r < RB; ++r) load_record(rec[r], a.st.rec + (size_t)slot[r] * REC_WORDS);
+    for (int r = 0; r < RB; ++r) {
+      if (!sched_index_ok(a.status, slot[r] <= a.st.zero_slot, SCHED_CHK_SLOT)) slot[r] = a.st.zero_slot;
+      load_record(rec[r], a.st.rec + (size_t)slot[r] * REC_WORDS);
+    }
     if (rb == 0 && pre_loaded) {
+      if (!sched_index_ok(a.status, pre_slot <= a.st.zero_slot, SCHED_CHK_SLOT)) pre_slot = a.st.zero_slot;
       pre_lo = __ldcg((const uint4 *)(a.st.rec + (size_t)pre_slot * REC_WORDS));
       pre_hi = __ldcg((const uint4 *)(a.st.rec + (size_t)pre_slot * REC_WORDS) + 1);
     }
@@ -990,7 +1001,8 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       const bool dist = ((w >> 11) & 0x7FFu) >= 2u;
       if (dist) s_mark[j] = MARK_DIST;
       if (rec[r][0] == REC_OVERFLOW) {
-        s_ovf[atomicAdd(&s_novf, 1)] = (uint16_t)j;
+        const int at = atomicAdd(&s_novf, 1);
+        if (sched_index_ok(a.status, at < J, SCHED_CHK_LIST)) s_ovf[at] = (uint16_t)j;
         continue;
       }
 #pragma unroll
@@ -1012,6 +1024,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
     uint4 lo = pre_lo, hi = pre_hi;
     if (!pre_loaded) {
       src = (INIT && !fail) ? a.init_src + (uint32_t)j : ((mj >> 15) ? __ldcg(pin_b + j) : __ldcg(pin_a + j));
+      if (!sched_index_ok(a.status, src <= a.st.zero_slot, SCHED_CHK_SLOT)) src = a.st.zero_slot;
       lo = __ldcg((const uint4 *)(a.st.rec + (size_t)src * REC_WORDS));
       hi = __ldcg((const uint4 *)(a.st.rec + (size_t)src * REC_WORDS) + 1);
     }
@@ -1043,7 +1056,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         mw = draw_call(a.key.k0, rkey, (uint32_t)j, c, a.gen, mut_slot);
         kc = max(0, min(a.k_cap ? a.k_cap[j] : a.k_max, a.k_max));
       }
-      list_perturb(NN, rl, mw, s_cap);
+      list_perturb(a.status, NN, rl, mw, s_cap);
       list_caps(a.cur, NN, a.n_max, rl, j, kc);
       slow = rl.n > REC_ENTRIES;
       if (!slow) {
@@ -1057,6 +1070,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         if (a.cur && rl.pn > 0) rl.nd += (int)(rl.pnew0 != cv0) - (int)(rl.pold0 != cv0);
         if (a.cur && rl.pn > 1) rl.nd += (int)(rl.pnew1 != cv1) - (int)(rl.pold1 != cv1);
         const uint32_t nslot = s_base_mut + (uint32_t)i;
+        if (!sched_index_ok(a.status, nslot < a.st.zero_slot && rl.n >= 0 && rl.n <= REC_ENTRIES, SCHED_CHK_SLOT)) continue;
         const uint32_t word = pack_summary(rl.K, rl.n, rl.nd);
         const float term = row_term_from(a.tp.pen != nullptr, a.tp.mode, a.tp.p, a.tp.floor_, x_sp, x_pen, rl.nd != 0);
         store_record(a.st.rec + (size_t)nslot * REC_WORDS, rl, term, word);
@@ -1067,7 +1081,10 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         for (int k = 0; k < rl.n; ++k) add_occupant(j, ent_node(rl.e[k]), ent_gpus(rl.e[k]), rl.n >= 2);
       }
     }
-    if (slow) s_slow[atomicAdd(&s_nslow, 1)] = (uint16_t)j;   // s_slot[j] is the source row, s_mark[j] >> 4 its number
+    if (slow) {   // s_slot[j] is the source row, s_mark[j] >> 4 its number
+      const int at = atomicAdd(&s_nslow, 1);
+      if (sched_index_ok(a.status, at < J, SCHED_CHK_LIST)) s_slow[at] = (uint16_t)j;
+    }
   }
   __syncthreads();
 
@@ -1207,7 +1224,8 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
           const int j = (int)(entry & 0x1FFFu);
           const int before = atomicOr(&s_mark[j], MARK_CHANGED);
           if ((before & MARK_CHANGED) == 0) {
-            s_mod[atomicAdd(&s_nmod, 1)] = (uint16_t)j;
+            const int at = atomicAdd(&s_nmod, 1);
+            if (sched_index_ok(a.status, at < J, SCHED_CHK_LIST)) s_mod[at] = (uint16_t)j;
             if ((before & MARK_OWN) == 0) atomicAdd(&s_nneed, 1);   // will want a slot of its own
           }
         }
@@ -1243,7 +1261,9 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
     }
     const bool fail2 = s_fail != 0;
     auto rewrite_row = [&](int j, int only_node, int only_value) {
+      if (!sched_index_ok(a.status, j >= 0 && j < J, SCHED_CHK_NODE)) return;
       const uint32_t src = s_slot[j];
+      if (!sched_index_ok(a.status, src <= a.st.zero_slot, SCHED_CHK_SLOT)) return;
       const bool own = (s_mark[j] & MARK_OWN) != 0;
       const uint4 lo = __ldcg((const uint4 *)(a.st.rec + (size_t)src * REC_WORDS));
       const uint4 hi = __ldcg((const uint4 *)(a.st.rec + (size_t)src * REC_WORDS) + 1);
@@ -1260,7 +1280,9 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
           if ((unsigned long long)dst + 1ull > limit) { atomicExch(a.status, SCHED_ERR_TOO_LARGE); return; }
         }
       }
+      if (!sched_index_ok(a.status, dst < a.st.zero_slot, SCHED_CHK_SLOT)) return;
       auto new_value = [&](int node, int v) -> int {
+        if (!sched_index_ok(a.status, node >= 0 && node < NN, SCHED_CHK_NODE)) return v;
         if (only_node >= 0) return node == only_node ? only_value : v;
         if (s_viol[node] != 1) return v;
         const int cnt = (int)(s_node[node] >> 48);
@@ -1464,6 +1486,7 @@ StoreView store_view(const sched_ctx *ctx) {
   v.pool = ctx->rs_pool; v.rec = ctx->rs_rec;
   v.half_cap = ctx->rs_half_cap;
   v.zero_slot = (uint32_t)(2 * ctx->rs_half_cap);
+  v.status = ctx->d_status;
   return v;
 }
 

@@ -53,6 +53,7 @@ def main(case: str, reps: int = 3, generations: int = 2):
         print("table_large", float(sp[0, 2, 1]))
     elif case == "round_large":
         cfg, cl, jobs, s, dj = _large(api, synth, torch)
+        s.set_store_budget(2 << 30)        # a small row pool: a profiler saves and restores device memory per pass
         cur = torch.from_numpy(cfg.cur()).cuda()
         best = torch.empty((cfg.num_jobs, cfg.num_nodes), dtype=torch.int16, device="cuda")
         bf = torch.zeros(1, dtype=torch.float32, device="cuda")

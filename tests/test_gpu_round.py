@@ -317,3 +317,27 @@ def test_host_entry_points_validate_their_arrays(gpu):
     assert e.value.code == -1
     run(jobs)                                          # the context is still usable
     s.close()
+
+
+@pytest.mark.parametrize("nodes,gpn,J", [(2, 2, 3), (2, 4, 2)])
+def test_search_against_the_brute_force_optimum(gpu, oracle, nodes, gpn, J, record_property):
+    """Clusters small enough to enumerate: the best fitness of the search can never exceed the
+    maximum of Eq. 14 over every feasible matrix; how close it gets is recorded, not required
+    (the method is a heuristic, Sec. 4.3)."""
+    import itertools
+    torch, api = gpu
+    cfg = synth.Config("quality", nodes, gpn, J, 40 + J, 16, 8, 32, 100, num_elite=2, mutate_prob=0.2)
+    cl, jobs = setup(cfg)
+    _, sp, _ = oracle.build_speedup_table(jobs, cl.node_capacity, cl.k_max, cl.n_max, cfg.grid_s, want_argmax=False)
+    mats = np.array(list(itertools.product(range(gpn + 1), repeat=J * nodes)), np.int16).reshape(-1, J, nodes)
+    ok = np.array([feasible(m, cl.node_capacity, jobs.k_cap, cl.n_max) for m in mats])
+    fit = oracle.eval_fitness(mats[ok], sp, cl.k_max, cl.n_max, cfg.p, cfg.speedup_floor)
+    optimum = float(fit.max())
+    for gens in (10, 100):
+        s, dj, best, bf, pop, f = _round(gpu, cfg, jobs, None, gens)
+        assert feasible(best, cl.node_capacity, jobs.k_cap, cl.n_max)
+        assert bf <= optimum * (1 + REL_TOL)
+        record_property("gap_after_%d_generations" % gens, 1.0 - bf / optimum)
+        if gens == 100:
+            assert bf >= 0.5 * optimum          # a search that found nothing would sit at the floor
+        s.close()
