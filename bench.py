@@ -46,8 +46,9 @@ HBM_FALLBACK_GBS = 6650.0
 # "rows": one dense large-workload generation (237.1 MB read + 257.1 MB written).
 # "fitness_stress": 16 dense stress candidates moved 544.8 + 3.5 MB; every candidate is streamed
 # once, so the figure is scaled by candidates / 16 to the chunk that is timed.
-# "generation_store": one row-store generation of the large workload.
-NCU_TRAFFIC_BYTES = {"rows": 494.2e6, "fitness_stress_per_candidate": 548.3e6 / 16, "generation_store": None}
+# "generation_store": one row-store generation of the large workload (3.4 - 3.6 MB read in
+# generations 6 to 8 of a 12-generation round).
+NCU_TRAFFIC_BYTES = {"rows": 494.2e6, "fitness_stress_per_candidate": 548.3e6 / 16, "generation_store": 3.5e6}
 
 
 def measured_peaks():
