@@ -1,16 +1,20 @@
 // Row store: the population of a running scheduling round kept as shared rows (Sec. 4.3).
 //
 // A generation copies almost every child row verbatim from one of two parents; only the
-// perturbed rows and the few rows the repair touches are new.  Here a row's contents live
-// once in a pool and a candidate is an array of row indices.  Next to each stored row sit
-// a 32-byte record: up to six occupied nodes, the row's summary (K, N, entries that differ
-// from the current allocation) and its term of the fitness sum (a stored row always serves
-// the same job, so the term is fixed for the round).  A generation reads 36 bytes per
-// unchanged row instead of the row, and writes 4.  New rows are appended to the pool (copy
-// on write); when a half of the pool runs low the live rows are copied to the other half.
+// perturbed rows and the few rows the repair touches are new.  Here every distinct row is
+// stored once and a candidate is an array of row indices ("slots").  A stored row is a
+// 32-byte record: up to six occupied nodes (node | GPUs << 12, ascending node order), the
+// row's term of the fitness sum (a stored row always serves the same job, so the term is
+// fixed for the round) and its summary (K, N, entries that differ from the current
+// allocation).  A row with at most six occupied nodes lives in its record alone; only a row
+// with more (first word 0xFFFFFFFF) also has its contents in the pool.  A generation reads
+// 36 bytes per unchanged row and writes 4.  New rows are appended (copy on write); when a
+// half of the slot space runs low the live rows are copied to the other half.
 //
 // One block evolves one candidate per generation: parent selection, row-wise crossover,
 // perturbation, per-row caps, interference and capacity repair, and the candidate's fitness.
+// Rows that change are edited as lists of occupied nodes, one thread per row.  The initial
+// population of a round is made by the same kernel from the current allocation's rows.
 // The operators, their random draws and the order of the fitness sums are the same as in
 // the dense kernels, so both paths produce identical populations and fitness bits.
 #include "common.cuh"
