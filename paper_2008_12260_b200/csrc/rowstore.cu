@@ -498,6 +498,27 @@ __device__ __noinline__ u32x4 draw_call(uint32_t k0, uint32_t k1, uint32_t idx, 
   return philox4x32_10(c, k0, k1);
 }
 
+// Two calls of the stream that differ only in their slot, rounds interleaved: the two chains of
+// dependent multiplies hide each other's latency (a row's crossover and perturbation draws).
+__device__ __noinline__ void draw_pair_call(uint32_t k0, uint32_t k1, uint32_t idx, uint32_t cand, uint32_t gen,
+                                            uint32_t slot_a, uint32_t slot_b, uint32_t &a_x, u32x4 &b) {
+  u32x4 ca = {idx, cand, gen, slot_a}, cb = {idx, cand, gen, slot_b};
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint64_t pa0 = (uint64_t)0xD2511F53u * ca.x, pa1 = (uint64_t)0xCD9E8D57u * ca.z;
+    const uint64_t pb0 = (uint64_t)0xD2511F53u * cb.x, pb1 = (uint64_t)0xCD9E8D57u * cb.z;
+    u32x4 na, nb;
+    na.x = (uint32_t)(pa1 >> 32) ^ ca.y ^ k0; na.y = (uint32_t)pa1; na.z = (uint32_t)(pa0 >> 32) ^ ca.w ^ k1; na.w = (uint32_t)pa0;
+    nb.x = (uint32_t)(pb1 >> 32) ^ cb.y ^ k0; nb.y = (uint32_t)pb1; nb.z = (uint32_t)(pb0 >> 32) ^ cb.w ^ k1; nb.w = (uint32_t)pb0;
+    ca = na;
+    cb = nb;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  a_x = ca.x;
+  b = cb;
+}
+
 // GPUs of the row on `node` (0 when the node is not occupied) and where its entry is or belongs
 __device__ __forceinline__ int list_find(const RowList &r, int node, int &pos, bool &found) {
   int v = 0;
@@ -816,9 +837,16 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
 #pragma unroll 1
     for (int j = tid; j < J; j += GEN_THREADS, ++r) {
       if (a.active && !a.active[j]) continue;
-      const bool sec = !INIT && (draw_call(a.key.k0, rkey, (uint32_t)j, c, a.gen, SLOT_XOVER).x >> 31);
+      bool sec = false;
+      u32x4 mw;
+      if (INIT) {
+        mw = draw_call(a.key.k0, rkey, (uint32_t)j, c, a.gen, mut_slot);
+      } else {
+        uint32_t xw;
+        draw_pair_call(a.key.k0, rkey, (uint32_t)j, c, a.gen, SLOT_XOVER, mut_slot, xw, mw);
+        sec = (xw >> 31) != 0u;
+      }
       if (sec) secbits |= 1u << r;
-      const u32x4 mw = draw_call(a.key.k0, rkey, (uint32_t)j, c, a.gen, mut_slot);
       if (mw.x < a.thr) {
         mutbits |= 1u << r;
         const int i = atomicAdd(&s_nmut, 1);
@@ -890,26 +918,30 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       prev = best;
     }
     if (tid == 0) s_parent = (int)(0xFFFFFFFFu - (uint32_t)(prev & 0xFFFFFFFFull));
-  } else if (warp < 4) {
-    // the ranks of the four drawn candidates, a warp each: every lane fetches its share of the keys
-    // (all loads in flight together) and counts those ordered before the warp's candidate
-    const int i = warp == 0 ? idx[0] : warp == 1 ? idx[1] : warp == 2 ? idx[2] : idx[3];
-    const uint32_t ki = order_key(__ldcg(a.fitness_bits + i));
-    int rk = 0;
+  } else {
+    // The ranks of the four drawn candidates, a warp each.  The keys are first staged in shared
+    // memory (the rows' slot and term arrays, unused until the rows are read) when they fit: every
+    // block of the grid asks for the same few lines at the same moment, so each key is fetched once
+    // per block rather than once per warp.
+    uint32_t *s_keys = s_slot;
+    const bool staged = (size_t)P * 4 <= (size_t)J * 8;
+    if (staged) {
 #pragma unroll 1
-    for (int o0 = lane; o0 < P; o0 += 32 * 8) {
-      uint32_t kk[8];
-#pragma unroll
-      for (int q = 0; q < 8; ++q) kk[q] = (o0 + 32 * q < P) ? __ldcg(a.fitness_bits + o0 + 32 * q) : 0u;
-#pragma unroll
-      for (int q = 0; q < 8; ++q) {
-        const int o = o0 + 32 * q;
-        const uint32_t ko = order_key(kk[q]);
-        rk += (o < P && (ko > ki || (ko == ki && o < i))) ? 1 : 0;
-      }
+      for (int i = tid; i < P; i += GEN_THREADS) s_keys[i] = order_key(__ldcg(a.fitness_bits + i));
+      __syncthreads();
     }
-    rk = warp_sum(rk);
-    if (lane == 0) s_rank4[warp] = rk;
+    if (warp < 4) {
+      const int i = warp == 0 ? idx[0] : warp == 1 ? idx[1] : warp == 2 ? idx[2] : idx[3];
+      const uint32_t ki = staged ? s_keys[i] : order_key(__ldcg(a.fitness_bits + i));
+      int rk = 0;
+#pragma unroll 4
+      for (int o = lane; o < P; o += 32) {
+        const uint32_t ko = staged ? s_keys[o] : order_key(__ldcg(a.fitness_bits + o));
+        rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
+      }
+      rk = warp_sum(rk);
+      if (lane == 0) s_rank4[warp] = rk;
+    }
   }
   if (tid == GEN_THREADS - 1) {
     const unsigned long long limit = (unsigned long long)(half_reg + 1u) * a.st.half_cap;
