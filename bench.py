@@ -40,6 +40,17 @@ FP32_LANES_PER_SM = 128          # CUDA cores per SM (compute capability 10.0)
 OPS_PER_POINT = 10               # fp32 lane-ops counted as useful per (job, K, class, m, s) point
 HBM_FALLBACK_GBS = 6650.0
 
+# the workload both arms (the CUDA path and the oracle as the reference) are quoted on
+CONFIG = {
+    "workload": "large: 256 nodes x 8 GPUs, 1024 jobs, grid 128x32, population 512, 200 generations, p=-1, "
+                "random current allocation, one scheduling round per step",
+    "per_rank": "one independent cluster per rank",
+    "arithmetic": "int16 matrices, fp32 tables and fitness on the GPU (the oracle computes in fp64)",
+    "l2": "every round rebuilds its 17 MB tables and a fresh population; inside a round the generations work on "
+          "the row store (records + indices, about 40 MB), L2-resident by design; the single-kernel sections flush "
+          "L2 or stream more than L2 per pass",
+}
+
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the committed ncu
 # summaries under profiles/ (not measured in this run); None = the kernel has changed since its
 # counters were taken.
@@ -343,12 +354,7 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": t_max / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "large: 256 nodes x 8 GPUs, 1024 jobs, grid 128x32, population 512, "
-                               "200 generations, p=-1, random current allocation, one scheduling round per step",
-                   "per_rank": "one independent cluster per rank", "arithmetic": "int16 matrices, fp32 tables and fitness",
-                   "l2": "every round rewrites its 268 MB dense initial population and rebuilds the 17 MB tables "
-                         "(more than L2 between timed steps); inside a round the generations work on the "
-                         "row store (records + indices, about 40 MB), L2-resident by design"},
+        "config": CONFIG,
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                 "ms_per_step": e2e_ms / args.steps, "api": "schedule_round_host (pinned host buffers)"},
@@ -749,9 +755,8 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round_s * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "large: 256 nodes x 8 GPUs, 1024 jobs, grid 128x32, population 512, "
-                               "200 generations, p=-1, random current allocation, one scheduling round per step",
-                   "note": "CPU oracle; each step times a bounded sample and extrapolates the round"},
+        "config": CONFIG,
+        "reference_note": "CPU oracle (fp64); each step times a bounded sample and extrapolates the round",
         "cpu_baseline": base,
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }

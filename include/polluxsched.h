@@ -269,6 +269,19 @@ int ga_generation(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_pop
                   const float *d_fitness_in, int16_t *d_pop_out, uint32_t round,
                   uint32_t generation);
 
+/* A slice of ga_generation: children first_child .. first_child + num_children - 1, bit for bit
+ * the children that ga_generation puts at those positions (a child depends on its own index,
+ * the parents and their fitness only).  This is how the population search of Sec. 4.3 shards
+ * by candidate over several GPUs: every GPU holds all parents and their fitness, makes its
+ * share of the children and evaluates them (eval_fitness with count = num_children), and the
+ * caller gathers children and fitness between generations (see dist.evolve_sharded in the
+ * Python package).  d_pop_in: int16 [P][J][num_nodes] and d_fitness_in: fp32 [P], all parents;
+ * d_children: int16 [num_children][J][num_nodes], must not overlap the parents.
+ * Errors: INVALID_ARG when the slice leaves [0, P). */
+int ga_generation_shard(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_pop_in, const float *d_fitness_in,
+                        int32_t first_child, int32_t num_children, int16_t *d_children, uint32_t round,
+                        uint32_t generation);
+
 /* A whole scheduling round: tables, re-allocation factors, initial population and its
  * fitness, `generations` x (ga_generation, eval_fitness), then the best candidate of the
  * last population.  d_cur: int16 [J][num_nodes] or NULL.  d_best: int16 [J][num_nodes],

@@ -20,7 +20,7 @@ ERRORS = {-1: "INVALID_ARG", -2: "BAD_CONFIG", -3: "CUDA", -4: "TIMEOUT", -5: "N
 EXPORTS = (
     "sched_init", "sched_fair_share", "sched_destroy", "sched_last_error", "sched_sync_status", "sched_launch_count",
     "build_speedup_table", "build_speedup_table_msample", "sched_set_racks", "build_speedup_table_rack", "eval_fitness_racks", "fit_throughput_model", "compute_realloc_factor", "autoscale_targets", "eval_fitness", "repair_population",
-    "init_population", "ga_generation", "schedule_round", "schedule_round_host",
+    "init_population", "ga_generation", "ga_generation_shard", "schedule_round", "schedule_round_host",
     "sched_get_population", "sched_get_round_tables", "sched_round_speedup_table", "eval_fitness_host",
     "sched_set_kernel_timing", "sched_num_kernel_kinds", "sched_kernel_kind_name",
     "sched_read_kernel_timing", "sched_measure_peaks", "sched_set_graphs", "sched_set_store_budget", "sched_store_moves", "eval_fitness_noalloc", "eval_fitness_noalloc_last_error",
@@ -79,6 +79,7 @@ def load_library(path: str = LIB_PATH):
     lib.repair_population.argtypes = [vp, C.POINTER(SchedJobs), vp, i32, u32, u32, u32]
     lib.init_population.argtypes = [vp, C.POINTER(SchedJobs), vp, u32, vp]
     lib.ga_generation.argtypes = [vp, C.POINTER(SchedJobs), vp, vp, vp, u32, u32]
+    lib.ga_generation_shard.argtypes = [vp, C.POINTER(SchedJobs), vp, vp, i32, i32, vp, u32, u32]
     lib.schedule_round.argtypes = [vp, C.POINTER(SchedJobs), vp, u32, i32, vp, vp]
     lib.schedule_round_host.argtypes = [vp, C.POINTER(SchedJobs), vp, u32, i32, vp, vp]
     lib.sched_get_population.argtypes = [vp, vp, vp]
@@ -296,6 +297,13 @@ class Scheduler:
         js = C.byref(jobs.struct) if jobs is not None else None
         self._check(_lib.ga_generation(self._ctx, js, _ptr(pop_in), _ptr(fitness_in), _ptr(pop_out),
                                        round, generation))
+
+    def ga_generation_shard(self, jobs, pop_in, fitness_in, children, *, first_child, round, generation,
+                            num_children=None):
+        n = children.shape[0] if num_children is None else num_children
+        js = C.byref(jobs.struct) if jobs is not None else None
+        self._check(_lib.ga_generation_shard(self._ctx, js, _ptr(pop_in), _ptr(fitness_in), first_child, n,
+                                             _ptr(children), round, generation))
 
     def schedule_round(self, jobs, cur, best, best_fitness, *, round, generations):
         self._check(_lib.schedule_round(self._ctx, C.byref(jobs.struct), _ptr(cur), round, generations,

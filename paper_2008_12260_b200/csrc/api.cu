@@ -549,6 +549,28 @@ int ga_generation(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_pop
                            d_pop_in, d_fitness_in, d_pop_out, generation);
 }
 
+int ga_generation_shard(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_pop_in, const float *d_fitness_in,
+                        int32_t first_child, int32_t num_children, int16_t *d_children, uint32_t round,
+                        uint32_t generation) {
+  REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "ga_generation_shard: ctx is NULL");
+  REQUIRE(ctx, d_pop_in && d_fitness_in, SCHED_ERR_INVALID_ARG,
+          "ga_generation_shard: d_pop_in and d_fitness_in must be non-NULL");
+  REQUIRE(ctx, first_child >= 0 && num_children >= 0 && (long long)first_child + num_children <= ctx->cfg.population,
+          SCHED_ERR_INVALID_ARG, "ga_generation_shard: children %d .. %d are not within the population of %d",
+          first_child, first_child + num_children, ctx->cfg.population);
+  if (num_children == 0 || ctx->cfg.num_jobs == 0) return SCHED_OK;
+  REQUIRE(ctx, d_children, SCHED_ERR_INVALID_ARG, "ga_generation_shard: d_children is NULL");
+  const size_t mat = (size_t)ctx->cfg.num_jobs * ctx->cfg.num_nodes;
+  REQUIRE(ctx, d_children + mat * num_children <= d_pop_in || d_pop_in + mat * ctx->cfg.population <= d_children,
+          SCHED_ERR_INVALID_ARG, "ga_generation_shard: parents and children must not overlap");
+  REQUIRE(ctx, (((uintptr_t)d_pop_in | (uintptr_t)d_children) & 1) == 0 && ((uintptr_t)d_fitness_in & 3) == 0,
+          SCHED_ERR_INVALID_ARG, "ga_generation_shard: a buffer is misaligned");
+  int rc = launch_set_round(ctx, round);
+  if (rc != SCHED_OK) return rc;
+  return launch_generation(ctx, d_jobs ? d_jobs->k_cap : nullptr, d_jobs ? d_jobs->active : nullptr, d_pop_in,
+                           d_fitness_in, d_children, generation, first_child, num_children);
+}
+
 // Everything a round enqueues on the stream (the round number is already in d_round).
 static int round_body(sched_ctx *ctx, const sched_jobs *d_jobs, const int16_t *d_cur, int32_t generations,
                       int16_t *d_best, float *d_best_fitness) {

@@ -293,7 +293,7 @@ int launch_init_population(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t
                            const int16_t *d_cur, int16_t *d_pop_out);
 int launch_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active,
                       const int16_t *d_pop_in, const float *d_fitness_in, int16_t *d_pop_out,
-                      uint32_t generation);
+                      uint32_t generation, int first_child = 0, int num_children = -1);
 int launch_set_round(sched_ctx *ctx, uint32_t round);
 int launch_fit(sched_ctx *ctx, int32_t num_jobs, const int32_t *d_offset, const int32_t *d_k, const int32_t *d_n,
                const int32_t *d_m, const int32_t *d_s, const float *d_t, const float *d_theta0,

@@ -1470,18 +1470,21 @@ int launch_init_population(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t
   return launch_rows_cols(ctx, a, d_pop_out, P, 0u, GEN_INIT);
 }
 
+// children first_child .. first_child + num_children - 1 (num_children < 0: all of them)
 int launch_generation(sched_ctx *ctx, const int32_t *d_k_cap, const uint8_t *d_active,
                       const int16_t *d_pop_in, const float *d_fitness_in, int16_t *d_pop_out,
-                      uint32_t generation) {
-  const int P = ctx->cfg.population;
+                      uint32_t generation, int first_child, int num_children) {
+  const int P = num_children < 0 ? ctx->cfg.population : num_children;
+  if (P == 0) return SCHED_OK;
   int rc = ensure_dflag(ctx, P);
   if (rc != SCHED_OK) return rc;
   RowsArgs a = base_rows_args(ctx, d_k_cap, d_active, P);
+  a.first_cand = (uint32_t)first_child;
   a.mode = ROWS_GENERATION; a.src = d_pop_in; a.dst = d_pop_out;
   a.fitness_bits = (const uint32_t *)d_fitness_in;
   a.thr = ctx->cfg.thr_mutate; a.gen = generation; a.key = make_key(ctx->cfg.seed, ctx->d_round);
   a.cur = ctx->round_cur; a.summ = ctx->round_summ; a.summ_in = ctx->round_summ_in;
-  return launch_rows_cols(ctx, a, d_pop_out, P, 0u, generation);
+  return launch_rows_cols(ctx, a, d_pop_out, P, (uint32_t)first_child, generation);
 }
 
 __global__ void set_round_kernel(uint32_t *dst, uint32_t value) { *dst = value; }

@@ -1,9 +1,14 @@
-"""Multi-process plumbing for the benchmark: one process per GPU, no data-path collective.
+"""Multi-process plumbing: one process per GPU.
 
-Scheduling rounds of different clusters (and candidates of one population) are independent
-problems, so ranks only meet to agree on the timing: a barrier on both sides of the timed
-region, the MAX over ranks of the elapsed time and the SUM of the units processed.  Works
-with `nccl` (CUDA tensors) and `gloo` (CPU tensors).
+Scheduling rounds of different clusters are independent problems, so in the benchmark ranks
+only meet to agree on the timing: a barrier on both sides of the timed region, the MAX over
+ranks of the elapsed time and the SUM of the units processed.
+
+One population can also be evolved by several ranks (`evolve_sharded`): the children of a
+generation are independent given the parents, so every rank makes and evaluates a contiguous
+slice of them and the slices are gathered (the one exchange step of the path: an all-gather
+of matrices and fitness) before the next generation.  The result equals the single-process
+search bit for bit.  Works with `nccl` (CUDA tensors) and `gloo` (CPU tensors).
 """
 from __future__ import annotations
 
@@ -58,3 +63,42 @@ def throughput(elapsed_ms: float, units: float, device="cpu"):
     """Whole-job throughput in units per second: all ranks' units over the slowest rank's time."""
     t, u = aggregate(elapsed_ms, units, device)
     return (u / (t * 1e-3)) if t > 0 else 0.0, t, u
+
+
+def all_gather_slices(local, total: int, world: int, rank: int):
+    """Concatenation over ranks of per-rank slices of unequal length (rank r holds the rows
+    shard_range(total, r, world) of the result).  Single process: returns `local`."""
+    import torch
+    import torch.distributed as dist
+
+    if world == 1 or not (dist.is_available() and dist.is_initialized()):
+        return local
+    longest = shard_range(total, 0, world)
+    longest = longest[1] - longest[0]
+    padded = torch.zeros((longest,) + tuple(local.shape[1:]), dtype=local.dtype, device=local.device)
+    padded[: local.shape[0]] = local
+    raw = padded.view(torch.uint8)                 # bytes: every backend gathers them, whatever the element type
+    parts = [torch.empty_like(raw) for _ in range(world)]
+    dist.all_gather(parts, raw)
+    out = []
+    for r in range(world):
+        b, e = shard_range(total, r, world)
+        out.append(parts[r].view(local.dtype).view(padded.shape)[: e - b])
+    return torch.cat(out)
+
+
+def evolve_sharded(make_children, evaluate, pop, fit, generations: int, rank: int, world: int, first_generation: int = 0):
+    """`generations` generations of one population over `world` ranks.
+
+    make_children(pop, fit, first_child, num_children, generation) -> the children's matrices,
+    evaluate(children) -> their fitness (both for this rank's slice only; on a GPU these are
+    Scheduler.ga_generation_shard and Scheduler.eval_fitness).  pop / fit: all parents, identical
+    on every rank.  Returns the final (pop, fit), again identical on every rank."""
+    P = pop.shape[0]
+    b, e = shard_range(P, rank, world)
+    for g in range(first_generation, first_generation + generations):
+        children = make_children(pop, fit, b, e - b, g)
+        cfit = evaluate(children)
+        pop = all_gather_slices(children, P, world, rank)
+        fit = all_gather_slices(cfit, P, world, rank)
+    return pop, fit
