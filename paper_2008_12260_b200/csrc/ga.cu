@@ -923,6 +923,327 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
 }
 
 // ---------------------------------------------------------------------------------------
+// Streaming row kernel: the row pass when no per-row summaries are wanted (the dense entry
+// points called on their own) and a row is a power-of-two number of 16-byte vectors.
+//
+// Almost every entry of a population is zero and almost every row is copied unchanged, so the
+// rows are moved as a stream - a warp reads its 32 rows as one flat run of vectors, four loads
+// per lane in flight, and stores them straight back out - and only the vectors that hold
+// something are looked at: they are compacted into a per-warp queue (ballot + popc) and
+// expanded one lane per entry, once to get each row's K, N and whether any entry leaves
+// [0, node size], and once more for the column totals and occupant lists.  A row that is
+// perturbed, has an entry out of range or breaks a row cap is rebuilt in shared memory by the
+// whole warp, written again, and its queue entries are replaced.  Same operators, draws and
+// results as rows2_kernel; block and grid shapes, column partials and the work list are shared
+// with it.
+// ---------------------------------------------------------------------------------------
+constexpr int STREAM_QCAP = 128;        // vectors a warp queues per tile
+
+// dynamic shared memory of the streaming kernel: per-node arrays sized by the cluster
+__host__ __device__ inline size_t stream_smem_bytes(int NN) {
+  return (size_t)8 * NN * 2          // a row per warp (rebuilt rows)
+         + (size_t)NN * 2            // node sizes
+         + (size_t)NN * 4 * 3        // GPUs placed, distributed jobs, occupants per node
+         + (size_t)NN * OCC_SLOTS * 4;
+}
+
+__global__ void __launch_bounds__(256, 4) rows_stream_kernel(Rows2Args aa) {
+  const RowsArgs &a = aa.r;
+  extern __shared__ __align__(16) unsigned char stream_smem[];
+  const int NN = a.num_nodes, J = a.J;
+  int16_t *s_rows = (int16_t *)stream_smem;                       // [8][NN] per-warp buffer for a row that is rebuilt
+  int16_t *s_cap = s_rows + (size_t)8 * NN;                       // node sizes floored at 0
+  int32_t *s_tot = (int32_t *)(s_cap + NN), *s_el = s_tot + NN, *s_cnt = s_el + NN;
+  uint32_t *s_occ = (uint32_t *)(s_cnt + NN);
+  __shared__ int s_parent[2];
+  __shared__ int s_rank4[4];
+  __shared__ __align__(16) uint4 s_qvec[8][STREAM_QCAP];
+  __shared__ uint32_t s_qmeta[8][STREAM_QCAP];       // row (bits 0..4) | vector of the row (8..13) | alive (31)
+  __shared__ int s_rowK[8][32], s_rowN[8][32], s_rowbad[8][32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int cl = blockIdx.y, batch = blockIdx.x;
+  const uint32_t c = a.first_cand + (uint32_t)cl;
+  const int row_vecs = NN >> 3;                      // a power of two, 1 .. 64
+  const int rv_log2 = 31 - __clz(row_vecs);
+  for (int i = threadIdx.x; i < NN; i += blockDim.x) {
+    s_tot[i] = 0; s_el[i] = 0; s_cnt[i] = 0;
+    s_cap[i] = (int16_t)max((int)a.cap[i], 0);
+  }
+  // ---- parents of this candidate (generation mode), found by the block itself (as rows2_kernel) ----
+  if (a.mode == ROWS_GENERATION) {
+    const int P = a.P;
+    if ((int)c < a.num_elite) {
+      for (int i = threadIdx.x; i < P; i += blockDim.x) {
+        const uint32_t ki = order_key(a.fitness_bits[i]);
+        int rk = 0;
+        for (int o = 0; o < P; ++o) {
+          const uint32_t ko = order_key(__ldg(a.fitness_bits + o));
+          rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
+        }
+        if (rk == (int)c) s_parent[0] = s_parent[1] = i;
+      }
+    } else {
+      const u32x4 sel = draw(a.key, 0u, c, a.gen, SLOT_SELECT);
+      const int idx[4] = {(int)bounded(sel.x, P), (int)bounded(sel.y, P), (int)bounded(sel.z, P),
+                          (int)bounded(sel.w, P)};
+      if (warp < 4) {
+        const int i = idx[warp];
+        const uint32_t ki = order_key(a.fitness_bits[i]);
+        int rk = 0;
+        for (int o = lane; o < P; o += 32) {
+          const uint32_t ko = order_key(__ldg(a.fitness_bits + o));
+          rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
+        }
+        rk = warp_sum(rk);
+        if (lane == 0) s_rank4[warp] = rk;
+      }
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        s_parent[0] = s_rank4[0] <= s_rank4[1] ? idx[0] : idx[1];
+        s_parent[1] = s_rank4[2] <= s_rank4[3] ? idx[2] : idx[3];
+      }
+    }
+  }
+  __syncthreads();
+
+  const int j0 = batch * 256 + warp * 32;
+  const int nrows = min(32, J - j0);          // may be <= 0 for trailing warps
+  // ---- per-lane set-up for row j0 + lane: the row's draws, 32 side by side ---------------------
+  bool act_l = false, mut_l = false, sec_l = false;
+  int kc_l = 0;
+  u32x4 mw = {0, 0, 0, 0};
+  if (lane < nrows) {
+    const int j = j0 + lane;
+    act_l = !a.active || a.active[j];
+    kc_l = max(0, min(a.k_cap ? a.k_cap[j] : a.k_max, a.k_max));
+    if (a.mode == ROWS_GENERATION) {
+      if ((int)c >= a.num_elite) {
+        sec_l = (draw(a.key, (uint32_t)j, c, a.gen, SLOT_XOVER).x >> 31) != 0u;
+        mw = draw(a.key, (uint32_t)j, c, a.gen, SLOT_MUTATE);
+        mut_l = mw.x < a.thr;
+      }
+    } else if (a.mode == ROWS_INIT && c > 0) {
+      mw = draw(a.key, (uint32_t)j, c, GEN_INIT, SLOT_INIT);
+      mut_l = mw.x < a.thr;
+    }
+  }
+  const unsigned act_mask = __ballot_sync(0xffffffffu, act_l);
+  const unsigned sec_mask = __ballot_sync(0xffffffffu, sec_l);
+  const unsigned mut_mask = __ballot_sync(0xffffffffu, mut_l && act_l);
+
+  // row j0 of the possible sources; per row only the offset r * NN is added
+  const size_t roff0 = (size_t)j0 * NN;
+  const int16_t *src_a = nullptr, *src_b = nullptr;
+  if (a.mode == ROWS_GENERATION) {
+    src_a = a.src + (size_t)s_parent[0] * J * NN + roff0;
+    src_b = a.src + (size_t)s_parent[1] * J * NN + roff0;
+  } else if (a.mode == ROWS_INIT) {
+    src_a = src_b = a.src ? a.src + roff0 : nullptr;
+  } else {
+    src_a = src_b = a.dst + (size_t)cl * J * NN + roff0;
+  }
+  int16_t *dst0 = a.dst + (size_t)cl * J * NN + roff0;
+  int16_t *row = s_rows + (size_t)warp * NN;
+  uint4 *qvec = s_qvec[warp];
+  uint32_t *qmeta = s_qmeta[warp];
+
+  const int total_vecs = max(nrows, 0) << rv_log2;      // the warp's rows as one run of vectors
+  // four vectors per lane of the tile at t0 (rows that are inactive or have no source read as empty)
+  auto fetch_tile = [&](int t0, uint4 (&y)[4]) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int t = t0 + q * 32 + lane;
+      const int r = t >> rv_log2, v = t & (row_vecs - 1);
+      y[q] = make_uint4(0u, 0u, 0u, 0u);
+      const int16_t *src = ((sec_mask >> (r & 31)) & 1u) ? src_b : src_a;
+      if (t < total_vecs && ((act_mask >> (r & 31)) & 1u) && src) y[q] = __ldg((const uint4 *)(src + (size_t)r * NN) + v);
+    }
+  };
+  for (int t0 = 0; t0 < total_vecs; t0 += 128) {
+    // rows of this tile: [r_first, r_first + rows_here); a tile never splits a row
+    const int r_first = t0 >> rv_log2;
+    const int rows_here = min(nrows - r_first, max(128 >> rv_log2, 1));
+    s_rowK[warp][lane] = 0; s_rowN[warp][lane] = 0; s_rowbad[warp][lane] = 0;
+    // ---- the stream: four vectors per lane in, queued if they hold anything, out ---------------
+    uint4 x[4];
+    fetch_tile(t0, x);
+    int qn = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int t = t0 + q * 32 + lane;
+      const int r = t >> rv_log2, v = t & (row_vecs - 1);
+      const bool in = t < total_vecs;
+      const bool nz = in && (x[q].x | x[q].y | x[q].z | x[q].w) != 0u;
+      const unsigned bal = __ballot_sync(0xffffffffu, nz);
+      if (nz) {
+        const int pos = qn + __popc(bal & ((1u << lane) - 1u));
+        qvec[pos] = x[q];
+        qmeta[pos] = (uint32_t)(r - r_first) | ((uint32_t)v << 8) | 0x80000000u;
+      }
+      qn += __popc(bal);
+      if (in) ((uint4 *)(dst0 + (size_t)r * NN))[v] = x[q];       // final for every row that is not rebuilt below
+    }
+    __syncwarp();
+    // ---- first look at the queued entries: each row's K and N, entries outside [0, node size] ----
+    for (int e = lane; e < qn * 8; e += 32) {
+      const int val = (int)((const int16_t *)qvec)[e];
+      if (val != 0) {
+        const uint32_t meta = qmeta[e >> 3];
+        const int rr = (int)(meta & 31u), n = (int)((meta >> 8) & 63u) * 8 + (e & 7);
+        const int cv = min(max(val, 0), (int)s_cap[n]);
+        if (cv != val) s_rowbad[warp][rr] = 1;
+        if (cv > 0) { atomicAdd(&s_rowK[warp][rr], cv); atomicAdd(&s_rowN[warp][rr], 1); }
+      }
+    }
+    __syncwarp();
+    // ---- rows that have to be rebuilt: perturbed, an entry out of range, or a row cap broken ----
+    bool need_l = false;
+    const int kc_r = __shfl_sync(0xffffffffu, kc_l, (r_first + lane) & 31);   // the cap of the tile's lane-th row
+    if (lane < rows_here) {
+      const int r = r_first + lane;
+      need_l = ((act_mask >> r) & 1u) &&
+               (((mut_mask >> r) & 1u) || s_rowbad[warp][lane] || s_rowK[warp][lane] > kc_r || s_rowN[warp][lane] > a.n_max);
+    }
+    unsigned need = __ballot_sync(0xffffffffu, need_l);
+    while (need) {
+      const int rl = __ffs(need) - 1;           // row within the tile
+      need &= need - 1;
+      const int rr = r_first + rl;
+      const int16_t *src = ((sec_mask >> rr) & 1u) ? src_b : src_a;
+      // the row, every entry forced into [0, node size]
+      for (int v = lane; v < row_vecs; v += 32) {
+        uint4 y = make_uint4(0u, 0u, 0u, 0u);
+        if (src) y = clamp_vec(__ldg((const uint4 *)(src + (size_t)rr * NN) + v), ((const uint4 *)s_cap)[v]);
+        ((uint4 *)row)[v] = y;
+      }
+      __syncwarp();
+      int rK = 0, rN = 0;
+      for (int n = lane; n < NN; n += 32) { rK += row[n]; rN += row[n] > 0; }
+      rK = __reduce_add_sync(0xffffffffu, rK);
+      rN = __reduce_add_sync(0xffffffffu, rN);
+      if ((mut_mask >> rr) & 1u) {
+        const uint32_t m1 = __shfl_sync(0xffffffffu, mw.y, rr), m2 = __shfl_sync(0xffffffffu, mw.z, rr),
+                       m3 = __shfl_sync(0xffffffffu, mw.w, rr);
+        const uint32_t op = bounded(m1, 3u);
+        if (op == 0u) {
+          const int n = (int)bounded(m3, (uint32_t)NN);
+          if (lane == 0) row[n] = (int16_t)min((int)row[n] + 1, (int)s_cap[n]);
+        } else if (rN > 0) {
+          const int ns = nth_occupied(row, NN, bounded(m2, (uint32_t)rN), lane);
+          if (op == 1u) {
+            if (lane == 0) row[ns] = (int16_t)(row[ns] - 1);
+          } else {
+            const int nd = (int)bounded(m3, (uint32_t)NN);
+            if (nd != ns && lane == 0) {
+              row[nd] = (int16_t)min((int)row[nd] + (int)row[ns], (int)s_cap[nd]);
+              row[ns] = 0;
+            }
+          }
+        }
+        __syncwarp();
+        rK = 0; rN = 0;
+        for (int n = lane; n < NN; n += 32) { rK += row[n]; rN += row[n] > 0; }
+        rK = __reduce_add_sync(0xffffffffu, rK);
+        rN = __reduce_add_sync(0xffffffffu, rN);
+      }
+      const int rkc = __shfl_sync(0xffffffffu, kc_l, rr);
+      if (rK > rkc || rN > a.n_max) {
+        if (lane == 0) {
+          int excess = rK - rkc;
+          rK = min(rK, rkc);
+          for (int n = NN - 1; n >= 0 && excess > 0; --n) {
+            const int take = min((int)row[n], excess);
+            row[n] = (int16_t)(row[n] - take);
+            excess -= take;
+          }
+          int occ = 0;
+          for (int n = 0; n < NN; ++n) {
+            if (row[n] > 0) {
+              ++occ;
+              if (occ > a.n_max) { rK -= row[n]; row[n] = 0; }
+            }
+          }
+          rN = min(occ, a.n_max);
+        }
+        rN = __shfl_sync(0xffffffffu, rN, 0);
+        rK = __shfl_sync(0xffffffffu, rK, 0);
+        __syncwarp();
+      }
+      if (lane == 0) { s_rowK[warp][rl] = rK; s_rowN[warp][rl] = rN; }
+      // the row's queued vectors are dropped; the row is written again and its occupants go
+      // straight into the column totals and lists
+      for (int e = lane; e < qn; e += 32)
+        if ((qmeta[e] & 31u) == (uint32_t)rl) qmeta[e] &= 0x7FFFFFFFu;
+      for (int v = lane; v < row_vecs; v += 32) ((uint4 *)(dst0 + (size_t)rr * NN))[v] = ((const uint4 *)row)[v];
+      for (int n = lane; n < NN; n += 32) {
+        const int val = row[n];
+        if (val > 0) {
+          atomicAdd(&s_tot[n], val);
+          if (rN >= 2) atomicAdd(&s_el[n], 1);
+          const int slot = atomicAdd(&s_cnt[n], 1);
+          if (slot < OCC_SLOTS)
+            s_occ[n * OCC_SLOTS + slot] = (uint32_t)(j0 + rr) | ((uint32_t)val << 20) | (rN >= 2 ? 0x80000000u : 0u);
+        }
+      }
+      __syncwarp();
+    }
+    // ---- second look: column totals, distributed-job counts and occupant lists --------------------
+    for (int e = lane; e < qn * 8; e += 32) {
+      const uint32_t meta = qmeta[e >> 3];
+      const int val = (int)((const int16_t *)qvec)[e];
+      if ((meta >> 31) && val > 0) {
+        const int rl = (int)(meta & 31u), n = (int)((meta >> 8) & 63u) * 8 + (e & 7);
+        const bool dist = s_rowN[warp][rl] >= 2;
+        atomicAdd(&s_tot[n], val);
+        if (dist) atomicAdd(&s_el[n], 1);
+        const int slot = atomicAdd(&s_cnt[n], 1);
+        if (slot < OCC_SLOTS)
+          s_occ[n * OCC_SLOTS + slot] = (uint32_t)(j0 + r_first + rl) | ((uint32_t)val << 20) | (dist ? 0x80000000u : 0u);
+      }
+    }
+    if (lane < rows_here) {
+      const int r = r_first + lane;
+      a.dflag[(size_t)cl * J + j0 + r] = (((act_mask >> r) & 1u) && s_rowN[warp][lane] >= 2) ? 1 : 0;
+    }
+    __syncwarp();
+  }
+
+  __syncthreads();
+  // ---- column partials and occupant lists of the block (as rows2_kernel) ----------------------
+  const size_t base = ((size_t)cl * aa.nbatch + batch) * NN;
+  for (int i = threadIdx.x; i < NN; i += blockDim.x) {
+    aa.colsum[base + i] = s_tot[i];
+    aa.colelig[base + i] = s_el[i];
+    aa.occ_count[base + i] = s_cnt[i];
+    const int cnt = min(s_cnt[i], OCC_SLOTS);
+    for (int k = 0; k < cnt; ++k) aa.occ_list[(base + i) * OCC_SLOTS + k] = s_occ[i * OCC_SLOTS + k];
+  }
+  __shared__ bool s_last_block;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned prev = atomicAdd(aa.cand_ticket + cl, 1u);
+    s_last_block = (prev == (unsigned)aa.nbatch - 1u);
+    if (s_last_block) aa.cand_ticket[cl] = 0u;
+  }
+  __syncthreads();
+  if (s_last_block) {
+    __threadfence();
+    for (int n = threadIdx.x; n < NN; n += blockDim.x) {
+      int total = 0, nelig = 0;
+      for (int b = 0; b < aa.nbatch; ++b) {
+        total += __ldcg(aa.colsum + ((size_t)cl * aa.nbatch + b) * NN + n);
+        nelig += __ldcg(aa.colelig + ((size_t)cl * aa.nbatch + b) * NN + n);
+      }
+      if (nelig >= 2 || total > (int)s_cap[n]) {
+        const unsigned slot = atomicAdd(aa.list_count, 1u);
+        aa.list[slot] = ((uint32_t)cl << 13) | (uint32_t)n;
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
 // Small problems (at most 256 jobs, at most 32 nodes): one block per candidate, one THREAD
 // per row.  A row is 16 to 64 bytes, so a thread reads its parent's row with one to four
 // vector loads, keeps it in its own line of shared memory, perturbs and caps it there, and
@@ -1365,6 +1686,34 @@ int launch_rows_cols(sched_ctx *ctx, RowsArgs &a, int16_t *pop, int count, uint3
   aa.fitness_out = ctx->ff_out;
   ctx->fit_done = aa.fuse != 0;
   dim3 grid((unsigned)nbatch, (unsigned)count);
+  const int row_vecs_all = NN / 8;
+  if (!aa.fuse && a.summ == nullptr && (row_vecs_all & (row_vecs_all - 1)) == 0) {
+    // no per-row summaries wanted (the entry points called on their own): the streaming kernel
+    const size_t smem = stream_smem_bytes(NN);
+    if (smem > 24 * 1024) {
+      cudaError_t e = cudaFuncSetAttribute(rows_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) {
+        set_error(ctx, "cudaFuncSetAttribute failed: %s", cudaGetErrorString(e));
+        return SCHED_ERR_CUDA;
+      }
+    }
+    SCHED_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->d_colcount, 0, sizeof(unsigned int), ctx->stream));
+    {
+      TimedLaunch tl_(ctx, KK_ROWS);
+      rows_stream_kernel<<<grid, 256, smem, ctx->stream>>>(aa);
+    }
+    SCHED_LAUNCH_CHECK(ctx);
+    ColfixArgs f;
+    f.pop = pop; f.dflag = ctx->d_dflag; f.cap = ctx->d_cap;
+    f.colsum = ctx->d_colsum; f.colelig = ctx->d_colelig; f.summ = nullptr;
+    f.J = a.J; f.num_nodes = NN; f.nbatch = nbatch;
+    f.gen = gen; f.first_cand = first_cand; f.key = make_key(ctx->cfg.seed, ctx->d_round);
+    f.list = ctx->d_collist; f.list_count = ctx->d_colcount;
+    f.cur = nullptr; f.occ_count = ctx->d_occcount; f.occ_list = ctx->d_occlist;
+    { TimedLaunch tl_(ctx, KK_COLS); colrepair_kernel<<<ctx->num_sms * 4, 128, 0, ctx->stream>>>(f); }
+    SCHED_LAUNCH_CHECK(ctx);
+    return SCHED_OK;
+  }
   if (aa.fuse && a.mode == ROWS_GENERATION && NN <= SMALL_MAX_NODES && a.J <= 8192) {
     // small problem inside a round: thread-per-row kernel, fitness included
     {

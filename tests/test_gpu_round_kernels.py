@@ -20,6 +20,10 @@ CASES = [
     # rows move to the other half several times
     synth.Config("store-compaction", 32, 8, 300, 11, 16, 8, 48, 24, num_elite=3, mutate_prob=0.5,
                  init_prob=0.3, with_history=True, random_cur=True),
+    # every row perturbed in every generation and a pool with room for two worst-case generations only:
+    # a candidate may take its full J + 16 slots per generation without the pool running out
+    synth.Config("store-all-perturbed", 16, 4, 280, 21, 16, 8, 20, 10, num_elite=1, mutate_prob=1.0,
+                 init_prob=1.0, with_history=True, random_cur=True),
     # few large nodes: more jobs on a node than a block lists per node (column scan through the
     # indices), and many GPUs per job
     synth.Config("store-crowded-nodes", 8, 64, 400, 12, 16, 8, 32, 12, num_elite=2, mutate_prob=0.3,
@@ -95,7 +99,7 @@ def test_store_round_equals_dense_stepwise_round(gpu, oracle, cfg):
     penalise = cur is not None
     rnd = 3
     s = api.scheduler_for(cfg, stream=torch.cuda.current_stream().cuda_stream)
-    if cfg.name == "store-compaction":
+    if cfg.name in ("store-compaction", "store-all-perturbed"):
         # a pool with room for two worst-case generations per half: the rows have to move every
         # other generation or so
         rows, worst = cfg.population * cfg.num_jobs, cfg.population * (cfg.num_jobs + 16)
@@ -118,7 +122,7 @@ def test_store_round_equals_dense_stepwise_round(gpu, oracle, cfg):
     assert np.array_equal(best.cpu().numpy(), pop[i]) and float(bf.item()) == fit[i]
     for c in range(cfg.population):
         assert feasible(pop[c], cl.node_capacity, jobs.k_cap, cl.n_max)
-    if cfg.name == "store-compaction":
+    if cfg.name in ("store-compaction", "store-all-perturbed"):
         assert s.store_moves() >= 3
     elif cfg.name.startswith("store-"):
         assert s.store_moves() == 0
