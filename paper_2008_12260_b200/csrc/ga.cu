@@ -1048,40 +1048,49 @@ __global__ void __launch_bounds__(256, 4) rows_stream_kernel(Rows2Args aa) {
   uint32_t *qmeta = s_qmeta[warp];
 
   const int total_vecs = max(nrows, 0) << rv_log2;      // the warp's rows as one run of vectors
-  // four vectors per lane of the tile at t0 (rows that are inactive or have no source read as empty)
-  auto fetch_tile = [&](int t0, uint4 (&y)[4]) {
+  // Rows are contiguous, so the warp's rows are one flat array of vectors in each source and in the
+  // destination: vector t of the run is element t of all three.  What depends on the lane and the
+  // slot q only (a tile never splits a row) is worked out once: the vector's row within the tile and
+  // its place in that row.
+  const uint4 *flat_a = (const uint4 *)src_a, *flat_b = (const uint4 *)src_b;
+  uint4 *flat_d = (uint4 *)dst0;
+  uint32_t meta_q[4];
+  int rel_row[4];
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int t = t0 + q * 32 + lane;
-      const int r = t >> rv_log2, v = t & (row_vecs - 1);
-      y[q] = make_uint4(0u, 0u, 0u, 0u);
-      const int16_t *src = ((sec_mask >> (r & 31)) & 1u) ? src_b : src_a;
-      if (t < total_vecs && ((act_mask >> (r & 31)) & 1u) && src) y[q] = __ldg((const uint4 *)(src + (size_t)r * NN) + v);
-    }
-  };
+  for (int q = 0; q < 4; ++q) {
+    const int u = q * 32 + lane;
+    rel_row[q] = u >> rv_log2;
+    meta_q[q] = (uint32_t)rel_row[q] | ((uint32_t)(u & (row_vecs - 1)) << 8) | 0x80000000u;
+  }
   for (int t0 = 0; t0 < total_vecs; t0 += 128) {
-    // rows of this tile: [r_first, r_first + rows_here); a tile never splits a row
+    // rows of this tile: [r_first, r_first + rows_here)
     const int r_first = t0 >> rv_log2;
     const int rows_here = min(nrows - r_first, max(128 >> rv_log2, 1));
     s_rowK[warp][lane] = 0; s_rowN[warp][lane] = 0; s_rowbad[warp][lane] = 0;
     // ---- the stream: four vectors per lane in, queued if they hold anything, out ---------------
+    // (rows that are inactive or have no source read as empty)
     uint4 x[4];
-    fetch_tile(t0, x);
-    int qn = 0;
+    bool in[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const int t = t0 + q * 32 + lane;
-      const int r = t >> rv_log2, v = t & (row_vecs - 1);
-      const bool in = t < total_vecs;
-      const bool nz = in && (x[q].x | x[q].y | x[q].z | x[q].w) != 0u;
+      const int r = r_first + rel_row[q];
+      in[q] = t < total_vecs;
+      x[q] = make_uint4(0u, 0u, 0u, 0u);
+      if (in[q] && ((act_mask >> (r & 31)) & 1u) && flat_a) x[q] = __ldg((((sec_mask >> (r & 31)) & 1u) ? flat_b : flat_a) + t);
+    }
+    int qn = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const bool nz = (x[q].x | x[q].y | x[q].z | x[q].w) != 0u;      // vectors outside the run are empty
       const unsigned bal = __ballot_sync(0xffffffffu, nz);
       if (nz) {
         const int pos = qn + __popc(bal & ((1u << lane) - 1u));
         qvec[pos] = x[q];
-        qmeta[pos] = (uint32_t)(r - r_first) | ((uint32_t)v << 8) | 0x80000000u;
+        qmeta[pos] = meta_q[q];
       }
       qn += __popc(bal);
-      if (in) ((uint4 *)(dst0 + (size_t)r * NN))[v] = x[q];       // final for every row that is not rebuilt below
+      if (in[q]) flat_d[t0 + q * 32 + lane] = x[q];       // final for every row that is not rebuilt below
     }
     __syncwarp();
     // ---- first look at the queued entries: each row's K and N, entries outside [0, node size] ----
