@@ -256,6 +256,13 @@ __device__ __forceinline__ uint32_t order_key(uint32_t bits) {
   return bits ^ ((bits >> 31) ? 0xFFFFFFFFu : 0x80000000u);
 }
 
+// The better-ranked of two candidates.  A rank is a candidate's position when the population is
+// ordered by fitness key descending, index ascending: a permutation, so comparing the two (key,
+// index) pairs answers the same question as comparing the two ranks, without counting either.
+__device__ __forceinline__ int tournament_winner(uint32_t key_i, int i, uint32_t key_j, int j) {
+  return (key_i > key_j || (key_i == key_j && i <= j)) ? i : j;
+}
+
 __device__ __forceinline__ int warp_sum(int v) { return __reduce_add_sync(0xffffffffu, v); }
 
 // node index of the t-th occupied entry (ascending) of a row held in shared memory

@@ -548,7 +548,6 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
   __shared__ int32_t s_tot[MAXN], s_el[MAXN], s_cnt[MAXN];
   __shared__ uint32_t s_occ[MAXN * OCC_SLOTS];
   __shared__ int s_parent[2];
-  __shared__ int s_rank4[4];
   __shared__ uint32_t s_summ[256];   // row summaries of the block's rows
   __shared__ float s_term[256];
   // per-warp queue of non-empty vectors waiting to be expanded into occupants
@@ -570,7 +569,7 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
   // ---- parents of this candidate (generation mode), found by the block itself -------------
   // rank(i) = number of candidates ordered before i (fitness descending, index ascending).
   // An elite child needs the candidate of rank c; any other child the better-ranked of two
-  // random pairs, i.e. the ranks of four candidates only.
+  // random pairs, which the two candidates' own keys and indices decide.
   if (a.mode == ROWS_GENERATION) {
     const int P = a.P;
     if ((int)c < a.num_elite) {
@@ -587,21 +586,12 @@ __global__ void __launch_bounds__(256, 4) rows2_kernel(Rows2Args aa) {
       const u32x4 sel = draw(a.key, 0u, c, a.gen, SLOT_SELECT);
       const int idx[4] = {(int)bounded(sel.x, P), (int)bounded(sel.y, P), (int)bounded(sel.z, P),
                           (int)bounded(sel.w, P)};
-      if (warp < 4) {
-        const int i = idx[warp];
-        const uint32_t ki = order_key(a.fitness_bits[i]);
-        int rk = 0;
-        for (int o = lane; o < P; o += 32) {
-          const uint32_t ko = order_key(__ldg(a.fitness_bits + o));
-          rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
-        }
-        rk = warp_sum(rk);
-        if (lane == 0) s_rank4[warp] = rk;
-      }
-      __syncthreads();
       if (threadIdx.x == 0) {
-        s_parent[0] = s_rank4[0] <= s_rank4[1] ? idx[0] : idx[1];
-        s_parent[1] = s_rank4[2] <= s_rank4[3] ? idx[2] : idx[3];
+        uint32_t k4[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) k4[q] = order_key(__ldg(a.fitness_bits + idx[q]));
+        s_parent[0] = tournament_winner(k4[0], idx[0], k4[1], idx[1]);
+        s_parent[1] = tournament_winner(k4[2], idx[2], k4[3], idx[3]);
       }
     }
   }
@@ -956,7 +946,6 @@ __global__ void __launch_bounds__(256, 4) rows_stream_kernel(Rows2Args aa) {
   int32_t *s_tot = (int32_t *)(s_cap + NN), *s_el = s_tot + NN, *s_cnt = s_el + NN;
   uint32_t *s_occ = (uint32_t *)(s_cnt + NN);
   __shared__ int s_parent[2];
-  __shared__ int s_rank4[4];
   __shared__ __align__(16) uint4 s_qvec[8][STREAM_QCAP];
   __shared__ uint32_t s_qmeta[8][STREAM_QCAP];       // row (bits 0..4) | vector of the row (8..13) | alive (31)
   __shared__ int s_rowK[8][32], s_rowN[8][32], s_rowbad[8][32];
@@ -986,21 +975,12 @@ __global__ void __launch_bounds__(256, 4) rows_stream_kernel(Rows2Args aa) {
       const u32x4 sel = draw(a.key, 0u, c, a.gen, SLOT_SELECT);
       const int idx[4] = {(int)bounded(sel.x, P), (int)bounded(sel.y, P), (int)bounded(sel.z, P),
                           (int)bounded(sel.w, P)};
-      if (warp < 4) {
-        const int i = idx[warp];
-        const uint32_t ki = order_key(a.fitness_bits[i]);
-        int rk = 0;
-        for (int o = lane; o < P; o += 32) {
-          const uint32_t ko = order_key(__ldg(a.fitness_bits + o));
-          rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
-        }
-        rk = warp_sum(rk);
-        if (lane == 0) s_rank4[warp] = rk;
-      }
-      __syncthreads();
       if (threadIdx.x == 0) {
-        s_parent[0] = s_rank4[0] <= s_rank4[1] ? idx[0] : idx[1];
-        s_parent[1] = s_rank4[2] <= s_rank4[3] ? idx[2] : idx[3];
+        uint32_t k4[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) k4[q] = order_key(__ldg(a.fitness_bits + idx[q]));
+        s_parent[0] = tournament_winner(k4[0], idx[0], k4[1], idx[1]);
+        s_parent[1] = tournament_winner(k4[2], idx[2], k4[3], idx[3]);
       }
     }
   }
@@ -1273,7 +1253,7 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
   __shared__ uint32_t s_summ[256];
   __shared__ uint8_t s_dirty[256];
   __shared__ float s_term[256];
-  __shared__ int s_parent[2], s_rank4[4];
+  __shared__ int s_parent[2];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int cl = blockIdx.x;
   const uint32_t c = a.first_cand + (uint32_t)cl;
@@ -1316,8 +1296,10 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
   }
   // from here on the parents' population and fitness are read: the grid that wrote them must be done
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (staged && tid < P) s_keys[tid] = order_key(__ldcg(a.fitness_bits + tid));
-  __syncthreads();
+  if (elite) {
+    if (staged && tid < P) s_keys[tid] = order_key(__ldcg(a.fitness_bits + tid));
+    __syncthreads();
+  }
   const bool early = !elite && row_vecs <= 2;
   uint4 cand[2][2] = {{make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)},
                       {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)}};
@@ -1345,8 +1327,8 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
   } else {
     const u32x4 sel = draw(a.key, 0u, c, a.gen, SLOT_SELECT);
     const int idx[4] = {(int)bounded(sel.x, P), (int)bounded(sel.y, P), (int)bounded(sel.z, P), (int)bounded(sel.w, P)};
-    // short rows: this thread's row of both candidates of its pair is fetched while the ranks
-    // are being worked out
+    // short rows: this thread's row of both candidates of its pair is fetched together with the
+    // candidates' keys
     if (early && j < J && on) {
       pair0 = idx[second ? 2 : 0];
       const uint4 *r0 = (const uint4 *)(a.src + ((size_t)pair0 * J + j) * NN);
@@ -1355,21 +1337,12 @@ __global__ void __launch_bounds__(256) generation_small_kernel(Rows2Args aa) {
       cand[1][0] = __ldcg(r1);
       if (row_vecs > 1) { cand[0][1] = __ldcg(r0 + 1); cand[1][1] = __ldcg(r1 + 1); }
     }
-    if (warp < 4) {
-      const int i = idx[warp];
-      const uint32_t ki = staged ? s_keys[i] : order_key(__ldcg(a.fitness_bits + i));
-      int rk = 0;
-      for (int o = lane; o < P; o += 32) {
-        const uint32_t ko = staged ? s_keys[o] : order_key(__ldcg(a.fitness_bits + o));
-        rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
-      }
-      rk = warp_sum(rk);
-      if (lane == 0) s_rank4[warp] = rk;
-    }
-    __syncthreads();
     if (tid == 0) {
-      s_parent[0] = s_rank4[0] <= s_rank4[1] ? idx[0] : idx[1];
-      s_parent[1] = s_rank4[2] <= s_rank4[3] ? idx[2] : idx[3];
+      uint32_t k4[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) k4[q] = order_key(__ldcg(a.fitness_bits + idx[q]));
+      s_parent[0] = tournament_winner(k4[0], idx[0], k4[1], idx[1]);
+      s_parent[1] = tournament_winner(k4[2], idx[2], k4[3], idx[3]);
     }
   }
   __syncthreads();

@@ -287,7 +287,9 @@ __global__ void __launch_bounds__(256) rowstore_build_cur_kernel(BuildCurArgs a)
       summarise_row<PPL>(g, s_row[grp], cur, K, N, nd, s_rec[grp]);
       const size_t slot = pass == 0 ? (size_t)a.J + j : (size_t)j;
       if (g.sub == 0) {
-        s_rec[grp][REC_SUMM] = pack_summary(K, N, nd);
+        // (before the row caps K may exceed its field: the row is only a perturbation's source then,
+        // and that path adds the entries up itself)
+        s_rec[grp][REC_SUMM] = pack_summary(min(K, 2047), N, nd);
         s_rec[grp][REC_TERM] = __float_as_uint(fitness_term(a.tp, j, K, N, nd != 0));
       }
       if (N > REC_ENTRIES) store_row(g, a.st.pool + slot * a.NN, s_row[grp]);
@@ -804,7 +806,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   uint4 *s_stash = (uint4 *)(smem + L.stash);         // per perturbed row: draw words y, z, w and the replica cap
   __shared__ int s_nmut, s_novf, s_nslow, s_nmod, s_nneed, s_ncow, s_fail, s_anyscan, s_po;
   __shared__ unsigned int s_base_mut, s_base_cow, s_base_cow2;
-  __shared__ int s_parent, s_rank4[4], s_red[GEN_WARPS + 1];
+  __shared__ int s_parent, s_red[GEN_WARPS + 1];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint32_t *my_list = (uint32_t *)s_rowbuf + tid * LIST_WORDS;
@@ -870,13 +872,14 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   // changes; one atomic, asked for now and needed once the parents are known -------------------
   unsigned int base_reg = 0, half_reg = 0;
   const int nmut = s_nmut;
-  if (tid == GEN_THREADS - 1) {          // a thread of a warp that has no rank to work out
+  if (tid == GEN_THREADS - 1) {
     half_reg = __ldcg(a.state + 1);
     base_reg = atomicAdd(a.state, (unsigned int)(nmut + COW_RESERVE));
   }
 
   // ---- parents: the candidate of rank c for an elite child, else the better-ranked of two
   // random pairs (rank = candidates ordered before, fitness descending, index ascending) ----
+  int par_a = 0, par_b = 0;
   if (INIT) {
     // every candidate descends from the current allocation
   } else if (elite) {
@@ -919,29 +922,12 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
     }
     if (tid == 0) s_parent = (int)(0xFFFFFFFFu - (uint32_t)(prev & 0xFFFFFFFFull));
   } else {
-    // The ranks of the four drawn candidates, a warp each.  The keys are first staged in shared
-    // memory (the rows' slot and term arrays, unused until the rows are read) when they fit: every
-    // block of the grid asks for the same few lines at the same moment, so each key is fetched once
-    // per block rather than once per warp.
-    uint32_t *s_keys = s_slot;
-    const bool staged = (size_t)P * 4 <= (size_t)J * 8;
-    if (staged) {
-#pragma unroll 1
-      for (int i = tid; i < P; i += GEN_THREADS) s_keys[i] = order_key(__ldcg(a.fitness_bits + i));
-      __syncthreads();
-    }
-    if (warp < 4) {
-      const int i = warp == 0 ? idx[0] : warp == 1 ? idx[1] : warp == 2 ? idx[2] : idx[3];
-      const uint32_t ki = staged ? s_keys[i] : order_key(__ldcg(a.fitness_bits + i));
-      int rk = 0;
-#pragma unroll 4
-      for (int o = lane; o < P; o += 32) {
-        const uint32_t ko = staged ? s_keys[o] : order_key(__ldcg(a.fitness_bits + o));
-        rk += (ko > ki || (ko == ki && o < i)) ? 1 : 0;
-      }
-      rk = warp_sum(rk);
-      if (lane == 0) s_rank4[warp] = rk;
-    }
+    // the four drawn candidates' keys (every thread asks for the same four words)
+    uint32_t k4[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) k4[q] = __ldcg(a.fitness_bits + idx[q]);
+    par_a = tournament_winner(order_key(k4[0]), idx[0], order_key(k4[1]), idx[1]);
+    par_b = tournament_winner(order_key(k4[2]), idx[2], order_key(k4[3]), idx[3]);
   }
   if (tid == GEN_THREADS - 1) {
     const unsigned long long limit = (unsigned long long)(half_reg + 1u) * a.st.half_cap;
@@ -954,14 +940,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   }
   __syncthreads();
   const bool fail = s_fail != 0;          // no slots: perturbed rows stay as their parents', nothing is repaired
-  int par_a = 0, par_b = 0;
-  if (!INIT) {
-    if (elite) { par_a = par_b = s_parent; }
-    else {
-      par_a = s_rank4[0] <= s_rank4[1] ? idx[0] : idx[1];
-      par_b = s_rank4[2] <= s_rank4[3] ? idx[2] : idx[3];
-    }
-  }
+  if (!INIT && elite) par_a = par_b = s_parent;
 
   // occupant (job j holds g GPUs on node n) into the node's totals and list
   auto add_occupant = [&](int j, int n, int g, bool dist) {
@@ -1082,6 +1061,11 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
     if (!slow) {
       RowList rl;
       list_from_record(rl, my_list, lo, hi);
+      // K from the entries: the row a perturbation starts from may hold more GPUs than the summary's
+      // field can say (the current allocation before the row caps)
+      rl.K = 0;
+#pragma unroll 1
+      for (int k = 0; k < rl.n; ++k) rl.K += ent_gpus(rl.e[k]);
       u32x4 mw;
       int kc;
       if (i < MUT_STASH) {

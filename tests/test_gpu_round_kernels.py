@@ -24,6 +24,10 @@ CASES = [
     # a candidate may take its full J + 16 slots per generation without the pool running out
     synth.Config("store-all-perturbed", 16, 4, 280, 21, 16, 8, 20, 10, num_elite=1, mutate_prob=1.0,
                  init_prob=1.0, with_history=True, random_cur=True),
+    # a current allocation that breaks every rule (node sizes, replica caps, interference) on large
+    # nodes: rows hold more GPUs before the row caps than a summary can say
+    synth.Config("store-infeasible-current", 8, 1500, 300, 22, 16, 8, 24, 6, num_elite=2, mutate_prob=0.3,
+                 init_prob=0.6, with_history=True, random_cur=False),
     # few large nodes: more jobs on a node than a block lists per node (column scan through the
     # indices), and many GPUs per job
     synth.Config("store-crowded-nodes", 8, 64, 400, 12, 16, 8, 32, 12, num_elite=2, mutate_prob=0.3,
@@ -96,6 +100,10 @@ def test_store_round_equals_dense_stepwise_round(gpu, oracle, cfg):
         jobs.active[6:] = 0
         jobs = setup_fair(jobs, cl)
     cur = cfg.cur(jobs) if cfg.random_cur else None
+    if cfg.name == "store-infeasible-current":
+        cur = synth.random_raw_population(1, cfg.num_jobs, cl, 77, density=0.5, v_hi=1400)[0]
+        jobs.k_cap[::3] = 2
+        assert cur.sum(axis=1).max() > 2047
     penalise = cur is not None
     rnd = 3
     s = api.scheduler_for(cfg, stream=torch.cuda.current_stream().cuda_stream)
