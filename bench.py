@@ -409,12 +409,26 @@ def bench_dense_generation(api, torch, dev, stream, cfg, cl, jobs, cur, hbm_peak
         a, b = b, a
     t = sched.read_kernel_timing()
     sched.close()
+    # a device-to-device copy of one population (the runtime's own copy, same 268 MB in and out,
+    # same stream): what a plain copy of this size reaches on this GPU, beside the row pass
+    copy_us = []
+    for _ in range(9):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        b.copy_(a)
+        e1.record(stream)
+        e1.synchronize()
+        copy_us.append(e0.elapsed_time(e1) * 1e3)
+    copy_us = sorted(copy_us)[len(copy_us) // 2]
     rows_ms = t["rows"][0] / reps
     cols_ms = t["cols"][0] / reps
     algo = 2.0 * P * J * NN * 2 + P * J * 5
     gbs = algo / (rows_ms * 1e-3) / 1e9
     return {"workload": "large shape, dense int16 [512][1024][256] in and out", "rows_us": round(rows_ms * 1e3, 2),
             "column_repair_us": round(cols_ms * 1e3, 2), "generations_per_sec": 1e3 / (rows_ms + cols_ms),
+            "plain_copy_same_size_us": round(copy_us, 2),
+            "plain_copy_note": "runtime device-to-device copy of one population, for context: the measured peak "
+                               "below was taken on buffers several times larger",
             "roofline": {"kernel": "rows", "bound": "hbm", "achieved": round(gbs, 1), "peak": hbm_peak,
                          "peak_source": "MEASURED_PEAKS.json hbm_gbs" if peak_src == "measured" else "recipe fallback",
                          "unit": "GB/s", "frac": round(gbs / hbm_peak, 4), "traffic": NCU_TRAFFIC_BYTES["rows"],
