@@ -500,25 +500,53 @@ __device__ __noinline__ u32x4 draw_call(uint32_t k0, uint32_t k1, uint32_t idx, 
   return philox4x32_10(c, k0, k1);
 }
 
-// Two calls of the stream that differ only in their slot, rounds interleaved: the two chains of
-// dependent multiplies hide each other's latency (a row's crossover and perturbation draws).
+// Two calls of the stream that differ only in their slot (the last counter word), rounds
+// interleaved: the two chains of dependent multiplies hide each other's latency (a row's crossover
+// and perturbation draws, a node's two repair draws).  Of the first call only word x is wanted.
+// What the two calls share is worked out once: round 0 entirely (the slot only enters its third
+// output word), the first product of round 1 and the second product of round 2; the last round of
+// the first call needs half a product.  35 products instead of 40.
 __device__ __noinline__ void draw_pair_call(uint32_t k0, uint32_t k1, uint32_t idx, uint32_t cand, uint32_t gen,
                                             uint32_t slot_a, uint32_t slot_b, uint32_t &a_x, u32x4 &b) {
-  u32x4 ca = {idx, cand, gen, slot_a}, cb = {idx, cand, gen, slot_b};
-#pragma unroll
-  for (int r = 0; r < 10; ++r) {
-    const uint64_t pa0 = (uint64_t)0xD2511F53u * ca.x, pa1 = (uint64_t)0xCD9E8D57u * ca.z;
-    const uint64_t pb0 = (uint64_t)0xD2511F53u * cb.x, pb1 = (uint64_t)0xCD9E8D57u * cb.z;
+  // (the two halves of a product as two 32-bit multiplies)
+  constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+  constexpr uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#define HI(m, v) __umulhi((m), (v))
+#define LO(m, v) ((m) * (v))
+  u32x4 ca, cb;
+  {
+    // round 0 on (idx, cand, gen, slot): x, y, w do not see the slot
+    const uint32_t x = HI(M1, gen) ^ cand ^ k0, y = LO(M1, gen), w = LO(M0, idx), h0 = HI(M0, idx);
+    const uint32_t za = h0 ^ slot_a ^ k1, zb = h0 ^ slot_b ^ k1;
+    k0 += W0; k1 += W1;
+    // round 1: the product of x is shared, so are the new z and w
+    ca.x = HI(M1, za) ^ y ^ k0; ca.y = LO(M1, za);
+    cb.x = HI(M1, zb) ^ y ^ k0; cb.y = LO(M1, zb);
+    ca.z = cb.z = HI(M0, x) ^ w ^ k1;
+    ca.w = cb.w = LO(M0, x);
+    k0 += W0; k1 += W1;
+    // round 2: the product of z is shared
+    const uint32_t h1 = HI(M1, ca.z), l1 = LO(M1, ca.z);
     u32x4 na, nb;
-    na.x = (uint32_t)(pa1 >> 32) ^ ca.y ^ k0; na.y = (uint32_t)pa1; na.z = (uint32_t)(pa0 >> 32) ^ ca.w ^ k1; na.w = (uint32_t)pa0;
-    nb.x = (uint32_t)(pb1 >> 32) ^ cb.y ^ k0; nb.y = (uint32_t)pb1; nb.z = (uint32_t)(pb0 >> 32) ^ cb.w ^ k1; nb.w = (uint32_t)pb0;
+    na.x = h1 ^ ca.y ^ k0; na.y = l1; na.z = HI(M0, ca.x) ^ ca.w ^ k1; na.w = LO(M0, ca.x);
+    nb.x = h1 ^ cb.y ^ k0; nb.y = l1; nb.z = HI(M0, cb.x) ^ cb.w ^ k1; nb.w = LO(M0, cb.x);
+    ca = na; cb = nb;
+    k0 += W0; k1 += W1;
+  }
+#pragma unroll
+  for (int r = 3; r < 9; ++r) {
+    u32x4 na, nb;
+    na.x = HI(M1, ca.z) ^ ca.y ^ k0; na.y = LO(M1, ca.z); na.z = HI(M0, ca.x) ^ ca.w ^ k1; na.w = LO(M0, ca.x);
+    nb.x = HI(M1, cb.z) ^ cb.y ^ k0; nb.y = LO(M1, cb.z); nb.z = HI(M0, cb.x) ^ cb.w ^ k1; nb.w = LO(M0, cb.x);
     ca = na;
     cb = nb;
-    k0 += 0x9E3779B9u;
-    k1 += 0xBB67AE85u;
+    k0 += W0; k1 += W1;
   }
-  a_x = ca.x;
-  b = cb;
+  // round 9: of the first call only x
+  a_x = HI(M1, ca.z) ^ ca.y ^ k0;
+  b.x = HI(M1, cb.z) ^ cb.y ^ k0; b.y = LO(M1, cb.z); b.z = HI(M0, cb.x) ^ cb.w ^ k1; b.w = LO(M0, cb.x);
+#undef HI
+#undef LO
 }
 
 // GPUs of the row on `node` (0 when the node is not occupied) and where its entry is or belongs
@@ -669,16 +697,16 @@ __device__ __noinline__ int row_value_at(const uint32_t *rec, const int16_t *poo
 }
 
 // what the per-node repair decides for the occupant held by this lane of a group (entry = job |
-// GPUs << 13 | distributed << 31 in the first have_n <= 16 lanes): the GPUs the job keeps on the node
-__device__ __forceinline__ int decide_entries(const GenArgs &a, uint32_t rkey, const Grp &g, uint32_t c, int nn, int tot,
-                                              int ne, int cap_n, uint32_t entry, int have_n) {
-  const int J = a.J;
+// GPUs << 13 | distributed << 31 in the first have_n <= 16 lanes): the GPUs the job keeps on the node.
+// o_intf, o_cap: the node's rotation offsets (its REPAIR_INTF and REPAIR_CAP draws, bounded by J).
+__device__ __forceinline__ int decide_entries(const Grp &g, int J, int o_intf, int o_cap, int tot, int ne, int cap_n,
+                                              uint32_t entry, int have_n) {
   const bool have = g.sub < have_n;
   const int j = (int)(entry & 0x1FFFu);
   int v = have ? (int)((entry >> 13) & 0x7FFu) : 0;
   const bool dist = have && (entry >> 31);
   if (ne >= 2) {
-    const int o = (int)bounded(draw_call(a.key.k0, rkey, (uint32_t)nn, c, a.gen, SLOT_REPAIR_INTF).x, (uint32_t)J);
+    const int o = o_intf;
     int t = J;
     if (dist && v > 0) { t = j - o; if (t < 0) t += J; }
     int best = t;
@@ -690,7 +718,7 @@ __device__ __forceinline__ int decide_entries(const GenArgs &a, uint32_t rkey, c
   }
   const int excess = tot - cap_n;
   if (excess > 0) {
-    const int o = (int)bounded(draw_call(a.key.k0, rkey, (uint32_t)nn, c, a.gen, SLOT_REPAIR_CAP).x, (uint32_t)J);
+    const int o = o_cap;
     int rot = 0x7fffffff;
     if (have) { rot = j - o; if (rot < 0) rot += J; }
     int ahead = 0;                       // GPUs of the occupants that come first in rotated order
@@ -1219,6 +1247,15 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         bad = (int)((acc_l >> 32) & 0xFFFFu) >= 2 || (int)(uint32_t)acc_l > (int)s_cap[n_l];
       }
       unsigned todo = __ballot_sync(0xffffffffu, bad);
+      // the violating nodes' two rotation offsets, drawn by their lanes side by side
+      int o_intf_l = 0, o_cap_l = 0;
+      if (bad) {
+        uint32_t xw;
+        u32x4 cw;
+        draw_pair_call(a.key.k0, rkey, (uint32_t)n_l, c, a.gen, SLOT_REPAIR_INTF, SLOT_REPAIR_CAP, xw, cw);
+        o_intf_l = (int)bounded(xw, (uint32_t)J);
+        o_cap_l = (int)bounded(cw.x, (uint32_t)J);
+      }
 #pragma unroll 1
       while (todo) {
       // the two lowest set bits: one node per group (the second group may have none)
@@ -1227,6 +1264,8 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       int b1 = -1;
       if (todo) { b1 = __ffs(todo) - 1; todo &= todo - 1; }
       const int bsel = (lane & GROUP) ? b1 : b0;
+      const int o_intf = __shfl_sync(0xffffffffu, o_intf_l, max(bsel, 0));
+      const int o_cap = __shfl_sync(0xffffffffu, o_cap_l, max(bsel, 0));
       if (bsel >= 0) {
       const int nn = nbase + bsel;
       const unsigned long long acc = s_node[nn];
@@ -1235,7 +1274,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         if (g.sub == 0) { s_viol[nn] = 2; s_anyscan = 1; }
       } else {
       const uint32_t entry = (g.sub < have_n) ? s_occ[nn * OCC + g.sub] : 0u;
-      const int v_new = decide_entries(a, rkey, g, c, nn, (int)(uint32_t)acc, (int)((acc >> 32) & 0xFFFFu), (int)s_cap[nn], entry, have_n);
+      const int v_new = decide_entries(g, J, o_intf, o_cap, (int)(uint32_t)acc, (int)((acc >> 32) & 0xFFFFu), (int)s_cap[nn], entry, have_n);
       if (g.sub < have_n) {
         // the entry now carries the decision: GPUs kept, and bit 24 when that is a change
         const bool changed = v_new != (int)((entry >> 13) & 0x7FFu);
@@ -1315,6 +1354,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       };
       RowList rl;
       list_from_record(rl, my_list, lo, hi);
+      float term;
       if (lo.x != REC_OVERFLOW) {
         int m = 0;                      // entries kept so far
 #pragma unroll 1
@@ -1322,13 +1362,27 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
           const int node = ent_node(rl.e[k]), v = ent_gpus(rl.e[k]);
           const int v_new = new_value(node, v);
           if (v_new != v) {
-            rl.nd += diff_delta(a.cur, NN, j, node, v, v_new);
+            // the first two changes are only noted: what the current allocation holds there is asked
+            // for below, together with the row's speedup
+            if (rl.pn == 0) { rl.pnode0 = node; rl.pold0 = v; rl.pnew0 = v_new; }
+            else if (rl.pn == 1) { rl.pnode1 = node; rl.pold1 = v; rl.pnew1 = v_new; }
+            else rl.nd += diff_delta(a.cur, NN, j, node, v, v_new);
+            ++rl.pn;
             rl.K += v_new - v;
           }
           rl.e[k] = 0u;
           if (v_new > 0) rl.e[m++] = (uint32_t)node | ((uint32_t)v_new << 12);
         }
         rl.n = m;
+        // K and N are final: speedup, penalty factor and the current allocation's values travel together
+        const float x_sp = __ldg(a.tp.table + fitness_table_index(a.tp, j, rl.K, rl.n));
+        const float x_pen = a.tp.pen ? __ldg(a.tp.pen + j) : 1.f;
+        int cv0 = 0, cv1 = 0;
+        if (a.cur && rl.pn > 0) cv0 = (int)__ldg(a.cur + (size_t)j * NN + rl.pnode0);
+        if (a.cur && rl.pn > 1) cv1 = (int)__ldg(a.cur + (size_t)j * NN + rl.pnode1);
+        if (a.cur && rl.pn > 0) rl.nd += (int)(rl.pnew0 != cv0) - (int)(rl.pold0 != cv0);
+        if (a.cur && rl.pn > 1) rl.nd += (int)(rl.pnew1 != cv1) - (int)(rl.pold1 != cv1);
+        term = row_term_from(a.tp.pen != nullptr, a.tp.mode, a.tp.p, a.tp.floor_, x_sp, x_pen, rl.nd != 0);
       } else {
         // contents only: pieces pass through this thread, patched on the way; the occupied nodes
         // that remain are listed, so that a row that now fits a record becomes one again
@@ -1365,10 +1419,9 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
 #pragma unroll
           for (int k = 1; k < LIST_MAX; ++k) rl.e[k] = 0u;
         }
+        term = row_term_of(a.tp.table, a.tp.pen, a.tp.k_max, a.tp.n_max, a.tp.mode, a.tp.p, a.tp.floor_, j, rl.K, rl.n, rl.nd);
       }
       const uint32_t word = pack_summary(rl.K, rl.n, rl.nd);
-      const float term = row_term_of(a.tp.table, a.tp.pen, a.tp.k_max, a.tp.n_max, a.tp.mode, a.tp.p, a.tp.floor_, j,
-                                     rl.K, rl.n, rl.nd);
       store_record(a.st.rec + (size_t)dst * REC_WORDS, rl, term, word);
       s_slot[j] = dst;
       s_term[j] = term;
