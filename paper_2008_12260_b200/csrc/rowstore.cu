@@ -993,11 +993,13 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
 
   // ---- rows, one thread each: the child row is the chosen parent's row -----------------------
   // RB rows per thread at a time, so that their dependent loads (index -> record) travel together.
-  // Perturbed rows are dealt out separately (row i of the block's list goes to lane i / 8 of warp
-  // i % 8); the loads of a thread's first perturbed row travel with those of its unperturbed rows.
+  // Perturbed rows are dealt out separately, row i of the block's list to thread i: a warp runs
+  // through the long path for a perturbed row once whether one of its lanes has such a row or all
+  // do, so the few there usually are share as few warps as possible.  The loads of a thread's first
+  // perturbed row travel with those of its unperturbed rows.
   const uint32_t *pin_a = a.ptr_in + (INIT ? (size_t)0 : (size_t)par_a * J);
   const uint32_t *pin_b = a.ptr_in + (INIT ? (size_t)0 : (size_t)par_b * J);
-  const int mine_first = lane * GEN_WARPS + warp;
+  const int mine_first = tid;
   bool pre_loaded = mine_first < nmut;
   uint32_t pre_slot = 0;
   uint4 pre_lo = make_uint4(0u, 0u, 0u, 0u), pre_hi = pre_lo;
@@ -1428,7 +1430,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       s_mark[j] |= MARK_OWN;
     };
     // Thread work for the two uses of rewrite_row, gathered so that the code exists once: first the
-    // rows the listed nodes changed (row i of the list to lane i / 8 of warp i % 8), then, node by
+    // rows the listed nodes changed (row i of the list to thread i), then, node by
     // node, the rows of the columns that had to be walked.
     const int rpt = (J + GEN_THREADS - 1) / GEN_THREADS;
     const int j_lo = min(J, tid * rpt), j_hi = min(J, j_lo + rpt);
