@@ -54,13 +54,13 @@ CONFIG = {
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the committed ncu
 # summaries under profiles/ (not measured in this run); None = the kernel has changed since its
 # counters were taken.
-# "rows": one dense large-workload generation of the streaming row kernel (228.2 MB read + 235.7 MB
+# "rows": one dense large-workload generation of the streaming row kernel (227.7 MB read + 233.7 MB
 # written: some parent rows are shared by several children and come from L2).
 # "fitness_stress": 16 dense stress candidates moved 544.8 + 3.5 MB; every candidate is streamed
 # once, so the figure is scaled by candidates / 16 to the chunk that is timed.
 # "generation_store": one row-store generation of the large workload (3.4 - 3.6 MB read in
 # generations 6 to 8 of a 12-generation round).
-NCU_TRAFFIC_BYTES = {"rows": 463.9e6, "fitness_stress_per_candidate": 548.3e6 / 16, "generation_store": 3.5e6}
+NCU_TRAFFIC_BYTES = {"rows": 461.4e6, "fitness_stress_per_candidate": 548.3e6 / 16, "generation_store": 3.5e6}
 
 
 def measured_peaks():
