@@ -238,7 +238,8 @@ int autoscale_targets(sched_ctx *ctx, const float *d_goodput, const int32_t *d_c
  * given, a row that differs from a non-empty current row is multiplied by the job's
  * factor; the result is raised to cfg.speedup_floor; the power mean with exponent p
  * over the active jobs is written to d_fitness[count] (p = 0: geometric mean; no active
- * job: 0).  d_active: uint8 [J], nullable.  `count` may differ from cfg.population. */
+ * job: 0; with num_jobs = 0 the matrices and the table are empty and d_pop, d_speedup may be
+ * NULL).  d_active: uint8 [J], nullable.  `count` may differ from cfg.population. */
 int eval_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const float *d_speedup,
                  const int16_t *d_cur, const float *d_realloc_factor, const uint8_t *d_active,
                  float p, float *d_fitness);

@@ -395,8 +395,8 @@ int eval_fitness_racks(sched_ctx *ctx, const int16_t *d_pop, int32_t count, cons
   REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "eval_fitness_racks: ctx is NULL");
   REQUIRE(ctx, ctx->d_rack, SCHED_ERR_INVALID_ARG, "eval_fitness_racks: no racks set (sched_set_racks)");
   REQUIRE(ctx, count >= 0, SCHED_ERR_INVALID_ARG, "eval_fitness_racks: count is negative");
-  REQUIRE(ctx, count == 0 || (d_pop && d_speedup && d_speedup_rack && d_fitness), SCHED_ERR_INVALID_ARG,
-          "eval_fitness_racks: d_pop, d_speedup, d_speedup_rack and d_fitness must be non-NULL");
+  REQUIRE(ctx, count == 0 || (d_fitness && (ctx->cfg.num_jobs == 0 || (d_pop && d_speedup && d_speedup_rack))),
+          SCHED_ERR_INVALID_ARG, "eval_fitness_racks: d_pop, d_speedup, d_speedup_rack and d_fitness must be non-NULL");
   REQUIRE(ctx, p == p, SCHED_ERR_INVALID_ARG, "eval_fitness_racks: p is NaN");
   REQUIRE(ctx, ((uintptr_t)d_pop & 1) == 0 && ((uintptr_t)d_cur & 1) == 0 && ((uintptr_t)d_speedup & 3) == 0 &&
                    ((uintptr_t)d_speedup_rack & 3) == 0 && ((uintptr_t)d_fitness & 3) == 0,
@@ -495,7 +495,7 @@ int eval_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const floa
                  float p, float *d_fitness) {
   REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "eval_fitness: ctx is NULL");
   REQUIRE(ctx, count >= 0, SCHED_ERR_INVALID_ARG, "eval_fitness: count is negative");
-  REQUIRE(ctx, count == 0 || (d_pop && d_speedup && d_fitness), SCHED_ERR_INVALID_ARG,
+  REQUIRE(ctx, count == 0 || (d_fitness && (ctx->cfg.num_jobs == 0 || (d_pop && d_speedup))), SCHED_ERR_INVALID_ARG,
           "eval_fitness: d_pop, d_speedup and d_fitness must be non-NULL");
   REQUIRE(ctx, p == p, SCHED_ERR_INVALID_ARG, "eval_fitness: p is NaN");
   REQUIRE(ctx, ((uintptr_t)d_pop & 1) == 0 && ((uintptr_t)d_cur & 1) == 0 &&
@@ -509,7 +509,7 @@ int eval_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const floa
 int repair_population(sched_ctx *ctx, const sched_jobs *d_jobs, int16_t *d_pop, int32_t count,
                       uint32_t first_candidate, uint32_t round, uint32_t generation) {
   REQUIRE(nullptr, ctx, SCHED_ERR_INVALID_ARG, "repair_population: ctx is NULL");
-  REQUIRE(ctx, count >= 0 && (count == 0 || d_pop), SCHED_ERR_INVALID_ARG,
+  REQUIRE(ctx, count >= 0 && (count == 0 || d_pop || ctx->cfg.num_jobs == 0), SCHED_ERR_INVALID_ARG,
           "repair_population: d_pop is NULL or count negative");
   REQUIRE(ctx, ((uintptr_t)d_pop & 1) == 0, SCHED_ERR_INVALID_ARG, "repair_population: d_pop misaligned");
   REQUIRE(ctx, (long long)count * ctx->cfg.num_jobs < (1LL << 31), SCHED_ERR_TOO_LARGE,

@@ -334,6 +334,10 @@ int launch_fitness(sched_ctx *ctx, const int16_t *d_pop, int32_t count, const fl
   const sched_config &c = ctx->cfg;
   const int J = c.num_jobs;
   if (count == 0) return SCHED_OK;
+  if (J == 0) {     // the mean over no jobs: 0 by definition
+    SCHED_CUDA_CHECK(ctx, cudaMemsetAsync(d_fitness, 0, (size_t)count * sizeof(float), ctx->stream));
+    return SCHED_OK;
+  }
 
   const bool penalise = d_cur && d_rf;
   if (penalise && J > 0 && !ctx->pen_ready) {
@@ -399,6 +403,10 @@ int launch_fitness_racks(sched_ctx *ctx, const int16_t *d_pop, int32_t count, co
   const sched_config &c = ctx->cfg;
   const int J = c.num_jobs;
   if (count == 0) return SCHED_OK;
+  if (J == 0) {     // the mean over no jobs: 0 by definition
+    SCHED_CUDA_CHECK(ctx, cudaMemsetAsync(d_fitness, 0, (size_t)count * sizeof(float), ctx->stream));
+    return SCHED_OK;
+  }
   const bool penalise = d_cur && d_rf;
   if (penalise && J > 0 && !ctx->pen_ready) {
     int rc = launch_penalty_prep(ctx, d_cur, d_rf);
