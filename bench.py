@@ -75,7 +75,8 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clocks / throttle reasons sampled every 200 ms while the timed region runs."""
+    """nvidia-smi clocks / throttle reasons sampled every 20 ms while the timed region runs (the region
+    is about 0.1 s long; the sampler is stopped right after it)."""
 
     FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -91,15 +92,32 @@ class ClockSampler:
             self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "200"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+                 "--format=csv,noheader,nounits", "-lms", "20"], stdout=self.tmp, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
+    def lines(self):
+        try:
+            with open(self.tmp.name) as f:
+                return [ln for ln in f.read().splitlines() if ln.count(",") >= 8]
+        except Exception:
+            return []
+
+    def wait_ready(self, seconds=2.0):
+        """Blocks until the sampler has printed its first line (it takes a while to start)."""
+        t0 = time.time()
+        while self.proc is not None and not self.lines() and time.time() - t0 < seconds:
+            time.sleep(0.01)
+
+    def mark(self):
+        """Number of samples taken so far: the timed region's samples lie between two marks."""
+        return len(self.lines())
+
+    def stop(self, first=0, last=None):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
-        time.sleep(0.25)
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -109,7 +127,13 @@ class ClockSampler:
         self.tmp.seek(0)
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.tmp.read().splitlines():
+        all_lines = [ln for ln in self.tmp.read().splitlines() if ln.count(",") >= 8]
+        # the samples between the two marks, and the one right after (a region shorter than the
+        # sampling interval would otherwise have none)
+        chosen = all_lines[first:(None if last is None else max(last, first) + 1)]
+        if not chosen or not last:          # (nothing was visible in the file while the region ran: keep all)
+            chosen = all_lines
+        for line in chosen:
             f = [x.strip() for x in line.split(",")]
             if len(f) < 9:
                 continue
@@ -231,18 +255,21 @@ def run_ours(args):
     torch.cuda.synchronize()
 
     sampler = ClockSampler(local_rank)
+    sampler.start()
+    sampler.wait_ready()
     launches0 = sched.launch_count()
     pdist.barrier()
     torch.cuda.synchronize()
-    sampler.start()
+    mark0 = sampler.mark()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for k in range(args.steps):
         step(100 + k)
     e1.record(stream)
     torch.cuda.synchronize()
+    mark1 = sampler.mark()
     pdist.barrier()
-    clocks = sampler.stop()
+    clocks = sampler.stop(mark0, mark1)
     elapsed_ms = e0.elapsed_time(e1)
     launches = sched.launch_count() - launches0
     sched.sync_status()
