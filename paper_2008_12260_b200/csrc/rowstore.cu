@@ -835,7 +835,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   __shared__ int s_nmut, s_novf, s_nslow, s_nmod, s_nneed, s_ncow, s_fail, s_anyscan, s_po;
   __shared__ unsigned int s_base_mut, s_base_cow, s_base_cow2;
   __shared__ int s_parent, s_red[GEN_WARPS + 1];
-  __shared__ uint32_t s_w0sec[32], s_w0mut[32];   // the first warp's draw bits, for the threads that take over its rows
+  __shared__ uint32_t s_w0sec[32], s_w0mut[32], s_w0act[32];   // the first warp's row bits, for the threads that take over its rows
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint32_t *my_list = (uint32_t *)s_rowbuf + tid * LIST_WORDS;
@@ -863,11 +863,18 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   __syncthreads();
   // every row's draws: which parent, perturbed or not; the perturbed rows are numbered
   uint32_t secbits = 0, mutbits = 0;   // bit r: this thread's r-th row (j = tid + r * GEN_THREADS)
+  uint32_t actbits = 0;                // the thread's rows that exist and belong to active jobs
+  {
+    int r = 0;
+#pragma unroll 1
+    for (int j = tid; j < J; j += GEN_THREADS, ++r)
+      if (!a.active || a.active[j]) actbits |= 1u << r;
+  }
   if (!elite) {
     int r = 0;
 #pragma unroll 1
     for (int j = tid; j < J; j += GEN_THREADS, ++r) {
-      if (a.active && !a.active[j]) continue;
+      if (!((actbits >> r) & 1u)) continue;
       bool sec = false;
       u32x4 mw;
       if (INIT) {
@@ -894,7 +901,7 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
     idx[0] = (int)bounded(sel.x, P); idx[1] = (int)bounded(sel.y, P);
     idx[2] = (int)bounded(sel.z, P); idx[3] = (int)bounded(sel.w, P);
   }
-  if (warp == 0) { s_w0sec[lane] = secbits; s_w0mut[lane] = mutbits; }
+  if (warp == 0) { s_w0sec[lane] = secbits; s_w0mut[lane] = mutbits; s_w0act[lane] = actbits; }
   __syncthreads();
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
@@ -1034,15 +1041,16 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
         jr[r] = tid + rr * GEN_THREADS;
         sec = ((secbits >> rr) & 1u) != 0u;
         mut[r] = ((mutbits >> rr) & 1u) != 0u;
+        on[r] = rr < 32 && ((actbits >> rr) & 1u) != 0u;
       } else {
         const int k = (tid - 32) + ((b - own_batches) * RB + r) * (GEN_THREADS - 32);   // k-th pair of the first warp
         const int t = k & 31, rr = k >> 5;
         jr[r] = (k < handed) ? t + rr * GEN_THREADS : J;
         sec = (k < handed) && ((s_w0sec[t] >> rr) & 1u) != 0u;
         mut[r] = (k < handed) && ((s_w0mut[t] >> rr) & 1u) != 0u;
+        on[r] = (k < handed) && ((s_w0act[t] >> rr) & 1u) != 0u;
       }
       const int j = jr[r];
-      on[r] = j < J && (!a.active || a.active[j]);
       slot[r] = a.st.zero_slot;
       if (on[r]) {
         if (INIT && mut[r]) slot[r] = a.init_src + (uint32_t)j;   // perturbation starts before the row caps
