@@ -835,7 +835,6 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   __shared__ int s_nmut, s_novf, s_nslow, s_nmod, s_nneed, s_ncow, s_fail, s_anyscan, s_po;
   __shared__ unsigned int s_base_mut, s_base_cow, s_base_cow2;
   __shared__ int s_parent, s_red[GEN_WARPS + 1];
-  __shared__ uint32_t s_w0sec[32], s_w0mut[32], s_w0act[32];   // the first warp's row bits, for the threads that take over its rows
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint32_t *my_list = (uint32_t *)s_rowbuf + tid * LIST_WORDS;
@@ -901,7 +900,6 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
     idx[0] = (int)bounded(sel.x, P); idx[1] = (int)bounded(sel.y, P);
     idx[2] = (int)bounded(sel.z, P); idx[3] = (int)bounded(sel.w, P);
   }
-  if (warp == 0) { s_w0sec[lane] = secbits; s_w0mut[lane] = mutbits; s_w0act[lane] = actbits; }
   __syncthreads();
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
@@ -1006,10 +1004,6 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   // through the long path for a perturbed row once whether one of its lanes has such a row or all
   // do, so the few there usually are share as few warps as possible.  The loads of a thread's first
   // perturbed row travel with those of its unperturbed rows.
-  // When one warp is enough for the perturbed rows (the usual case), the first warp does nothing
-  // else: the long path then starts as soon as the rows' records are in, and the first warp's
-  // unperturbed rows go, as a further batch, to the other threads, which have long finished theirs
-  // by the time the perturbed rows are done.
   const uint32_t *pin_a = a.ptr_in + (INIT ? (size_t)0 : (size_t)par_a * J);
   const uint32_t *pin_b = a.ptr_in + (INIT ? (size_t)0 : (size_t)par_b * J);
   const int mine_first = tid;
@@ -1023,33 +1017,19 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
   }
   constexpr int RB = 4;
   const int rows_per_thread = (J + GEN_THREADS - 1) / GEN_THREADS;
-  const bool freed = !elite && nmut > 0 && nmut <= 32;          // the first warp takes the perturbed rows only
   const int own_batches = (rows_per_thread + RB - 1) / RB;
-  const int handed = 32 * rows_per_thread;                       // (thread, row number) pairs of the first warp
-  const int handed_batches = freed ? (handed + (GEN_THREADS - 32) * RB - 1) / ((GEN_THREADS - 32) * RB) : 0;
-  bool pre_rec = false;
 #pragma unroll 1
-  for (int b = (freed && warp == 0) ? own_batches + handed_batches : 0; b < own_batches + handed_batches; ++b) {
+  for (int b = 0; b < own_batches; ++b) {
     uint32_t slot[RB];
     int jr[RB];
     bool on[RB], mut[RB];
 #pragma unroll
     for (int r = 0; r < RB; ++r) {
-      bool sec;
-      if (b < own_batches) {
-        const int rr = b * RB + r;                                // this thread's rr-th row
-        jr[r] = tid + rr * GEN_THREADS;
-        sec = ((secbits >> rr) & 1u) != 0u;
-        mut[r] = ((mutbits >> rr) & 1u) != 0u;
-        on[r] = rr < 32 && ((actbits >> rr) & 1u) != 0u;
-      } else {
-        const int k = (tid - 32) + ((b - own_batches) * RB + r) * (GEN_THREADS - 32);   // k-th pair of the first warp
-        const int t = k & 31, rr = k >> 5;
-        jr[r] = (k < handed) ? t + rr * GEN_THREADS : J;
-        sec = (k < handed) && ((s_w0sec[t] >> rr) & 1u) != 0u;
-        mut[r] = (k < handed) && ((s_w0mut[t] >> rr) & 1u) != 0u;
-        on[r] = (k < handed) && ((s_w0act[t] >> rr) & 1u) != 0u;
-      }
+      const int rr = b * RB + r;                                // this thread's rr-th row
+      jr[r] = tid + rr * GEN_THREADS;
+      const bool sec = ((secbits >> rr) & 1u) != 0u;
+      mut[r] = ((mutbits >> rr) & 1u) != 0u;
+      on[r] = rr < 32 && ((actbits >> rr) & 1u) != 0u;
       const int j = jr[r];
       slot[r] = a.st.zero_slot;
       if (on[r]) {
@@ -1067,7 +1047,6 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
       if (!sched_index_ok(a.status, pre_slot <= a.st.zero_slot, SCHED_CHK_SLOT)) pre_slot = a.st.zero_slot;
       pre_lo = __ldcg((const uint4 *)(a.st.rec + (size_t)pre_slot * REC_WORDS));
       pre_hi = __ldcg((const uint4 *)(a.st.rec + (size_t)pre_slot * REC_WORDS) + 1);
-      pre_rec = true;
     }
 #pragma unroll
     for (int r = 0; r < RB; ++r) {
@@ -1101,8 +1080,8 @@ __global__ void __launch_bounds__(GEN_THREADS, 4) generation_store_kernel(GenArg
     const int j = (int)(mj & 0x1FFFu);
     uint32_t src = pre_slot;
     uint4 lo = pre_lo, hi = pre_hi;
-    if (!pre_loaded) src = (INIT && !fail) ? a.init_src + (uint32_t)j : ((mj >> 15) ? __ldcg(pin_b + j) : __ldcg(pin_a + j));
-    if (!pre_loaded || !pre_rec) {
+    if (!pre_loaded) {
+      src = (INIT && !fail) ? a.init_src + (uint32_t)j : ((mj >> 15) ? __ldcg(pin_b + j) : __ldcg(pin_a + j));
       if (!sched_index_ok(a.status, src <= a.st.zero_slot, SCHED_CHK_SLOT)) src = a.st.zero_slot;
       lo = __ldcg((const uint4 *)(a.st.rec + (size_t)src * REC_WORDS));
       hi = __ldcg((const uint4 *)(a.st.rec + (size_t)src * REC_WORDS) + 1);
