@@ -504,7 +504,7 @@ __device__ __noinline__ u32x4 draw_call(uint32_t k0, uint32_t k1, uint32_t idx, 
 // interleaved: the two chains of dependent multiplies hide each other's latency (a row's crossover
 // and perturbation draws, a node's two repair draws).  Of the first call only word x is wanted.
 // What the two calls share is worked out once: round 0 entirely (the slot only enters its third
-// output word), the first product of round 1 and the second product of round 2; the last round of
+// output word), the first product of the second round and the second product of the third; the last round of
 // the first call needs half a product.  35 products instead of 40.
 __device__ __noinline__ void draw_pair_call(uint32_t k0, uint32_t k1, uint32_t idx, uint32_t cand, uint32_t gen,
                                             uint32_t slot_a, uint32_t slot_b, uint32_t &a_x, u32x4 &b) {
@@ -515,17 +515,17 @@ __device__ __noinline__ void draw_pair_call(uint32_t k0, uint32_t k1, uint32_t i
 #define LO(m, v) ((m) * (v))
   u32x4 ca, cb;
   {
-    // round 0 on (idx, cand, gen, slot): x, y, w do not see the slot
+    // first round, on (idx, cand, gen, slot): x, y, w do not see the slot
     const uint32_t x = HI(M1, gen) ^ cand ^ k0, y = LO(M1, gen), w = LO(M0, idx), h0 = HI(M0, idx);
     const uint32_t za = h0 ^ slot_a ^ k1, zb = h0 ^ slot_b ^ k1;
     k0 += W0; k1 += W1;
-    // round 1: the product of x is shared, so are the new z and w
+    // second round: the product of x is shared, so are the new z and w
     ca.x = HI(M1, za) ^ y ^ k0; ca.y = LO(M1, za);
     cb.x = HI(M1, zb) ^ y ^ k0; cb.y = LO(M1, zb);
     ca.z = cb.z = HI(M0, x) ^ w ^ k1;
     ca.w = cb.w = LO(M0, x);
     k0 += W0; k1 += W1;
-    // round 2: the product of z is shared
+    // third round: the product of z is shared
     const uint32_t h1 = HI(M1, ca.z), l1 = LO(M1, ca.z);
     u32x4 na, nb;
     na.x = h1 ^ ca.y ^ k0; na.y = l1; na.z = HI(M0, ca.x) ^ ca.w ^ k1; na.w = LO(M0, ca.x);
@@ -542,7 +542,7 @@ __device__ __noinline__ void draw_pair_call(uint32_t k0, uint32_t k1, uint32_t i
     cb = nb;
     k0 += W0; k1 += W1;
   }
-  // round 9: of the first call only x
+  // last round: of the first call only x
   a_x = HI(M1, ca.z) ^ ca.y ^ k0;
   b.x = HI(M1, cb.z) ^ cb.y ^ k0; b.y = LO(M1, cb.z); b.z = HI(M0, cb.x) ^ cb.w ^ k1; b.w = LO(M0, cb.x);
 #undef HI
