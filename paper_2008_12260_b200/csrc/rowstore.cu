@@ -503,7 +503,7 @@ __device__ __noinline__ u32x4 draw_call(uint32_t k0, uint32_t k1, uint32_t idx, 
 // Two calls of the stream that differ only in their slot (the last counter word), rounds
 // interleaved: the two chains of dependent multiplies hide each other's latency (a row's crossover
 // and perturbation draws, a node's two repair draws).  Of the first call only word x is wanted.
-// What the two calls share is worked out once: round 0 entirely (the slot only enters its third
+// What the two calls share is worked out once: the first round entirely (the slot only enters its third
 // output word), the first product of the second round and the second product of the third; the last round of
 // the first call needs half a product.  35 products instead of 40.
 __device__ __noinline__ void draw_pair_call(uint32_t k0, uint32_t k1, uint32_t idx, uint32_t cand, uint32_t gen,
